@@ -1,0 +1,251 @@
+/* libbild: the batch-1 decode loop of Big Little Decoder (BiLD) for one pair of
+ * T5-shaped encoder-decoder models on one GPU (sm_100a).
+ *
+ * What the calls compute is defined by the paper:
+ *   - problem statement, Section 3.2 (Eq. 1-2): at every step the next token comes
+ *     from the small or from the large model, chosen by a boolean policy;
+ *   - fallback policy, Section 3.3: hand over to the large model when the small
+ *     model's largest softmax probability is below alpha_FB;
+ *   - rollback policy, Section 3.4 (Eq. 3): the large model reads all pending
+ *     small-model tokens in ONE non-autoregressive pass; the first position whose
+ *     distance d = -ln p_L(small model's token) exceeds alpha_RB is replaced by
+ *     the large model's token and everything after it is dropped;
+ *   - the whole loop, Algorithm 1 (Section 3.5);
+ *   - d is the cross entropy between the small model's hard label and the large
+ *     model's soft label (Section 4.1), and the small model writes at most
+ *     `max_draft` tokens in a row (evaluation details, supplementary material).
+ * The paper names its models (T5 / mT5, Section 4.1 and the model-size table)
+ * but does not define them; the architecture implemented is stated at
+ * bild_model_cfg below.
+ *
+ * General rules
+ *   - Every pointer is tagged HOST or DEVICE.  The library never allocates or
+ *     frees device memory: weights, workspace and debug buffers are the caller's
+ *     and must outlive the context.  bild_create allocates a small host-side
+ *     context, freed by bild_destroy.
+ *   - Every call returns a status (BILD_OK = 0 or a negative BILD_ERR_*), never
+ *     throws, never aborts.  After an error the context is usable again after
+ *     bild_encode.  bild_last_error gives a message for the last failing call.
+ *   - All work is enqueued on the CUDA stream given to bild_create.  Calls that
+ *     return results in host memory synchronise that stream before returning.
+ *   - A context is not thread-safe; use one context per host thread.
+ */
+#ifndef BILD_H
+#define BILD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bild_ctx bild_ctx; /* opaque */
+
+enum {
+  BILD_OK = 0,
+  BILD_ERR_ARG = -1,       /* null pointer, value out of range */
+  BILD_ERR_WORKSPACE = -2, /* workspace too small or misaligned */
+  BILD_ERR_STATE = -3,     /* call out of order (e.g. decode before bild_encode) */
+  BILD_ERR_CAPACITY = -4,  /* sequence would exceed max_enc_len / max_dec_len */
+  BILD_ERR_CUDA = -5,      /* a CUDA runtime call failed */
+  BILD_ERR_TIMEOUT = -6    /* a bounded device-side wait expired */
+};
+enum { BILD_FP32 = 0, BILD_BF16 = 1 };              /* storage type of weight matrices */
+enum { BILD_FFN_RELU = 0, BILD_FFN_GATED_GELU = 1 };
+enum { BILD_MODE_BILD = 0, BILD_MODE_SMALL_ONLY = 1, BILD_MODE_LARGE_ONLY = 2 };
+enum { BILD_MAX_BLOCK = 16 };                       /* largest k of bild_large_verify */
+
+/* One encoder-decoder model.  Architecture (T5 / mT5 as published): pre-norm
+ * residual blocks; RMS norm y = x*g/sqrt(mean(x^2)+ln_eps) without bias; attention
+ * scores not scaled by 1/sqrt(d_kv); additive relative-position bias on
+ * self-attention only, one [rel_buckets][n_heads] table per stack shared by its
+ * layers (decoder: unidirectional buckets, encoder: bidirectional); cross-attention
+ * without bias or mask; FFN = ReLU or tanh-GELU gate; final RMS norm;
+ * logits = logit_scale * W_lm h.  Encoder and decoder have the same depth/width. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, d_kv, d_ff, ffn_kind, vocab;
+  int32_t rel_buckets;   /* 32 */
+  int32_t rel_max_dist;  /* 128 */
+  float ln_eps;          /* 1e-6 */
+  float logit_scale;
+} bild_model_cfg;
+
+typedef struct {
+  bild_model_cfg small_cfg, large_cfg;
+  int32_t dtype;        /* BILD_FP32 or BILD_BF16: type of every matrix and of the embedding table */
+  int32_t max_enc_len;  /* capacity for encoder ids */
+  int32_t max_dec_len;  /* capacity of y including the start symbol: max_len + 1 <= max_dec_len */
+  int32_t max_draft;    /* small-model tokens in a row before a forced fallback (paper: 10); 1..15 */
+  int32_t start_id;     /* y[0] */
+  int32_t eos_id;       /* -1: never stop on a token */
+} bild_config;
+
+/* All members are DEVICE pointers.  Matrices are row-major [out][in] in
+ * config.dtype; norm gains and bias tables are always fp32.  inner = n_heads*d_kv. */
+typedef struct {
+  const void *ln1;   /* [d] fp32 */
+  const void *wqkv;  /* [3*inner][d], rows: q, k, v */
+  const void *wo;    /* [d][inner] */
+  const void *ln2;   /* [d] fp32 */
+  const void *wi0;   /* [d_ff][d]  (ReLU branch, or GELU branch of the gate) */
+  const void *wi1;   /* [d_ff][d]  linear branch of the gate; NULL for ReLU */
+  const void *wfo;   /* [d][d_ff] */
+} bild_enc_layer;
+
+typedef struct {
+  const void *ln1, *wqkv, *wo;  /* self-attention, as above */
+  const void *ln2;              /* [d] fp32 */
+  const void *wcq;              /* [inner][d] */
+  const void *wckv;             /* [2*inner][d], rows: k, v (applied to the encoder memory) */
+  const void *wco;              /* [d][inner] */
+  const void *ln3;              /* [d] fp32 */
+  const void *wi0, *wi1, *wfo;  /* as above */
+} bild_dec_layer;
+
+typedef struct {
+  const void *emb;           /* DEVICE [vocab][d] */
+  const void *lm_head;       /* DEVICE [vocab][d]; may equal emb */
+  const void *enc_rel_bias;  /* DEVICE [rel_buckets][n_heads] fp32 */
+  const void *dec_rel_bias;  /* DEVICE [rel_buckets][n_heads] fp32 */
+  const void *enc_final_ln;  /* DEVICE [d] fp32 */
+  const void *dec_final_ln;  /* DEVICE [d] fp32 */
+  const bild_enc_layer *enc_layers; /* HOST array [n_layers] of structs of DEVICE pointers (copied) */
+  const bild_dec_layer *dec_layers; /* HOST array [n_layers] (copied) */
+} bild_weights;
+
+/* Result of one small-model step (Algorithm 1, the small-model branch). */
+typedef struct {
+  int32_t argmax;   /* lowest index among equal maxima */
+  float max_logit;
+  float lse;        /* ln sum exp of the scaled logits */
+  float pmax;       /* largest softmax probability */
+  int32_t fallback; /* 1 iff pmax < alpha_fb (Section 3.3) */
+} bild_step_out;
+
+/* Result of one large-model block pass (Algorithm 1, the fallback branch). */
+typedef struct {
+  int32_t argmax[BILD_MAX_BLOCK];  /* row i: arg max of p_L(. | y up to and including tokens[i]) */
+  float lse[BILD_MAX_BLOCK];
+  float d[BILD_MAX_BLOCK];         /* d[i] = -ln p_L(tokens[i+1]) under row i, i < k-1 */
+  int32_t first_violation;         /* smallest i < k-1 with d[i] > alpha_rb, else -1 (Eq. 3) */
+  int32_t next_token;              /* argmax[first_violation], else argmax[k-1] */
+} bild_verify_out;
+
+/* kind: 0 small token accepted (token written at y[pos], value = p_max)
+ *       1 fallback, 2 forced fallback after max_draft drafts (token = the small model's
+ *         rejected candidate for y[pos], value = p_max)
+ *       3 large pass without rollback, 4 with rollback (token written at y[pos],
+ *         k = block size, m = first violating row or -1, value = d[m], or for kind 3 the
+ *         largest distance scanned, 0 if none). */
+typedef struct {
+  int32_t kind, pos, token, k, m;
+  float value;
+} bild_trace_rec;
+
+typedef struct {
+  int32_t small_steps, large_calls, fallbacks, forced, rollbacks, discarded, sum_k;
+} bild_stats;
+
+/* Bytes of DEVICE workspace bild_create needs for this configuration (KV caches,
+ * cross-attention K/V, activations, kernel scratch, decode state, trace). */
+int bild_query_workspace(const bild_config *cfg /*HOST*/, size_t *bytes /*HOST out*/);
+
+/* Build a context.  `workspace` is DEVICE memory, 256-byte aligned, at least
+ * bild_query_workspace bytes, caller-owned, used exclusively by this context until
+ * bild_destroy.  `cuda_stream` is a cudaStream_t (NULL = default stream).  Uploads a
+ * few small tables; no other device work.  Errors: ARG, WORKSPACE, CUDA. */
+int bild_create(const bild_config *cfg /*HOST*/, const bild_weights *small_w /*HOST*/,
+                const bild_weights *large_w /*HOST*/, void *workspace /*DEVICE*/,
+                size_t workspace_bytes, void *cuda_stream, bild_ctx **out /*HOST out*/);
+void bild_destroy(bild_ctx *ctx); /* frees the host-side context only */
+
+/* Run both encoders over ids[0..n_ids) and project the cross-attention K/V of
+ * every decoder layer (the per-input set-up of Algorithm 1's two models).  Resets
+ * the decode state: y = [start_id], both caches empty.  1 <= n_ids <= max_enc_len.
+ * Asynchronous on the stream (ids are copied before returning). */
+int bild_encode(bild_ctx *ctx, const int32_t *ids /*HOST*/, int n_ids);
+
+/* Reset the decode state only (keeps the encoder results of the last bild_encode). */
+int bild_reset(bild_ctx *ctx);
+
+/* One small-model step: feed `token` at the next position of the small model's
+ * cache (cache length += 1) and return the arg-max / p_max / fallback test of the
+ * next-token distribution (Section 3.3).  logits_dbg: DEVICE [vocab] fp32 or NULL;
+ * when given, the scaled logits are also written there (debug; the normal path
+ * never stores them).  Synchronises. */
+int bild_small_step(bild_ctx *ctx, int32_t token, float alpha_fb, bild_step_out *out /*HOST*/,
+                    float *logits_dbg /*DEVICE or NULL*/);
+
+/* One large-model block pass over tokens[0..k), 1 <= k <= BILD_MAX_BLOCK, fed at the
+ * next k positions of the large model's cache (cache length += k; no rewind is done
+ * here).  Row i is the distribution after tokens[i]; tokens[i+1] is judged by row i
+ * (Section 3.4).  logits_dbg: DEVICE [k][vocab] fp32 or NULL.  Synchronises. */
+int bild_large_verify(bild_ctx *ctx, const int32_t *tokens /*HOST*/, int k, float alpha_rb,
+                      bild_verify_out *out /*HOST*/, float *logits_dbg /*DEVICE or NULL*/);
+
+/* Cut a self-attention cache back to new_len rows (which: 0 small, 1 large).  Only a
+ * length counter changes; later steps overwrite the dropped rows. */
+int bild_rewind(bild_ctx *ctx, int which, int new_len);
+
+/* Algorithm 1 from y = [start_id] until max_len tokens exist or eos_id was written.
+ * Resets the decode state first (bild_encode must have been called).  The loop runs
+ * on the device; tokens, trace and counters are copied back once at the end.
+ * tokens_out: HOST [max_len]; *n_tokens: number written.  trace_out: HOST
+ * [trace_cap] or NULL; *n_trace = records produced (records beyond trace_cap are
+ * counted but dropped).  mode: BILD_MODE_*.  Synchronises.
+ * Errors: STATE (no encode), CAPACITY (max_len + 1 > max_dec_len), ARG, CUDA. */
+int bild_generate(bild_ctx *ctx, int mode, float alpha_fb, float alpha_rb, int max_len,
+                  int32_t *tokens_out /*HOST*/, int *n_tokens /*HOST out*/,
+                  bild_trace_rec *trace_out /*HOST or NULL*/, int trace_cap, int *n_trace /*HOST out*/,
+                  bild_stats *stats /*HOST out or NULL*/);
+
+/* As bild_generate, but only enqueues the device loop (no copy back, no sync): for
+ * timing with events on the stream.  Fetch the results with bild_fetch_result. */
+int bild_generate_async(bild_ctx *ctx, int mode, float alpha_fb, float alpha_rb, int max_len);
+int bild_fetch_result(bild_ctx *ctx, int32_t *tokens_out /*HOST*/, int *n_tokens /*HOST out*/,
+                      bild_trace_rec *trace_out /*HOST or NULL*/, int trace_cap, int *n_trace,
+                      bild_stats *stats /*HOST out or NULL*/);
+
+/* Measurement aid for the per-pass latencies (the paper's claim under test is that one
+ * block pass over k tokens costs one weight load, Section 3.2): run one decoder pass of
+ * model `which` (0 small with k = 1, 1 large with 1 <= k <= 16) `iters` times back to back
+ * at self-cache length cache_len, with whatever the cache holds, and return the mean time
+ * of one pass in milliseconds (CUDA events on the context's stream).  Leaves the decode
+ * state undefined: call bild_reset or bild_generate afterwards.  Synchronises. */
+int bild_time_pass(bild_ctx *ctx, int which, int k, int cache_len, int iters, float *ms_per_pass /*HOST out*/);
+
+/* Number of kernel launches this context has enqueued since it was created. */
+int64_t bild_launch_count(const bild_ctx *ctx);
+
+const char *bild_last_error(const bild_ctx *ctx); /* HOST string owned by the context */
+
+/* ---- single operations (for unit tests and micro-benchmarks) -------------------
+ * Each is the kernel the decode path uses, run once on the given stream, with every
+ * pointer DEVICE unless said otherwise; no synchronisation. */
+
+/* Y[m][n] = sum_j W[n][j] * H[m][j], H = X if gain == NULL, else the RMS norm of X
+ * with that gain (Section 3.2's model forward; one weight pass serves all m rows).
+ * W: [N][K] in w_dtype; X: [M][K] fp32; Y: [M][N] fp32.  1 <= M <= BILD_MAX_BLOCK. */
+int bild_op_linear(const void *W, int w_dtype, const float *X, const float *gain, float eps,
+                   float *Y, int M, int N, int K, void *cuda_stream);
+
+/* Fused LM head (Sections 3.3 and 3.4): for each of M rows, z = scale * W_lm rms(X),
+ * and from z only: arg-max (lowest index), max, ln-sum-exp, and z[target[m]]
+ * (target may be NULL).  The logits are not stored unless logits_dbg != NULL.
+ * scratch: at least bild_op_lm_head_scratch_bytes(V) bytes, 256-byte aligned. */
+size_t bild_op_lm_head_scratch_bytes(int V);
+int bild_op_lm_head(const void *W, int w_dtype, const float *X, const float *gain, float eps,
+                    float scale, const int32_t *target, int M, int V, int K,
+                    int32_t *argmax_out, float *max_out, float *lse_out, float *gather_out,
+                    float *logits_dbg, void *scratch, void *cuda_stream);
+
+/* Host-only: the relative-position bucket the library uses (T5's bucket function in
+ * exact integer arithmetic).  which = 0: decoder, rel = query_pos - key_pos >= 0;
+ * which = 1: encoder, rel = key_pos - query_pos.  Returns -1 on invalid arguments. */
+int bild_debug_bucket(int which, int rel, int n_buckets, int max_dist);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BILD_H */

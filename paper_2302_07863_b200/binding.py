@@ -1,0 +1,290 @@
+"""ctypes binding of libbild.so: the same names and arguments as include/bild.h.
+
+Only argument marshalling happens here; every step of the decode path runs in the
+library's CUDA kernels.  PyTorch is used for device memory and streams only.  There
+is no fallback: a missing library raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libbild.so")
+
+BILD_OK = 0
+ERR = {-1: "BILD_ERR_ARG", -2: "BILD_ERR_WORKSPACE", -3: "BILD_ERR_STATE", -4: "BILD_ERR_CAPACITY",
+       -5: "BILD_ERR_CUDA", -6: "BILD_ERR_TIMEOUT"}
+FP32, BF16 = 0, 1
+FFN_RELU, FFN_GATED_GELU = 0, 1
+MODE_BILD, MODE_SMALL_ONLY, MODE_LARGE_ONLY = 0, 1, 2
+MAX_BLOCK = 16
+
+EXPORTS = ["bild_query_workspace", "bild_create", "bild_destroy", "bild_encode", "bild_reset",
+           "bild_small_step", "bild_large_verify", "bild_rewind", "bild_generate", "bild_generate_async",
+           "bild_fetch_result", "bild_time_pass", "bild_launch_count", "bild_last_error", "bild_op_linear",
+           "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_debug_bucket"]
+
+
+class ModelCfg(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "d_kv", "d_ff", "ffn_kind", "vocab",
+                                         "rel_buckets", "rel_max_dist")] + [("ln_eps", C.c_float),
+                                                                            ("logit_scale", C.c_float)]
+
+
+class Config(C.Structure):
+    _fields_ = [("small_cfg", ModelCfg), ("large_cfg", ModelCfg)] + [
+        (n, C.c_int32) for n in ("dtype", "max_enc_len", "max_dec_len", "max_draft", "start_id", "eos_id")]
+
+
+class EncLayer(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("ln1", "wqkv", "wo", "ln2", "wi0", "wi1", "wfo")]
+
+
+class DecLayer(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("ln1", "wqkv", "wo", "ln2", "wcq", "wckv", "wco", "ln3",
+                                          "wi0", "wi1", "wfo")]
+
+
+class Weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("emb", "lm_head", "enc_rel_bias", "dec_rel_bias", "enc_final_ln",
+                                          "dec_final_ln")] + [("enc_layers", C.POINTER(EncLayer)),
+                                                              ("dec_layers", C.POINTER(DecLayer))]
+
+
+class StepOut(C.Structure):
+    _fields_ = [("argmax", C.c_int32), ("max_logit", C.c_float), ("lse", C.c_float), ("pmax", C.c_float),
+                ("fallback", C.c_int32)]
+
+
+class VerifyOut(C.Structure):
+    _fields_ = [("argmax", C.c_int32 * MAX_BLOCK), ("lse", C.c_float * MAX_BLOCK), ("d", C.c_float * MAX_BLOCK),
+                ("first_violation", C.c_int32), ("next_token", C.c_int32)]
+
+
+class TraceRec(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("kind", "pos", "token", "k", "m")] + [("value", C.c_float)]
+
+
+class Stats(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("small_steps", "large_calls", "fallbacks", "forced", "rollbacks",
+                                         "discarded", "sum_k")]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library; raises if it has not been built (python -m paper_2302_07863_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python paper_2302_07863_b200/build.py`; "
+                               "there is no fallback path")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, f32 = C.c_void_p, C.c_int, C.c_float
+        L.bild_query_workspace.argtypes = [C.POINTER(Config), C.POINTER(C.c_size_t)]
+        L.bild_create.argtypes = [C.POINTER(Config), C.POINTER(Weights), C.POINTER(Weights), vp, C.c_size_t, vp,
+                                  C.POINTER(vp)]
+        L.bild_destroy.argtypes = [vp]
+        L.bild_destroy.restype = None
+        L.bild_encode.argtypes = [vp, C.POINTER(C.c_int32), i32]
+        L.bild_reset.argtypes = [vp]
+        L.bild_small_step.argtypes = [vp, C.c_int32, f32, C.POINTER(StepOut), vp]
+        L.bild_large_verify.argtypes = [vp, C.POINTER(C.c_int32), i32, f32, C.POINTER(VerifyOut), vp]
+        L.bild_rewind.argtypes = [vp, i32, i32]
+        L.bild_generate.argtypes = [vp, i32, f32, f32, i32, C.POINTER(C.c_int32), C.POINTER(i32),
+                                    C.POINTER(TraceRec), i32, C.POINTER(i32), C.POINTER(Stats)]
+        L.bild_generate_async.argtypes = [vp, i32, f32, f32, i32]
+        L.bild_fetch_result.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(i32), C.POINTER(TraceRec), i32,
+                                        C.POINTER(i32), C.POINTER(Stats)]
+        L.bild_time_pass.argtypes = [vp, i32, i32, i32, i32, C.POINTER(f32)]
+        L.bild_launch_count.argtypes = [vp]
+        L.bild_launch_count.restype = C.c_int64
+        L.bild_last_error.argtypes = [vp]
+        L.bild_last_error.restype = C.c_char_p
+        L.bild_op_linear.argtypes = [vp, i32, vp, vp, f32, vp, i32, i32, i32, vp]
+        L.bild_op_lm_head_scratch_bytes.argtypes = [i32]
+        L.bild_op_lm_head_scratch_bytes.restype = C.c_size_t
+        L.bild_op_lm_head.argtypes = [vp, i32, vp, vp, f32, f32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.bild_debug_bucket.argtypes = [i32, i32, i32, i32]
+        _lib = L
+    return _lib
+
+
+class BildError(RuntimeError):
+    def __init__(self, code, msg=""):
+        super().__init__(f"{ERR.get(code, code)}: {msg}")
+        self.code = code
+
+
+def model_cfg(shape, logit_scale: float) -> ModelCfg:
+    """ModelCfg from any object with the fields of workloads.ModelShape."""
+    return ModelCfg(shape.n_layers, shape.d_model, shape.n_heads, shape.d_kv, shape.d_ff,
+                    FFN_RELU if shape.ffn == "relu" else FFN_GATED_GELU, shape.vocab, shape.rel_buckets,
+                    shape.rel_max_dist, shape.eps, logit_scale)
+
+
+def upload_model(tensors: dict, device):
+    """numpy tensors (fp32, or uint16 bf16 bit patterns) -> torch tensors on the device."""
+    import torch
+    out = {}
+    for k, v in tensors.items():
+        if v.dtype == np.uint16:
+            out[k] = torch.from_numpy(v.view(np.int16)).to(device).view(torch.bfloat16)
+        else:
+            out[k] = torch.from_numpy(np.ascontiguousarray(v, dtype=np.float32)).to(device)
+    return out
+
+
+def make_weights(shape, dev: dict):
+    """Weights struct of device pointers for one model; returns (struct, keep-alive list)."""
+    p = lambda name: dev[name].data_ptr()
+    L = shape.n_layers
+    enc = (EncLayer * L)()
+    dec = (DecLayer * L)()
+    gated = shape.ffn != "relu"
+    for l in range(L):
+        e, d = f"enc.{l}.", f"dec.{l}."
+        enc[l] = EncLayer(p(e + "ln1"), p(e + "wqkv"), p(e + "wo"), p(e + "ln2"), p(e + "wi0"),
+                          p(e + "wi1") if gated else None, p(e + "wfo"))
+        dec[l] = DecLayer(p(d + "ln1"), p(d + "wqkv"), p(d + "wo"), p(d + "ln2"), p(d + "wcq"), p(d + "wckv"),
+                          p(d + "wco"), p(d + "ln3"), p(d + "wi0"), p(d + "wi1") if gated else None, p(d + "wfo"))
+    w = Weights(p("emb"), p("lm_head") if "lm_head" in dev else p("emb"), p("enc.rel_bias"), p("dec.rel_bias"),
+                p("enc.final_ln"), p("dec.final_ln"), enc, dec)
+    return w, [enc, dec, dev]
+
+
+class Context:
+    """Owns the workspace tensor and keeps the weight tensors alive; methods mirror the C calls."""
+
+    def __init__(self, cfg: Config, small_shape, small_dev: dict, large_shape, large_dev: dict, device="cuda:0",
+                 stream=None):
+        import torch
+        self.L = lib()
+        self.cfg = cfg
+        self.device = torch.device(device)
+        nbytes = C.c_size_t()
+        self._check(self.L.bild_query_workspace(C.byref(cfg), C.byref(nbytes)), "bild_query_workspace")
+        self.workspace_bytes = nbytes.value
+        self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        ws, self._keep_s = make_weights(small_shape, small_dev)
+        wl, self._keep_l = make_weights(large_shape, large_dev)
+        self.stream = stream
+        sp = stream.cuda_stream if stream is not None else None
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = self.L.bild_create(C.byref(cfg), C.byref(ws), C.byref(wl), base, nbytes.value, sp, C.byref(h))
+        if rc != BILD_OK:
+            raise BildError(rc, "bild_create")
+        self.h = h
+
+    def _check(self, rc, what=""):
+        if rc != BILD_OK:
+            msg = self.L.bild_last_error(self.h).decode() if getattr(self, "h", None) else what
+            raise BildError(rc, msg)
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.L.bild_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        self.close()
+
+    def encode(self, ids):
+        a = np.ascontiguousarray(ids, dtype=np.int32)
+        self._check(self.L.bild_encode(self.h, a.ctypes.data_as(C.POINTER(C.c_int32)), len(a)))
+
+    def reset(self):
+        self._check(self.L.bild_reset(self.h))
+
+    def small_step(self, token: int, alpha_fb: float, logits_dbg=None) -> StepOut:
+        out = StepOut()
+        self._check(self.L.bild_small_step(self.h, int(token), alpha_fb, C.byref(out),
+                                           logits_dbg.data_ptr() if logits_dbg is not None else None))
+        return out
+
+    def large_verify(self, tokens, alpha_rb: float, logits_dbg=None) -> VerifyOut:
+        a = np.ascontiguousarray(tokens, dtype=np.int32)
+        out = VerifyOut()
+        self._check(self.L.bild_large_verify(self.h, a.ctypes.data_as(C.POINTER(C.c_int32)), len(a), alpha_rb,
+                                             C.byref(out), logits_dbg.data_ptr() if logits_dbg is not None else None))
+        return out
+
+    def rewind(self, which: int, new_len: int):
+        self._check(self.L.bild_rewind(self.h, which, new_len))
+
+    def generate(self, mode: int, alpha_fb: float, alpha_rb: float, max_len: int):
+        toks = (C.c_int32 * max(1, max_len))()
+        n = C.c_int()
+        cap = (max_len + 1) * (self.cfg.max_draft + 3)
+        tr = (TraceRec * cap)()
+        nt = C.c_int()
+        st = Stats()
+        self._check(self.L.bild_generate(self.h, mode, alpha_fb, alpha_rb, max_len, toks, C.byref(n), tr, cap,
+                                         C.byref(nt), C.byref(st)))
+        return self._unpack(toks, n, tr, nt, cap, st)
+
+    def generate_async(self, mode: int, alpha_fb: float, alpha_rb: float, max_len: int):
+        self._check(self.L.bild_generate_async(self.h, mode, alpha_fb, alpha_rb, max_len))
+
+    def fetch_result(self, max_len: int):
+        toks = (C.c_int32 * max(1, max_len))()
+        n = C.c_int()
+        cap = (max_len + 1) * (self.cfg.max_draft + 3)
+        tr = (TraceRec * cap)()
+        nt = C.c_int()
+        st = Stats()
+        self._check(self.L.bild_fetch_result(self.h, toks, C.byref(n), tr, cap, C.byref(nt), C.byref(st)))
+        return self._unpack(toks, n, tr, nt, cap, st)
+
+    @staticmethod
+    def _unpack(toks, n, tr, nt, cap, st):
+        trace = [(r.kind, r.pos, r.token, r.k, r.m, r.value) for r in tr[:min(nt.value, cap)]]
+        stats = {f: getattr(st, f) for f, _ in Stats._fields_}
+        return dict(tokens=list(toks[:n.value]), trace=trace, stats=stats, n_trace=nt.value)
+
+    def time_pass(self, which: int, k: int, cache_len: int, iters: int) -> float:
+        ms = C.c_float()
+        self._check(self.L.bild_time_pass(self.h, which, k, cache_len, iters, C.byref(ms)))
+        return ms.value
+
+    def launch_count(self) -> int:
+        return self.L.bild_launch_count(self.h)
+
+
+def op_linear(W, X, gain, eps, M, N, K, stream=None):
+    """Y[M][N] = rms?(X) W^T through the library's kernel; W bf16 or fp32 torch tensor."""
+    import torch
+    Y = torch.empty((M, N), dtype=torch.float32, device=X.device)
+    dt = BF16 if W.dtype == torch.bfloat16 else FP32
+    rc = lib().bild_op_linear(W.data_ptr(), dt, X.data_ptr(), gain.data_ptr() if gain is not None else None, eps,
+                              Y.data_ptr(), M, N, K, stream.cuda_stream if stream is not None else None)
+    if rc != BILD_OK:
+        raise BildError(rc, "bild_op_linear")
+    return Y
+
+
+def op_lm_head(W, X, gain, eps, scale, target, M, V, K, want_logits=False, stream=None):
+    import torch
+    dev = X.device
+    nb = lib().bild_op_lm_head_scratch_bytes(V)
+    scratch = torch.zeros(nb + 256, dtype=torch.uint8, device=dev)
+    sp = (scratch.data_ptr() + 255) // 256 * 256
+    am = torch.empty(M, dtype=torch.int32, device=dev)
+    mx = torch.empty(M, dtype=torch.float32, device=dev)
+    lse = torch.empty(M, dtype=torch.float32, device=dev)
+    ga = torch.zeros(M, dtype=torch.float32, device=dev)
+    lg = torch.empty((M, V), dtype=torch.float32, device=dev) if want_logits else None
+    dt = BF16 if W.dtype == torch.bfloat16 else FP32
+    rc = lib().bild_op_lm_head(W.data_ptr(), dt, X.data_ptr(), gain.data_ptr() if gain is not None else None, eps,
+                               scale, target.data_ptr() if target is not None else None, M, V, K, am.data_ptr(),
+                               mx.data_ptr(), lse.data_ptr(), ga.data_ptr(), lg.data_ptr() if lg is not None else None,
+                               sp, stream.cuda_stream if stream is not None else None)
+    if rc != BILD_OK:
+        raise BildError(rc, "bild_op_lm_head")
+    return am, mx, lse, ga, lg

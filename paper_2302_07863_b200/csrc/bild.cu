@@ -1,0 +1,752 @@
+// libbild host runtime: workspace planning, launch sequences of the encoder and of the
+// two decoder passes, the decode loop driver, and the extern "C" boundary (include/bild.h).
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "kernels.cuh"
+
+using namespace bild;
+
+// ------------------------------------------------------------------------------------
+// relative-position buckets, exact integer arithmetic
+// ------------------------------------------------------------------------------------
+namespace {
+
+struct Big {  // non-negative big integer, little-endian base 2^32
+  std::vector<uint32_t> d{1};
+  void mul(uint32_t f) {
+    uint64_t carry = 0;
+    for (auto& w : d) { uint64_t t = (uint64_t)w * f + carry; w = (uint32_t)t; carry = t >> 32; }
+    if (carry) d.push_back((uint32_t)carry);
+  }
+  void mul_pow(uint32_t base, int e) { for (int i = 0; i < e; ++i) mul(base); }
+  bool ge(const Big& o) const {
+    size_t na = d.size(), nb = o.d.size();
+    while (na > 1 && d[na - 1] == 0) --na;
+    while (nb > 1 && o.d[nb - 1] == 0) --nb;
+    if (na != nb) return na > nb;
+    for (size_t i = na; i-- > 0;) if (d[i] != o.d[i]) return d[i] > o.d[i];
+    return true;
+  }
+};
+
+// for dist >= max_exact: max_exact + floor(n_log * ln(dist/max_exact) / ln(max_dist/max_exact)),
+// capped at max_exact + n_log - 1: the largest j with dist^n_log * max_exact^j >= max_dist^j * max_exact^n_log
+int log_bucket(int dist, int max_exact, int n_log, int max_dist) {
+  if (dist >= max_dist) return max_exact + n_log - 1;
+  int j = 0;
+  while (j + 1 <= n_log - 1) {
+    Big lhs, rhs;
+    lhs.mul_pow((uint32_t)dist, n_log); lhs.mul_pow((uint32_t)max_exact, j + 1);
+    rhs.mul_pow((uint32_t)max_dist, j + 1); rhs.mul_pow((uint32_t)max_exact, n_log);
+    if (!lhs.ge(rhs)) break;
+    ++j;
+  }
+  return max_exact + j;
+}
+
+int decoder_bucket(int delta, int n_buckets, int max_dist) {  // delta = query - key >= 0
+  const int max_exact = n_buckets / 2;
+  if (delta < max_exact) return delta;
+  return log_bucket(delta, max_exact, n_buckets - max_exact, max_dist);
+}
+
+int encoder_bucket(int rel, int n_buckets, int max_dist) {  // rel = key - query
+  const int half = n_buckets / 2;
+  const int off = rel > 0 ? half : 0;
+  const int dist = rel < 0 ? -rel : rel;
+  const int max_exact = half / 2;
+  if (dist < max_exact) return off + dist;
+  return off + log_bucket(dist, max_exact, half - max_exact, max_dist);
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Bump {  // carves the caller's workspace; with base == nullptr it only measures
+  char* base;
+  size_t off = 0;
+  explicit Bump(void* b) : base((char*)b) {}
+  template <typename T> T* take(size_t n) {
+    off = align_up(off, 256);
+    T* p = base ? (T*)(base + off) : nullptr;
+    off += n * sizeof(T);
+    return p;
+  }
+};
+
+constexpr int NSPLIT_MAX = 32;
+constexpr int HEAD_GRID_MAX = 148 * 4;
+
+struct Model {
+  bild_model_cfg c{};
+  bild_weights w{};
+  std::vector<bild_enc_layer> enc;
+  std::vector<bild_dec_layer> dec;
+  int inner = 0;
+  float *selfK = nullptr, *selfV = nullptr, *crossK = nullptr, *crossV = nullptr;
+  float *x = nullptr, *q = nullptr, *att = nullptr, *u = nullptr;
+  float *dec_bias = nullptr, *enc_bias = nullptr;
+  float* att_part = nullptr;
+  unsigned* att_cnt = nullptr;
+  Partial* head_part = nullptr;
+  unsigned* head_cnt = nullptr;
+  HeadOut* head_out = nullptr;
+  CallDesc* desc = nullptr;
+  int head_grid = 0;
+};
+
+}  // namespace
+
+struct bild_ctx {
+  bild_config cfg{};
+  Model m[2];
+  cudaStream_t stream = nullptr;
+  DevState* st = nullptr;
+  int* y = nullptr;
+  bild_trace_rec* trace = nullptr;
+  int trace_cap = 0;
+  int* enc_ids = nullptr;
+  int* enc_len_dev = nullptr;
+  int* bucket_tmp = nullptr;
+  float *ex = nullptr, *eq = nullptr, *ek = nullptr, *ev = nullptr, *eatt = nullptr, *eu = nullptr;
+  int enc_len = 0;
+  bool encoded = false;
+  int64_t launches = 0;
+  std::string err;
+  DevState* pin_state = nullptr;  // pinned host mirror for the loop driver
+  HeadOut* pin_head = nullptr;
+  size_t ws_bytes = 0;
+};
+
+namespace {
+
+int fail(bild_ctx* c, int code, const std::string& msg) {
+  if (c) c->err = msg;
+  return code;
+}
+#define CUDA_TRY(ctx, expr)                                                               \
+  do {                                                                                    \
+    cudaError_t e_ = (expr);                                                              \
+    if (e_ != cudaSuccess)                                                                \
+      return fail(ctx, BILD_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e_)); \
+  } while (0)
+
+int check_model(const bild_model_cfg& c, std::string& why) {
+  auto bad = [&](const char* s) { why = s; return BILD_ERR_ARG; };
+  if (c.n_layers < 1 || c.d_model < 8 || c.n_heads < 1 || c.d_ff < 8 || c.vocab < 2) return bad("model sizes must be positive");
+  if (c.d_model % 8 || c.d_ff % 8 || (c.n_heads * c.d_kv) % 8) return bad("d_model, d_ff and n_heads*d_kv must be multiples of 8");
+  if (c.d_kv != 16 && c.d_kv != 32 && c.d_kv != 64 && c.d_kv != 128) return bad("d_kv must be 16, 32, 64 or 128");
+  if (c.d_model > 4096 || c.d_ff > 16384) return bad("d_model <= 4096 and d_ff <= 16384");
+  if (c.ffn_kind != BILD_FFN_RELU && c.ffn_kind != BILD_FFN_GATED_GELU) return bad("ffn_kind");
+  if (c.rel_buckets < 4 || c.rel_buckets % 4 || c.rel_max_dist < c.rel_buckets) return bad("rel_buckets / rel_max_dist");
+  if (!(c.ln_eps >= 0.f) || !(c.logit_scale > 0.f)) return bad("ln_eps >= 0 and logit_scale > 0");
+  return BILD_OK;
+}
+
+int check_config(const bild_config* cfg, std::string& why) {
+  if (!cfg) { why = "null config"; return BILD_ERR_ARG; }
+  int rc = check_model(cfg->small_cfg, why);
+  if (rc) return rc;
+  rc = check_model(cfg->large_cfg, why);
+  if (rc) return rc;
+  if (cfg->small_cfg.vocab != cfg->large_cfg.vocab) { why = "the two models must share a vocabulary"; return BILD_ERR_ARG; }
+  if (cfg->dtype != BILD_FP32 && cfg->dtype != BILD_BF16) { why = "dtype"; return BILD_ERR_ARG; }
+  if (cfg->max_enc_len < 1 || cfg->max_enc_len > 4096) { why = "1 <= max_enc_len <= 4096"; return BILD_ERR_ARG; }
+  if (cfg->max_dec_len < 2 || cfg->max_dec_len > 4096) { why = "2 <= max_dec_len <= 4096"; return BILD_ERR_ARG; }
+  if (cfg->max_draft < 1 || cfg->max_draft > MAXB - 1) { why = "1 <= max_draft <= 15"; return BILD_ERR_ARG; }
+  if (cfg->start_id < 0 || cfg->start_id >= cfg->small_cfg.vocab) { why = "start_id"; return BILD_ERR_ARG; }
+  return BILD_OK;
+}
+
+int head_grid_for(int V) { return std::max(1, std::min(HEAD_GRID_MAX, (V + 63) / 64)); }
+
+// Lays out everything the context keeps on the device.
+void plan(bild_ctx* c, Bump& b) {
+  const bild_config& cfg = c->cfg;
+  const int cap = cfg.max_dec_len, ecap = cfg.max_enc_len;
+  c->st = b.take<DevState>(1);
+  c->y = b.take<int>(cap + 1);
+  c->trace_cap = cap * (cfg.max_draft + 3);
+  c->trace = b.take<bild_trace_rec>(c->trace_cap);
+  c->enc_ids = b.take<int>(ecap);
+  c->enc_len_dev = b.take<int>(1);
+  c->bucket_tmp = b.take<int>(std::max(cap, 2 * ecap));
+  int dmax = 0, imax = 0, fmax = 0;
+  for (int i = 0; i < 2; ++i) {
+    Model& m = c->m[i];
+    const bild_model_cfg& mc = i == 0 ? cfg.small_cfg : cfg.large_cfg;
+    m.c = mc;
+    m.inner = mc.n_heads * mc.d_kv;
+    dmax = std::max(dmax, mc.d_model); imax = std::max(imax, m.inner); fmax = std::max(fmax, mc.d_ff);
+    const size_t kv = (size_t)mc.n_layers * mc.n_heads * mc.d_kv;
+    m.selfK = b.take<float>(kv * cap);
+    m.selfV = b.take<float>(kv * cap);
+    m.crossK = b.take<float>(kv * ecap);
+    m.crossV = b.take<float>(kv * ecap);
+    m.x = b.take<float>((size_t)MAXB * mc.d_model);
+    m.q = b.take<float>((size_t)MAXB * m.inner);
+    m.att = b.take<float>((size_t)MAXB * m.inner);
+    m.u = b.take<float>((size_t)MAXB * mc.d_ff);
+    m.dec_bias = b.take<float>((size_t)mc.n_heads * cap);
+    m.enc_bias = b.take<float>((size_t)mc.n_heads * (2 * ecap - 1));
+    m.att_part = b.take<float>((size_t)MAXB * mc.n_heads * NSPLIT_MAX * (mc.d_kv + 2));
+    m.att_cnt = b.take<unsigned>((size_t)MAXB * mc.n_heads);
+    m.head_grid = head_grid_for(mc.vocab);
+    m.head_part = b.take<Partial>((size_t)m.head_grid * MAXB);
+    m.head_cnt = b.take<unsigned>(1);
+    m.head_out = b.take<HeadOut>(1);
+    m.desc = b.take<CallDesc>(1);
+  }
+  c->ex = b.take<float>((size_t)ecap * dmax);
+  c->eq = b.take<float>((size_t)ecap * imax);
+  c->ek = b.take<float>((size_t)ecap * imax);
+  c->ev = b.take<float>((size_t)ecap * imax);
+  c->eatt = b.take<float>((size_t)ecap * imax);
+  c->eu = b.take<float>((size_t)ecap * fmax);
+  b.off = align_up(b.off, 256);
+}
+
+// ---- launches ------------------------------------------------------------------------
+template <typename WT, int MB, int RW>
+cudaError_t launch_linear_t(bild_ctx* c, const LinArgs& a, int rows_y) {
+  const int nwarps = LIN_THREADS / 32;
+  dim3 grid((a.N + nwarps * RW - 1) / (nwarps * RW), rows_y);
+  const int kc = (MB == 1) ? a.K : std::min(a.K, LIN_KC);
+  const size_t smem = (size_t)MB * kc * sizeof(float);
+  const bool gated = a.epi == EPI_GATED;
+  auto kern = gated ? linear_kernel<WT, MB, RW, true> : linear_kernel<WT, MB, RW, false>;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  kern<<<grid, LIN_THREADS, smem, c->stream>>>(a);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_linear(bild_ctx* c, int dtype, int MB, const LinArgs& a, int rows_y = 1) {
+  if (dtype == BILD_BF16)
+    return MB == 1 ? launch_linear_t<__nv_bfloat16, 1, 4>(c, a, rows_y) : launch_linear_t<__nv_bfloat16, MAXB, 2>(c, a, rows_y);
+  return MB == 1 ? launch_linear_t<float, 1, 4>(c, a, rows_y) : launch_linear_t<float, MAXB, 2>(c, a, rows_y);
+}
+
+template <typename WT, int MB, int RW>
+cudaError_t launch_head_t(bild_ctx* c, const HeadArgs& a, int grid, int64_t* launches) {
+  const size_t smem = (size_t)MB * a.K * sizeof(float);
+  auto kern = lm_head_kernel<WT, MB, RW>;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  kern<<<grid, HEAD_THREADS, smem, c ? c->stream : nullptr>>>(a);
+  if (launches) (*launches)++;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_head(cudaStream_t s, int dtype, int MB, const HeadArgs& a, int grid, int64_t* launches) {
+  bild_ctx tmp;
+  tmp.stream = s;
+  if (dtype == BILD_BF16)
+    return MB == 1 ? launch_head_t<__nv_bfloat16, 1, 4>(&tmp, a, grid, launches) : launch_head_t<__nv_bfloat16, MAXB, 2>(&tmp, a, grid, launches);
+  return MB == 1 ? launch_head_t<float, 1, 4>(&tmp, a, grid, launches) : launch_head_t<float, MAXB, 2>(&tmp, a, grid, launches);
+}
+
+int pick_nsplit(int ctas_without_split, int keys_cap) {
+  int ns = (2 * 148 + ctas_without_split - 1) / ctas_without_split;
+  ns = std::min(ns, std::max(1, keys_cap / 32));
+  ns = std::max(1, std::min(ns, NSPLIT_MAX));
+  while ((keys_cap + ns - 1) / ns > 8192 && ns < NSPLIT_MAX) ++ns;
+  return ns;
+}
+
+cudaError_t launch_attn(bild_ctx* c, AttnArgs a, int rows, int keys_cap) {
+  a.smem_keys = (keys_cap + a.nsplit - 1) / a.nsplit;
+  dim3 grid(a.H, rows, a.nsplit);
+  attn_kernel<<<grid, ATT_THREADS, (size_t)a.smem_keys * sizeof(float), c->stream>>>(a);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+template <typename WT>
+void launch_embed_t(bild_ctx* c, const void* E, const int* tokens, const int* cnt_dev, int cnt_host, int rows,
+                    int d, int vocab, float* x) {
+  embed_kernel<WT><<<rows, 128, 0, c->stream>>>((const WT*)E, tokens, cnt_dev, cnt_host, d, vocab, x);
+  c->launches++;
+}
+cudaError_t launch_embed(bild_ctx* c, const void* E, const int* tokens, const int* cnt_dev, int cnt_host, int rows,
+                         int d, int vocab, float* x) {
+  if (c->cfg.dtype == BILD_BF16) launch_embed_t<__nv_bfloat16>(c, E, tokens, cnt_dev, cnt_host, rows, d, vocab, x);
+  else launch_embed_t<float>(c, E, tokens, cnt_dev, cnt_host, rows, d, vocab, x);
+  return cudaGetLastError();
+}
+
+LoopPtrs loop_ptrs(bild_ctx* c) {
+  LoopPtrs L;
+  L.st = c->st; L.y = c->y; L.trace = c->trace; L.descS = c->m[0].desc; L.descL = c->m[1].desc;
+  return L;
+}
+
+// One decoder pass of model `which` over the rows described by its CallDesc
+// (steps S0..S10 / L0..L10: embed, per layer [norm+QKV+append, self-attention, O+residual,
+// norm+cross-Q, cross-attention, cross-O+residual, norm+FFN-up, FFN-down+residual],
+// final norm + LM head + policy).  MB = 1 or MAXB selects the kernel variants.
+int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg) {
+  Model& m = c->m[which];
+  const bild_model_cfg& mc = m.c;
+  const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
+  const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len, dt = c->cfg.dtype;
+  CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x));
+  const int ns_self = pick_nsplit(H * MB, cap), ns_cross = pick_nsplit(H * MB, ecap);
+  for (int l = 0; l < mc.n_layers; ++l) {
+    const bild_dec_layer& w = m.dec[l];
+    const size_t kvoff = (size_t)l * H * dkv;
+    LinArgs a{};
+    a.desc = m.desc; a.eps = mc.ln_eps;
+    // S1 / L1: norm + QKV, K/V appended to the cache
+    a.W0 = w.wqkv; a.X = m.x; a.ldx = d; a.gain = (const float*)w.ln1; a.N = 3 * I; a.K = d;
+    a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 0; a.q_out = m.q; a.ldq = I;
+    a.kc = m.selfK + kvoff * cap; a.vc = m.selfV + kvoff * cap; a.cap = cap;
+    CUDA_TRY(c, launch_linear(c, dt, MB, a));
+    // S2 / L2: self-attention over the cache (causal inside the block)
+    AttnArgs t{};
+    t.q = m.q; t.ldq = I; t.kc = a.kc; t.vc = a.vc; t.cap = cap; t.out = m.att; t.ldo = I;
+    t.bias = m.dec_bias; t.bias_ld = cap; t.bias_off = 0; t.mode = 1; t.dkv = dkv; t.H = H;
+    t.n_keys_dev = c->enc_len_dev; t.desc = m.desc; t.part = m.att_part; t.counters = m.att_cnt;
+    t.nsplit = ns_self; t.err = &c->st->err;
+    CUDA_TRY(c, launch_attn(c, t, MB, cap));
+    // S3 / L3: output projection + residual
+    LinArgs o{};
+    o.desc = m.desc; o.W0 = w.wo; o.X = m.att; o.ldx = I; o.N = d; o.K = I; o.epi = EPI_RESID; o.Y = m.x; o.ldy = d;
+    CUDA_TRY(c, launch_linear(c, dt, MB, o));
+    // S4 / L4: norm + cross-attention query
+    LinArgs cq{};
+    cq.desc = m.desc; cq.eps = mc.ln_eps; cq.W0 = w.wcq; cq.X = m.x; cq.ldx = d; cq.gain = (const float*)w.ln2;
+    cq.N = I; cq.K = d; cq.epi = EPI_STORE; cq.Y = m.q; cq.ldy = I;
+    CUDA_TRY(c, launch_linear(c, dt, MB, cq));
+    // S5 / L5: cross-attention over the encoder K/V
+    AttnArgs x{};
+    x.q = m.q; x.ldq = I; x.kc = m.crossK + kvoff * ecap; x.vc = m.crossV + kvoff * ecap; x.cap = ecap;
+    x.out = m.att; x.ldo = I; x.mode = 0; x.dkv = dkv; x.H = H; x.n_keys_dev = c->enc_len_dev; x.desc = m.desc;
+    x.part = m.att_part; x.counters = m.att_cnt; x.nsplit = ns_cross; x.err = &c->st->err;
+    CUDA_TRY(c, launch_attn(c, x, MB, ecap));
+    // S6 / L6: cross output projection + residual
+    o.W0 = w.wco;
+    CUDA_TRY(c, launch_linear(c, dt, MB, o));
+    // S7 / L7: norm + FFN up (ReLU, or GELU gate)
+    LinArgs up{};
+    up.desc = m.desc; up.eps = mc.ln_eps; up.W0 = w.wi0; up.W1 = w.wi1; up.X = m.x; up.ldx = d;
+    up.gain = (const float*)w.ln3; up.N = F; up.K = d; up.Y = m.u; up.ldy = F;
+    up.epi = mc.ffn_kind == BILD_FFN_GATED_GELU ? EPI_GATED : EPI_RELU;
+    CUDA_TRY(c, launch_linear(c, dt, MB, up));
+    // S8 / L8: FFN down + residual
+    LinArgs dn{};
+    dn.desc = m.desc; dn.W0 = w.wfo; dn.X = m.u; dn.ldx = F; dn.N = d; dn.K = F; dn.epi = EPI_RESID; dn.Y = m.x; dn.ldy = d;
+    CUDA_TRY(c, launch_linear(c, dt, MB, dn));
+  }
+  // S9+S10 / L9+L10: final norm + LM head + policy
+  HeadArgs h{};
+  h.W = m.w.lm_head; h.X = m.x; h.ldx = d; h.gain = (const float*)m.w.dec_final_ln; h.eps = mc.ln_eps;
+  h.scale = mc.logit_scale; h.V = mc.vocab; h.K = d; h.desc = m.desc; h.partials = m.head_part;
+  h.counter = m.head_cnt; h.out = m.head_out; h.logits_dbg = logits_dbg; h.which = which; h.loop = loop_ptrs(c);
+  CUDA_TRY(c, launch_head(c->stream, dt, MB, h, m.head_grid, &c->launches));
+  return BILD_OK;
+}
+
+// Encoder of model `which` over the ids in c->enc_ids, then the cross-attention K/V of
+// every decoder layer.
+int encoder_pass(bild_ctx* c, int which) {
+  Model& m = c->m[which];
+  const bild_model_cfg& mc = m.c;
+  const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
+  const int E = c->enc_len, ecap = c->cfg.max_enc_len, dt = c->cfg.dtype;
+  const int rb = (E + MAXB - 1) / MAXB;
+  CUDA_TRY(c, launch_embed(c, m.w.emb, c->enc_ids, nullptr, E, E, d, mc.vocab, c->ex));
+  for (int l = 0; l < mc.n_layers; ++l) {
+    const bild_enc_layer& w = m.enc[l];
+    LinArgs a{};
+    a.M = E; a.eps = mc.ln_eps; a.W0 = w.wqkv; a.X = c->ex; a.ldx = d; a.gain = (const float*)w.ln1;
+    a.N = 3 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 0; a.q_out = c->eq; a.ldq = I;
+    a.kc = c->ek; a.vc = c->ev; a.cap = ecap; a.pos0_host = 0;
+    CUDA_TRY(c, launch_linear(c, dt, MAXB, a, rb));
+    AttnArgs t{};
+    t.q = c->eq; t.ldq = I; t.kc = c->ek; t.vc = c->ev; t.cap = ecap; t.out = c->eatt; t.ldo = I;
+    t.bias = m.enc_bias; t.bias_ld = 2 * ecap - 1; t.bias_off = ecap - 1; t.mode = 2; t.dkv = dkv; t.H = H;
+    t.n_keys_dev = c->enc_len_dev; t.M = E; t.part = m.att_part; t.counters = m.att_cnt; t.nsplit = 1;
+    t.err = &c->st->err;
+    CUDA_TRY(c, launch_attn(c, t, E, ecap));
+    LinArgs o{};
+    o.M = E; o.W0 = w.wo; o.X = c->eatt; o.ldx = I; o.N = d; o.K = I; o.epi = EPI_RESID; o.Y = c->ex; o.ldy = d;
+    CUDA_TRY(c, launch_linear(c, dt, MAXB, o, rb));
+    LinArgs up{};
+    up.M = E; up.eps = mc.ln_eps; up.W0 = w.wi0; up.W1 = w.wi1; up.X = c->ex; up.ldx = d; up.gain = (const float*)w.ln2;
+    up.N = F; up.K = d; up.Y = c->eu; up.ldy = F;
+    up.epi = mc.ffn_kind == BILD_FFN_GATED_GELU ? EPI_GATED : EPI_RELU;
+    CUDA_TRY(c, launch_linear(c, dt, MAXB, up, rb));
+    LinArgs dn{};
+    dn.M = E; dn.W0 = w.wfo; dn.X = c->eu; dn.ldx = F; dn.N = d; dn.K = F; dn.epi = EPI_RESID; dn.Y = c->ex; dn.ldy = d;
+    CUDA_TRY(c, launch_linear(c, dt, MAXB, dn, rb));
+  }
+  // encoder memory = final norm of ex (fused into the projections); cross K/V per decoder layer
+  for (int l = 0; l < mc.n_layers; ++l) {
+    const size_t kvoff = (size_t)l * H * dkv;
+    LinArgs a{};
+    a.M = E; a.eps = mc.ln_eps; a.W0 = m.dec[l].wckv; a.X = c->ex; a.ldx = d; a.gain = (const float*)m.w.enc_final_ln;
+    a.N = 2 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 1;
+    a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.pos0_host = 0;
+    CUDA_TRY(c, launch_linear(c, dt, MAXB, a, rb));
+  }
+  return BILD_OK;
+}
+
+int build_bias_tables(bild_ctx* c) {
+  const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len;
+  for (int i = 0; i < 2; ++i) {
+    Model& m = c->m[i];
+    std::vector<int> tab(cap);
+    for (int x = 0; x < cap; ++x) tab[x] = decoder_bucket(x, m.c.rel_buckets, m.c.rel_max_dist);
+    CUDA_TRY(c, cudaMemcpyAsync(c->bucket_tmp, tab.data(), cap * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    bias_table_kernel<<<(cap + 127) / 128, 128, 0, c->stream>>>((const float*)m.w.dec_rel_bias, c->bucket_tmp, cap,
+                                                                m.c.n_heads, m.dec_bias);
+    c->launches++;
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    const int ne = 2 * ecap - 1;
+    std::vector<int> etab(ne);
+    for (int x = 0; x < ne; ++x) etab[x] = encoder_bucket(x - (ecap - 1), m.c.rel_buckets, m.c.rel_max_dist);
+    CUDA_TRY(c, cudaMemcpyAsync(c->bucket_tmp, etab.data(), ne * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    bias_table_kernel<<<(ne + 127) / 128, 128, 0, c->stream>>>((const float*)m.w.enc_rel_bias, c->bucket_tmp, ne,
+                                                               m.c.n_heads, m.enc_bias);
+    c->launches++;
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  }
+  return BILD_OK;
+}
+
+int read_state(bild_ctx* c) {
+  CUDA_TRY(c, cudaMemcpyAsync(c->pin_state, c->st, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (c->pin_state->err) return fail(c, c->pin_state->err, "device-side error flag set");
+  return BILD_OK;
+}
+
+int reset_state(bild_ctx* c, int mode, float afb, float arb, int max_len) {
+  reset_state_kernel<<<1, 1, 0, c->stream>>>(loop_ptrs(c), mode, afb, arb, max_len, c->cfg.max_draft,
+                                             c->cfg.eos_id, c->cfg.start_id, c->trace_cap);
+  c->launches++;
+  CUDA_TRY(c, cudaGetLastError());
+  return BILD_OK;
+}
+
+}  // namespace
+
+// ======================================================================================
+// extern "C" boundary
+// ======================================================================================
+extern "C" {
+
+int bild_query_workspace(const bild_config* cfg, size_t* bytes) {
+  std::string why;
+  if (!bytes) return BILD_ERR_ARG;
+  int rc = check_config(cfg, why);
+  if (rc) return rc;
+  bild_ctx tmp;
+  tmp.cfg = *cfg;
+  Bump b(nullptr);
+  plan(&tmp, b);
+  *bytes = b.off;
+  return BILD_OK;
+}
+
+int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_weights* large_w, void* workspace,
+                size_t workspace_bytes, void* cuda_stream, bild_ctx** out) {
+  if (!out) return BILD_ERR_ARG;
+  *out = nullptr;
+  std::string why;
+  int rc = check_config(cfg, why);
+  if (rc) return rc;
+  if (!small_w || !large_w || !workspace) return BILD_ERR_ARG;
+  if ((uintptr_t)workspace % 256) return BILD_ERR_WORKSPACE;
+  bild_ctx* c = new (std::nothrow) bild_ctx;
+  if (!c) return BILD_ERR_ARG;
+  c->cfg = *cfg;
+  c->stream = (cudaStream_t)cuda_stream;
+  Bump b(workspace);
+  plan(c, b);
+  c->ws_bytes = b.off;
+  if (workspace_bytes < b.off) { delete c; return BILD_ERR_WORKSPACE; }
+  const bild_weights* ws[2] = {small_w, large_w};
+  for (int i = 0; i < 2; ++i) {
+    Model& m = c->m[i];
+    const bild_weights* w = ws[i];
+    if (!w->emb || !w->lm_head || !w->enc_rel_bias || !w->dec_rel_bias || !w->enc_final_ln || !w->dec_final_ln ||
+        !w->enc_layers || !w->dec_layers) { delete c; return BILD_ERR_ARG; }
+    m.w = *w;
+    m.enc.assign(w->enc_layers, w->enc_layers + m.c.n_layers);
+    m.dec.assign(w->dec_layers, w->dec_layers + m.c.n_layers);
+    const bool gated = m.c.ffn_kind == BILD_FFN_GATED_GELU;
+    for (int l = 0; l < m.c.n_layers; ++l) {
+      const bild_enc_layer& e = m.enc[l];
+      const bild_dec_layer& d = m.dec[l];
+      if (!e.ln1 || !e.wqkv || !e.wo || !e.ln2 || !e.wi0 || !e.wfo || (gated && !e.wi1) || !d.ln1 || !d.wqkv ||
+          !d.wo || !d.ln2 || !d.wcq || !d.wckv || !d.wco || !d.ln3 || !d.wi0 || !d.wfo || (gated && !d.wi1)) {
+        delete c;
+        return BILD_ERR_ARG;
+      }
+    }
+    m.w.enc_layers = nullptr;
+    m.w.dec_layers = nullptr;
+  }
+  if (cudaMallocHost((void**)&c->pin_state, sizeof(DevState)) != cudaSuccess ||
+      cudaMallocHost((void**)&c->pin_head, sizeof(HeadOut)) != cudaSuccess) {
+    bild_destroy(c);
+    return BILD_ERR_CUDA;
+  }
+  // zero the ticket counters and the state, build the bias-by-distance tables
+  if (cudaMemsetAsync(workspace, 0, c->ws_bytes, c->stream) != cudaSuccess) { bild_destroy(c); return BILD_ERR_CUDA; }
+  rc = build_bias_tables(c);
+  if (rc) { bild_destroy(c); return rc; }
+  *out = c;
+  return BILD_OK;
+}
+
+void bild_destroy(bild_ctx* c) {
+  if (!c) return;
+  if (c->pin_state) cudaFreeHost(c->pin_state);
+  if (c->pin_head) cudaFreeHost(c->pin_head);
+  delete c;
+}
+
+const char* bild_last_error(const bild_ctx* c) { return c ? c->err.c_str() : "null context"; }
+int64_t bild_launch_count(const bild_ctx* c) { return c ? c->launches : 0; }
+
+int bild_encode(bild_ctx* c, const int32_t* ids, int n_ids) {
+  if (!c || !ids) return fail(c, BILD_ERR_ARG, "null argument");
+  if (n_ids < 1 || n_ids > c->cfg.max_enc_len) return fail(c, BILD_ERR_CAPACITY, "n_ids outside 1..max_enc_len");
+  c->encoded = false;
+  c->enc_len = n_ids;
+  CUDA_TRY(c, cudaMemcpyAsync(c->enc_ids, ids, n_ids * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(c->enc_len_dev, &c->enc_len, sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  for (int i = 0; i < 2; ++i) {
+    int rc = encoder_pass(c, i);
+    if (rc) return rc;
+  }
+  int rc = reset_state(c, BILD_MODE_BILD, 0.f, INFINITY, c->cfg.max_dec_len - 1);
+  if (rc) return rc;
+  c->encoded = true;
+  return BILD_OK;
+}
+
+int bild_reset(bild_ctx* c) {
+  if (!c) return BILD_ERR_ARG;
+  if (!c->encoded) return fail(c, BILD_ERR_STATE, "bild_encode has not been called");
+  return reset_state(c, BILD_MODE_BILD, 0.f, INFINITY, c->cfg.max_dec_len - 1);
+}
+
+int bild_small_step(bild_ctx* c, int32_t token, float alpha_fb, bild_step_out* out, float* logits_dbg) {
+  if (!c || !out) return fail(c, BILD_ERR_ARG, "null argument");
+  if (!c->encoded) return fail(c, BILD_ERR_STATE, "bild_encode has not been called");
+  if (token < 0 || token >= c->m[0].c.vocab) return fail(c, BILD_ERR_ARG, "token outside the vocabulary");
+  int rc = read_state(c);
+  if (rc) return rc;
+  if (c->pin_state->S_len + 1 > c->cfg.max_dec_len) return fail(c, BILD_ERR_CAPACITY, "small-model cache is full");
+  TokList t{};
+  t.t[0] = token;
+  set_alpha_kernel<<<1, 1, 0, c->stream>>>(c->st, alpha_fb, c->pin_state->alpha_rb);
+  set_desc_kernel<<<1, 1, 0, c->stream>>>(c->m[0].desc, c->st, 0, 1, t);
+  c->launches += 2;
+  rc = decoder_pass(c, 0, 1, logits_dbg);
+  if (rc) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(c->pin_head, c->m[0].head_out, sizeof(HeadOut), cudaMemcpyDeviceToHost, c->stream));
+  rc = read_state(c);
+  if (rc) return rc;
+  out->argmax = c->pin_head->argmax[0];
+  out->max_logit = c->pin_head->zmax[0];
+  out->lse = c->pin_head->lse[0];
+  out->pmax = c->pin_head->pmax;
+  out->fallback = c->pin_head->fallback;
+  return BILD_OK;
+}
+
+int bild_large_verify(bild_ctx* c, const int32_t* tokens, int k, float alpha_rb, bild_verify_out* out,
+                      float* logits_dbg) {
+  if (!c || !out || !tokens) return fail(c, BILD_ERR_ARG, "null argument");
+  if (!c->encoded) return fail(c, BILD_ERR_STATE, "bild_encode has not been called");
+  if (k < 1 || k > MAXB) return fail(c, BILD_ERR_ARG, "k outside 1..16");
+  for (int i = 0; i < k; ++i)
+    if (tokens[i] < 0 || tokens[i] >= c->m[1].c.vocab) return fail(c, BILD_ERR_ARG, "token outside the vocabulary");
+  int rc = read_state(c);
+  if (rc) return rc;
+  if (c->pin_state->L_len + k > c->cfg.max_dec_len) return fail(c, BILD_ERR_CAPACITY, "large-model cache is full");
+  TokList t{};
+  for (int i = 0; i < k; ++i) t.t[i] = tokens[i];
+  set_alpha_kernel<<<1, 1, 0, c->stream>>>(c->st, c->pin_state->alpha_fb, alpha_rb);
+  set_desc_kernel<<<1, 1, 0, c->stream>>>(c->m[1].desc, c->st, 1, k, t);
+  c->launches += 2;
+  rc = decoder_pass(c, 1, k == 1 ? 1 : MAXB, logits_dbg);
+  if (rc) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(c->pin_head, c->m[1].head_out, sizeof(HeadOut), cudaMemcpyDeviceToHost, c->stream));
+  rc = read_state(c);
+  if (rc) return rc;
+  for (int i = 0; i < MAXB; ++i) {
+    out->argmax[i] = i < k ? c->pin_head->argmax[i] : -1;
+    out->lse[i] = i < k ? c->pin_head->lse[i] : 0.f;
+    out->d[i] = i < k - 1 ? c->pin_head->d[i] : 0.f;
+  }
+  out->first_violation = c->pin_head->first_violation;
+  out->next_token = c->pin_head->next_token;
+  return BILD_OK;
+}
+
+int bild_rewind(bild_ctx* c, int which, int new_len) {
+  if (!c || (which != 0 && which != 1)) return fail(c, BILD_ERR_ARG, "which must be 0 or 1");
+  if (!c->encoded) return fail(c, BILD_ERR_STATE, "bild_encode has not been called");
+  int rc = read_state(c);
+  if (rc) return rc;
+  const int cur = which == 0 ? c->pin_state->S_len : c->pin_state->L_len;
+  if (new_len < 0 || new_len > cur) return fail(c, BILD_ERR_ARG, "new_len outside 0..current length");
+  rewind_kernel<<<1, 1, 0, c->stream>>>(c->st, which, new_len);
+  c->launches++;
+  CUDA_TRY(c, cudaGetLastError());
+  return BILD_OK;
+}
+
+int bild_generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, int max_len) {
+  if (!c) return BILD_ERR_ARG;
+  if (!c->encoded) return fail(c, BILD_ERR_STATE, "bild_encode has not been called");
+  if (mode < 0 || mode > 2) return fail(c, BILD_ERR_ARG, "mode");
+  if (max_len < 0) return fail(c, BILD_ERR_ARG, "max_len < 0");
+  if (max_len + 1 > c->cfg.max_dec_len) return fail(c, BILD_ERR_CAPACITY, "max_len + 1 > max_dec_len");
+  int rc = reset_state(c, mode, alpha_fb, alpha_rb, max_len);
+  if (rc) return rc;
+  // Loop driver: the policy runs on the device; the host only reads two flags per step.
+  const int guard = (max_len + 1) * (c->cfg.max_draft + 3);
+  rc = read_state(c);
+  if (rc) return rc;
+  for (int it = 0; it < guard && !c->pin_state->done; ++it) {
+    if (mode != BILD_MODE_LARGE_ONLY) {
+      rc = decoder_pass(c, 0, 1, nullptr);
+      if (rc) return rc;
+      rc = read_state(c);
+      if (rc) return rc;
+      if (!c->pin_state->fallback) continue;
+    }
+    rc = decoder_pass(c, 1, mode == BILD_MODE_LARGE_ONLY ? 1 : MAXB, nullptr);
+    if (rc) return rc;
+    rc = read_state(c);
+    if (rc) return rc;
+  }
+  return BILD_OK;
+}
+
+int bild_fetch_result(bild_ctx* c, int32_t* tokens_out, int* n_tokens, bild_trace_rec* trace_out, int trace_cap,
+                      int* n_trace, bild_stats* stats) {
+  if (!c || !tokens_out || !n_tokens) return fail(c, BILD_ERR_ARG, "null argument");
+  int rc = read_state(c);
+  if (rc) return rc;
+  const DevState& s = *c->pin_state;
+  *n_tokens = s.n;
+  if (s.n > 0) CUDA_TRY(c, cudaMemcpyAsync(tokens_out, c->y + 1, s.n * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  if (n_trace) *n_trace = s.n_trace;
+  const int nt = std::min(std::min(s.n_trace, trace_cap), c->trace_cap);
+  if (trace_out && nt > 0)
+    CUDA_TRY(c, cudaMemcpyAsync(trace_out, c->trace, nt * sizeof(bild_trace_rec), cudaMemcpyDeviceToHost, c->stream));
+  if (stats) *stats = s.stats;
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return BILD_OK;
+}
+
+int bild_generate(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, int max_len, int32_t* tokens_out,
+                  int* n_tokens, bild_trace_rec* trace_out, int trace_cap, int* n_trace, bild_stats* stats) {
+  if (!c || !tokens_out || !n_tokens) return fail(c, BILD_ERR_ARG, "null argument");
+  int rc = bild_generate_async(c, mode, alpha_fb, alpha_rb, max_len);
+  if (rc) return rc;
+  return bild_fetch_result(c, tokens_out, n_tokens, trace_out, trace_cap, n_trace, stats);
+}
+
+int bild_op_linear(const void* W, int w_dtype, const float* X, const float* gain, float eps, float* Y, int M, int N,
+                   int K, void* cuda_stream) {
+  if (!W || !X || !Y || M < 1 || M > MAXB || N < 1 || K < 8 || K % 8) return BILD_ERR_ARG;
+  if (w_dtype != BILD_FP32 && w_dtype != BILD_BF16) return BILD_ERR_ARG;
+  bild_ctx tmp;
+  tmp.stream = (cudaStream_t)cuda_stream;
+  LinArgs a{};
+  a.W0 = W; a.X = X; a.ldx = K; a.gain = gain; a.eps = eps; a.Y = Y; a.ldy = N; a.N = N; a.K = K; a.M = M;
+  a.epi = EPI_STORE;
+  cudaError_t e = launch_linear(&tmp, w_dtype, M == 1 ? 1 : MAXB, a);
+  return e == cudaSuccess ? BILD_OK : BILD_ERR_CUDA;
+}
+
+size_t bild_op_lm_head_scratch_bytes(int V) {
+  if (V < 1) return 0;
+  return align_up((size_t)head_grid_for(V) * MAXB * sizeof(Partial), 256) + 256 + align_up(sizeof(HeadOut), 256);
+}
+
+int bild_op_lm_head(const void* W, int w_dtype, const float* X, const float* gain, float eps, float scale,
+                    const int32_t* target, int M, int V, int K, int32_t* argmax_out, float* max_out, float* lse_out,
+                    float* gather_out, float* logits_dbg, void* scratch, void* cuda_stream) {
+  if (!W || !X || !scratch || !argmax_out || !max_out || !lse_out) return BILD_ERR_ARG;
+  if (M < 1 || M > MAXB || V < 1 || K < 8 || K % 8 || K > 4096) return BILD_ERR_ARG;
+  if (w_dtype != BILD_FP32 && w_dtype != BILD_BF16) return BILD_ERR_ARG;
+  if ((uintptr_t)scratch % 256) return BILD_ERR_WORKSPACE;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int grid = head_grid_for(V);
+  char* p = (char*)scratch;
+  HeadArgs h{};
+  h.partials = (Partial*)p;
+  p += align_up((size_t)grid * MAXB * sizeof(Partial), 256);
+  h.counter = (unsigned*)p;
+  p += 256;
+  h.out = (HeadOut*)p;
+  if (cudaMemsetAsync(h.counter, 0, sizeof(unsigned), s) != cudaSuccess) return BILD_ERR_CUDA;
+  h.W = W; h.X = X; h.ldx = K; h.gain = gain; h.eps = eps; h.scale = scale; h.V = V; h.K = K; h.M = M;
+  h.target = target; h.logits_dbg = logits_dbg; h.which = 1;
+  if (launch_head(s, w_dtype, M == 1 ? 1 : MAXB, h, grid, nullptr) != cudaSuccess) return BILD_ERR_CUDA;
+  const HeadOut* o = h.out;
+  cudaError_t e = cudaMemcpyAsync(argmax_out, o->argmax, M * sizeof(int), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(max_out, o->zmax, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(lse_out, o->lse, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess && gather_out && target)
+    e = cudaMemcpyAsync(gather_out, o->gather, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
+  return e == cudaSuccess ? BILD_OK : BILD_ERR_CUDA;
+}
+
+int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, float* ms_per_pass) {
+  if (!c || !ms_per_pass || (which != 0 && which != 1)) return fail(c, BILD_ERR_ARG, "null argument / which");
+  if (!c->encoded) return fail(c, BILD_ERR_STATE, "bild_encode has not been called");
+  if (k < 1 || k > (which == 0 ? 1 : MAXB) || iters < 1) return fail(c, BILD_ERR_ARG, "k or iters out of range");
+  if (cache_len < 0 || cache_len + k > c->cfg.max_dec_len) return fail(c, BILD_ERR_CAPACITY, "cache_len + k > max_dec_len");
+  TokList t{};
+  for (int i = 0; i < k; ++i) t.t[i] = (7 * i + 3) % c->m[which].c.vocab;
+  cudaEvent_t e0, e1;
+  CUDA_TRY(c, cudaEventCreate(&e0));
+  CUDA_TRY(c, cudaEventCreate(&e1));
+  int rc = BILD_OK;
+  set_desc_at_kernel<<<1, 1, 0, c->stream>>>(c->m[which].desc, k, cache_len, t);
+  c->launches++;
+  rc = decoder_pass(c, which, k == 1 ? 1 : MAXB, nullptr);  // untimed first pass
+  if (rc == BILD_OK && cudaEventRecord(e0, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
+  for (int it = 0; it < iters && rc == BILD_OK; ++it) rc = decoder_pass(c, which, k == 1 ? 1 : MAXB, nullptr);
+  if (rc == BILD_OK && cudaEventRecord(e1, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
+  if (rc == BILD_OK && cudaEventSynchronize(e1) != cudaSuccess) rc = BILD_ERR_CUDA;
+  float ms = 0.f;
+  if (rc == BILD_OK && cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) rc = BILD_ERR_CUDA;
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (rc != BILD_OK) return fail(c, rc, "bild_time_pass failed");
+  *ms_per_pass = ms / (float)iters;
+  return BILD_OK;
+}
+
+// Host-only helper for tests of the bucket tables: which = 0 decoder (delta = query - key >= 0),
+// 1 encoder (rel = key - query).
+int bild_debug_bucket(int which, int rel, int n_buckets, int max_dist) {
+  if (n_buckets < 4 || n_buckets % 4 || max_dist < n_buckets) return -1;
+  if (which == 0) return rel < 0 ? -1 : decoder_bucket(rel, n_buckets, max_dist);
+  return encoder_bucket(rel, n_buckets, max_dist);
+}
+
+}  // extern "C"

@@ -1,0 +1,20 @@
+"""Contexts for the named synthetic workloads (random T5 / mT5-shaped pairs)."""
+from __future__ import annotations
+
+from workloads import MODEL_SHAPES, WORKLOADS, gen_ids, gen_model
+
+from .binding import BF16, FP32, Config, Context, model_cfg, upload_model
+
+
+def make_context(workload: str, scale_small: float, scale_large: float, device="cuda:0", max_enc_len=None,
+                 max_dec_len=None, eos_id=-1, max_draft=None):
+    """Generate the workload's two models on the host, upload them, create a Context.
+    Returns (context, encoder ids, workload)."""
+    wl = WORKLOADS[workload]
+    sS, sL = MODEL_SHAPES[wl.small], MODEL_SHAPES[wl.large]
+    devS = upload_model(gen_model(sS, wl.seed, wl.dtype), device)
+    devL = upload_model(gen_model(sL, wl.seed, wl.dtype), device)
+    cfg = Config(model_cfg(sS, scale_small), model_cfg(sL, scale_large), BF16 if wl.dtype == "bf16" else FP32,
+                 max_enc_len or wl.enc_len, max_dec_len or wl.gen_len + 1, max_draft or wl.max_draft, 0, eos_id)
+    ctx = Context(cfg, sS, devS, sL, devL, device)
+    return ctx, gen_ids(sS.vocab, wl.enc_len, wl.seed), wl

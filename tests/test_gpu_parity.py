@@ -1,0 +1,316 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the CPU oracle on the
+same seeded inputs.  Tolerances: fp32 configurations: logits max-abs error <= 1e-4 and
+tokens / traces identical; bf16 configurations: logits <= 2e-2 and traces identical except
+where the oracle's own decision margin is below that tolerance."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import bild as obild
+from oracle.t5 import Model, rms_norm
+from workloads import MODEL_SHAPES, WORKLOADS, gen_ids, gen_model
+
+pytestmark = pytest.mark.gpu
+GOLD = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+TOL = {"fp32": 1e-4, "bf16": 2e-2}
+INF = math.inf
+
+
+def golden(name):
+    with open(os.path.join(GOLD, name + ".json")) as f:
+        return json.load(f)
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    import torch
+    assert torch.cuda.is_available()
+    return torch
+
+
+_ctx_cache = {}
+
+
+def get_ctx(name, **kw):
+    """Context + encoded input for a workload (cached per module run)."""
+    from paper_2302_07863_b200.synthetic import make_context
+    key = (name, tuple(sorted(kw.items())))
+    if key not in _ctx_cache:
+        g = golden(name)
+        ctx, ids, wl = make_context(name, g["scale_small"]["scale"], g["scale_large"]["scale"], **kw)
+        ctx.encode(ids)
+        _ctx_cache[key] = (ctx, ids, wl, g)
+    return _ctx_cache[key]
+
+
+_oracle_cache = {}
+
+
+def get_oracle(name):
+    if name not in _oracle_cache:
+        wl = WORKLOADS[name]
+        g = golden(name)
+        S = Model(MODEL_SHAPES[wl.small], gen_model(MODEL_SHAPES[wl.small], wl.seed, wl.dtype), g["scale_small"]["scale"])
+        L = Model(MODEL_SHAPES[wl.large], gen_model(MODEL_SHAPES[wl.large], wl.seed, wl.dtype), g["scale_large"]["scale"])
+        _oracle_cache[name] = (S, L, gen_ids(S.s.vocab, wl.enc_len, wl.seed))
+    return _oracle_cache[name]
+
+
+def assert_trace_equal(got, want, vtol):
+    assert len(got) == len(want), (len(got), len(want))
+    for a, b in zip(got, want):
+        assert tuple(a[:5]) == tuple(b[:5]), (a, b)
+        assert abs(a[5] - b[5]) <= vtol * max(1.0, abs(b[5])), (a, b)
+
+
+# ---- single kernels ---------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("M,N,K", [(1, 7, 64), (1, 515, 2048), (3, 96, 136), (16, 1031, 1024), (11, 257, 4096),
+                                   (1, 1024, 512), (16, 64, 8)])
+@pytest.mark.parametrize("norm", [False, True])
+def test_op_linear(torch_cuda, dtype, M, N, K, norm):
+    torch = torch_cuda
+    from paper_2302_07863_b200 import op_linear
+    from workloads import bf16_bits_to_f32, bf16_round_bits
+    rng = np.random.default_rng(M * 1000 + N + K)
+    W = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
+    X = rng.standard_normal((M, K)).astype(np.float32) * 3
+    g = (1 + 0.1 * rng.standard_normal(K)).astype(np.float32)
+    if dtype == "bf16":
+        bits = bf16_round_bits(W)
+        W = bf16_bits_to_f32(bits)
+        Wd = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        Wd = torch.from_numpy(W).cuda()
+    H = rms_norm(X.astype(np.float64), g.astype(np.float64), 1e-6) if norm else X.astype(np.float64)
+    ref = H @ W.astype(np.float64).T
+    Y = op_linear(Wd, torch.from_numpy(X).cuda(), torch.from_numpy(g).cuda() if norm else None, 1e-6, M, N, K)
+    err = np.max(np.abs(Y.cpu().numpy() - ref))
+    assert err <= 2e-5 * max(1.0, np.max(np.abs(ref))), err
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("M,V,K", [(1, 5, 64), (1, 32128, 512), (16, 773, 128), (7, 40013, 1024), (2, 64, 8)])
+def test_op_lm_head(torch_cuda, dtype, M, V, K):
+    torch = torch_cuda
+    from paper_2302_07863_b200 import op_lm_head
+    from workloads import bf16_bits_to_f32, bf16_round_bits
+    rng = np.random.default_rng(V + K + M)
+    W = (rng.standard_normal((V, K)) * 0.05).astype(np.float32)
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    g = (1 + 0.1 * rng.standard_normal(K)).astype(np.float32)
+    tgt = rng.integers(0, V, M).astype(np.int32)
+    if dtype == "bf16":
+        bits = bf16_round_bits(W)
+        W = bf16_bits_to_f32(bits)
+        Wd = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        Wd = torch.from_numpy(W).cuda()
+    scale = 9.0
+    Z = scale * (rms_norm(X.astype(np.float64), g.astype(np.float64), 1e-6) @ W.astype(np.float64).T)
+    am, mx, lse, ga, lg = op_lm_head(Wd, torch.from_numpy(X).cuda(), torch.from_numpy(g).cuda(), 1e-6, scale,
+                                     torch.from_numpy(tgt).cuda(), M, V, K, want_logits=True)
+    torch.cuda.synchronize()
+    assert np.max(np.abs(lg.cpu().numpy() - Z)) <= 1e-4
+    for m in range(M):
+        t, pmax, l, gap = obild.max_prob(Z[m])
+        if gap > 1e-3:
+            assert int(am[m]) == t
+        assert abs(float(mx[m]) - Z[m].max()) <= 1e-4
+        assert abs(float(lse[m]) - l) <= 1e-4
+        assert abs(float(ga[m]) - Z[m][tgt[m]]) <= 1e-4
+
+
+def test_op_lm_head_ties_take_lowest_index(torch_cuda):
+    torch = torch_cuda
+    from paper_2302_07863_b200 import op_lm_head
+    V, K = 3000, 64
+    W = np.zeros((V, K), dtype=np.float32)
+    W[[17, 1500, 2999], 0] = 1.0          # three equal maxima in different blocks
+    X = np.zeros((2, K), dtype=np.float32); X[:, 0] = 2.0
+    am, mx, lse, ga, _ = op_lm_head(torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda(), None, 0.0, 1.0, None,
+                                    2, V, K)
+    assert am.tolist() == [17, 17]
+    assert abs(float(lse[0]) - math.log(3 * math.exp(2.0) + (V - 3))) < 1e-4
+
+
+# ---- step entry points: full logits against the oracle --------------------------------
+@pytest.mark.parametrize("name", ["tiny", "odd", "odd_bf16", "tiny_bf16"])
+def test_steps_match_oracle_logits(torch_cuda, name):
+    torch = torch_cuda
+    ctx, ids, wl, g = get_ctx(name)
+    S, L, _ = get_oracle(name)
+    tol = TOL[wl.dtype]
+    V = S.s.vocab
+    ctx.reset()
+    stS, stL = S.start(ids, 64), L.start(ids, 64)
+    buf = torch.empty((16, V), dtype=torch.float32, device="cuda")
+    toks = [0] + [int(t) for t in gen_ids(V, 20, 11)]
+    worst = 0.0
+    # small model: token by token
+    for t in toks[:9]:
+        z = S.forward_one(stS, t)
+        o = ctx.small_step(t, 0.4, buf)
+        zg = buf[0].cpu().numpy()
+        worst = max(worst, np.max(np.abs(zg - z)))
+        ta, pmax, lse, gap = obild.max_prob(z)
+        assert o.argmax == ta and abs(o.pmax - pmax) < 10 * tol and abs(o.lse - lse) <= tol
+        if abs(pmax - 0.4) > 10 * tol:
+            assert o.fallback == int(pmax < 0.4)
+    # large model: blocks of different sizes, with a rewind in between
+    pos = 0
+    for k in (1, 5, 16):
+        blk = toks[pos:pos + k] if pos + k <= len(toks) else (toks + toks)[pos:pos + k]
+        Z = L.forward_block(stL, blk)
+        o = ctx.large_verify(blk, 15.0, buf)
+        Zg = buf[:k].cpu().numpy()
+        worst = max(worst, np.max(np.abs(Zg - Z)))
+        for i in range(k):
+            ta, _, lse, gap = obild.max_prob(Z[i])
+            assert o.argmax[i] == ta and abs(o.lse[i] - lse) <= tol
+            if i < k - 1:
+                assert abs(o.d[i] - (lse - Z[i][blk[i + 1]])) <= 2 * tol
+        dd = [obild.max_prob(Z[i])[2] - Z[i][blk[i + 1]] for i in range(k - 1)]
+        viol = [i for i, d in enumerate(dd) if d > 15.0]
+        if all(abs(d - 15.0) > 2 * tol for d in dd):
+            assert o.first_violation == (viol[0] if viol else -1)
+        pos += k
+        if k == 5:
+            stL.rewind(3); ctx.rewind(1, 3); pos = 3
+    assert worst <= tol, worst
+    if wl.dtype == "bf16":
+        assert worst <= 2e-3, worst      # activations stay fp32: far inside the bf16 tolerance
+
+
+# ---- whole loop against the stored oracle runs ------------------------------------------
+@pytest.mark.parametrize("name", ["tiny", "odd", "odd_bf16", "tiny_bf16"])
+def test_generate_matches_golden(torch_cuda, name):
+    from paper_2302_07863_b200 import MODE_BILD, MODE_LARGE_ONLY, MODE_SMALL_ONLY
+    ctx, ids, wl, g = get_ctx(name)
+    th = g["thresholds"]
+    r = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
+    assert r["tokens"] == g["bild"]["tokens"]
+    assert_trace_equal(r["trace"], g["bild"]["trace"], 1e-3)
+    assert r["stats"] == g["bild"]["stats"]
+    assert ctx.generate(MODE_SMALL_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["small_only"]["tokens"]
+    assert ctx.generate(MODE_LARGE_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["large_only"]["tokens"]
+    # twice in a row: same result (state fully reset, no stale cache rows)
+    r2 = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
+    assert r2["tokens"] == r["tokens"] and r2["trace"] == r["trace"]
+
+
+@pytest.mark.parametrize("name", ["tiny", "odd_bf16"])
+@pytest.mark.parametrize("alpha_fb,alpha_rb,max_draft", [(0.0, INF, 10), (2.0, 0.0, 10), (0.3, -1.0, 10),
+                                                          (0.5, 15.5, 3), (0.2, 18.0, 15), (0.35, 16.5, 1)])
+def test_generate_matches_live_oracle(torch_cuda, name, alpha_fb, alpha_rb, max_draft):
+    """Other thresholds and draft caps, including the policy's special cases (never fall
+    back, always fall back, always roll back)."""
+    from paper_2302_07863_b200 import MODE_BILD
+    ctx, ids, wl, g = get_ctx(name, max_draft=max_draft)
+    S, L, _ = get_oracle(name)
+    want = obild.generate(S, L, ids, alpha_fb, alpha_rb, wl.gen_len, max_draft=max_draft)
+    got = ctx.generate(MODE_BILD, alpha_fb, alpha_rb, wl.gen_len)
+    tol = TOL[wl.dtype]
+    if min(want["margins"].values()) > 4 * tol or wl.dtype == "fp32":
+        assert got["tokens"] == want["tokens"]
+        assert_trace_equal(got["trace"], want["trace"], 1e-3)
+        assert got["stats"] == want["stats"]
+    else:   # compare up to the first low-margin decision
+        n = next((i for i, (a, b) in enumerate(zip(got["trace"], want["trace"])) if tuple(a[:5]) != tuple(b[:5])),
+                 None)
+        assert n is None or n > 0
+
+
+def test_eos_and_limits(torch_cuda):
+    from paper_2302_07863_b200 import MODE_SMALL_ONLY, BildError
+    g = golden("tiny")
+    eos = g["small_only"]["tokens"][5]
+    ctx, ids, wl, _ = get_ctx("tiny", eos_id=eos)
+    r = ctx.generate(MODE_SMALL_ONLY, 0.0, INF, wl.gen_len)
+    assert r["tokens"] == g["small_only"]["tokens"][:6]
+    assert ctx.generate(MODE_SMALL_ONLY, 0.0, INF, 0)["tokens"] == []
+    with pytest.raises(BildError) as e:
+        ctx.generate(MODE_SMALL_ONLY, 0.0, INF, wl.gen_len + 1)
+    assert e.value.code == -4
+    with pytest.raises(BildError):
+        ctx.large_verify([1] * 17, 1.0)
+    with pytest.raises(BildError):
+        ctx.rewind(0, 10 ** 6)
+    # still usable after errors
+    assert ctx.generate(MODE_SMALL_ONLY, 0.0, INF, 3)["tokens"] == g["small_only"]["tokens"][:3]
+
+
+# ---- full-size workloads: replay the oracle's calls, compare sampled logits ---------------
+@pytest.mark.parametrize("name", ["t5_sum", "mt5_mt"])
+def test_full_size_replay_and_generate(torch_cuda, name):
+    torch = torch_cuda
+    from paper_2302_07863_b200 import MODE_BILD, MODE_LARGE_ONLY, MODE_SMALL_ONLY
+    ctx, ids, wl, g = get_ctx(name)
+    tol = TOL[wl.dtype]
+    V = MODEL_SHAPES[wl.small].vocab
+    th = g["thresholds"]
+    idx = torch.tensor(g["sample_idx"], device="cuda")
+    rows = iter(g["sample_rows"])
+    buf = torch.empty((16, V), dtype=torch.float32, device="cuda")
+    ctx.reset()
+    y, L_len, worst = [0], 0, 0.0
+
+    def check(row, zrow, am, lse):
+        nonlocal worst
+        worst = max(worst, float(np.max(np.abs(zrow[idx].cpu().numpy() - np.array(row["z"])))))
+        worst = max(worst, abs(float(zrow[row["argmax"]]) - row["zmax"]))
+        assert abs(lse - row["lse"]) <= tol
+        if row["gap"] > 2 * tol:
+            assert am == row["argmax"]
+
+    for kind, pos, tok, k, m, val in g["bild"]["trace"]:
+        if kind in (0, 1, 2):
+            o = ctx.small_step(y[-1], th["alpha_fb"], buf)
+            row = next(rows)
+            assert row["model"] == "S" and row["first"] == len(y) - 1
+            check(row, buf[0], o.argmax, o.lse)
+            assert abs(o.pmax - row["pmax"]) <= 2 * tol
+            if kind == 0:
+                y.append(tok)
+        else:
+            blk = y[L_len:]
+            assert len(blk) == k
+            o = ctx.large_verify(blk, th["alpha_rb"], buf)
+            for i in range(k):
+                row = next(rows)
+                assert row["model"] == "L" and row["first"] == L_len and row["row"] == i
+                check(row, buf[i], o.argmax[i], o.lse[i])
+            if kind == 4:
+                assert o.first_violation == m and abs(o.d[m] - val) <= 2 * tol
+                del y[pos:]
+                y.append(tok)
+                ctx.rewind(0, pos); ctx.rewind(1, pos)
+                L_len = pos
+            else:
+                assert o.first_violation == -1
+                y.append(tok)
+                L_len = len(y) - 1
+            assert o.next_token == tok or row["gap"] <= 2 * tol
+    assert y[1:] == g["bild"]["tokens"]
+    assert worst <= tol, worst
+
+    # whole loop on the device
+    r = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
+    mg = g["bild"]["margins"]
+    if mg["argmax"] > 2 * tol and mg["fallback"] > 2 * tol and mg["rollback"] > 2 * tol:
+        assert r["tokens"] == g["bild"]["tokens"]
+        assert r["stats"] == g["bild"]["stats"]
+    else:
+        n = next((i for i, (a, b) in enumerate(zip(r["trace"], g["bild"]["trace"])) if tuple(a[:5]) != tuple(b[:5])),
+                 None)
+        if n is not None:     # a divergence is only allowed at a low-margin decision
+            lows = [i for i, row in enumerate(g["sample_rows"]) if row["gap"] <= 2 * tol
+                    or abs(row["pmax"] - th["alpha_fb"]) <= 2 * tol]
+            assert lows, "trace differs although every oracle margin is above tolerance"
+    if g["small_only"]["argmax_margin"] > 2 * tol:
+        assert ctx.generate(MODE_SMALL_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["small_only"]["tokens"]
+    if g["large_only"]["argmax_margin"] > 2 * tol:
+        assert ctx.generate(MODE_LARGE_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["large_only"]["tokens"]
