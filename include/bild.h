@@ -240,6 +240,29 @@ int bild_op_lm_head(const void *W, int w_dtype, const float *X, const float *gai
                     int32_t *argmax_out, float *max_out, float *lse_out, float *gather_out,
                     float *logits_dbg, void *scratch, void *cuda_stream);
 
+/* The paper has no counterpart for this call; it exists for callers that cannot allocate.
+ * Same computation and outputs as bild_op_lm_head, but the kernel's scratch (block
+ * partials, ticket counter, result record) is a fixed 128 KiB array inside the library's
+ * device image, so the caller passes no scratch and nothing is allocated here: no
+ * cudaMalloc / cudaFree, no allocating library routine.  Meant for a decode worker inside
+ * a serving process whose allocator already owns the device's memory, or for a
+ * latency-critical loop where cudaMalloc's device-wide synchronisation is not acceptable.
+ *   - Limits: M <= 16, V <= 1048576, K <= 4096 (multiple of 8); beyond them the call
+ *     returns BILD_ERR_CAPACITY (and says why on stderr) - use bild_op_lm_head then.
+ *   - Every GPU that loads the library holds the 128 KiB until the process exits.
+ *   - The first call on a device looks the array's device address up (a runtime call that
+ *     is not a stream operation), so make that first call before any stream capture, with
+ *     the intended device current.
+ *   - All calls on a device share the one array and it keeps the previous call's
+ *     contents; the call clears what must start at zero on the given stream.  Two calls
+ *     whose kernels overlap on the GPU (different streams, no ordering) race on it and
+ *     give wrong results: order them.
+ *   - No logits debug dump.  Asynchronous on the stream; all pointers DEVICE. */
+int bild_op_lm_head_static(const void *W, int w_dtype, const float *X, const float *gain, float eps,
+                           float scale, const int32_t *target, int M, int V, int K,
+                           int32_t *argmax_out, float *max_out, float *lse_out, float *gather_out,
+                           void *cuda_stream);
+
 /* Host-only: the relative-position bucket the library uses (T5's bucket function in
  * exact integer arithmetic).  which = 0: decoder, rel = query_pos - key_pos >= 0;
  * which = 1: encoder, rel = key_pos - query_pos.  Returns -1 on invalid arguments. */

@@ -25,7 +25,7 @@ MAX_BLOCK = 16
 EXPORTS = ["bild_query_workspace", "bild_create", "bild_destroy", "bild_encode", "bild_reset",
            "bild_small_step", "bild_large_verify", "bild_rewind", "bild_generate", "bild_generate_async",
            "bild_fetch_result", "bild_time_pass", "bild_launch_count", "bild_last_error", "bild_op_linear",
-           "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_debug_bucket"]
+           "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_op_lm_head_static", "bild_debug_bucket"]
 
 
 class ModelCfg(C.Structure):
@@ -109,6 +109,7 @@ def lib() -> C.CDLL:
         L.bild_op_lm_head_scratch_bytes.argtypes = [i32]
         L.bild_op_lm_head_scratch_bytes.restype = C.c_size_t
         L.bild_op_lm_head.argtypes = [vp, i32, vp, vp, f32, f32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.bild_op_lm_head_static.argtypes = [vp, i32, vp, vp, f32, f32, vp, i32, i32, i32, vp, vp, vp, vp, vp]
         L.bild_debug_bucket.argtypes = [i32, i32, i32, i32]
         _lib = L
     return _lib
@@ -288,3 +289,24 @@ def op_lm_head(W, X, gain, eps, scale, target, M, V, K, want_logits=False, strea
     if rc != BILD_OK:
         raise BildError(rc, "bild_op_lm_head")
     return am, mx, lse, ga, lg
+
+
+def op_lm_head_static(W, X, gain, eps, scale, target, M, V, K, stream=None):
+    """bild_op_lm_head_static: the fused LM head for callers that cannot allocate scratch
+    (a worker inside a process whose allocator owns the device, or a loop that must not
+    hit cudaMalloc's device-wide synchronisation).  Only the four small output tensors are
+    created here, by the test harness; the library call itself allocates nothing."""
+    import torch
+    dev = X.device
+    am = torch.empty(M, dtype=torch.int32, device=dev)
+    mx = torch.empty(M, dtype=torch.float32, device=dev)
+    lse = torch.empty(M, dtype=torch.float32, device=dev)
+    ga = torch.zeros(M, dtype=torch.float32, device=dev)
+    dt = BF16 if W.dtype == torch.bfloat16 else FP32
+    rc = lib().bild_op_lm_head_static(W.data_ptr(), dt, X.data_ptr(), gain.data_ptr() if gain is not None else None,
+                                      eps, scale, target.data_ptr() if target is not None else None, M, V, K,
+                                      am.data_ptr(), mx.data_ptr(), lse.data_ptr(), ga.data_ptr(),
+                                      stream.cuda_stream if stream is not None else None)
+    if rc != BILD_OK:
+        raise BildError(rc, "bild_op_lm_head_static")
+    return am, mx, lse, ga

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbild.so")
-SOURCES = ["bild.cu"]
+SOURCES = ["bild.cu", "no_alloc.cu"]
 
 
 def _newest(paths):
