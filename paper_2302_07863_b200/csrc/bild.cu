@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -121,6 +122,15 @@ struct bild_ctx {
   DevState* pin_state = nullptr;  // pinned host mirror for the loop driver
   HeadOut* pin_head = nullptr;
   size_t ws_bytes = 0;
+  // device-side loop: WHILE { small pass; IF (fallback) { large block pass } } and WHILE { large pass }
+  cudaGraph_t graph[2] = {nullptr, nullptr};
+  cudaGraphExec_t exec[2] = {nullptr, nullptr};
+  int64_t per_pass[2] = {0, 0};      // kernel launches in one small / one large pass of the graphs
+  int64_t per_pass_large1 = 0;
+  int64_t* cnt = &launches;         // where launches are counted (redirected while capturing)
+  cudaStream_t cap_stream = nullptr;  // capture only (the legacy default stream cannot capture); nothing runs on it
+  bool host_loop = false;            // debug: drive the loop from the host, one read-back per step
+  int graph_run_mode = -1;           // mode of a graph run whose launches are not yet counted
 };
 
 namespace {
@@ -225,7 +235,7 @@ cudaError_t launch_linear_t(bild_ctx* c, const LinArgs& a, int rows_y) {
     if (e != cudaSuccess) return e;
   }
   kern<<<grid, LIN_THREADS, smem, c->stream>>>(a);
-  c->launches++;
+  (*c->cnt)++;
   return cudaGetLastError();
 }
 
@@ -268,7 +278,7 @@ cudaError_t launch_attn(bild_ctx* c, AttnArgs a, int rows, int keys_cap) {
   a.smem_keys = (keys_cap + a.nsplit - 1) / a.nsplit;
   dim3 grid(a.H, rows, a.nsplit);
   attn_kernel<<<grid, ATT_THREADS, (size_t)a.smem_keys * sizeof(float), c->stream>>>(a);
-  c->launches++;
+  (*c->cnt)++;
   return cudaGetLastError();
 }
 
@@ -276,7 +286,7 @@ template <typename WT>
 void launch_embed_t(bild_ctx* c, const void* E, const int* tokens, const int* cnt_dev, int cnt_host, int rows,
                     int d, int vocab, float* x) {
   embed_kernel<WT><<<rows, 128, 0, c->stream>>>((const WT*)E, tokens, cnt_dev, cnt_host, d, vocab, x);
-  c->launches++;
+  (*c->cnt)++;
 }
 cudaError_t launch_embed(bild_ctx* c, const void* E, const int* tokens, const int* cnt_dev, int cnt_host, int rows,
                          int d, int vocab, float* x) {
@@ -295,7 +305,8 @@ LoopPtrs loop_ptrs(bild_ctx* c) {
 // (steps S0..S10 / L0..L10: embed, per layer [norm+QKV+append, self-attention, O+residual,
 // norm+cross-Q, cross-attention, cross-O+residual, norm+FFN-up, FFN-down+residual],
 // final norm + LM head + policy).  MB = 1 or MAXB selects the kernel variants.
-int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg) {
+int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned long long cond_while = 0,
+                 unsigned long long cond_if = 0) {
   Model& m = c->m[which];
   const bild_model_cfg& mc = m.c;
   const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
@@ -353,7 +364,8 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg) {
   h.W = m.w.lm_head; h.X = m.x; h.ldx = d; h.gain = (const float*)m.w.dec_final_ln; h.eps = mc.ln_eps;
   h.scale = mc.logit_scale; h.V = mc.vocab; h.K = d; h.desc = m.desc; h.partials = m.head_part;
   h.counter = m.head_cnt; h.out = m.head_out; h.logits_dbg = logits_dbg; h.which = which; h.loop = loop_ptrs(c);
-  CUDA_TRY(c, launch_head(c->stream, dt, MB, h, m.head_grid, &c->launches));
+  h.cond_while = cond_while; h.cond_if = cond_if;
+  CUDA_TRY(c, launch_head(c->stream, dt, MB, h, m.head_grid, c->cnt));
   return BILD_OK;
 }
 
@@ -412,7 +424,7 @@ int build_bias_tables(bild_ctx* c) {
     CUDA_TRY(c, cudaMemcpyAsync(c->bucket_tmp, tab.data(), cap * sizeof(int), cudaMemcpyHostToDevice, c->stream));
     bias_table_kernel<<<(cap + 127) / 128, 128, 0, c->stream>>>((const float*)m.w.dec_rel_bias, c->bucket_tmp, cap,
                                                                 m.c.n_heads, m.dec_bias);
-    c->launches++;
+    (*c->cnt)++;
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     const int ne = 2 * ecap - 1;
     std::vector<int> etab(ne);
@@ -420,8 +432,83 @@ int build_bias_tables(bild_ctx* c) {
     CUDA_TRY(c, cudaMemcpyAsync(c->bucket_tmp, etab.data(), ne * sizeof(int), cudaMemcpyHostToDevice, c->stream));
     bias_table_kernel<<<(ne + 127) / 128, 128, 0, c->stream>>>((const float*)m.w.enc_rel_bias, c->bucket_tmp, ne,
                                                                m.c.n_heads, m.enc_bias);
-    c->launches++;
+    (*c->cnt)++;
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  }
+  return BILD_OK;
+}
+
+// Adds a conditional node to `g` after `deps` and returns its body graph.
+int add_cond(bild_ctx* c, cudaGraph_t g, const cudaGraphNode_t* deps, size_t ndeps, cudaGraphConditionalHandle h,
+             cudaGraphConditionalNodeType type, cudaGraph_t* body) {
+  cudaGraphNodeParams p = {cudaGraphNodeTypeConditional};
+  p.conditional.handle = h;
+  p.conditional.type = type;
+  p.conditional.size = 1;
+  cudaGraphNode_t node;
+  CUDA_TRY(c, cudaGraphAddNode(&node, g, deps, ndeps, &p));
+  *body = p.conditional.phGraph_out[0];
+  return BILD_OK;
+}
+
+// Captures one decoder pass into `body`; returns the leaf nodes of the capture.
+int capture_pass(bild_ctx* c, cudaGraph_t body, int which, int MB, unsigned long long hw, unsigned long long hi,
+                 std::vector<cudaGraphNode_t>* leaves, int64_t* count) {
+  if (!c->cap_stream) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
+  CUDA_TRY(c, cudaStreamBeginCaptureToGraph(c->cap_stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed));
+  int64_t n = 0;
+  cudaStream_t user_stream = c->stream;
+  c->stream = c->cap_stream;
+  c->cnt = &n;
+  int rc = decoder_pass(c, which, MB, nullptr, hw, hi);
+  c->cnt = &c->launches;
+  c->stream = user_stream;
+  if (rc == BILD_OK && leaves) {
+    cudaStreamCaptureStatus st;
+    const cudaGraphNode_t* deps = nullptr;
+    size_t nd = 0;
+    if (cudaStreamGetCaptureInfo(c->cap_stream, &st, nullptr, nullptr, &deps, &nd) != cudaSuccess) rc = BILD_ERR_CUDA;
+    else leaves->assign(deps, deps + nd);
+  }
+  cudaGraph_t got = nullptr;
+  cudaError_t e = cudaStreamEndCapture(c->cap_stream, &got);
+  if (rc != BILD_OK) return rc;
+  if (e != cudaSuccess) return fail(c, BILD_ERR_CUDA, std::string("cudaStreamEndCapture: ") + cudaGetErrorString(e));
+  *count = n;
+  return BILD_OK;
+}
+
+// Builds the two device-side loops (CUDA graphs with conditional nodes).  The head
+// kernel's last block sets the WHILE handle to "not done" and the IF handle to "fallback".
+int build_graphs(bild_ctx* c) {
+  if (c->exec[0]) return BILD_OK;
+  {  // BiLD (and small-only): WHILE { small pass ; IF { large block pass } }
+    CUDA_TRY(c, cudaGraphCreate(&c->graph[0], 0));
+    cudaGraphConditionalHandle hw, hi;
+    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hw, c->graph[0], 1, cudaGraphCondAssignDefault));
+    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi, c->graph[0], 0, cudaGraphCondAssignDefault));
+    cudaGraph_t body = nullptr, ifbody = nullptr;
+    int rc = add_cond(c, c->graph[0], nullptr, 0, hw, cudaGraphCondTypeWhile, &body);
+    if (rc) return rc;
+    std::vector<cudaGraphNode_t> leaves;
+    rc = capture_pass(c, body, 0, 1, hw, hi, &leaves, &c->per_pass[0]);
+    if (rc) return rc;
+    rc = add_cond(c, body, leaves.data(), leaves.size(), hi, cudaGraphCondTypeIf, &ifbody);
+    if (rc) return rc;
+    rc = capture_pass(c, ifbody, 1, MAXB, hw, 0, nullptr, &c->per_pass[1]);
+    if (rc) return rc;
+    CUDA_TRY(c, cudaGraphInstantiate(&c->exec[0], c->graph[0], 0));
+  }
+  {  // large-only greedy: WHILE { large pass with k = 1 }
+    CUDA_TRY(c, cudaGraphCreate(&c->graph[1], 0));
+    cudaGraphConditionalHandle hw;
+    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hw, c->graph[1], 1, cudaGraphCondAssignDefault));
+    cudaGraph_t body = nullptr;
+    int rc = add_cond(c, c->graph[1], nullptr, 0, hw, cudaGraphCondTypeWhile, &body);
+    if (rc) return rc;
+    rc = capture_pass(c, body, 1, 1, hw, 0, nullptr, &c->per_pass_large1);
+    if (rc) return rc;
+    CUDA_TRY(c, cudaGraphInstantiate(&c->exec[1], c->graph[1], 0));
   }
   return BILD_OK;
 }
@@ -429,6 +516,13 @@ int build_bias_tables(bild_ctx* c) {
 int read_state(bild_ctx* c) {
   CUDA_TRY(c, cudaMemcpyAsync(c->pin_state, c->st, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (c->graph_run_mode >= 0) {  // a finished graph run: count the kernels it launched
+    const bild_stats& t = c->pin_state->stats;
+    c->launches += c->graph_run_mode == BILD_MODE_LARGE_ONLY
+                       ? t.large_calls * c->per_pass_large1
+                       : t.small_steps * c->per_pass[0] + t.large_calls * c->per_pass[1];
+    c->graph_run_mode = -1;
+  }
   if (c->pin_state->err) return fail(c, c->pin_state->err, "device-side error flag set");
   return BILD_OK;
 }
@@ -436,7 +530,7 @@ int read_state(bild_ctx* c) {
 int reset_state(bild_ctx* c, int mode, float afb, float arb, int max_len) {
   reset_state_kernel<<<1, 1, 0, c->stream>>>(loop_ptrs(c), mode, afb, arb, max_len, c->cfg.max_draft,
                                              c->cfg.eos_id, c->cfg.start_id, c->trace_cap);
-  c->launches++;
+  (*c->cnt)++;
   CUDA_TRY(c, cudaGetLastError());
   return BILD_OK;
 }
@@ -474,6 +568,9 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   if (!c) return BILD_ERR_ARG;
   c->cfg = *cfg;
   c->stream = (cudaStream_t)cuda_stream;
+  c->cnt = &c->launches;
+  const char* hl = std::getenv("BILD_HOST_LOOP");
+  c->host_loop = hl && hl[0] == '1';
   Bump b(workspace);
   plan(c, b);
   c->ws_bytes = b.off;
@@ -515,6 +612,11 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
 
 void bild_destroy(bild_ctx* c) {
   if (!c) return;
+  for (int i = 0; i < 2; ++i) {
+    if (c->exec[i]) cudaGraphExecDestroy(c->exec[i]);
+    if (c->graph[i]) cudaGraphDestroy(c->graph[i]);
+  }
+  if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
   if (c->pin_state) cudaFreeHost(c->pin_state);
   if (c->pin_head) cudaFreeHost(c->pin_head);
   delete c;
@@ -609,7 +711,7 @@ int bild_rewind(bild_ctx* c, int which, int new_len) {
   const int cur = which == 0 ? c->pin_state->S_len : c->pin_state->L_len;
   if (new_len < 0 || new_len > cur) return fail(c, BILD_ERR_ARG, "new_len outside 0..current length");
   rewind_kernel<<<1, 1, 0, c->stream>>>(c->st, which, new_len);
-  c->launches++;
+  (*c->cnt)++;
   CUDA_TRY(c, cudaGetLastError());
   return BILD_OK;
 }
@@ -620,9 +722,20 @@ int bild_generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, i
   if (mode < 0 || mode > 2) return fail(c, BILD_ERR_ARG, "mode");
   if (max_len < 0) return fail(c, BILD_ERR_ARG, "max_len < 0");
   if (max_len + 1 > c->cfg.max_dec_len) return fail(c, BILD_ERR_CAPACITY, "max_len + 1 > max_dec_len");
+  if (!c->host_loop) {
+    // device-side loop: no host involvement between the first and the last token
+    int rc = build_graphs(c);
+    if (rc) return rc;
+    rc = reset_state(c, mode, alpha_fb, alpha_rb, max_len);
+    if (rc) return rc;
+    if (max_len == 0 || c->cfg.start_id == c->cfg.eos_id) return BILD_OK;
+    CUDA_TRY(c, cudaGraphLaunch(c->exec[mode == BILD_MODE_LARGE_ONLY ? 1 : 0], c->stream));
+    c->graph_run_mode = mode;
+    return BILD_OK;
+  }
   int rc = reset_state(c, mode, alpha_fb, alpha_rb, max_len);
   if (rc) return rc;
-  // Loop driver: the policy runs on the device; the host only reads two flags per step.
+  // Debug loop driver: the policy still runs on the device; the host reads two flags per step.
   const int guard = (max_len + 1) * (c->cfg.max_draft + 3);
   rc = read_state(c);
   if (rc) return rc;
@@ -726,7 +839,7 @@ int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, floa
   CUDA_TRY(c, cudaEventCreate(&e1));
   int rc = BILD_OK;
   set_desc_at_kernel<<<1, 1, 0, c->stream>>>(c->m[which].desc, k, cache_len, t);
-  c->launches++;
+  (*c->cnt)++;
   rc = decoder_pass(c, which, k == 1 ? 1 : MAXB, nullptr);  // untimed first pass
   if (rc == BILD_OK && cudaEventRecord(e0, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
   for (int it = 0; it < iters && rc == BILD_OK; ++it) rc = decoder_pass(c, which, k == 1 ? 1 : MAXB, nullptr);

@@ -49,7 +49,7 @@ struct DevState {
   float alpha_fb, alpha_rb;
   int n_trace, trace_cap;
   bild_stats stats;
-  int pad;
+  int passes;   // decoder passes taken by the running loop (guards against a runaway loop)
 };
 
 struct Partial {  // running soft-max statistics of a slice of the vocabulary

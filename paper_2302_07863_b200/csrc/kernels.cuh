@@ -389,6 +389,14 @@ __device__ inline void policy_tests(HeadOut* o, const CallDesc* desc, const DevS
 __device__ inline void policy_step(const LoopPtrs& L, const HeadOut* o, const CallDesc* desc, int which) {
   DevState* st = L.st;
   int* y = L.y;
+  // Every pass adds a token or consumes a pending draft, so a run takes at most
+  // (max_len + 1) * (max_draft + 2) passes; beyond that the loop is stopped with an error.
+  if (++st->passes > (st->max_len + 1) * (st->max_draft + 2) + 8) {
+    st->err = BILD_ERR_TIMEOUT;
+    st->done = 1;
+    st->fallback = 0;
+    return;
+  }
   if (which == 0) {
     const int t = o->argmax[0];
     st->stats.small_steps++;
@@ -459,6 +467,8 @@ struct HeadArgs {
   float* logits_dbg;
   int which;  // 0 small, 1 large
   LoopPtrs loop;  // loop.st may be nullptr (single-operation entry point)
+  // handles of the graph's WHILE (loop goes on) and IF (large pass wanted) nodes; 0 = not in a graph
+  unsigned long long cond_while, cond_if;
 };
 
 constexpr int HEAD_THREADS = 256;
@@ -597,6 +607,8 @@ __global__ void __launch_bounds__(HEAD_THREADS) lm_head_kernel(HeadArgs a) {
       if (a.desc->run_policy) policy_step(a.loop, o, a.desc, a.which);
       else if (a.which == 0) a.loop.st->S_len = a.desc->pos0 + 1;
       else a.loop.st->L_len = a.desc->pos0 + a.desc->k;
+      if (a.cond_while) cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
+      if (a.cond_if) cudaGraphSetConditional(a.cond_if, a.loop.st->fallback ? 1u : 0u);
     }
   }
 }
@@ -644,6 +656,7 @@ __global__ void reset_state_kernel(LoopPtrs L, int mode, float alpha_fb, float a
   st->alpha_fb = alpha_fb; st->alpha_rb = alpha_rb;
   st->n_trace = 0; st->trace_cap = trace_cap;
   st->stats = bild_stats{0, 0, 0, 0, 0, 0, 0};
+  st->passes = 0;
   L.y[0] = start_id;
   st->done = (max_len <= 0 || start_id == eos_id) ? 1 : 0;
   if (mode == BILD_MODE_LARGE_ONLY) next_large(L); else next_small(L);
