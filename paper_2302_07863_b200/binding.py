@@ -24,7 +24,7 @@ MAX_BLOCK = 16
 
 EXPORTS = ["bild_query_workspace", "bild_create", "bild_destroy", "bild_encode", "bild_reset",
            "bild_small_step", "bild_large_verify", "bild_rewind", "bild_generate", "bild_generate_async",
-           "bild_fetch_result", "bild_time_pass", "bild_launch_count", "bild_last_error", "bild_op_linear",
+           "bild_fetch_result", "bild_time_pass", "bild_uses_tensor_cores", "bild_launch_count", "bild_last_error", "bild_op_linear",
            "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_op_lm_head_static", "bild_debug_bucket"]
 
 
@@ -101,6 +101,7 @@ def lib() -> C.CDLL:
         L.bild_fetch_result.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(i32), C.POINTER(TraceRec), i32,
                                         C.POINTER(i32), C.POINTER(Stats)]
         L.bild_time_pass.argtypes = [vp, i32, i32, i32, i32, C.POINTER(f32)]
+        L.bild_uses_tensor_cores.argtypes = [vp]
         L.bild_launch_count.argtypes = [vp]
         L.bild_launch_count.restype = C.c_int64
         L.bild_last_error.argtypes = [vp]
@@ -253,6 +254,9 @@ class Context:
         ms = C.c_float()
         self._check(self.L.bild_time_pass(self.h, which, k, cache_len, iters, C.byref(ms)))
         return ms.value
+
+    def uses_tensor_cores(self) -> bool:
+        return bool(self.L.bild_uses_tensor_cores(self.h))
 
     def launch_count(self) -> int:
         return self.L.bild_launch_count(self.h)

@@ -9,7 +9,8 @@
 #include <string>
 #include <vector>
 
-#include "kernels.cuh"
+#include "decode_kernels.cuh"
+#include "umma_linear.cuh"
 
 using namespace bild;
 
@@ -99,6 +100,9 @@ struct Model {
   HeadOut* head_out = nullptr;
   CallDesc* desc = nullptr;
   int head_grid = 0;
+  // TMA descriptors of the decoder's weight matrices (bf16 only): per layer qkv, o, cq, co, wi0, wi1, fo
+  std::vector<CUtensorMap> tmaps;
+  bool umma = false;
 };
 
 }  // namespace
@@ -129,6 +133,7 @@ struct bild_ctx {
   int64_t per_pass_large1 = 0;
   int64_t* cnt = &launches;         // where launches are counted (redirected while capturing)
   cudaStream_t cap_stream = nullptr;  // capture only (the legacy default stream cannot capture); nothing runs on it
+  bool use_pdl = true;               // launch pass kernels with programmatic stream serialization
   bool host_loop = false;            // debug: drive the loop from the host, one read-back per step
   int graph_run_mode = -1;           // mode of a graph run whose launches are not yet counted
 };
@@ -151,7 +156,7 @@ int check_model(const bild_model_cfg& c, std::string& why) {
   if (c.n_layers < 1 || c.d_model < 8 || c.n_heads < 1 || c.d_ff < 8 || c.vocab < 2) return bad("model sizes must be positive");
   if (c.d_model % 8 || c.d_ff % 8 || (c.n_heads * c.d_kv) % 8) return bad("d_model, d_ff and n_heads*d_kv must be multiples of 8");
   if (c.d_kv != 16 && c.d_kv != 32 && c.d_kv != 64 && c.d_kv != 128) return bad("d_kv must be 16, 32, 64 or 128");
-  if (c.d_model > 4096 || c.d_ff > 16384) return bad("d_model <= 4096 and d_ff <= 16384");
+  if (c.d_model > 2048 || c.d_ff > 16384) return bad("d_model <= 2048 and d_ff <= 16384");
   if (c.ffn_kind != BILD_FFN_RELU && c.ffn_kind != BILD_FFN_GATED_GELU) return bad("ffn_kind");
   if (c.rel_buckets < 4 || c.rel_buckets % 4 || c.rel_max_dist < c.rel_buckets) return bad("rel_buckets / rel_max_dist");
   if (!(c.ln_eps >= 0.f) || !(c.logit_scale > 0.f)) return bad("ln_eps >= 0 and logit_scale > 0");
@@ -166,7 +171,7 @@ int check_config(const bild_config* cfg, std::string& why) {
   if (rc) return rc;
   if (cfg->small_cfg.vocab != cfg->large_cfg.vocab) { why = "the two models must share a vocabulary"; return BILD_ERR_ARG; }
   if (cfg->dtype != BILD_FP32 && cfg->dtype != BILD_BF16) { why = "dtype"; return BILD_ERR_ARG; }
-  if (cfg->max_enc_len < 1 || cfg->max_enc_len > 4096) { why = "1 <= max_enc_len <= 4096"; return BILD_ERR_ARG; }
+  if (cfg->max_enc_len < 1 || cfg->max_enc_len > 2048) { why = "1 <= max_enc_len <= 2048"; return BILD_ERR_ARG; }
   if (cfg->max_dec_len < 2 || cfg->max_dec_len > 4096) { why = "2 <= max_dec_len <= 4096"; return BILD_ERR_ARG; }
   if (cfg->max_draft < 1 || cfg->max_draft > MAXB - 1) { why = "1 <= max_draft <= 15"; return BILD_ERR_ARG; }
   if (cfg->start_id < 0 || cfg->start_id >= cfg->small_cfg.vocab) { why = "start_id"; return BILD_ERR_ARG; }
@@ -222,6 +227,43 @@ void plan(bild_ctx* c, Bump& b) {
 }
 
 // ---- launches ------------------------------------------------------------------------
+// Every kernel of a pass is launched so that it may start while its predecessor drains
+// (programmatic dependent launch); each of them waits before touching dependent data.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(bild_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = c->use_pdl ? 1 : 0;
+  (*c->cnt)++;
+  return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
+template <typename WT, int RW>
+cudaError_t launch_gemv_t(bild_ctx* c, const LinArgs& a) {
+  const int nwarps = GEMV_THREADS / 32;
+  dim3 grid((a.N + nwarps * RW - 1) / (nwarps * RW));
+  if (a.epi == EPI_GATED) return launch_k(c, gemv_kernel<WT, RW, true>, grid, dim3(GEMV_THREADS), 0, a);
+  return launch_k(c, gemv_kernel<WT, RW, false>, grid, dim3(GEMV_THREADS), 0, a);
+}
+
+template <int MB>
+cudaError_t launch_battn_t(bild_ctx* c, BAttnArgs a, int row_blocks, int keys_cap) {
+  a.smem_keys = (keys_cap + a.nsplit - 1) / a.nsplit;
+  const size_t smem = (size_t)MB * a.smem_keys * sizeof(float);
+  if (smem > 16 * 1024) {  // static shared memory of the kernel takes about 17 KB of the default 48 KB
+    cudaError_t e = cudaFuncSetAttribute(battn_kernel<MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  return launch_k(c, battn_kernel<MB>, dim3(a.H, a.nsplit, row_blocks), dim3(BATT_THREADS), smem, a);
+}
+cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a, int row_blocks, int keys_cap) {
+  return MB == 1 ? launch_battn_t<1>(c, a, row_blocks, keys_cap) : launch_battn_t<MAXB>(c, a, row_blocks, keys_cap);
+}
+
 template <typename WT, int MB, int RW>
 cudaError_t launch_linear_t(bild_ctx* c, const LinArgs& a, int rows_y) {
   const int nwarps = LIN_THREADS / 32;
@@ -234,15 +276,16 @@ cudaError_t launch_linear_t(bild_ctx* c, const LinArgs& a, int rows_y) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  kern<<<grid, LIN_THREADS, smem, c->stream>>>(a);
-  (*c->cnt)++;
-  return cudaGetLastError();
+  if (gated) return launch_k(c, linear_kernel<WT, MB, RW, true>, grid, dim3(LIN_THREADS), smem, a);
+  return launch_k(c, linear_kernel<WT, MB, RW, false>, grid, dim3(LIN_THREADS), smem, a);
 }
 
+// MB == 1: the GEMV of the small-model step (and of the large model at k = 1);
+// otherwise the small-M GEMM over up to MAXB rows per row block.
 cudaError_t launch_linear(bild_ctx* c, int dtype, int MB, const LinArgs& a, int rows_y = 1) {
   if (dtype == BILD_BF16)
-    return MB == 1 ? launch_linear_t<__nv_bfloat16, 1, 4>(c, a, rows_y) : launch_linear_t<__nv_bfloat16, MAXB, 2>(c, a, rows_y);
-  return MB == 1 ? launch_linear_t<float, 1, 4>(c, a, rows_y) : launch_linear_t<float, MAXB, 2>(c, a, rows_y);
+    return MB == 1 ? launch_gemv_t<__nv_bfloat16, 2>(c, a) : launch_linear_t<__nv_bfloat16, MAXB, 2>(c, a, rows_y);
+  return MB == 1 ? launch_gemv_t<float, 2>(c, a) : launch_linear_t<float, MAXB, 2>(c, a, rows_y);
 }
 
 template <typename WT, int MB, int RW>
@@ -253,9 +296,8 @@ cudaError_t launch_head_t(bild_ctx* c, const HeadArgs& a, int grid, int64_t* lau
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  kern<<<grid, HEAD_THREADS, smem, c ? c->stream : nullptr>>>(a);
   if (launches) (*launches)++;
-  return cudaGetLastError();
+  return launch_k(c, kern, dim3(grid), dim3(HEAD_THREADS), smem, a);
 }
 
 cudaError_t launch_head(cudaStream_t s, int dtype, int MB, const HeadArgs& a, int grid, int64_t* launches) {
@@ -267,32 +309,130 @@ cudaError_t launch_head(cudaStream_t s, int dtype, int MB, const HeadArgs& a, in
 }
 
 int pick_nsplit(int ctas_without_split, int keys_cap) {
-  int ns = (2 * 148 + ctas_without_split - 1) / ctas_without_split;
+  int ns = (148 + ctas_without_split - 1) / ctas_without_split;
   ns = std::min(ns, std::max(1, keys_cap / 32));
   ns = std::max(1, std::min(ns, NSPLIT_MAX));
-  while ((keys_cap + ns - 1) / ns > 8192 && ns < NSPLIT_MAX) ++ns;
+  while ((keys_cap + ns - 1) / ns > 1024 && ns < NSPLIT_MAX) ++ns;   // scores of MAXB rows stay under 64 KB
   return ns;
 }
 
-cudaError_t launch_attn(bild_ctx* c, AttnArgs a, int rows, int keys_cap) {
-  a.smem_keys = (keys_cap + a.nsplit - 1) / a.nsplit;
-  dim3 grid(a.H, rows, a.nsplit);
-  attn_kernel<<<grid, ATT_THREADS, (size_t)a.smem_keys * sizeof(float), c->stream>>>(a);
-  (*c->cnt)++;
-  return cudaGetLastError();
-}
-
-template <typename WT>
-void launch_embed_t(bild_ctx* c, const void* E, const int* tokens, const int* cnt_dev, int cnt_host, int rows,
-                    int d, int vocab, float* x) {
-  embed_kernel<WT><<<rows, 128, 0, c->stream>>>((const WT*)E, tokens, cnt_dev, cnt_host, d, vocab, x);
-  (*c->cnt)++;
-}
 cudaError_t launch_embed(bild_ctx* c, const void* E, const int* tokens, const int* cnt_dev, int cnt_host, int rows,
                          int d, int vocab, float* x) {
-  if (c->cfg.dtype == BILD_BF16) launch_embed_t<__nv_bfloat16>(c, E, tokens, cnt_dev, cnt_host, rows, d, vocab, x);
-  else launch_embed_t<float>(c, E, tokens, cnt_dev, cnt_host, rows, d, vocab, x);
-  return cudaGetLastError();
+  if (c->cfg.dtype == BILD_BF16)
+    return launch_k(c, embed_kernel<__nv_bfloat16>, dim3(rows), dim3(128), 0, (const __nv_bfloat16*)E, tokens, cnt_dev,
+                    cnt_host, d, vocab, x);
+  return launch_k(c, embed_kernel<float>, dim3(rows), dim3(128), 0, (const float*)E, tokens, cnt_dev, cnt_host, d,
+                  vocab, x);
+}
+
+// ---- tensor-core path of the block pass ---------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Descriptor of a row-major bf16 matrix [N][K] for boxes of 128 rows x 64 columns, 128-byte swizzle.
+bool make_tmap(EncodeTiledFn enc, const void* W, int N, int K, CUtensorMap* out) {
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)N};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {UM_KB, UM_TILE_M};
+  cuuint32_t es[2] = {1, 1};
+  return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(W), dims, strides, box, es,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+enum { TM_QKV = 0, TM_O, TM_CQ, TM_CO, TM_WI0, TM_WI1, TM_FO, TM_PER_LAYER };
+
+// Builds the descriptors of one model; leaves m.umma false when the shapes do not fit the kernel.
+void setup_umma(bild_ctx* c, Model& m) {
+  m.umma = false;
+  const char* off = std::getenv("BILD_NO_UMMA");
+  if (off && off[0] == '1') return;
+  if (c->cfg.dtype != BILD_BF16) return;
+  const bild_model_cfg& mc = m.c;
+  if (mc.d_model % UM_KB || m.inner % UM_KB || mc.d_ff % UM_KB) return;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) {
+    cudaGetLastError();
+    return;
+  }
+  EncodeTiledFn enc = (EncodeTiledFn)fn;
+  const bool gated = mc.ffn_kind == BILD_FFN_GATED_GELU;
+  m.tmaps.resize((size_t)mc.n_layers * TM_PER_LAYER);
+  for (int l = 0; l < mc.n_layers; ++l) {
+    const bild_dec_layer& w = m.dec[l];
+    CUtensorMap* t = &m.tmaps[(size_t)l * TM_PER_LAYER];
+    bool ok = make_tmap(enc, w.wqkv, 3 * m.inner, mc.d_model, &t[TM_QKV]) &&
+              make_tmap(enc, w.wo, mc.d_model, m.inner, &t[TM_O]) &&
+              make_tmap(enc, w.wcq, m.inner, mc.d_model, &t[TM_CQ]) &&
+              make_tmap(enc, w.wco, mc.d_model, m.inner, &t[TM_CO]) &&
+              make_tmap(enc, w.wi0, mc.d_ff, mc.d_model, &t[TM_WI0]) &&
+              make_tmap(enc, gated ? w.wi1 : w.wi0, mc.d_ff, mc.d_model, &t[TM_WI1]) &&
+              make_tmap(enc, w.wfo, mc.d_model, mc.d_ff, &t[TM_FO]);
+    if (!ok) { m.tmaps.clear(); return; }
+  }
+  const int maxsm = 227 * 1024;
+  if (cudaFuncSetAttribute(umma_linear_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, maxsm) != cudaSuccess ||
+      cudaFuncSetAttribute(umma_linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, maxsm) != cudaSuccess) {
+    cudaGetLastError();
+    m.tmaps.clear();
+    return;
+  }
+  m.umma = true;
+}
+
+// Split of K over a cluster: enough blocks to pull the matrix at full bandwidth, at most 16 k blocks each.
+bool umma_plan(int N, int K, bool gated, int* cs_out, int* nkb_out) {
+  const int tiles = (N + UM_TILE_M - 1) / UM_TILE_M;
+  int best = 0;
+  for (int cs = 1; cs <= (gated ? 4 : 8); cs *= 2) {
+    if (K % (UM_KB * cs)) break;
+    const int nkb = K / UM_KB / cs;
+    if (nkb > 16 || umma_smem_bytes(gated, nkb, cs) > 227 * 1024) continue;
+    best = cs;
+    if (tiles * cs >= 96) break;
+  }
+  if (!best) return false;
+  *cs_out = best;
+  *nkb_out = K / UM_KB / best;
+  return true;
+}
+
+cudaError_t launch_umma(bild_ctx* c, const LinArgs& a, const CUtensorMap& t0, const CUtensorMap& t1, int cs, int nkb) {
+  const bool gated = a.epi == EPI_GATED;
+  UmmaArgs u;
+  u.lin = a; u.cs = cs; u.nkb = nkb; u.err = &c->st->err;
+  const int tiles = (a.N + UM_TILE_M - 1) / UM_TILE_M;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(tiles * cs); cfg.blockDim = dim3(UM_THREADS);
+  cfg.dynamicSmemBytes = umma_smem_bytes(gated, nkb, cs); cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (c->use_pdl) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (cs > 1) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = cs; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = at; cfg.numAttrs = na;
+  (*c->cnt)++;
+  if (gated) return cudaLaunchKernelEx(&cfg, umma_linear_kernel<true>, u, t0, t1);
+  return cudaLaunchKernelEx(&cfg, umma_linear_kernel<false>, u, t0, t1);
+}
+
+// Linear layer of a decoder pass: tensor cores for the bf16 block pass, SIMT otherwise.
+cudaError_t launch_dec_linear(bild_ctx* c, Model& m, int MB, const LinArgs& a, int layer, int which_map) {
+  int cs, nkb;
+  if (MB != 1 && m.umma && umma_plan(a.N, a.K, a.epi == EPI_GATED, &cs, &nkb)) {
+    const CUtensorMap* t = &m.tmaps[(size_t)layer * TM_PER_LAYER];
+    return launch_umma(c, a, t[which_map], t[which_map == TM_WI0 ? TM_WI1 : which_map], cs, nkb);
+  }
+  return launch_linear(c, c->cfg.dtype, MB, a);
 }
 
 LoopPtrs loop_ptrs(bild_ctx* c) {
@@ -312,7 +452,7 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
   const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len, dt = c->cfg.dtype;
   CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x));
-  const int ns_self = pick_nsplit(H * MB, cap), ns_cross = pick_nsplit(H * MB, ecap);
+  const int ns_self = pick_nsplit(H, cap), ns_cross = pick_nsplit(H, ecap);
   for (int l = 0; l < mc.n_layers; ++l) {
     const bild_dec_layer& w = m.dec[l];
     const size_t kvoff = (size_t)l * H * dkv;
@@ -322,42 +462,42 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
     a.W0 = w.wqkv; a.X = m.x; a.ldx = d; a.gain = (const float*)w.ln1; a.N = 3 * I; a.K = d;
     a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 0; a.q_out = m.q; a.ldq = I;
     a.kc = m.selfK + kvoff * cap; a.vc = m.selfV + kvoff * cap; a.cap = cap;
-    CUDA_TRY(c, launch_linear(c, dt, MB, a));
+    CUDA_TRY(c, launch_dec_linear(c, m, MB, a, l, TM_QKV));
     // S2 / L2: self-attention over the cache (causal inside the block)
-    AttnArgs t{};
+    BAttnArgs t{};
     t.q = m.q; t.ldq = I; t.kc = a.kc; t.vc = a.vc; t.cap = cap; t.out = m.att; t.ldo = I;
     t.bias = m.dec_bias; t.bias_ld = cap; t.bias_off = 0; t.mode = 1; t.dkv = dkv; t.H = H;
     t.n_keys_dev = c->enc_len_dev; t.desc = m.desc; t.part = m.att_part; t.counters = m.att_cnt;
     t.nsplit = ns_self; t.err = &c->st->err;
-    CUDA_TRY(c, launch_attn(c, t, MB, cap));
+    CUDA_TRY(c, launch_battn(c, MB, t, 1, cap));
     // S3 / L3: output projection + residual
     LinArgs o{};
     o.desc = m.desc; o.W0 = w.wo; o.X = m.att; o.ldx = I; o.N = d; o.K = I; o.epi = EPI_RESID; o.Y = m.x; o.ldy = d;
-    CUDA_TRY(c, launch_linear(c, dt, MB, o));
+    CUDA_TRY(c, launch_dec_linear(c, m, MB, o, l, TM_O));
     // S4 / L4: norm + cross-attention query
     LinArgs cq{};
     cq.desc = m.desc; cq.eps = mc.ln_eps; cq.W0 = w.wcq; cq.X = m.x; cq.ldx = d; cq.gain = (const float*)w.ln2;
     cq.N = I; cq.K = d; cq.epi = EPI_STORE; cq.Y = m.q; cq.ldy = I;
-    CUDA_TRY(c, launch_linear(c, dt, MB, cq));
+    CUDA_TRY(c, launch_dec_linear(c, m, MB, cq, l, TM_CQ));
     // S5 / L5: cross-attention over the encoder K/V
-    AttnArgs x{};
+    BAttnArgs x{};
     x.q = m.q; x.ldq = I; x.kc = m.crossK + kvoff * ecap; x.vc = m.crossV + kvoff * ecap; x.cap = ecap;
     x.out = m.att; x.ldo = I; x.mode = 0; x.dkv = dkv; x.H = H; x.n_keys_dev = c->enc_len_dev; x.desc = m.desc;
     x.part = m.att_part; x.counters = m.att_cnt; x.nsplit = ns_cross; x.err = &c->st->err;
-    CUDA_TRY(c, launch_attn(c, x, MB, ecap));
+    CUDA_TRY(c, launch_battn(c, MB, x, 1, ecap));
     // S6 / L6: cross output projection + residual
     o.W0 = w.wco;
-    CUDA_TRY(c, launch_linear(c, dt, MB, o));
+    CUDA_TRY(c, launch_dec_linear(c, m, MB, o, l, TM_CO));
     // S7 / L7: norm + FFN up (ReLU, or GELU gate)
     LinArgs up{};
     up.desc = m.desc; up.eps = mc.ln_eps; up.W0 = w.wi0; up.W1 = w.wi1; up.X = m.x; up.ldx = d;
     up.gain = (const float*)w.ln3; up.N = F; up.K = d; up.Y = m.u; up.ldy = F;
     up.epi = mc.ffn_kind == BILD_FFN_GATED_GELU ? EPI_GATED : EPI_RELU;
-    CUDA_TRY(c, launch_linear(c, dt, MB, up));
+    CUDA_TRY(c, launch_dec_linear(c, m, MB, up, l, TM_WI0));
     // S8 / L8: FFN down + residual
     LinArgs dn{};
     dn.desc = m.desc; dn.W0 = w.wfo; dn.X = m.u; dn.ldx = F; dn.N = d; dn.K = F; dn.epi = EPI_RESID; dn.Y = m.x; dn.ldy = d;
-    CUDA_TRY(c, launch_linear(c, dt, MB, dn));
+    CUDA_TRY(c, launch_dec_linear(c, m, MB, dn, l, TM_FO));
   }
   // S9+S10 / L9+L10: final norm + LM head + policy
   HeadArgs h{};
@@ -385,12 +525,12 @@ int encoder_pass(bild_ctx* c, int which) {
     a.N = 3 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 0; a.q_out = c->eq; a.ldq = I;
     a.kc = c->ek; a.vc = c->ev; a.cap = ecap; a.pos0_host = 0;
     CUDA_TRY(c, launch_linear(c, dt, MAXB, a, rb));
-    AttnArgs t{};
+    BAttnArgs t{};
     t.q = c->eq; t.ldq = I; t.kc = c->ek; t.vc = c->ev; t.cap = ecap; t.out = c->eatt; t.ldo = I;
     t.bias = m.enc_bias; t.bias_ld = 2 * ecap - 1; t.bias_off = ecap - 1; t.mode = 2; t.dkv = dkv; t.H = H;
     t.n_keys_dev = c->enc_len_dev; t.M = E; t.part = m.att_part; t.counters = m.att_cnt; t.nsplit = 1;
     t.err = &c->st->err;
-    CUDA_TRY(c, launch_attn(c, t, E, ecap));
+    CUDA_TRY(c, launch_battn(c, MAXB, t, rb, ecap));
     LinArgs o{};
     o.M = E; o.W0 = w.wo; o.X = c->eatt; o.ldx = I; o.N = d; o.K = I; o.epi = EPI_RESID; o.Y = c->ex; o.ldy = d;
     CUDA_TRY(c, launch_linear(c, dt, MAXB, o, rb));
@@ -480,8 +620,31 @@ int capture_pass(bild_ctx* c, cudaGraph_t body, int which, int MB, unsigned long
 
 // Builds the two device-side loops (CUDA graphs with conditional nodes).  The head
 // kernel's last block sets the WHILE handle to "not done" and the IF handle to "fallback".
+int build_graphs_once(bild_ctx* c);
+
+void drop_graphs(bild_ctx* c) {
+  for (int i = 0; i < 2; ++i) {
+    if (c->exec[i]) cudaGraphExecDestroy(c->exec[i]);
+    if (c->graph[i]) cudaGraphDestroy(c->graph[i]);
+    c->exec[i] = nullptr;
+    c->graph[i] = nullptr;
+  }
+}
+
 int build_graphs(bild_ctx* c) {
-  if (c->exec[0]) return BILD_OK;
+  if (c->exec[0] && c->exec[1]) return BILD_OK;
+  int rc = build_graphs_once(c);
+  if (rc != BILD_OK && c->use_pdl) {  // programmatic edges refused inside the loop bodies: plain edges
+    drop_graphs(c);
+    cudaGetLastError();
+    c->use_pdl = false;
+    rc = build_graphs_once(c);
+  }
+  if (rc != BILD_OK) drop_graphs(c);
+  return rc;
+}
+
+int build_graphs_once(bild_ctx* c) {
   {  // BiLD (and small-only): WHILE { small pass ; IF { large block pass } }
     CUDA_TRY(c, cudaGraphCreate(&c->graph[0], 0));
     cudaGraphConditionalHandle hw, hi;
@@ -571,6 +734,8 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   c->cnt = &c->launches;
   const char* hl = std::getenv("BILD_HOST_LOOP");
   c->host_loop = hl && hl[0] == '1';
+  const char* np = std::getenv("BILD_NO_PDL");
+  c->use_pdl = !(np && np[0] == '1');
   Bump b(workspace);
   plan(c, b);
   c->ws_bytes = b.off;
@@ -596,6 +761,7 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
     }
     m.w.enc_layers = nullptr;
     m.w.dec_layers = nullptr;
+    if (i == 1) setup_umma(c, m);
   }
   if (cudaMallocHost((void**)&c->pin_state, sizeof(DevState)) != cudaSuccess ||
       cudaMallocHost((void**)&c->pin_head, sizeof(HeadOut)) != cudaSuccess) {
@@ -612,15 +778,14 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
 
 void bild_destroy(bild_ctx* c) {
   if (!c) return;
-  for (int i = 0; i < 2; ++i) {
-    if (c->exec[i]) cudaGraphExecDestroy(c->exec[i]);
-    if (c->graph[i]) cudaGraphDestroy(c->graph[i]);
-  }
+  drop_graphs(c);
   if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
   if (c->pin_state) cudaFreeHost(c->pin_state);
   if (c->pin_head) cudaFreeHost(c->pin_head);
   delete c;
 }
+
+int bild_uses_tensor_cores(const bild_ctx* c) { return c && c->m[1].umma ? 1 : 0; }
 
 const char* bild_last_error(const bild_ctx* c) { return c ? c->err.c_str() : "null context"; }
 int64_t bild_launch_count(const bild_ctx* c) { return c ? c->launches : 0; }
@@ -840,11 +1005,22 @@ int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, floa
   int rc = BILD_OK;
   set_desc_at_kernel<<<1, 1, 0, c->stream>>>(c->m[which].desc, k, cache_len, t);
   (*c->cnt)++;
-  rc = decoder_pass(c, which, k == 1 ? 1 : MAXB, nullptr);  // untimed first pass
+  // the pass as a CUDA graph (as the decode loop runs it), replayed `iters` times
+  cudaGraph_t g = nullptr;
+  cudaGraphExec_t ex = nullptr;
+  if (cudaGraphCreate(&g, 0) != cudaSuccess) rc = BILD_ERR_CUDA;
+  int64_t n_launch = 0;
+  if (rc == BILD_OK) rc = capture_pass(c, g, which, k == 1 ? 1 : MAXB, 0, 0, nullptr, &n_launch);
+  if (rc == BILD_OK && cudaGraphInstantiate(&ex, g, 0) != cudaSuccess) rc = BILD_ERR_CUDA;
+  if (rc == BILD_OK && cudaGraphLaunch(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;  // untimed first pass
   if (rc == BILD_OK && cudaEventRecord(e0, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
-  for (int it = 0; it < iters && rc == BILD_OK; ++it) rc = decoder_pass(c, which, k == 1 ? 1 : MAXB, nullptr);
+  for (int it = 0; it < iters && rc == BILD_OK; ++it)
+    if (cudaGraphLaunch(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && cudaEventRecord(e1, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && cudaEventSynchronize(e1) != cudaSuccess) rc = BILD_ERR_CUDA;
+  if (rc == BILD_OK) c->launches += n_launch * (iters + 1);
+  if (ex) cudaGraphExecDestroy(ex);
+  if (g) cudaGraphDestroy(g);
   float ms = 0.f;
   if (rc == BILD_OK && cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) rc = BILD_ERR_CUDA;
   cudaEventDestroy(e0);

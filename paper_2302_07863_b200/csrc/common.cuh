@@ -99,6 +99,12 @@ __device__ __forceinline__ void load8(const float* p, float (&w)[8]) {
   w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
 }
 
+// Programmatic dependent launch: let the next kernel in the stream start its prologue,
+// and wait until everything the previous kernel wrote is visible.  Both are no-ops in a
+// kernel that was launched without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 

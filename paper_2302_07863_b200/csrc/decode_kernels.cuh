@@ -1,0 +1,294 @@
+// Latency-tuned kernels of the decode passes: the M = 1 weight-streaming GEMV of the
+// small-model step and the block attention that reads each cached key/value once for all
+// rows of the block.  All of them support programmatic dependent launch: what does not
+// depend on the previous kernel (the weight loads) is issued before the dependency wait.
+#pragma once
+#include "kernels.cuh"
+
+namespace bild {
+
+// ---------------------------------------------------------------------------------
+// GEMV for one activation row (steps S1, S3, S4, S6, S7, S8 of the small-model step):
+//   v[n] = inv_rms * sum_j W[n][j] * x[j] * g[j]        (inv_rms = 1, g = 1 without norm)
+// One warp owns RW weight rows.  Its first PRE*256 columns are loaded into registers
+// before the dependency wait; x, g and the sum of squares are taken in the same pass, so
+// there is no shared memory and no block-wide barrier.  Same epilogues as linear_kernel.
+// ---------------------------------------------------------------------------------
+constexpr int GEMV_THREADS = 128;
+constexpr int GEMV_PRE = 4;  // column chunks (of 256) whose weights are fetched ahead
+
+template <typename WT, int RW, bool GATED>
+__global__ void __launch_bounds__(GEMV_THREADS) gemv_kernel(LinArgs a) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = GEMV_THREADS / 32;
+  const int n0 = (blockIdx.x * nwarps + warp) * RW;
+  const int K = a.K;
+  const WT* W0 = (const WT*)a.W0;
+  const WT* W1 = (const WT*)a.W1;
+  const bool active = n0 < a.N;
+  float pre0[RW][GEMV_PRE][8], pre1[GATED ? RW : 1][GATED ? GEMV_PRE : 1][8];
+  if (active) {
+#pragma unroll
+    for (int r = 0; r < RW; ++r) {
+      const size_t row = (size_t)min(n0 + r, a.N - 1) * K;
+#pragma unroll
+      for (int p = 0; p < GEMV_PRE; ++p) {
+        const int c = p * 256 + lane * 8;
+        if (c < K) {
+          load8(W0 + row + c, pre0[r][p]);
+          if (GATED) load8(W1 + row + c, pre1[r][p]);
+        }
+      }
+    }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  if (!active) return;
+  const float* X = a.X;
+  float acc0[RW], acc1[GATED ? RW : 1], ss = 0.f;
+#pragma unroll
+  for (int r = 0; r < RW; ++r) { acc0[r] = 0.f; if (GATED) acc1[r] = 0.f; }
+
+  auto fma8 = [&](const float (&w)[8], const float (&h)[8]) {
+    return w[0] * h[0] + w[1] * h[1] + w[2] * h[2] + w[3] * h[3] + w[4] * h[4] + w[5] * h[5] + w[6] * h[6] + w[7] * h[7];
+  };
+  auto load_h = [&](int c, float (&h)[8]) {
+    const float4 x0 = *reinterpret_cast<const float4*>(X + c);
+    const float4 x1 = *reinterpret_cast<const float4*>(X + c + 4);
+    h[0] = x0.x; h[1] = x0.y; h[2] = x0.z; h[3] = x0.w; h[4] = x1.x; h[5] = x1.y; h[6] = x1.z; h[7] = x1.w;
+    if (a.gain) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ss += h[i] * h[i];
+      const float4 g0 = *reinterpret_cast<const float4*>(a.gain + c);
+      const float4 g1 = *reinterpret_cast<const float4*>(a.gain + c + 4);
+      h[0] *= g0.x; h[1] *= g0.y; h[2] *= g0.z; h[3] *= g0.w; h[4] *= g1.x; h[5] *= g1.y; h[6] *= g1.z; h[7] *= g1.w;
+    }
+  };
+#pragma unroll
+  for (int p = 0; p < GEMV_PRE; ++p) {
+    const int c = p * 256 + lane * 8;
+    if (c < K) {
+      float h[8];
+      load_h(c, h);
+#pragma unroll
+      for (int r = 0; r < RW; ++r) {
+        acc0[r] += fma8(pre0[r][p], h);
+        if (GATED) acc1[r] += fma8(pre1[r][p], h);
+      }
+    }
+  }
+  for (int c = GEMV_PRE * 256 + lane * 8; c < K; c += 256) {
+    float h[8];
+    load_h(c, h);
+#pragma unroll
+    for (int r = 0; r < RW; ++r) {
+      float w[8];
+      const size_t row = (size_t)min(n0 + r, a.N - 1) * K;
+      load8(W0 + row + c, w);
+      acc0[r] += fma8(w, h);
+      if (GATED) { load8(W1 + row + c, w); acc1[r] += fma8(w, h); }
+    }
+  }
+  float inv = 1.f;
+  if (a.gain) inv = 1.f / sqrtf(warp_sum(ss) / (float)K + a.eps);
+  float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+  for (int r = 0; r < RW; ++r) {
+    const float s0 = warp_sum(acc0[r]) * inv;
+    if (lane == r) v0 = s0;
+    if (GATED) { const float s1 = warp_sum(acc1[r]) * inv; if (lane == r) v1 = s1; }
+  }
+  if (lane >= RW) return;
+  const int n = n0 + lane;
+  if (n >= a.N) return;
+  const int pos0 = a.desc ? a.desc->pos0 : a.pos0_host;
+  switch (a.epi) {
+    case EPI_STORE: a.Y[n] = v0; break;
+    case EPI_RELU: a.Y[n] = fmaxf(v0, 0.f); break;
+    case EPI_GATED: a.Y[n] = gelu_tanh(v0) * v1; break;
+    case EPI_RESID: a.Y[n] += v0; break;
+    default: {
+      const int part = a.first_part + n / a.inner;
+      const int rr = n % a.inner;
+      if (part == 0) {
+        a.q_out[rr] = v0;
+      } else {
+        const int h = rr / a.dkv, c = rr % a.dkv;
+        if (pos0 < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + pos0) * a.dkv + c] = v0;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// Block attention (steps S2, S5, L2, L5 and the encoder's self-attention): one block per
+// (head, key split, block of MB query rows) reads every key and value of its split ONCE
+// and serves all MB rows from it.
+//   scores : one thread per key, the key row in registers, MB dot products
+//   softmax: one warp per row (max, exp, sum) in a fixed order
+//   values : thread (channel c, group g) accumulates keys j = g mod ng for all MB rows
+// Splits write (max, sum, weighted values) per row to scratch; the split that takes the
+// last ticket of its (head, row block) merges them in split order.
+// mode 0 cross (all E keys), 1 decoder self (row i sees keys 0..pos0+i, bias by distance),
+// mode 2 encoder self (all E keys, bias by signed distance).
+// ---------------------------------------------------------------------------------
+struct BAttnArgs {
+  const float* q;
+  int ldq;
+  const float* kc;
+  const float* vc;
+  int cap;
+  float* out;
+  int ldo;
+  const float* bias;
+  int bias_ld, bias_off;
+  int mode, dkv, H;
+  const int* n_keys_dev;
+  int M;                 // rows when desc == nullptr
+  const CallDesc* desc;
+  float* part;           // [row block][H][nsplit][MB][2 + dkv]
+  unsigned* counters;    // [row block][H]
+  int nsplit, smem_keys;
+  int* err;
+};
+
+constexpr int BATT_THREADS = 128;
+
+template <int MB>
+__global__ void __launch_bounds__(BATT_THREADS) battn_kernel(BAttnArgs a) {
+  extern __shared__ float s_dyn[];          // scores / probabilities [MB][smem_keys]
+  __shared__ float s_q[MB][128];
+  __shared__ float s_m[MB], s_l[MB];
+  __shared__ float s_red[BATT_THREADS / 16][MB][16 + 1];   // value partials of the key groups (dkv = 16 chunks)
+  __shared__ int s_last;
+  const int h = blockIdx.x, sp = blockIdx.y, rb = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int dkv = a.dkv;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int M = a.desc ? a.desc->k : a.M;
+  const int m0 = rb * MB;
+  const int mrows = min(MB, M - m0);
+  if (mrows <= 0) return;
+  const int pos0 = a.desc ? a.desc->pos0 : 0;
+  // keys any row of this block may see
+  int n = (a.mode == 1) ? pos0 + m0 + mrows : *a.n_keys_dev;
+  n = min(n, a.cap);
+  const int chunk = (n + a.nsplit - 1) / a.nsplit;
+  const int j0 = sp * chunk, j1 = min(n, j0 + chunk);
+  const int nk = max(0, j1 - j0);
+  if (chunk > a.smem_keys) {
+    if (tid == 0) *a.err = BILD_ERR_CAPACITY;
+    return;
+  }
+  const float* K = a.kc + (size_t)h * a.cap * dkv;
+  const float* V = a.vc + (size_t)h * a.cap * dkv;
+  for (int idx = tid; idx < mrows * dkv; idx += BATT_THREADS) {
+    const int i = idx / dkv, e = idx - i * dkv;
+    s_q[i][e] = a.q[(size_t)(m0 + i) * a.ldq + h * dkv + e];
+  }
+  __syncthreads();
+  const int sk = a.smem_keys;
+  // ---- scores ----
+  for (int jj = tid; jj < nk; jj += BATT_THREADS) {
+    const int j = j0 + jj;
+    float acc[MB];
+#pragma unroll
+    for (int i = 0; i < MB; ++i) acc[i] = 0.f;
+    const float4* kr = reinterpret_cast<const float4*>(K + (size_t)j * dkv);
+    for (int e = 0; e < dkv / 4; ++e) {
+      const float4 kv = kr[e];
+#pragma unroll
+      for (int i = 0; i < MB; ++i) {
+        const float4 qv = *reinterpret_cast<const float4*>(&s_q[i][4 * e]);
+        acc[i] += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < MB; ++i) {
+      if (i < mrows) {
+        float sc = acc[i];
+        const int qi = m0 + i;
+        if (a.mode == 1) sc = (j <= pos0 + qi) ? sc + a.bias[(size_t)h * a.bias_ld + (pos0 + qi - j)] : -INFINITY;
+        else if (a.mode == 2) sc += a.bias[(size_t)h * a.bias_ld + (j - qi + a.bias_off)];
+        s_dyn[i * sk + jj] = sc;
+      }
+    }
+  }
+  __syncthreads();
+  // ---- softmax statistics, one warp per row ----
+  for (int i = warp; i < mrows; i += BATT_THREADS / 32) {
+    float mx = -INFINITY;
+    for (int jj = lane; jj < nk; jj += 32) mx = fmaxf(mx, s_dyn[i * sk + jj]);
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int jj = lane; jj < nk; jj += 32) {
+      const float sc = s_dyn[i * sk + jj];
+      const float p = (sc == -INFINITY) ? 0.f : expf(sc - mx);
+      s_dyn[i * sk + jj] = p;
+      sum += p;
+    }
+    sum = warp_sum(sum);
+    if (lane == 0) { s_m[i] = mx; s_l[i] = sum; }
+  }
+  __syncthreads();
+  // ---- weighted values ----
+  const int ng = BATT_THREADS / dkv;
+  const int c = tid % dkv, g = tid / dkv;
+  float acc[MB];
+#pragma unroll
+  for (int i = 0; i < MB; ++i) acc[i] = 0.f;
+  for (int jj = g; jj < nk; jj += ng) {
+    const float v = V[(size_t)(j0 + jj) * dkv + c];
+#pragma unroll
+    for (int i = 0; i < MB; ++i) acc[i] += s_dyn[i * sk + jj] * v;
+  }
+  // reduce the ng key groups in group order through shared memory (reusing s_dyn is not
+  // possible: other threads may still read it), 16 channels at a time
+  float* P = a.part + ((((size_t)rb * a.H + h) * a.nsplit + sp) * MB) * (dkv + 2);
+  for (int c0 = 0; c0 < dkv; c0 += 16) {
+    __syncthreads();
+    if (c >= c0 && c < c0 + 16)
+#pragma unroll
+      for (int i = 0; i < MB; ++i) s_red[g][i][c - c0] = acc[i];
+    __syncthreads();
+    for (int idx = tid; idx < mrows * 16; idx += BATT_THREADS) {
+      const int i = idx / 16, cc = idx % 16;
+      float t = 0.f;
+      for (int gg = 0; gg < ng; ++gg) t += s_red[gg][i][cc];
+      if (a.nsplit == 1) a.out[(size_t)(m0 + i) * a.ldo + h * dkv + c0 + cc] = t / s_l[i];
+      else P[(size_t)i * (dkv + 2) + 2 + c0 + cc] = t;
+    }
+  }
+  if (a.nsplit == 1) return;
+  if (tid < mrows) { P[(size_t)tid * (dkv + 2)] = s_m[tid]; P[(size_t)tid * (dkv + 2) + 1] = s_l[tid]; }
+  __threadfence();
+  __syncthreads();
+  const int slot = rb * a.H + h;
+  if (tid == 0) {
+    const unsigned t = atomicAdd(&a.counters[slot], 1u);
+    s_last = (t == (unsigned)a.nsplit - 1);
+    if (s_last) a.counters[slot] = 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const float* P0 = a.part + (((size_t)rb * a.H + h) * a.nsplit * MB) * (dkv + 2);
+  for (int idx = tid; idx < mrows * dkv; idx += BATT_THREADS) {
+    const int i = idx / dkv, cc = idx - i * dkv;
+    float gm = -INFINITY;
+    for (int s = 0; s < a.nsplit; ++s) gm = fmaxf(gm, __ldcg(&P0[((size_t)s * MB + i) * (dkv + 2)]));
+    float num = 0.f, den = 0.f;
+    for (int s = 0; s < a.nsplit; ++s) {
+      const float* Ps = P0 + ((size_t)s * MB + i) * (dkv + 2);
+      const float l = __ldcg(&Ps[1]);
+      if (l > 0.f) {
+        const float w = expf(__ldcg(&Ps[0]) - gm);
+        den += l * w;
+        num += __ldcg(&Ps[2 + cc]) * w;
+      }
+    }
+    a.out[(size_t)(m0 + i) * a.ldo + h * dkv + cc] = num / den;
+  }
+}
+
+}  // namespace bild

@@ -14,6 +14,8 @@ __global__ void embed_kernel(const WT* __restrict__ E, const int* __restrict__ t
                              const int* __restrict__ count_dev, int count_host, int d,
                              int vocab, float* __restrict__ x) {
   const int m = blockIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   const int M = count_dev ? *count_dev : count_host;
   if (m >= M) return;
   int t = tokens[m];
@@ -65,6 +67,8 @@ __global__ void __launch_bounds__(LIN_THREADS) linear_kernel(LinArgs a) {
   extern __shared__ float sH[];  // [MB][kc]
   __shared__ float s_scale[MB];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = LIN_THREADS / 32;
+  pdl_launch_dependents();
+  pdl_wait();
   const int M = a.desc ? a.desc->k : a.M;
   const int m0 = blockIdx.y * MB;
   const int mrows = min(MB, M - m0);
@@ -480,6 +484,8 @@ __global__ void __launch_bounds__(HEAD_THREADS) lm_head_kernel(HeadArgs a) {
   __shared__ Partial s_part[HEAD_THREADS / 32][32];
   __shared__ int s_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = HEAD_THREADS / 32;
+  pdl_launch_dependents();
+  pdl_wait();
   const int M = a.desc ? a.desc->k : a.M;
   const int mrows = min(MB, M);
   const int K = a.K, V = a.V;

@@ -1,0 +1,325 @@
+// Block linear layer of the large-model pass on the 5th-generation tensor cores
+// (steps L1, L3, L4, L6, L7, L8): Y^T = W X^T for up to 16 token rows ("swap-AB": the weight's
+// output dimension rides the MMA's M = 128 axis, the tokens its N = 16 axis).
+//   * the bf16 weight tile [128 rows][64 k] arrives by TMA (128-byte swizzle) into a ring of
+//     shared-memory stages, the first stages before the dependency wait of the launch;
+//   * the fp32 activations (times the norm gain) are split into bf16 hi + bf16 lo and both
+//     are multiplied against the same weight tile, so the weights are read once and the
+//     product carries ~16 mantissa bits of the activation;
+//   * accumulators live in tensor memory (one 16-column block per weight matrix);
+//   * K is split over the CTAs of a thread-block cluster; their partial tiles (and partial
+//     sums of squares for the RMS norm) are summed in rank order in the leader's shared
+//     memory, so the result does not depend on timing;
+//   * every wait on an mbarrier is bounded: on expiry an error code is recorded and the
+//     block carries on to its barriers and frees its tensor memory.
+#pragma once
+#include <cuda.h>
+
+#include "kernels.cuh"
+
+namespace bild {
+
+constexpr int UM_THREADS = 128;
+constexpr int UM_TILE_M = 128;   // weight rows per CTA
+constexpr int UM_KB = 64;        // k per stage = one 128-byte swizzle atom of bf16
+constexpr int UM_STAGES = 8;
+constexpr int UM_MAX_KB = 24;    // k blocks per CTA (activation tiles are resident)
+constexpr uint32_t UM_SPIN_LIMIT = 1u << 20;
+
+struct UmmaArgs {
+  LinArgs lin;       // same operands / epilogues as linear_kernel (W pointers unused here)
+  int cs;            // cluster size along K
+  int nkb;           // k blocks (of 64) per CTA
+  int* err;
+};
+
+// ---- raw PTX helpers --------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait; returns false (and the caller records an error) if the phase never completes.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t addr = smem_u32(bar);
+  for (uint32_t it = 0; it < UM_SPIN_LIMIT; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+// K-major operand tile with 128-byte swizzle: rows are 128 bytes, 8-row atoms are 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);   // start address
+  d |= (uint64_t)1 << 16;                    // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset between 8-row atoms
+  d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
+  return d;
+}
+// bf16 x bf16 -> fp32, A and B K-major, M = 128, N = 16
+constexpr uint32_t UM_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(UM_IDESC), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster_f4(uint32_t local_addr, uint32_t rank, float4 v) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_cluster_f1(uint32_t local_addr, uint32_t rank, float v) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
+// Shared-memory plan (bytes) for a launch; the kernel carves the same layout.
+__host__ __device__ inline size_t umma_smem_bytes(bool gated, int nkb, int cs) {
+  const size_t a = (size_t)(gated ? 3 : 6) * (gated ? 2 : 1) * 16384;   // weight stages
+  const size_t b = (size_t)nkb * 4096;                                  // activations hi + lo
+  const size_t red = (size_t)(cs > 1 ? cs - 1 : 0) * UM_TILE_M * 16 * 4 * (gated ? 2 : 1);
+  return 1024 /*alignment slack*/ + a + b + red + 1024 /*ss partials, barriers, tmem slot*/;
+}
+
+template <bool GATED>
+__global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, const __grid_constant__ CUtensorMap tm0,
+                                                                 const __grid_constant__ CUtensorMap tm1) {
+  constexpr int NST = GATED ? 3 : 6;
+  constexpr int NMAT = GATED ? 2 : 1;
+  extern __shared__ unsigned char um_raw[];
+  const LinArgs& a = u.lin;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cs = u.cs, nkb = u.nkb;
+  const uint32_t rank = cs > 1 ? cluster_rank() : 0;
+  const int tile = blockIdx.x / cs;
+  const int n_base = tile * UM_TILE_M;
+  const int k_base = (int)rank * nkb * UM_KB;
+
+  unsigned char* base = (unsigned char*)(((uintptr_t)um_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char* sA = base;                                      // [NST][NMAT][16 KB]
+  unsigned char* sB = sA + (size_t)NST * NMAT * 16384;           // [nkb][hi 2 KB | lo 2 KB]
+  float* sRed = (float*)(sB + (size_t)nkb * 4096);               // [cs-1][NMAT][128][16]
+  float* sSS = sRed + (size_t)(cs > 1 ? cs - 1 : 0) * NMAT * UM_TILE_M * 16;   // [8][16]
+  uint64_t* full = (uint64_t*)(sSS + 8 * 16);
+  uint64_t* empty = full + NST;
+  uint64_t* done = empty + NST;
+  uint32_t* tmem_slot = (uint32_t*)(done + 1);
+
+  if (tid == 0) {
+    for (int i = 0; i < NST; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    mbar_init(done, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 32;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = *tmem_slot;
+  // every block of the cluster must be running before anyone stores into a peer's shared memory
+  if (cs > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+
+  // weights do not depend on the previous kernel: fill the ring before the dependency wait
+  if (tid == 0) {
+    for (int kb = 0; kb < nkb && kb < NST; ++kb) {
+      mbar_expect_tx(&full[kb], NMAT * 16384);
+      tma_load_2d(sA + (size_t)kb * NMAT * 16384, &tm0, k_base + kb * UM_KB, n_base, &full[kb]);
+      if (GATED) tma_load_2d(sA + (size_t)kb * NMAT * 16384 + 16384, &tm1, k_base + kb * UM_KB, n_base, &full[kb]);
+    }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  if (cs > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+
+  // ---- activations: x * gain -> bf16 hi / lo tiles (swizzled), partial sums of squares ----
+  const int M = a.desc ? a.desc->k : a.M;
+  const int mrows = min(MAXB, M);
+  const int kl = nkb * UM_KB;
+  for (int m = warp; m < MAXB; m += UM_THREADS / 32) {
+    float ss = 0.f;
+    for (int c = lane * 8; c < kl; c += 256) {
+      float h[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) h[i] = 0.f;
+      if (m < mrows) {
+        const float* xp = a.X + (size_t)m * a.ldx + k_base + c;
+        const float4 x0 = *reinterpret_cast<const float4*>(xp);
+        const float4 x1 = *reinterpret_cast<const float4*>(xp + 4);
+        h[0] = x0.x; h[1] = x0.y; h[2] = x0.z; h[3] = x0.w; h[4] = x1.x; h[5] = x1.y; h[6] = x1.z; h[7] = x1.w;
+        if (a.gain) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) ss += h[i] * h[i];
+          const float4 g0 = *reinterpret_cast<const float4*>(a.gain + k_base + c);
+          const float4 g1 = *reinterpret_cast<const float4*>(a.gain + k_base + c + 4);
+          h[0] *= g0.x; h[1] *= g0.y; h[2] *= g0.z; h[3] *= g0.w; h[4] *= g1.x; h[5] *= g1.y; h[6] *= g1.z; h[7] *= g1.w;
+        }
+      }
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(h[2 * i]), h1 = __float2bfloat16_rn(h[2 * i + 1]);
+        const __nv_bfloat16 l0 = __float2bfloat16_rn(h[2 * i] - __bfloat162float(h0));
+        const __nv_bfloat16 l1 = __float2bfloat16_rn(h[2 * i + 1] - __bfloat162float(h1));
+        hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+        lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+      }
+      const int kb = c / UM_KB, chunk = (c % UM_KB) / 8;
+      const uint32_t off = (uint32_t)kb * 4096 + (m >> 3) * 1024 + (m & 7) * 128 + ((chunk ^ (m & 7)) << 4);
+      *reinterpret_cast<uint4*>(sB + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(sB + off + 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
+    ss = warp_sum(ss);
+    if (lane == 0) {
+      if (rank == 0) sSS[m] = ss;
+      else st_cluster_f1(smem_u32(&sSS[rank * 16 + m]), 0, ss);
+    }
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+
+  // ---- producer (rest of the ring) and MMA issue ----
+  if (tid == 0) {
+    for (int kb = NST; kb < nkb; ++kb) {
+      const int st = kb % NST;
+      if (!mbar_wait(&empty[st], ((kb / NST) - 1) & 1)) *u.err = BILD_ERR_TIMEOUT;
+      mbar_expect_tx(&full[st], NMAT * 16384);
+      tma_load_2d(sA + (size_t)st * NMAT * 16384, &tm0, k_base + kb * UM_KB, n_base, &full[st]);
+      if (GATED) tma_load_2d(sA + (size_t)st * NMAT * 16384 + 16384, &tm1, k_base + kb * UM_KB, n_base, &full[st]);
+    }
+  } else if (tid == 32) {
+    for (int kb = 0; kb < nkb; ++kb) {
+      const int st = kb % NST;
+      if (!mbar_wait(&full[st], (kb / NST) & 1)) *u.err = BILD_ERR_TIMEOUT;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t a0 = smem_u32(sA + (size_t)st * NMAT * 16384);
+      const uint32_t bh = smem_u32(sB + (size_t)kb * 4096);
+#pragma unroll
+      for (int kk = 0; kk < UM_KB / 16; ++kk) {
+        const uint64_t dbh = umma_desc_sw128(bh + kk * 32), dbl = umma_desc_sw128(bh + 2048 + kk * 32);
+        const uint64_t da0 = umma_desc_sw128(a0 + kk * 32);
+        umma_bf16(tmem, da0, dbh, (kb | kk) ? 1u : 0u);
+        umma_bf16(tmem, da0, dbl, 1u);
+        if (GATED) {
+          const uint64_t da1 = umma_desc_sw128(a0 + 16384 + kk * 32);
+          umma_bf16(tmem + 16, da1, dbh, (kb | kk) ? 1u : 0u);
+          umma_bf16(tmem + 16, da1, dbl, 1u);
+        }
+      }
+      umma_commit(&empty[st]);   // the stage may be refilled once these MMAs have read it
+    }
+    umma_commit(done);
+  }
+  __syncwarp();
+  if (!mbar_wait(done, 0)) *u.err = BILD_ERR_TIMEOUT;
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+  // ---- accumulators: thread t holds weight row n_base + t for the 16 token rows ----
+  float acc0[16], acc1[16];
+  tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16), acc0);
+  if (GATED) tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + 16, acc1);
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+
+  if (cs > 1) {
+    if (rank != 0) {
+      float* dst = sRed + ((size_t)(rank - 1) * NMAT * UM_TILE_M + tid) * 16;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) st_cluster_f4(smem_u32(dst + 4 * i), 0, make_float4(acc0[4 * i], acc0[4 * i + 1], acc0[4 * i + 2], acc0[4 * i + 3]));
+      if (GATED) {
+        float* dst1 = dst + (size_t)UM_TILE_M * 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) st_cluster_f4(smem_u32(dst1 + 4 * i), 0, make_float4(acc1[4 * i], acc1[4 * i + 1], acc1[4 * i + 2], acc1[4 * i + 3]));
+      }
+    }
+    cluster_sync_all();
+  }
+  if (rank == 0) {
+    for (int r = 1; r < cs; ++r) {   // fixed order: rank 1, 2, ...
+      const float* src = sRed + ((size_t)(r - 1) * NMAT * UM_TILE_M + tid) * 16;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) acc0[i] += src[i];
+      if (GATED) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc1[i] += src[(size_t)UM_TILE_M * 16 + i];
+      }
+    }
+    const int n = n_base + tid;
+    const int pos0 = a.desc ? a.desc->pos0 : a.pos0_host;
+    if (n < a.N) {
+#pragma unroll
+      for (int m = 0; m < MAXB; ++m) {
+        if (m < mrows) {
+          float inv = 1.f;
+          if (a.gain) {
+            float ss = 0.f;
+            for (int r = 0; r < cs; ++r) ss += sSS[r * 16 + m];
+            inv = 1.f / sqrtf(ss / (float)a.K + a.eps);
+          }
+          const float v0 = acc0[m] * inv;
+          switch (a.epi) {
+            case EPI_STORE: a.Y[(size_t)m * a.ldy + n] = v0; break;
+            case EPI_RELU: a.Y[(size_t)m * a.ldy + n] = fmaxf(v0, 0.f); break;
+            case EPI_GATED: a.Y[(size_t)m * a.ldy + n] = gelu_tanh(v0) * (GATED ? acc1[m] * inv : 0.f); break;
+            case EPI_RESID: a.Y[(size_t)m * a.ldy + n] += v0; break;
+            default: {
+              const int part = a.first_part + n / a.inner;
+              const int rr = n % a.inner;
+              if (part == 0) {
+                a.q_out[(size_t)m * a.ldq + rr] = v0;
+              } else {
+                const int h = rr / a.dkv, c = rr % a.dkv;
+                const int row = pos0 + m;
+                if (row < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + row) * a.dkv + c] = v0;
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 32;" ::"r"(tmem) : "memory");
+}
+
+}  // namespace bild

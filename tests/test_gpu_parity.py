@@ -145,6 +145,8 @@ def test_steps_match_oracle_logits(torch_cuda, name):
     S, L, _ = get_oracle(name)
     tol = TOL[wl.dtype]
     V = S.s.vocab
+    # the block pass of a bf16 pair with 64-multiple widths must run on the tensor-core kernel
+    assert ctx.uses_tensor_cores() == (name == "tiny_bf16")
     ctx.reset()
     stS, stL = S.start(ids, 64), L.start(ids, 64)
     buf = torch.empty((16, V), dtype=torch.float32, device="cuda")
@@ -249,6 +251,7 @@ def test_full_size_replay_and_generate(torch_cuda, name):
     torch = torch_cuda
     from paper_2302_07863_b200 import MODE_BILD, MODE_LARGE_ONLY, MODE_SMALL_ONLY
     ctx, ids, wl, g = get_ctx(name)
+    assert ctx.uses_tensor_cores()
     tol = TOL[wl.dtype]
     V = MODEL_SHAPES[wl.small].vocab
     th = g["thresholds"]
