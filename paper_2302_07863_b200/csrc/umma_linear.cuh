@@ -115,7 +115,7 @@ __device__ __forceinline__ void st_cluster_f1(uint32_t local_addr, uint32_t rank
 
 // Shared-memory plan (bytes) for a launch; the kernel carves the same layout.
 __host__ __device__ inline size_t umma_smem_bytes(bool gated, int nkb, int cs) {
-  const size_t a = (size_t)(gated ? 3 : 6) * (gated ? 2 : 1) * 16384;   // weight stages
+  const size_t a = (size_t)(gated ? 4 : 8) * (gated ? 2 : 1) * 16384;   // weight stages
   const size_t b = (size_t)nkb * 4096;                                  // activations hi + lo
   const size_t red = (size_t)(cs > 1 ? cs - 1 : 0) * UM_TILE_M * 16 * 4 * (gated ? 2 : 1);
   return 1024 /*alignment slack*/ + a + b + red + 1024 /*ss partials, barriers, tmem slot*/;
@@ -124,7 +124,7 @@ __host__ __device__ inline size_t umma_smem_bytes(bool gated, int nkb, int cs) {
 template <bool GATED>
 __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, const __grid_constant__ CUtensorMap tm0,
                                                                  const __grid_constant__ CUtensorMap tm1) {
-  constexpr int NST = GATED ? 3 : 6;
+  constexpr int NST = GATED ? 4 : 8;
   constexpr int NMAT = GATED ? 2 : 1;
   extern __shared__ unsigned char um_raw[];
   const LinArgs& a = u.lin;
@@ -177,43 +177,58 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
   const int M = a.desc ? a.desc->k : a.M;
   const int mrows = min(MAXB, M);
   const int kl = nkb * UM_KB;
-  for (int m = warp; m < MAXB; m += UM_THREADS / 32) {
-    float ss = 0.f;
+  {  // warp w owns rows w, w+4, w+8, w+12; the loads of all four rows are issued together
+    float ssr[4] = {0.f, 0.f, 0.f, 0.f};
     for (int c = lane * 8; c < kl; c += 256) {
-      float h[8];
+      float4 g0 = make_float4(1.f, 1.f, 1.f, 1.f), g1 = g0;
+      if (a.gain) {
+        g0 = *reinterpret_cast<const float4*>(a.gain + k_base + c);
+        g1 = *reinterpret_cast<const float4*>(a.gain + k_base + c + 4);
+      }
+      float4 xa[4], xb[4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) h[i] = 0.f;
-      if (m < mrows) {
-        const float* xp = a.X + (size_t)m * a.ldx + k_base + c;
-        const float4 x0 = *reinterpret_cast<const float4*>(xp);
-        const float4 x1 = *reinterpret_cast<const float4*>(xp + 4);
-        h[0] = x0.x; h[1] = x0.y; h[2] = x0.z; h[3] = x0.w; h[4] = x1.x; h[5] = x1.y; h[6] = x1.z; h[7] = x1.w;
-        if (a.gain) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) ss += h[i] * h[i];
-          const float4 g0 = *reinterpret_cast<const float4*>(a.gain + k_base + c);
-          const float4 g1 = *reinterpret_cast<const float4*>(a.gain + k_base + c + 4);
-          h[0] *= g0.x; h[1] *= g0.y; h[2] *= g0.z; h[3] *= g0.w; h[4] *= g1.x; h[5] *= g1.y; h[6] *= g1.z; h[7] *= g1.w;
+      for (int r = 0; r < 4; ++r) {
+        const int m = warp + 4 * r;
+        xa[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        xb[r] = xa[r];
+        if (m < mrows) {
+          const float* xp = a.X + (size_t)m * a.ldx + k_base + c;
+          xa[r] = *reinterpret_cast<const float4*>(xp);
+          xb[r] = *reinterpret_cast<const float4*>(xp + 4);
         }
       }
-      uint32_t hi[4], lo[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const __nv_bfloat16 h0 = __float2bfloat16_rn(h[2 * i]), h1 = __float2bfloat16_rn(h[2 * i + 1]);
-        const __nv_bfloat16 l0 = __float2bfloat16_rn(h[2 * i] - __bfloat162float(h0));
-        const __nv_bfloat16 l1 = __float2bfloat16_rn(h[2 * i + 1] - __bfloat162float(h1));
-        hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-        lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-      }
       const int kb = c / UM_KB, chunk = (c % UM_KB) / 8;
-      const uint32_t off = (uint32_t)kb * 4096 + (m >> 3) * 1024 + (m & 7) * 128 + ((chunk ^ (m & 7)) << 4);
-      *reinterpret_cast<uint4*>(sB + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-      *reinterpret_cast<uint4*>(sB + off + 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int m = warp + 4 * r;
+        float h[8] = {xa[r].x, xa[r].y, xa[r].z, xa[r].w, xb[r].x, xb[r].y, xb[r].z, xb[r].w};
+        if (a.gain) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) ssr[r] += h[i] * h[i];
+          h[0] *= g0.x; h[1] *= g0.y; h[2] *= g0.z; h[3] *= g0.w; h[4] *= g1.x; h[5] *= g1.y; h[6] *= g1.z; h[7] *= g1.w;
+        }
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(h[2 * i]), h1 = __float2bfloat16_rn(h[2 * i + 1]);
+          const __nv_bfloat16 l0 = __float2bfloat16_rn(h[2 * i] - __bfloat162float(h0));
+          const __nv_bfloat16 l1 = __float2bfloat16_rn(h[2 * i + 1] - __bfloat162float(h1));
+          hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+          lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+        }
+        const uint32_t off = (uint32_t)kb * 4096 + (m >> 3) * 1024 + (m & 7) * 128 + ((chunk ^ (m & 7)) << 4);
+        *reinterpret_cast<uint4*>(sB + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(sB + off + 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      }
     }
-    ss = warp_sum(ss);
-    if (lane == 0) {
-      if (rank == 0) sSS[m] = ss;
-      else st_cluster_f1(smem_u32(&sSS[rank * 16 + m]), 0, ss);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int m = warp + 4 * r;
+      const float ss = warp_sum(ssr[r]);
+      if (lane == 0) {
+        if (rank == 0) sSS[m] = ss;
+        else st_cluster_f1(smem_u32(&sSS[rank * 16 + m]), 0, ss);
+      }
     }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -263,56 +278,68 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
 
   if (cs > 1) {
     if (rank != 0) {
-      float* dst = sRed + ((size_t)(rank - 1) * NMAT * UM_TILE_M + tid) * 16;
+      // layout [rank-1][matrix][token i][row tid]: consecutive threads, consecutive words
+      float* dst = sRed + (size_t)(rank - 1) * NMAT * UM_TILE_M * 16 + tid;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) st_cluster_f4(smem_u32(dst + 4 * i), 0, make_float4(acc0[4 * i], acc0[4 * i + 1], acc0[4 * i + 2], acc0[4 * i + 3]));
+      for (int i = 0; i < 16; ++i) st_cluster_f1(smem_u32(dst + i * UM_TILE_M), 0, acc0[i]);
       if (GATED) {
-        float* dst1 = dst + (size_t)UM_TILE_M * 16;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) st_cluster_f4(smem_u32(dst1 + 4 * i), 0, make_float4(acc1[4 * i], acc1[4 * i + 1], acc1[4 * i + 2], acc1[4 * i + 3]));
+        for (int i = 0; i < 16; ++i) st_cluster_f1(smem_u32(dst + (16 + i) * UM_TILE_M), 0, acc1[i]);
       }
     }
     cluster_sync_all();
   }
   if (rank == 0) {
     for (int r = 1; r < cs; ++r) {   // fixed order: rank 1, 2, ...
-      const float* src = sRed + ((size_t)(r - 1) * NMAT * UM_TILE_M + tid) * 16;
+      const float* src = sRed + (size_t)(r - 1) * NMAT * UM_TILE_M * 16 + tid;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) acc0[i] += src[i];
+      for (int i = 0; i < 16; ++i) acc0[i] += src[i * UM_TILE_M];
       if (GATED) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) acc1[i] += src[(size_t)UM_TILE_M * 16 + i];
+        for (int i = 0; i < 16; ++i) acc1[i] += src[(16 + i) * UM_TILE_M];
       }
     }
     const int n = n_base + tid;
     const int pos0 = a.desc ? a.desc->pos0 : a.pos0_host;
     if (n < a.N) {
+      float v0[MAXB], v1[MAXB];
 #pragma unroll
       for (int m = 0; m < MAXB; ++m) {
-        if (m < mrows) {
-          float inv = 1.f;
-          if (a.gain) {
-            float ss = 0.f;
-            for (int r = 0; r < cs; ++r) ss += sSS[r * 16 + m];
-            inv = 1.f / sqrtf(ss / (float)a.K + a.eps);
+        float inv = 1.f;
+        if (a.gain && m < mrows) {
+          float ss = 0.f;
+          for (int r = 0; r < cs; ++r) ss += sSS[r * 16 + m];
+          inv = 1.f / sqrtf(ss / (float)a.K + a.eps);
+        }
+        v0[m] = acc0[m] * inv;
+        v1[m] = GATED ? acc1[m] * inv : 0.f;
+      }
+      if (a.epi == EPI_RESID) {   // all reads of the residual stream first, then the writes
+        float old[MAXB];
+#pragma unroll
+        for (int m = 0; m < MAXB; ++m) old[m] = m < mrows ? a.Y[(size_t)m * a.ldy + n] : 0.f;
+#pragma unroll
+        for (int m = 0; m < MAXB; ++m)
+          if (m < mrows) a.Y[(size_t)m * a.ldy + n] = old[m] + v0[m];
+      } else if (a.epi == EPI_HEADS) {
+        const int part = a.first_part + n / a.inner;
+        const int rr = n % a.inner;
+        const int h = rr / a.dkv, c = rr % a.dkv;
+#pragma unroll
+        for (int m = 0; m < MAXB; ++m) {
+          if (m < mrows) {
+            if (part == 0) a.q_out[(size_t)m * a.ldq + rr] = v0[m];
+            else if (pos0 + m < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + pos0 + m) * a.dkv + c] = v0[m];
           }
-          const float v0 = acc0[m] * inv;
-          switch (a.epi) {
-            case EPI_STORE: a.Y[(size_t)m * a.ldy + n] = v0; break;
-            case EPI_RELU: a.Y[(size_t)m * a.ldy + n] = fmaxf(v0, 0.f); break;
-            case EPI_GATED: a.Y[(size_t)m * a.ldy + n] = gelu_tanh(v0) * (GATED ? acc1[m] * inv : 0.f); break;
-            case EPI_RESID: a.Y[(size_t)m * a.ldy + n] += v0; break;
-            default: {
-              const int part = a.first_part + n / a.inner;
-              const int rr = n % a.inner;
-              if (part == 0) {
-                a.q_out[(size_t)m * a.ldq + rr] = v0;
-              } else {
-                const int h = rr / a.dkv, c = rr % a.dkv;
-                const int row = pos0 + m;
-                if (row < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + row) * a.dkv + c] = v0;
-              }
-            }
+        }
+      } else {
+#pragma unroll
+        for (int m = 0; m < MAXB; ++m) {
+          if (m < mrows) {
+            float y = v0[m];
+            if (a.epi == EPI_RELU) y = fmaxf(y, 0.f);
+            else if (a.epi == EPI_GATED) y = gelu_tanh(y) * v1[m];
+            a.Y[(size_t)m * a.ldy + n] = y;
           }
         }
       }
