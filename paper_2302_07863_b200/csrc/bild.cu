@@ -243,9 +243,12 @@ cudaError_t launch_k(bild_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block,
 }
 
 template <typename WT, int RW>
-cudaError_t launch_gemv_t(bild_ctx* c, const LinArgs& a) {
-  const int nwarps = GEMV_THREADS / 32;
-  dim3 grid((a.N + nwarps * RW - 1) / (nwarps * RW));
+cudaError_t launch_gemv_t(bild_ctx* c, const LinArgs& a0) {
+  LinArgs a = a0;
+  // enough warps along K that every warp's slice (<= 1024 columns) is requested in one batch
+  a.ksplit = (a.K % 32 == 0 && a.K > 2048) ? 4 : (a.K % 16 == 0 && a.K > 1024) ? 2 : 1;
+  const int groups = (GEMV_THREADS / 32) / a.ksplit;
+  dim3 grid((a.N + groups * RW - 1) / (groups * RW));
   if (a.epi == EPI_GATED) return launch_k(c, gemv_kernel<WT, RW, true>, grid, dim3(GEMV_THREADS), 0, a);
   return launch_k(c, gemv_kernel<WT, RW, false>, grid, dim3(GEMV_THREADS), 0, a);
 }

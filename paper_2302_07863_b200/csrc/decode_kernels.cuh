@@ -17,11 +17,18 @@ namespace bild {
 constexpr int GEMV_THREADS = 128;
 constexpr int GEMV_PRE = 4;  // column chunks (of 256) whose weights are fetched ahead
 
+// a.ksplit (1, 2 or 4) warps share one group of RW rows, each taking a contiguous K / ksplit
+// columns, so that for K up to 4096 every weight byte of the block is requested in one batch
+// before the dependency wait; their partial sums are added in warp order through shared memory.
 template <typename WT, int RW, bool GATED>
 __global__ void __launch_bounds__(GEMV_THREADS) gemv_kernel(LinArgs a) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = GEMV_THREADS / 32;
-  const int n0 = (blockIdx.x * nwarps + warp) * RW;
-  const int K = a.K;
+  constexpr int NW = GEMV_THREADS / 32;
+  __shared__ float s_part[NW][2 * RW + 1];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int ks = a.ksplit > 1 ? a.ksplit : 1;
+  const int group = warp / ks, kw = warp - group * ks;
+  const int n0 = (blockIdx.x * (NW / ks) + group) * RW;
+  const int K = a.K, kl = K / ks, kbeg = kw * kl;
   const WT* W0 = (const WT*)a.W0;
   const WT* W1 = (const WT*)a.W1;
   const bool active = n0 < a.N;
@@ -29,11 +36,11 @@ __global__ void __launch_bounds__(GEMV_THREADS) gemv_kernel(LinArgs a) {
   if (active) {
 #pragma unroll
     for (int r = 0; r < RW; ++r) {
-      const size_t row = (size_t)min(n0 + r, a.N - 1) * K;
+      const size_t row = (size_t)min(n0 + r, a.N - 1) * K + kbeg;
 #pragma unroll
       for (int p = 0; p < GEMV_PRE; ++p) {
         const int c = p * 256 + lane * 8;
-        if (c < K) {
+        if (c < kl) {
           load8(W0 + row + c, pre0[r][p]);
           if (GATED) load8(W1 + row + c, pre1[r][p]);
         }
@@ -42,8 +49,8 @@ __global__ void __launch_bounds__(GEMV_THREADS) gemv_kernel(LinArgs a) {
   }
   pdl_launch_dependents();
   pdl_wait();
-  if (!active) return;
-  const float* X = a.X;
+  const float* X = a.X + kbeg;
+  const float* G = a.gain ? a.gain + kbeg : nullptr;
   float acc0[RW], acc1[GATED ? RW : 1], ss = 0.f;
 #pragma unroll
   for (int r = 0; r < RW; ++r) { acc0[r] = 0.f; if (GATED) acc1[r] = 0.f; }
@@ -55,47 +62,78 @@ __global__ void __launch_bounds__(GEMV_THREADS) gemv_kernel(LinArgs a) {
     const float4 x0 = *reinterpret_cast<const float4*>(X + c);
     const float4 x1 = *reinterpret_cast<const float4*>(X + c + 4);
     h[0] = x0.x; h[1] = x0.y; h[2] = x0.z; h[3] = x0.w; h[4] = x1.x; h[5] = x1.y; h[6] = x1.z; h[7] = x1.w;
-    if (a.gain) {
+    if (G) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) ss += h[i] * h[i];
-      const float4 g0 = *reinterpret_cast<const float4*>(a.gain + c);
-      const float4 g1 = *reinterpret_cast<const float4*>(a.gain + c + 4);
+      const float4 g0 = *reinterpret_cast<const float4*>(G + c);
+      const float4 g1 = *reinterpret_cast<const float4*>(G + c + 4);
       h[0] *= g0.x; h[1] *= g0.y; h[2] *= g0.z; h[3] *= g0.w; h[4] *= g1.x; h[5] *= g1.y; h[6] *= g1.z; h[7] *= g1.w;
     }
   };
+  if (active) {
+    float hp[GEMV_PRE][8];
 #pragma unroll
-  for (int p = 0; p < GEMV_PRE; ++p) {
-    const int c = p * 256 + lane * 8;
-    if (c < K) {
+    for (int p = 0; p < GEMV_PRE; ++p) {
+      const int c = p * 256 + lane * 8;
+      if (c < kl) load_h(c, hp[p]);
+    }
+#pragma unroll
+    for (int p = 0; p < GEMV_PRE; ++p) {
+      const int c = p * 256 + lane * 8;
+      if (c < kl) {
+#pragma unroll
+        for (int r = 0; r < RW; ++r) {
+          acc0[r] += fma8(pre0[r][p], hp[p]);
+          if (GATED) acc1[r] += fma8(pre1[r][p], hp[p]);
+        }
+      }
+    }
+    for (int c = GEMV_PRE * 256 + lane * 8; c < kl; c += 256) {   // only for K / ksplit > 1024
       float h[8];
       load_h(c, h);
 #pragma unroll
       for (int r = 0; r < RW; ++r) {
-        acc0[r] += fma8(pre0[r][p], h);
-        if (GATED) acc1[r] += fma8(pre1[r][p], h);
+        float w[8];
+        const size_t row = (size_t)min(n0 + r, a.N - 1) * K + kbeg;
+        load8(W0 + row + c, w);
+        acc0[r] += fma8(w, h);
+        if (GATED) { load8(W1 + row + c, w); acc1[r] += fma8(w, h); }
       }
     }
   }
-  for (int c = GEMV_PRE * 256 + lane * 8; c < K; c += 256) {
-    float h[8];
-    load_h(c, h);
 #pragma unroll
-    for (int r = 0; r < RW; ++r) {
-      float w[8];
-      const size_t row = (size_t)min(n0 + r, a.N - 1) * K;
-      load8(W0 + row + c, w);
-      acc0[r] += fma8(w, h);
-      if (GATED) { load8(W1 + row + c, w); acc1[r] += fma8(w, h); }
+  for (int r = 0; r < RW; ++r) {
+    acc0[r] = warp_sum(acc0[r]);
+    if (GATED) acc1[r] = warp_sum(acc1[r]);
+  }
+  ss = warp_sum(ss);
+  if (ks > 1) {
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < RW; ++r) { s_part[warp][r] = acc0[r]; s_part[warp][RW + r] = GATED ? acc1[r] : 0.f; }
+      s_part[warp][2 * RW] = ss;
+    }
+    __syncthreads();
+    if (kw != 0) return;
+    ss = 0.f;
+#pragma unroll
+    for (int r = 0; r < RW; ++r) { acc0[r] = 0.f; if (GATED) acc1[r] = 0.f; }
+    for (int w2 = 0; w2 < ks; ++w2) {   // fixed order
+#pragma unroll
+      for (int r = 0; r < RW; ++r) {
+        acc0[r] += s_part[group * ks + w2][r];
+        if (GATED) acc1[r] += s_part[group * ks + w2][RW + r];
+      }
+      ss += s_part[group * ks + w2][2 * RW];
     }
   }
+  if (!active) return;
   float inv = 1.f;
-  if (a.gain) inv = 1.f / sqrtf(warp_sum(ss) / (float)K + a.eps);
+  if (a.gain) inv = 1.f / sqrtf(ss / (float)K + a.eps);
   float v0 = 0.f, v1 = 0.f;
 #pragma unroll
   for (int r = 0; r < RW; ++r) {
-    const float s0 = warp_sum(acc0[r]) * inv;
-    if (lane == r) v0 = s0;
-    if (GATED) { const float s1 = warp_sum(acc1[r]) * inv; if (lane == r) v1 = s1; }
+    if (lane == r) { v0 = acc0[r] * inv; if (GATED) v1 = acc1[r] * inv; }
   }
   if (lane >= RW) return;
   const int n = n0 + lane;
@@ -195,12 +233,20 @@ __global__ void __launch_bounds__(BATT_THREADS) battn_kernel(BAttnArgs a) {
 #pragma unroll
     for (int i = 0; i < MB; ++i) acc[i] = 0.f;
     const float4* kr = reinterpret_cast<const float4*>(K + (size_t)j * dkv);
-    for (int e = 0; e < dkv / 4; ++e) {
-      const float4 kv = kr[e];
+    const int nq4 = dkv / 4;
+    for (int e0 = 0; e0 < nq4; e0 += 8) {   // eight independent 16-byte loads in flight
+      float4 kv[8];
 #pragma unroll
-      for (int i = 0; i < MB; ++i) {
-        const float4 qv = *reinterpret_cast<const float4*>(&s_q[i][4 * e]);
-        acc[i] += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
+      for (int u2 = 0; u2 < 8; ++u2) kv[u2] = (e0 + u2 < nq4) ? kr[e0 + u2] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u2 = 0; u2 < 8; ++u2) {
+        if (e0 + u2 < nq4) {
+#pragma unroll
+          for (int i = 0; i < MB; ++i) {
+            const float4 qv = *reinterpret_cast<const float4*>(&s_q[i][4 * (e0 + u2)]);
+            acc[i] += kv[u2].x * qv.x + kv[u2].y * qv.y + kv[u2].z * qv.z + kv[u2].w * qv.w;
+          }
+        }
       }
     }
 #pragma unroll
@@ -237,10 +283,17 @@ __global__ void __launch_bounds__(BATT_THREADS) battn_kernel(BAttnArgs a) {
   float acc[MB];
 #pragma unroll
   for (int i = 0; i < MB; ++i) acc[i] = 0.f;
-  for (int jj = g; jj < nk; jj += ng) {
-    const float v = V[(size_t)(j0 + jj) * dkv + c];
+  for (int jj = g; jj < nk; jj += 4 * ng) {   // four values in flight per thread
+    float v[4];
 #pragma unroll
-    for (int i = 0; i < MB; ++i) acc[i] += s_dyn[i * sk + jj] * v;
+    for (int u2 = 0; u2 < 4; ++u2) v[u2] = (jj + u2 * ng < nk) ? V[(size_t)(j0 + jj + u2 * ng) * dkv + c] : 0.f;
+#pragma unroll
+    for (int u2 = 0; u2 < 4; ++u2) {
+      if (jj + u2 * ng < nk) {
+#pragma unroll
+        for (int i = 0; i < MB; ++i) acc[i] += s_dyn[i * sk + jj + u2 * ng] * v[u2];
+      }
+    }
   }
   // reduce the ng key groups in group order through shared memory (reusing s_dyn is not
   // possible: other threads may still read it), 16 channels at a time

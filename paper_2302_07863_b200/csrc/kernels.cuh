@@ -57,6 +57,7 @@ struct LinArgs {
   float* vc;
   int cap;
   int pos0_host;
+  int ksplit;             // gemv_kernel only: warps sharing one row group along K (0 or 1 = none)
 };
 
 constexpr int LIN_THREADS = 256;
