@@ -253,18 +253,22 @@ cudaError_t launch_gemv_t(bild_ctx* c, const LinArgs& a0) {
   return launch_k(c, gemv_kernel<WT, RW, false>, grid, dim3(GEMV_THREADS), 0, a);
 }
 
-template <int MB>
+template <int MB, bool STAGE>
 cudaError_t launch_battn_t(bild_ctx* c, BAttnArgs a, int row_blocks, int keys_cap) {
-  a.smem_keys = (keys_cap + a.nsplit - 1) / a.nsplit;
-  const size_t smem = (size_t)MB * a.smem_keys * sizeof(float);
-  if (smem > 16 * 1024) {  // static shared memory of the kernel takes about 17 KB of the default 48 KB
-    cudaError_t e = cudaFuncSetAttribute(battn_kernel<MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  a.smem_keys = ((keys_cap + a.nsplit - 1) / a.nsplit + 3) / 4 * 4;
+  size_t smem = (size_t)MB * a.smem_keys * sizeof(float);
+  if (STAGE) smem += (size_t)a.smem_keys * (2 * a.dkv + 4) * sizeof(float);
+  if (smem > 16 * 1024) {  // the kernel's static shared memory takes about 17 KB of the default 48 KB
+    cudaError_t e = cudaFuncSetAttribute(battn_kernel<MB, STAGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  return launch_k(c, battn_kernel<MB>, dim3(a.H, a.nsplit, row_blocks), dim3(BATT_THREADS), smem, a);
+  return launch_k(c, battn_kernel<MB, STAGE>, dim3(a.H, a.nsplit, row_blocks), dim3(BATT_THREADS), smem, a);
 }
+// Decoder attention stages its keys / values in shared memory (at most 128 keys per split);
+// the encoder's self-attention (mode 2, all keys in one block) reads them from global memory.
 cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a, int row_blocks, int keys_cap) {
-  return MB == 1 ? launch_battn_t<1>(c, a, row_blocks, keys_cap) : launch_battn_t<MAXB>(c, a, row_blocks, keys_cap);
+  if (a.mode == 2) return launch_battn_t<MAXB, false>(c, a, row_blocks, keys_cap);
+  return MB == 1 ? launch_battn_t<1, true>(c, a, row_blocks, keys_cap) : launch_battn_t<MAXB, true>(c, a, row_blocks, keys_cap);
 }
 
 template <typename WT, int MB, int RW>
@@ -315,7 +319,7 @@ int pick_nsplit(int ctas_without_split, int keys_cap) {
   int ns = (148 + ctas_without_split - 1) / ctas_without_split;
   ns = std::min(ns, std::max(1, keys_cap / 32));
   ns = std::max(1, std::min(ns, NSPLIT_MAX));
-  while ((keys_cap + ns - 1) / ns > 1024 && ns < NSPLIT_MAX) ++ns;   // scores of MAXB rows stay under 64 KB
+  while ((keys_cap + ns - 1) / ns > 128 && ns < NSPLIT_MAX) ++ns;   // staged keys / values stay under 72 KB
   return ns;
 }
 
@@ -455,7 +459,9 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
   const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len, dt = c->cfg.dtype;
   CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x));
-  const int ns_self = pick_nsplit(H, cap), ns_cross = pick_nsplit(H, ecap);
+  // self-attention: one block per head up to 128 cached rows (no merge step); cross-attention:
+  // enough splits of the encoder keys to occupy the SMs
+  const int ns_self = std::max(1, (cap + 127) / 128), ns_cross = pick_nsplit(H, ecap);
   for (int l = 0; l < mc.n_layers; ++l) {
     const bild_dec_layer& w = m.dec[l];
     const size_t kvoff = (size_t)l * H * dkv;

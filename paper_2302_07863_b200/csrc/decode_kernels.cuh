@@ -191,9 +191,16 @@ struct BAttnArgs {
 
 constexpr int BATT_THREADS = 128;
 
-template <int MB>
+// STAGE: the block's keys and values are first copied to shared memory with cp.async (for
+// cross-attention before the dependency wait, since the encoder K/V never change during
+// decoding), and scores and weighted values are then computed from shared memory.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+
+template <int MB, bool STAGE>
 __global__ void __launch_bounds__(BATT_THREADS) battn_kernel(BAttnArgs a) {
-  extern __shared__ float s_dyn[];          // scores / probabilities [MB][smem_keys]
+  extern __shared__ float s_dyn[];          // scores [MB][sk] | keys [sk][dkv + 4] | values [sk][dkv]
   __shared__ float s_q[MB][128];
   __shared__ float s_m[MB], s_l[MB];
   __shared__ float s_red[BATT_THREADS / 16][MB][16 + 1];   // value partials of the key groups (dkv = 16 chunks)
@@ -201,6 +208,25 @@ __global__ void __launch_bounds__(BATT_THREADS) battn_kernel(BAttnArgs a) {
   const int h = blockIdx.x, sp = blockIdx.y, rb = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int dkv = a.dkv;
+  const int sk = a.smem_keys;
+  float* sK = s_dyn + MB * sk;
+  float* sV = sK + sk * (dkv + 4);
+  auto stage_kv = [&](int first, int count) {
+    const float* Kg = a.kc + ((size_t)h * a.cap + first) * dkv;
+    const float* Vg = a.vc + ((size_t)h * a.cap + first) * dkv;
+    const int q4 = dkv / 4;
+    for (int idx = tid; idx < count * q4; idx += BATT_THREADS) {
+      const int jj = idx / q4, e = idx - jj * q4;
+      cp_async16(sK + jj * (dkv + 4) + 4 * e, Kg + (size_t)jj * dkv + 4 * e);
+      cp_async16(sV + jj * dkv + 4 * e, Vg + (size_t)jj * dkv + 4 * e);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  if (STAGE && a.mode == 0) {   // static data: fetch before waiting for the previous kernel
+    const int n_all = min(*a.n_keys_dev, a.cap);
+    const int ch = (n_all + a.nsplit - 1) / a.nsplit;
+    if (ch <= sk) stage_kv(sp * ch, max(0, min(n_all, sp * ch + ch) - sp * ch));
+  }
   pdl_launch_dependents();
   pdl_wait();
   const int M = a.desc ? a.desc->k : a.M;
@@ -220,19 +246,21 @@ __global__ void __launch_bounds__(BATT_THREADS) battn_kernel(BAttnArgs a) {
   }
   const float* K = a.kc + (size_t)h * a.cap * dkv;
   const float* V = a.vc + (size_t)h * a.cap * dkv;
+  if (STAGE && a.mode != 0) stage_kv(j0, nk);
   for (int idx = tid; idx < mrows * dkv; idx += BATT_THREADS) {
     const int i = idx / dkv, e = idx - i * dkv;
     s_q[i][e] = a.q[(size_t)(m0 + i) * a.ldq + h * dkv + e];
   }
+  if (STAGE) asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
-  const int sk = a.smem_keys;
   // ---- scores ----
   for (int jj = tid; jj < nk; jj += BATT_THREADS) {
     const int j = j0 + jj;
     float acc[MB];
 #pragma unroll
     for (int i = 0; i < MB; ++i) acc[i] = 0.f;
-    const float4* kr = reinterpret_cast<const float4*>(K + (size_t)j * dkv);
+    const float4* kr = STAGE ? reinterpret_cast<const float4*>(sK + jj * (dkv + 4))
+                             : reinterpret_cast<const float4*>(K + (size_t)j * dkv);
     const int nq4 = dkv / 4;
     for (int e0 = 0; e0 < nq4; e0 += 8) {   // eight independent 16-byte loads in flight
       float4 kv[8];
@@ -286,7 +314,8 @@ __global__ void __launch_bounds__(BATT_THREADS) battn_kernel(BAttnArgs a) {
   for (int jj = g; jj < nk; jj += 4 * ng) {   // four values in flight per thread
     float v[4];
 #pragma unroll
-    for (int u2 = 0; u2 < 4; ++u2) v[u2] = (jj + u2 * ng < nk) ? V[(size_t)(j0 + jj + u2 * ng) * dkv + c] : 0.f;
+    for (int u2 = 0; u2 < 4; ++u2)
+      v[u2] = (jj + u2 * ng < nk) ? (STAGE ? sV[(jj + u2 * ng) * dkv + c] : V[(size_t)(j0 + jj + u2 * ng) * dkv + c]) : 0.f;
 #pragma unroll
     for (int u2 = 0; u2 < 4; ++u2) {
       if (jj + u2 * ng < nk) {

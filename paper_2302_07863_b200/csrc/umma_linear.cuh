@@ -71,8 +71,8 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
   return d;
 }
-// bf16 x bf16 -> fp32, A and B K-major, M = 128, N = 16
-constexpr uint32_t UM_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+// bf16 x bf16 -> fp32, A and B K-major, M = 128, N = 32 (16 token rows of hi, then 16 of lo)
+constexpr uint32_t UM_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
 
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
   asm volatile(
@@ -126,6 +126,7 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
                                                                  const __grid_constant__ CUtensorMap tm1) {
   constexpr int NST = GATED ? 4 : 8;
   constexpr int NMAT = GATED ? 2 : 1;
+  constexpr int TCOLS = 32 * NMAT;   // accumulator columns in tensor memory: [hi 16 | lo 16] per matrix
   extern __shared__ unsigned char um_raw[];
   const LinArgs& a = u.lin;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -151,7 +152,7 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 32;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TCOLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -173,9 +174,17 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
   pdl_wait();
   if (cs > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 
-  // ---- activations: x * gain -> bf16 hi / lo tiles (swizzled), partial sums of squares ----
+  // Everything that needs a round trip to memory is requested here at once: the descriptor,
+  // the residual rows this block will update, and (below) the activations.  All MAXB rows of
+  // the activation buffers exist, so they are loaded without waiting for the row count; rows
+  // beyond it only feed accumulator columns that the epilogue ignores.
   const int M = a.desc ? a.desc->k : a.M;
-  const int mrows = min(MAXB, M);
+  const int pos0 = a.desc ? a.desc->pos0 : a.pos0_host;
+  float old[MAXB];
+  if (rank == 0 && a.epi == EPI_RESID && n_base + tid < a.N) {
+#pragma unroll
+    for (int m = 0; m < MAXB; ++m) old[m] = a.Y[(size_t)m * a.ldy + n_base + tid];
+  }
   const int kl = nkb * UM_KB;
   {  // warp w owns rows w, w+4, w+8, w+12; the loads of all four rows are issued together
     float ssr[4] = {0.f, 0.f, 0.f, 0.f};
@@ -189,13 +198,9 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
         const int m = warp + 4 * r;
-        xa[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-        xb[r] = xa[r];
-        if (m < mrows) {
-          const float* xp = a.X + (size_t)m * a.ldx + k_base + c;
-          xa[r] = *reinterpret_cast<const float4*>(xp);
-          xb[r] = *reinterpret_cast<const float4*>(xp + 4);
-        }
+        const float* xp = a.X + (size_t)m * a.ldx + k_base + c;
+        xa[r] = *reinterpret_cast<const float4*>(xp);
+        xb[r] = *reinterpret_cast<const float4*>(xp + 4);
       }
       const int kb = c / UM_KB, chunk = (c % UM_KB) / 8;
 #pragma unroll
@@ -252,15 +257,11 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
       const uint32_t bh = smem_u32(sB + (size_t)kb * 4096);
 #pragma unroll
       for (int kk = 0; kk < UM_KB / 16; ++kk) {
-        const uint64_t dbh = umma_desc_sw128(bh + kk * 32), dbl = umma_desc_sw128(bh + 2048 + kk * 32);
-        const uint64_t da0 = umma_desc_sw128(a0 + kk * 32);
-        umma_bf16(tmem, da0, dbh, (kb | kk) ? 1u : 0u);
-        umma_bf16(tmem, da0, dbl, 1u);
-        if (GATED) {
-          const uint64_t da1 = umma_desc_sw128(a0 + 16384 + kk * 32);
-          umma_bf16(tmem + 16, da1, dbh, (kb | kk) ? 1u : 0u);
-          umma_bf16(tmem + 16, da1, dbl, 1u);
-        }
+        // one MMA covers hi (token rows 0..15) and lo (rows 16..31) of the activation tile,
+        // so each weight tile is read from shared memory once
+        const uint64_t db = umma_desc_sw128(bh + kk * 32);
+        umma_bf16(tmem, umma_desc_sw128(a0 + kk * 32), db, (kb | kk) ? 1u : 0u);
+        if (GATED) umma_bf16(tmem + 32, umma_desc_sw128(a0 + 16384 + kk * 32), db, (kb | kk) ? 1u : 0u);
       }
       umma_commit(&empty[st]);   // the stage may be refilled once these MMAs have read it
     }
@@ -272,8 +273,20 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
 
   // ---- accumulators: thread t holds weight row n_base + t for the 16 token rows ----
   float acc0[16], acc1[16];
-  tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16), acc0);
-  if (GATED) tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + 16, acc1);
+  {
+    float lo16[16];
+    const uint32_t t0 = tmem + ((uint32_t)(warp * 32) << 16);
+    tmem_ld16(t0, acc0);
+    tmem_ld16(t0 + 16, lo16);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc0[i] += lo16[i];
+    if (GATED) {
+      tmem_ld16(t0 + 32, acc1);
+      tmem_ld16(t0 + 48, lo16);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) acc1[i] += lo16[i];
+    }
+  }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 
   if (cs > 1) {
@@ -300,7 +313,7 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
       }
     }
     const int n = n_base + tid;
-    const int pos0 = a.desc ? a.desc->pos0 : a.pos0_host;
+    const int mrows = min(MAXB, M);
     if (n < a.N) {
       float v0[MAXB], v1[MAXB];
 #pragma unroll
@@ -314,10 +327,7 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
         v0[m] = acc0[m] * inv;
         v1[m] = GATED ? acc1[m] * inv : 0.f;
       }
-      if (a.epi == EPI_RESID) {   // all reads of the residual stream first, then the writes
-        float old[MAXB];
-#pragma unroll
-        for (int m = 0; m < MAXB; ++m) old[m] = m < mrows ? a.Y[(size_t)m * a.ldy + n] : 0.f;
+      if (a.epi == EPI_RESID) {   // the old values were requested right after the dependency wait
 #pragma unroll
         for (int m = 0; m < MAXB; ++m)
           if (m < mrows) a.Y[(size_t)m * a.ldy + n] = old[m] + v0[m];
@@ -346,7 +356,7 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
     }
   }
   __syncthreads();
-  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 32;" ::"r"(tmem) : "memory");
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(TCOLS) : "memory");
 }
 
 }  // namespace bild
