@@ -133,6 +133,7 @@ struct bild_ctx {
   int64_t per_pass_large1 = 0;
   int64_t* cnt = &launches;         // where launches are counted (redirected while capturing)
   cudaStream_t cap_stream = nullptr;  // capture only (the legacy default stream cannot capture); nothing runs on it
+  bool block_simt = false;           // block pass on the SIMT block GEMV instead of the tensor-core kernel
   bool use_pdl = true;               // launch pass kernels with programmatic stream serialization
   bool host_loop = false;            // debug: drive the loop from the host, one read-back per step
   int graph_run_mode = -1;           // mode of a graph run whose launches are not yet counted
@@ -287,6 +288,28 @@ cudaError_t launch_linear_t(bild_ctx* c, const LinArgs& a, int rows_y) {
   return launch_k(c, linear_kernel<WT, MB, RW, false>, grid, dim3(LIN_THREADS), smem, a);
 }
 
+// Block GEMV (SIMT) for up to MAXB token rows: one block per RW weight rows, warps split K.
+template <typename WT, int PC>
+cudaError_t launch_gemvk_pc(bild_ctx* c, const LinArgs& a, int ks) {
+  dim3 grid((a.N + 1) / 2), block(32 * ks);
+  if (a.epi == EPI_GATED) return launch_k(c, gemvk_kernel<WT, 2, PC, true>, grid, block, 0, a);
+  return launch_k(c, gemvk_kernel<WT, 2, PC, false>, grid, block, 0, a);
+}
+// false if K cannot be split into at most 16 warps of at most 4 chunks with 8-column alignment
+template <typename WT>
+bool launch_gemvk_t(bild_ctx* c, const LinArgs& a, cudaError_t* err) {
+  int ks = 0;
+  for (int w = std::max(1, (a.K + 255) / 256); w <= 16; ++w)
+    if (a.K % (8 * w) == 0) { ks = w; break; }
+  if (!ks)
+    for (int w = 16; w >= 1; --w)
+      if (a.K % (8 * w) == 0) { ks = w; break; }
+  const int pc = (a.K / ks + 255) / 256;
+  if (pc > 4) return false;
+  *err = pc == 1 ? launch_gemvk_pc<WT, 1>(c, a, ks) : pc == 2 ? launch_gemvk_pc<WT, 2>(c, a, ks) : launch_gemvk_pc<WT, 4>(c, a, ks);
+  return true;
+}
+
 // MB == 1: the GEMV of the small-model step (and of the large model at k = 1);
 // otherwise the small-M GEMM over up to MAXB rows per row block.
 cudaError_t launch_linear(bild_ctx* c, int dtype, int MB, const LinArgs& a, int rows_y = 1) {
@@ -435,6 +458,10 @@ cudaError_t launch_umma(bild_ctx* c, const LinArgs& a, const CUtensorMap& t0, co
 // Linear layer of a decoder pass: tensor cores for the bf16 block pass, SIMT otherwise.
 cudaError_t launch_dec_linear(bild_ctx* c, Model& m, int MB, const LinArgs& a, int layer, int which_map) {
   int cs, nkb;
+  if (MB != 1 && c->block_simt) {
+    cudaError_t e = cudaSuccess;
+    if (c->cfg.dtype == BILD_BF16 ? launch_gemvk_t<__nv_bfloat16>(c, a, &e) : launch_gemvk_t<float>(c, a, &e)) return e;
+  }
   if (MB != 1 && m.umma && umma_plan(a.N, a.K, a.epi == EPI_GATED, &cs, &nkb)) {
     const CUtensorMap* t = &m.tmaps[(size_t)layer * TM_PER_LAYER];
     return launch_umma(c, a, t[which_map], t[which_map == TM_WI0 ? TM_WI1 : which_map], cs, nkb);
@@ -743,6 +770,8 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   c->cnt = &c->launches;
   const char* hl = std::getenv("BILD_HOST_LOOP");
   c->host_loop = hl && hl[0] == '1';
+  const char* bs = std::getenv("BILD_BLOCK_SIMT");
+  c->block_simt = bs && bs[0] == '1';
   const char* np = std::getenv("BILD_NO_PDL");
   c->use_pdl = !(np && np[0] == '1');
   Bump b(workspace);

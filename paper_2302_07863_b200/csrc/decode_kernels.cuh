@@ -158,6 +158,160 @@ __global__ void __launch_bounds__(GEMV_THREADS) gemv_kernel(LinArgs a) {
 }
 
 // ---------------------------------------------------------------------------------
+// The same GEMV for a block of up to MAXB token rows (steps L1, L3, L4, L6, L7, L8 when the
+// block pass is latency-bound): one block owns RW weight rows, its warps split K so that each
+// warp's weights (<= GEMV_PRE chunks of 256 columns) sit in registers before the dependency
+// wait.  Token rows are then taken four at a time against those registers; the loads of the
+// next four rows are in flight while the current four are reduced.  Partial sums of the
+// warps are added in warp order through shared memory.
+// ---------------------------------------------------------------------------------
+constexpr int GEMVK_TG = 4;   // token rows per step
+
+template <typename WT, int RW, int PC, bool GATED>   // PC: chunks of 256 columns per warp
+__global__ void __launch_bounds__(512) gemvk_kernel(LinArgs a) {
+  constexpr int NV = RW * (GATED ? 2 : 1) * GEMVK_TG + GEMVK_TG;   // values per warp and step: sums + squares
+  __shared__ float s_part[2][16][NV];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int ks = blockDim.x >> 5;
+  const int n0 = blockIdx.x * RW;
+  const int K = a.K, kl = K / ks, kbeg = warp * kl;
+  const WT* W0 = (const WT*)a.W0;
+  const WT* W1 = (const WT*)a.W1;
+  float pre0[RW][PC][8], pre1[GATED ? RW : 1][GATED ? PC : 1][8];
+#pragma unroll
+  for (int r = 0; r < RW; ++r) {
+    const size_t row = (size_t)min(n0 + r, a.N - 1) * K + kbeg;
+#pragma unroll
+    for (int p = 0; p < PC; ++p) {
+      const int c = p * 256 + lane * 8;
+      if (c < kl) {
+        load8(W0 + row + c, pre0[r][p]);
+        if (GATED) load8(W1 + row + c, pre1[r][p]);
+      }
+    }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  // requested together: the row count, the gains, the first four activation rows, and (for the
+  // threads that write results) the residual values they will update
+  const int M = a.desc ? a.desc->k : a.M;
+  const int pos0 = a.desc ? a.desc->pos0 : a.pos0_host;
+  const int out_r = threadIdx.x / GEMVK_TG, out_m = threadIdx.x % GEMVK_TG;   // writer threads: tid < RW * TG
+  const bool writer = threadIdx.x < RW * GEMVK_TG && n0 + out_r < a.N;
+  float old[MAXB / GEMVK_TG];
+  if (writer && a.epi == EPI_RESID) {
+#pragma unroll
+    for (int g = 0; g < MAXB / GEMVK_TG; ++g) old[g] = a.Y[(size_t)(g * GEMVK_TG + out_m) * a.ldy + n0 + out_r];
+  }
+  float gn[PC][8];
+#pragma unroll
+  for (int p = 0; p < PC; ++p) {
+    const int c = p * 256 + lane * 8;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) gn[p][i] = 1.f;
+    if (a.gain && c < kl) {
+      const float4 g0 = *reinterpret_cast<const float4*>(a.gain + kbeg + c);
+      const float4 g1 = *reinterpret_cast<const float4*>(a.gain + kbeg + c + 4);
+      gn[p][0] = g0.x; gn[p][1] = g0.y; gn[p][2] = g0.z; gn[p][3] = g0.w;
+      gn[p][4] = g1.x; gn[p][5] = g1.y; gn[p][6] = g1.z; gn[p][7] = g1.w;
+    }
+  }
+  float4 xa[GEMVK_TG][PC], xb[GEMVK_TG][PC];
+  auto load_rows = [&](int m_first) {   // all MAXB rows of the activation buffer exist
+#pragma unroll
+    for (int t = 0; t < GEMVK_TG; ++t)
+#pragma unroll
+      for (int p = 0; p < PC; ++p) {
+        const int c = p * 256 + lane * 8;
+        if (c < kl) {
+          const float* xp = a.X + (size_t)(m_first + t) * a.ldx + kbeg + c;
+          xa[t][p] = *reinterpret_cast<const float4*>(xp);
+          xb[t][p] = *reinterpret_cast<const float4*>(xp + 4);
+        }
+      }
+  };
+  load_rows(0);
+  const int groups = (min(M, MAXB) + GEMVK_TG - 1) / GEMVK_TG;
+#pragma unroll
+  for (int g = 0; g < MAXB / GEMVK_TG; ++g) {
+    if (g >= groups) break;   // uniform over the block
+    float acc0[RW][GEMVK_TG], acc1[GATED ? RW : 1][GEMVK_TG], ss[GEMVK_TG];
+#pragma unroll
+    for (int t = 0; t < GEMVK_TG; ++t) {
+      ss[t] = 0.f;
+#pragma unroll
+      for (int r = 0; r < RW; ++r) { acc0[r][t] = 0.f; if (GATED) acc1[r][t] = 0.f; }
+#pragma unroll
+      for (int p = 0; p < PC; ++p) {
+        const int c = p * 256 + lane * 8;
+        if (c < kl) {
+          float h[8] = {xa[t][p].x, xa[t][p].y, xa[t][p].z, xa[t][p].w, xb[t][p].x, xb[t][p].y, xb[t][p].z, xb[t][p].w};
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { ss[t] += h[i] * h[i]; h[i] *= gn[p][i]; }
+#pragma unroll
+          for (int r = 0; r < RW; ++r) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              acc0[r][t] += pre0[r][p][i] * h[i];
+              if (GATED) acc1[r][t] += pre1[r][p][i] * h[i];
+            }
+          }
+        }
+      }
+    }
+    if (g + 1 < groups) load_rows((g + 1) * GEMVK_TG);   // in flight during the reduction below
+    float* sp = s_part[g & 1][warp];
+#pragma unroll
+    for (int t = 0; t < GEMVK_TG; ++t) {
+#pragma unroll
+      for (int r = 0; r < RW; ++r) {
+        const float v = warp_sum(acc0[r][t]);
+        if (lane == 0) sp[r * GEMVK_TG + t] = v;
+        if (GATED) {
+          const float v1 = warp_sum(acc1[r][t]);
+          if (lane == 0) sp[(RW + r) * GEMVK_TG + t] = v1;
+        }
+      }
+      const float sv = warp_sum(ss[t]);
+      if (lane == 0) sp[NV - GEMVK_TG + t] = sv;
+    }
+    __syncthreads();
+    const int m = g * GEMVK_TG + out_m;
+    if (writer && m < M) {
+      float v0 = 0.f, v1 = 0.f, sq = 0.f;
+      for (int w2 = 0; w2 < ks; ++w2) {   // fixed order
+        const float* q = s_part[g & 1][w2];
+        v0 += q[out_r * GEMVK_TG + out_m];
+        if (GATED) v1 += q[(RW + out_r) * GEMVK_TG + out_m];
+        sq += q[NV - GEMVK_TG + out_m];
+      }
+      if (a.gain) {
+        const float inv = 1.f / sqrtf(sq / (float)K + a.eps);
+        v0 *= inv;
+        v1 *= inv;
+      }
+      const int n = n0 + out_r;
+      switch (a.epi) {
+        case EPI_STORE: a.Y[(size_t)m * a.ldy + n] = v0; break;
+        case EPI_RELU: a.Y[(size_t)m * a.ldy + n] = fmaxf(v0, 0.f); break;
+        case EPI_GATED: a.Y[(size_t)m * a.ldy + n] = gelu_tanh(v0) * v1; break;
+        case EPI_RESID: a.Y[(size_t)m * a.ldy + n] = old[g] + v0; break;
+        default: {
+          const int part = a.first_part + n / a.inner;
+          const int rr = n % a.inner;
+          if (part == 0) {
+            a.q_out[(size_t)m * a.ldq + rr] = v0;
+          } else {
+            const int h = rr / a.dkv, c = rr % a.dkv;
+            if (pos0 + m < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + pos0 + m) * a.dkv + c] = v0;
+          }
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------
 // Block attention (steps S2, S5, L2, L5 and the encoder's self-attention): one block per
 // (head, key split, block of MB query rows) reads every key and value of its split ONCE
 // and serves all MB rows from it.
