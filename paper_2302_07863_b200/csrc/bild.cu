@@ -243,15 +243,27 @@ cudaError_t launch_k(bild_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block,
   return cudaLaunchKernelEx(&cfg, kern, args...);
 }
 
-template <typename WT, int RW>
+int ilog2(int v) { int s = 0; while ((1 << s) < v) ++s; return s; }
+
+// Warps per row group: one 256-column chunk per warp where K allows it (K <= 4096).
+int gemv_ksplit(int K) {
+  for (int w = std::max(1, (K + 255) / 256); w <= 16; ++w)
+    if (K % (8 * w) == 0) return w;
+  for (int w = 16; w >= 1; --w)
+    if (K % (8 * w) == 0) return w;
+  return 1;
+}
+
+template <typename WT>
 cudaError_t launch_gemv_t(bild_ctx* c, const LinArgs& a0) {
   LinArgs a = a0;
-  // enough warps along K that every warp's slice (<= 1024 columns) is requested in one batch
-  a.ksplit = (a.K % 32 == 0 && a.K > 2048) ? 4 : (a.K % 16 == 0 && a.K > 1024) ? 2 : 1;
-  const int groups = (GEMV_THREADS / 32) / a.ksplit;
-  dim3 grid((a.N + groups * RW - 1) / (groups * RW));
-  if (a.epi == EPI_GATED) return launch_k(c, gemv_kernel<WT, RW, true>, grid, dim3(GEMV_THREADS), 0, a);
-  return launch_k(c, gemv_kernel<WT, RW, false>, grid, dim3(GEMV_THREADS), 0, a);
+  a.ksplit = gemv_ksplit(a.K);
+  a.dkv_shift = ilog2(std::max(1, a.dkv));
+  const int groups = std::max(1, 4 / a.ksplit);
+  a.groups = groups; a.kl = a.K / a.ksplit; a.inv_k = 1.f / (float)a.K;
+  dim3 grid((a.N + 2 * groups - 1) / (2 * groups)), block(32 * a.ksplit * groups);
+  if (a.epi == EPI_GATED) return launch_k(c, gemv_kernel<WT, true>, grid, block, 0, a);
+  return launch_k(c, gemv_kernel<WT, false>, grid, block, 0, a);
 }
 
 template <int MB, bool STAGE>
@@ -267,9 +279,18 @@ cudaError_t launch_battn_t(bild_ctx* c, BAttnArgs a, int row_blocks, int keys_ca
 }
 // Decoder attention stages its keys / values in shared memory (at most 128 keys per split);
 // the encoder's self-attention (mode 2, all keys in one block) reads them from global memory.
-cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a, int row_blocks, int keys_cap) {
-  if (a.mode == 2) return launch_battn_t<MAXB, false>(c, a, row_blocks, keys_cap);
-  return MB == 1 ? launch_battn_t<1, true>(c, a, row_blocks, keys_cap) : launch_battn_t<MAXB, true>(c, a, row_blocks, keys_cap);
+cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_blocks, int keys_cap) {
+  if (a0.mode == 2) return launch_battn_t<MAXB, false>(c, a0, row_blocks, keys_cap);
+  BAttnArgs a = a0;
+  a.smem_keys = ((keys_cap + a.nsplit - 1) / a.nsplit + 3) / 4 * 4;
+  const size_t smem = sizeof(float) * ((size_t)MB * a.dkv + (size_t)MB * a.smem_keys + (size_t)a.smem_keys * (2 * a.dkv + 4));
+  if (smem > 40 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(dattn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (e != cudaSuccess) return e;
+  }
+  DAttnArgs d;
+  d.b = a; d.MB = MB; d.dkv_shift = ilog2(a.dkv);
+  return launch_k(c, dattn_kernel, dim3(a.H, a.nsplit), dim3(DATT_THREADS), smem, d);
 }
 
 template <typename WT, int MB, int RW>
@@ -290,7 +311,9 @@ cudaError_t launch_linear_t(bild_ctx* c, const LinArgs& a, int rows_y) {
 
 // Block GEMV (SIMT) for up to MAXB token rows: one block per RW weight rows, warps split K.
 template <typename WT, int PC>
-cudaError_t launch_gemvk_pc(bild_ctx* c, const LinArgs& a, int ks) {
+cudaError_t launch_gemvk_pc(bild_ctx* c, const LinArgs& a0, int ks) {
+  LinArgs a = a0;
+  a.dkv_shift = ilog2(std::max(1, a.dkv));
   dim3 grid((a.N + 1) / 2), block(32 * ks);
   if (a.epi == EPI_GATED) return launch_k(c, gemvk_kernel<WT, 2, PC, true>, grid, block, 0, a);
   return launch_k(c, gemvk_kernel<WT, 2, PC, false>, grid, block, 0, a);
@@ -314,8 +337,8 @@ bool launch_gemvk_t(bild_ctx* c, const LinArgs& a, cudaError_t* err) {
 // otherwise the small-M GEMM over up to MAXB rows per row block.
 cudaError_t launch_linear(bild_ctx* c, int dtype, int MB, const LinArgs& a, int rows_y = 1) {
   if (dtype == BILD_BF16)
-    return MB == 1 ? launch_gemv_t<__nv_bfloat16, 2>(c, a) : launch_linear_t<__nv_bfloat16, MAXB, 2>(c, a, rows_y);
-  return MB == 1 ? launch_gemv_t<float, 2>(c, a) : launch_linear_t<float, MAXB, 2>(c, a, rows_y);
+    return MB == 1 ? launch_gemv_t<__nv_bfloat16>(c, a) : launch_linear_t<__nv_bfloat16, MAXB, 2>(c, a, rows_y);
+  return MB == 1 ? launch_gemv_t<float>(c, a) : launch_linear_t<float, MAXB, 2>(c, a, rows_y);
 }
 
 template <typename WT, int MB, int RW>

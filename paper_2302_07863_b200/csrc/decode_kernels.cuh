@@ -14,147 +14,97 @@ namespace bild {
 // before the dependency wait; x, g and the sum of squares are taken in the same pass, so
 // there is no shared memory and no block-wide barrier.  Same epilogues as linear_kernel.
 // ---------------------------------------------------------------------------------
-constexpr int GEMV_THREADS = 128;
-constexpr int GEMV_PRE = 4;  // column chunks (of 256) whose weights are fetched ahead
+// Kernel code is kept small on purpose: the kernels of a layer alternate every few
+// microseconds and their instructions have to stay in the SMs' instruction caches.
+constexpr int GEMV_PRE = 4;   // (block GEMV) column chunks of 256 whose weights are fetched ahead
 
-// a.ksplit (1, 2 or 4) warps share one group of RW rows, each taking a contiguous K / ksplit
-// columns, so that for K up to 4096 every weight byte of the block is requested in one batch
-// before the dependency wait; their partial sums are added in warp order through shared memory.
-template <typename WT, int RW, bool GATED>
-__global__ void __launch_bounds__(GEMV_THREADS) gemv_kernel(LinArgs a) {
-  constexpr int NW = GEMV_THREADS / 32;
-  __shared__ float s_part[NW][2 * RW + 1];
+// Where output row n of a packed q|k|v (or k|v) projection goes: part 0 = q, 1 = k, 2 = v.
+__device__ __forceinline__ void heads_store(const LinArgs& a, int n, int m, int pos0, float v) {
+  int part = a.first_part, rr = n;
+  if (rr >= a.inner) { rr -= a.inner; ++part; }
+  if (rr >= a.inner) { rr -= a.inner; ++part; }
+  if (part == 0) {
+    a.q_out[(size_t)m * a.ldq + rr] = v;
+  } else {
+    const int h = rr >> a.dkv_shift, c = rr & (a.dkv - 1);
+    const int row = pos0 + m;
+    if (row < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + row) * a.dkv + c] = v;
+  }
+}
+
+// One group of 2 weight rows is shared by a.ksplit warps, each taking K / ksplit (<= 256 when
+// K <= 4096) contiguous columns, so every weight byte is requested before the dependency
+// wait with one 128-bit load per lane and row.  Partial sums are added in warp order.
+template <typename WT, bool GATED>
+__global__ void __launch_bounds__(512) gemv_kernel(LinArgs a) {
+  __shared__ float s_part[16][5];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int ks = a.ksplit > 1 ? a.ksplit : 1;
-  const int group = warp / ks, kw = warp - group * ks;
-  const int n0 = (blockIdx.x * (NW / ks) + group) * RW;
-  const int K = a.K, kl = K / ks, kbeg = kw * kl;
-  const WT* W0 = (const WT*)a.W0;
-  const WT* W1 = (const WT*)a.W1;
-  const bool active = n0 < a.N;
-  float pre0[RW][GEMV_PRE][8], pre1[GATED ? RW : 1][GATED ? GEMV_PRE : 1][8];
-  if (active) {
-#pragma unroll
-    for (int r = 0; r < RW; ++r) {
-      const size_t row = (size_t)min(n0 + r, a.N - 1) * K + kbeg;
-#pragma unroll
-      for (int p = 0; p < GEMV_PRE; ++p) {
-        const int c = p * 256 + lane * 8;
-        if (c < kl) {
-          load8(W0 + row + c, pre0[r][p]);
-          if (GATED) load8(W1 + row + c, pre1[r][p]);
-        }
-      }
-    }
+  const int ks = a.ksplit;
+  // more than one group per block only for ksplit 1 or 2 (host: groups = max(1, 4 / ksplit))
+  const int group = a.groups == 1 ? 0 : (ks == 1 ? warp : warp >> 1);
+  const int kw = a.groups == 1 ? warp : (ks == 1 ? 0 : warp & 1);
+  const int n0 = (blockIdx.x * a.groups + group) * 2;
+  const int K = a.K, kl = a.kl, kbeg = kw * kl;
+  const int c0 = lane * 8;
+  const int r0 = min(n0, a.N - 1), r1 = min(n0 + 1, a.N - 1);
+  const WT* W0 = (const WT*)a.W0 + kbeg;
+  const WT* W1 = (const WT*)a.W1 + kbeg;
+  float w00[8], w01[8], w10[8], w11[8];
+  if (c0 < kl) {
+    load8(W0 + (size_t)r0 * K + c0, w00);
+    load8(W0 + (size_t)r1 * K + c0, w01);
+    if (GATED) { load8(W1 + (size_t)r0 * K + c0, w10); load8(W1 + (size_t)r1 * K + c0, w11); }
   }
   pdl_launch_dependents();
   pdl_wait();
   const float* X = a.X + kbeg;
   const float* G = a.gain ? a.gain + kbeg : nullptr;
-  float acc0[RW], acc1[GATED ? RW : 1], ss = 0.f;
-#pragma unroll
-  for (int r = 0; r < RW; ++r) { acc0[r] = 0.f; if (GATED) acc1[r] = 0.f; }
-
-  auto fma8 = [&](const float (&w)[8], const float (&h)[8]) {
-    return w[0] * h[0] + w[1] * h[1] + w[2] * h[2] + w[3] * h[3] + w[4] * h[4] + w[5] * h[5] + w[6] * h[6] + w[7] * h[7];
-  };
-  auto load_h = [&](int c, float (&h)[8]) {
+  float a00 = 0.f, a01 = 0.f, a10 = 0.f, a11 = 0.f, ss = 0.f;
+#pragma unroll 1
+  for (int c = c0; c < kl; c += 256) {
+    if (c != c0) {   // columns beyond the first 256 of this warp (K > 4096 only)
+      load8(W0 + (size_t)r0 * K + c, w00);
+      load8(W0 + (size_t)r1 * K + c, w01);
+      if (GATED) { load8(W1 + (size_t)r0 * K + c, w10); load8(W1 + (size_t)r1 * K + c, w11); }
+    }
     const float4 x0 = *reinterpret_cast<const float4*>(X + c);
     const float4 x1 = *reinterpret_cast<const float4*>(X + c + 4);
-    h[0] = x0.x; h[1] = x0.y; h[2] = x0.z; h[3] = x0.w; h[4] = x1.x; h[5] = x1.y; h[6] = x1.z; h[7] = x1.w;
+    float h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
     if (G) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) ss += h[i] * h[i];
       const float4 g0 = *reinterpret_cast<const float4*>(G + c);
       const float4 g1 = *reinterpret_cast<const float4*>(G + c + 4);
-      h[0] *= g0.x; h[1] *= g0.y; h[2] *= g0.z; h[3] *= g0.w; h[4] *= g1.x; h[5] *= g1.y; h[6] *= g1.z; h[7] *= g1.w;
-    }
-  };
-  if (active) {
-    float hp[GEMV_PRE][8];
+      const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
 #pragma unroll
-    for (int p = 0; p < GEMV_PRE; ++p) {
-      const int c = p * 256 + lane * 8;
-      if (c < kl) load_h(c, hp[p]);
+      for (int i = 0; i < 8; ++i) { ss += h[i] * h[i]; h[i] *= g[i]; }
     }
 #pragma unroll
-    for (int p = 0; p < GEMV_PRE; ++p) {
-      const int c = p * 256 + lane * 8;
-      if (c < kl) {
-#pragma unroll
-        for (int r = 0; r < RW; ++r) {
-          acc0[r] += fma8(pre0[r][p], hp[p]);
-          if (GATED) acc1[r] += fma8(pre1[r][p], hp[p]);
-        }
-      }
-    }
-    for (int c = GEMV_PRE * 256 + lane * 8; c < kl; c += 256) {   // only for K / ksplit > 1024
-      float h[8];
-      load_h(c, h);
-#pragma unroll
-      for (int r = 0; r < RW; ++r) {
-        float w[8];
-        const size_t row = (size_t)min(n0 + r, a.N - 1) * K + kbeg;
-        load8(W0 + row + c, w);
-        acc0[r] += fma8(w, h);
-        if (GATED) { load8(W1 + row + c, w); acc1[r] += fma8(w, h); }
-      }
+    for (int i = 0; i < 8; ++i) {
+      a00 += w00[i] * h[i];
+      a01 += w01[i] * h[i];
+      if (GATED) { a10 += w10[i] * h[i]; a11 += w11[i] * h[i]; }
     }
   }
-#pragma unroll
-  for (int r = 0; r < RW; ++r) {
-    acc0[r] = warp_sum(acc0[r]);
-    if (GATED) acc1[r] = warp_sum(acc1[r]);
-  }
-  ss = warp_sum(ss);
+  a00 = warp_sum(a00); a01 = warp_sum(a01); ss = warp_sum(ss);
+  if (GATED) { a10 = warp_sum(a10); a11 = warp_sum(a11); }
   if (ks > 1) {
-    if (lane == 0) {
-#pragma unroll
-      for (int r = 0; r < RW; ++r) { s_part[warp][r] = acc0[r]; s_part[warp][RW + r] = GATED ? acc1[r] : 0.f; }
-      s_part[warp][2 * RW] = ss;
-    }
+    if (lane == 0) { s_part[warp][0] = a00; s_part[warp][1] = a01; s_part[warp][2] = a10; s_part[warp][3] = a11; s_part[warp][4] = ss; }
     __syncthreads();
     if (kw != 0) return;
-    ss = 0.f;
-#pragma unroll
-    for (int r = 0; r < RW; ++r) { acc0[r] = 0.f; if (GATED) acc1[r] = 0.f; }
-    for (int w2 = 0; w2 < ks; ++w2) {   // fixed order
-#pragma unroll
-      for (int r = 0; r < RW; ++r) {
-        acc0[r] += s_part[group * ks + w2][r];
-        if (GATED) acc1[r] += s_part[group * ks + w2][RW + r];
-      }
-      ss += s_part[group * ks + w2][2 * RW];
+    a00 = a01 = a10 = a11 = ss = 0.f;
+    for (int w2 = group * ks; w2 < group * ks + ks; ++w2) {   // fixed order
+      a00 += s_part[w2][0]; a01 += s_part[w2][1]; a10 += s_part[w2][2]; a11 += s_part[w2][3]; ss += s_part[w2][4];
     }
   }
-  if (!active) return;
-  float inv = 1.f;
-  if (a.gain) inv = 1.f / sqrtf(ss / (float)K + a.eps);
-  float v0 = 0.f, v1 = 0.f;
-#pragma unroll
-  for (int r = 0; r < RW; ++r) {
-    if (lane == r) { v0 = acc0[r] * inv; if (GATED) v1 = acc1[r] * inv; }
-  }
-  if (lane >= RW) return;
+  if (lane > 1) return;
   const int n = n0 + lane;
   if (n >= a.N) return;
-  const int pos0 = a.desc ? a.desc->pos0 : a.pos0_host;
-  switch (a.epi) {
-    case EPI_STORE: a.Y[n] = v0; break;
-    case EPI_RELU: a.Y[n] = fmaxf(v0, 0.f); break;
-    case EPI_GATED: a.Y[n] = gelu_tanh(v0) * v1; break;
-    case EPI_RESID: a.Y[n] += v0; break;
-    default: {
-      const int part = a.first_part + n / a.inner;
-      const int rr = n % a.inner;
-      if (part == 0) {
-        a.q_out[rr] = v0;
-      } else {
-        const int h = rr / a.dkv, c = rr % a.dkv;
-        if (pos0 < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + pos0) * a.dkv + c] = v0;
-      }
-    }
-  }
+  const float inv = a.gain ? rsqrtf(ss * a.inv_k + a.eps) : 1.f;
+  const float v0 = (lane ? a01 : a00) * inv;
+  if (a.epi == EPI_RESID) a.Y[n] += v0;
+  else if (a.epi == EPI_STORE) a.Y[n] = v0;
+  else if (a.epi == EPI_RELU) a.Y[n] = fmaxf(v0, 0.f);
+  else if (a.epi == EPI_GATED) { if (GATED) a.Y[n] = gelu_tanh(v0) * ((lane ? a11 : a10) * inv); }
+  else heads_store(a, n, 0, a.desc ? a.desc->pos0 : a.pos0_host, v0);
 }
 
 // ---------------------------------------------------------------------------------
@@ -286,7 +236,7 @@ __global__ void __launch_bounds__(512) gemvk_kernel(LinArgs a) {
         sq += q[NV - GEMVK_TG + out_m];
       }
       if (a.gain) {
-        const float inv = 1.f / sqrtf(sq / (float)K + a.eps);
+        const float inv = rsqrtf(sq / (float)K + a.eps);
         v0 *= inv;
         v1 *= inv;
       }
@@ -296,16 +246,7 @@ __global__ void __launch_bounds__(512) gemvk_kernel(LinArgs a) {
         case EPI_RELU: a.Y[(size_t)m * a.ldy + n] = fmaxf(v0, 0.f); break;
         case EPI_GATED: a.Y[(size_t)m * a.ldy + n] = gelu_tanh(v0) * v1; break;
         case EPI_RESID: a.Y[(size_t)m * a.ldy + n] = old[g] + v0; break;
-        default: {
-          const int part = a.first_part + n / a.inner;
-          const int rr = n % a.inner;
-          if (part == 0) {
-            a.q_out[(size_t)m * a.ldq + rr] = v0;
-          } else {
-            const int h = rr / a.dkv, c = rr % a.dkv;
-            if (pos0 + m < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + pos0 + m) * a.dkv + c] = v0;
-          }
-        }
+        default: heads_store(a, n, m, pos0, v0);
       }
     }
   }
@@ -524,6 +465,146 @@ __global__ void __launch_bounds__(BATT_THREADS) battn_kernel(BAttnArgs a) {
       }
     }
     a.out[(size_t)(m0 + i) * a.ldo + h * dkv + cc] = num / den;
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// Decode attention, compact version of the block attention above for the decoder passes
+// (modes 0 and 1 only).  Keys and values of the block's split are staged in shared memory
+// (cross-attention: before the dependency wait), scores are taken one (row, key) pair per
+// thread, soft-max one warp per row, values one (row, channel) pair per thread.  Loops are
+// kept rolled: the kernel runs for a few microseconds and its instructions must stay cached.
+// ---------------------------------------------------------------------------------
+constexpr int DATT_THREADS = 128;
+
+struct DAttnArgs {
+  BAttnArgs b;
+  int MB;          // rows of the q / out buffers and of the scratch layout (1 or MAXB)
+  int dkv_shift;   // log2(dkv)
+};
+
+__device__ __forceinline__ void dattn_stage(const BAttnArgs& a, int h, int j0, int nk, int dshift, float* sK, float* sV) {
+  const int dkv = a.dkv, kst = dkv + 4, q4s = dshift - 2;
+  const float* Kg = a.kc + ((size_t)h * a.cap + j0) * dkv;
+  const float* Vg = a.vc + ((size_t)h * a.cap + j0) * dkv;
+#pragma unroll 1
+  for (int idx = threadIdx.x; idx < (nk << q4s); idx += DATT_THREADS) {
+    const int jj = idx >> q4s, e4 = (idx & ((1 << q4s) - 1)) << 2;
+    cp_async16(sK + jj * kst + e4, Kg + jj * dkv + e4);
+    cp_async16(sV + jj * dkv + e4, Vg + jj * dkv + e4);
+  }
+}
+
+__global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
+  extern __shared__ float s_dyn[];   // q [MB][dkv] | scores [MB][sk] | keys [sk][dkv + 4] | values [sk][dkv]
+  __shared__ float s_m[MAXB], s_l[MAXB];
+  __shared__ int s_last;
+  const BAttnArgs& a = d.b;
+  const int MB = d.MB, dshift = d.dkv_shift;
+  const int h = blockIdx.x, sp = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int dkv = a.dkv, sk = a.smem_keys, kst = dkv + 4;
+  float* sQ = s_dyn;
+  float* sS = sQ + MB * dkv;
+  float* sK = sS + MB * sk;
+  float* sV = sK + sk * kst;
+  int j0 = 0, nk = 0;
+  if (a.mode == 0) {   // encoder keys never change while decoding: fetch before the dependency wait
+    const int n_all = min(*a.n_keys_dev, a.cap);
+    const int ch = (n_all + a.nsplit - 1) / a.nsplit;
+    j0 = sp * ch;
+    nk = min(max(0, min(n_all, j0 + ch) - j0), sk);
+    dattn_stage(a, h, j0, nk, dshift, sK, sV);
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  const int M = min(a.desc->k, MB), pos0 = a.desc->pos0;
+  if (a.mode == 1) {
+    const int n_all = min(pos0 + M, a.cap);
+    const int ch = (n_all + a.nsplit - 1) / a.nsplit;
+    j0 = sp * ch;
+    nk = min(max(0, min(n_all, j0 + ch) - j0), sk);
+    dattn_stage(a, h, j0, nk, dshift, sK, sV);
+  }
+#pragma unroll 1
+  for (int idx = tid; idx < (M << (dshift - 2)); idx += DATT_THREADS) {
+    const int i = idx >> (dshift - 2), e4 = (idx & ((dkv >> 2) - 1)) << 2;
+    cp_async16(sQ + i * dkv + e4, a.q + (size_t)i * a.ldq + h * dkv + e4);
+  }
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_all;" ::: "memory");
+  __syncthreads();
+  // warp w owns rows w, w+4, ...: scores (lanes over keys), soft-max, values (lanes over channels)
+  float* P = a.part + (((size_t)h * a.nsplit + sp) * MB) * (dkv + 2);
+#pragma unroll 1
+  for (int i = warp; i < M; i += DATT_THREADS / 32) {
+    const float4* qr = reinterpret_cast<const float4*>(sQ + i * dkv);
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int jj = lane; jj < nk; jj += 32) {
+      const float4* kr = reinterpret_cast<const float4*>(sK + jj * kst);
+      float acc = 0.f;
+#pragma unroll 4
+      for (int e = 0; e < (dkv >> 2); ++e) {
+        const float4 kv = kr[e], qv = qr[e];
+        acc += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
+      }
+      const int j = j0 + jj;
+      if (a.mode == 1) acc = (j <= pos0 + i) ? acc + a.bias[(size_t)h * a.bias_ld + (pos0 + i - j)] : -INFINITY;
+      sS[i * sk + jj] = acc;
+      mx = fmaxf(mx, acc);
+    }
+    mx = warp_max(mx);
+    float sum = 0.f;
+#pragma unroll 1
+    for (int jj = lane; jj < nk; jj += 32) {
+      const float sc = sS[i * sk + jj];
+      const float pr = (sc == -INFINITY) ? 0.f : __expf(sc - mx);
+      sS[i * sk + jj] = pr;
+      sum += pr;
+    }
+    sum = warp_sum(sum);
+    __syncwarp();
+    const float rl = a.nsplit == 1 ? __frcp_rn(sum) : 1.f;
+#pragma unroll 1
+    for (int c = lane; c < dkv; c += 32) {
+      float acc = 0.f;
+#pragma unroll 4
+      for (int jj = 0; jj < nk; ++jj) acc += sS[i * sk + jj] * sV[jj * dkv + c];
+      if (a.nsplit == 1) a.out[(size_t)i * a.ldo + h * dkv + c] = acc * rl;
+      else P[(size_t)i * (dkv + 2) + 2 + c] = acc;
+    }
+    if (a.nsplit > 1 && lane == 0) { P[(size_t)i * (dkv + 2)] = mx; P[(size_t)i * (dkv + 2) + 1] = sum; }
+  }
+  if (a.nsplit == 1) return;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned t = atomicAdd(&a.counters[h], 1u);
+    s_last = (t == (unsigned)a.nsplit - 1);
+    if (s_last) a.counters[h] = 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const float* P0 = a.part + ((size_t)h * a.nsplit * MB) * (dkv + 2);
+#pragma unroll 1
+  for (int i = warp; i < M; i += DATT_THREADS / 32) {
+    float gm = -INFINITY;
+#pragma unroll 1
+    for (int s2 = 0; s2 < a.nsplit; ++s2) gm = fmaxf(gm, __ldcg(&P0[((size_t)s2 * MB + i) * (dkv + 2)]));
+#pragma unroll 1
+    for (int c = lane; c < dkv; c += 32) {
+      float num = 0.f, den = 0.f;
+#pragma unroll 1
+      for (int s2 = 0; s2 < a.nsplit; ++s2) {   // split order
+        const float* Ps = P0 + ((size_t)s2 * MB + i) * (dkv + 2);
+        const float l = __ldcg(&Ps[1]);
+        const float w = l > 0.f ? __expf(__ldcg(&Ps[0]) - gm) : 0.f;
+        den += l * w;
+        num += __ldcg(&Ps[2 + c]) * w;
+      }
+      a.out[(size_t)i * a.ldo + h * dkv + c] = num * __frcp_rn(den);
+    }
   }
 }
 

@@ -57,7 +57,10 @@ struct LinArgs {
   float* vc;
   int cap;
   int pos0_host;
-  int ksplit;             // gemv_kernel only: warps sharing one row group along K (0 or 1 = none)
+  int ksplit;             // gemv_kernel only: warps sharing one row group along K
+  int dkv_shift;          // log2(dkv)
+  int groups, kl;         // gemv_kernel only: row groups per block, columns per warp
+  float inv_k;            // 1 / K
 };
 
 constexpr int LIN_THREADS = 256;
