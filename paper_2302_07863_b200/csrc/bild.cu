@@ -173,7 +173,7 @@ int check_config(const bild_config* cfg, std::string& why) {
   if (cfg->small_cfg.vocab != cfg->large_cfg.vocab) { why = "the two models must share a vocabulary"; return BILD_ERR_ARG; }
   if (cfg->dtype != BILD_FP32 && cfg->dtype != BILD_BF16) { why = "dtype"; return BILD_ERR_ARG; }
   if (cfg->max_enc_len < 1 || cfg->max_enc_len > 2048) { why = "1 <= max_enc_len <= 2048"; return BILD_ERR_ARG; }
-  if (cfg->max_dec_len < 2 || cfg->max_dec_len > 4096) { why = "2 <= max_dec_len <= 4096"; return BILD_ERR_ARG; }
+  if (cfg->max_dec_len < 2 || cfg->max_dec_len > 2048) { why = "2 <= max_dec_len <= 2048"; return BILD_ERR_ARG; }
   if (cfg->max_draft < 1 || cfg->max_draft > MAXB - 1) { why = "1 <= max_draft <= 15"; return BILD_ERR_ARG; }
   if (cfg->start_id < 0 || cfg->start_id >= cfg->small_cfg.vocab) { why = "start_id"; return BILD_ERR_ARG; }
   return BILD_OK;
@@ -283,14 +283,31 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
   if (a0.mode == 2) return launch_battn_t<MAXB, false>(c, a0, row_blocks, keys_cap);
   BAttnArgs a = a0;
   a.smem_keys = ((keys_cap + a.nsplit - 1) / a.nsplit + 3) / 4 * 4;
-  const size_t smem = sizeof(float) * ((size_t)MB * a.dkv + (size_t)MB * a.smem_keys + (size_t)a.smem_keys * (2 * a.dkv + 4));
+  const size_t smem = sizeof(float) * ((size_t)MB * a.dkv + (size_t)MB * a.smem_keys + (size_t)a.smem_keys * (2 * a.dkv + 4) +
+                                       (a.nsplit > 1 ? (size_t)a.nsplit * MB * (a.dkv + 2) : 0));
   if (smem > 40 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(dattn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(dattn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
   }
   DAttnArgs d;
   d.b = a; d.MB = MB; d.dkv_shift = ilog2(a.dkv);
-  return launch_k(c, dattn_kernel, dim3(a.H, a.nsplit), dim3(DATT_THREADS), smem, d);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.H, a.nsplit); cfg.blockDim = dim3(DATT_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (c->use_pdl) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (a.nsplit > 1) {   // the splits of one head are one cluster
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = 1; at[na].val.clusterDim.y = a.nsplit; at[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = at; cfg.numAttrs = na;
+  (*c->cnt)++;
+  return cudaLaunchKernelEx(&cfg, dattn_kernel, d);
 }
 
 template <typename WT, int MB, int RW>
@@ -361,11 +378,11 @@ cudaError_t launch_head(cudaStream_t s, int dtype, int MB, const HeadArgs& a, in
   return MB == 1 ? launch_head_t<float, 1, 4>(&tmp, a, grid, launches) : launch_head_t<float, MAXB, 2>(&tmp, a, grid, launches);
 }
 
-int pick_nsplit(int ctas_without_split, int keys_cap) {
-  int ns = (148 + ctas_without_split - 1) / ctas_without_split;
-  ns = std::min(ns, std::max(1, keys_cap / 32));
-  ns = std::max(1, std::min(ns, NSPLIT_MAX));
-  while ((keys_cap + ns - 1) / ns > 128 && ns < NSPLIT_MAX) ++ns;   // staged keys / values stay under 72 KB
+// Key splits per head for decoder attention: the splits of a head form one cluster (<= 8 blocks),
+// each staging at most 256 keys; more splits until about one block per SM.
+int pick_nsplit(int heads, int keys_cap) {
+  int ns = 1;
+  while (ns < 8 && (heads * ns < 148 / 2 || (keys_cap + ns - 1) / ns > 256) && keys_cap / (ns * 2) >= 16) ns *= 2;
   return ns;
 }
 
@@ -511,7 +528,9 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x));
   // self-attention: one block per head up to 128 cached rows (no merge step); cross-attention:
   // enough splits of the encoder keys to occupy the SMs
-  const int ns_self = std::max(1, (cap + 127) / 128), ns_cross = pick_nsplit(H, ecap);
+  int ns_self = 1;
+  while (ns_self < 8 && (cap + ns_self - 1) / ns_self > 256) ns_self *= 2;
+  const int ns_cross = pick_nsplit(H, ecap);
   for (int l = 0; l < mc.n_layers; ++l) {
     const bild_dec_layer& w = m.dec[l];
     const size_t kvoff = (size_t)l * H * dkv;

@@ -495,23 +495,25 @@ __device__ __forceinline__ void dattn_stage(const BAttnArgs& a, int h, int j0, i
   }
 }
 
+// grid (heads, splits); the splits of a head form one thread-block cluster, whose blocks hand
+// their partial results to the first block through distributed shared memory.
 __global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
-  extern __shared__ float s_dyn[];   // q [MB][dkv] | scores [MB][sk] | keys [sk][dkv + 4] | values [sk][dkv]
-  __shared__ float s_m[MAXB], s_l[MAXB];
-  __shared__ int s_last;
+  extern __shared__ float s_dyn[];   // q [MB][dkv] | scores [MB][sk] | keys [sk][dkv+4] | values [sk][dkv] | merge [ns][MB][dkv+2]
   const BAttnArgs& a = d.b;
   const int MB = d.MB, dshift = d.dkv_shift;
-  const int h = blockIdx.x, sp = blockIdx.y;
+  const int h = blockIdx.x, sp = blockIdx.y, ns = a.nsplit;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int dkv = a.dkv, sk = a.smem_keys, kst = dkv + 4;
+  const int dkv = a.dkv, sk = a.smem_keys, kst = dkv + 4, pst = dkv + 2;
   float* sQ = s_dyn;
   float* sS = sQ + MB * dkv;
   float* sK = sS + MB * sk;
   float* sV = sK + sk * kst;
+  float* sM = sV + sk * dkv;
+  if (ns > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   int j0 = 0, nk = 0;
   if (a.mode == 0) {   // encoder keys never change while decoding: fetch before the dependency wait
     const int n_all = min(*a.n_keys_dev, a.cap);
-    const int ch = (n_all + a.nsplit - 1) / a.nsplit;
+    const int ch = (n_all + ns - 1) / ns;
     j0 = sp * ch;
     nk = min(max(0, min(n_all, j0 + ch) - j0), sk);
     dattn_stage(a, h, j0, nk, dshift, sK, sV);
@@ -521,7 +523,7 @@ __global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
   const int M = min(a.desc->k, MB), pos0 = a.desc->pos0;
   if (a.mode == 1) {
     const int n_all = min(pos0 + M, a.cap);
-    const int ch = (n_all + a.nsplit - 1) / a.nsplit;
+    const int ch = (n_all + ns - 1) / ns;
     j0 = sp * ch;
     nk = min(max(0, min(n_all, j0 + ch) - j0), sk);
     dattn_stage(a, h, j0, nk, dshift, sK, sV);
@@ -533,8 +535,8 @@ __global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
   }
   asm volatile("cp.async.commit_group;\n\tcp.async.wait_all;" ::: "memory");
   __syncthreads();
+  if (ns > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
   // warp w owns rows w, w+4, ...: scores (lanes over keys), soft-max, values (lanes over channels)
-  float* P = a.part + (((size_t)h * a.nsplit + sp) * MB) * (dkv + 2);
 #pragma unroll 1
   for (int i = warp; i < M; i += DATT_THREADS / 32) {
     const float4* qr = reinterpret_cast<const float4*>(sQ + i * dkv);
@@ -564,44 +566,36 @@ __global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
     }
     sum = warp_sum(sum);
     __syncwarp();
-    const float rl = a.nsplit == 1 ? __frcp_rn(sum) : 1.f;
+    const float rl = ns == 1 ? __frcp_rn(sum) : 1.f;
+    float* mrow = sM + ((size_t)sp * MB + i) * pst;   // this block's slot in the first block's merge area
 #pragma unroll 1
     for (int c = lane; c < dkv; c += 32) {
       float acc = 0.f;
 #pragma unroll 4
       for (int jj = 0; jj < nk; ++jj) acc += sS[i * sk + jj] * sV[jj * dkv + c];
-      if (a.nsplit == 1) a.out[(size_t)i * a.ldo + h * dkv + c] = acc * rl;
-      else P[(size_t)i * (dkv + 2) + 2 + c] = acc;
+      if (ns == 1) a.out[(size_t)i * a.ldo + h * dkv + c] = acc * rl;
+      else st_cluster_f1(smem_u32(mrow + 2 + c), 0, acc);
     }
-    if (a.nsplit > 1 && lane == 0) { P[(size_t)i * (dkv + 2)] = mx; P[(size_t)i * (dkv + 2) + 1] = sum; }
+    if (ns > 1 && lane == 0) { st_cluster_f1(smem_u32(mrow), 0, mx); st_cluster_f1(smem_u32(mrow + 1), 0, sum); }
   }
-  if (a.nsplit == 1) return;
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned t = atomicAdd(&a.counters[h], 1u);
-    s_last = (t == (unsigned)a.nsplit - 1);
-    if (s_last) a.counters[h] = 0;
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  const float* P0 = a.part + ((size_t)h * a.nsplit * MB) * (dkv + 2);
+  if (ns == 1) return;
+  cluster_sync_all();
+  if (sp != 0) return;
 #pragma unroll 1
   for (int i = warp; i < M; i += DATT_THREADS / 32) {
     float gm = -INFINITY;
 #pragma unroll 1
-    for (int s2 = 0; s2 < a.nsplit; ++s2) gm = fmaxf(gm, __ldcg(&P0[((size_t)s2 * MB + i) * (dkv + 2)]));
+    for (int s2 = 0; s2 < ns; ++s2) gm = fmaxf(gm, sM[((size_t)s2 * MB + i) * pst]);
 #pragma unroll 1
     for (int c = lane; c < dkv; c += 32) {
       float num = 0.f, den = 0.f;
 #pragma unroll 1
-      for (int s2 = 0; s2 < a.nsplit; ++s2) {   // split order
-        const float* Ps = P0 + ((size_t)s2 * MB + i) * (dkv + 2);
-        const float l = __ldcg(&Ps[1]);
-        const float w = l > 0.f ? __expf(__ldcg(&Ps[0]) - gm) : 0.f;
+      for (int s2 = 0; s2 < ns; ++s2) {   // split order
+        const float* Ps = sM + ((size_t)s2 * MB + i) * pst;
+        const float l = Ps[1];
+        const float w = l > 0.f ? __expf(Ps[0] - gm) : 0.f;
         den += l * w;
-        num += __ldcg(&Ps[2 + c]) * w;
+        num += Ps[2 + c] * w;
       }
       a.out[(size_t)i * a.ldo + h * dkv + c] = num * __frcp_rn(den);
     }
