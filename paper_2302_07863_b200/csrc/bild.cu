@@ -284,7 +284,8 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
   BAttnArgs a = a0;
   a.smem_keys = ((keys_cap + a.nsplit - 1) / a.nsplit + 3) / 4 * 4;
   const size_t smem = sizeof(float) * ((size_t)MB * a.dkv + (size_t)MB * a.smem_keys + (size_t)a.smem_keys * (2 * a.dkv + 4) +
-                                       (a.nsplit > 1 ? (size_t)a.nsplit * MB * (a.dkv + 2) : 0));
+                                       (size_t)a.nsplit * (MB == 1 ? 4 : 1) * MB * (a.dkv + 2));
+  const int threads = MB == 1 ? 128 : 256;
   if (smem > 40 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(dattn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
@@ -292,7 +293,7 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
   DAttnArgs d;
   d.b = a; d.MB = MB; d.dkv_shift = ilog2(a.dkv);
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(a.H, a.nsplit); cfg.blockDim = dim3(DATT_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+  cfg.gridDim = dim3(a.H, a.nsplit); cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
   cudaLaunchAttribute at[2];
   int na = 0;
   if (c->use_pdl) {

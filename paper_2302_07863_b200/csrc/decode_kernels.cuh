@@ -488,7 +488,7 @@ __device__ __forceinline__ void dattn_stage(const BAttnArgs& a, int h, int j0, i
   const float* Kg = a.kc + ((size_t)h * a.cap + j0) * dkv;
   const float* Vg = a.vc + ((size_t)h * a.cap + j0) * dkv;
 #pragma unroll 1
-  for (int idx = threadIdx.x; idx < (nk << q4s); idx += DATT_THREADS) {
+  for (int idx = threadIdx.x; idx < (nk << q4s); idx += blockDim.x) {
     const int jj = idx >> q4s, e4 = (idx & ((1 << q4s) - 1)) << 2;
     cp_async16(sK + jj * kst + e4, Kg + jj * dkv + e4);
     cp_async16(sV + jj * dkv + e4, Vg + jj * dkv + e4);
@@ -496,14 +496,17 @@ __device__ __forceinline__ void dattn_stage(const BAttnArgs& a, int h, int j0, i
 }
 
 // grid (heads, splits); the splits of a head form one thread-block cluster, whose blocks hand
-// their partial results to the first block through distributed shared memory.
-__global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
-  extern __shared__ float s_dyn[];   // q [MB][dkv] | scores [MB][sk] | keys [sk][dkv+4] | values [sk][dkv] | merge [ns][MB][dkv+2]
+// their partial results to the first block through distributed shared memory.  Inside a block
+// warp w owns rows w, w+nw, ...; for a single row (MB == 1) the block's warps instead share the
+// row, each taking every nw-th key and writing its own slot of the merge area.
+__global__ void __launch_bounds__(256) dattn_kernel(DAttnArgs d) {
+  extern __shared__ float s_dyn[];   // q [MB][dkv] | scores [MB][sk] | keys [sk][dkv+4] | values [sk][dkv] | merge [slots][MB][dkv+2]
   const BAttnArgs& a = d.b;
   const int MB = d.MB, dshift = d.dkv_shift;
   const int h = blockIdx.x, sp = blockIdx.y, ns = a.nsplit;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
   const int dkv = a.dkv, sk = a.smem_keys, kst = dkv + 4, pst = dkv + 2;
+  const int wsplit = MB == 1 ? nw : 1;   // warps sharing one row
   float* sQ = s_dyn;
   float* sS = sQ + MB * dkv;
   float* sK = sS + MB * sk;
@@ -520,6 +523,12 @@ __global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
   }
   pdl_launch_dependents();
   pdl_wait();
+  // all MB rows of the query buffer exist: stage them without waiting for the row count
+#pragma unroll 1
+  for (int idx = tid; idx < (MB << (dshift - 2)); idx += blockDim.x) {
+    const int i = idx >> (dshift - 2), e4 = (idx & ((dkv >> 2) - 1)) << 2;
+    cp_async16(sQ + i * dkv + e4, a.q + (size_t)i * a.ldq + h * dkv + e4);
+  }
   const int M = min(a.desc->k, MB), pos0 = a.desc->pos0;
   if (a.mode == 1) {
     const int n_all = min(pos0 + M, a.cap);
@@ -528,21 +537,18 @@ __global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
     nk = min(max(0, min(n_all, j0 + ch) - j0), sk);
     dattn_stage(a, h, j0, nk, dshift, sK, sV);
   }
-#pragma unroll 1
-  for (int idx = tid; idx < (M << (dshift - 2)); idx += DATT_THREADS) {
-    const int i = idx >> (dshift - 2), e4 = (idx & ((dkv >> 2) - 1)) << 2;
-    cp_async16(sQ + i * dkv + e4, a.q + (size_t)i * a.ldq + h * dkv + e4);
-  }
   asm volatile("cp.async.commit_group;\n\tcp.async.wait_all;" ::: "memory");
   __syncthreads();
   if (ns > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-  // warp w owns rows w, w+4, ...: scores (lanes over keys), soft-max, values (lanes over channels)
+  const int slots = ns * wsplit;
+  const int i_first = wsplit > 1 ? 0 : warp, i_step = wsplit > 1 ? 1 : nw;
+  const int k_first = wsplit > 1 ? warp : 0, k_step = wsplit;   // this warp's keys: k_first, k_first + k_step, ...
 #pragma unroll 1
-  for (int i = warp; i < M; i += DATT_THREADS / 32) {
+  for (int i = i_first; i < M; i += i_step) {
     const float4* qr = reinterpret_cast<const float4*>(sQ + i * dkv);
     float mx = -INFINITY;
 #pragma unroll 1
-    for (int jj = lane; jj < nk; jj += 32) {
+    for (int jj = k_first + lane * k_step; jj < nk; jj += 32 * k_step) {
       const float4* kr = reinterpret_cast<const float4*>(sK + jj * kst);
       float acc = 0.f;
 #pragma unroll 4
@@ -558,7 +564,7 @@ __global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
     mx = warp_max(mx);
     float sum = 0.f;
 #pragma unroll 1
-    for (int jj = lane; jj < nk; jj += 32) {
+    for (int jj = k_first + lane * k_step; jj < nk; jj += 32 * k_step) {
       const float sc = sS[i * sk + jj];
       const float pr = (sc == -INFINITY) ? 0.f : __expf(sc - mx);
       sS[i * sk + jj] = pr;
@@ -566,31 +572,42 @@ __global__ void __launch_bounds__(DATT_THREADS) dattn_kernel(DAttnArgs d) {
     }
     sum = warp_sum(sum);
     __syncwarp();
-    const float rl = ns == 1 ? __frcp_rn(sum) : 1.f;
-    float* mrow = sM + ((size_t)sp * MB + i) * pst;   // this block's slot in the first block's merge area
+    const bool direct = slots == 1;
+    const float rl = direct ? __frcp_rn(sum) : 1.f;
+    float* mrow = sM + ((size_t)(sp * wsplit + (wsplit > 1 ? warp : 0)) * MB + i) * pst;   // slot in the first block
 #pragma unroll 1
     for (int c = lane; c < dkv; c += 32) {
-      float acc = 0.f;
-#pragma unroll 4
-      for (int jj = 0; jj < nk; ++jj) acc += sS[i * sk + jj] * sV[jj * dkv + c];
-      if (ns == 1) a.out[(size_t)i * a.ldo + h * dkv + c] = acc * rl;
-      else st_cluster_f1(smem_u32(mrow + 2 + c), 0, acc);
+      float acc0 = 0.f, acc1 = 0.f;   // two chains, added in a fixed order
+      int jj = k_first;
+#pragma unroll 2
+      for (; jj + k_step < nk; jj += 2 * k_step) {
+        acc0 += sS[i * sk + jj] * sV[jj * dkv + c];
+        acc1 += sS[i * sk + jj + k_step] * sV[(jj + k_step) * dkv + c];
+      }
+      if (jj < nk) acc0 += sS[i * sk + jj] * sV[jj * dkv + c];
+      const float acc = acc0 + acc1;
+      if (direct) a.out[(size_t)i * a.ldo + h * dkv + c] = acc * rl;
+      else if (ns > 1) st_cluster_f1(smem_u32(mrow + 2 + c), 0, acc);
+      else mrow[2 + c] = acc;
     }
-    if (ns > 1 && lane == 0) { st_cluster_f1(smem_u32(mrow), 0, mx); st_cluster_f1(smem_u32(mrow + 1), 0, sum); }
+    if (!direct && lane == 0) {
+      if (ns > 1) { st_cluster_f1(smem_u32(mrow), 0, mx); st_cluster_f1(smem_u32(mrow + 1), 0, sum); }
+      else { mrow[0] = mx; mrow[1] = sum; }
+    }
   }
-  if (ns == 1) return;
-  cluster_sync_all();
+  if (slots == 1) return;
+  if (ns > 1) cluster_sync_all(); else __syncthreads();
   if (sp != 0) return;
 #pragma unroll 1
-  for (int i = warp; i < M; i += DATT_THREADS / 32) {
+  for (int i = warp; i < M; i += nw) {
     float gm = -INFINITY;
 #pragma unroll 1
-    for (int s2 = 0; s2 < ns; ++s2) gm = fmaxf(gm, sM[((size_t)s2 * MB + i) * pst]);
+    for (int s2 = 0; s2 < slots; ++s2) gm = fmaxf(gm, sM[((size_t)s2 * MB + i) * pst]);
 #pragma unroll 1
     for (int c = lane; c < dkv; c += 32) {
       float num = 0.f, den = 0.f;
 #pragma unroll 1
-      for (int s2 = 0; s2 < ns; ++s2) {   // split order
+      for (int s2 = 0; s2 < slots; ++s2) {   // slot order
         const float* Ps = sM + ((size_t)s2 * MB + i) * pst;
         const float l = Ps[1];
         const float w = l > 0.f ? __expf(Ps[0] - gm) : 0.f;
