@@ -285,7 +285,7 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
   a.smem_keys = ((keys_cap + a.nsplit - 1) / a.nsplit + 3) / 4 * 4;
   const size_t smem = sizeof(float) * ((size_t)MB * a.dkv + (size_t)MB * a.smem_keys + (size_t)a.smem_keys * (2 * a.dkv + 4) +
                                        (size_t)a.nsplit * (MB == 1 ? 4 : 1) * MB * (a.dkv + 2));
-  const int threads = MB == 1 ? 128 : 256;
+  const int threads = MB == 1 ? 32 : 256;
   if (smem > 40 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(dattn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;

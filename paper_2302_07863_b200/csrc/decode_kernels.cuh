@@ -506,7 +506,7 @@ __global__ void __launch_bounds__(256) dattn_kernel(DAttnArgs d) {
   const int h = blockIdx.x, sp = blockIdx.y, ns = a.nsplit;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
   const int dkv = a.dkv, sk = a.smem_keys, kst = dkv + 4, pst = dkv + 2;
-  const int wsplit = MB == 1 ? nw : 1;   // warps sharing one row
+  const int wsplit = 1;   // warps sharing one row (sharing did not pay: the merge grows with the slots)
   float* sQ = s_dyn;
   float* sS = sQ + MB * dkv;
   float* sK = sS + MB * sk;
@@ -542,13 +542,14 @@ __global__ void __launch_bounds__(256) dattn_kernel(DAttnArgs d) {
   if (ns > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
   const int slots = ns * wsplit;
   const int i_first = wsplit > 1 ? 0 : warp, i_step = wsplit > 1 ? 1 : nw;
-  const int k_first = wsplit > 1 ? warp : 0, k_step = wsplit;   // this warp's keys: k_first, k_first + k_step, ...
+  // this warp's keys: a contiguous range [k_lo, k_hi)
+  const int k_lo = wsplit > 1 ? (nk * warp) / nw : 0, k_hi = wsplit > 1 ? (nk * (warp + 1)) / nw : nk;
 #pragma unroll 1
   for (int i = i_first; i < M; i += i_step) {
     const float4* qr = reinterpret_cast<const float4*>(sQ + i * dkv);
     float mx = -INFINITY;
 #pragma unroll 1
-    for (int jj = k_first + lane * k_step; jj < nk; jj += 32 * k_step) {
+    for (int jj = k_lo + lane; jj < k_hi; jj += 32) {
       const float4* kr = reinterpret_cast<const float4*>(sK + jj * kst);
       float acc = 0.f;
 #pragma unroll 4
@@ -564,7 +565,7 @@ __global__ void __launch_bounds__(256) dattn_kernel(DAttnArgs d) {
     mx = warp_max(mx);
     float sum = 0.f;
 #pragma unroll 1
-    for (int jj = k_first + lane * k_step; jj < nk; jj += 32 * k_step) {
+    for (int jj = k_lo + lane; jj < k_hi; jj += 32) {
       const float sc = sS[i * sk + jj];
       const float pr = (sc == -INFINITY) ? 0.f : __expf(sc - mx);
       sS[i * sk + jj] = pr;
@@ -578,13 +579,13 @@ __global__ void __launch_bounds__(256) dattn_kernel(DAttnArgs d) {
 #pragma unroll 1
     for (int c = lane; c < dkv; c += 32) {
       float acc0 = 0.f, acc1 = 0.f;   // two chains, added in a fixed order
-      int jj = k_first;
+      int jj = k_lo;
 #pragma unroll 2
-      for (; jj + k_step < nk; jj += 2 * k_step) {
+      for (; jj + 1 < k_hi; jj += 2) {
         acc0 += sS[i * sk + jj] * sV[jj * dkv + c];
-        acc1 += sS[i * sk + jj + k_step] * sV[(jj + k_step) * dkv + c];
+        acc1 += sS[i * sk + jj + 1] * sV[(jj + 1) * dkv + c];
       }
-      if (jj < nk) acc0 += sS[i * sk + jj] * sV[jj * dkv + c];
+      if (jj < k_hi) acc0 += sS[i * sk + jj] * sV[jj * dkv + c];
       const float acc = acc0 + acc1;
       if (direct) a.out[(size_t)i * a.ldo + h * dkv + c] = acc * rl;
       else if (ns > 1) st_cluster_f1(smem_u32(mrow + 2 + c), 0, acc);
