@@ -500,6 +500,16 @@ cudaError_t launch_umma(bild_ctx* c, const LinArgs& a, const CUtensorMap& t0, co
 cudaError_t launch_dec_linear(bild_ctx* c, Model& m, int MB, const LinArgs& a, int layer, int which_map) {
   int cs, nkb;
   if (MB != 1 && c->block_simt) {
+    const int ks = gemv_ksplit(a.K);
+    if (a.K / ks <= 256) {   // compact block GEMV: one chunk per warp
+      LinArgs b = a;
+      b.ksplit = ks; b.kl = a.K / ks; b.inv_k = 1.f / (float)a.K; b.groups = 1; b.dkv_shift = ilog2(std::max(1, a.dkv));
+      dim3 grid((a.N + 1) / 2), block(32 * ks);
+      const bool gated = a.epi == EPI_GATED;
+      if (c->cfg.dtype == BILD_BF16)
+        return gated ? launch_k(c, gemvb_kernel<__nv_bfloat16, true>, grid, block, 0, b) : launch_k(c, gemvb_kernel<__nv_bfloat16, false>, grid, block, 0, b);
+      return gated ? launch_k(c, gemvb_kernel<float, true>, grid, block, 0, b) : launch_k(c, gemvb_kernel<float, false>, grid, block, 0, b);
+    }
     cudaError_t e = cudaSuccess;
     if (c->cfg.dtype == BILD_BF16 ? launch_gemvk_t<__nv_bfloat16>(c, a, &e) : launch_gemvk_t<float>(c, a, &e)) return e;
   }

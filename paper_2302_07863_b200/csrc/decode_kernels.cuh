@@ -108,6 +108,99 @@ __global__ void __launch_bounds__(512) gemv_kernel(LinArgs a) {
 }
 
 // ---------------------------------------------------------------------------------
+// Block GEMV, compact: the GEMV above with a loop over the token rows of the block (steps L1,
+// L3, L4, L6, L7, L8).  The weights of the warp stay in registers (fetched before the
+// dependency wait); token rows are taken four at a time, all four loads in flight at once.
+// The first four rows are requested before the row count is known: all MAXB rows of the
+// activation buffers exist.  Requires K <= 4096 (one 256-column chunk per warp).
+// ---------------------------------------------------------------------------------
+template <typename WT, bool GATED>
+__global__ void __launch_bounds__(512) gemvb_kernel(LinArgs a) {
+  __shared__ float s_part[MAXB][16][5];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int ks = a.ksplit;                 // all warps of the block share one group of 2 rows
+  const int n0 = blockIdx.x * 2;
+  const int K = a.K, kl = a.kl, kbeg = warp * kl;
+  const int c0 = lane * 8;
+  const bool act = c0 < kl;
+  const int r0 = min(n0, a.N - 1), r1 = min(n0 + 1, a.N - 1);
+  const WT* W0 = (const WT*)a.W0 + kbeg;
+  const WT* W1 = (const WT*)a.W1 + kbeg;
+  float w00[8], w01[8], w10[8], w11[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { w00[i] = w01[i] = 0.f; if (GATED) w10[i] = w11[i] = 0.f; }
+  if (act) {
+    load8(W0 + (size_t)r0 * K + c0, w00);
+    load8(W0 + (size_t)r1 * K + c0, w01);
+    if (GATED) { load8(W1 + (size_t)r0 * K + c0, w10); load8(W1 + (size_t)r1 * K + c0, w11); }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  const int out_m = threadIdx.x >> 1, out_r = threadIdx.x & 1;   // writer threads: tid < 2 * M
+  float old = 0.f;
+  if (threadIdx.x < 2 * MAXB && a.epi == EPI_RESID && n0 + out_r < a.N) old = a.Y[(size_t)out_m * a.ldy + n0 + out_r];
+  float g[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) g[i] = 1.f;
+  if (a.gain && act) {
+    const float4 g0 = *reinterpret_cast<const float4*>(a.gain + kbeg + c0);
+    const float4 g1 = *reinterpret_cast<const float4*>(a.gain + kbeg + c0 + 4);
+    g[0] = g0.x; g[1] = g0.y; g[2] = g0.z; g[3] = g0.w; g[4] = g1.x; g[5] = g1.y; g[6] = g1.z; g[7] = g1.w;
+  }
+  const float* X = a.X + kbeg + c0;
+  int M = 4;   // rows 0..3 first; the true count arrives with them
+#pragma unroll 1
+  for (int m0 = 0; m0 < M; m0 += 4) {
+    float4 xa[4], xb[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      xa[t] = xb[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (act) {
+        xa[t] = *reinterpret_cast<const float4*>(X + (size_t)(m0 + t) * a.ldx);
+        xb[t] = *reinterpret_cast<const float4*>(X + (size_t)(m0 + t) * a.ldx + 4);
+      }
+    }
+    if (m0 == 0) M = min(a.desc ? a.desc->k : a.M, MAXB);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      float h[8] = {xa[t].x, xa[t].y, xa[t].z, xa[t].w, xb[t].x, xb[t].y, xb[t].z, xb[t].w};
+      float a00 = 0.f, a01 = 0.f, a10 = 0.f, a11 = 0.f, ss = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        ss += h[i] * h[i];
+        h[i] *= g[i];
+        a00 += w00[i] * h[i];
+        a01 += w01[i] * h[i];
+        if (GATED) { a10 += w10[i] * h[i]; a11 += w11[i] * h[i]; }
+      }
+      a00 = warp_sum(a00); a01 = warp_sum(a01); ss = warp_sum(ss);
+      if (GATED) { a10 = warp_sum(a10); a11 = warp_sum(a11); }
+      if (lane == 0) {
+        float* sp = s_part[m0 + t][warp];
+        sp[0] = a00; sp[1] = a01; sp[2] = a10; sp[3] = a11; sp[4] = ss;
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x >= 2 * M) return;
+  const int n = n0 + out_r;
+  if (n >= a.N) return;
+  float v0 = 0.f, v1 = 0.f, sq = 0.f;
+#pragma unroll 1
+  for (int w2 = 0; w2 < ks; ++w2) {   // fixed order
+    const float* sp = s_part[out_m][w2];
+    v0 += sp[out_r]; v1 += sp[2 + out_r]; sq += sp[4];
+  }
+  const float inv = a.gain ? rsqrtf(sq * a.inv_k + a.eps) : 1.f;
+  v0 *= inv;
+  if (a.epi == EPI_RESID) a.Y[(size_t)out_m * a.ldy + n] = old + v0;
+  else if (a.epi == EPI_STORE) a.Y[(size_t)out_m * a.ldy + n] = v0;
+  else if (a.epi == EPI_RELU) a.Y[(size_t)out_m * a.ldy + n] = fmaxf(v0, 0.f);
+  else if (a.epi == EPI_GATED) { if (GATED) a.Y[(size_t)out_m * a.ldy + n] = gelu_tanh(v0) * (v1 * inv); }
+  else heads_store(a, n, out_m, a.desc ? a.desc->pos0 : a.pos0_host, v0);
+}
+
+// ---------------------------------------------------------------------------------
 // The same GEMV for a block of up to MAXB token rows (steps L1, L3, L4, L6, L7, L8 when the
 // block pass is latency-bound): one block owns RW weight rows, its warps split K so that each
 // warp's weights (<= GEMV_PRE chunks of 256 columns) sit in registers before the dependency

@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
   unsigned char* sB = sA + (size_t)NST * NMAT * 16384;           // [nkb][hi 2 KB | lo 2 KB]
   float* sRed = (float*)(sB + (size_t)nkb * 4096);               // [cs-1][NMAT][128][16]
   float* sSS = sRed + (size_t)(cs > 1 ? cs - 1 : 0) * NMAT * UM_TILE_M * 16;   // [8][16]
-  uint64_t* full = (uint64_t*)(sSS + 8 * 16);
+  uint64_t* full = (uint64_t*)(sSS + 9 * 16);   // [8][16] sums of squares per rank, [16] 1/rms
   uint64_t* empty = full + NST;
   uint64_t* done = empty + NST;
   uint32_t* tmem_slot = (uint32_t*)(done + 1);
@@ -166,44 +166,56 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
     for (int m = 0; m < MAXB; ++m) old[m] = a.Y[(size_t)m * a.ldy + n_base + tid];
   }
   const int kl = nkb * UM_KB;
-  {  // warp w owns rows w, w+4, w+8, w+12; the loads of all four rows are issued together
+  {  // warp w owns rows w, w+4, w+8, w+12.  Two column chunks (2 x 256) of all four rows are
+     // requested before any of them is converted, so a block with up to 512 columns needs one
+     // round trip to L2 for its activations.
     float ssr[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int c = lane * 8; c < kl; c += 256) {
-      float4 g0 = make_float4(1.f, 1.f, 1.f, 1.f), g1 = g0;
-      if (a.gain) {
-        g0 = *reinterpret_cast<const float4*>(a.gain + k_base + c);
-        g1 = *reinterpret_cast<const float4*>(a.gain + k_base + c + 4);
-      }
-      float4 xa[4], xb[4];
+#pragma unroll 1
+    for (int cb = lane * 8; cb < kl; cb += 512) {
+      float4 xa[2][4], xb[2][4], g0[2], g1[2];
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        const int m = warp + 4 * r;
-        const float* xp = a.X + (size_t)m * a.ldx + k_base + c;
-        xa[r] = *reinterpret_cast<const float4*>(xp);
-        xb[r] = *reinterpret_cast<const float4*>(xp + 4);
-      }
-      const int kb = c / UM_KB, chunk = (c % UM_KB) / 8;
+      for (int j = 0; j < 2; ++j) {
+        const int c = cb + 256 * j;
+        g0[j] = g1[j] = make_float4(1.f, 1.f, 1.f, 1.f);
+        if (c < kl) {
+          if (a.gain) {
+            g0[j] = *reinterpret_cast<const float4*>(a.gain + k_base + c);
+            g1[j] = *reinterpret_cast<const float4*>(a.gain + k_base + c + 4);
+          }
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        const int m = warp + 4 * r;
-        float h[8] = {xa[r].x, xa[r].y, xa[r].z, xa[r].w, xb[r].x, xb[r].y, xb[r].z, xb[r].w};
-        if (a.gain) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) ssr[r] += h[i] * h[i];
-          h[0] *= g0.x; h[1] *= g0.y; h[2] *= g0.z; h[3] *= g0.w; h[4] *= g1.x; h[5] *= g1.y; h[6] *= g1.z; h[7] *= g1.w;
+          for (int r = 0; r < 4; ++r) {
+            const float* xp = a.X + (size_t)(warp + 4 * r) * a.ldx + k_base + c;
+            xa[j][r] = *reinterpret_cast<const float4*>(xp);
+            xb[j][r] = *reinterpret_cast<const float4*>(xp + 4);
+          }
         }
-        uint32_t hi[4], lo[4];
+      }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const __nv_bfloat16 h0 = __float2bfloat16_rn(h[2 * i]), h1 = __float2bfloat16_rn(h[2 * i + 1]);
-          const __nv_bfloat16 l0 = __float2bfloat16_rn(h[2 * i] - __bfloat162float(h0));
-          const __nv_bfloat16 l1 = __float2bfloat16_rn(h[2 * i + 1] - __bfloat162float(h1));
-          hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-          lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+      for (int j = 0; j < 2; ++j) {
+        const int c = cb + 256 * j;
+        if (c < kl) {
+          const int kb = c / UM_KB, chunk = (c % UM_KB) / 8;
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            const int m = warp + 4 * r;
+            float h[8] = {xa[j][r].x, xa[j][r].y, xa[j][r].z, xa[j][r].w, xb[j][r].x, xb[j][r].y, xb[j][r].z, xb[j][r].w};
+            const float gg[8] = {g0[j].x, g0[j].y, g0[j].z, g0[j].w, g1[j].x, g1[j].y, g1[j].z, g1[j].w};
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              ssr[r] += h[2 * i] * h[2 * i] + h[2 * i + 1] * h[2 * i + 1];
+              const float e0 = h[2 * i] * gg[2 * i], e1 = h[2 * i + 1] * gg[2 * i + 1];
+              const __nv_bfloat16 h0 = __float2bfloat16_rn(e0), h1 = __float2bfloat16_rn(e1);
+              const __nv_bfloat16 l0 = __float2bfloat16_rn(e0 - __bfloat162float(h0));
+              const __nv_bfloat16 l1 = __float2bfloat16_rn(e1 - __bfloat162float(h1));
+              hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+              lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+            }
+            const uint32_t off = (uint32_t)kb * 4096 + (m >> 3) * 1024 + (m & 7) * 128 + ((chunk ^ (m & 7)) << 4);
+            *reinterpret_cast<uint4*>(sB + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(sB + off + 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          }
         }
-        const uint32_t off = (uint32_t)kb * 4096 + (m >> 3) * 1024 + (m & 7) * 128 + ((chunk ^ (m & 7)) << 4);
-        *reinterpret_cast<uint4*>(sB + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(sB + off + 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
     }
 #pragma unroll
@@ -292,45 +304,47 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
         for (int i = 0; i < 16; ++i) acc1[i] += src[(16 + i) * UM_TILE_M];
       }
     }
+    // 1 / rms per token row: threads 0..15 add the ranks' sums of squares in rank order
+    if (tid < MAXB) {
+      float ss = 0.f;
+      for (int r = 0; r < cs; ++r) ss += sSS[r * 16 + tid];
+      sSS[8 * 16 + tid] = a.gain ? rsqrtf(ss / (float)a.K + a.eps) : 1.f;
+    }
+    __syncthreads();
+  }
+  if (rank == 0) {
     const int n = n_base + tid;
     const int mrows = min(MAXB, M);
+    const float* sInv = sSS + 8 * 16;
     if (n < a.N) {
-      float v0[MAXB], v1[MAXB];
-#pragma unroll
-      for (int m = 0; m < MAXB; ++m) {
-        float inv = 1.f;
-        if (a.gain && m < mrows) {
-          float ss = 0.f;
-          for (int r = 0; r < cs; ++r) ss += sSS[r * 16 + m];
-          inv = 1.f / sqrtf(ss / (float)a.K + a.eps);
-        }
-        v0[m] = acc0[m] * inv;
-        v1[m] = GATED ? acc1[m] * inv : 0.f;
-      }
       if (a.epi == EPI_RESID) {   // the old values were requested right after the dependency wait
 #pragma unroll
         for (int m = 0; m < MAXB; ++m)
-          if (m < mrows) a.Y[(size_t)m * a.ldy + n] = old[m] + v0[m];
+          if (m < mrows) a.Y[(size_t)m * a.ldy + n] = old[m] + acc0[m] * sInv[m];
       } else if (a.epi == EPI_HEADS) {
-        const int part = a.first_part + n / a.inner;
-        const int rr = n % a.inner;
+        int part = a.first_part, rr = n;
+        if (rr >= a.inner) { rr -= a.inner; ++part; }
+        if (rr >= a.inner) { rr -= a.inner; ++part; }
         const int h = rr / a.dkv, c = rr % a.dkv;
 #pragma unroll
         for (int m = 0; m < MAXB; ++m) {
           if (m < mrows) {
-            if (part == 0) a.q_out[(size_t)m * a.ldq + rr] = v0[m];
-            else if (pos0 + m < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + pos0 + m) * a.dkv + c] = v0[m];
+            const float v = acc0[m] * sInv[m];
+            if (part == 0) a.q_out[(size_t)m * a.ldq + rr] = v;
+            else if (pos0 + m < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)h * a.cap + pos0 + m) * a.dkv + c] = v;
           }
         }
       } else {
+#pragma unroll 1
+        for (int m = 0; m < mrows; ++m) {
+          // registers cannot be indexed in a rolled loop: pick the row's values with selects
+          float y = 0.f, y1 = 0.f;
 #pragma unroll
-        for (int m = 0; m < MAXB; ++m) {
-          if (m < mrows) {
-            float y = v0[m];
-            if (a.epi == EPI_RELU) y = fmaxf(y, 0.f);
-            else if (a.epi == EPI_GATED) y = gelu_tanh(y) * v1[m];
-            a.Y[(size_t)m * a.ldy + n] = y;
-          }
+          for (int q = 0; q < MAXB; ++q) { if (q == m) { y = acc0[q]; if (GATED) y1 = acc1[q]; } }
+          y *= sInv[m];
+          if (a.epi == EPI_RELU) y = fmaxf(y, 0.f);
+          else if (a.epi == EPI_GATED) { if (GATED) y = gelu_tanh(y) * (y1 * sInv[m]); }
+          a.Y[(size_t)m * a.ldy + n] = y;
         }
       }
     }
