@@ -218,12 +218,13 @@ void plan(bild_ctx* c, Bump& b) {
     m.head_out = b.take<HeadOut>(1);
     m.desc = b.take<CallDesc>(1);
   }
-  c->ex = b.take<float>((size_t)ecap * dmax);
-  c->eq = b.take<float>((size_t)ecap * imax);
+  const size_t ecap16 = (size_t)(ecap + MAXB - 1) / MAXB * MAXB;   // whole blocks of MAXB rows
+  c->ex = b.take<float>(ecap16 * dmax);
+  c->eq = b.take<float>(ecap16 * imax);
   c->ek = b.take<float>((size_t)ecap * imax);
   c->ev = b.take<float>((size_t)ecap * imax);
-  c->eatt = b.take<float>((size_t)ecap * imax);
-  c->eu = b.take<float>((size_t)ecap * fmax);
+  c->eatt = b.take<float>(ecap16 * imax);
+  c->eu = b.take<float>(ecap16 * fmax);
   b.off = align_up(b.off, 256);
 }
 
@@ -412,7 +413,7 @@ bool make_tmap(EncodeTiledFn enc, const void* W, int N, int K, CUtensorMap* out)
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-enum { TM_QKV = 0, TM_O, TM_CQ, TM_CO, TM_WI0, TM_WI1, TM_FO, TM_PER_LAYER };
+enum { TM_QKV = 0, TM_O, TM_CQ, TM_CO, TM_WI0, TM_WI1, TM_FO, TM_CKV, TM_EQKV, TM_EO, TM_EWI0, TM_EWI1, TM_EFO, TM_PER_LAYER };
 
 // Builds the descriptors of one model; leaves m.umma false when the shapes do not fit the kernel.
 void setup_umma(bild_ctx* c, Model& m) {
@@ -440,7 +441,14 @@ void setup_umma(bild_ctx* c, Model& m) {
               make_tmap(enc, w.wco, mc.d_model, m.inner, &t[TM_CO]) &&
               make_tmap(enc, w.wi0, mc.d_ff, mc.d_model, &t[TM_WI0]) &&
               make_tmap(enc, gated ? w.wi1 : w.wi0, mc.d_ff, mc.d_model, &t[TM_WI1]) &&
-              make_tmap(enc, w.wfo, mc.d_model, mc.d_ff, &t[TM_FO]);
+              make_tmap(enc, w.wfo, mc.d_model, mc.d_ff, &t[TM_FO]) &&
+              make_tmap(enc, w.wckv, 2 * m.inner, mc.d_model, &t[TM_CKV]);
+    const bild_enc_layer& e = m.enc[l];
+    ok = ok && make_tmap(enc, e.wqkv, 3 * m.inner, mc.d_model, &t[TM_EQKV]) &&
+         make_tmap(enc, e.wo, mc.d_model, m.inner, &t[TM_EO]) &&
+         make_tmap(enc, e.wi0, mc.d_ff, mc.d_model, &t[TM_EWI0]) &&
+         make_tmap(enc, gated ? e.wi1 : e.wi0, mc.d_ff, mc.d_model, &t[TM_EWI1]) &&
+         make_tmap(enc, e.wfo, mc.d_model, mc.d_ff, &t[TM_EFO]);
     if (!ok) { m.tmaps.clear(); return; }
   }
   const int maxsm = 227 * 1024;
@@ -470,13 +478,14 @@ bool umma_plan(int N, int K, bool gated, int* cs_out, int* nkb_out) {
   return true;
 }
 
-cudaError_t launch_umma(bild_ctx* c, const LinArgs& a, const CUtensorMap& t0, const CUtensorMap& t1, int cs, int nkb) {
+cudaError_t launch_umma(bild_ctx* c, const LinArgs& a, const CUtensorMap& t0, const CUtensorMap& t1, int cs, int nkb,
+                        int row_blocks = 1) {
   const bool gated = a.epi == EPI_GATED;
   UmmaArgs u;
   u.lin = a; u.cs = cs; u.nkb = nkb; u.err = &c->st->err;
   const int tiles = (a.N + UM_TILE_M - 1) / UM_TILE_M;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(tiles * cs); cfg.blockDim = dim3(UM_THREADS);
+  cfg.gridDim = dim3(tiles * cs, row_blocks); cfg.blockDim = dim3(UM_THREADS);
   cfg.dynamicSmemBytes = umma_smem_bytes(gated, nkb, cs); cfg.stream = c->stream;
   cudaLaunchAttribute at[2];
   int na = 0;
@@ -518,6 +527,16 @@ cudaError_t launch_dec_linear(bild_ctx* c, Model& m, int MB, const LinArgs& a, i
     return launch_umma(c, a, t[which_map], t[which_map == TM_WI0 ? TM_WI1 : which_map], cs, nkb);
   }
   return launch_linear(c, c->cfg.dtype, MB, a);
+}
+
+// Linear layer of the encoder over rb blocks of MAXB rows.
+cudaError_t launch_enc_linear(bild_ctx* c, Model& m, const LinArgs& a, int rb, int layer, int which_map) {
+  int cs, nkb;
+  if (m.umma && umma_plan(a.N, a.K, a.epi == EPI_GATED, &cs, &nkb)) {
+    const CUtensorMap* t = &m.tmaps[(size_t)layer * TM_PER_LAYER];
+    return launch_umma(c, a, t[which_map], t[which_map == TM_EWI0 ? TM_EWI1 : which_map], cs, nkb, rb);
+  }
+  return launch_linear(c, c->cfg.dtype, MAXB, a, rb);
 }
 
 LoopPtrs loop_ptrs(bild_ctx* c) {
@@ -613,7 +632,7 @@ int encoder_pass(bild_ctx* c, int which) {
     a.M = E; a.eps = mc.ln_eps; a.W0 = w.wqkv; a.X = c->ex; a.ldx = d; a.gain = (const float*)w.ln1;
     a.N = 3 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 0; a.q_out = c->eq; a.ldq = I;
     a.kc = c->ek; a.vc = c->ev; a.cap = ecap; a.pos0_host = 0;
-    CUDA_TRY(c, launch_linear(c, dt, MAXB, a, rb));
+    CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_EQKV));
     BAttnArgs t{};
     t.q = c->eq; t.ldq = I; t.kc = c->ek; t.vc = c->ev; t.cap = ecap; t.out = c->eatt; t.ldo = I;
     t.bias = m.enc_bias; t.bias_ld = 2 * ecap - 1; t.bias_off = ecap - 1; t.mode = 2; t.dkv = dkv; t.H = H;
@@ -622,15 +641,15 @@ int encoder_pass(bild_ctx* c, int which) {
     CUDA_TRY(c, launch_battn(c, MAXB, t, rb, ecap));
     LinArgs o{};
     o.M = E; o.W0 = w.wo; o.X = c->eatt; o.ldx = I; o.N = d; o.K = I; o.epi = EPI_RESID; o.Y = c->ex; o.ldy = d;
-    CUDA_TRY(c, launch_linear(c, dt, MAXB, o, rb));
+    CUDA_TRY(c, launch_enc_linear(c, m, o, rb, l, TM_EO));
     LinArgs up{};
     up.M = E; up.eps = mc.ln_eps; up.W0 = w.wi0; up.W1 = w.wi1; up.X = c->ex; up.ldx = d; up.gain = (const float*)w.ln2;
     up.N = F; up.K = d; up.Y = c->eu; up.ldy = F;
     up.epi = mc.ffn_kind == BILD_FFN_GATED_GELU ? EPI_GATED : EPI_RELU;
-    CUDA_TRY(c, launch_linear(c, dt, MAXB, up, rb));
+    CUDA_TRY(c, launch_enc_linear(c, m, up, rb, l, TM_EWI0));
     LinArgs dn{};
     dn.M = E; dn.W0 = w.wfo; dn.X = c->eu; dn.ldx = F; dn.N = d; dn.K = F; dn.epi = EPI_RESID; dn.Y = c->ex; dn.ldy = d;
-    CUDA_TRY(c, launch_linear(c, dt, MAXB, dn, rb));
+    CUDA_TRY(c, launch_enc_linear(c, m, dn, rb, l, TM_EFO));
   }
   // encoder memory = final norm of ex (fused into the projections); cross K/V per decoder layer
   for (int l = 0; l < mc.n_layers; ++l) {
@@ -639,7 +658,7 @@ int encoder_pass(bild_ctx* c, int which) {
     a.M = E; a.eps = mc.ln_eps; a.W0 = m.dec[l].wckv; a.X = c->ex; a.ldx = d; a.gain = (const float*)m.w.enc_final_ln;
     a.N = 2 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 1;
     a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.pos0_host = 0;
-    CUDA_TRY(c, launch_linear(c, dt, MAXB, a, rb));
+    CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_CKV));
   }
   return BILD_OK;
 }
@@ -852,7 +871,7 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
     }
     m.w.enc_layers = nullptr;
     m.w.dec_layers = nullptr;
-    if (i == 1) setup_umma(c, m);
+    setup_umma(c, m);
   }
   if (cudaMallocHost((void**)&c->pin_state, sizeof(DevState)) != cudaSuccess ||
       cudaMallocHost((void**)&c->pin_head, sizeof(HeadOut)) != cudaSuccess) {

@@ -108,7 +108,14 @@ __global__ void __launch_bounds__(UM_THREADS) umma_linear_kernel(UmmaArgs u, con
   constexpr int NMAT = GATED ? 2 : 1;
   constexpr int TCOLS = 32 * NMAT;   // accumulator columns in tensor memory: [hi 16 | lo 16] per matrix
   extern __shared__ unsigned char um_raw[];
-  const LinArgs& a = u.lin;
+  // blockIdx.y selects a block of MAXB token rows (encoder: many blocks; decoder passes: one)
+  LinArgs a = u.lin;
+  const int row0 = blockIdx.y * MAXB;
+  a.X += (size_t)row0 * a.ldx;
+  if (a.Y) a.Y += (size_t)row0 * a.ldy;
+  if (a.q_out) a.q_out += (size_t)row0 * a.ldq;
+  a.pos0_host += row0;
+  a.M -= row0;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int cs = u.cs, nkb = u.nkb;
   const uint32_t rank = cs > 1 ? cluster_rank() : 0;
