@@ -214,10 +214,11 @@ def main():
         res["r"] = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
 
     sampler = ClockSampler(local) if rank == 0 else None
+    ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
     l0 = ctx.launch_count()
     ms = run(step_resident, a.steps, a.warmup)
-    launches = (ctx.launch_count() - l0) * a.steps // (a.steps + a.warmup)
     r = ctx.fetch_result(wl.gen_len)
+    launches = (ctx.launch_count() - l0) * a.steps // (a.steps + a.warmup)
     ntok = len(r["tokens"])
     ms_e2e = run(step_e2e, max(2, a.steps // 4), 1)
     e2e_steps = max(2, a.steps // 4)

@@ -136,7 +136,7 @@ struct bild_ctx {
   bool block_simt = false;           // block pass on the SIMT block GEMV instead of the tensor-core kernel
   bool use_pdl = true;               // launch pass kernels with programmatic stream serialization
   bool host_loop = false;            // debug: drive the loop from the host, one read-back per step
-  int graph_run_mode = -1;           // mode of a graph run whose launches are not yet counted
+  int64_t graph_counted = 0;         // launches of the loop graphs already added to `launches`
 };
 
 namespace {
@@ -180,6 +180,8 @@ int check_config(const bild_config* cfg, std::string& why) {
 }
 
 int head_grid_for(int V) { return std::max(1, std::min(HEAD_GRID_MAX, (V + 63) / 64)); }
+// partial records either head kernel may write (block head: grid x MAXB; single-row head: up to V / 8 blocks)
+size_t head_partial_count(int V) { return std::max((size_t)head_grid_for(V) * MAXB, (size_t)(V + 7) / 8 + 8); }
 
 // Lays out everything the context keeps on the device.
 void plan(bild_ctx* c, Bump& b) {
@@ -213,7 +215,7 @@ void plan(bild_ctx* c, Bump& b) {
     m.att_part = b.take<float>((size_t)MAXB * mc.n_heads * NSPLIT_MAX * (mc.d_kv + 2));
     m.att_cnt = b.take<unsigned>((size_t)MAXB * mc.n_heads);
     m.head_grid = head_grid_for(mc.vocab);
-    m.head_part = b.take<Partial>((size_t)m.head_grid * MAXB);
+    m.head_part = b.take<Partial>(head_partial_count(mc.vocab));
     m.head_cnt = b.take<unsigned>(1);
     m.head_out = b.take<HeadOut>(1);
     m.desc = b.take<CallDesc>(1);
@@ -372,9 +374,32 @@ cudaError_t launch_head_t(bild_ctx* c, const HeadArgs& a, int grid, int64_t* lau
   return launch_k(c, kern, dim3(grid), dim3(HEAD_THREADS), smem, a);
 }
 
+template <typename WT, int NCH, int RPW>
+cudaError_t launch_head1_t(bild_ctx* c, const HeadArgs& a, int64_t* launches) {
+  const int rows = (HEAD1_THREADS / 32) * RPW;
+  if (launches) (*launches)++;
+  return launch_k(c, head1_kernel<WT, NCH, RPW>, dim3((a.V + rows - 1) / rows), dim3(HEAD1_THREADS), 0, a);
+}
+// blocks of the single-row head for a vocabulary of V rows and K columns (0: shape not covered)
+int head1_grid(int V, int K) {
+  const int nch = (K + 255) / 256;
+  const int rpw = nch <= 2 ? 4 : nch <= 4 ? 2 : nch <= 8 ? 1 : 0;
+  return rpw ? (V + 8 * rpw - 1) / (8 * rpw) : 0;
+}
+template <typename WT>
+cudaError_t launch_head1(bild_ctx* c, const HeadArgs& a, int64_t* launches) {
+  const int nch = (a.K + 255) / 256;
+  if (nch <= 1) return launch_head1_t<WT, 1, 4>(c, a, launches);
+  if (nch <= 2) return launch_head1_t<WT, 2, 4>(c, a, launches);
+  if (nch <= 4) return launch_head1_t<WT, 4, 2>(c, a, launches);
+  return launch_head1_t<WT, 8, 1>(c, a, launches);
+}
+
 cudaError_t launch_head(cudaStream_t s, int dtype, int MB, const HeadArgs& a, int grid, int64_t* launches) {
   bild_ctx tmp;
   tmp.stream = s;
+  if (MB == 1 && head1_grid(a.V, a.K) > 0)
+    return dtype == BILD_BF16 ? launch_head1<__nv_bfloat16>(&tmp, a, launches) : launch_head1<float>(&tmp, a, launches);
   if (dtype == BILD_BF16)
     return MB == 1 ? launch_head_t<__nv_bfloat16, 1, 4>(&tmp, a, grid, launches) : launch_head_t<__nv_bfloat16, MAXB, 2>(&tmp, a, grid, launches);
   return MB == 1 ? launch_head_t<float, 1, 4>(&tmp, a, grid, launches) : launch_head_t<float, MAXB, 2>(&tmp, a, grid, launches);
@@ -787,12 +812,11 @@ int build_graphs_once(bild_ctx* c) {
 int read_state(bild_ctx* c) {
   CUDA_TRY(c, cudaMemcpyAsync(c->pin_state, c->st, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-  if (c->graph_run_mode >= 0) {  // a finished graph run: count the kernels it launched
-    const bild_stats& t = c->pin_state->stats;
-    c->launches += c->graph_run_mode == BILD_MODE_LARGE_ONLY
-                       ? t.large_calls * c->per_pass_large1
-                       : t.small_steps * c->per_pass[0] + t.large_calls * c->per_pass[1];
-    c->graph_run_mode = -1;
+  {  // kernels launched by the loop graphs so far (the device counts the passes they ran)
+    const long long* cp = c->pin_state->cum_passes;
+    const int64_t total = cp[0] * c->per_pass[0] + cp[1] * c->per_pass[1] + cp[2] * c->per_pass_large1;
+    c->launches += total - c->graph_counted;
+    c->graph_counted = total;
   }
   if (c->pin_state->err) return fail(c, c->pin_state->err, "device-side error flag set");
   return BILD_OK;
@@ -1005,7 +1029,6 @@ int bild_generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, i
     if (rc) return rc;
     if (max_len == 0 || c->cfg.start_id == c->cfg.eos_id) return BILD_OK;
     CUDA_TRY(c, cudaGraphLaunch(c->exec[mode == BILD_MODE_LARGE_ONLY ? 1 : 0], c->stream));
-    c->graph_run_mode = mode;
     return BILD_OK;
   }
   int rc = reset_state(c, mode, alpha_fb, alpha_rb, max_len);
@@ -1070,7 +1093,7 @@ int bild_op_linear(const void* W, int w_dtype, const float* X, const float* gain
 
 size_t bild_op_lm_head_scratch_bytes(int V) {
   if (V < 1) return 0;
-  return align_up((size_t)head_grid_for(V) * MAXB * sizeof(Partial), 256) + 256 + align_up(sizeof(HeadOut), 256);
+  return align_up(head_partial_count(V) * sizeof(Partial), 256) + 256 + align_up(sizeof(HeadOut), 256);
 }
 
 int bild_op_lm_head(const void* W, int w_dtype, const float* X, const float* gain, float eps, float scale,
@@ -1085,7 +1108,7 @@ int bild_op_lm_head(const void* W, int w_dtype, const float* X, const float* gai
   char* p = (char*)scratch;
   HeadArgs h{};
   h.partials = (Partial*)p;
-  p += align_up((size_t)grid * MAXB * sizeof(Partial), 256);
+  p += align_up(head_partial_count(V) * sizeof(Partial), 256);
   h.counter = (unsigned*)p;
   p += 256;
   h.out = (HeadOut*)p;

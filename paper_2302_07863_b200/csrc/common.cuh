@@ -50,6 +50,8 @@ struct DevState {
   int n_trace, trace_cap;
   bild_stats stats;
   int passes;   // decoder passes taken by the running loop (guards against a runaway loop)
+  int pad0;
+  long long cum_passes[3];   // passes run from the loop graphs since create: small, large block, large single row
 };
 
 struct Partial {  // running soft-max statistics of a slice of the vocabulary

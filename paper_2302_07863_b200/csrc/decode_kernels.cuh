@@ -562,6 +562,135 @@ __global__ void __launch_bounds__(BATT_THREADS) battn_kernel(BAttnArgs a) {
 }
 
 // ---------------------------------------------------------------------------------
+// LM head for one row (steps S9 + S10, and the large model at k = 1): a GEMV over the
+// vocabulary fused with the online max / arg-max / sum-exp.  Every warp owns RPW consecutive
+// vocabulary rows whose weights are all requested before the dependency wait (the head is
+// the largest matrix of the step, so its load overlaps the last layers of the pass).  The
+// block writes one partial; the block with the last ticket merges all partials (each thread
+// loads its share at once, then a fixed-order tree) and runs the policy code.
+// ---------------------------------------------------------------------------------
+constexpr int HEAD1_THREADS = 256;
+
+template <typename WT, int NCH, int RPW>   // NCH chunks of 256 columns per row, RPW rows per warp
+__global__ void __launch_bounds__(HEAD1_THREADS) head1_kernel(HeadArgs a) {
+  constexpr int NW = HEAD1_THREADS / 32;
+  __shared__ Partial s_p[HEAD1_THREADS];
+  __shared__ int s_last;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int K = a.K, V = a.V;
+  const int n0 = (blockIdx.x * NW + warp) * RPW;
+  const WT* W = (const WT*)a.W;
+  float w[RPW][NCH][8];
+#pragma unroll
+  for (int r = 0; r < RPW; ++r)
+#pragma unroll
+    for (int p = 0; p < NCH; ++p) {
+      const int c = p * 256 + lane * 8;
+      if (c < K) load8(W + (size_t)min(n0 + r, V - 1) * K + c, w[r][p]);
+    }
+  pdl_launch_dependents();
+  pdl_wait();
+  const int target = a.desc ? a.desc->targets[0] : (a.target ? a.target[0] : -1);
+  float acc[RPW], ss = 0.f;
+#pragma unroll
+  for (int r = 0; r < RPW; ++r) acc[r] = 0.f;
+#pragma unroll
+  for (int p = 0; p < NCH; ++p) {
+    const int c = p * 256 + lane * 8;
+    if (c < K) {
+      const float4 x0 = *reinterpret_cast<const float4*>(a.X + c), x1 = *reinterpret_cast<const float4*>(a.X + c + 4);
+      float h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+      if (a.gain) {
+        const float4 g0 = *reinterpret_cast<const float4*>(a.gain + c), g1 = *reinterpret_cast<const float4*>(a.gain + c + 4);
+        const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { ss += h[i] * h[i]; h[i] *= g[i]; }
+      }
+#pragma unroll
+      for (int r = 0; r < RPW; ++r)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[r] += w[r][p][i] * h[i];
+    }
+  }
+  ss = warp_sum(ss);
+  const float mul = (a.gain ? rsqrtf(ss / (float)K + a.eps) : 1.f) * a.scale;
+  Partial run;
+  run.m = -INFINITY; run.s = 0.f; run.idx = 0x7fffffff;
+#pragma unroll
+  for (int r = 0; r < RPW; ++r) {
+    const float z = warp_sum(acc[r]) * mul;
+    const int n = n0 + r;
+    if (n < V) {
+      if (z > run.m) { run.s = run.s * __expf(run.m - z) + 1.f; run.m = z; run.idx = n; }
+      else run.s += __expf(z - run.m);
+      if (lane == 0) {
+        if (n == target) a.out->gather[0] = z;
+        if (a.logits_dbg) a.logits_dbg[n] = z;
+      }
+    }
+  }
+  if (lane == 0) s_p[warp] = run;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    Partial p = s_p[0];
+    for (int w2 = 1; w2 < NW; ++w2) p = combine(p, s_p[w2]);
+    a.partials[blockIdx.x] = p;
+    __threadfence();
+    const unsigned t = atomicAdd(a.counter, 1u);
+    s_last = (t == gridDim.x - 1);
+    if (s_last) *a.counter = 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // merge: every thread requests its partials together, then combines them in index order
+  {
+    Partial q[8];
+    const int nb = (int)gridDim.x;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int b = threadIdx.x + j * HEAD1_THREADS;
+      q[j].m = -INFINITY; q[j].s = 0.f; q[j].idx = 0x7fffffff;
+      if (b < nb) { q[j].m = __ldcg(&a.partials[b].m); q[j].s = __ldcg(&a.partials[b].s); q[j].idx = __ldcg(&a.partials[b].idx); }
+    }
+    Partial p = q[0];
+#pragma unroll
+    for (int j = 1; j < 8; ++j) p = combine(p, q[j]);
+    for (int b = threadIdx.x + 8 * HEAD1_THREADS; b < nb; b += HEAD1_THREADS) {   // very large vocabularies
+      Partial t2;
+      t2.m = __ldcg(&a.partials[b].m); t2.s = __ldcg(&a.partials[b].s); t2.idx = __ldcg(&a.partials[b].idx);
+      p = combine(p, t2);
+    }
+    s_p[threadIdx.x] = p;
+  }
+  __syncthreads();
+  for (int stride = HEAD1_THREADS / 2; stride > 0; stride >>= 1) {
+    if (threadIdx.x < stride) s_p[threadIdx.x] = combine(s_p[threadIdx.x], s_p[threadIdx.x + stride]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const Partial p = s_p[0];
+    HeadOut* o = a.out;
+    o->argmax[0] = p.idx;
+    o->zmax[0] = p.m;
+    o->lse[0] = p.m + logf(p.s);
+    o->pmax = 1.f / p.s;
+    o->gather[0] = __ldcg(&o->gather[0]);
+    if (a.loop.st) {
+      policy_tests(o, a.desc, a.loop.st, a.which);
+      if (a.desc->run_policy) policy_step(a.loop, o, a.desc, a.which);
+      else if (a.which == 0) a.loop.st->S_len = a.desc->pos0 + 1;
+      else a.loop.st->L_len = a.desc->pos0 + a.desc->k;
+      if (a.cond_while) {
+        a.loop.st->cum_passes[a.which == 0 ? 0 : 2]++;
+        cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
+      }
+      if (a.cond_if) cudaGraphSetConditional(a.cond_if, a.loop.st->fallback ? 1u : 0u);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------
 // Decode attention, compact version of the block attention above for the decoder passes
 // (modes 0 and 1 only).  Keys and values of the block's split are staged in shared memory
 // (cross-attention: before the dependency wait), scores are taken one (row, key) pair per

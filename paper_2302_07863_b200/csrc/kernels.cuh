@@ -617,7 +617,10 @@ __global__ void __launch_bounds__(HEAD_THREADS) lm_head_kernel(HeadArgs a) {
       if (a.desc->run_policy) policy_step(a.loop, o, a.desc, a.which);
       else if (a.which == 0) a.loop.st->S_len = a.desc->pos0 + 1;
       else a.loop.st->L_len = a.desc->pos0 + a.desc->k;
-      if (a.cond_while) cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
+      if (a.cond_while) {
+        a.loop.st->cum_passes[a.which == 0 ? 0 : (MB == 1 ? 2 : 1)]++;
+        cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
+      }
       if (a.cond_if) cudaGraphSetConditional(a.cond_if, a.loop.st->fallback ? 1u : 0u);
     }
   }
