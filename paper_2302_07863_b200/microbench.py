@@ -1,0 +1,73 @@
+"""Per-pass micro-benchmark of the decoder passes (time, achieved HBM GB/s, fraction of peak).
+
+    python -m paper_2302_07863_b200.microbench --workload t5_sum --k 1,2,4,8,16 --cache 64,256,1024
+
+For every (k, cache length) it replays the large model's block pass as a CUDA graph
+(bild_time_pass) and prints one JSON line; `--small` adds the small model's single step.
+Bytes are the algorithmic bytes of the pass: every weight matrix and the LM head once, the
+cached self-attention rows and the cross-attention K/V of every layer, the k embedding rows.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+
+
+def pass_bytes(s, w_bytes, kv_bytes, cache_rows, enc_len, k):
+    g = 3 if s.ffn == "gated_gelu" else 2
+    I, d, F, V, L = s.inner, s.d_model, s.d_ff, s.vocab, s.n_layers
+    weights = w_bytes * (L * (6 * I * d + g * d * F) + V * d)
+    kv = kv_bytes * L * (2 * (cache_rows + k) * I + 2 * enc_len * I)
+    return weights + kv + w_bytes * k * d
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="t5_sum")
+    ap.add_argument("--k", default="1,2,4,8,16")
+    ap.add_argument("--cache", default="64,256,1024")
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--small", action="store_true")
+    ap.add_argument("--peak-gbs", type=float, default=0.0)
+    a = ap.parse_args()
+    import torch
+    assert torch.cuda.is_available(), "needs a CUDA device"
+    from workloads import MODEL_SHAPES, WORKLOADS
+    from paper_2302_07863_b200 import build
+    from paper_2302_07863_b200.synthetic import make_context
+    build.build()
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with open(os.path.join(root, "tests", "golden", a.workload + ".json")) as f:
+        g = json.load(f)
+    peak = a.peak_gbs
+    if not peak:
+        p = os.path.join(root, "MEASURED_PEAKS.json")
+        peak = float(json.load(open(p))["hbm_gbs"]) if os.path.exists(p) else 6650.0
+    ks = [int(x) for x in a.k.split(",")]
+    caches = [int(x) for x in a.cache.split(",")]
+    wl = WORKLOADS[a.workload]
+    ctx, ids, _ = make_context(a.workload, g["scale_small"]["scale"], g["scale_large"]["scale"],
+                               max_dec_len=max(caches) + 16 + 1)
+    ctx.encode(ids)
+    wb = 2 if wl.dtype == "bf16" else 4
+    sS, sL = MODEL_SHAPES[wl.small], MODEL_SHAPES[wl.large]
+    for cache in caches:
+        if a.small:
+            ms = ctx.time_pass(0, 1, cache, a.iters)
+            b = pass_bytes(sS, wb, 4, cache, wl.enc_len, 1)
+            print(json.dumps({"pass": "small step", "k": 1, "cache": cache, "us": ms * 1e3, "GBs": b / ms / 1e6,
+                              "frac_of_peak": b / ms / 1e6 / peak, "bytes": b}))
+        for k in ks:
+            ms = ctx.time_pass(1, k, cache, a.iters)
+            b = pass_bytes(sL, wb, 4, cache, wl.enc_len, k)
+            print(json.dumps({"pass": "large block pass", "k": k, "cache": cache, "us": ms * 1e3, "GBs": b / ms / 1e6,
+                              "frac_of_peak": b / ms / 1e6 / peak, "bytes": b,
+                              "tensor_cores": ctx.uses_tensor_cores() and k > 1}))
+
+
+if __name__ == "__main__":
+    main()
