@@ -487,9 +487,17 @@ void setup_umma(bild_ctx* c, Model& m) {
 }
 
 // Split of K over a cluster: enough blocks to pull the matrix at full bandwidth, at most 16 k blocks each.
-bool umma_plan(int N, int K, bool gated, int* cs_out, int* nkb_out) {
+bool umma_plan(int N, int K, bool gated, int* cs_out, int* nkb_out, bool many_row_blocks = false) {
   const int tiles = (N + UM_TILE_M - 1) / UM_TILE_M;
   int best = 0;
+  if (many_row_blocks) {   // encoder: row blocks already give enough CTAs; the smallest split of K that fits
+    for (int cs = 1; cs <= (gated ? 4 : 8); cs *= 2) {
+      if (K % (UM_KB * cs)) break;
+      const int nkb = K / UM_KB / cs;
+      if (nkb <= 16 && umma_smem_bytes(gated, nkb, cs) <= 227 * 1024) { *cs_out = cs; *nkb_out = nkb; return true; }
+    }
+    return false;
+  }
   for (int cs = 1; cs <= (gated ? 4 : 8); cs *= 2) {
     if (K % (UM_KB * cs)) break;
     const int nkb = K / UM_KB / cs;
@@ -557,7 +565,7 @@ cudaError_t launch_dec_linear(bild_ctx* c, Model& m, int MB, const LinArgs& a, i
 // Linear layer of the encoder over rb blocks of MAXB rows.
 cudaError_t launch_enc_linear(bild_ctx* c, Model& m, const LinArgs& a, int rb, int layer, int which_map) {
   int cs, nkb;
-  if (m.umma && umma_plan(a.N, a.K, a.epi == EPI_GATED, &cs, &nkb)) {
+  if (m.umma && umma_plan(a.N, a.K, a.epi == EPI_GATED, &cs, &nkb, rb >= 4)) {
     const CUtensorMap* t = &m.tmaps[(size_t)layer * TM_PER_LAYER];
     return launch_umma(c, a, t[which_map], t[which_map == TM_EWI0 ? TM_EWI1 : which_map], cs, nkb, rb);
   }
