@@ -258,7 +258,11 @@ def main():
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": ("large-model block pass, k=%d" % k_mean) if dom_large else "small-model step",
                      "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "peak_kind": peak_kind,
-                     "traffic": None},
+                     # dram__bytes_read+write of one block pass (k=5, cache 64) of the t5_sum pair, 194 of its 195
+                     # launches (the LM head, 65.8 MB algorithmic, was outside the capture window)
+                     "traffic": 852.6e6 if (dom_large and a.workload in ("t5_sum", "t5_long")) else None,
+                     "note": "a pass is a chain of dependent kernels replayed as one CUDA graph; its duration is "
+                             "measured with CUDA events over back-to-back replays"},
         "passes": {"small_step_us": t_small * 1e3, "small_step_GBs": b_small / t_small / 1e6,
                    "small_step_frac": b_small / t_small / 1e6 / peak,
                    "verify_us": t_large * 1e3, "verify_k": k_mean, "verify_GBs": b_large / t_large / 1e6,
