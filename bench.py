@@ -182,9 +182,10 @@ def main():
     ctx.encode(ids_pinned.numpy())
     torch.cuda.synchronize()
 
+    from paper_2302_07863_b200 import replicas
+
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier(dist if world > 1 else None, world)
         torch.cuda.synchronize()
 
     def run(fn, steps, warmup):
@@ -197,12 +198,7 @@ def main():
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return replicas.max_over_ranks(dist if world > 1 else None, world, e0.elapsed_time(e1), device="cuda")
 
     def step_resident():
         ctx.generate_async(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
@@ -246,13 +242,13 @@ def main():
     if rank != 0:
         return
     out = {
-        "metric": METRIC, "value": world * ntok * a.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": replicas.whole_job_rate(ntok * a.steps, world, ms), "unit": UNIT, "n_gpus": world,
         "steps": a.steps, "warmup": a.warmup, "ms_per_step": ms / a.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights, f32 activations and KV cache" if wb == 2 else "f32",
         "data": "synthetic", "gpu_launches": int(launches),
         "config": dict(cfg_common, l2="inputs larger than L2: every step re-reads "
                        f"{(b_large + b_small) / 1e6:.0f} MB of weights and K/V", parallelism="replicas only"),
-        "e2e": {"value": world * ntok * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT,
+        "e2e": {"value": replicas.whole_job_rate(ntok * e2e_steps, world, ms_e2e), "unit": UNIT,
                 "h2d_bytes_per_step": int(ids_pinned.numel() * 4),
                 "d2h_bytes_per_step": int(4 * ntok + 24 * r["n_trace"] + 2 * 96)},
         "clocks": clocks,

@@ -226,6 +226,29 @@ def test_generate_matches_live_oracle(torch_cuda, name, alpha_fb, alpha_rb, max_
         assert n is None or n > 0
 
 
+@pytest.mark.parametrize("env", ["BILD_BLOCK_SIMT", "BILD_HOST_LOOP", "BILD_NO_PDL", "BILD_NO_UMMA"])
+@pytest.mark.parametrize("name", ["tiny_bf16", "odd"])
+def test_alternative_paths_match_golden(torch_cuda, name, env):
+    """The switchable paths (SIMT block GEMV, host-driven loop, plain launches, SIMT block
+    linear) give the same tokens and trace as the default path's golden run."""
+    from paper_2302_07863_b200 import MODE_BILD
+    from paper_2302_07863_b200.synthetic import make_context
+    g = golden(name)
+    os.environ[env] = "1"
+    try:
+        ctx, ids, wl = make_context(name, g["scale_small"]["scale"], g["scale_large"]["scale"])
+    finally:
+        del os.environ[env]
+    ctx.encode(ids)
+    th = g["thresholds"]
+    r = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
+    assert r["tokens"] == g["bild"]["tokens"]
+    assert_trace_equal(r["trace"], g["bild"]["trace"], 1e-3)
+    assert r["stats"] == g["bild"]["stats"]
+    assert ctx.launch_count() > 0
+    ctx.close()
+
+
 def test_eos_and_limits(torch_cuda):
     from paper_2302_07863_b200 import MODE_SMALL_ONLY, BildError
     g = golden("tiny")
