@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "decode_kernels.cuh"
+#include "mega_pass.cuh"
 #include "umma_linear.cuh"
 
 using namespace bild;
@@ -103,6 +104,13 @@ struct Model {
   // TMA descriptors of the decoder's weight matrices (bf16 only): per layer qkv, o, cq, co, wi0, wi1, fo
   std::vector<CUtensorMap> tmaps;
   bool umma = false;
+  // whole-pass persistent kernel (bf16 only)
+  MegaLayer* mega_layers = nullptr;
+  unsigned* mega_sync = nullptr;
+  float* mega_part = nullptr;
+  bool mega = false;
+  MegaArgs mega_args{};
+  int mega_grid = 0;
 };
 
 }  // namespace
@@ -136,6 +144,7 @@ struct bild_ctx {
   bool block_simt = false;           // block pass on the SIMT block GEMV instead of the tensor-core kernel
   bool use_pdl = true;               // launch pass kernels with programmatic stream serialization
   bool host_loop = false;            // debug: drive the loop from the host, one read-back per step
+  bool mega_coop = true;             // launch the whole-pass kernel with the cooperative attribute
   int64_t graph_counted = 0;         // launches of the loop graphs already added to `launches`
 };
 
@@ -219,6 +228,9 @@ void plan(bild_ctx* c, Bump& b) {
     m.head_cnt = b.take<unsigned>(1);
     m.head_out = b.take<HeadOut>(1);
     m.desc = b.take<CallDesc>(1);
+    m.mega_layers = b.take<MegaLayer>(mc.n_layers);
+    m.mega_sync = b.take<unsigned>(4);
+    m.mega_part = b.take<float>(MG_ACT / sizeof(float));
   }
   const size_t ecap16 = (size_t)(ecap + MAXB - 1) / MAXB * MAXB;   // whole blocks of MAXB rows
   c->ex = b.take<float>(ecap16 * dmax);
@@ -486,6 +498,77 @@ void setup_umma(bild_ctx* c, Model& m) {
   m.umma = true;
 }
 
+// Decides whether the decoder passes of model `m` run as the persistent whole-pass kernel and
+// prepares its arguments (the per-layer pointer table lives in the workspace).
+int setup_mega(bild_ctx* c, Model& m) {
+  m.mega = false;
+  const char* off = std::getenv("BILD_NO_MEGA");
+  if (off && off[0] == '1') return BILD_OK;
+  if (c->cfg.dtype != BILD_BF16) return BILD_OK;
+  const bild_model_cfg& mc = m.c;
+  const int d = mc.d_model, I = m.inner, F = mc.d_ff;
+  const bool gated = mc.ffn_kind == BILD_FFN_GATED_GELU;
+  if (d % 8 || I % 8 || F % 8 || d * 2 > MG_SLOT || I * 2 > MG_SLOT || F * 2 > MG_SLOT) return BILD_OK;
+  int dev = 0, sms = 0, smem_max = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return BILD_OK;
+  }
+  const int nslots = std::min(MG_MAX_SLOTS, (smem_max - MG_ACT - MG_PSUM - MG_MISC) / MG_SLOT);
+  if (nslots < 4 || sms < 1) return BILD_OK;
+  // every stage's slice must fit the ring with room to fetch ahead, and its rows the partial-sum area
+  const int Ns[6] = {3 * I, d, I, d, F, d}, Ks[6] = {d, I, d, I, d, F};
+  for (int p = 0; p < 6; ++p) {
+    const int rows = (Ns[p] + sms - 1) / sms, nmat = (p == 4 && gated) ? 2 : 1;
+    const int rps = MG_SLOT / (Ks[p] * 2);
+    const int slots = (rows + rps - 1) / rps * nmat;
+    if (slots > nslots - 2 || rows * nmat > 4 * MG_QUADS) return BILD_OK;
+  }
+  auto aligned = [](const void* p) { return ((uintptr_t)p & 15) == 0; };
+  std::vector<MegaLayer> tab(mc.n_layers);
+  for (int l = 0; l < mc.n_layers; ++l) {
+    const bild_dec_layer& w = m.dec[l];
+    if (!aligned(w.wqkv) || !aligned(w.wo) || !aligned(w.wcq) || !aligned(w.wco) || !aligned(w.wi0) || !aligned(w.wfo) ||
+        (gated && !aligned(w.wi1)) || !aligned(w.ln1) || !aligned(w.ln2) || !aligned(w.ln3)) return BILD_OK;
+    MegaLayer& t = tab[l];
+    t.wqkv = (const __nv_bfloat16*)w.wqkv; t.wo = (const __nv_bfloat16*)w.wo; t.wcq = (const __nv_bfloat16*)w.wcq;
+    t.wco = (const __nv_bfloat16*)w.wco; t.wi0 = (const __nv_bfloat16*)w.wi0; t.wi1 = (const __nv_bfloat16*)w.wi1;
+    t.wfo = (const __nv_bfloat16*)w.wfo;
+    t.ln1 = (const float*)w.ln1; t.ln2 = (const float*)w.ln2; t.ln3 = (const float*)w.ln3;
+  }
+  if (!aligned(m.w.emb)) return BILD_OK;
+  if (cudaFuncSetAttribute(mega_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mega_smem_bytes(nslots)) != cudaSuccess) {
+    cudaGetLastError();
+    return BILD_OK;
+  }
+  CUDA_TRY(c, cudaMemcpyAsync(m.mega_layers, tab.data(), tab.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  MegaArgs& a = m.mega_args;
+  a.layers = m.mega_layers; a.n_layers = mc.n_layers;
+  a.d = d; a.I = I; a.F = F; a.H = mc.n_heads; a.dkv = mc.d_kv; a.dkv_shift = ilog2(mc.d_kv); a.gated = gated ? 1 : 0;
+  a.vocab = mc.vocab; a.eps = mc.ln_eps; a.desc = m.desc; a.emb = (const __nv_bfloat16*)m.w.emb;
+  a.x = m.x; a.q = m.q; a.att = m.att; a.u = m.u; a.part = m.mega_part;
+  a.selfK = m.selfK; a.selfV = m.selfV; a.crossK = m.crossK; a.crossV = m.crossV;
+  a.cap = c->cfg.max_dec_len; a.ecap = c->cfg.max_enc_len; a.dec_bias = m.dec_bias; a.enc_len = c->enc_len_dev;
+  a.sync = m.mega_sync; a.err = &c->st->err; a.nslots = nslots;
+  m.mega_grid = sms;
+  m.mega = true;
+  return BILD_OK;
+}
+
+cudaError_t launch_mega(bild_ctx* c, Model& m) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(m.mega_grid); cfg.blockDim = dim3(MG_THREADS);
+  cfg.dynamicSmemBytes = mega_smem_bytes(m.mega_args.nslots); cfg.stream = c->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeCooperative;   // all blocks resident at once: they wait for one another
+  at[0].val.cooperative = 1;
+  cfg.attrs = at; cfg.numAttrs = c->mega_coop ? 1 : 0;
+  (*c->cnt)++;
+  return cudaLaunchKernelEx(&cfg, mega_pass_kernel, m.mega_args);
+}
+
 // Split of K over a cluster: enough blocks to pull the matrix at full bandwidth, at most 16 k blocks each.
 bool umma_plan(int N, int K, bool gated, int* cs_out, int* nkb_out, bool many_row_blocks = false) {
   const int tiles = (N + UM_TILE_M - 1) / UM_TILE_M;
@@ -588,13 +671,15 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   const bild_model_cfg& mc = m.c;
   const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
   const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len, dt = c->cfg.dtype;
+  if (m.mega) CUDA_TRY(c, launch_mega(c, m));
+  else
   CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x));
   // self-attention: one block per head up to 128 cached rows (no merge step); cross-attention:
   // enough splits of the encoder keys to occupy the SMs
   int ns_self = 1;
   while (ns_self < 8 && (cap + ns_self - 1) / ns_self > 256) ns_self *= 2;
   const int ns_cross = pick_nsplit(H, ecap);
-  for (int l = 0; l < mc.n_layers; ++l) {
+  for (int l = 0; l < (m.mega ? 0 : mc.n_layers); ++l) {
     const bild_dec_layer& w = m.dec[l];
     const size_t kvoff = (size_t)l * H * dkv;
     LinArgs a{};
@@ -774,14 +859,19 @@ void drop_graphs(bild_ctx* c) {
 
 int build_graphs(bild_ctx* c) {
   if (c->exec[0] && c->exec[1]) return BILD_OK;
-  int rc = build_graphs_once(c);
-  if (rc != BILD_OK && c->use_pdl) {  // programmatic edges refused inside the loop bodies: plain edges
+  // what a loop body refuses (programmatic edges, cooperative kernel nodes) is dropped step by step
+  const bool want_pdl = c->use_pdl, want_coop = c->mega_coop;
+  const bool tries[3][2] = {{want_pdl, want_coop}, {want_pdl, false}, {false, false}};
+  int rc = BILD_ERR_CUDA;
+  for (int t = 0; t < 3; ++t) {
+    if (t > 0 && tries[t][0] == tries[t - 1][0] && tries[t][1] == tries[t - 1][1]) continue;
+    c->use_pdl = tries[t][0];
+    c->mega_coop = tries[t][1];
+    rc = build_graphs_once(c);
+    if (rc == BILD_OK) return rc;
     drop_graphs(c);
     cudaGetLastError();
-    c->use_pdl = false;
-    rc = build_graphs_once(c);
   }
-  if (rc != BILD_OK) drop_graphs(c);
   return rc;
 }
 
@@ -912,6 +1002,10 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   }
   // zero the ticket counters and the state, build the bias-by-distance tables
   if (cudaMemsetAsync(workspace, 0, c->ws_bytes, c->stream) != cudaSuccess) { bild_destroy(c); return BILD_ERR_CUDA; }
+  for (int i = 0; i < 2; ++i) {
+    rc = setup_mega(c, c->m[i]);
+    if (rc) { bild_destroy(c); return rc; }
+  }
   rc = build_bias_tables(c);
   if (rc) { bild_destroy(c); return rc; }
   *out = c;
