@@ -107,7 +107,9 @@ struct Model {
   // whole-pass persistent kernel (bf16 only)
   MegaLayer* mega_layers = nullptr;
   unsigned* mega_sync = nullptr;
-  float* mega_part = nullptr;
+  uint2* mega_ll = nullptr;          // all (value, epoch) areas, contiguous
+  size_t mega_ll_pairs = 0;
+  int64_t mega_launch_bound = 0;     // launches since the areas and the epoch base were last cleared
   bool mega = false;
   MegaArgs mega_args{};
   int mega_grid = 0;
@@ -145,6 +147,7 @@ struct bild_ctx {
   bool use_pdl = true;               // launch pass kernels with programmatic stream serialization
   bool host_loop = false;            // debug: drive the loop from the host, one read-back per step
   bool mega_coop = true;             // launch the whole-pass kernel with the cooperative attribute
+  bool capturing = false;            // launches are being recorded into a graph, not run
   int64_t graph_counted = 0;         // launches of the loop graphs already added to `launches`
 };
 
@@ -230,7 +233,8 @@ void plan(bild_ctx* c, Bump& b) {
     m.desc = b.take<CallDesc>(1);
     m.mega_layers = b.take<MegaLayer>(mc.n_layers);
     m.mega_sync = b.take<unsigned>(4);
-    m.mega_part = b.take<float>(MG_ACT / sizeof(float));
+    m.mega_ll_pairs = (size_t)MAXB * (6 * m.inner + 3 * mc.d_model + mc.d_ff) + 2 * mega_record_pairs(MG_MAX_BLOCKS, mc.d_kv);
+    m.mega_ll = b.take<uint2>(m.mega_ll_pairs);
   }
   const size_t ecap16 = (size_t)(ecap + MAXB - 1) / MAXB * MAXB;   // whole blocks of MAXB rows
   c->ex = b.take<float>(ecap16 * dmax);
@@ -516,14 +520,15 @@ int setup_mega(bild_ctx* c, Model& m) {
     return BILD_OK;
   }
   const int nslots = std::min(MG_MAX_SLOTS, (smem_max - MG_ACT - MG_PSUM - MG_MISC) / MG_SLOT);
-  if (nslots < 4 || sms < 1) return BILD_OK;
+  if (nslots < 4 || sms < 1 || sms > MG_MAX_BLOCKS) return BILD_OK;
+  if (mc.n_heads * 4 > sms || (d + sms - 1) / sms > MG_XRES || 8 * mc.n_layers + 2 > MG_EPOCHS_PER_LAUNCH) return BILD_OK;
   // every stage's slice must fit the ring with room to fetch ahead, and its rows the partial-sum area
   const int Ns[6] = {3 * I, d, I, d, F, d}, Ks[6] = {d, I, d, I, d, F};
   for (int p = 0; p < 6; ++p) {
     const int rows = (Ns[p] + sms - 1) / sms, nmat = (p == 4 && gated) ? 2 : 1;
     const int rps = MG_SLOT / (Ks[p] * 2);
     const int slots = (rows + rps - 1) / rps * nmat;
-    if (slots > nslots - 2 || rows * nmat > 4 * MG_QUADS) return BILD_OK;
+    if (slots > nslots - 2 || rows * nmat > 4 * MG_QUADS || mc.n_layers > MG_MAX_LAYERS) return BILD_OK;
   }
   auto aligned = [](const void* p) { return ((uintptr_t)p & 15) == 0; };
   std::vector<MegaLayer> tab(mc.n_layers);
@@ -548,7 +553,15 @@ int setup_mega(bild_ctx* c, Model& m) {
   a.layers = m.mega_layers; a.n_layers = mc.n_layers;
   a.d = d; a.I = I; a.F = F; a.H = mc.n_heads; a.dkv = mc.d_kv; a.dkv_shift = ilog2(mc.d_kv); a.gated = gated ? 1 : 0;
   a.vocab = mc.vocab; a.eps = mc.ln_eps; a.desc = m.desc; a.emb = (const __nv_bfloat16*)m.w.emb;
-  a.x = m.x; a.q = m.q; a.att = m.att; a.u = m.u; a.part = m.mega_part;
+  a.x = m.x;
+  {
+    uint2* p = m.mega_ll;
+    auto take = [&](size_t n) { uint2* r = p; p += n; return r; };
+    const size_t rec = mega_record_pairs(MG_MAX_BLOCKS, mc.d_kv);
+    a.ll.qkv1 = take((size_t)MAXB * 3 * I); a.ll.a2 = take((size_t)MAXB * I); a.ll.r2 = take(rec);
+    a.ll.x3 = take((size_t)MAXB * d); a.ll.q4 = take((size_t)MAXB * I); a.ll.a5 = take((size_t)MAXB * I); a.ll.r5 = take(rec);
+    a.ll.x6 = take((size_t)MAXB * d); a.ll.u7 = take((size_t)MAXB * F); a.ll.x8 = take((size_t)MAXB * d);
+  }
   a.selfK = m.selfK; a.selfV = m.selfV; a.crossK = m.crossK; a.crossV = m.crossV;
   a.cap = c->cfg.max_dec_len; a.ecap = c->cfg.max_enc_len; a.dec_bias = m.dec_bias; a.enc_len = c->enc_len_dev;
   a.sync = m.mega_sync; a.err = &c->st->err; a.nslots = nslots;
@@ -557,7 +570,23 @@ int setup_mega(bild_ctx* c, Model& m) {
   return BILD_OK;
 }
 
+// The epochs are 32-bit and grow by MG_EPOCHS_PER_LAUNCH per launch: long before they could wrap,
+// the areas and the launch counter are cleared (stream-ordered, between passes).
+cudaError_t mega_epoch_budget(bild_ctx* c, Model& m, int64_t launches) {
+  if (!m.mega) return cudaSuccess;
+  m.mega_launch_bound += launches;
+  if (m.mega_launch_bound < (int64_t)2000000) return cudaSuccess;
+  m.mega_launch_bound = launches;
+  cudaError_t e = cudaMemsetAsync(m.mega_ll, 0, m.mega_ll_pairs * sizeof(uint2), c->stream);
+  if (e != cudaSuccess) return e;
+  return cudaMemsetAsync(m.mega_sync, 0, 4 * sizeof(unsigned), c->stream);
+}
+
 cudaError_t launch_mega(bild_ctx* c, Model& m) {
+  if (!c->capturing) {
+    cudaError_t e = mega_epoch_budget(c, m, 1);
+    if (e != cudaSuccess) return e;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(m.mega_grid); cfg.blockDim = dim3(MG_THREADS);
   cfg.dynamicSmemBytes = mega_smem_bytes(m.mega_args.nslots); cfg.stream = c->stream;
@@ -826,7 +855,9 @@ int capture_pass(bild_ctx* c, cudaGraph_t body, int which, int MB, unsigned long
   cudaStream_t user_stream = c->stream;
   c->stream = c->cap_stream;
   c->cnt = &n;
+  c->capturing = true;
   int rc = decoder_pass(c, which, MB, nullptr, hw, hi);
+  c->capturing = false;
   c->cnt = &c->launches;
   c->stream = user_stream;
   if (rc == BILD_OK && leaves) {
@@ -1130,6 +1161,10 @@ int bild_generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, i
     rc = reset_state(c, mode, alpha_fb, alpha_rb, max_len);
     if (rc) return rc;
     if (max_len == 0 || c->cfg.start_id == c->cfg.eos_id) return BILD_OK;
+    // passes the loop may run: bounded by the guard of the device-side policy
+    const int64_t bound = (int64_t)(max_len + 2) * (c->cfg.max_draft + 3) + 16;
+    CUDA_TRY(c, mega_epoch_budget(c, c->m[0], bound));
+    CUDA_TRY(c, mega_epoch_budget(c, c->m[1], bound));
     CUDA_TRY(c, cudaGraphLaunch(c->exec[mode == BILD_MODE_LARGE_ONLY ? 1 : 0], c->stream));
     return BILD_OK;
   }
@@ -1247,6 +1282,7 @@ int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, floa
   int64_t n_launch = 0;
   if (rc == BILD_OK) rc = capture_pass(c, g, which, k == 1 ? 1 : MAXB, 0, 0, nullptr, &n_launch);
   if (rc == BILD_OK && cudaGraphInstantiate(&ex, g, 0) != cudaSuccess) rc = BILD_ERR_CUDA;
+  if (rc == BILD_OK && mega_epoch_budget(c, c->m[which], iters + 1) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && cudaGraphLaunch(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;  // untimed first pass
   if (rc == BILD_OK && cudaEventRecord(e0, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
   for (int it = 0; it < iters && rc == BILD_OK; ++it)

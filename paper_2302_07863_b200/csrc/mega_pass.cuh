@@ -1,44 +1,65 @@
 // One decoder pass (steps S0..S8 / L0..L8 of every layer) as ONE persistent kernel, bf16 weights.
 //
-// A decoder pass at batch 1 is a chain of ~8 dependent stages per layer, each of which moves
-// far less data than it takes to hide the memory latency, so a chain of separate kernels is
-// bound by launch and memory latency.  Here one block per SM stays resident for the whole
-// pass:
+// A decoder pass at batch 1 is a chain of 8 dependent stages per layer, each of which moves far
+// less data than it takes to hide the memory latency, so a chain of separate kernels is bound
+// by launch and memory latency.  Here one block per SM stays resident for the whole pass:
 //   * a producer warp streams the block's slice of every weight matrix, in program order,
-//     through a ring of shared-memory slots with bulk (TMA) copies.  The weights do not
-//     depend on the activations, so the stream runs ahead of the dependency chain and a
-//     stage finds its weights already on chip;
-//   * eight consumer warps run the stages.  Stages are separated by a grid-wide barrier (an
-//     arrive counter in global memory); the k activation rows a stage needs are pulled into
-//     shared memory with one bulk copy right after the barrier;
-//   * a linear stage splits the output rows over the blocks (no cross-block reduction);
-//     inside a block a work item is 4 weight rows x 256 columns for all token rows, partial
-//     sums are added in a fixed order;
-//   * attention splits (head, row group, key range) over the blocks, keys and values are
-//     staged in 64-key chunks (double buffered) with a running soft-max; key splits leave
-//     (max, sum, weighted values) records that the following output projection merges while
-//     it loads its input.
-// Every wait (grid barrier, mbarrier) gives up after a fixed number of polls: the block
-// then records BILD_ERR_TIMEOUT, stops waiting anywhere, and runs to the end.
+//     through a ring of shared-memory slots with bulk (TMA) copies.  The weights do not depend
+//     on the activations, so the stream runs ahead of the dependency chain and a stage finds
+//     its weights already on chip;
+//   * eight consumer warps run the stages.  There is no grid-wide barrier: every activation
+//     that crosses blocks travels as an 8-byte (value, epoch) pair written with one store, and
+//     a reader polls the pairs it needs until they carry the epoch of the stage it is in
+//     (one epoch per stage and launch).  A stage therefore starts in a block as soon as that
+//     block's own inputs have arrived, one L2 round trip after they were written;
+//   * a linear stage splits the output rows over the blocks (no cross-block reduction); inside
+//     a block a work item is 4 weight rows x 256 columns for all token rows, partial sums are
+//     added in a fixed order.  The block that owns a slice of the model dimension keeps the
+//     residual stream of that slice in shared memory;
+//   * attention splits (head, row group, key range) over the blocks; cached keys / values are
+//     staged in 64-key chunks (bulk copies, double buffered, issued before the queries arrive)
+//     with a running soft-max, the rows of the current block of tokens arrive as pairs; the
+//     first split of a (head, row group) merges the others' (max, sum, weighted values).
+// Every wait gives up after a fixed number of polls: the block then records BILD_ERR_TIMEOUT,
+// stops waiting anywhere, and runs to the end.
 #pragma once
 #include "common.cuh"
 
 namespace bild {
 
 constexpr int MG_CONSUMERS = 256;                   // 8 consumer warps
-constexpr int MG_THREADS = MG_CONSUMERS + 32;       // + the producer warp
+constexpr int MG_THREADS = MG_CONSUMERS;
+constexpr int MG_FEEDER = MG_CONSUMERS - 1;        // the thread that issues the weight copies
 constexpr int MG_SLOT = 8192;                       // bytes per ring slot
 constexpr int MG_ACT = 80 * 1024;                   // activation staging
-constexpr int MG_QUADS = 16;                        // weight-row quads per stage and block (64 rows)
-constexpr int MG_PSUM = MG_QUADS * 8 * 32 * 4;      // partial sums [quad][warp][32]
+constexpr int MG_QUADS = 12;                        // weight-row quads per stage and block (48 rows)
+constexpr int MG_PSUM = MG_QUADS * 8 * 32 * 4;      // partial sums [quad][warp][32]; attention scratch
 constexpr int MG_MAX_SLOTS = 20;
-constexpr int MG_MISC = 1024;
-constexpr int MG_PST_PAD = 4;                       // record = [max, sum, -, -, values[dkv]]
+constexpr int MG_MAX_BLOCKS = 256;                 // record areas are sized for this many blocks
+constexpr int MG_MISC = 7168;
+constexpr int MG_MAX_LAYERS = 56;                  // the per-layer pointer table is copied to shared memory
+constexpr int MG_PST_PAD = 4;                       // record = [max, sum, 0, 0, values[dkv]]
+constexpr int MG_XRES = 16;                         // columns of the model dimension one block may own
 constexpr unsigned MG_SPIN = 1u << 20;
+constexpr int MG_EPOCHS_PER_LAUNCH = 1024;          // > 8 * layers
 
 struct MegaLayer {
   const __nv_bfloat16 *wqkv, *wo, *wcq, *wco, *wi0, *wi1, *wfo;
   const float *ln1, *ln2, *ln3;
+};
+
+// (value, epoch) pairs of the eight stage outputs, each for MAXB token rows
+struct MegaLL {
+  uint2 *qkv1;  // [H][MAXB][3][dkv]  query | key | value of the rows of this pass, by head
+  uint2 *a2;    // [MAXB][I]      self-attention output
+  uint2 *r2;    // records of the key splits, self-attention
+  uint2 *x3;    // [MAXB][d]
+  uint2 *q4;    // [H][MAXB][dkv]  cross-attention queries, by head
+  uint2 *a5;    // [MAXB][I]
+  uint2 *r5;
+  uint2 *x6;    // [MAXB][d]
+  uint2 *u7;    // [MAXB][F]
+  uint2 *x8;    // [MAXB][d]
 };
 
 struct MegaArgs {
@@ -48,18 +69,21 @@ struct MegaArgs {
   float eps;
   const CallDesc* desc;
   const __nv_bfloat16* emb;
-  float *x, *q, *att, *u, *part;
+  float* x;                   // [MAXB][d] residual stream after the last layer (input of the LM head)
   float *selfK, *selfV;
   const float *crossK, *crossV;
   int cap, ecap;
   const float* dec_bias;      // [H][cap] by distance
   const int* enc_len;
-  unsigned* sync;             // [0], [1]: arrive counters (alternating between launches); [2]: which one is next
+  unsigned* sync;             // [0]: launches so far (epoch base)
   int* err;
   int nslots;
+  MegaLL ll;
 };
 
 inline size_t mega_smem_bytes(int nslots) { return (size_t)nslots * MG_SLOT + MG_ACT + MG_PSUM + MG_MISC; }
+// pairs in one record area: per (head, row group) up to 7 later splits x 4 rows
+inline size_t mega_record_pairs(int blocks, int dkv) { return (size_t)blocks * 32 * (dkv + MG_PST_PAD); }
 
 // ---- small PTX helpers ----------------------------------------------------------------
 __device__ __forceinline__ void mg_mbar_init(uint32_t bar, uint32_t count) {
@@ -81,22 +105,26 @@ __device__ __forceinline__ void mg_bulk_g2s(uint32_t dst, const void* src, uint3
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void mg_fence_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
-__device__ __forceinline__ unsigned mg_ld_acquire(const unsigned* p) {
-  unsigned v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+__device__ __forceinline__ void mg_csync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }   // consumer warps only
+__device__ __forceinline__ void mg_ll_store(uint2* p, float v, uint32_t ep) {
+  asm volatile("st.volatile.global.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(__float_as_uint(v)), "r"(ep) : "memory");
+}
+__device__ __forceinline__ uint4 mg_ll_load2(const uint2* p) {   // two pairs, 16-byte aligned
+  uint4 v;
+  asm volatile("ld.volatile.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void mg_red_release(unsigned* p, unsigned v) {
-  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ void mg_csync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }   // consumer warps only
 
 // Block-wide state in shared memory.
 struct MegaShared {
-  unsigned long long full[MG_MAX_SLOTS], empty[MG_MAX_SLOTS], actbar, kvbar[2];
+  unsigned long long full[MG_MAX_SLOTS], kvbar[2];   // full[i]: all slices of the i-th (mod) linear stage have landed
+  MegaLayer layers[MG_MAX_LAYERS];
+  int slice[6][2];                      // rows of the six matrices that belong to this block
   float inv[MAXB];                      // 1 / rms of the staged rows
+  float ssq[8][MAXB];                   // sum of squares of the staged rows, per warp
   float amax[4], asum[4], ascale[4];    // running soft-max of the unit's rows
+  unsigned rowoff[4 * MG_QUADS];        // byte offset of every slice row in the ring
+  float xres[MAXB][MG_XRES];            // residual stream of the columns this block owns
   int failed;
 };
 
@@ -106,11 +134,44 @@ __device__ __forceinline__ void mg_fail(MegaShared* sh, int* err) {
 }
 // bounded mbarrier wait; after a failure nothing waits any more
 __device__ __forceinline__ void mg_wait(MegaShared* sh, int* err, unsigned long long* bar, uint32_t parity) {
-  if (*(volatile int*)&sh->failed) return;
   const uint32_t b = smem_u32(bar);
+  if (mg_mbar_try(b, parity)) return;
+  if (*(volatile int*)&sh->failed) return;
   for (unsigned it = 0; it < MG_SPIN; ++it)
     if (mg_mbar_try(b, parity)) return;
   mg_fail(sh, err);
+}
+
+// Polls the n2 16-byte units (two pairs each) at src until they carry epoch ep and writes the
+// 2 * n2 values to dst (shared memory, same order).  All consumer threads call it; at most 8
+// units per thread are in flight at a time.
+__device__ __noinline__ void mg_ll_fetch(const uint2* src, int n2, float* dst, uint32_t ep, MegaShared* sh, int* err) {
+  const int tid = threadIdx.x;
+#pragma unroll 1
+  for (int b0 = tid; b0 < n2; b0 += MG_CONSUMERS * 8) {
+    unsigned pend = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (b0 + j * MG_CONSUMERS < n2) pend |= 1u << j;
+    unsigned it = 0;
+    while (pend) {
+      uint4 v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (pend & (1u << j)) v[j] = mg_ll_load2(src + 2 * (size_t)(b0 + j * MG_CONSUMERS));
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if ((pend & (1u << j)) && v[j].y == ep && v[j].w == ep) {
+          *reinterpret_cast<float2*>(dst + 2 * (size_t)(b0 + j * MG_CONSUMERS)) =
+              make_float2(__uint_as_float(v[j].x), __uint_as_float(v[j].z));
+          pend &= ~(1u << j);
+        }
+      if (pend && (++it > MG_SPIN || *(volatile int*)&sh->failed)) {
+        if (it > MG_SPIN) mg_fail(sh, err);
+        break;
+      }
+    }
+  }
 }
 
 // The six weight matrices of a layer in the order the stages use them.
@@ -137,61 +198,57 @@ __device__ __forceinline__ void mg_slice(int N, int b, int G, int* r0, int* r1) 
   *r1 = (int)(((long long)(b + 1) * N) / G);
 }
 
-// ---- producer: the block's weight slices, in program order, through the ring -----------
-__device__ void mg_producer(const MegaArgs& a, MegaShared* sh, unsigned char* ring) {
-  const int G = gridDim.x, b = blockIdx.x, ns = a.nslots;
-  unsigned fill = 0;
-  for (int l = 0; l < a.n_layers; ++l) {
-    const MegaLayer L = a.layers[l];
-    for (int p = 0; p < 6; ++p) {
-      const MegaLin w = mg_lin(a, L, p);
-      int r0, r1;
-      mg_slice(w.N, b, G, &r0, &r1);
-      const int rowbytes = w.K * 2, rps = MG_SLOT / rowbytes;
-      for (int mat = 0; mat < (w.W1 ? 2 : 1); ++mat) {
-        const __nv_bfloat16* W = mat ? w.W1 : w.W0;
-        for (int r = r0; r < r1; r += rps) {
-          const int nr = min(rps, r1 - r);
-          const int slot = fill % ns;
-          mg_wait(sh, a.err, &sh->empty[slot], ((fill / ns) & 1) ^ 1);
-          const uint32_t bar = smem_u32(&sh->full[slot]);
-          mg_mbar_expect(bar, (uint32_t)(nr * rowbytes));
-          mg_bulk_g2s(smem_u32(ring + (size_t)slot * MG_SLOT), W + (size_t)r * w.K, (uint32_t)(nr * rowbytes), bar);
-          ++fill;
-        }
+// ---- the block's weight slices, in program order, through the ring ------------------------
+// One thread owns the stream: it fills every slot at the start and refills the slots of a stage
+// as soon as the stage has used them (it frees them itself, so it never waits).
+struct MegaFeed {
+  int l, p, mat, r, r1, rps, K;          // next copy: layer, matrix, row range of this block's slice
+  const __nv_bfloat16* W;
+  int slot;                              // next slot to fill
+  int stage;                             // linear stages of this block fully issued so far (mod MG_MAX_SLOTS)
+  bool second;                           // the matrix under way has a successor in the same stage
+  bool done;
+};
+__device__ __forceinline__ void mg_feed_open(const MegaArgs& a, const MegaShared* sh, MegaFeed& f) {   // positions f at (f.l, f.p, f.mat)
+  while (f.l < a.n_layers) {
+    const MegaLin w = mg_lin(a, sh->layers[f.l], f.p);
+    const int r0 = sh->slice[f.p][0];
+    f.r1 = sh->slice[f.p][1];
+    if (f.r1 > r0) {
+      f.r = r0; f.K = w.K; f.rps = MG_SLOT / (w.K * 2); f.W = f.mat ? w.W1 : w.W0;
+      f.second = w.W1 && f.mat == 0;
+      return;
+    }
+    if (++f.p == 6) { f.p = 0; ++f.l; }   // no rows of this matrix belong to the block
+  }
+  f.done = true;
+}
+__device__ __forceinline__ void mg_feed_init(const MegaArgs& a, const MegaShared* sh, MegaFeed& f) {
+  f.l = 0; f.p = 0; f.mat = 0; f.slot = 0; f.stage = 0; f.done = false;
+  mg_feed_open(a, sh, f);
+}
+// fills `count` slots (fewer if the program ends); the last copy of a stage also arrives on its barrier
+__device__ __noinline__ void mg_feed(const MegaArgs& a, MegaShared* sh, unsigned char* ring, MegaFeed& f, int count) {
+  for (int i = 0; i < count && !f.done; ++i) {
+    const int nr = min(f.rps, f.r1 - f.r);
+    const uint32_t bytes = (uint32_t)(nr * f.K * 2);
+    const uint32_t bar = smem_u32(&sh->full[f.stage]);
+    const bool last = f.r + nr >= f.r1 && !f.second;
+    if (last) mg_mbar_expect(bar, bytes);
+    else asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+    mg_bulk_g2s(smem_u32(ring + (size_t)f.slot * MG_SLOT), f.W + (size_t)f.r * f.K, bytes, bar);
+    if (++f.slot == a.nslots) f.slot = 0;
+    f.r += nr;
+    if (f.r >= f.r1) {
+      if (f.second) f.mat = 1;
+      else {
+        f.mat = 0;
+        if (++f.p == 6) { f.p = 0; ++f.l; }
+        if (++f.stage == MG_MAX_SLOTS) f.stage = 0;
       }
+      mg_feed_open(a, sh, f);
     }
   }
-  // nothing may still be in flight into this block's shared memory when it exits
-  const unsigned first = fill > (unsigned)ns ? fill - ns : 0;
-  for (unsigned f = first; f < fill; ++f) {
-    const uint32_t bar = smem_u32(&sh->full[f % ns]);
-    for (unsigned it = 0; it < MG_SPIN; ++it)
-      if (mg_mbar_try(bar, (f / ns) & 1)) break;
-  }
-}
-
-// ---- grid barrier ------------------------------------------------------------------------
-struct MegaBarrier {
-  unsigned* ctr;
-  unsigned done;    // barriers passed so far
-};
-// all consumer threads call both; global writes made before arrive are visible after wait
-__device__ __forceinline__ void mg_arrive(MegaBarrier& gb) {
-  mg_fence_async();   // this thread's global stores, for bulk copies issued by other blocks
-  mg_csync();
-  if (threadIdx.x == 0) mg_red_release(gb.ctr, 1u);
-}
-__device__ __forceinline__ void mg_wait_grid(MegaBarrier& gb, MegaShared* sh, int* err) {
-  ++gb.done;
-  if (threadIdx.x == 0 && !*(volatile int*)&sh->failed) {
-    const unsigned target = gb.done * gridDim.x;
-    unsigned it = 0;
-    while (mg_ld_acquire(gb.ctr) < target)
-      if (++it > MG_SPIN) { mg_fail(sh, err); break; }
-    mg_fence_async();
-  }
-  mg_csync();
 }
 
 // ---- sum of NP register values across the warp, one shuffle per halving ------------------
@@ -215,85 +272,67 @@ __device__ __forceinline__ float mg_treduce(float (&v)[NP], int lane) {
   return r;
 }
 
-// Where slice row r of the running stage sits in the ring.
-struct MegaRows {
-  unsigned char* ring;
-  int ns, slot0, rps, rowbytes;
-  int n0, slots0;     // gated: rows >= n0 belong to the second matrix, which starts slots0 slots later
-  __device__ __forceinline__ const unsigned char* row(int r) const {
-    int s = slot0;
-    if (r >= n0) { r -= n0; s += slots0; }
-    s += r / rps;
-    return ring + (size_t)(s % ns) * MG_SLOT + (size_t)(r % rps) * rowbytes;
-  }
-};
-
-// Work items of a linear stage: (quad of weight rows, 256 columns) x MG token rows.
+// Work items of a linear stage: (quad of weight rows, 256 columns) x MG token rows.  Item it
+// belongs to quad it / nkb and column block it % nkb; warp w takes items w, w + 8, ...  (rows past
+// the end of the slice repeat its last row; nobody reads their sums)
 template <int MG>
-__device__ __forceinline__ void mg_items(const MegaRows& R, int nrows, int K, const float* Xs, float* psum, int warp, int lane) {
+__device__ __forceinline__ void mg_items(const unsigned char* ring, const unsigned* rowoff, int nrows, int K, const float* Xs,
+                                         float* psum, int warp, int lane) {
   constexpr int NA = 4 * MG;
   constexpr int NP = NA <= 4 ? 4 : NA <= 8 ? 8 : NA <= 16 ? 16 : 32;
-  const int nkb = (K + 255) >> 8, nq = (nrows + 3) >> 2, nitems = nq * nkb;
-  float acc[NP];
-#pragma unroll
-  for (int i = 0; i < NP; ++i) acc[i] = 0.f;
-  int cur = -1;
+  constexpr int SH = NP == 32 ? 0 : NP == 16 ? 1 : NP == 8 ? 2 : 3;
+  const int nkb = (K + 255) >> 8, nq = (nrows + 3) >> 2;
 #pragma unroll 1
-  for (int it = warp; it < nitems; it += 8) {
-    const int qd = it / nkb, kb = it - qd * nkb;
-    if (qd != cur) {
-      if (cur >= 0) {
-        const float r = mg_treduce<NP>(acc, lane);
-        if ((lane & (32 / NP - 1)) == 0) psum[(cur * 8 + warp) * 32 + (lane >> (NP == 32 ? 0 : NP == 16 ? 1 : NP == 8 ? 2 : 3))] = r;
+  for (int qd = 0; qd < nq; ++qd) {
+    int kb = (warp - qd * nkb) & 7;   // first column block of this quad that falls to this warp
+    if (kb >= nkb) continue;
+    float acc[NP];
 #pragma unroll
-        for (int i = 0; i < NP; ++i) acc[i] = 0.f;
-      }
-      cur = qd;
-    }
-    const int kofs = (kb << 8) + lane * 8;
-    if (kofs < K) {
-      uint4 w[4];
+    for (int i = 0; i < NP; ++i) acc[i] = 0.f;
+    unsigned off[4];
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        const int row = qd * 4 + r;
-        w[r] = row < nrows ? *reinterpret_cast<const uint4*>(R.row(row) + (size_t)kofs * 2) : make_uint4(0, 0, 0, 0);
-      }
+    for (int r = 0; r < 4; ++r) off[r] = rowoff[min(qd * 4 + r, nrows - 1)];
+#pragma unroll 1
+    for (; kb < nkb; kb += 8) {
+      const int kofs = (kb << 8) + lane * 8;
+      if (kofs < K) {
+        uint4 w[4];
 #pragma unroll
-      for (int m = 0; m < MG; ++m) {
-        const float4 x0 = *reinterpret_cast<const float4*>(Xs + (size_t)m * K + kofs);
-        const float4 x1 = *reinterpret_cast<const float4*>(Xs + (size_t)m * K + kofs + 4);
+        for (int r = 0; r < 4; ++r) w[r] = *reinterpret_cast<const uint4*>(ring + off[r] + (size_t)kofs * 2);
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          float s = acc[r * MG + m];
-          s += __uint_as_float(w[r].x << 16) * x0.x;
-          s += __uint_as_float(w[r].x & 0xffff0000u) * x0.y;
-          s += __uint_as_float(w[r].y << 16) * x0.z;
-          s += __uint_as_float(w[r].y & 0xffff0000u) * x0.w;
-          s += __uint_as_float(w[r].z << 16) * x1.x;
-          s += __uint_as_float(w[r].z & 0xffff0000u) * x1.y;
-          s += __uint_as_float(w[r].w << 16) * x1.z;
-          s += __uint_as_float(w[r].w & 0xffff0000u) * x1.w;
-          acc[r * MG + m] = s;
+        for (int m = 0; m < MG; ++m) {
+          const float4 x0 = *reinterpret_cast<const float4*>(Xs + (size_t)m * K + kofs);
+          const float4 x1 = *reinterpret_cast<const float4*>(Xs + (size_t)m * K + kofs + 4);
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            float s = acc[r * MG + m];
+            s += __uint_as_float(w[r].x << 16) * x0.x;
+            s += __uint_as_float(w[r].x & 0xffff0000u) * x0.y;
+            s += __uint_as_float(w[r].y << 16) * x0.z;
+            s += __uint_as_float(w[r].y & 0xffff0000u) * x0.w;
+            s += __uint_as_float(w[r].z << 16) * x1.x;
+            s += __uint_as_float(w[r].z & 0xffff0000u) * x1.y;
+            s += __uint_as_float(w[r].w << 16) * x1.z;
+            s += __uint_as_float(w[r].w & 0xffff0000u) * x1.w;
+            acc[r * MG + m] = s;
+          }
         }
       }
     }
-  }
-  if (cur >= 0) {
     const float r = mg_treduce<NP>(acc, lane);
-    if ((lane & (32 / NP - 1)) == 0) psum[(cur * 8 + warp) * 32 + (lane >> (NP == 32 ? 0 : NP == 16 ? 1 : NP == 8 ? 2 : 3))] = r;
+    if ((lane & (32 / NP - 1)) == 0) psum[(qd * 8 + warp) * 32 + (lane >> SH)] = r;
   }
 }
 
-__device__ __forceinline__ void mg_items_dyn(int mg, const MegaRows& R, int nrows, int K, const float* Xs, float* psum, int warp, int lane) {
-  switch (mg) {
-    case 1: mg_items<1>(R, nrows, K, Xs, psum, warp, lane); break;
-    case 2: mg_items<2>(R, nrows, K, Xs, psum, warp, lane); break;
-    case 3: mg_items<3>(R, nrows, K, Xs, psum, warp, lane); break;
-    case 4: mg_items<4>(R, nrows, K, Xs, psum, warp, lane); break;
-    case 5: mg_items<5>(R, nrows, K, Xs, psum, warp, lane); break;
-    case 6: mg_items<6>(R, nrows, K, Xs, psum, warp, lane); break;
-    case 7: mg_items<7>(R, nrows, K, Xs, psum, warp, lane); break;
-    default: mg_items<8>(R, nrows, K, Xs, psum, warp, lane); break;
+// Token rows are taken 1, 2, 4 or 8 at a time (rows beyond mg hold stale values whose sums nobody reads).
+__device__ __forceinline__ int mg_round_rows(int mg) { return mg <= 2 ? mg : mg <= 4 ? 4 : 8; }
+__device__ __forceinline__ void mg_items_dyn(int mgr, const unsigned char* ring, const unsigned* rowoff, int nrows, int K,
+                                             const float* Xs, float* psum, int warp, int lane) {
+  switch (mgr) {
+    case 1: mg_items<1>(ring, rowoff, nrows, K, Xs, psum, warp, lane); break;
+    case 2: mg_items<2>(ring, rowoff, nrows, K, Xs, psum, warp, lane); break;
+    case 4: mg_items<4>(ring, rowoff, nrows, K, Xs, psum, warp, lane); break;
+    default: mg_items<8>(ring, rowoff, nrows, K, Xs, psum, warp, lane); break;
   }
 }
 
@@ -301,91 +340,84 @@ __device__ __forceinline__ void mg_items_dyn(int mg, const MegaRows& R, int nrow
 struct MegaAttnPlan {
   int rg;      // rows per unit
   int nrg;     // row groups
-  int ns;      // key splits (1: the unit writes the finished rows)
+  int ns;      // key splits
   int ck;      // keys per staged chunk
+  int per;     // keys per split
 };
 __device__ __forceinline__ MegaAttnPlan mg_attn_plan(const MegaArgs& a, int M, int nkeys, int G) {
   MegaAttnPlan p;
   const int rgmax = max(1, min(4, 256 >> a.dkv_shift));
   p.nrg = (M + rgmax - 1) / rgmax;
   p.rg = (M + p.nrg - 1) / p.nrg;
-  p.ck = min(64, 4096 >> a.dkv_shift);
-  const int pst = a.dkv + MG_PST_PAD;
+  p.ck = a.dkv > 64 ? 16 : 64;   // chunk buffers (2 x keys + values) take at most 64 KB of the staging area
   int ns = max(1, G / (a.H * p.nrg));
   ns = min(ns, max(1, nkeys / 32));
-  const int room = MG_ACT - M * a.I * 4;
-  ns = min(ns, max(1, room / (M * a.H * pst * 4)));
-  if (M > 8) ns = 1;   // the merging projection stages all rows at once
-  p.ns = max(1, ns);
+  p.ns = min(ns, 8);
+  p.per = (nkeys + p.ns - 1) / p.ns;
   return p;
 }
 
 // ---- attention stage ---------------------------------------------------------------------
 // mode 0: cross (all encoder keys, no bias), mode 1: self (row i sees keys 0..pos0+i, bias by distance)
-__device__ void mg_attention(const MegaArgs& a, MegaShared* sh, float* act, float* scratch, MegaBarrier& gb, int layer,
-                             int mode, int M, int pos0, unsigned& kvfill) {
+__device__ void mg_attention(const MegaArgs& a, MegaShared* sh, float* act, float* scratch, int layer, int mode, int M, int pos0,
+                             int nkeys, const MegaAttnPlan& P, const uint2* llin, uint2* llout, uint2* llrec, uint32_t ep_in,
+                             uint32_t ep_out, unsigned& kvfill, unsigned char* ring, MegaFeed& feed, int& pending) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, H = a.H, dkv = a.dkv, dsh = a.dkv_shift;
-  const int nkeys = mode == 0 ? min(*a.enc_len, a.ecap) : min(pos0 + M, a.cap);
-  const MegaAttnPlan P = mg_attn_plan(a, M, nkeys, G);
   const int units = H * P.nrg * P.ns;
   const int kcap = mode == 0 ? a.ecap : a.cap;
   const size_t kvoff = (size_t)layer * H * dkv * kcap;
-  const float* Kb = (mode == 0 ? a.crossK : a.selfK) + kvoff;
-  const float* Vb = (mode == 0 ? a.crossV : a.selfV) + kvoff;
-  const int ck = P.ck, chunk_floats = ck * dkv;
-  float* sQ = scratch;                    // [rg][dkv]
-  float* sS = scratch + 4 * 128;          // [rg][ck]
-  const int pst = dkv + MG_PST_PAD;
-  bool waited = false;
+  const int ck = P.ck, chunk_floats = ck * dkv, pst = dkv + MG_PST_PAD;
+  float* sS = scratch;                    // [rg][ck] scores, then probabilities
+  float* sBias = scratch + 4 * 64;        // bias by distance, the distances this unit meets
+  const int ck_sh = 31 - __clz(ck);
+  const int bias_cap = MG_PSUM / 4 - 4 * 64;
+  float* sIn = act + 4 * chunk_floats;    // what arrives as pairs: self [M][q | k | v][dkv], cross [rows][dkv]
+  float* sRec = act;                      // records of the other splits (after the chunks are done)
+  const int in_st = mode == 1 ? 3 * dkv : dkv;   // floats between the rows of sIn
 #pragma unroll 1
-  for (int u = blockIdx.x; u < units || !waited; u += G) {
-    const bool active = u < units;
-    int h = 0, g = 0, sp = 0, j0 = 0, j1 = 0, nchunks = 0;
-    if (active) {
-      h = u % H;
-      const int rest = u / H;
-      g = rest % P.nrg;
-      sp = rest / P.nrg;
-      const int per = (nkeys + P.ns - 1) / P.ns;
-      j0 = sp * per;
-      j1 = min(nkeys, j0 + per);
-      nchunks = j1 > j0 ? (j1 - j0 + ck - 1) / ck : 0;
-    }
-    const float* Kh = Kb + (size_t)h * kcap * dkv;
-    const float* Vh = Vb + (size_t)h * kcap * dkv;
-    auto issue = [&](int c) {   // thread 0: chunk c of this unit into buffer (kvfill & 1)
-      const int nk = min(ck, j1 - (j0 + c * ck));
-      const unsigned buf = kvfill & 1;
-      const uint32_t bar = smem_u32(&sh->kvbar[buf]);
-      const uint32_t bytes = (uint32_t)(nk * dkv * 4);
-      mg_mbar_expect(bar, 2 * bytes);
-      mg_bulk_g2s(smem_u32(act + (size_t)buf * 2 * chunk_floats), Kh + (size_t)(j0 + c * ck) * dkv, bytes, bar);
-      mg_bulk_g2s(smem_u32(act + (size_t)buf * 2 * chunk_floats + chunk_floats), Vh + (size_t)(j0 + c * ck) * dkv, bytes, bar);
-      ++kvfill;
-    };
-    // cross keys / values never change while decoding: the first chunks may start before the barrier
-    const bool early = mode == 0 && !waited;
-    unsigned fill0 = kvfill;
-    if (early && tid == 0 && active) {
-      if (nchunks > 0) issue(0);
-      if (nchunks > 1) issue(1);
-    }
-    if (!waited) { mg_wait_grid(gb, sh, a.err); waited = true; }
-    if (!active) break;
-    if (tid == 0) {
-      if (!early) {
-        if (nchunks > 0) issue(0);
-        if (nchunks > 1) issue(1);
-      }
-    }
-    if (tid != 0) kvfill = fill0 + min(nchunks, 2);   // every thread tracks the fill count
+  for (int u = blockIdx.x; u < units; u += G) {
+    mg_csync();   // the scratch area may still be read as the partial sums of the stage before
+    if (tid == MG_FEEDER && pending) mg_feed(a, sh, ring, feed, pending);
+    pending = 0;
+    const int h = u % H, rest = u / H, g = rest % P.nrg, sp = rest / P.nrg;
+    const int j0 = min(nkeys, sp * P.per), j1 = min(nkeys, j0 + P.per);
+    const int jo1 = mode == 1 ? min(j1, pos0) : j1;                 // cached keys [j0, jo1)
+    const int jn0 = mode == 1 ? max(j0, pos0) : j1;                 // keys of this pass [jn0, j1)
+    const int nold = jo1 > j0 ? (jo1 - j0 + ck - 1) >> ck_sh : 0;
+    const int nchunks = nold + (j1 > jn0 ? 1 : 0);
+    const float* Kh = (mode == 0 ? a.crossK : a.selfK) + kvoff + (size_t)h * kcap * dkv;
+    const float* Vh = (mode == 0 ? a.crossV : a.selfV) + kvoff + (size_t)h * kcap * dkv;
     const int i0 = g * P.rg, nr = min(P.rg, M - i0);
-    // queries of the unit's rows
-    for (int idx = tid; idx < nr * (dkv >> 2); idx += MG_CONSUMERS) {
-      const int i = idx / (dkv >> 2), e4 = (idx - i * (dkv >> 2)) << 2;
-      *reinterpret_cast<float4*>(sQ + i * dkv + e4) =
-          __ldcg(reinterpret_cast<const float4*>(a.q + (size_t)(i0 + i) * a.I + h * dkv + e4));
+    // the cache does not change during the pass: its first chunks start before the queries arrive
+    const unsigned fill0 = kvfill;
+    int issued = 0;   // cached chunks requested so far
+    auto issue_to = [&](int upto) {
+#pragma unroll 1
+      for (; issued < upto; ++issued, ++kvfill) {
+        if (tid != 0) continue;
+        const int jc = j0 + (issued << ck_sh), nk = min(ck, jo1 - jc);
+        const unsigned buf = kvfill & 1;
+        const uint32_t bar = smem_u32(&sh->kvbar[buf]), bytes = (uint32_t)(nk * dkv * 4);
+        mg_mbar_expect(bar, 2 * bytes);
+        mg_bulk_g2s(smem_u32(act + (size_t)buf * 2 * chunk_floats), Kh + (size_t)jc * dkv, bytes, bar);
+        mg_bulk_g2s(smem_u32(act + (size_t)buf * 2 * chunk_floats + chunk_floats), Vh + (size_t)jc * dkv, bytes, bar);
+      }
+    };
+    issue_to(min(nold, 2));
+    // bias of the distances pos0 + i - j of this unit (a static table)
+    const int dmin = max(0, pos0 + i0 - (j1 - 1)), dmax = pos0 + i0 + nr - 1 - j0;
+    const bool bias_staged = mode == 1 && dmax - dmin + 1 <= bias_cap;
+    if (bias_staged)
+      for (int dd = dmin + tid; dd <= dmax; dd += MG_CONSUMERS) sBias[dd - dmin] = __ldg(a.dec_bias + (size_t)h * a.cap + dd);
+    // what arrives as pairs: all rows of this head (self: the new keys / values are among them), or the unit's queries
+    const float* sQ;
+    if (mode == 1) {
+      mg_ll_fetch(llin + (size_t)h * MAXB * 3 * dkv, (M * 3 * dkv) >> 1, sIn, ep_in, sh, a.err);
+      sQ = sIn + (size_t)i0 * 3 * dkv;
+    } else {
+      mg_ll_fetch(llin + ((size_t)h * MAXB + i0) * dkv, (nr * dkv) >> 1, sIn, ep_in, sh, a.err);
+      sQ = sIn;
     }
     if (tid < 4) { sh->amax[tid] = -INFINITY; sh->asum[tid] = 0.f; sh->ascale[tid] = 1.f; }
     // thread <-> (row, channel) of the weighted values
@@ -395,47 +427,52 @@ __device__ void mg_attention(const MegaArgs& a, MegaShared* sh, float* act, floa
     mg_csync();
     unsigned use = fill0;
 #pragma unroll 1
-    for (int c = 0; c < nchunks; ++c, ++use) {
+    for (int c = 0; c < nchunks; ++c) {
+      const bool cached = c < nold;
       const unsigned buf = use & 1;
-      const float* sK = act + (size_t)buf * 2 * chunk_floats;
-      const float* sV = sK + chunk_floats;
-      const int jc = j0 + c * ck, nk = min(ck, j1 - jc);
-      mg_wait(sh, a.err, &sh->kvbar[buf], (use >> 1) & 1);
+      const float* sK = cached ? act + (size_t)buf * 2 * chunk_floats : sIn + (size_t)(jn0 - pos0) * 3 * dkv + dkv;
+      const float* sV = cached ? sK + chunk_floats : sK + dkv;
+      const int kst = cached ? dkv : 3 * dkv;
+      const int jc = cached ? j0 + (c << ck_sh) : jn0, nk = cached ? min(ck, jo1 - jc) : j1 - jn0;
+      if (cached) mg_wait(sh, a.err, &sh->kvbar[buf], (use >> 1) & 1);
       // scores: one (row, key) pair per thread; the columns are visited in a rotated order so that
       // the threads of a quarter warp hit different banks
-      for (int idx = tid; idx < nr * ck; idx += MG_CONSUMERS) {
-        const int i = idx / ck, jj = idx - i * ck;
-        float s = -INFINITY;
-        if (jj < nk) {
-          const int j = jc + jj;
-          const bool seen = mode == 0 || j <= pos0 + i0 + i;
-          if (seen) {
-            float accs = 0.f;
-            const int nq4 = dkv >> 2;
+#pragma unroll 1
+      for (int idx = tid; idx < (nr << ck_sh); idx += MG_CONSUMERS) {
+        const int i = idx >> ck_sh, jj = idx & (ck - 1);
+        float sc = -INFINITY;
+        const int j = jc + jj;
+        if (jj < nk && (mode == 0 || j <= pos0 + i0 + i)) {
+          float accs = 0.f;
+          const int nq4 = dkv >> 2;
 #pragma unroll 4
-            for (int e = 0; e < nq4; ++e) {
-              const int er = ((e + jj) & (nq4 - 1)) << 2;
-              const float4 kv = *reinterpret_cast<const float4*>(sK + jj * dkv + er);
-              const float4 qv = *reinterpret_cast<const float4*>(sQ + i * dkv + er);
-              accs += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
-            }
-            if (mode == 1) accs += a.dec_bias[(size_t)h * a.cap + (pos0 + i0 + i - j)];
-            s = accs;
+          for (int e = 0; e < nq4; ++e) {
+            const int er = ((e + jj) & (nq4 - 1)) << 2;
+            const float4 kv = *reinterpret_cast<const float4*>(sK + jj * kst + er);
+            const float4 qv = *reinterpret_cast<const float4*>(sQ + i * in_st + er);
+            accs += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
           }
+          if (mode == 1) {
+            const int dd = pos0 + i0 + i - j;
+            accs += bias_staged ? sBias[dd - dmin] : __ldg(a.dec_bias + (size_t)h * a.cap + dd);
+          }
+          sc = accs;
         }
-        sS[i * ck + jj] = s;
+        sS[idx] = sc;
       }
       mg_csync();
       if (warp < nr) {   // running soft-max of row `warp`
         float mx = -INFINITY;
-        for (int jj = lane; jj < ck; jj += 32) mx = fmaxf(mx, sS[warp * ck + jj]);
+#pragma unroll 1
+        for (int jj = lane; jj < ck; jj += 32) mx = fmaxf(mx, sS[(warp << ck_sh) + jj]);
         mx = warp_max(mx);
         const float mo = sh->amax[warp], mn = fmaxf(mo, mx);
         float sum = 0.f;
+#pragma unroll 1
         for (int jj = lane; jj < ck; jj += 32) {
-          const float sc = sS[warp * ck + jj];
-          const float pr = sc == -INFINITY ? 0.f : __expf(sc - mn);
-          sS[warp * ck + jj] = pr;
+          const float scv = sS[(warp << ck_sh) + jj];
+          const float pr = scv == -INFINITY ? 0.f : __expf(scv - mn);
+          sS[(warp << ck_sh) + jj] = pr;
           sum += pr;
         }
         sum = warp_sum(sum);
@@ -449,64 +486,101 @@ __device__ void mg_attention(const MegaArgs& a, MegaShared* sh, float* act, floa
       mg_csync();
       if (pv_on) {
         float a0 = 0.f, a1 = 0.f;
-        const float* pr = sS + pv_i * ck;
+        const float* pr = sS + (pv_i << ck_sh);
         int jj = 0;
-#pragma unroll 4
+#pragma unroll 2
         for (; jj + 1 < nk; jj += 2) {
-          a0 += pr[jj] * sV[jj * dkv + pv_c];
-          a1 += pr[jj + 1] * sV[(jj + 1) * dkv + pv_c];
+          a0 += pr[jj] * sV[jj * kst + pv_c];
+          a1 += pr[jj + 1] * sV[(jj + 1) * kst + pv_c];
         }
-        if (jj < nk) a0 += pr[jj] * sV[jj * dkv + pv_c];
+        if (jj < nk) a0 += pr[jj] * sV[jj * kst + pv_c];
         pv_acc = pv_acc * sh->ascale[pv_i] + (a0 + a1);
       }
       mg_csync();   // the chunk's buffer and the probabilities are free again
-      if (tid == 0 && c + 2 < nchunks) issue(c + 2);
-      if (tid != 0 && c + 2 < nchunks) ++kvfill;
-    }
-    if (pv_on) {
-      const int i = i0 + pv_i;
-      if (P.ns == 1) {
-        const float l = sh->asum[pv_i];
-        a.att[(size_t)i * a.I + h * dkv + pv_c] = l > 0.f ? pv_acc / l : 0.f;
-      } else {
-        float* rec = a.part + ((size_t)(i * H + h) * P.ns + sp) * pst;
-        rec[MG_PST_PAD + pv_c] = pv_acc;
-        if (pv_c == 0) { rec[0] = sh->amax[pv_i]; rec[1] = sh->asum[pv_i]; }
+      if (cached) {
+        issue_to(min(nold, c + 3));
+        ++use;
       }
+    }
+    // finish: a lone split writes the rows, later splits leave records, the first split merges them
+    const int slot = (h * P.nrg + g) * 32 * pst;   // pairs: [split - 1][row < rg][pst], at most 7 x 4 rows
+    if (sp > 0) {
+      if (pv_i < P.rg) {
+        uint2* rec = llrec + slot + ((size_t)(sp - 1) * P.rg + pv_i) * pst;
+        mg_ll_store(rec + MG_PST_PAD + pv_c, pv_on ? pv_acc : 0.f, ep_out);
+        if (pv_c < MG_PST_PAD)
+          mg_ll_store(rec + pv_c, pv_c == 0 ? (pv_on ? sh->amax[pv_i] : -INFINITY) : pv_c == 1 ? (pv_on ? sh->asum[pv_i] : 0.f) : 0.f, ep_out);
+      }
+    } else {
+      float mx = pv_on ? sh->amax[pv_i] : -INFINITY, l = pv_on ? sh->asum[pv_i] : 0.f;
+      if (P.ns > 1) {
+        mg_ll_fetch(llrec + slot, ((P.ns - 1) * P.rg * pst) >> 1, sRec, ep_out, sh, a.err);
+        mg_csync();
+        if (pv_on) {
+          float gm = mx;
+#pragma unroll 1
+          for (int s2 = 1; s2 < P.ns; ++s2) gm = fmaxf(gm, sRec[((s2 - 1) * P.rg + pv_i) * pst]);
+          const float w0 = mx == -INFINITY ? 0.f : __expf(mx - gm);
+          float num = pv_acc * w0, den = l * w0;
+#pragma unroll 1
+          for (int s2 = 1; s2 < P.ns; ++s2) {
+            const float* rec = sRec + ((s2 - 1) * P.rg + pv_i) * pst;
+            const float wgt = rec[1] > 0.f ? __expf(rec[0] - gm) : 0.f;
+            den += rec[1] * wgt;
+            num += rec[MG_PST_PAD + pv_c] * wgt;
+          }
+          pv_acc = num;
+          l = den;
+        }
+      }
+      if (pv_on) mg_ll_store(llout + (size_t)(i0 + pv_i) * a.I + h * dkv + pv_c, l > 0.f ? pv_acc / l : 0.f, ep_out);
     }
     mg_csync();
   }
-  mg_arrive(gb);
 }
 
 // ---- linear stage ------------------------------------------------------------------------
-enum { MG_SRC_EMB = 0, MG_SRC_X, MG_SRC_ATT, MG_SRC_ATT_PARTS, MG_SRC_U };
 enum { MG_EPI_QKV = 0, MG_EPI_RESID, MG_EPI_Q, MG_EPI_FFN };
 
-__device__ void mg_linear(const MegaArgs& a, MegaShared* sh, unsigned char* ring, float* act, float* psum, MegaBarrier& gb,
-                          const MegaLin& w, int src, const float* gain, int epi, int layer, int M, int pos0,
-                          const MegaAttnPlan& AP, bool wait_first, bool arrive_last, unsigned& fill, unsigned& actuse) {
+// src == nullptr: the input rows are the embeddings of the tokens (first stage of the pass)
+__device__ void mg_linear(const MegaArgs& a, MegaShared* sh, unsigned char* ring, float* act, float* psum, const MegaLin& w,
+                          int which, const uint2* src, uint32_t ep_in, const float* gain, int epi, uint2* dst, uint32_t ep_out, int layer,
+                          int M, int pos0, bool write_x, int& slot, unsigned& stage, MegaFeed& feed, int& pending) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int G = gridDim.x, K = w.K;
-  int r0, r1;
-  mg_slice(w.N, blockIdx.x, G, &r0, &r1);
+  const int K = w.K;
+  const int r0 = sh->slice[which][0], r1 = sh->slice[which][1];
   const int n = r1 - r0, nmat = w.W1 ? 2 : 1;
-  MegaRows R;
-  R.ring = ring; R.ns = a.nslots; R.slot0 = fill % a.nslots; R.rowbytes = K * 2; R.rps = MG_SLOT / R.rowbytes;
-  const int slots_mat = (n + R.rps - 1) / R.rps;
-  R.n0 = nmat == 2 ? n : 0x7fffffff; R.slots0 = slots_mat;
-  const int nslots_stage = slots_mat * nmat, nrows = n * nmat;
-  // before the barrier: clear the partial sums
-  for (int i = tid; i < MG_PSUM / 4; i += MG_CONSUMERS) psum[i] = 0.f;
-  if (wait_first) mg_wait_grid(gb, sh, a.err); else mg_csync();
+  if (n == 0) return;   // nothing to produce: the block needs neither the input nor any weights
+  const int rowbytes = K * 2, rps = MG_SLOT / rowbytes;
+  const int slots_mat = (n + rps - 1) / rps, nslots_stage = slots_mat * nmat, nrows = n * nmat;
+  if (tid < nrows) {   // where each slice row sits in the ring
+    int r = tid, s = slot;
+    if (r >= n) { r -= n; s += slots_mat; }
+    s += r / rps;
+    if (s >= a.nslots) s -= a.nslots;
+    if (s >= a.nslots) s -= a.nslots;
+    sh->rowoff[tid] = (unsigned)(s * MG_SLOT + (r % rps) * rowbytes);
+  }
+  // the slots the previous linear stage handed back take the next slices while the inputs arrive
+  if (tid == MG_FEEDER && pending) mg_feed(a, sh, ring, feed, pending);
+  pending = nslots_stage;
+  const int nkb = (K + 255) >> 8;
+  float4 gv[2];   // gains of the columns this thread scales (K <= 2048 where a norm precedes)
+  if (gain) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int c = tid * 4 + j * 1024;
+      gv[j] = c < K ? __ldg(reinterpret_cast<const float4*>(gain + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
   // token rows in groups that fit the staging area
-  int rgl = min(8, MG_ACT / (K * 4));
-  if (src == MG_SRC_ATT_PARTS) rgl = min(rgl, M);   // plan guarantees records + rows fit for all M rows
+  const int cap_rows = MG_ACT / (K * 4);
+  const int rgl = cap_rows >= 8 ? 8 : cap_rows >= 4 ? 4 : cap_rows >= 2 ? 2 : 1;
 #pragma unroll 1
   for (int m0 = 0; m0 < M; m0 += rgl) {
     const int mg = min(rgl, M - m0);
     float* Xs = act;
-    if (src == MG_SRC_EMB) {
+    if (!src) {
       for (int idx = tid; idx < mg * (K >> 3); idx += MG_CONSUMERS) {
         const int m = idx / (K >> 3), c8 = (idx - m * (K >> 3)) << 3;
         int t = a.desc->tokens[m0 + m];
@@ -516,78 +590,50 @@ __device__ void mg_linear(const MegaArgs& a, MegaShared* sh, unsigned char* ring
         *reinterpret_cast<float4*>(Xs + (size_t)m * K + c8) = make_float4(v[0], v[1], v[2], v[3]);
         *reinterpret_cast<float4*>(Xs + (size_t)m * K + c8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
       }
-      // the residual stream starts as the embedding: every block writes its share of the columns
-      mg_csync();
-      int c_lo, c_hi;
-      mg_slice(K, blockIdx.x, G, &c_lo, &c_hi);
-      for (int idx = tid; idx < mg * (c_hi - c_lo); idx += MG_CONSUMERS) {
-        const int m = idx / (c_hi - c_lo), c = c_lo + idx - m * (c_hi - c_lo);
-        a.x[(size_t)(m0 + m) * a.d + c] = Xs[(size_t)m * K + c];
-      }
-    } else if (src == MG_SRC_ATT_PARTS) {
-      const int pst = a.dkv + MG_PST_PAD;
-      const uint32_t bytes = (uint32_t)(M * a.H * AP.ns * pst * 4);
-      float* stage = act + (size_t)M * K;     // K == I
-      if (tid == 0) {
-        const uint32_t bar = smem_u32(&sh->actbar);
-        mg_mbar_expect(bar, bytes);
-        mg_bulk_g2s(smem_u32(stage), a.part, bytes, bar);
-      }
-      mg_wait(sh, a.err, &sh->actbar, actuse & 1);
-      ++actuse;
-      for (int idx = tid; idx < M * K; idx += MG_CONSUMERS) {
-        const int i = idx / K, nn = idx - i * K, h = nn >> a.dkv_shift, c = nn & (a.dkv - 1);
-        const float* rec = stage + (size_t)(i * a.H + h) * AP.ns * pst;
-        float gm = -INFINITY;
-        for (int s = 0; s < AP.ns; ++s) gm = fmaxf(gm, rec[s * pst]);
-        float num = 0.f, den = 0.f;
-        for (int s = 0; s < AP.ns; ++s) {
-          const float l = rec[s * pst + 1];
-          const float wgt = l > 0.f ? __expf(rec[s * pst] - gm) : 0.f;
-          den += l * wgt;
-          num += rec[s * pst + MG_PST_PAD + c] * wgt;
-        }
-        Xs[idx] = den > 0.f ? num / den : 0.f;
-      }
     } else {
-      const float* srcp = src == MG_SRC_X ? a.x : src == MG_SRC_ATT ? a.att : a.u;
-      const uint32_t bytes = (uint32_t)(mg * K * 4);
-      if (tid == 0) {
-        const uint32_t bar = smem_u32(&sh->actbar);
-        mg_mbar_expect(bar, bytes);
-        mg_bulk_g2s(smem_u32(Xs), srcp + (size_t)m0 * K, bytes, bar);
-      }
-      mg_wait(sh, a.err, &sh->actbar, actuse & 1);
-      ++actuse;
+      mg_ll_fetch(src + (size_t)m0 * K, (mg * K) >> 1, Xs, ep_in, sh, a.err);
     }
-    if (src == MG_SRC_EMB || src == MG_SRC_ATT_PARTS) mg_csync();
+    mg_csync();
     if (gain) {   // T5 norm: x * g / sqrt(mean(x^2) + eps); the division is applied to the dot products
-      for (int m = warp; m < mg; m += 8) {
+      // thread t scales columns 4t .. 4t+3 (+ 1024, ...) of every row; the gains were requested before the rows arrived
+      for (int m = 0; m < mg; ++m) {
         float ss = 0.f;
-        for (int c = lane * 4; c < K; c += 128) {
-          float4 v = *reinterpret_cast<float4*>(Xs + (size_t)m * K + c);
-          const float4 gv = __ldg(reinterpret_cast<const float4*>(gain + c));
-          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-          v.x *= gv.x; v.y *= gv.y; v.z *= gv.z; v.w *= gv.w;
-          *reinterpret_cast<float4*>(Xs + (size_t)m * K + c) = v;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int c = tid * 4 + j * 1024;
+          if (c < K) {
+            float4 v = *reinterpret_cast<float4*>(Xs + (size_t)m * K + c);
+            ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+            v.x *= gv[j].x; v.y *= gv[j].y; v.z *= gv[j].z; v.w *= gv[j].w;
+            *reinterpret_cast<float4*>(Xs + (size_t)m * K + c) = v;
+          }
         }
         ss = warp_sum(ss);
-        if (lane == 0) sh->inv[m] = rsqrtf(ss / (float)K + a.eps);
+        if (lane == 0) sh->ssq[warp][m] = ss;
       }
       mg_csync();
+      if (tid < mg) {
+        float ss = 0.f;
+#pragma unroll
+        for (int wv = 0; wv < 8; ++wv) ss += sh->ssq[wv][tid];
+        sh->inv[tid] = rsqrtf(ss / (float)K + a.eps);
+      }
     }
-    if (m0 == 0)
-      for (int s = 0; s < nslots_stage; ++s) mg_wait(sh, a.err, &sh->full[(fill + s) % a.nslots], ((fill + s) / a.nslots) & 1);
-    mg_items_dyn(mg, R, nrows, K, Xs, psum, warp, lane);
+    if (m0 == 0) mg_wait(sh, a.err, &sh->full[stage % MG_MAX_SLOTS], (stage / MG_MAX_SLOTS) & 1);
+    const int mgr = mg_round_rows(mg);
+    mg_items_dyn(mgr, ring, sh->rowoff, nrows, K, Xs, psum, warp, lane);
     mg_csync();
-    // epilogue: one (output row, token row) pair per thread, partial sums added in warp order
-    for (int idx = tid; idx < n * mg; idx += MG_CONSUMERS) {
-      const int r = idx / mg, m = idx - r * mg;
+    // epilogue: (output row r, token row m); the partial sums of a quad are added in warp order
+    for (int m = tid >> 6; m < mg; m += 4) {
+      const int r = tid & 63;
+      if (r >= n) continue;
       auto total = [&](int row) {
-        const float* p = psum + (size_t)((row >> 2) * 8) * 32 + (row & 3) * mg + m;
+        const int qd = row >> 2, first = qd * nkb;
+        const float* p = psum + (size_t)(qd * 8) * 32 + (row & 3) * mgr + m;
         float s = 0.f;
 #pragma unroll
-        for (int wv = 0; wv < 8; ++wv) s += p[wv * 32];
+        for (int wv = 0; wv < 8; ++wv)
+          if (((wv - first) & 7) < nkb) s += p[wv * 32];   // warp wv took part in this quad
         return s;
       };
       float v = total(r);
@@ -597,35 +643,29 @@ __device__ void mg_linear(const MegaArgs& a, MegaShared* sh, unsigned char* ring
         int part = 0, rr = nn;
         if (rr >= a.I) { rr -= a.I; ++part; }
         if (rr >= a.I) { rr -= a.I; ++part; }
-        if (part == 0) a.q[(size_t)mm * a.I + rr] = v;
-        else {
-          const int h = rr >> a.dkv_shift, c = rr & (a.dkv - 1), row = pos0 + mm;
-          if (row < a.cap) (part == 1 ? a.selfK : a.selfV)[(((size_t)layer * a.H + h) * a.cap + row) * a.dkv + c] = v;
-        }
+        const int h = rr >> a.dkv_shift, c = rr & (a.dkv - 1), row = pos0 + mm;
+        mg_ll_store(dst + (((size_t)h * MAXB + mm) * 3 + part) * a.dkv + c, v, ep_out);
+        if (part > 0 && row < a.cap) (part == 1 ? a.selfK : a.selfV)[(((size_t)layer * a.H + h) * a.cap + row) * a.dkv + c] = v;
       } else if (epi == MG_EPI_RESID) {
-        a.x[(size_t)mm * a.d + nn] += v;
+        const float xn = sh->xres[mm][r] + v;
+        sh->xres[mm][r] = xn;
+        mg_ll_store(dst + (size_t)mm * a.d + nn, xn, ep_out);
+        if (write_x) a.x[(size_t)mm * a.d + nn] = xn;
       } else if (epi == MG_EPI_Q) {
-        a.q[(size_t)mm * a.I + nn] = v;
+        mg_ll_store(dst + ((size_t)(nn >> a.dkv_shift) * MAXB + mm) * a.dkv + (nn & (a.dkv - 1)), v, ep_out);
       } else {
-        if (nmat == 2) {
-          const float v1 = total(n + r) * sh->inv[m];
-          a.u[(size_t)mm * a.F + nn] = gelu_tanh(v) * v1;
-        } else {
-          a.u[(size_t)mm * a.F + nn] = fmaxf(v, 0.f);
-        }
+        float uo;
+        if (nmat == 2) uo = gelu_tanh(v) * (total(n + r) * sh->inv[m]);
+        else uo = fmaxf(v, 0.f);
+        mg_ll_store(dst + (size_t)mm * a.F + nn, uo, ep_out);
       }
     }
-    if (m0 + rgl < M) {   // another group of token rows follows
-      mg_csync();
-      for (int i = tid; i < MG_PSUM / 4; i += MG_CONSUMERS) psum[i] = 0.f;
-      mg_csync();
-    }
+    if (m0 + rgl < M) mg_csync();   // another group of token rows: staged rows and partial sums are reused
   }
-  mg_csync();   // all warps are done with the weights (and the staged rows)
-  if (tid == 0)
-    for (int s = 0; s < nslots_stage; ++s) mg_mbar_arrive(smem_u32(&sh->empty[(fill + s) % a.nslots]));
-  fill += nslots_stage;
-  if (arrive_last) mg_arrive(gb);
+  slot += nslots_stage;
+  if (slot >= a.nslots) slot -= a.nslots;
+  if (slot >= a.nslots) slot -= a.nslots;
+  ++stage;
 }
 
 // ---- the pass ----------------------------------------------------------------------------
@@ -637,49 +677,81 @@ __global__ void __launch_bounds__(MG_THREADS, 1) mega_pass_kernel(MegaArgs a) {
   MegaShared* sh = reinterpret_cast<MegaShared*>(psum + MG_PSUM / 4);
   const int tid = threadIdx.x;
   if (tid == 0) {
-    for (int i = 0; i < a.nslots; ++i) { mg_mbar_init(smem_u32(&sh->full[i]), 1); mg_mbar_init(smem_u32(&sh->empty[i]), 1); }
-    mg_mbar_init(smem_u32(&sh->actbar), 1);
+    for (int i = 0; i < MG_MAX_SLOTS; ++i) mg_mbar_init(smem_u32(&sh->full[i]), 1);
     mg_mbar_init(smem_u32(&sh->kvbar[0]), 1);
     mg_mbar_init(smem_u32(&sh->kvbar[1]), 1);
     sh->failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (tid < 6) {
+    const int Ns[6] = {3 * a.I, a.d, a.I, a.d, a.F, a.d};
+    mg_slice(Ns[tid], blockIdx.x, gridDim.x, &sh->slice[tid][0], &sh->slice[tid][1]);
+  }
+  for (int i = tid; i < a.n_layers * (int)(sizeof(MegaLayer) / 8); i += MG_CONSUMERS)
+    reinterpret_cast<unsigned long long*>(sh->layers)[i] = reinterpret_cast<const unsigned long long*>(a.layers)[i];
   __syncthreads();
-  if (tid >= MG_CONSUMERS) {
-    if (tid == MG_CONSUMERS) mg_producer(a, sh, ring);
-    return;
+  MegaFeed feed;
+  feed.done = true; feed.slot = 0; feed.stage = 0;
+  if (tid == MG_FEEDER) {   // the weights do not wait for anything: start the stream
+    mg_feed_init(a, sh, feed);
+    mg_feed(a, sh, ring, feed, a.nslots);
   }
   const int M = max(1, min(a.desc->k, MAXB)), pos0 = a.desc->pos0;
-  const unsigned par = a.sync[2] & 1u;
-  MegaBarrier gb;
-  gb.ctr = a.sync + par;
-  gb.done = 0;
-  if (blockIdx.x == 0 && tid == 0) a.sync[par ^ 1u] = 0;   // the next launch counts from zero
-  unsigned fill = 0, actuse = 0, kvfill = 0;
+  const unsigned seq = *(volatile unsigned*)a.sync;
+  const uint32_t ep0 = seq * MG_EPOCHS_PER_LAUNCH + 1;
+  int slot = 0;
+  unsigned stage = 0, kvfill = 0;
+  int pending = 0;   // slots to refill at the next opportunity
   const int G = gridDim.x;
   const int ekeys = min(*a.enc_len, a.ecap), skeys = min(pos0 + M, a.cap);
   const MegaAttnPlan plan_self = mg_attn_plan(a, M, skeys, G), plan_cross = mg_attn_plan(a, M, ekeys, G);
-#pragma unroll 1
-  for (int l = 0; l < a.n_layers; ++l) {
-    const MegaLayer L = a.layers[l];
-    const bool last = l + 1 == a.n_layers;
-    // norm + QKV, K/V appended to the cache
-    mg_linear(a, sh, ring, act, psum, gb, mg_lin(a, L, 0), l == 0 ? MG_SRC_EMB : MG_SRC_X, L.ln1, MG_EPI_QKV, l, M, pos0,
-              plan_self, l != 0, true, fill, actuse);
-    mg_attention(a, sh, act, psum, gb, l, 1, M, pos0, kvfill);
-    mg_linear(a, sh, ring, act, psum, gb, mg_lin(a, L, 1), plan_self.ns > 1 ? MG_SRC_ATT_PARTS : MG_SRC_ATT, nullptr,
-              MG_EPI_RESID, l, M, pos0, plan_self, true, true, fill, actuse);
-    mg_linear(a, sh, ring, act, psum, gb, mg_lin(a, L, 2), MG_SRC_X, L.ln2, MG_EPI_Q, l, M, pos0, plan_self, true, true,
-              fill, actuse);
-    mg_attention(a, sh, act, psum, gb, l, 0, M, pos0, kvfill);
-    mg_linear(a, sh, ring, act, psum, gb, mg_lin(a, L, 3), plan_cross.ns > 1 ? MG_SRC_ATT_PARTS : MG_SRC_ATT, nullptr,
-              MG_EPI_RESID, l, M, pos0, plan_cross, true, true, fill, actuse);
-    mg_linear(a, sh, ring, act, psum, gb, mg_lin(a, L, 4), MG_SRC_X, L.ln3, MG_EPI_FFN, l, M, pos0, plan_self, true, true,
-              fill, actuse);
-    mg_linear(a, sh, ring, act, psum, gb, mg_lin(a, L, 5), MG_SRC_U, nullptr, MG_EPI_RESID, l, M, pos0, plan_self, true,
-              !last, fill, actuse);
+  {   // the residual stream starts as the embedding: this block keeps the columns it owns
+    const int c_lo = sh->slice[1][0], c_hi = sh->slice[1][1];
+    for (int idx = tid; idx < M * MG_XRES; idx += MG_CONSUMERS) {
+      const int m = idx / MG_XRES, c = idx - m * MG_XRES;
+      if (c < c_hi - c_lo) {
+        int t = a.desc->tokens[m];
+        t = t < 0 ? 0 : (t >= a.vocab ? a.vocab - 1 : t);
+        sh->xres[m][c] = __bfloat162float(a.emb[(size_t)t * a.d + c_lo + c]);
+      }
+    }
   }
-  if (blockIdx.x == 0 && tid == 0) a.sync[2] = par ^ 1u;
+  // stage s of layer l writes epoch ep0 + 8 l + s; stages 1 and 4 are the attentions
+  const int n_stages = 8 * a.n_layers;
+#pragma unroll 1
+  for (int st = 0; st < n_stages; ++st) {
+    const int l = st >> 3, sg = st & 7;
+    const uint32_t ep_out = ep0 + st, ep_in = ep_out - 1;
+    if (sg == 1 || sg == 4) {
+      const bool self = sg == 1;
+      mg_attention(a, sh, act, psum, l, self ? 1 : 0, M, pos0, self ? skeys : ekeys, self ? plan_self : plan_cross,
+                   self ? a.ll.qkv1 : a.ll.q4, self ? a.ll.a2 : a.ll.a5, self ? a.ll.r2 : a.ll.r5, ep_in, ep_out, kvfill, ring, feed,
+                   pending);
+    } else {
+      const MegaLayer& L = sh->layers[l];
+      const int p = sg == 0 ? 0 : sg == 2 ? 1 : sg == 3 ? 2 : sg - 2;     // which of the six matrices
+      const uint2* src = sg == 0 ? (l == 0 ? nullptr : a.ll.x8) : sg == 2 ? a.ll.a2 : sg == 3 ? a.ll.x3 : sg == 5 ? a.ll.a5
+                         : sg == 6 ? a.ll.x6 : a.ll.u7;
+      uint2* dst = sg == 0 ? a.ll.qkv1 : sg == 2 ? a.ll.x3 : sg == 3 ? a.ll.q4 : sg == 5 ? a.ll.x6 : sg == 6 ? a.ll.u7 : a.ll.x8;
+      const float* gain = sg == 0 ? L.ln1 : sg == 3 ? L.ln2 : sg == 6 ? L.ln3 : nullptr;
+      const int epi = sg == 0 ? MG_EPI_QKV : sg == 3 ? MG_EPI_Q : sg == 6 ? MG_EPI_FFN : MG_EPI_RESID;
+      mg_linear(a, sh, ring, act, psum, mg_lin(a, L, p), p, src, ep_in, gain, epi, dst, ep_out, l, M, pos0,
+                sg == 7 && l + 1 == a.n_layers, slot, stage, feed, pending);
+    }
+  }
+  // Every slice that was issued has been waited for by its stage (the program ends with the last
+  // stage), so nothing is in flight into this block's shared memory when it exits - unless a wait
+  // gave up: then the stages' barriers are polled once more, each with a limit.
+  if (tid == MG_FEEDER && *(volatile int*)&sh->failed) {
+    for (unsigned st2 = stage > (unsigned)MG_MAX_SLOTS ? stage - MG_MAX_SLOTS : 0; st2 < stage; ++st2) {
+      const uint32_t bar = smem_u32(&sh->full[st2 % MG_MAX_SLOTS]);
+      for (unsigned it = 0; it < MG_SPIN; ++it)
+        if (mg_mbar_try(bar, (st2 / MG_MAX_SLOTS) & 1)) break;
+    }
+  }
+  // the launch counter moves on once every block has read it: block 0 gets here only after it has
+  // consumed values that every working block produced
+  if (blockIdx.x == 0 && tid == 0) *(volatile unsigned*)a.sync = seq + 1;
 }
 
 }  // namespace bild
