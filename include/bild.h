@@ -215,8 +215,10 @@ int bild_fetch_result(bild_ctx *ctx, int32_t *tokens_out /*HOST*/, int *n_tokens
  * state undefined: call bild_reset or bild_generate afterwards.  Synchronises. */
 int bild_time_pass(bild_ctx *ctx, int which, int k, int cache_len, int iters, float *ms_per_pass /*HOST out*/);
 
-/* 1 if the large model's block pass (k > 1) runs its linear layers on the tcgen05 tensor-core
- * kernel (bf16 weights, d_model / inner / d_ff multiples of 64), 0 if on the SIMT kernels. */
+/* 1 if the tcgen05 tensor-core kernel is in use for this context (bf16 weights, d_model / inner /
+ * d_ff multiples of 64): it runs the encoder's linear layers, and those of the large model's
+ * block pass (k > 1) when the row-slice kernel is switched off (BILD_SLICE=0); 0 if everything
+ * runs on the SIMT kernels. */
 int bild_uses_tensor_cores(const bild_ctx *ctx);
 
 /* Number of kernel launches this context has enqueued since it was created. */

@@ -11,6 +11,7 @@
 
 #include "decode_kernels.cuh"
 #include "mega_pass.cuh"
+#include "slice_linear.cuh"
 #include "umma_linear.cuh"
 
 using namespace bild;
@@ -146,6 +147,10 @@ struct bild_ctx {
   bool block_simt = false;           // block pass on the SIMT block GEMV instead of the tensor-core kernel
   bool use_pdl = true;               // launch pass kernels with programmatic stream serialization
   bool host_loop = false;            // debug: drive the loop from the host, one read-back per step
+  int slice_mode = 2;                // row-slice linear kernel: 0 off, 1 block passes, 2 block and single-row passes
+  int sms = 0;
+  size_t slice_smem_set = 0;
+  size_t slice_min_bytes = 3000 * 1024;   // single-row passes: smaller matrices stay on the GEMV (measured)
   bool mega_coop = true;             // launch the whole-pass kernel with the cooperative attribute
   bool capturing = false;            // launches are being recorded into a graph, not run
   int64_t graph_counted = 0;         // launches of the loop graphs already added to `launches`
@@ -506,8 +511,10 @@ void setup_umma(bild_ctx* c, Model& m) {
 // prepares its arguments (the per-layer pointer table lives in the workspace).
 int setup_mega(bild_ctx* c, Model& m) {
   m.mega = false;
-  const char* off = std::getenv("BILD_NO_MEGA");
-  if (off && off[0] == '1') return BILD_OK;
+  // Opt-in: on B200 the stage-to-stage exchange through L2 (about 2 us per hop) makes the persistent
+  // pass slower than the chain of kernels, whose boundaries cost less.
+  const char* on = std::getenv("BILD_MEGA");
+  if (!(on && on[0] == '1')) return BILD_OK;
   if (c->cfg.dtype != BILD_BF16) return BILD_OK;
   const bild_model_cfg& mc = m.c;
   const int d = mc.d_model, I = m.inner, F = mc.d_ff;
@@ -650,9 +657,44 @@ cudaError_t launch_umma(bild_ctx* c, const LinArgs& a, const CUtensorMap& t0, co
   return cudaLaunchKernelEx(&cfg, umma_linear_kernel<false>, u, t0, t1);
 }
 
+// Row-slice kernel (one block per SM, weights fetched ahead of the dependency wait); false if the shape does not fit.
+bool launch_slice(bild_ctx* c, int MB, const LinArgs& a0, cudaError_t* err) {
+  if (c->cfg.dtype != BILD_BF16 || c->sms < 1 || !a0.desc) return false;
+  const LinArgs& a = a0;
+  const int nmat = a.epi == EPI_GATED ? 2 : 1;
+  const int rows = (a.N + c->sms - 1) / c->sms;
+  if (a.K % 8 || a.ldx != a.K || rows * nmat > 4 * SL_QUADS || (a.gain && a.K > 2048)) return false;
+  if (((uintptr_t)a.W0 & 15) || (nmat == 2 && ((uintptr_t)a.W1 & 15)) || ((uintptr_t)a.X & 15) || (a.gain && ((uintptr_t)a.gain & 15))) return false;
+  SliceArgs s;
+  s.lin = a;
+  s.lin.dkv_shift = ilog2(std::max(1, a.dkv));
+  s.err = &c->st->err;
+  s.w_bytes = (int)align_up((size_t)rows * nmat * a.K * 2, 1024);
+  int xr = MB == 1 ? 1 : 8;
+  while (xr > 1 && (size_t)xr * a.K * 4 > 64 * 1024) xr /= 2;
+  s.x_rows = xr;
+  const size_t smem = slice_smem_bytes(s.w_bytes, xr, a.K);
+  if (smem > 200 * 1024) return false;
+  if (smem > 48 * 1024 && smem > c->slice_smem_set) {
+    if (cudaFuncSetAttribute(slice_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    c->slice_smem_set = 200 * 1024;
+  }
+  *err = launch_k(c, slice_linear_kernel, dim3(c->sms), dim3(SL_THREADS), smem, s);
+  return true;
+}
+
 // Linear layer of a decoder pass: tensor cores for the bf16 block pass, SIMT otherwise.
 cudaError_t launch_dec_linear(bild_ctx* c, Model& m, int MB, const LinArgs& a, int layer, int which_map) {
   int cs, nkb;
+  // single-row passes: only matrices large enough that a block's slice is worth a bulk copy
+  const bool big = (size_t)a.N * a.K * 2 >= c->slice_min_bytes;
+  if (c->slice_mode >= (MB == 1 ? 2 : 1) && (MB != 1 || big) && !c->block_simt) {
+    cudaError_t e = cudaSuccess;
+    if (launch_slice(c, MB, a, &e)) return e;
+  }
   if (MB != 1 && c->block_simt) {
     const int ks = gemv_ksplit(a.K);
     if (a.K / ks <= 256) {   // compact block GEMV: one chunk per warp
@@ -997,6 +1039,17 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   c->host_loop = hl && hl[0] == '1';
   const char* bs = std::getenv("BILD_BLOCK_SIMT");
   c->block_simt = bs && bs[0] == '1';
+  const char* sl = std::getenv("BILD_SLICE");
+  if (sl && sl[0] >= '0' && sl[0] <= '2') c->slice_mode = sl[0] - '0';
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      cudaGetLastError();
+      c->sms = 0;
+    }
+  }
+  const char* sm = std::getenv("BILD_SLICE_MIN_KB");
+  if (sm) c->slice_min_bytes = (size_t)std::atoi(sm) * 1024;
   const char* np = std::getenv("BILD_NO_PDL");
   c->use_pdl = !(np && np[0] == '1');
   Bump b(workspace);

@@ -65,8 +65,7 @@ def main():
             ms = ctx.time_pass(1, k, cache, a.iters)
             b = pass_bytes(sL, wb, 4, cache, wl.enc_len, k)
             print(json.dumps({"pass": "large block pass", "k": k, "cache": cache, "us": ms * 1e3, "GBs": b / ms / 1e6,
-                              "frac_of_peak": b / ms / 1e6 / peak, "bytes": b,
-                              "tensor_cores": ctx.uses_tensor_cores() and k > 1}))
+                              "frac_of_peak": b / ms / 1e6 / peak, "bytes": b}))
 
 
 if __name__ == "__main__":

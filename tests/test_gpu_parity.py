@@ -226,7 +226,7 @@ def test_generate_matches_live_oracle(torch_cuda, name, alpha_fb, alpha_rb, max_
         assert n is None or n > 0
 
 
-@pytest.mark.parametrize("env", ["BILD_BLOCK_SIMT", "BILD_HOST_LOOP", "BILD_NO_PDL", "BILD_NO_UMMA"])
+@pytest.mark.parametrize("env", ["BILD_BLOCK_SIMT", "BILD_HOST_LOOP", "BILD_NO_PDL", "BILD_NO_UMMA", "BILD_MEGA"])
 @pytest.mark.parametrize("name", ["tiny_bf16", "odd"])
 def test_alternative_paths_match_golden(torch_cuda, name, env):
     """The switchable paths (SIMT block GEMV, host-driven loop, plain launches, SIMT block
