@@ -12,6 +12,7 @@
 #include "decode_kernels.cuh"
 #include "mega_pass.cuh"
 #include "slice_linear.cuh"
+#include "unit_attention.cuh"
 #include "umma_linear.cuh"
 
 using namespace bild;
@@ -150,6 +151,9 @@ struct bild_ctx {
   int slice_mode = 2;                // row-slice linear kernel: 0 off, 1 block passes, 2 block and single-row passes
   int sms = 0;
   size_t slice_smem_set = 0;
+  bool unit_attn = true;             // decoder attention on the 256-thread chunked kernel
+  bool uattn_smem_set = false;
+  int slice_mma_min = 3;
   size_t slice_min_bytes = 3000 * 1024;   // single-row passes: smaller matrices stay on the GEMV (measured)
   bool mega_coop = true;             // launch the whole-pass kernel with the cooperative attribute
   bool capturing = false;            // launches are being recorded into a graph, not run
@@ -305,6 +309,36 @@ cudaError_t launch_battn_t(bild_ctx* c, BAttnArgs a, int row_blocks, int keys_ca
 // the encoder's self-attention (mode 2, all keys in one block) reads them from global memory.
 cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_blocks, int keys_cap) {
   if (a0.mode == 2) return launch_battn_t<MAXB, false>(c, a0, row_blocks, keys_cap);
+  if (c->unit_attn && a0.dkv <= 64 && a0.dkv >= 16) {   // 256-thread kernel with bulk-copied key / value chunks
+    DAttnArgs d;
+    d.b = a0; d.MB = MB; d.dkv_shift = ilog2(a0.dkv);
+    const int bias_len = a0.mode == 1 ? (((keys_cap + a0.nsplit - 1) / a0.nsplit + MAXB + 15) / 16 * 16) : 0;
+    const size_t smem = uattn_smem_floats(MB, a0.dkv, a0.nsplit, bias_len) * sizeof(float);
+    if (smem <= 200 * 1024) {
+      if (smem > 48 * 1024 && !c->uattn_smem_set) {
+        cudaError_t e = cudaFuncSetAttribute(uattn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        c->uattn_smem_set = true;
+      }
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(a0.H, a0.nsplit); cfg.blockDim = dim3(UA_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+      cudaLaunchAttribute at[2];
+      int na = 0;
+      if (c->use_pdl) {
+        at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+      }
+      if (a0.nsplit > 1) {   // the splits of one head are one cluster
+        at[na].id = cudaLaunchAttributeClusterDimension;
+        at[na].val.clusterDim.x = 1; at[na].val.clusterDim.y = a0.nsplit; at[na].val.clusterDim.z = 1;
+        ++na;
+      }
+      cfg.attrs = at; cfg.numAttrs = na;
+      (*c->cnt)++;
+      return cudaLaunchKernelEx(&cfg, uattn_kernel, d, bias_len);
+    }
+  }
   BAttnArgs a = a0;
   a.smem_keys = ((keys_cap + a.nsplit - 1) / a.nsplit + 3) / 4 * 4;
   const size_t smem = sizeof(float) * ((size_t)MB * a.dkv + (size_t)MB * a.smem_keys + (size_t)a.smem_keys * (2 * a.dkv + 4) +
@@ -669,10 +703,11 @@ bool launch_slice(bild_ctx* c, int MB, const LinArgs& a0, cudaError_t* err) {
   s.lin = a;
   s.lin.dkv_shift = ilog2(std::max(1, a.dkv));
   s.err = &c->st->err;
-  s.w_bytes = (int)align_up((size_t)rows * nmat * a.K * 2, 1024);
-  int xr = MB == 1 ? 1 : 8;
-  while (xr > 1 && (size_t)xr * a.K * 4 > 64 * 1024) xr /= 2;
+  s.w_bytes = (int)slice_w_bytes(rows * nmat, a.K);
+  int xr = MB == 1 ? 1 : MAXB;   // token rows staged at once: at most 81 KB (5 rows of 4096 columns)
+  while (xr > 1 && (size_t)xr * (a.K + SL_XPAD) * 4 > 81 * 1024) --xr;
   s.x_rows = xr;
+  s.mma_min = c->slice_mma_min;
   const size_t smem = slice_smem_bytes(s.w_bytes, xr, a.K);
   if (smem > 200 * 1024) return false;
   if (smem > 48 * 1024 && smem > c->slice_smem_set) {
@@ -1048,6 +1083,10 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
       c->sms = 0;
     }
   }
+  const char* ua = std::getenv("BILD_UNIT_ATTN");
+  if (ua && ua[0] == '0') c->unit_attn = false;
+  const char* mm = std::getenv("BILD_SLICE_MMA_MIN");
+  if (mm) c->slice_mma_min = std::min(5, std::max(2, std::atoi(mm)));
   const char* sm = std::getenv("BILD_SLICE_MIN_KB");
   if (sm) c->slice_min_bytes = (size_t)std::atoi(sm) * 1024;
   const char* np = std::getenv("BILD_NO_PDL");

@@ -6,8 +6,14 @@
 //     the kernel before it is still running;
 //   * after the wait the token rows (a few KB) follow with a second bulk copy; every block needs
 //     all of them, so they are read 148 times from L2 instead of once per pair of rows;
-//   * a work item is 4 weight rows x 256 columns for all token rows of the group; warp w takes
-//     items w, w + 8, ...; the partial sums of a quad are added in warp order (fixed);
+//   * one or two token rows: a work item is 4 weight rows x 256 columns for all token rows of
+//     the group; warp w takes items w, w + 8, ...; the partial sums of a quad are added in warp
+//     order (fixed);
+//   * more token rows: the block's 16-row tiles of the slice times 8-token tiles go through
+//     mma.sync m16n8k16 (bf16 weights straight from shared memory, each activation split into
+//     a bf16 head and a bf16 remainder, fp32 accumulation), the K range split over the warps of
+//     a tile and added in warp order.  Rows in shared memory are padded so that the fragment
+//     loads do not collide on banks;
 //   * the epilogues are those of the other linear kernels (store, ReLU, GELU gate, residual add,
 //     scatter to q / the KV cache).
 #pragma once
@@ -32,10 +38,16 @@ struct SliceArgs {
   LinArgs lin;
   int* err;
   int w_bytes;     // shared memory reserved for the weight slice
-  int x_rows;      // token rows per group (1, 2, 4 or 8)
+  int x_rows;      // token rows per group
+  int mma_min;     // groups of at least this many token rows go through the tensor cores
 };
 
-inline size_t slice_smem_bytes(int w_bytes, int x_rows, int K) { return (size_t)w_bytes + (size_t)x_rows * K * 4 + SL_PSUM + SL_MISC; }
+constexpr int SL_WPAD = 16;   // bytes added to every weight row in shared memory
+constexpr int SL_XPAD = 8;    // floats added to every token row in shared memory
+inline size_t slice_w_bytes(int rows, int K) { return ((size_t)rows * (K * 2 + SL_WPAD) + 1023) / 1024 * 1024; }
+inline size_t slice_smem_bytes(int w_bytes, int x_rows, int K) {
+  return (size_t)w_bytes + (size_t)x_rows * (K + SL_XPAD) * 4 + SL_PSUM + SL_MISC;
+}
 
 __device__ __forceinline__ void sl_wait(SliceShared* sh, int* err, unsigned long long* bar, uint32_t parity) {
   const uint32_t b = smem_u32(bar);
@@ -50,8 +62,8 @@ __device__ __forceinline__ void sl_wait(SliceShared* sh, int* err, unsigned long
 // Item it belongs to quad it / nkb and column block it % nkb (rows past the end of the slice repeat
 // its last row; nobody reads their sums).
 template <int MG>
-__device__ __forceinline__ void sl_items(const unsigned char* sW, int rowbytes, int nrows, int K, const float* Xs, float* psum,
-                                         int warp, int lane) {
+__device__ __forceinline__ void sl_items(const unsigned char* sW, int rowbytes, int nrows, int K, const float* Xs, int xst,
+                                         float* psum, int warp, int lane) {
   constexpr int NA = 4 * MG;
   constexpr int NP = NA <= 4 ? 4 : NA <= 8 ? 8 : NA <= 16 ? 16 : 32;
   constexpr int SH = NP == 32 ? 0 : NP == 16 ? 1 : NP == 8 ? 2 : 3;
@@ -75,8 +87,8 @@ __device__ __forceinline__ void sl_items(const unsigned char* sW, int rowbytes, 
         for (int r = 0; r < 4; ++r) w[r] = *reinterpret_cast<const uint4*>(rowp[r] + (size_t)kofs * 2);
 #pragma unroll
         for (int m = 0; m < MG; ++m) {
-          const float4 x0 = *reinterpret_cast<const float4*>(Xs + (size_t)m * K + kofs);
-          const float4 x1 = *reinterpret_cast<const float4*>(Xs + (size_t)m * K + kofs + 4);
+          const float4 x0 = *reinterpret_cast<const float4*>(Xs + (size_t)m * xst + kofs);
+          const float4 x1 = *reinterpret_cast<const float4*>(Xs + (size_t)m * xst + kofs + 4);
 #pragma unroll
           for (int r = 0; r < 4; ++r) {
             float s = acc[r * MG + m];
@@ -98,31 +110,87 @@ __device__ __forceinline__ void sl_items(const unsigned char* sW, int rowbytes, 
   }
 }
 
+// Tensor-core variant for NT tiles of 8 token rows.  Warp w works on row tile w / KS and on
+// the w % KS-th part of K (KS = 8, 4 or 2 for 1, 2 or 3 row tiles); its 16 x 8 accumulators go to
+// psum[(w * NT + nt) * 128 + lane * 4 ..] in the fragment layout of the instruction.
+__device__ __forceinline__ uint32_t sl_pack_bf16(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+template <int NT>
+__device__ __forceinline__ void sl_mma(const unsigned char* sW, int rowst, int nrows, int K, const float* Xs, int xst, int mg,
+                                       float* psum, int warp, int lane) {
+  const int MT = (nrows + 15) >> 4, ks_sh = MT == 1 ? 3 : MT == 2 ? 2 : 1, KS = 1 << ks_sh;
+  if (warp >= MT * KS) return;
+  const int mt = warp >> ks_sh, ks = warp & (KS - 1);
+  const int steps = (K + 15) >> 4, per = (steps + KS - 1) >> ks_sh;
+  const int s0 = ks * per, s1 = min(steps, s0 + per);
+  const int g = lane >> 2, t = lane & 3;
+  const unsigned char* pa0 = sW + (size_t)min(mt * 16 + g, nrows - 1) * rowst + t * 4;
+  const unsigned char* pa1 = sW + (size_t)min(mt * 16 + g + 8, nrows - 1) * rowst + t * 4;
+  const float* xb[NT];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) xb[nt] = Xs + (size_t)min(nt * 8 + g, mg - 1) * xst + 2 * t;
+  float c[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll 2
+  for (int st = s0; st < s1; ++st) {
+    const int k0 = st << 4;
+    const bool tail = k0 + 8 >= K;   // K is a multiple of 8: the second half of the last step may not exist
+    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(pa0 + k0 * 2);
+    const uint32_t a1 = *reinterpret_cast<const uint32_t*>(pa1 + k0 * 2);
+    const uint32_t a2 = tail ? 0u : *reinterpret_cast<const uint32_t*>(pa0 + k0 * 2 + 16);
+    const uint32_t a3 = tail ? 0u : *reinterpret_cast<const uint32_t*>(pa1 + k0 * 2 + 16);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float2 x0 = *reinterpret_cast<const float2*>(xb[nt] + k0);
+      const float2 x1 = tail ? make_float2(0.f, 0.f) : *reinterpret_cast<const float2*>(xb[nt] + k0 + 8);
+      const uint32_t h0 = sl_pack_bf16(x0.x, x0.y), h1 = sl_pack_bf16(x1.x, x1.y);
+      const uint32_t l0 = sl_pack_bf16(x0.x - __uint_as_float(h0 << 16), x0.y - __uint_as_float(h0 & 0xffff0000u));
+      const uint32_t l1 = sl_pack_bf16(x1.x - __uint_as_float(h1 << 16), x1.y - __uint_as_float(h1 & 0xffff0000u));
+      asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                   : "+f"(c[nt][0]), "+f"(c[nt][1]), "+f"(c[nt][2]), "+f"(c[nt][3])
+                   : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(h0), "r"(h1));
+      asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                   : "+f"(c[nt][0]), "+f"(c[nt][1]), "+f"(c[nt][2]), "+f"(c[nt][3])
+                   : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(l0), "r"(l1));
+    }
+  }
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+    *reinterpret_cast<float4*>(psum + ((size_t)(warp * NT + nt) * 32 + lane) * 4) = make_float4(c[nt][0], c[nt][1], c[nt][2], c[nt][3]);
+}
+
 __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
   extern __shared__ __align__(1024) unsigned char sl_smem[];
   const LinArgs& a = s.lin;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, K = a.K;
   const int r0 = (int)(((long long)blockIdx.x * a.N) / G), r1 = (int)(((long long)(blockIdx.x + 1) * a.N) / G);
-  const int n = r1 - r0, nmat = a.epi == EPI_GATED ? 2 : 1, nrows = n * nmat, rowbytes = K * 2;
+  const int n = r1 - r0, nmat = a.epi == EPI_GATED ? 2 : 1, nrows = n * nmat, rowbytes = K * 2 + SL_WPAD, xst = K + SL_XPAD;
   if (n == 0) {   // more blocks than rows
     pdl_launch_dependents();
     return;
   }
   unsigned char* sW = sl_smem;
   float* Xs = reinterpret_cast<float*>(sl_smem + s.w_bytes);
-  float* psum = Xs + (size_t)s.x_rows * K;
+  float* psum = Xs + (size_t)s.x_rows * xst;
   SliceShared* sh = reinterpret_cast<SliceShared*>(psum + SL_PSUM / 4);
   if (tid == 0) {
     mg_mbar_init(smem_u32(&sh->wbar), 1);
     mg_mbar_init(smem_u32(&sh->xbar), 1);
     sh->failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    // the weights depend on nothing: request them before waiting for the kernel in front
-    const uint32_t bytes = (uint32_t)(n * rowbytes);
-    mg_mbar_expect(smem_u32(&sh->wbar), bytes * nmat);
-    mg_bulk_g2s(smem_u32(sW), (const __nv_bfloat16*)a.W0 + (size_t)r0 * K, bytes, smem_u32(&sh->wbar));
-    if (nmat == 2) mg_bulk_g2s(smem_u32(sW + bytes), (const __nv_bfloat16*)a.W1 + (size_t)r0 * K, bytes, smem_u32(&sh->wbar));
+    mg_mbar_expect(smem_u32(&sh->wbar), (uint32_t)(nrows * K * 2));
+  }
+  __syncthreads();
+  // the weights depend on nothing: request them before waiting for the kernel in front, one copy per
+  // row (the rows are padded in shared memory)
+  if (tid < nrows) {
+    const int r = tid < n ? tid : tid - n;
+    const __nv_bfloat16* W = (const __nv_bfloat16*)(tid < n ? a.W0 : a.W1);
+    mg_bulk_g2s(smem_u32(sW + (size_t)tid * rowbytes), W + (size_t)(r0 + r) * K, (uint32_t)(K * 2), smem_u32(&sh->wbar));
   }
   float4 gv[2];   // gains of the columns this thread scales (K <= 2048 where a norm precedes)
   if (a.gain) {
@@ -132,7 +200,6 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
       gv[j] = c < K ? __ldg(reinterpret_cast<const float4*>(a.gain + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
-  __syncthreads();
   pdl_launch_dependents();
   pdl_wait();
   const int M = min(a.desc->k, MAXB), pos0 = a.desc->pos0;
@@ -141,11 +208,11 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
 #pragma unroll 1
   for (int m0 = 0; m0 < M; m0 += rgl, ++xuse) {
     const int mg = min(rgl, M - m0);
-    if (tid == 0) {
+    if (tid == 0) mg_mbar_expect(smem_u32(&sh->xbar), (uint32_t)(mg * K * 4));
+    __syncthreads();   // the barrier expects the bytes (and the group before is done with the rows)
+    if (tid < mg) {
       asm volatile("fence.proxy.async;" ::: "memory");   // rows written by the kernel in front, read by the copy engine
-      const uint32_t bytes = (uint32_t)(mg * K * 4);
-      mg_mbar_expect(smem_u32(&sh->xbar), bytes);
-      mg_bulk_g2s(smem_u32(Xs), a.X + (size_t)m0 * a.ldx, bytes, smem_u32(&sh->xbar));
+      mg_bulk_g2s(smem_u32(Xs + (size_t)tid * xst), a.X + (size_t)(m0 + tid) * a.ldx, (uint32_t)(K * 4), smem_u32(&sh->xbar));
     }
     sl_wait(sh, s.err, &sh->xbar, xuse & 1);
     if (a.gain) {   // T5 norm: x * g / sqrt(mean(x^2) + eps); the division is applied to the dot products
@@ -155,10 +222,10 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
         for (int j = 0; j < 2; ++j) {
           const int c = tid * 4 + j * 1024;
           if (c < K) {
-            float4 v = *reinterpret_cast<float4*>(Xs + (size_t)m * K + c);
+            float4 v = *reinterpret_cast<float4*>(Xs + (size_t)m * xst + c);
             ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
             v.x *= gv[j].x; v.y *= gv[j].y; v.z *= gv[j].z; v.w *= gv[j].w;
-            *reinterpret_cast<float4*>(Xs + (size_t)m * K + c) = v;
+            *reinterpret_cast<float4*>(Xs + (size_t)m * xst + c) = v;
           }
         }
         ss = warp_sum(ss);
@@ -173,25 +240,39 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
       }
     }
     if (m0 == 0) sl_wait(sh, s.err, &sh->wbar, 0);
-    const int mgr = mg_round_rows(mg);
-    switch (mgr) {
-      case 1: sl_items<1>(sW, rowbytes, nrows, K, Xs, psum, warp, lane); break;
-      case 2: sl_items<2>(sW, rowbytes, nrows, K, Xs, psum, warp, lane); break;
-      case 4: sl_items<4>(sW, rowbytes, nrows, K, Xs, psum, warp, lane); break;
-      default: sl_items<8>(sW, rowbytes, nrows, K, Xs, psum, warp, lane); break;
+    const bool tc = mg >= s.mma_min;   // tensor cores for the larger groups
+    const int mgr = mg;
+    if (tc) {
+      if (!a.gain) __syncthreads();   // (with a norm the rows were synchronised above)
+      if (mg <= 8) sl_mma<1>(sW, rowbytes, nrows, K, Xs, xst, mg, psum, warp, lane);
+      else sl_mma<2>(sW, rowbytes, nrows, K, Xs, xst, mg, psum, warp, lane);
+    } else {
+      switch (mgr) {
+        case 1: sl_items<1>(sW, rowbytes, nrows, K, Xs, xst, psum, warp, lane); break;
+        case 2: sl_items<2>(sW, rowbytes, nrows, K, Xs, xst, psum, warp, lane); break;
+        case 3: sl_items<3>(sW, rowbytes, nrows, K, Xs, xst, psum, warp, lane); break;
+        default: sl_items<4>(sW, rowbytes, nrows, K, Xs, xst, psum, warp, lane); break;
+      }
     }
     __syncthreads();
-    // epilogue: (output row r, token row m); the partial sums of a quad are added in warp order
+    // epilogue: (output row r, token row m); partial sums are added in warp order
+    const int MT = (nrows + 15) >> 4, ks_sh = MT == 1 ? 3 : MT == 2 ? 2 : 1, NT = mg <= 8 ? 1 : 2;
     for (int m = tid >> 6; m < mg; m += 4) {
       const int r = tid & 63;
       if (r >= n) continue;
       auto total = [&](int row) {
-        const int qd = row >> 2, first = qd * nkb;
-        const float* p = psum + (size_t)(qd * 8) * 32 + (row & 3) * mgr + m;
         float t = 0.f;
+        if (tc) {   // fragment layout: row = group (+ 8), token = 2 * (lane & 3) (+ 1)
+          const int mt = row >> 4, rr = row & 15, col = m & 7;
+          const float* p = psum + ((size_t)((mt << ks_sh) * NT + (m >> 3)) * 32 + (rr & 7) * 4 + (col >> 1)) * 4 + (rr >> 3) * 2 + (col & 1);
+          for (int ks = 0; ks < (1 << ks_sh); ++ks) t += p[(size_t)ks * NT * 128];
+        } else {
+          const int qd = row >> 2, first = qd * nkb;
+          const float* p = psum + (size_t)(qd * 8) * 32 + (row & 3) * mgr + m;
 #pragma unroll
-        for (int wv = 0; wv < 8; ++wv)
-          if (((wv - first) & 7) < nkb) t += p[wv * 32];   // warp wv took part in this quad
+          for (int wv = 0; wv < 8; ++wv)
+            if (((wv - first) & 7) < nkb) t += p[wv * 32];   // warp wv took part in this quad
+        }
         return t;
       };
       float v = total(r);

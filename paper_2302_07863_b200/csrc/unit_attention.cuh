@@ -1,0 +1,212 @@
+// Decoder attention (steps S2, S5 and L2, L5) for up to MAXB query rows, 256 threads per block.
+// grid (heads, key splits); the splits of a head form one thread-block cluster whose blocks hand
+// (max, sum, weighted values) to the first block through distributed shared memory.
+//   * keys and values of the block's key range are staged in 64-key chunks with bulk (TMA)
+//     copies, double buffered; for cross-attention (the encoder K/V never change while decoding)
+//     the first chunks are requested before the dependency wait of the programmatic launch;
+//   * per chunk: scores one (row, key) pair per thread and turn (columns visited in a rotated
+//     order, so that the threads of a quarter warp hit different banks), running soft-max one
+//     warp per row, weighted values one (row, channel) pair per thread and group of rows.
+#pragma once
+#include "decode_kernels.cuh"
+#include "mega_pass.cuh"
+
+namespace bild {
+
+constexpr int UA_THREADS = 256;
+constexpr int UA_CK = 64;   // keys per staged chunk
+
+struct UAttnShared {
+  unsigned long long kvbar[2];
+  float amax[MAXB], asum[MAXB], ascale[MAXB];
+  int failed;
+};
+
+// floats of dynamic shared memory
+inline size_t uattn_smem_floats(int MB, int dkv, int nsplit, int bias_len) {
+  return (size_t)4 * UA_CK * dkv + (size_t)MB * dkv + (size_t)MB * UA_CK + (size_t)bias_len + (size_t)nsplit * MB * (dkv + 2) +
+         (sizeof(UAttnShared) + 3) / 4 + 8;
+}
+
+__global__ void __launch_bounds__(UA_THREADS) uattn_kernel(DAttnArgs d, int bias_len) {
+  extern __shared__ __align__(1024) float ua_smem[];
+  const BAttnArgs& a = d.b;
+  const int MB = d.MB, dsh = d.dkv_shift, dkv = a.dkv;
+  const int h = blockIdx.x, sp = blockIdx.y, ns = a.nsplit;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int chunk_floats = UA_CK * dkv, pst = dkv + 2;
+  float* sKV = ua_smem;                               // [2 buffers][keys | values][UA_CK][dkv]
+  float* sQ = sKV + 4 * chunk_floats;                 // [MB][dkv]
+  float* sS = sQ + MB * dkv;                          // [MB][UA_CK]
+  float* sBias = sS + MB * UA_CK;                      // [bias_len]
+  float* sM = sBias + bias_len;                       // [ns][MB][pst] (used in the first block of the cluster)
+  UAttnShared* sh = reinterpret_cast<UAttnShared*>(sM + (size_t)ns * MB * pst + ((ns * MB * pst) & 1));
+  if (tid == 0) {
+    mg_mbar_init(smem_u32(&sh->kvbar[0]), 1);
+    mg_mbar_init(smem_u32(&sh->kvbar[1]), 1);
+    sh->failed = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (ns > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  __syncthreads();
+  const float* Kh = a.kc + (size_t)h * a.cap * dkv;
+  const float* Vh = a.vc + (size_t)h * a.cap * dkv;
+  int j0 = 0, j1 = 0, nchunks = 0, issued = 0;
+  auto issue_to = [&](int upto) {   // thread 0: request chunks [issued, upto)
+#pragma unroll 1
+    for (; issued < upto; ++issued) {
+      if (tid != 0) continue;
+      const int jc = j0 + issued * UA_CK, nk = min(UA_CK, j1 - jc), buf = issued & 1;
+      const uint32_t bar = smem_u32(&sh->kvbar[buf]), bytes = (uint32_t)(nk * dkv * 4);
+      mg_mbar_expect(bar, 2 * bytes);
+      mg_bulk_g2s(smem_u32(sKV + (size_t)buf * 2 * chunk_floats), Kh + (size_t)jc * dkv, bytes, bar);
+      mg_bulk_g2s(smem_u32(sKV + (size_t)buf * 2 * chunk_floats + chunk_floats), Vh + (size_t)jc * dkv, bytes, bar);
+    }
+  };
+  auto set_range = [&](int n_all) {
+    const int per = (n_all + ns - 1) / ns;
+    j0 = min(n_all, sp * per);
+    j1 = min(n_all, j0 + per);
+    nchunks = (j1 - j0 + UA_CK - 1) / UA_CK;
+  };
+  if (a.mode == 0) {   // encoder keys: before the dependency wait
+    set_range(min(*a.n_keys_dev, a.cap));
+    issue_to(min(nchunks, 2));
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  const int M = min(a.desc->k, MB), pos0 = a.desc->pos0;
+  if (a.mode == 1) {
+    set_range(min(pos0 + M, a.cap));
+    if (tid == 0) asm volatile("fence.proxy.async;" ::: "memory");   // cache rows written by the kernel in front
+    issue_to(min(nchunks, 2));
+  }
+  for (int idx = tid; idx < (M << (dsh - 2)); idx += UA_THREADS) {
+    const int i = idx >> (dsh - 2), e4 = (idx & ((dkv >> 2) - 1)) << 2;
+    *reinterpret_cast<float4*>(sQ + i * dkv + e4) = __ldcg(reinterpret_cast<const float4*>(a.q + (size_t)i * a.ldq + h * dkv + e4));
+  }
+  // bias of the distances pos0 + i - j this block meets (a static table)
+  const int dmin = max(0, pos0 - (j1 - 1)), dmax = pos0 + M - 1 - j0;
+  const bool bias_staged = a.mode == 1 && dmax - dmin + 1 <= bias_len;
+  if (bias_staged)
+    for (int dd = dmin + tid; dd <= dmax; dd += UA_THREADS) sBias[dd - dmin] = __ldg(a.bias + (size_t)h * a.bias_ld + dd);
+  if (tid < MAXB) { sh->amax[tid] = -INFINITY; sh->asum[tid] = 0.f; sh->ascale[tid] = 1.f; }
+  const int RG = min(4, UA_THREADS >> dsh);           // query rows per group
+  const int ngroups = (M + RG - 1) / RG;
+  const int pv_i = tid >> dsh, pv_c = tid & (dkv - 1);   // thread <-> (row of the group, channel)
+  float pv_acc[4] = {0.f, 0.f, 0.f, 0.f};               // one per group (MAXB / RG <= 4 when dkv <= 64)
+  __syncthreads();
+#pragma unroll 1
+  for (int c = 0; c < nchunks; ++c) {
+    const int buf = c & 1;
+    const float* sK = sKV + (size_t)buf * 2 * chunk_floats;
+    const float* sV = sK + chunk_floats;
+    const int jc = j0 + c * UA_CK, nk = min(UA_CK, j1 - jc);
+    {   // bounded wait for the chunk
+      const uint32_t bar = smem_u32(&sh->kvbar[buf]);
+      bool ok = mg_mbar_try(bar, (c >> 1) & 1);
+      if (!ok && !*(volatile int*)&sh->failed) {
+        for (unsigned it = 0; it < MG_SPIN && !ok; ++it) ok = mg_mbar_try(bar, (c >> 1) & 1);
+        if (!ok) { sh->failed = 1; atomicExch(a.err, (int)BILD_ERR_TIMEOUT); }
+      }
+    }
+    // scores of all rows: one (row, key) pair per thread and turn
+#pragma unroll 1
+    for (int idx = tid; idx < M * UA_CK; idx += UA_THREADS) {
+      const int i = idx >> 6, jj = idx & (UA_CK - 1);
+      float sc = -INFINITY;
+      const int j = jc + jj;
+      if (jj < nk && (a.mode == 0 || j <= pos0 + i)) {
+        float accs = 0.f;
+        const int nq4 = dkv >> 2;
+#pragma unroll 4
+        for (int e = 0; e < nq4; ++e) {
+          const int er = ((e + jj) & (nq4 - 1)) << 2;
+          const float4 kv = *reinterpret_cast<const float4*>(sK + jj * dkv + er);
+          const float4 qv = *reinterpret_cast<const float4*>(sQ + i * dkv + er);
+          accs += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
+        }
+        if (a.mode == 1) {
+          const int dd = pos0 + i - j;
+          accs += bias_staged ? sBias[dd - dmin] : __ldg(a.bias + (size_t)h * a.bias_ld + dd);
+        }
+        sc = accs;
+      }
+      sS[idx] = sc;
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int row = warp; row < M; row += UA_THREADS / 32) {   // running soft-max, one warp per row
+      const float s0 = sS[row * UA_CK + lane], s1 = sS[row * UA_CK + 32 + lane];
+      const float mx = warp_max(fmaxf(s0, s1));
+      const float mo = sh->amax[row], mn = fmaxf(mo, mx);
+      const float p0 = s0 == -INFINITY ? 0.f : __expf(s0 - mn), p1 = s1 == -INFINITY ? 0.f : __expf(s1 - mn);
+      sS[row * UA_CK + lane] = p0;
+      sS[row * UA_CK + 32 + lane] = p1;
+      const float sum = warp_sum(p0 + p1);
+      if (lane == 0) {
+        const float scale = mo == -INFINITY ? 0.f : __expf(mo - mn);
+        sh->ascale[row] = scale;
+        sh->asum[row] = sh->asum[row] * scale + sum;
+        sh->amax[row] = mn;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int gp = 0; gp < 4; ++gp) {   // weighted values: thread <-> (row gp * RG + pv_i, channel pv_c)
+      const int i = gp * RG + pv_i;
+      if (gp >= ngroups || pv_i >= RG || i >= M) continue;
+      float a0 = 0.f, a1 = 0.f;
+      const float* pr = sS + i * UA_CK;
+      int jj = 0;
+#pragma unroll 4
+      for (; jj + 1 < nk; jj += 2) {
+        a0 += pr[jj] * sV[jj * dkv + pv_c];
+        a1 += pr[jj + 1] * sV[(jj + 1) * dkv + pv_c];
+      }
+      if (jj < nk) a0 += pr[jj] * sV[jj * dkv + pv_c];
+      pv_acc[gp] = pv_acc[gp] * sh->ascale[i] + (a0 + a1);
+    }
+    __syncthreads();   // probabilities and the chunk's buffer are free again
+    issue_to(min(nchunks, c + 3));
+  }
+  // finish: a lone split writes the rows; otherwise every split hands its sums to the first block
+  // (which is known to be running once the cluster barrier entered at the start completes)
+  if (ns > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+#pragma unroll
+  for (int gp = 0; gp < 4; ++gp) {
+    if (gp >= ngroups) break;
+    const int i = gp * RG + pv_i;
+    if (pv_i >= RG || i >= M) continue;
+    if (ns == 1) {
+      const float l = sh->asum[i];
+      a.out[(size_t)i * a.ldo + h * dkv + pv_c] = l > 0.f ? pv_acc[gp] / l : 0.f;
+    } else {
+      float* mrow = sM + ((size_t)sp * MB + i) * pst;
+      st_cluster_f1(smem_u32(mrow + 2 + pv_c), 0, pv_acc[gp]);
+      if (pv_c == 0) { st_cluster_f1(smem_u32(mrow), 0, sh->amax[i]); st_cluster_f1(smem_u32(mrow + 1), 0, sh->asum[i]); }
+    }
+  }
+  if (ns == 1) return;
+  cluster_sync_all();
+  if (sp != 0) return;
+#pragma unroll 1
+  for (int idx = tid; idx < (M << dsh); idx += UA_THREADS) {
+    const int i = idx >> dsh, c = idx & (dkv - 1);
+    float gm = -INFINITY;
+#pragma unroll 1
+    for (int s2 = 0; s2 < ns; ++s2) gm = fmaxf(gm, sM[((size_t)s2 * MB + i) * pst]);
+    float num = 0.f, den = 0.f;
+#pragma unroll 1
+    for (int s2 = 0; s2 < ns; ++s2) {   // split order
+      const float* Ps = sM + ((size_t)s2 * MB + i) * pst;
+      const float l = Ps[1];
+      const float w = l > 0.f ? __expf(Ps[0] - gm) : 0.f;
+      den += l * w;
+      num += Ps[2 + c] * w;
+    }
+    a.out[(size_t)i * a.ldo + h * dkv + c] = den > 0.f ? num / den : 0.f;
+  }
+}
+
+}  // namespace bild
