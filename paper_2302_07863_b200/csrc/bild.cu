@@ -13,6 +13,7 @@
 #include "mega_pass.cuh"
 #include "slice_linear.cuh"
 #include "unit_attention.cuh"
+#include "slice_head.cuh"
 #include "umma_linear.cuh"
 
 using namespace bild;
@@ -153,6 +154,8 @@ struct bild_ctx {
   size_t slice_smem_set = 0;
   bool unit_attn = true;             // decoder attention on the 256-thread chunked kernel
   bool uattn_smem_set = false;
+  int slice_head = 1;                // tensor-core LM head: 0 off, 1 block passes, 2 also single-row passes
+  bool slice_head_smem_set = false;
   int slice_mma_min = 3;
   size_t slice_min_bytes = 3000 * 1024;   // single-row passes: smaller matrices stay on the GEMV (measured)
   bool mega_coop = true;             // launch the whole-pass kernel with the cooperative attribute
@@ -202,7 +205,10 @@ int check_config(const bild_config* cfg, std::string& why) {
 
 int head_grid_for(int V) { return std::max(1, std::min(HEAD_GRID_MAX, (V + 63) / 64)); }
 // partial records either head kernel may write (block head: grid x MAXB; single-row head: up to V / 8 blocks)
-size_t head_partial_count(int V) { return std::max((size_t)head_grid_for(V) * MAXB, (size_t)(V + 7) / 8 + 8); }
+size_t head_partial_count(int V) {
+  // block head: grid x MAXB; single-row head: up to V / 8 blocks; one-block-per-SM head: SMs x MAXB
+  return std::max(std::max((size_t)head_grid_for(V) * MAXB, (size_t)(V + 7) / 8 + 8), (size_t)MG_MAX_BLOCKS * MAXB);
+}
 
 // Lays out everything the context keeps on the device.
 void plan(bild_ctx* c, Bump& b) {
@@ -837,6 +843,18 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   h.scale = mc.logit_scale; h.V = mc.vocab; h.K = d; h.desc = m.desc; h.partials = m.head_part;
   h.counter = m.head_cnt; h.out = m.head_out; h.logits_dbg = logits_dbg; h.which = which; h.loop = loop_ptrs(c);
   h.cond_while = cond_while; h.cond_if = cond_if;
+  const size_t sh_smem = slice_head_smem_bytes(d);
+  if (c->slice_head >= (MB == 1 ? 2 : 1) && dt == BILD_BF16 && c->sms > 0 && c->sms <= MG_MAX_BLOCKS && sh_smem <= 200 * 1024 &&
+      d % 8 == 0 && ((uintptr_t)m.w.lm_head & 15) == 0) {
+    // tensor-core head, one block per SM
+    if (!c->slice_head_smem_set) {
+      CUDA_TRY(c, cudaFuncSetAttribute(slice_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+      c->slice_head_smem_set = true;
+    }
+    CUDA_TRY(c, launch_k(c, slice_head_kernel, dim3(c->sms), dim3(SH_THREADS), sh_smem, h, which == 0 ? 0 : (MB == 1 ? 2 : 1),
+                         &c->st->err));
+    return BILD_OK;
+  }
   CUDA_TRY(c, launch_head(c->stream, dt, MB, h, m.head_grid, c->cnt));
   return BILD_OK;
 }
@@ -1083,6 +1101,8 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
       c->sms = 0;
     }
   }
+  const char* shd = std::getenv("BILD_SLICE_HEAD");
+  if (shd && shd[0] >= '0' && shd[0] <= '2') c->slice_head = shd[0] - '0';
   const char* ua = std::getenv("BILD_UNIT_ATTN");
   if (ua && ua[0] == '0') c->unit_attn = false;
   const char* mm = std::getenv("BILD_SLICE_MMA_MIN");

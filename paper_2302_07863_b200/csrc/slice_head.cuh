@@ -1,0 +1,194 @@
+// Fused LM head (steps S9+S10 / L9+L10) for up to MAXB rows, bf16 weights, one block per SM.
+//   z[m][n] = scale * sum_j W[n][j] * rms_norm(x_m)[j]
+// Block b owns the vocabulary rows [b V / G, (b + 1) V / G).  They stream through a ring of
+// 16-row tiles in shared memory (one bulk copy per row, rows padded against bank conflicts; the
+// first tiles are requested before the dependency wait of the programmatic launch).  A tile
+// times the (up to 16) normalised token rows goes through mma.sync m16n8k16 (each activation as
+// a bf16 head and a bf16 remainder, fp32 accumulation), K split over the 8 warps and added in
+// warp order.  Thread (row r, token m) then folds the logit into its running (max, arg max,
+// sum exp), picks up the target token's logit, and at the end the 16 threads of a token combine
+// in a fixed order.  The logits never reach memory unless a debug buffer is given.  The last
+// block to finish merges the per-block partials, applies the policy tests and advances the
+// decode loop, exactly as the other head kernels do.
+#pragma once
+#include "slice_linear.cuh"
+
+namespace bild {
+
+constexpr int SH_THREADS = 256;
+constexpr int SH_TILES = 3;   // ring depth
+
+struct SliceHeadShared {
+  unsigned long long full[SH_TILES];
+  float scale[MAXB];
+  int last, failed;
+};
+
+__host__ __device__ inline size_t slice_head_tile_bytes(int K) { return (size_t)16 * (K * 2 + SL_WPAD); }
+inline size_t slice_head_smem_bytes(int K) {
+  return SH_TILES * slice_head_tile_bytes(K) + (size_t)MAXB * (K + SL_XPAD) * 4 + 2 * 8 * 2 * 128 * 4 + 1024;
+}
+
+// pass_kind: index of the pass counter the kernel bumps when it runs inside a loop graph
+__global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int pass_kind, int* err) {
+  extern __shared__ __align__(1024) unsigned char shd_smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int K = a.K, V = a.V, G = gridDim.x;
+  const int rowst = K * 2 + SL_WPAD, xst = K + SL_XPAD;
+  const size_t tile_bytes = slice_head_tile_bytes(K);
+  unsigned char* sW = shd_smem;
+  float* Xs = reinterpret_cast<float*>(shd_smem + SH_TILES * tile_bytes);
+  float* psum = Xs + (size_t)MAXB * xst;                 // [2][8 warps][2][32 lanes][4]
+  SliceHeadShared* sh = reinterpret_cast<SliceHeadShared*>(psum + 2 * 8 * 2 * 128);
+  const int nb = (int)(((long long)blockIdx.x * V) / G), ne = (int)(((long long)(blockIdx.x + 1) * V) / G);
+  const int ntiles = (ne - nb + 15) >> 4;
+  const __nv_bfloat16* W = (const __nv_bfloat16*)a.W;
+  if (tid == 0) {
+    for (int i = 0; i < SH_TILES; ++i) mg_mbar_init(smem_u32(&sh->full[i]), 1);
+    sh->failed = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  // warp 0 requests tile t: lane 0 announces the bytes, lanes 0..15 copy one row each (rows past the
+  // end of the slice repeat its last row; their logits are masked)
+  auto request = [&](int t) {
+    if (warp != 0 || t >= ntiles) return;
+    const int slot = t % SH_TILES;
+    if (lane == 0) mg_mbar_expect(smem_u32(&sh->full[slot]), (uint32_t)(16 * K * 2));
+    __syncwarp();
+    if (lane < 16) {
+      const int n = min(nb + t * 16 + lane, ne - 1);
+      mg_bulk_g2s(smem_u32(sW + slot * tile_bytes + (size_t)lane * rowst), W + (size_t)n * K, (uint32_t)(K * 2),
+                  smem_u32(&sh->full[slot]));
+    }
+  };
+  if (ntiles > 0)
+    for (int t = 0; t < SH_TILES; ++t) request(t);
+  pdl_launch_dependents();
+  pdl_wait();
+  const int M = min(a.desc ? a.desc->k : a.M, MAXB);
+  const int* target = a.desc ? a.desc->targets : a.target;
+  // normalised token rows: x * g / rms (the head's own norm), fp32 in shared memory
+  for (int m = warp; m < M; m += SH_THREADS / 32) {
+    float ss = 0.f;
+    for (int j = lane * 4; j < K; j += 128) {
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(a.X + (size_t)m * a.ldx + j));
+      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      *reinterpret_cast<float4*>(Xs + (size_t)m * xst + j) = v;
+    }
+    ss = warp_sum(ss);
+    const float sc = a.gain ? rsqrtf(ss / (float)K + a.eps) : 1.f;
+    __syncwarp();
+    for (int j = lane * 4; j < K; j += 128) {
+      float4 v = *reinterpret_cast<float4*>(Xs + (size_t)m * xst + j);
+      float4 g = a.gain ? __ldg(reinterpret_cast<const float4*>(a.gain + j)) : make_float4(1.f, 1.f, 1.f, 1.f);
+      v.x *= g.x * sc; v.y *= g.y * sc; v.z *= g.z * sc; v.w *= g.w * sc;
+      *reinterpret_cast<float4*>(Xs + (size_t)m * xst + j) = v;
+    }
+  }
+  __syncthreads();
+  // thread <-> (row r of the tile, token m)
+  const int er = tid & 15, em = tid >> 4;
+  const int my_target = (em < M && target) ? target[em] : -1;
+  Partial run;
+  run.m = -INFINITY; run.s = 0.f; run.idx = 0x7fffffff;
+  const int NT = M <= 8 ? 1 : 2;
+#pragma unroll 1
+  for (int t = 0; t < ntiles; ++t) {
+    const int slot = t % SH_TILES;
+    {   // bounded wait for the tile
+      const uint32_t bar = smem_u32(&sh->full[slot]), par = (t / SH_TILES) & 1;
+      bool ok = mg_mbar_try(bar, par);
+      if (!ok && !*(volatile int*)&sh->failed) {
+        for (unsigned it = 0; it < MG_SPIN && !ok; ++it) ok = mg_mbar_try(bar, par);
+        if (!ok) { sh->failed = 1; atomicExch(err, (int)BILD_ERR_TIMEOUT); }
+      }
+    }
+    float* ps = psum + (t & 1) * (8 * 2 * 128);
+    if (NT == 1) sl_mma<1>(sW + slot * tile_bytes, rowst, 16, K, Xs, xst, M, ps, warp, lane);
+    else sl_mma<2>(sW + slot * tile_bytes, rowst, 16, K, Xs, xst, M, ps, warp, lane);
+    __syncthreads();   // partial sums complete; every warp is done with the tile
+    request(t + SH_TILES);
+    if (em < M) {
+      // fragment layout of the accumulators: row = group (+ 8), token = 2 * (lane & 3) (+ 1)
+      const int col = em & 7;
+      const float* p = ps + ((size_t)(em >> 3) * 32 + (er & 7) * 4 + (col >> 1)) * 4 + (er >> 3) * 2 + (col & 1);
+      float z = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) z += p[(size_t)w * NT * 128];
+      const int n = nb + t * 16 + er;
+      if (n < ne) {
+        z *= a.scale;
+        if (z > run.m) { run.s = run.s * expf(run.m - z) + 1.f; run.m = z; run.idx = n; }
+        else run.s += expf(z - run.m);
+        if (n == my_target) a.out->gather[em] = z;
+        if (a.logits_dbg) a.logits_dbg[(size_t)em * V + n] = z;
+      }
+    }
+    // the other half of psum is written next; this half is reused two tiles later, after another barrier
+  }
+  // the 16 threads of a token combine (lanes 0..15 / 16..31 of a warp), lower row index first
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) {
+    Partial q;
+    q.m = __shfl_xor_sync(0xffffffffu, run.m, o);
+    q.s = __shfl_xor_sync(0xffffffffu, run.s, o);
+    q.idx = __shfl_xor_sync(0xffffffffu, run.idx, o);
+    run = ((lane & o) == 0) ? combine(run, q) : combine(q, run);
+  }
+  if (er == 0 && em < M) a.partials[(size_t)blockIdx.x * MAXB + em] = run;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned tk = atomicAdd(a.counter, 1u);
+    sh->last = (tk == gridDim.x - 1);
+    if (sh->last) *a.counter = 0;
+  }
+  __syncthreads();
+  if (!sh->last) return;
+  __threadfence();
+  for (int m = warp; m < M; m += SH_THREADS / 32) {
+    Partial p;
+    p.m = -INFINITY; p.s = 0.f; p.idx = 0x7fffffff;
+    for (int b = lane; b < (int)gridDim.x; b += 32) {
+      Partial q;
+      const Partial* src = &a.partials[(size_t)b * MAXB + m];
+      q.m = __ldcg(&src->m); q.s = __ldcg(&src->s); q.idx = __ldcg(&src->idx);
+      p = combine(p, q);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      Partial q;
+      q.m = __shfl_xor_sync(0xffffffffu, p.m, o);
+      q.s = __shfl_xor_sync(0xffffffffu, p.s, o);
+      q.idx = __shfl_xor_sync(0xffffffffu, p.idx, o);
+      p = ((lane & o) == 0) ? combine(p, q) : combine(q, p);
+    }
+    if (lane == 0) {
+      a.out->argmax[m] = p.idx;
+      a.out->zmax[m] = p.m;
+      a.out->lse[m] = p.m + logf(p.s);
+      if (m == 0) a.out->pmax = 1.f / p.s;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    HeadOut* o = a.out;
+    // gather[] was written by other blocks before their tickets: read around L1
+    for (int m = 0; m < M; ++m) o->gather[m] = __ldcg(&o->gather[m]);
+    if (a.loop.st) {
+      policy_tests(o, a.desc, a.loop.st, a.which);
+      if (a.desc->run_policy) policy_step(a.loop, o, a.desc, a.which);
+      else if (a.which == 0) a.loop.st->S_len = a.desc->pos0 + 1;
+      else a.loop.st->L_len = a.desc->pos0 + a.desc->k;
+      if (a.cond_while) {
+        a.loop.st->cum_passes[pass_kind]++;
+        cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
+      }
+      if (a.cond_if) cudaGraphSetConditional(a.cond_if, a.loop.st->fallback ? 1u : 0u);
+    }
+  }
+}
+
+}  // namespace bild
