@@ -269,7 +269,7 @@ def test_eos_and_limits(torch_cuda):
 
 
 # ---- full-size workloads: replay the oracle's calls, compare sampled logits ---------------
-@pytest.mark.parametrize("name", ["t5_sum", "mt5_mt"])
+@pytest.mark.parametrize("name", ["t5_sum", "mt5_mt", "t5_long"])
 def test_full_size_replay_and_generate(torch_cuda, name):
     torch = torch_cuda
     from paper_2302_07863_b200 import MODE_BILD, MODE_LARGE_ONLY, MODE_SMALL_ONLY
@@ -340,3 +340,26 @@ def test_full_size_replay_and_generate(torch_cuda, name):
         assert ctx.generate(MODE_SMALL_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["small_only"]["tokens"]
     if g["large_only"]["argmax_margin"] > 2 * tol:
         assert ctx.generate(MODE_LARGE_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["large_only"]["tokens"]
+
+
+@pytest.mark.gpu
+def test_persistent_pass_full_size(torch_cuda):
+    """The opt-in whole-pass persistent kernel (BILD_MEGA=1) reproduces the stored oracle run of the
+    summarisation workload: same tokens and statistics where every decision margin is above tolerance."""
+    from paper_2302_07863_b200 import MODE_BILD
+    from paper_2302_07863_b200.synthetic import make_context
+    g = golden("t5_sum")
+    os.environ["BILD_MEGA"] = "1"
+    try:
+        ctx, ids, wl = make_context("t5_sum", g["scale_small"]["scale"], g["scale_large"]["scale"])
+    finally:
+        del os.environ["BILD_MEGA"]
+    ctx.encode(ids)
+    th = g["thresholds"]
+    tol = TOL[wl.dtype]
+    r = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
+    mg = g["bild"]["margins"]
+    if mg["argmax"] > 2 * tol and mg["fallback"] > 2 * tol and mg["rollback"] > 2 * tol:
+        assert r["tokens"] == g["bild"]["tokens"]
+        assert r["stats"] == g["bild"]["stats"]
+    ctx.close()
