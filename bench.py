@@ -254,9 +254,10 @@ def main():
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": ("large-model block pass, k=%d" % k_mean) if dom_large else "small-model step",
                      "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "peak_kind": peak_kind,
-                     # dram__bytes_read+write of one block pass (k=5, cache 64) of the t5_sum pair, 194 of its 195
-                     # launches (the LM head, 65.8 MB algorithmic, was outside the capture window)
-                     "traffic": 852.6e6 if (dom_large and a.workload in ("t5_sum", "t5_long")) else None,
+                     # dram__bytes_read+write of one block pass (k=5, cache 64) of the t5_sum pair: 191 of its 194
+                     # launches (one of the 144 linear layers, 2 MB, and the LM head, 65.8 MB algorithmic, were
+                     # outside the capture window); 814 MB algorithmic for the same launches
+                     "traffic": 828.5e6 if (dom_large and a.workload in ("t5_sum", "t5_long")) else None,
                      "note": "a pass is a chain of dependent kernels replayed as one CUDA graph; its duration is "
                              "measured with CUDA events over back-to-back replays"},
         "passes": {"small_step_us": t_small * 1e3, "small_step_GBs": b_small / t_small / 1e6,
