@@ -15,6 +15,7 @@
 #include "unit_attention.cuh"
 #include "slice_head.cuh"
 #include "umma_linear.cuh"
+#include "enc_gemm.cuh"
 
 using namespace bild;
 
@@ -107,6 +108,9 @@ struct Model {
   // TMA descriptors of the decoder's weight matrices (bf16 only): per layer qkv, o, cq, co, wi0, wi1, fo
   std::vector<CUtensorMap> tmaps;
   bool umma = false;
+  // encoder GEMM: descriptors of the bf16 head / remainder matrices of the layer input, by row length (d, inner, d_ff)
+  CUtensorMap tmH[3][2];
+  bool enc_gemm = false;
   // whole-pass persistent kernel (bf16 only)
   MegaLayer* mega_layers = nullptr;
   unsigned* mega_sync = nullptr;
@@ -132,6 +136,7 @@ struct bild_ctx {
   int* enc_len_dev = nullptr;
   int* bucket_tmp = nullptr;
   float *ex = nullptr, *eq = nullptr, *ek = nullptr, *ev = nullptr, *eatt = nullptr, *eu = nullptr;
+  __nv_bfloat16 *exh = nullptr, *exl = nullptr;   // bf16 head / remainder of the encoder's current layer input
   int enc_len = 0;
   bool encoded = false;
   int64_t launches = 0;
@@ -258,6 +263,9 @@ void plan(bild_ctx* c, Bump& b) {
   c->ev = b.take<float>((size_t)ecap * imax);
   c->eatt = b.take<float>(ecap16 * imax);
   c->eu = b.take<float>(ecap16 * fmax);
+  const size_t ecap128 = (size_t)(ecap + EG_TOK - 1) / EG_TOK * EG_TOK;   // whole tiles of 128 tokens
+  c->exh = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(dmax, imax), fmax));
+  c->exl = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(dmax, imax), fmax));
   b.off = align_up(b.off, 256);
 }
 
@@ -314,11 +322,10 @@ cudaError_t launch_battn_t(bild_ctx* c, BAttnArgs a, int row_blocks, int keys_ca
 // Decoder attention stages its keys / values in shared memory (at most 128 keys per split);
 // the encoder's self-attention (mode 2, all keys in one block) reads them from global memory.
 cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_blocks, int keys_cap) {
-  if (a0.mode == 2) return launch_battn_t<MAXB, false>(c, a0, row_blocks, keys_cap);
-  if (c->unit_attn && a0.dkv <= 64 && a0.dkv >= 16) {   // 256-thread kernel with bulk-copied key / value chunks
+  if (c->unit_attn && a0.mode != 2 && a0.dkv <= 64 && a0.dkv >= 16) {   // 256-thread kernel with bulk-copied key / value chunks
     DAttnArgs d;
     d.b = a0; d.MB = MB; d.dkv_shift = ilog2(a0.dkv);
-    const int bias_len = a0.mode == 1 ? (((keys_cap + a0.nsplit - 1) / a0.nsplit + MAXB + 15) / 16 * 16) : 0;
+    const int bias_len = a0.mode != 0 ? (((keys_cap + a0.nsplit - 1) / a0.nsplit + MAXB + 15) / 16 * 16) : 0;
     const size_t smem = uattn_smem_floats(MB, a0.dkv, a0.nsplit, bias_len) * sizeof(float);
     if (smem <= 200 * 1024) {
       if (smem > 48 * 1024 && !c->uattn_smem_set) {
@@ -327,7 +334,7 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
         c->uattn_smem_set = true;
       }
       cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(a0.H, a0.nsplit); cfg.blockDim = dim3(UA_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+      cfg.gridDim = dim3(a0.H, a0.nsplit, row_blocks); cfg.blockDim = dim3(UA_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
       cudaLaunchAttribute at[2];
       int na = 0;
       if (c->use_pdl) {
@@ -345,6 +352,7 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
       return cudaLaunchKernelEx(&cfg, uattn_kernel, d, bias_len);
     }
   }
+  if (a0.mode == 2) return launch_battn_t<MAXB, false>(c, a0, row_blocks, keys_cap);
   BAttnArgs a = a0;
   a.smem_keys = ((keys_cap + a.nsplit - 1) / a.nsplit + 3) / 4 * 4;
   const size_t smem = sizeof(float) * ((size_t)MB * a.dkv + (size_t)MB * a.smem_keys + (size_t)a.smem_keys * (2 * a.dkv + 4) +
@@ -545,6 +553,20 @@ void setup_umma(bild_ctx* c, Model& m) {
     return;
   }
   m.umma = true;
+  // encoder GEMM over 128-token tiles
+  m.enc_gemm = false;
+  const char* eg = std::getenv("BILD_ENC_GEMM");
+  if (eg && eg[0] == '0') return;
+  const int ecap128 = (c->cfg.max_enc_len + EG_TOK - 1) / EG_TOK * EG_TOK;
+  const int Ks[3] = {mc.d_model, m.inner, mc.d_ff};
+  for (int i = 0; i < 3; ++i)
+    if (!make_tmap(enc, c->exh, ecap128, Ks[i], &m.tmH[i][0]) || !make_tmap(enc, c->exl, ecap128, Ks[i], &m.tmH[i][1])) return;
+  if (cudaFuncSetAttribute(enc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)eg_smem_bytes<false>()) != cudaSuccess ||
+      cudaFuncSetAttribute(enc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)eg_smem_bytes<true>()) != cudaSuccess) {
+    cudaGetLastError();
+    return;
+  }
+  m.enc_gemm = true;
 }
 
 // Decides whether the decoder passes of model `m` run as the persistent whole-pass kernel and
@@ -757,9 +779,30 @@ cudaError_t launch_dec_linear(bild_ctx* c, Model& m, int MB, const LinArgs& a, i
   return launch_linear(c, c->cfg.dtype, MB, a);
 }
 
+// Encoder linear layer on 128-token tiles: split the (normalised) input into bf16 head + remainder, then the GEMM.
+// `split` false: the input was split by an earlier call with the same input and norm.
+cudaError_t launch_enc_gemm(bild_ctx* c, Model& m, const LinArgs& a, int layer, int which_map, bool split) {
+  const int E = a.M, tiles_tok = (E + EG_TOK - 1) / EG_TOK;
+  const int ki = a.K == m.c.d_model ? 0 : a.K == m.inner ? 1 : 2;
+  if (split) {
+    cudaError_t e = launch_k(c, norm_split_kernel, dim3(tiles_tok * EG_TOK / 4), dim3(128), 0, a.X, a.ldx, a.gain, a.eps, E, a.K,
+                             c->exh, c->exl);
+    if (e != cudaSuccess) return e;
+  }
+  const CUtensorMap* t = &m.tmaps[(size_t)layer * TM_PER_LAYER];
+  const bool gated = a.epi == EPI_GATED;
+  dim3 grid((a.N + UM_TILE_M - 1) / UM_TILE_M, tiles_tok);
+  if (gated)
+    return launch_k(c, enc_gemm_kernel<true>, grid, dim3(EG_THREADS), eg_smem_bytes<true>(), a, &c->st->err, t[which_map],
+                    t[which_map == TM_EWI0 ? TM_EWI1 : which_map], m.tmH[ki][0], m.tmH[ki][1]);
+  return launch_k(c, enc_gemm_kernel<false>, grid, dim3(EG_THREADS), eg_smem_bytes<false>(), a, &c->st->err, t[which_map],
+                  t[which_map], m.tmH[ki][0], m.tmH[ki][1]);
+}
+
 // Linear layer of the encoder over rb blocks of MAXB rows.
-cudaError_t launch_enc_linear(bild_ctx* c, Model& m, const LinArgs& a, int rb, int layer, int which_map) {
+cudaError_t launch_enc_linear(bild_ctx* c, Model& m, const LinArgs& a, int rb, int layer, int which_map, bool split = true) {
   int cs, nkb;
+  if (m.enc_gemm && (a.K == m.c.d_model || a.K == m.inner || a.K == m.c.d_ff)) return launch_enc_gemm(c, m, a, layer, which_map, split);
   if (m.umma && umma_plan(a.N, a.K, a.epi == EPI_GATED, &cs, &nkb, rb >= 4)) {
     const CUtensorMap* t = &m.tmaps[(size_t)layer * TM_PER_LAYER];
     return launch_umma(c, a, t[which_map], t[which_map == TM_EWI0 ? TM_EWI1 : which_map], cs, nkb, rb);
@@ -900,7 +943,7 @@ int encoder_pass(bild_ctx* c, int which) {
     a.M = E; a.eps = mc.ln_eps; a.W0 = m.dec[l].wckv; a.X = c->ex; a.ldx = d; a.gain = (const float*)m.w.enc_final_ln;
     a.N = 2 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 1;
     a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.pos0_host = 0;
-    CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_CKV));
+    CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_CKV, l == 0));   // the normalised encoder output is split once
   }
   return BILD_OK;
 }

@@ -1,0 +1,210 @@
+// Linear layers of the encoder (set-up step: encoder stack and the cross-attention K/V of every
+// decoder layer) on the 5th-generation tensor cores, for hundreds of token rows at once:
+//   Y^T[n][tok] = sum_j W[n][j] * H[tok][j],   H = rms_norm(X) * g  or  H = X
+//   * `norm_split_kernel` writes H once per layer input as two bf16 matrices, H_hi = bf16(H) and
+//     H_lo = bf16(H - H_hi) (rows padded with zeros to whole tiles of 128 tokens), so that the
+//     product keeps ~16 mantissa bits of the activation while the weights stay bf16;
+//   * `enc_gemm_kernel`: one CTA per (128 weight rows, 128 tokens) tile.  Weight tile, H_hi tile
+//     and H_lo tile [128][64] arrive by TMA (128-byte swizzle) into a ring of stages; one elected
+//     thread issues tcgen05.mma M128 N256 K16: the H_hi and H_lo tiles sit back to back in the
+//     stage and form one 256-row operand, so each weight tile is read once per k step; the
+//     accumulator in tensor memory has 128 columns for hi and 128 for lo (a second accumulator
+//     for the gate matrix of a gated FFN); the epilogue reads 16 token columns of both at a time, adds them and applies store / ReLU / GELU gate / residual add /
+//     scatter to q and the K/V layout, writing 32 consecutive outputs of one token per warp;
+//   * every wait on an mbarrier is bounded (error code, then the block carries on and frees its
+//     tensor memory).
+#pragma once
+#include "umma_linear.cuh"
+
+namespace bild {
+
+constexpr int EG_THREADS = 128;
+constexpr int EG_TOK = 128;   // tokens per tile
+
+// H_hi / H_lo of one row per warp; rows >= M are written as zeros (the last tile's padding)
+__global__ void __launch_bounds__(128) norm_split_kernel(const float* __restrict__ X, int ldx, const float* __restrict__ gain,
+                                                         float eps, int M, int K, __nv_bfloat16* __restrict__ Hh,
+                                                         __nv_bfloat16* __restrict__ Hl) {
+  const int lane = threadIdx.x & 31, row = blockIdx.x * 4 + (threadIdx.x >> 5);
+  pdl_launch_dependents();
+  pdl_wait();
+  __nv_bfloat16* oh = Hh + (size_t)row * K;
+  __nv_bfloat16* ol = Hl + (size_t)row * K;
+  if (row >= M) {
+    for (int c = lane * 8; c < K; c += 256) {
+      *reinterpret_cast<uint4*>(oh + c) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(ol + c) = make_uint4(0, 0, 0, 0);
+    }
+    return;
+  }
+  const float* x = X + (size_t)row * ldx;
+  float inv = 1.f;
+  if (gain) {
+    float ss = 0.f;
+    for (int c = lane * 4; c < K; c += 128) {
+      const float4 v = *reinterpret_cast<const float4*>(x + c);
+      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    ss = warp_sum(ss);
+    inv = rsqrtf(ss / (float)K + eps);
+  }
+  for (int c = lane * 8; c < K; c += 256) {
+    const float4 a0 = *reinterpret_cast<const float4*>(x + c), a1 = *reinterpret_cast<const float4*>(x + c + 4);
+    float h[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    if (gain) {
+      const float4 g0 = *reinterpret_cast<const float4*>(gain + c), g1 = *reinterpret_cast<const float4*>(gain + c + 4);
+      const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) h[i] = h[i] * g[i] * inv;
+    }
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(h[2 * i]), h1 = __float2bfloat16_rn(h[2 * i + 1]);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(h[2 * i] - __bfloat162float(h0));
+      const __nv_bfloat16 l1 = __float2bfloat16_rn(h[2 * i + 1] - __bfloat162float(h1));
+      hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    }
+    *reinterpret_cast<uint4*>(oh + c) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(ol + c) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
+}
+
+// bf16 x bf16 -> fp32, A and B K-major, M = 128, N = 256 (128 token rows of hi, then 128 of lo)
+constexpr uint32_t EG_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+__device__ __forceinline__ void eg_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(EG_IDESC), "r"(accumulate) : "memory");
+}
+
+template <bool GATED>
+__host__ __device__ constexpr int eg_stages() { return GATED ? 3 : 4; }
+template <bool GATED>
+constexpr size_t eg_smem_bytes() { return 1024 + (size_t)eg_stages<GATED>() * (GATED ? 4 : 3) * 16384 + 256; }
+
+template <bool GATED>
+__global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* err, const __grid_constant__ CUtensorMap tmW0,
+                                                              const __grid_constant__ CUtensorMap tmW1,
+                                                              const __grid_constant__ CUtensorMap tmHh,
+                                                              const __grid_constant__ CUtensorMap tmHl) {
+  constexpr int NST = eg_stages<GATED>();
+  constexpr int NMAT = GATED ? 2 : 1;
+  constexpr int STAGE = (NMAT + 2) * 16384;
+  constexpr int TCOLS = 256 * NMAT;
+  extern __shared__ unsigned char eg_raw[];
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int n_base = blockIdx.x * UM_TILE_M, tok0 = blockIdx.y * EG_TOK;
+  const int nkb = a.K / UM_KB;
+  unsigned char* base = (unsigned char*)(((uintptr_t)eg_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = (uint64_t*)(base + (size_t)NST * STAGE);
+  uint64_t* empty = full + NST;
+  uint64_t* done = empty + NST;
+  uint32_t* tmem_slot = (uint32_t*)(done + 1);
+  if (tid == 0) {
+    for (int i = 0; i < NST; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    mbar_init(done, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TCOLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = *tmem_slot;
+  auto load_stage = [&](int kb) {   // thread 0: weight tile(s) and both activation tiles of k block kb
+    unsigned char* st = base + (size_t)(kb % NST) * STAGE;
+    uint64_t* bar = &full[kb % NST];
+    mbar_expect_tx(bar, STAGE);
+    tma_load_2d(st, &tmW0, kb * UM_KB, n_base, bar);
+    if (GATED) tma_load_2d(st + 16384, &tmW1, kb * UM_KB, n_base, bar);
+    tma_load_2d(st + NMAT * 16384, &tmHh, kb * UM_KB, tok0, bar);
+    tma_load_2d(st + (NMAT + 1) * 16384, &tmHl, kb * UM_KB, tok0, bar);
+  };
+  pdl_launch_dependents();
+  pdl_wait();   // the activation tiles were written by the kernel in front
+  if (tid == 0) {
+    asm volatile("fence.proxy.async;" ::: "memory");   // rows written with ordinary stores, read by the copy engine
+    for (int kb = 0; kb < nkb; ++kb) {
+      if (kb >= NST && !mbar_wait(&empty[kb % NST], ((kb / NST) - 1) & 1)) *err = BILD_ERR_TIMEOUT;
+      load_stage(kb);
+    }
+  } else if (tid == 32) {
+    for (int kb = 0; kb < nkb; ++kb) {
+      const int st = kb % NST;
+      if (!mbar_wait(&full[st], (kb / NST) & 1)) *err = BILD_ERR_TIMEOUT;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t a0 = smem_u32(base + (size_t)st * STAGE);
+      const uint32_t bh = a0 + NMAT * 16384;   // hi tile, lo tile right behind it: one operand of 256 rows
+#pragma unroll
+      for (int kk = 0; kk < UM_KB / 16; ++kk) {
+        const uint64_t db = umma_desc_sw128(bh + kk * 32);
+        eg_mma(tmem, umma_desc_sw128(a0 + kk * 32), db, (kb | kk) ? 1u : 0u);
+        if (GATED) eg_mma(tmem + 256, umma_desc_sw128(a0 + 16384 + kk * 32), db, (kb | kk) ? 1u : 0u);
+      }
+      umma_commit(&empty[st]);   // the stage may be refilled once these MMAs have read it
+    }
+    umma_commit(done);
+  }
+  __syncwarp();
+  if (!mbar_wait(done, 0)) *err = BILD_ERR_TIMEOUT;
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+  // ---- epilogue: thread t holds weight row n_base + t; 16 token columns at a time ----
+  const int n = n_base + tid;
+  const bool row_ok = n < a.N;
+  const uint32_t t0 = tmem + ((uint32_t)(warp * 32) << 16);
+  int part = a.first_part, rr = n;
+  if (a.epi == EPI_HEADS) {
+    if (rr >= a.inner) { rr -= a.inner; ++part; }
+    if (rr >= a.inner) { rr -= a.inner; ++part; }
+  }
+  const int hh = a.epi == EPI_HEADS ? rr / a.dkv : 0, hc = a.epi == EPI_HEADS ? rr % a.dkv : 0;
+#pragma unroll 1
+  for (int c0 = 0; c0 < EG_TOK; c0 += 16) {
+    float v0[16], v1[16], lo16[16];
+    tmem_ld16(t0 + c0, v0);
+    tmem_ld16(t0 + 128 + c0, lo16);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v0[j] += lo16[j];
+    if (GATED) {
+      tmem_ld16(t0 + 256 + c0, v1);
+      tmem_ld16(t0 + 384 + c0, lo16);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v1[j] += lo16[j];
+    }
+    if (!row_ok) continue;
+    if (a.epi == EPI_RESID) {   // all 16 old values are requested before any of them is needed
+      float old[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) old[j] = tok0 + c0 + j < a.M ? __ldcg(a.Y + (size_t)(tok0 + c0 + j) * a.ldy + n) : 0.f;
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (tok0 + c0 + j < a.M) a.Y[(size_t)(tok0 + c0 + j) * a.ldy + n] = old[j] + v0[j];
+      continue;
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const int tok = tok0 + c0 + j;
+      if (tok >= a.M) break;
+      float y = v0[j];
+      if (a.epi == EPI_STORE) a.Y[(size_t)tok * a.ldy + n] = y;
+      else if (a.epi == EPI_RELU) a.Y[(size_t)tok * a.ldy + n] = fmaxf(y, 0.f);
+      else if (a.epi == EPI_GATED) { if (GATED) a.Y[(size_t)tok * a.ldy + n] = gelu_tanh(y) * v1[j]; }
+      else {
+        const int row = a.pos0_host + tok;
+        if (part == 0) a.q_out[(size_t)tok * a.ldq + rr] = y;
+        else if (row < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)hh * a.cap + row) * a.dkv + hc] = y;
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(TCOLS) : "memory");
+}
+
+}  // namespace bild

@@ -1,6 +1,9 @@
-// Decoder attention (steps S2, S5 and L2, L5) for up to MAXB query rows, 256 threads per block.
-// grid (heads, key splits); the splits of a head form one thread-block cluster whose blocks hand
-// (max, sum, weighted values) to the first block through distributed shared memory.
+// Attention for up to MAXB query rows per block, 256 threads: the decoder's self- and cross-attention
+// (steps S2, S5 and L2, L5) and the encoder's self-attention (set-up).
+// grid (heads, key splits, blocks of query rows); the splits of a head form one thread-block cluster
+// whose blocks hand (max, sum, weighted values) to the first block through distributed shared memory.
+// mode 0 cross (all encoder keys, no bias), 1 decoder self (row i sees keys 0..pos0+i, bias by
+// distance), 2 encoder self (all keys, bias by signed distance; rows blockIdx.z * MB ...).
 //   * keys and values of the block's key range are staged in 64-key chunks with bulk (TMA)
 //     copies, double buffered; for cross-attention (the encoder K/V never change while decoding)
 //     the first chunks are requested before the dependency wait of the programmatic launch;
@@ -75,19 +78,22 @@ __global__ void __launch_bounds__(UA_THREADS) uattn_kernel(DAttnArgs d, int bias
   }
   pdl_launch_dependents();
   pdl_wait();
-  const int M = min(a.desc->k, MB), pos0 = a.desc->pos0;
-  if (a.mode == 1) {
-    set_range(min(pos0 + M, a.cap));
+  const int row0 = blockIdx.z * MB;   // first query row of this block (encoder: many blocks of rows)
+  const int M = min((a.desc ? a.desc->k : a.M) - row0, MB), pos0 = a.desc ? a.desc->pos0 : 0;
+  if (a.mode != 0) {
+    set_range(a.mode == 1 ? min(pos0 + M, a.cap) : min(*a.n_keys_dev, a.cap));
     if (tid == 0) asm volatile("fence.proxy.async;" ::: "memory");   // cache rows written by the kernel in front
     issue_to(min(nchunks, 2));
   }
   for (int idx = tid; idx < (M << (dsh - 2)); idx += UA_THREADS) {
     const int i = idx >> (dsh - 2), e4 = (idx & ((dkv >> 2) - 1)) << 2;
-    *reinterpret_cast<float4*>(sQ + i * dkv + e4) = __ldcg(reinterpret_cast<const float4*>(a.q + (size_t)i * a.ldq + h * dkv + e4));
+    *reinterpret_cast<float4*>(sQ + i * dkv + e4) =
+        __ldcg(reinterpret_cast<const float4*>(a.q + (size_t)(row0 + i) * a.ldq + h * dkv + e4));
   }
-  // bias of the distances pos0 + i - j this block meets (a static table)
-  const int dmin = max(0, pos0 - (j1 - 1)), dmax = pos0 + M - 1 - j0;
-  const bool bias_staged = a.mode == 1 && dmax - dmin + 1 <= bias_len;
+  // bias entries this block meets (a static table): decoder index pos0 + i - j, encoder index off + j - (row0 + i)
+  const int dmin = a.mode == 1 ? max(0, pos0 - (j1 - 1)) : a.bias_off + j0 - (row0 + M - 1);
+  const int dmax = a.mode == 1 ? pos0 + M - 1 - j0 : a.bias_off + (j1 - 1) - row0;
+  const bool bias_staged = a.mode != 0 && dmax - dmin + 1 <= bias_len;
   if (bias_staged)
     for (int dd = dmin + tid; dd <= dmax; dd += UA_THREADS) sBias[dd - dmin] = __ldg(a.bias + (size_t)h * a.bias_ld + dd);
   if (tid < MAXB) { sh->amax[tid] = -INFINITY; sh->asum[tid] = 0.f; sh->ascale[tid] = 1.f; }
@@ -116,7 +122,7 @@ __global__ void __launch_bounds__(UA_THREADS) uattn_kernel(DAttnArgs d, int bias
       const int i = idx >> 6, jj = idx & (UA_CK - 1);
       float sc = -INFINITY;
       const int j = jc + jj;
-      if (jj < nk && (a.mode == 0 || j <= pos0 + i)) {
+      if (jj < nk && (a.mode != 1 || j <= pos0 + i)) {
         float accs = 0.f;
         const int nq4 = dkv >> 2;
 #pragma unroll 4
@@ -126,8 +132,8 @@ __global__ void __launch_bounds__(UA_THREADS) uattn_kernel(DAttnArgs d, int bias
           const float4 qv = *reinterpret_cast<const float4*>(sQ + i * dkv + er);
           accs += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
         }
-        if (a.mode == 1) {
-          const int dd = pos0 + i - j;
+        if (a.mode != 0) {
+          const int dd = a.mode == 1 ? pos0 + i - j : a.bias_off + j - (row0 + i);
           accs += bias_staged ? sBias[dd - dmin] : __ldg(a.bias + (size_t)h * a.bias_ld + dd);
         }
         sc = accs;
@@ -180,7 +186,7 @@ __global__ void __launch_bounds__(UA_THREADS) uattn_kernel(DAttnArgs d, int bias
     if (pv_i >= RG || i >= M) continue;
     if (ns == 1) {
       const float l = sh->asum[i];
-      a.out[(size_t)i * a.ldo + h * dkv + pv_c] = l > 0.f ? pv_acc[gp] / l : 0.f;
+      a.out[(size_t)(row0 + i) * a.ldo + h * dkv + pv_c] = l > 0.f ? pv_acc[gp] / l : 0.f;
     } else {
       float* mrow = sM + ((size_t)sp * MB + i) * pst;
       st_cluster_f1(smem_u32(mrow + 2 + pv_c), 0, pv_acc[gp]);
@@ -205,7 +211,7 @@ __global__ void __launch_bounds__(UA_THREADS) uattn_kernel(DAttnArgs d, int bias
       den += l * w;
       num += Ps[2 + c] * w;
     }
-    a.out[(size_t)i * a.ldo + h * dkv + c] = den > 0.f ? num / den : 0.f;
+    a.out[(size_t)(row0 + i) * a.ldo + h * dkv + c] = den > 0.f ? num / den : 0.f;
   }
 }
 
