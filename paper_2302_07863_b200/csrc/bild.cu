@@ -16,6 +16,7 @@
 #include "slice_head.cuh"
 #include "umma_linear.cuh"
 #include "enc_gemm.cuh"
+#include "enc_attention.cuh"
 
 using namespace bild;
 
@@ -159,6 +160,7 @@ struct bild_ctx {
   size_t slice_smem_set = 0;
   bool unit_attn = true;             // decoder attention on the 256-thread chunked kernel
   bool uattn_smem_set = false;
+  bool enc_attn_mma = true;          // encoder self-attention on the mma.sync kernel (d_kv = 64)
   int slice_head = 1;                // tensor-core LM head: 0 off, 1 block passes, 2 also single-row passes
   bool slice_head_smem_set = false;
   int slice_mma_min = 3;
@@ -351,6 +353,14 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
       (*c->cnt)++;
       return cudaLaunchKernelEx(&cfg, uattn_kernel, d, bias_len);
     }
+  }
+  if (a0.mode == 2 && a0.dkv == EA_D && c->enc_attn_mma) {   // encoder: 64-row tiles on mma.sync
+    const size_t smem = enc_attn_smem_bytes(keys_cap);
+    if (smem > 48 * 1024) {
+      cudaError_t e = cudaFuncSetAttribute(enc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
+    return launch_k(c, enc_attn_kernel, dim3(a0.H, (a0.M + EA_ROWS - 1) / EA_ROWS), dim3(EA_THREADS), smem, a0);
   }
   if (a0.mode == 2) return launch_battn_t<MAXB, false>(c, a0, row_blocks, keys_cap);
   BAttnArgs a = a0;
@@ -1146,6 +1156,8 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   }
   const char* shd = std::getenv("BILD_SLICE_HEAD");
   if (shd && shd[0] >= '0' && shd[0] <= '2') c->slice_head = shd[0] - '0';
+  const char* ea = std::getenv("BILD_ENC_ATTN_MMA");
+  if (ea && ea[0] == '0') c->enc_attn_mma = false;
   const char* ua = std::getenv("BILD_UNIT_ATTN");
   if (ua && ua[0] == '0') c->unit_attn = false;
   const char* mm = std::getenv("BILD_SLICE_MMA_MIN");

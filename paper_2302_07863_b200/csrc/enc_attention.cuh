@@ -1,0 +1,191 @@
+// Self-attention of the encoder (set-up step) for d_kv = 64: softmax(Q K^T + bias) V per head over
+// all encoder positions, bias by signed relative position.
+// One block per (head, 64 query rows), 4 warps of 16 rows each; keys and values are visited in tiles
+// of 64 with a running soft-max (no score matrix in memory).  Both products run on mma.sync
+// m16n8k16 with every fp32 operand split into a bf16 head and a bf16 remainder and three products
+// kept (head x head, head x remainder, remainder x head), i.e. ~16 mantissa bits per operand:
+//   * the key tile is staged as [key][d] (the "col" operand of Q K^T), the value tile transposed as
+//     [d][key] (the "col" operand of P V), both as head and remainder, rows padded against bank
+//     conflicts;
+//   * the score fragment of a warp (16 rows x 64 keys) stays in registers, is turned into
+//     probabilities and re-used as the left operand of P V (accumulator fragment of two 8-key
+//     tiles = operand fragment of one 16-key step).
+#pragma once
+#include "decode_kernels.cuh"
+
+namespace bild {
+
+constexpr int EA_THREADS = 128;
+constexpr int EA_ROWS = 64;    // query rows per block
+constexpr int EA_KEYS = 64;    // keys per tile
+constexpr int EA_D = 64;       // d_kv
+constexpr int EA_PAD = 8;      // bf16 elements of padding per staged row
+
+__device__ __forceinline__ uint32_t ea_pack(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+__device__ __forceinline__ void ea_split(float a, float b, uint32_t& hi, uint32_t& lo) {
+  hi = ea_pack(a, b);
+  lo = ea_pack(a - __uint_as_float(hi << 16), b - __uint_as_float(hi & 0xffff0000u));
+}
+__device__ __forceinline__ void ea_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+inline size_t enc_attn_smem_bytes(int max_keys) {
+  return (size_t)4 * EA_KEYS * (EA_D + EA_PAD) * 2 + (size_t)(max_keys + EA_ROWS) * 4;
+}
+
+// q [E][ldq], kc / vc [H][cap][64], out [E][ldo]; bias [H][bias_ld] indexed by bias_off + key - query
+__global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a) {
+  extern __shared__ __align__(16) unsigned char ea_smem[];
+  constexpr int ST = EA_D + EA_PAD;   // staged row length (bf16 elements)
+  __nv_bfloat16* sKh = reinterpret_cast<__nv_bfloat16*>(ea_smem);   // [key][d]
+  __nv_bfloat16* sKl = sKh + EA_KEYS * ST;
+  __nv_bfloat16* sVh = sKl + EA_KEYS * ST;                          // [d][key]
+  __nv_bfloat16* sVl = sVh + EA_D * ST;
+  float* sBias = reinterpret_cast<float*>(sVl + EA_D * ST);        // [E + 63]: entry (key - query + r0 + 63)
+  const int h = blockIdx.x, r0 = blockIdx.y * EA_ROWS;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int E = min(min(a.M, *a.n_keys_dev), a.cap);
+  for (int i = tid; i < E + EA_ROWS - 1; i += EA_THREADS) {
+    // key - query for query r0 + 63 - ... : entry i stands for key - query = i - (r0 + 63)
+    const int rel = i - (r0 + EA_ROWS - 1);
+    const int idx = a.bias_off + rel;
+    sBias[i] = (idx >= 0 && idx < a.bias_ld) ? __ldg(a.bias + (size_t)h * a.bias_ld + idx) : 0.f;
+  }
+  // this warp's queries as left-operand fragments (head and remainder), kept for the whole kernel
+  const int row_a = min(r0 + warp * 16 + g, E - 1), row_b = min(r0 + warp * 16 + g + 8, E - 1);
+  uint32_t qh[4][4], ql[4][4];
+  {
+    const float* qa = a.q + (size_t)row_a * a.ldq + h * EA_D;
+    const float* qb = a.q + (size_t)row_b * a.ldq + h * EA_D;
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      const float2 x0 = *reinterpret_cast<const float2*>(qa + ks * 16 + 2 * t);
+      const float2 x1 = *reinterpret_cast<const float2*>(qb + ks * 16 + 2 * t);
+      const float2 x2 = *reinterpret_cast<const float2*>(qa + ks * 16 + 8 + 2 * t);
+      const float2 x3 = *reinterpret_cast<const float2*>(qb + ks * 16 + 8 + 2 * t);
+      ea_split(x0.x, x0.y, qh[ks][0], ql[ks][0]);
+      ea_split(x1.x, x1.y, qh[ks][1], ql[ks][1]);
+      ea_split(x2.x, x2.y, qh[ks][2], ql[ks][2]);
+      ea_split(x3.x, x3.y, qh[ks][3], ql[ks][3]);
+    }
+  }
+  float o[8][4];   // 16 rows x 64 channels of weighted values (unnormalised)
+#pragma unroll
+  for (int dt = 0; dt < 8; ++dt) o[dt][0] = o[dt][1] = o[dt][2] = o[dt][3] = 0.f;
+  float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;   // rows g and g + 8 of the warp
+  const float* Kg = a.kc + (size_t)h * a.cap * EA_D;
+  const float* Vg = a.vc + (size_t)h * a.cap * EA_D;
+  const int qa_pos = r0 + warp * 16 + g, qb_pos = qa_pos + 8;
+#pragma unroll 1
+  for (int k0 = 0; k0 < E; k0 += EA_KEYS) {
+    __syncthreads();   // the previous tile is no longer read
+    // stage the tile: 64 keys x 64 channels, 16 float4 per row; thread -> (key, quarter of the row)
+    for (int idx = tid; idx < EA_KEYS * (EA_D / 4); idx += EA_THREADS) {
+      const int key = idx >> 4, c4 = (idx & 15) << 2;
+      const int kg = min(k0 + key, E - 1);
+      const float4 kv = __ldcg(reinterpret_cast<const float4*>(Kg + (size_t)kg * EA_D + c4));
+      const float4 vv = __ldcg(reinterpret_cast<const float4*>(Vg + (size_t)kg * EA_D + c4));
+      uint32_t h0, l0, h1, l1;
+      ea_split(kv.x, kv.y, h0, l0);
+      ea_split(kv.z, kv.w, h1, l1);
+      *reinterpret_cast<uint2*>(sKh + key * ST + c4) = make_uint2(h0, h1);
+      *reinterpret_cast<uint2*>(sKl + key * ST + c4) = make_uint2(l0, l1);
+      const float ve[4] = {vv.x, vv.y, vv.z, vv.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat16 vh = __float2bfloat16_rn(ve[e]);
+        sVh[(c4 + e) * ST + key] = vh;
+        sVl[(c4 + e) * ST + key] = __float2bfloat16_rn(ve[e] - __bfloat162float(vh));
+      }
+    }
+    __syncthreads();
+    // scores of 16 rows x 64 keys
+    float s[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+      const __nv_bfloat16* kh = sKh + (nt * 8 + g) * ST + 2 * t;
+      const __nv_bfloat16* kl = sKl + (nt * 8 + g) * ST + 2 * t;
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+        const uint32_t bh0 = *reinterpret_cast<const uint32_t*>(kh + ks * 16), bh1 = *reinterpret_cast<const uint32_t*>(kh + ks * 16 + 8);
+        const uint32_t bl0 = *reinterpret_cast<const uint32_t*>(kl + ks * 16), bl1 = *reinterpret_cast<const uint32_t*>(kl + ks * 16 + 8);
+        ea_mma(s[nt], qh[ks][0], qh[ks][1], qh[ks][2], qh[ks][3], bh0, bh1);
+        ea_mma(s[nt], qh[ks][0], qh[ks][1], qh[ks][2], qh[ks][3], bl0, bl1);
+        ea_mma(s[nt], ql[ks][0], ql[ks][1], ql[ks][2], ql[ks][3], bh0, bh1);
+      }
+    }
+    // bias, mask of the keys past the end, tile maxima
+    float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int key = k0 + nt * 8 + 2 * t + e;
+        const bool ok = key < E;
+        // entry (key - query + r0 + 63)
+        s[nt][e] = ok ? s[nt][e] + sBias[key - qa_pos + r0 + EA_ROWS - 1] : -INFINITY;
+        s[nt][2 + e] = ok ? s[nt][2 + e] + sBias[key - qb_pos + r0 + EA_ROWS - 1] : -INFINITY;
+        mx_a = fmaxf(mx_a, s[nt][e]);
+        mx_b = fmaxf(mx_b, s[nt][2 + e]);
+      }
+    }
+    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1)); mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1)); mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+    const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
+    const float sc_a = m_a == -INFINITY ? 0.f : __expf(m_a - mn_a), sc_b = m_b == -INFINITY ? 0.f : __expf(m_b - mn_b);
+    m_a = mn_a; m_b = mn_b;
+    float sum_a = 0.f, sum_b = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float pa = s[nt][e] == -INFINITY ? 0.f : __expf(s[nt][e] - mn_a);
+        const float pb = s[nt][2 + e] == -INFINITY ? 0.f : __expf(s[nt][2 + e] - mn_b);
+        s[nt][e] = pa; s[nt][2 + e] = pb;
+        sum_a += pa; sum_b += pb;
+      }
+    }
+    l_a = l_a * sc_a + sum_a;   // (this thread's share of the row; the quad is added at the end)
+    l_b = l_b * sc_b + sum_b;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) { o[dt][0] *= sc_a; o[dt][1] *= sc_a; o[dt][2] *= sc_b; o[dt][3] *= sc_b; }
+    // weighted values: probabilities of two 8-key tiles are the operand of one 16-key step
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t ph[4], pl[4];
+      ea_split(s[2 * j][0], s[2 * j][1], ph[0], pl[0]);
+      ea_split(s[2 * j][2], s[2 * j][3], ph[1], pl[1]);
+      ea_split(s[2 * j + 1][0], s[2 * j + 1][1], ph[2], pl[2]);
+      ea_split(s[2 * j + 1][2], s[2 * j + 1][3], ph[3], pl[3]);
+#pragma unroll
+      for (int dt = 0; dt < 8; ++dt) {
+        const __nv_bfloat16* vh = sVh + (dt * 8 + g) * ST + j * 16 + 2 * t;
+        const __nv_bfloat16* vl = sVl + (dt * 8 + g) * ST + j * 16 + 2 * t;
+        const uint32_t bh0 = *reinterpret_cast<const uint32_t*>(vh), bh1 = *reinterpret_cast<const uint32_t*>(vh + 8);
+        const uint32_t bl0 = *reinterpret_cast<const uint32_t*>(vl), bl1 = *reinterpret_cast<const uint32_t*>(vl + 8);
+        ea_mma(o[dt], ph[0], ph[1], ph[2], ph[3], bh0, bh1);
+        ea_mma(o[dt], ph[0], ph[1], ph[2], ph[3], bl0, bl1);
+        ea_mma(o[dt], pl[0], pl[1], pl[2], pl[3], bh0, bh1);
+      }
+    }
+  }
+  l_a += __shfl_xor_sync(0xffffffffu, l_a, 1); l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
+  l_b += __shfl_xor_sync(0xffffffffu, l_b, 1); l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
+  const float ia = l_a > 0.f ? 1.f / l_a : 0.f, ib = l_b > 0.f ? 1.f / l_b : 0.f;
+#pragma unroll
+  for (int dt = 0; dt < 8; ++dt) {
+    if (qa_pos < E) *reinterpret_cast<float2*>(a.out + (size_t)qa_pos * a.ldo + h * EA_D + dt * 8 + 2 * t) = make_float2(o[dt][0] * ia, o[dt][1] * ia);
+    if (qb_pos < E) *reinterpret_cast<float2*>(a.out + (size_t)qb_pos * a.ldo + h * EA_D + dt * 8 + 2 * t) = make_float2(o[dt][2] * ib, o[dt][3] * ib);
+  }
+}
+
+}  // namespace bild
