@@ -110,7 +110,7 @@ struct Model {
   std::vector<CUtensorMap> tmaps;
   bool umma = false;
   // encoder GEMM: descriptors of the bf16 head / remainder matrices of the layer input, by row length (d, inner, d_ff)
-  CUtensorMap tmH[3][2];
+  CUtensorMap tmH[2][3][2];   // [buffer pair][row length d / inner / d_ff][head, remainder]
   bool enc_gemm = false;
   // whole-pass persistent kernel (bf16 only)
   MegaLayer* mega_layers = nullptr;
@@ -137,7 +137,7 @@ struct bild_ctx {
   int* enc_len_dev = nullptr;
   int* bucket_tmp = nullptr;
   float *ex = nullptr, *eq = nullptr, *ek = nullptr, *ev = nullptr, *eatt = nullptr, *eu = nullptr;
-  __nv_bfloat16 *exh = nullptr, *exl = nullptr;   // bf16 head / remainder of the encoder's current layer input
+  __nv_bfloat16 *exh[2] = {nullptr, nullptr}, *exl[2] = {nullptr, nullptr};   // two pairs (bf16 head, remainder) of encoder layer inputs
   int enc_len = 0;
   bool encoded = false;
   int64_t launches = 0;
@@ -266,8 +266,10 @@ void plan(bild_ctx* c, Bump& b) {
   c->eatt = b.take<float>(ecap16 * imax);
   c->eu = b.take<float>(ecap16 * fmax);
   const size_t ecap128 = (size_t)(ecap + EG_TOK - 1) / EG_TOK * EG_TOK;   // whole tiles of 128 tokens
-  c->exh = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(dmax, imax), fmax));
-  c->exl = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(dmax, imax), fmax));
+  for (int i = 0; i < 2; ++i) {
+    c->exh[i] = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(dmax, imax), fmax));
+    c->exl[i] = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(dmax, imax), fmax));
+  }
   b.off = align_up(b.off, 256);
 }
 
@@ -323,7 +325,8 @@ cudaError_t launch_battn_t(bild_ctx* c, BAttnArgs a, int row_blocks, int keys_ca
 }
 // Decoder attention stages its keys / values in shared memory (at most 128 keys per split);
 // the encoder's self-attention (mode 2, all keys in one block) reads them from global memory.
-cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_blocks, int keys_cap) {
+cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_blocks, int keys_cap, __nv_bfloat16* oh = nullptr,
+                         __nv_bfloat16* ol = nullptr) {
   if (c->unit_attn && a0.mode != 2 && a0.dkv <= 64 && a0.dkv >= 16) {   // 256-thread kernel with bulk-copied key / value chunks
     DAttnArgs d;
     d.b = a0; d.MB = MB; d.dkv_shift = ilog2(a0.dkv);
@@ -360,7 +363,7 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
       cudaError_t e = cudaFuncSetAttribute(enc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
     }
-    return launch_k(c, enc_attn_kernel, dim3(a0.H, (a0.M + EA_ROWS - 1) / EA_ROWS), dim3(EA_THREADS), smem, a0);
+    return launch_k(c, enc_attn_kernel, dim3(a0.H, (a0.M + EA_ROWS - 1) / EA_ROWS), dim3(EA_THREADS), smem, a0, oh, ol);
   }
   if (a0.mode == 2) return launch_battn_t<MAXB, false>(c, a0, row_blocks, keys_cap);
   BAttnArgs a = a0;
@@ -569,8 +572,9 @@ void setup_umma(bild_ctx* c, Model& m) {
   if (eg && eg[0] == '0') return;
   const int ecap128 = (c->cfg.max_enc_len + EG_TOK - 1) / EG_TOK * EG_TOK;
   const int Ks[3] = {mc.d_model, m.inner, mc.d_ff};
-  for (int i = 0; i < 3; ++i)
-    if (!make_tmap(enc, c->exh, ecap128, Ks[i], &m.tmH[i][0]) || !make_tmap(enc, c->exl, ecap128, Ks[i], &m.tmH[i][1])) return;
+  for (int pr = 0; pr < 2; ++pr)
+    for (int i = 0; i < 3; ++i)
+      if (!make_tmap(enc, c->exh[pr], ecap128, Ks[i], &m.tmH[pr][i][0]) || !make_tmap(enc, c->exl[pr], ecap128, Ks[i], &m.tmH[pr][i][1])) return;
   if (cudaFuncSetAttribute(enc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)eg_smem_bytes<false>()) != cudaSuccess ||
       cudaFuncSetAttribute(enc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)eg_smem_bytes<true>()) != cudaSuccess) {
     cudaGetLastError();
@@ -790,29 +794,34 @@ cudaError_t launch_dec_linear(bild_ctx* c, Model& m, int MB, const LinArgs& a, i
 }
 
 // Encoder linear layer on 128-token tiles: split the (normalised) input into bf16 head + remainder, then the GEMM.
-// `split` false: the input was split by an earlier call with the same input and norm.
-cudaError_t launch_enc_gemm(bild_ctx* c, Model& m, const LinArgs& a, int layer, int which_map, bool split) {
+// The input pair is buffer `pair`; `split` false: it already holds the input (written by the kernel in front or by
+// an earlier call); `out_pair` >= 0: a ReLU / gated epilogue writes its output as the pair `out_pair` instead of fp32.
+cudaError_t launch_enc_gemm(bild_ctx* c, Model& m, const LinArgs& a, int layer, int which_map, bool split, int pair, int out_pair) {
   const int E = a.M, tiles_tok = (E + EG_TOK - 1) / EG_TOK;
   const int ki = a.K == m.c.d_model ? 0 : a.K == m.inner ? 1 : 2;
   if (split) {
     cudaError_t e = launch_k(c, norm_split_kernel, dim3(tiles_tok * EG_TOK / 4), dim3(128), 0, a.X, a.ldx, a.gain, a.eps, E, a.K,
-                             c->exh, c->exl);
+                             c->exh[pair], c->exl[pair]);
     if (e != cudaSuccess) return e;
   }
   const CUtensorMap* t = &m.tmaps[(size_t)layer * TM_PER_LAYER];
   const bool gated = a.epi == EPI_GATED;
+  __nv_bfloat16* oh = out_pair >= 0 ? c->exh[out_pair] : nullptr;
+  __nv_bfloat16* ol = out_pair >= 0 ? c->exl[out_pair] : nullptr;
   dim3 grid((a.N + UM_TILE_M - 1) / UM_TILE_M, tiles_tok);
   if (gated)
-    return launch_k(c, enc_gemm_kernel<true>, grid, dim3(EG_THREADS), eg_smem_bytes<true>(), a, &c->st->err, t[which_map],
-                    t[which_map == TM_EWI0 ? TM_EWI1 : which_map], m.tmH[ki][0], m.tmH[ki][1]);
-  return launch_k(c, enc_gemm_kernel<false>, grid, dim3(EG_THREADS), eg_smem_bytes<false>(), a, &c->st->err, t[which_map],
-                  t[which_map], m.tmH[ki][0], m.tmH[ki][1]);
+    return launch_k(c, enc_gemm_kernel<true>, grid, dim3(EG_THREADS), eg_smem_bytes<true>(), a, &c->st->err, oh, ol, t[which_map],
+                    t[which_map == TM_EWI0 ? TM_EWI1 : which_map], m.tmH[pair][ki][0], m.tmH[pair][ki][1]);
+  return launch_k(c, enc_gemm_kernel<false>, grid, dim3(EG_THREADS), eg_smem_bytes<false>(), a, &c->st->err, oh, ol, t[which_map],
+                  t[which_map], m.tmH[pair][ki][0], m.tmH[pair][ki][1]);
 }
 
 // Linear layer of the encoder over rb blocks of MAXB rows.
-cudaError_t launch_enc_linear(bild_ctx* c, Model& m, const LinArgs& a, int rb, int layer, int which_map, bool split = true) {
+cudaError_t launch_enc_linear(bild_ctx* c, Model& m, const LinArgs& a, int rb, int layer, int which_map, bool split = true,
+                              int pair = 0, int out_pair = -1) {
   int cs, nkb;
-  if (m.enc_gemm && (a.K == m.c.d_model || a.K == m.inner || a.K == m.c.d_ff)) return launch_enc_gemm(c, m, a, layer, which_map, split);
+  if (m.enc_gemm && (a.K == m.c.d_model || a.K == m.inner || a.K == m.c.d_ff))
+    return launch_enc_gemm(c, m, a, layer, which_map, split, pair, out_pair);
   if (m.umma && umma_plan(a.N, a.K, a.epi == EPI_GATED, &cs, &nkb, rb >= 4)) {
     const CUtensorMap* t = &m.tmaps[(size_t)layer * TM_PER_LAYER];
     return launch_umma(c, a, t[which_map], t[which_map == TM_EWI0 ? TM_EWI1 : which_map], cs, nkb, rb);
@@ -927,24 +936,27 @@ int encoder_pass(bild_ctx* c, int which) {
     a.M = E; a.eps = mc.ln_eps; a.W0 = w.wqkv; a.X = c->ex; a.ldx = d; a.gain = (const float*)w.ln1;
     a.N = 3 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 0; a.q_out = c->eq; a.ldq = I;
     a.kc = c->ek; a.vc = c->ev; a.cap = ecap; a.pos0_host = 0;
-    CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_EQKV));
+    // with the GEMM path the layer inputs alternate between two (bf16 head, remainder) buffer pairs:
+    // norm(x) -> pair 0 -> QKV; attention -> pair 1 -> O; norm(x) -> pair 0 -> FFN-up -> pair 1 -> FFN-down
+    const bool fuse = m.enc_gemm && c->enc_attn_mma && dkv == EA_D;
+    CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_EQKV, true, 0));
     BAttnArgs t{};
     t.q = c->eq; t.ldq = I; t.kc = c->ek; t.vc = c->ev; t.cap = ecap; t.out = c->eatt; t.ldo = I;
     t.bias = m.enc_bias; t.bias_ld = 2 * ecap - 1; t.bias_off = ecap - 1; t.mode = 2; t.dkv = dkv; t.H = H;
     t.n_keys_dev = c->enc_len_dev; t.M = E; t.part = m.att_part; t.counters = m.att_cnt; t.nsplit = 1;
     t.err = &c->st->err;
-    CUDA_TRY(c, launch_battn(c, MAXB, t, rb, ecap));
+    CUDA_TRY(c, launch_battn(c, MAXB, t, rb, ecap, fuse ? c->exh[1] : nullptr, fuse ? c->exl[1] : nullptr));
     LinArgs o{};
     o.M = E; o.W0 = w.wo; o.X = c->eatt; o.ldx = I; o.N = d; o.K = I; o.epi = EPI_RESID; o.Y = c->ex; o.ldy = d;
-    CUDA_TRY(c, launch_enc_linear(c, m, o, rb, l, TM_EO));
+    CUDA_TRY(c, launch_enc_linear(c, m, o, rb, l, TM_EO, !fuse, 1));
     LinArgs up{};
     up.M = E; up.eps = mc.ln_eps; up.W0 = w.wi0; up.W1 = w.wi1; up.X = c->ex; up.ldx = d; up.gain = (const float*)w.ln2;
     up.N = F; up.K = d; up.Y = c->eu; up.ldy = F;
     up.epi = mc.ffn_kind == BILD_FFN_GATED_GELU ? EPI_GATED : EPI_RELU;
-    CUDA_TRY(c, launch_enc_linear(c, m, up, rb, l, TM_EWI0));
+    CUDA_TRY(c, launch_enc_linear(c, m, up, rb, l, TM_EWI0, true, 0, m.enc_gemm ? 1 : -1));
     LinArgs dn{};
     dn.M = E; dn.W0 = w.wfo; dn.X = c->eu; dn.ldx = F; dn.N = d; dn.K = F; dn.epi = EPI_RESID; dn.Y = c->ex; dn.ldy = d;
-    CUDA_TRY(c, launch_enc_linear(c, m, dn, rb, l, TM_EFO));
+    CUDA_TRY(c, launch_enc_linear(c, m, dn, rb, l, TM_EFO, !m.enc_gemm, 1));
   }
   // encoder memory = final norm of ex (fused into the projections); cross K/V per decoder layer
   for (int l = 0; l < mc.n_layers; ++l) {
@@ -953,7 +965,7 @@ int encoder_pass(bild_ctx* c, int which) {
     a.M = E; a.eps = mc.ln_eps; a.W0 = m.dec[l].wckv; a.X = c->ex; a.ldx = d; a.gain = (const float*)m.w.enc_final_ln;
     a.N = 2 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 1;
     a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.pos0_host = 0;
-    CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_CKV, l == 0));   // the normalised encoder output is split once
+    CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_CKV, l == 0, 0));   // the normalised encoder output is split once
   }
   return BILD_OK;
 }

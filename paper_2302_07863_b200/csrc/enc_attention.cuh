@@ -40,7 +40,9 @@ inline size_t enc_attn_smem_bytes(int max_keys) {
 }
 
 // q [E][ldq], kc / vc [H][cap][64], out [E][ldo]; bias [H][bias_ld] indexed by bias_off + key - query
-__global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a) {
+// oh / ol != nullptr: the output is written as its bf16 head and remainder [E][H * 64] (what the
+// output projection reads) instead of fp32
+__global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_bfloat16* oh, __nv_bfloat16* ol) {
   extern __shared__ __align__(16) unsigned char ea_smem[];
   constexpr int ST = EA_D + EA_PAD;   // staged row length (bf16 elements)
   __nv_bfloat16* sKh = reinterpret_cast<__nv_bfloat16*>(ea_smem);   // [key][d]
@@ -181,10 +183,26 @@ __global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a) {
   l_a += __shfl_xor_sync(0xffffffffu, l_a, 1); l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
   l_b += __shfl_xor_sync(0xffffffffu, l_b, 1); l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
   const float ia = l_a > 0.f ? 1.f / l_a : 0.f, ib = l_b > 0.f ? 1.f / l_b : 0.f;
+  const int ldh = a.H * EA_D;
 #pragma unroll
   for (int dt = 0; dt < 8; ++dt) {
-    if (qa_pos < E) *reinterpret_cast<float2*>(a.out + (size_t)qa_pos * a.ldo + h * EA_D + dt * 8 + 2 * t) = make_float2(o[dt][0] * ia, o[dt][1] * ia);
-    if (qb_pos < E) *reinterpret_cast<float2*>(a.out + (size_t)qb_pos * a.ldo + h * EA_D + dt * 8 + 2 * t) = make_float2(o[dt][2] * ib, o[dt][3] * ib);
+    const int col = h * EA_D + dt * 8 + 2 * t;
+    if (oh) {
+      uint32_t hv, lv;
+      if (qa_pos < E) {
+        ea_split(o[dt][0] * ia, o[dt][1] * ia, hv, lv);
+        *reinterpret_cast<uint32_t*>(oh + (size_t)qa_pos * ldh + col) = hv;
+        *reinterpret_cast<uint32_t*>(ol + (size_t)qa_pos * ldh + col) = lv;
+      }
+      if (qb_pos < E) {
+        ea_split(o[dt][2] * ib, o[dt][3] * ib, hv, lv);
+        *reinterpret_cast<uint32_t*>(oh + (size_t)qb_pos * ldh + col) = hv;
+        *reinterpret_cast<uint32_t*>(ol + (size_t)qb_pos * ldh + col) = lv;
+      }
+    } else {
+      if (qa_pos < E) *reinterpret_cast<float2*>(a.out + (size_t)qa_pos * a.ldo + col) = make_float2(o[dt][0] * ia, o[dt][1] * ia);
+      if (qb_pos < E) *reinterpret_cast<float2*>(a.out + (size_t)qb_pos * a.ldo + col) = make_float2(o[dt][2] * ib, o[dt][3] * ib);
+    }
   }
 }
 

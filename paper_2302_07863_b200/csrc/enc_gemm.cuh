@@ -11,6 +11,8 @@
 //     accumulator in tensor memory has 128 columns for hi and 128 for lo (a second accumulator
 //     for the gate matrix of a gated FFN); the epilogue reads 16 token columns of both at a time, adds them and applies store / ReLU / GELU gate / residual add /
 //     scatter to q and the K/V layout, writing 32 consecutive outputs of one token per warp;
+//   * the FFN's first matrix can write its output directly as the bf16 head / remainder pair that
+//     the second matrix reads (no fp32 round trip, no separate split);
 //   * every wait on an mbarrier is bounded (error code, then the block carries on and frees its
 //     tensor memory).
 #pragma once
@@ -86,7 +88,8 @@ template <bool GATED>
 constexpr size_t eg_smem_bytes() { return 1024 + (size_t)eg_stages<GATED>() * (GATED ? 4 : 3) * 16384 + 256; }
 
 template <bool GATED>
-__global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* err, const __grid_constant__ CUtensorMap tmW0,
+__global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* err, __nv_bfloat16* oh, __nv_bfloat16* ol,
+                                                              const __grid_constant__ CUtensorMap tmW0,
                                                               const __grid_constant__ CUtensorMap tmW1,
                                                               const __grid_constant__ CUtensorMap tmHh,
                                                               const __grid_constant__ CUtensorMap tmHl) {
@@ -193,9 +196,17 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
       if (tok >= a.M) break;
       float y = v0[j];
       if (a.epi == EPI_STORE) a.Y[(size_t)tok * a.ldy + n] = y;
-      else if (a.epi == EPI_RELU) a.Y[(size_t)tok * a.ldy + n] = fmaxf(y, 0.f);
-      else if (a.epi == EPI_GATED) { if (GATED) a.Y[(size_t)tok * a.ldy + n] = gelu_tanh(y) * v1[j]; }
-      else {
+      else if (a.epi == EPI_RELU || a.epi == EPI_GATED) {
+        if (a.epi == EPI_RELU) y = fmaxf(y, 0.f);
+        else if (GATED) y = gelu_tanh(y) * v1[j];
+        if (oh) {   // the next layer reads this as bf16 head + remainder: write that form directly
+          const __nv_bfloat16 hv = __float2bfloat16_rn(y);
+          oh[(size_t)tok * a.N + n] = hv;
+          ol[(size_t)tok * a.N + n] = __float2bfloat16_rn(y - __bfloat162float(hv));
+        } else {
+          a.Y[(size_t)tok * a.ldy + n] = y;
+        }
+      } else {
         const int row = a.pos0_host + tok;
         if (part == 0) a.q_out[(size_t)tok * a.ldq + rr] = y;
         else if (row < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)hh * a.cap + row) * a.dkv + hc] = y;
