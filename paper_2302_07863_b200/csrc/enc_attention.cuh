@@ -89,23 +89,31 @@ __global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_
 #pragma unroll 1
   for (int k0 = 0; k0 < E; k0 += EA_KEYS) {
     __syncthreads();   // the previous tile is no longer read
-    // stage the tile: 64 keys x 64 channels, 16 float4 per row; thread -> (key, quarter of the row)
+    // stage the tile.  Keys: thread -> (key, 4 channels), rows written 8 bytes at a time.
     for (int idx = tid; idx < EA_KEYS * (EA_D / 4); idx += EA_THREADS) {
       const int key = idx >> 4, c4 = (idx & 15) << 2;
       const int kg = min(k0 + key, E - 1);
       const float4 kv = __ldcg(reinterpret_cast<const float4*>(Kg + (size_t)kg * EA_D + c4));
-      const float4 vv = __ldcg(reinterpret_cast<const float4*>(Vg + (size_t)kg * EA_D + c4));
       uint32_t h0, l0, h1, l1;
       ea_split(kv.x, kv.y, h0, l0);
       ea_split(kv.z, kv.w, h1, l1);
       *reinterpret_cast<uint2*>(sKh + key * ST + c4) = make_uint2(h0, h1);
       *reinterpret_cast<uint2*>(sKl + key * ST + c4) = make_uint2(l0, l1);
-      const float ve[4] = {vv.x, vv.y, vv.z, vv.w};
+    }
+    // Values, transposed: thread -> (pair of keys, 4 channels) with the key pair varying fastest, so that a
+    // warp writes 32 consecutive words of one transposed row
+    for (int idx = tid; idx < (EA_KEYS / 2) * (EA_D / 4); idx += EA_THREADS) {
+      const int kp = idx & 31, c4 = (idx >> 5) << 2;
+      const int ka = min(k0 + 2 * kp, E - 1), kb = min(k0 + 2 * kp + 1, E - 1);
+      const float4 va = *reinterpret_cast<const float4*>(Vg + (size_t)ka * EA_D + c4);
+      const float4 vb = *reinterpret_cast<const float4*>(Vg + (size_t)kb * EA_D + c4);
+      const float ea[4] = {va.x, va.y, va.z, va.w}, eb[4] = {vb.x, vb.y, vb.z, vb.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const __nv_bfloat16 vh = __float2bfloat16_rn(ve[e]);
-        sVh[(c4 + e) * ST + key] = vh;
-        sVl[(c4 + e) * ST + key] = __float2bfloat16_rn(ve[e] - __bfloat162float(vh));
+        uint32_t hv, lv;
+        ea_split(ea[e], eb[e], hv, lv);
+        *reinterpret_cast<uint32_t*>(sVh + (c4 + e) * ST + 2 * kp) = hv;
+        *reinterpret_cast<uint32_t*>(sVl + (c4 + e) * ST + 2 * kp) = lv;
       }
     }
     __syncthreads();
