@@ -226,15 +226,20 @@ def test_generate_matches_live_oracle(torch_cuda, name, alpha_fb, alpha_rb, max_
         assert n is None or n > 0
 
 
-@pytest.mark.parametrize("env", ["BILD_BLOCK_SIMT", "BILD_HOST_LOOP", "BILD_NO_PDL", "BILD_NO_UMMA", "BILD_MEGA"])
+@pytest.mark.parametrize("env", ["BILD_BLOCK_SIMT=1", "BILD_HOST_LOOP=1", "BILD_NO_PDL=1", "BILD_NO_UMMA=1", "BILD_MEGA=1",
+                                 "BILD_SLICE=0", "BILD_SLICE=2", "BILD_SLICE_MMA_MIN=5", "BILD_UNIT_ATTN=0", "BILD_SLICE_HEAD=0",
+                                 "BILD_SLICE_HEAD=2", "BILD_ENC_GEMM=0"])
 @pytest.mark.parametrize("name", ["tiny_bf16", "odd"])
 def test_alternative_paths_match_golden(torch_cuda, name, env):
-    """The switchable paths (SIMT block GEMV, host-driven loop, plain launches, SIMT block
-    linear) give the same tokens and trace as the default path's golden run."""
+    """The switchable paths (SIMT block GEMV, host-driven loop, plain launches, no tcgen05 kernels, persistent
+    pass, row-slice kernel off / also for single rows, SIMT items up to 4 rows, earlier attention kernel, earlier
+    block head, tensor-core head for single rows, encoder on the 16-row kernel) give the same tokens and trace as
+    the stored oracle run."""
+    env, env_value = env.split("=")
     from paper_2302_07863_b200 import MODE_BILD
     from paper_2302_07863_b200.synthetic import make_context
     g = golden(name)
-    os.environ[env] = "1"
+    os.environ[env] = env_value
     try:
         ctx, ids, wl = make_context(name, g["scale_small"]["scale"], g["scale_large"]["scale"])
     finally:
