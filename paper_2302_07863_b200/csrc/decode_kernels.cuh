@@ -57,6 +57,9 @@ __global__ void __launch_bounds__(512) gemv_kernel(LinArgs a) {
   }
   pdl_launch_dependents();
   pdl_wait();
+  // the value a residual epilogue adds to is requested now, not when the sums are ready
+  float y_old = 0.f;
+  if (a.epi == EPI_RESID && lane < 2 && n0 + lane < a.N) y_old = __ldcg(a.Y + n0 + lane);
   const float* X = a.X + kbeg;
   const float* G = a.gain ? a.gain + kbeg : nullptr;
   float a00 = 0.f, a01 = 0.f, a10 = 0.f, a11 = 0.f, ss = 0.f;
@@ -100,7 +103,7 @@ __global__ void __launch_bounds__(512) gemv_kernel(LinArgs a) {
   if (n >= a.N) return;
   const float inv = a.gain ? rsqrtf(ss * a.inv_k + a.eps) : 1.f;
   const float v0 = (lane ? a01 : a00) * inv;
-  if (a.epi == EPI_RESID) a.Y[n] += v0;
+  if (a.epi == EPI_RESID) a.Y[n] = y_old + v0;
   else if (a.epi == EPI_STORE) a.Y[n] = v0;
   else if (a.epi == EPI_RELU) a.Y[n] = fmaxf(v0, 0.f);
   else if (a.epi == EPI_GATED) { if (GATED) a.Y[n] = gelu_tanh(v0) * ((lane ? a11 : a10) * inv); }

@@ -208,6 +208,15 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
 #pragma unroll 1
   for (int m0 = 0; m0 < M; m0 += rgl, ++xuse) {
     const int mg = min(rgl, M - m0);
+    // the values a residual epilogue adds to are requested now, not when the sums are ready
+    float y_old[4] = {0.f, 0.f, 0.f, 0.f};
+    if (a.epi == EPI_RESID && (tid & 63) < n) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int m = (tid >> 6) + 4 * i;
+        if (m < mg) y_old[i] = __ldcg(a.Y + (size_t)(m0 + m) * a.ldy + r0 + (tid & 63));
+      }
+    }
     if (tid == 0) mg_mbar_expect(smem_u32(&sh->xbar), (uint32_t)(mg * K * 4));
     __syncthreads();   // the barrier expects the bytes (and the group before is done with the rows)
     if (tid < mg) {
@@ -257,7 +266,10 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
     __syncthreads();
     // epilogue: (output row r, token row m); partial sums are added in warp order
     const int MT = (nrows + 15) >> 4, ks_sh = MT == 1 ? 3 : MT == 2 ? 2 : 1, NT = mg <= 8 ? 1 : 2;
-    for (int m = tid >> 6; m < mg; m += 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int m = (tid >> 6) + 4 * i;
+      if (m >= mg) break;
       const int r = tid & 63;
       if (r >= n) continue;
       auto total = [&](int row) {
@@ -278,7 +290,7 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
       float v = total(r);
       if (a.gain) v *= sh->inv[m];
       const int nn = r0 + r, mm = m0 + m;
-      if (a.epi == EPI_RESID) a.Y[(size_t)mm * a.ldy + nn] += v;
+      if (a.epi == EPI_RESID) a.Y[(size_t)mm * a.ldy + nn] = y_old[i] + v;
       else if (a.epi == EPI_STORE) a.Y[(size_t)mm * a.ldy + nn] = v;
       else if (a.epi == EPI_RELU) a.Y[(size_t)mm * a.ldy + nn] = fmaxf(v, 0.f);
       else if (a.epi == EPI_GATED) a.Y[(size_t)mm * a.ldy + nn] = gelu_tanh(v) * (total(n + r) * (a.gain ? sh->inv[m] : 1.f));
