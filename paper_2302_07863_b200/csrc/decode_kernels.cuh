@@ -55,6 +55,13 @@ __global__ void __launch_bounds__(512) gemv_kernel(LinArgs a) {
     load8(W0 + (size_t)r1 * K + c0, w01);
     if (GATED) { load8(W1 + (size_t)r0 * K + c0, w10); load8(W1 + (size_t)r1 * K + c0, w11); }
   }
+  // the norm gains are weights too: fetched before the dependency wait
+  float gpre[8] = {1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f};
+  if (a.gain && c0 < kl) {
+    const float4 g0 = __ldg(reinterpret_cast<const float4*>(a.gain + kbeg + c0));
+    const float4 g1 = __ldg(reinterpret_cast<const float4*>(a.gain + kbeg + c0 + 4));
+    gpre[0] = g0.x; gpre[1] = g0.y; gpre[2] = g0.z; gpre[3] = g0.w; gpre[4] = g1.x; gpre[5] = g1.y; gpre[6] = g1.z; gpre[7] = g1.w;
+  }
   pdl_launch_dependents();
   pdl_wait();
   // the value a residual epilogue adds to is requested now, not when the sums are ready
@@ -74,11 +81,13 @@ __global__ void __launch_bounds__(512) gemv_kernel(LinArgs a) {
     const float4 x1 = *reinterpret_cast<const float4*>(X + c + 4);
     float h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
     if (G) {
-      const float4 g0 = *reinterpret_cast<const float4*>(G + c);
-      const float4 g1 = *reinterpret_cast<const float4*>(G + c + 4);
-      const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+      if (c != c0) {
+        const float4 g0 = *reinterpret_cast<const float4*>(G + c);
+        const float4 g1 = *reinterpret_cast<const float4*>(G + c + 4);
+        gpre[0] = g0.x; gpre[1] = g0.y; gpre[2] = g0.z; gpre[3] = g0.w; gpre[4] = g1.x; gpre[5] = g1.y; gpre[6] = g1.z; gpre[7] = g1.w;
+      }
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { ss += h[i] * h[i]; h[i] *= g[i]; }
+      for (int i = 0; i < 8; ++i) { ss += h[i] * h[i]; h[i] *= gpre[i]; }
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -591,6 +600,17 @@ __global__ void __launch_bounds__(HEAD1_THREADS) head1_kernel(HeadArgs a) {
       const int c = p * 256 + lane * 8;
       if (c < K) load8(W + (size_t)min(n0 + r, V - 1) * K + c, w[r][p]);
     }
+  float gn[NCH][8];   // the norm gains are weights too
+  if (a.gain) {
+#pragma unroll
+    for (int p = 0; p < NCH; ++p) {
+      const int c = p * 256 + lane * 8;
+      if (c < K) {
+        const float4 g0 = __ldg(reinterpret_cast<const float4*>(a.gain + c)), g1 = __ldg(reinterpret_cast<const float4*>(a.gain + c + 4));
+        gn[p][0] = g0.x; gn[p][1] = g0.y; gn[p][2] = g0.z; gn[p][3] = g0.w; gn[p][4] = g1.x; gn[p][5] = g1.y; gn[p][6] = g1.z; gn[p][7] = g1.w;
+      }
+    }
+  }
   pdl_launch_dependents();
   pdl_wait();
   const int target = a.desc ? a.desc->targets[0] : (a.target ? a.target[0] : -1);
@@ -604,10 +624,8 @@ __global__ void __launch_bounds__(HEAD1_THREADS) head1_kernel(HeadArgs a) {
       const float4 x0 = *reinterpret_cast<const float4*>(a.X + c), x1 = *reinterpret_cast<const float4*>(a.X + c + 4);
       float h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
       if (a.gain) {
-        const float4 g0 = *reinterpret_cast<const float4*>(a.gain + c), g1 = *reinterpret_cast<const float4*>(a.gain + c + 4);
-        const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { ss += h[i] * h[i]; h[i] *= g[i]; }
+        for (int i = 0; i < 8; ++i) { ss += h[i] * h[i]; h[i] *= gn[p][i]; }
       }
 #pragma unroll
       for (int r = 0; r < RPW; ++r)
