@@ -119,22 +119,33 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
-  auto load_stage = [&](int kb) {   // thread 0: weight tile(s) and both activation tiles of k block kb
+  // thread 0 feeds the ring; the weight tiles depend on nothing and are requested before the dependency wait
+  // for the first NST stages, the activation tiles of those stages follow after it (same barrier per stage)
+  auto load_weights = [&](int kb) {
     unsigned char* st = base + (size_t)(kb % NST) * STAGE;
     uint64_t* bar = &full[kb % NST];
     mbar_expect_tx(bar, STAGE);
     tma_load_2d(st, &tmW0, kb * UM_KB, n_base, bar);
     if (GATED) tma_load_2d(st + 16384, &tmW1, kb * UM_KB, n_base, bar);
+  };
+  auto load_acts = [&](int kb) {
+    unsigned char* st = base + (size_t)(kb % NST) * STAGE;
+    uint64_t* bar = &full[kb % NST];
     tma_load_2d(st + NMAT * 16384, &tmHh, kb * UM_KB, tok0, bar);
     tma_load_2d(st + (NMAT + 1) * 16384, &tmHl, kb * UM_KB, tok0, bar);
   };
+  if (tid == 0)
+    for (int kb = 0; kb < nkb && kb < NST; ++kb) load_weights(kb);
   pdl_launch_dependents();
   pdl_wait();   // the activation tiles were written by the kernel in front
   if (tid == 0) {
     asm volatile("fence.proxy.async;" ::: "memory");   // rows written with ordinary stores, read by the copy engine
     for (int kb = 0; kb < nkb; ++kb) {
-      if (kb >= NST && !mbar_wait(&empty[kb % NST], ((kb / NST) - 1) & 1)) *err = BILD_ERR_TIMEOUT;
-      load_stage(kb);
+      if (kb >= NST) {
+        if (!mbar_wait(&empty[kb % NST], ((kb / NST) - 1) & 1)) *err = BILD_ERR_TIMEOUT;
+        load_weights(kb);
+      }
+      load_acts(kb);
     }
   } else if (tid == 32) {
     for (int kb = 0; kb < nkb; ++kb) {
