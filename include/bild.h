@@ -211,8 +211,11 @@ int bild_fetch_result(bild_ctx *ctx, int32_t *tokens_out /*HOST*/, int *n_tokens
  * block pass over k tokens costs one weight load, Section 3.2): run one decoder pass of
  * model `which` (0 small with k = 1, 1 large with 1 <= k <= 16) `iters` times back to back
  * at self-cache length cache_len, with whatever the cache holds, and return the mean time
- * of one pass in milliseconds (CUDA events on the context's stream).  Leaves the decode
- * state undefined: call bild_reset or bild_generate afterwards.  Synchronises. */
+ * of one pass in milliseconds (CUDA events on the context's stream).  One untimed pass
+ * runs first; with iters < 0 it does not (|iters| timed passes), so that the first timed pass
+ * finds the caches as the previous work left them ("L2-cold" step after a large pass).
+ * Leaves the decode state undefined: call bild_reset or bild_generate afterwards.
+ * Synchronises. */
 int bild_time_pass(bild_ctx *ctx, int which, int k, int cache_len, int iters, float *ms_per_pass /*HOST out*/);
 
 /* 1 if the tcgen05 tensor-core kernel is in use for this context (bf16 weights, d_model / inner /

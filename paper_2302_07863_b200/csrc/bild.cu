@@ -1444,6 +1444,8 @@ int bild_op_lm_head(const void* W, int w_dtype, const float* X, const float* gai
 int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, float* ms_per_pass) {
   if (!c || !ms_per_pass || (which != 0 && which != 1)) return fail(c, BILD_ERR_ARG, "null argument / which");
   if (!c->encoded) return fail(c, BILD_ERR_STATE, "bild_encode has not been called");
+  const bool cold = iters < 0;   // no untimed first pass: the caches hold whatever ran before
+  if (cold) iters = -iters;
   if (k < 1 || k > (which == 0 ? 1 : MAXB) || iters < 1) return fail(c, BILD_ERR_ARG, "k or iters out of range");
   if (cache_len < 0 || cache_len + k > c->cfg.max_dec_len) return fail(c, BILD_ERR_CAPACITY, "cache_len + k > max_dec_len");
   TokList t{};
@@ -1462,13 +1464,14 @@ int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, floa
   if (rc == BILD_OK) rc = capture_pass(c, g, which, k == 1 ? 1 : MAXB, 0, 0, nullptr, &n_launch);
   if (rc == BILD_OK && cudaGraphInstantiate(&ex, g, 0) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && mega_epoch_budget(c, c->m[which], iters + 1) != cudaSuccess) rc = BILD_ERR_CUDA;
-  if (rc == BILD_OK && cudaGraphLaunch(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;  // untimed first pass
+  if (rc == BILD_OK && cudaGraphUpload(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
+  if (rc == BILD_OK && !cold && cudaGraphLaunch(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;  // untimed first pass
   if (rc == BILD_OK && cudaEventRecord(e0, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
   for (int it = 0; it < iters && rc == BILD_OK; ++it)
     if (cudaGraphLaunch(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && cudaEventRecord(e1, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && cudaEventSynchronize(e1) != cudaSuccess) rc = BILD_ERR_CUDA;
-  if (rc == BILD_OK) c->launches += n_launch * (iters + 1);
+  if (rc == BILD_OK) c->launches += n_launch * (iters + (cold ? 0 : 1));
   if (ex) cudaGraphExecDestroy(ex);
   if (g) cudaGraphDestroy(g);
   float ms = 0.f;

@@ -32,6 +32,7 @@ def main():
     ap.add_argument("--cache", default="64,256,1024")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--small", action="store_true")
+    ap.add_argument("--dist", type=int, default=0, help="also time N single passes per point: median, p10, p90")
     ap.add_argument("--peak-gbs", type=float, default=0.0)
     a = ap.parse_args()
     import torch
@@ -55,17 +56,41 @@ def main():
     ctx.encode(ids)
     wb = 2 if wl.dtype == "bf16" else 4
     sS, sL = MODEL_SHAPES[wl.small], MODEL_SHAPES[wl.large]
+    def dist(which, k, cache, cold_after=None):
+        """median / p10 / p90 (us) of a.dist single passes; cold_after: run that large pass before each one"""
+        if not a.dist:
+            return {}
+        ts = []
+        for _ in range(a.dist):
+            if cold_after is not None:
+                ctx.time_pass(1, cold_after, cache, 1)
+                ts.append(ctx.time_pass(which, k, cache, -1) * 1e3)
+            else:
+                ts.append(ctx.time_pass(which, k, cache, 1) * 1e3)
+        ts.sort()
+        q = lambda f: ts[min(len(ts) - 1, int(f * len(ts)))]
+        return {"median_us": q(0.5), "p10_us": q(0.1), "p90_us": q(0.9), "n": len(ts)}
+
+    nominal = 8000.0   # GB/s, the nominal HBM3e figure
     for cache in caches:
         if a.small:
             ms = ctx.time_pass(0, 1, cache, a.iters)
             b = pass_bytes(sS, wb, 4, cache, wl.enc_len, 1)
-            print(json.dumps({"pass": "small step", "k": 1, "cache": cache, "us": ms * 1e3, "GBs": b / ms / 1e6,
-                              "frac_of_peak": b / ms / 1e6 / peak, "bytes": b}))
+            rec = {"pass": "small step", "k": 1, "cache": cache, "us": ms * 1e3, "GBs": b / ms / 1e6,
+                   "frac_of_peak": b / ms / 1e6 / peak, "frac_of_nominal": b / ms / 1e6 / nominal, "bytes": b}
+            rec.update(dist(0, 1, cache))
+            print(json.dumps(rec))
+            if a.dist:   # the small model's weights fit in L2: time the step right after a large pass as well
+                rec = {"pass": "small step after a large pass (L2-cold)", "k": 1, "cache": cache, "bytes": b}
+                rec.update(dist(0, 1, cache, cold_after=4))
+                print(json.dumps(rec))
         for k in ks:
             ms = ctx.time_pass(1, k, cache, a.iters)
             b = pass_bytes(sL, wb, 4, cache, wl.enc_len, k)
-            print(json.dumps({"pass": "large block pass", "k": k, "cache": cache, "us": ms * 1e3, "GBs": b / ms / 1e6,
-                              "frac_of_peak": b / ms / 1e6 / peak, "bytes": b}))
+            rec = {"pass": "large block pass", "k": k, "cache": cache, "us": ms * 1e3, "GBs": b / ms / 1e6,
+                   "frac_of_peak": b / ms / 1e6 / peak, "frac_of_nominal": b / ms / 1e6 / nominal, "bytes": b}
+            rec.update(dist(1, k, cache))
+            print(json.dumps(rec))
 
 
 if __name__ == "__main__":
