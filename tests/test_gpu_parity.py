@@ -206,10 +206,13 @@ def test_generate_matches_golden(torch_cuda, name):
 
 @pytest.mark.parametrize("name", ["tiny", "odd_bf16"])
 @pytest.mark.parametrize("alpha_fb,alpha_rb,max_draft", [(0.0, INF, 10), (2.0, 0.0, 10), (0.3, -1.0, 10),
-                                                          (0.5, 15.5, 3), (0.2, 18.0, 15), (0.35, 16.5, 1)])
+                                                          (0.5, 15.5, 3), (0.2, 18.0, 15), (0.35, 16.5, 1),
+                                                          (0.0, 16.5, 5), (0.3, INF, 10)])
 def test_generate_matches_live_oracle(torch_cuda, name, alpha_fb, alpha_rb, max_draft):
     """Other thresholds and draft caps, including the policy's special cases (never fall
-    back, always fall back, always roll back)."""
+    back, always fall back, always roll back) and the two ablations of Section 4.4: no
+    fallback policy with a hand-over after a fixed number of small steps (alpha_fb = 0,
+    max_draft = window), and no rollback policy (alpha_rb = +inf)."""
     from paper_2302_07863_b200 import MODE_BILD
     ctx, ids, wl, g = get_ctx(name, max_draft=max_draft)
     S, L, _ = get_oracle(name)
