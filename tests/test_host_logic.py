@@ -84,3 +84,22 @@ def test_create_rejects_bad_arguments_without_a_gpu(L):
     assert L.bild_last_error(None) == b"null context"
     assert L.bild_op_linear(None, 0, None, None, 0.0, None, 1, 1, 8, None) == -1
     assert L.bild_op_lm_head_scratch_bytes(32128) > 0
+
+
+def test_model_analysis_counts():
+    """Analytic FLOPs / memory operations of the stored runs: the byte model agrees with the one the
+    benchmarks use, and BiLD trades slightly more FLOPs for several times fewer memory operations
+    than the large model alone (the direction of the paper's model-analysis figure)."""
+    from workloads import MODEL_SHAPES
+    from paper_2302_07863_b200 import microbench, model_analysis
+    s = MODEL_SHAPES["t5_l"]
+    for k, cache in [(1, 0), (5, 64), (16, 1024)]:
+        assert model_analysis.pass_counts(s, 2, 4, cache, 512, k)[1] == microbench.pass_bytes(s, 2, 4, cache, 512, k)
+    # one row, no cache, no encoder: 2 flops per weight plus one key
+    f, _ = model_analysis.pass_counts(s, 2, 4, 0, 0, 1)
+    params = s.n_layers * (6 * s.inner * s.d_model + 2 * s.d_model * s.d_ff) + s.vocab * s.d_model
+    assert f == 2 * params + 4 * s.inner * s.n_layers
+    r = model_analysis.analyse("t5_sum")["normalised"]
+    assert 1.0 < r["flops"] < 1.5
+    assert r["memory_operations"] < 0.5
+    assert abs(r["arithmetic_intensity"] - r["flops"] / r["memory_operations"]) < 1e-9
