@@ -2,7 +2,8 @@
 //   z[m][n] = scale * sum_j W[n][j] * rms_norm(x_m)[j]
 // Block b owns the vocabulary rows [b V / G, (b + 1) V / G).  They stream through a ring of
 // 16-row tiles in shared memory (one bulk copy per row, rows padded against bank conflicts; the
-// first tiles are requested before the dependency wait of the programmatic launch).  A tile
+// first tiles are requested before the dependency wait of the programmatic launch) by a ninth warp
+// that does nothing else (issuing a tile's copies costs about as much as multiplying it).  A tile
 // times the (up to 16) normalised token rows goes through mma.sync m16n8k16 (each activation as
 // a bf16 head and a bf16 remainder, fp32 accumulation), K split over the 8 warps and added in
 // warp order.  Thread (row r, token m) then folds the logit into its running (max, arg max,
@@ -15,11 +16,12 @@
 
 namespace bild {
 
-constexpr int SH_THREADS = 256;
+constexpr int SH_COMPUTE = 256;             // 8 warps multiply, reduce and fold
+constexpr int SH_THREADS = SH_COMPUTE + 32;  // + one warp that only requests tiles
 constexpr int SH_TILES = 3;   // ring depth
 
 struct SliceHeadShared {
-  unsigned long long full[SH_TILES];
+  unsigned long long full[SH_TILES], empty[SH_TILES];
   float scale[MAXB];
   int last, failed;
 };
@@ -44,15 +46,16 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
   const int ntiles = (ne - nb + 15) >> 4;
   const __nv_bfloat16* W = (const __nv_bfloat16*)a.W;
   if (tid == 0) {
-    for (int i = 0; i < SH_TILES; ++i) mg_mbar_init(smem_u32(&sh->full[i]), 1);
+    for (int i = 0; i < SH_TILES; ++i) { mg_mbar_init(smem_u32(&sh->full[i]), 1); mg_mbar_init(smem_u32(&sh->empty[i]), 1); }
     sh->failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  // warp 0 requests tile t: lane 0 announces the bytes, lanes 0..15 copy one row each (rows past the
-  // end of the slice repeat its last row; their logits are masked)
+  // the last warp requests tile t: lane 0 announces the bytes, lanes 0..15 copy one row each (rows past
+  // the end of the slice repeat its last row; their logits are masked).  Issuing the copies takes about
+  // as long as multiplying a tile, which is why the eight computing warps do not do it themselves.
   auto request = [&](int t) {
-    if (warp != 0 || t >= ntiles) return;
+    if (t >= ntiles) return;
     const int slot = t % SH_TILES;
     if (lane == 0) mg_mbar_expect(smem_u32(&sh->full[slot]), (uint32_t)(16 * K * 2));
     __syncwarp();
@@ -62,14 +65,27 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
                   smem_u32(&sh->full[slot]));
     }
   };
-  if (ntiles > 0)
-    for (int t = 0; t < SH_TILES; ++t) request(t);
   pdl_launch_dependents();
+  if (warp == SH_COMPUTE / 32) {   // producer: the weights depend on nothing, so it never waits for the kernel in front
+    for (int t = 0; t < SH_TILES; ++t) request(t);
+#pragma unroll 1
+    for (int t = SH_TILES; t < ntiles; ++t) {
+      const int slot = t % SH_TILES;
+      const uint32_t bar = smem_u32(&sh->empty[slot]), par = ((t / SH_TILES) - 1) & 1;
+      bool ok = mg_mbar_try(bar, par);
+      if (!ok && !*(volatile int*)&sh->failed) {
+        for (unsigned it = 0; it < MG_SPIN && !ok; ++it) ok = mg_mbar_try(bar, par);
+        if (!ok && lane == 0) { sh->failed = 1; atomicExch(err, (int)BILD_ERR_TIMEOUT); }
+      }
+      request(t);
+    }
+    return;
+  }
   pdl_wait();
   const int M = min(a.desc ? a.desc->k : a.M, MAXB);
   const int* target = a.desc ? a.desc->targets : a.target;
   // normalised token rows: x * g / rms (the head's own norm), fp32 in shared memory
-  for (int m = warp; m < M; m += SH_THREADS / 32) {
+  for (int m = warp; m < M; m += SH_COMPUTE / 32) {
     float ss = 0.f;
     for (int j = lane * 4; j < K; j += 128) {
       const float4 v = __ldcg(reinterpret_cast<const float4*>(a.X + (size_t)m * a.ldx + j));
@@ -86,7 +102,7 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
       *reinterpret_cast<float4*>(Xs + (size_t)m * xst + j) = v;
     }
   }
-  __syncthreads();
+  mg_csync();
   // thread <-> (row r of the tile, token m)
   const int er = tid & 15, em = tid >> 4;
   const int my_target = (em < M && target) ? target[em] : -1;
@@ -107,8 +123,8 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
     float* ps = psum + (t & 1) * (8 * 2 * 128);
     if (NT == 1) sl_mma<1>(sW + slot * tile_bytes, rowst, 16, K, Xs, xst, M, ps, warp, lane);
     else sl_mma<2>(sW + slot * tile_bytes, rowst, 16, K, Xs, xst, M, ps, warp, lane);
-    __syncthreads();   // partial sums complete; every warp is done with the tile
-    request(t + SH_TILES);
+    mg_csync();   // partial sums complete; every warp is done with the tile
+    if (tid == 0) mg_mbar_arrive(smem_u32(&sh->empty[slot]));   // the producer may refill it
     if (em < M) {
       // fragment layout of the accumulators: row = group (+ 8), token = 2 * (lane & 3) (+ 1)
       const int col = em & 7;
@@ -138,16 +154,16 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
   }
   if (er == 0 && em < M) a.partials[(size_t)blockIdx.x * MAXB + em] = run;
   __threadfence();
-  __syncthreads();
+  mg_csync();
   if (tid == 0) {
     const unsigned tk = atomicAdd(a.counter, 1u);
     sh->last = (tk == gridDim.x - 1);
     if (sh->last) *a.counter = 0;
   }
-  __syncthreads();
+  mg_csync();
   if (!sh->last) return;
   __threadfence();
-  for (int m = warp; m < M; m += SH_THREADS / 32) {
+  for (int m = warp; m < M; m += SH_COMPUTE / 32) {
     Partial p;
     p.m = -INFINITY; p.s = 0.f; p.idx = 0x7fffffff;
     for (int b = lane; b < (int)gridDim.x; b += 32) {
@@ -171,7 +187,7 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
       if (m == 0) a.out->pmax = 1.f / p.s;
     }
   }
-  __syncthreads();
+  mg_csync();
   if (tid == 0) {
     __threadfence();
     HeadOut* o = a.out;
