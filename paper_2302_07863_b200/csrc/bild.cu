@@ -161,7 +161,7 @@ struct bild_ctx {
   bool unit_attn = true;             // decoder attention on the 256-thread chunked kernel
   bool uattn_smem_set = false;
   bool enc_attn_mma = true;          // encoder self-attention on the mma.sync kernel (d_kv = 64)
-  int slice_head = 1;                // tensor-core LM head: 0 off, 1 block passes, 2 also single-row passes
+  int slice_head = 2;                // tensor-core LM head: 0 off, 1 block passes, 2 also single-row passes (large heads)
   bool slice_head_smem_set = false;
   int slice_mma_min = 3;
   size_t slice_min_bytes = 3000 * 1024;   // single-row passes: smaller matrices stay on the GEMV (measured)
@@ -906,7 +906,9 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   h.counter = m.head_cnt; h.out = m.head_out; h.logits_dbg = logits_dbg; h.which = which; h.loop = loop_ptrs(c);
   h.cond_while = cond_while; h.cond_if = cond_if;
   const size_t sh_smem = slice_head_smem_bytes(d);
-  if (c->slice_head >= (MB == 1 ? 2 : 1) && dt == BILD_BF16 && c->sms > 0 && c->sms <= MG_MAX_BLOCKS && sh_smem <= 200 * 1024 &&
+  // single-row passes: only heads of 48 MB and more (measured: the 33 MB head of the T5-small shape is faster on the GEMV head)
+  const bool big_head = (size_t)mc.vocab * d * 2 >= ((size_t)48 << 20);
+  if (c->slice_head >= (MB == 1 ? 2 : 1) && (MB != 1 || big_head) && dt == BILD_BF16 && c->sms > 0 && c->sms <= MG_MAX_BLOCKS && sh_smem <= 200 * 1024 &&
       d % 8 == 0 && ((uintptr_t)m.w.lm_head & 15) == 0) {
     // tensor-core head, one block per SM
     if (!c->slice_head_smem_set) {
