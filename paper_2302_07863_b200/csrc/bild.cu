@@ -905,7 +905,8 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   h.scale = mc.logit_scale; h.V = mc.vocab; h.K = d; h.desc = m.desc; h.partials = m.head_part;
   h.counter = m.head_cnt; h.out = m.head_out; h.logits_dbg = logits_dbg; h.which = which; h.loop = loop_ptrs(c);
   h.cond_while = cond_while; h.cond_if = cond_if;
-  const size_t sh_smem = slice_head_smem_bytes(d);
+  const int head_tr = (MB == 1 && d <= 512) ? 32 : 16;   // rows per tile of the tensor-core head
+  const size_t sh_smem = slice_head_smem_bytes(d, head_tr);
   // single-row passes: only heads of 48 MB and more (measured: the 33 MB head of the T5-small shape is faster on the GEMV head)
   const bool big_head = (size_t)mc.vocab * d * 2 >= ((size_t)48 << 20);
   if (c->slice_head >= (MB == 1 ? 2 : 1) && (MB != 1 || big_head) && dt == BILD_BF16 && c->sms > 0 && c->sms <= MG_MAX_BLOCKS && sh_smem <= 200 * 1024 &&
@@ -916,7 +917,7 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
       c->slice_head_smem_set = true;
     }
     CUDA_TRY(c, launch_k(c, slice_head_kernel, dim3(c->sms), dim3(SH_THREADS), sh_smem, h, which == 0 ? 0 : (MB == 1 ? 2 : 1),
-                         &c->st->err));
+                         &c->st->err, head_tr));
     return BILD_OK;
   }
   CUDA_TRY(c, launch_head(c->stream, dt, MB, h, m.head_grid, c->cnt));

@@ -26,24 +26,26 @@ struct SliceHeadShared {
   int last, failed;
 };
 
-__host__ __device__ inline size_t slice_head_tile_bytes(int K) { return (size_t)16 * (K * 2 + SL_WPAD); }
-inline size_t slice_head_smem_bytes(int K) {
-  return SH_TILES * slice_head_tile_bytes(K) + (size_t)MAXB * (K + SL_XPAD) * 4 + 2 * 8 * 2 * 128 * 4 + 1024;
+// tile_rows: 16, or 32 for short rows and at most 8 token rows (half as many barriers per byte)
+__host__ __device__ inline size_t slice_head_tile_bytes(int K, int tile_rows) { return (size_t)tile_rows * (K * 2 + SL_WPAD); }
+inline size_t slice_head_smem_bytes(int K, int tile_rows) {
+  return SH_TILES * slice_head_tile_bytes(K, tile_rows) + (size_t)MAXB * (K + SL_XPAD) * 4 + 2 * 8 * 2 * 128 * 4 + 1024;
 }
 
 // pass_kind: index of the pass counter the kernel bumps when it runs inside a loop graph
-__global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int pass_kind, int* err) {
+__global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int pass_kind, int* err, int TR) {
   extern __shared__ __align__(1024) unsigned char shd_smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K, V = a.V, G = gridDim.x;
   const int rowst = K * 2 + SL_WPAD, xst = K + SL_XPAD;
-  const size_t tile_bytes = slice_head_tile_bytes(K);
+  const size_t tile_bytes = slice_head_tile_bytes(K, TR);
+  const int tr_sh = TR == 32 ? 5 : 4;
   unsigned char* sW = shd_smem;
   float* Xs = reinterpret_cast<float*>(shd_smem + SH_TILES * tile_bytes);
   float* psum = Xs + (size_t)MAXB * xst;                 // [2][8 warps][2][32 lanes][4]
   SliceHeadShared* sh = reinterpret_cast<SliceHeadShared*>(psum + 2 * 8 * 2 * 128);
   const int nb = (int)(((long long)blockIdx.x * V) / G), ne = (int)(((long long)(blockIdx.x + 1) * V) / G);
-  const int ntiles = (ne - nb + 15) >> 4;
+  const int ntiles = (ne - nb + TR - 1) >> tr_sh;
   const __nv_bfloat16* W = (const __nv_bfloat16*)a.W;
   if (tid == 0) {
     for (int i = 0; i < SH_TILES; ++i) { mg_mbar_init(smem_u32(&sh->full[i]), 1); mg_mbar_init(smem_u32(&sh->empty[i]), 1); }
@@ -57,10 +59,10 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
   auto request = [&](int t) {
     if (t >= ntiles) return;
     const int slot = t % SH_TILES;
-    if (lane == 0) mg_mbar_expect(smem_u32(&sh->full[slot]), (uint32_t)(16 * K * 2));
+    if (lane == 0) mg_mbar_expect(smem_u32(&sh->full[slot]), (uint32_t)(TR * K * 2));
     __syncwarp();
-    if (lane < 16) {
-      const int n = min(nb + t * 16 + lane, ne - 1);
+    if (lane < TR) {
+      const int n = min(nb + t * TR + lane, ne - 1);
       mg_bulk_g2s(smem_u32(sW + slot * tile_bytes + (size_t)lane * rowst), W + (size_t)n * K, (uint32_t)(K * 2),
                   smem_u32(&sh->full[slot]));
     }
@@ -104,7 +106,8 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
   }
   mg_csync();
   // thread <-> (row r of the tile, token m)
-  const int er = tid & 15, em = tid >> 4;
+  const int er = tid & (TR - 1), em = tid >> tr_sh;
+  const int ks_sh = TR == 32 ? 2 : 3;   // the K range of a 16-row tile is split over 8 (4) warps
   const int my_target = (em < M && target) ? target[em] : -1;
   Partial run;
   run.m = -INFINITY; run.s = 0.f; run.idx = 0x7fffffff;
@@ -121,18 +124,17 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
       }
     }
     float* ps = psum + (t & 1) * (8 * 2 * 128);
-    if (NT == 1) sl_mma<1>(sW + slot * tile_bytes, rowst, 16, K, Xs, xst, M, ps, warp, lane);
-    else sl_mma<2>(sW + slot * tile_bytes, rowst, 16, K, Xs, xst, M, ps, warp, lane);
+    if (NT == 1) sl_mma<1>(sW + slot * tile_bytes, rowst, TR, K, Xs, xst, M, ps, warp, lane);
+    else sl_mma<2>(sW + slot * tile_bytes, rowst, TR, K, Xs, xst, M, ps, warp, lane);
     mg_csync();   // partial sums complete; every warp is done with the tile
     if (tid == 0) mg_mbar_arrive(smem_u32(&sh->empty[slot]));   // the producer may refill it
     if (em < M) {
       // fragment layout of the accumulators: row = group (+ 8), token = 2 * (lane & 3) (+ 1)
-      const int col = em & 7;
-      const float* p = ps + ((size_t)(em >> 3) * 32 + (er & 7) * 4 + (col >> 1)) * 4 + (er >> 3) * 2 + (col & 1);
+      const int col = em & 7, mt = er >> 4, rr = er & 15;
+      const float* p = ps + ((size_t)((mt << ks_sh) * NT + (em >> 3)) * 32 + (rr & 7) * 4 + (col >> 1)) * 4 + (rr >> 3) * 2 + (col & 1);
       float z = 0.f;
-#pragma unroll
-      for (int w = 0; w < 8; ++w) z += p[(size_t)w * NT * 128];
-      const int n = nb + t * 16 + er;
+      for (int w = 0; w < (1 << ks_sh); ++w) z += p[(size_t)w * NT * 128];
+      const int n = nb + t * TR + er;
       if (n < ne) {
         z *= a.scale;
         if (z > run.m) { run.s = run.s * expf(run.m - z) + 1.f; run.m = z; run.idx = n; }
@@ -143,9 +145,8 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
     }
     // the other half of psum is written next; this half is reused two tiles later, after another barrier
   }
-  // the 16 threads of a token combine (lanes 0..15 / 16..31 of a warp), lower row index first
-#pragma unroll
-  for (int o = 8; o > 0; o >>= 1) {
+  // the 16 (32) threads of a token combine (half a warp or a warp), lower row index first
+  for (int o = TR >> 1; o > 0; o >>= 1) {
     Partial q;
     q.m = __shfl_xor_sync(0xffffffffu, run.m, o);
     q.s = __shfl_xor_sync(0xffffffffu, run.s, o);
