@@ -163,6 +163,7 @@ struct bild_ctx {
   bool enc_attn_mma = true;          // encoder self-attention on the mma.sync kernel (d_kv = 64)
   int slice_head = 2;                // tensor-core LM head: 0 off, 1 block passes, 2 also single-row passes (large heads)
   bool slice_head_smem_set = false;
+  size_t slice_head_min_bytes = (size_t)32 << 20;
   int slice_mma_min = 3;
   size_t slice_min_bytes = 3000 * 1024;   // single-row passes: smaller matrices stay on the GEMV (measured)
   bool mega_coop = true;             // launch the whole-pass kernel with the cooperative attribute
@@ -907,8 +908,8 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   h.cond_while = cond_while; h.cond_if = cond_if;
   const int head_tr = (MB == 1 && d <= 512) ? 32 : 16;   // rows per tile of the tensor-core head
   const size_t sh_smem = slice_head_smem_bytes(d, head_tr);
-  // single-row passes: only heads of 48 MB and more (measured: the 33 MB head of the T5-small shape is faster on the GEMV head)
-  const bool big_head = (size_t)mc.vocab * d * 2 >= ((size_t)48 << 20);
+  // single-row passes: only heads of 32 MB and more (smaller ones stay on the GEMV head)
+  const bool big_head = (size_t)mc.vocab * d * 2 >= c->slice_head_min_bytes;
   if (c->slice_head >= (MB == 1 ? 2 : 1) && (MB != 1 || big_head) && dt == BILD_BF16 && c->sms > 0 && c->sms <= MG_MAX_BLOCKS && sh_smem <= 200 * 1024 &&
       d % 8 == 0 && ((uintptr_t)m.w.lm_head & 15) == 0) {
     // tensor-core head, one block per SM
@@ -1169,6 +1170,8 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
       c->sms = 0;
     }
   }
+  const char* shm = std::getenv("BILD_SLICE_HEAD_MIN_MB");
+  if (shm) c->slice_head_min_bytes = (size_t)std::max(0, std::atoi(shm)) << 20;
   const char* shd = std::getenv("BILD_SLICE_HEAD");
   if (shd && shd[0] >= '0' && shd[0] <= '2') c->slice_head = shd[0] - '0';
   const char* ea = std::getenv("BILD_ENC_ATTN_MMA");
