@@ -371,3 +371,21 @@ def test_persistent_pass_full_size(torch_cuda):
         assert r["tokens"] == g["bild"]["tokens"]
         assert r["stats"] == g["bild"]["stats"]
     ctx.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", ["tiny", "tiny_bf16"])
+def test_large_cache_capacity_matches_golden(torch_cuda, name):
+    """A context sized for the longest sequences (2048 decoder positions, 2048 encoder positions) splits the
+    keys of every attention over eight blocks per head; tokens, trace and statistics do not change."""
+    from paper_2302_07863_b200 import MODE_BILD
+    from paper_2302_07863_b200.synthetic import make_context
+    g = golden(name)
+    ctx, ids, wl = make_context(name, g["scale_small"]["scale"], g["scale_large"]["scale"], max_enc_len=2048, max_dec_len=2048)
+    ctx.encode(ids)
+    th = g["thresholds"]
+    r = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
+    assert r["tokens"] == g["bild"]["tokens"]
+    assert_trace_equal(r["trace"], g["bild"]["trace"], 1e-3)
+    assert r["stats"] == g["bild"]["stats"]
+    ctx.close()
