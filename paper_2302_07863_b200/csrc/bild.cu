@@ -841,7 +841,7 @@ LoopPtrs loop_ptrs(bild_ctx* c) {
 // norm+cross-Q, cross-attention, cross-O+residual, norm+FFN-up, FFN-down+residual],
 // final norm + LM head + policy).  MB = 1 or MAXB selects the kernel variants.
 int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned long long cond_while = 0,
-                 unsigned long long cond_if = 0) {
+                 unsigned long long cond_if = 0, unsigned long long cond_if1 = 0) {
   Model& m = c->m[which];
   const bild_model_cfg& mc = m.c;
   const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
@@ -905,7 +905,7 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   h.W = m.w.lm_head; h.X = m.x; h.ldx = d; h.gain = (const float*)m.w.dec_final_ln; h.eps = mc.ln_eps;
   h.scale = mc.logit_scale; h.V = mc.vocab; h.K = d; h.desc = m.desc; h.partials = m.head_part;
   h.counter = m.head_cnt; h.out = m.head_out; h.logits_dbg = logits_dbg; h.which = which; h.loop = loop_ptrs(c);
-  h.cond_while = cond_while; h.cond_if = cond_if;
+  h.cond_while = cond_while; h.cond_if = cond_if; h.cond_if1 = cond_if1;
   const int head_tr = (MB == 1 && d <= 512) ? 32 : 16;   // rows per tile of the tensor-core head
   const size_t sh_smem = slice_head_smem_bytes(d, head_tr);
   // single-row passes: only heads of 32 MB and more (smaller ones stay on the GEMV head)
@@ -1012,7 +1012,7 @@ int add_cond(bild_ctx* c, cudaGraph_t g, const cudaGraphNode_t* deps, size_t nde
 
 // Captures one decoder pass into `body`; returns the leaf nodes of the capture.
 int capture_pass(bild_ctx* c, cudaGraph_t body, int which, int MB, unsigned long long hw, unsigned long long hi,
-                 std::vector<cudaGraphNode_t>* leaves, int64_t* count) {
+                 std::vector<cudaGraphNode_t>* leaves, int64_t* count, unsigned long long hi1 = 0) {
   if (!c->cap_stream) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
   CUDA_TRY(c, cudaStreamBeginCaptureToGraph(c->cap_stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed));
   int64_t n = 0;
@@ -1020,7 +1020,7 @@ int capture_pass(bild_ctx* c, cudaGraph_t body, int which, int MB, unsigned long
   c->stream = c->cap_stream;
   c->cnt = &n;
   c->capturing = true;
-  int rc = decoder_pass(c, which, MB, nullptr, hw, hi);
+  int rc = decoder_pass(c, which, MB, nullptr, hw, hi, hi1);
   c->capturing = false;
   c->cnt = &c->launches;
   c->stream = user_stream;
@@ -1071,21 +1071,29 @@ int build_graphs(bild_ctx* c) {
 }
 
 int build_graphs_once(bild_ctx* c) {
-  {  // BiLD (and small-only): WHILE { small pass ; IF { large block pass } }
+  {  // BiLD (and small-only): WHILE { small pass ; IF { large block pass } ; IF { large single-row pass } }
     CUDA_TRY(c, cudaGraphCreate(&c->graph[0], 0));
-    cudaGraphConditionalHandle hw, hi;
+    cudaGraphConditionalHandle hw, hi, hi1;
     CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hw, c->graph[0], 1, cudaGraphCondAssignDefault));
     CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi, c->graph[0], 0, cudaGraphCondAssignDefault));
-    cudaGraph_t body = nullptr, ifbody = nullptr;
+    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi1, c->graph[0], 0, cudaGraphCondAssignDefault));
+    cudaGraph_t body = nullptr, ifbody = nullptr, if1body = nullptr;
     int rc = add_cond(c, c->graph[0], nullptr, 0, hw, cudaGraphCondTypeWhile, &body);
     if (rc) return rc;
     std::vector<cudaGraphNode_t> leaves;
-    rc = capture_pass(c, body, 0, 1, hw, hi, &leaves, &c->per_pass[0]);
+    rc = capture_pass(c, body, 0, 1, hw, hi, &leaves, &c->per_pass[0], hi1);
     if (rc) return rc;
     rc = add_cond(c, body, leaves.data(), leaves.size(), hi, cudaGraphCondTypeIf, &ifbody);
     if (rc) return rc;
     rc = capture_pass(c, ifbody, 1, MAXB, hw, 0, nullptr, &c->per_pass[1]);
     if (rc) return rc;
+    // a fallback right after a large pass verifies one row: that pass runs on the single-row kernels
+    rc = add_cond(c, body, leaves.data(), leaves.size(), hi1, cudaGraphCondTypeIf, &if1body);
+    if (rc) return rc;
+    int64_t n1 = 0;
+    rc = capture_pass(c, if1body, 1, 1, hw, 0, nullptr, &n1);
+    if (rc) return rc;
+    c->per_pass_large1 = n1;
     CUDA_TRY(c, cudaGraphInstantiate(&c->exec[0], c->graph[0], 0));
   }
   {  // large-only greedy: WHILE { large pass with k = 1 }

@@ -706,7 +706,10 @@ __global__ void __launch_bounds__(HEAD1_THREADS) head1_kernel(HeadArgs a) {
         a.loop.st->cum_passes[a.which == 0 ? 0 : 2]++;
         cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
       }
-      if (a.cond_if) cudaGraphSetConditional(a.cond_if, a.loop.st->fallback ? 1u : 0u);
+      // the large pass wanted next: the single-row graph branch if it has one row (and that branch exists), else the block branch
+      const bool one_row = a.cond_if1 && a.loop.st->fallback && a.loop.descL->k == 1;
+      if (a.cond_if) cudaGraphSetConditional(a.cond_if, (a.loop.st->fallback && !one_row) ? 1u : 0u);
+      if (a.cond_if1) cudaGraphSetConditional(a.cond_if1, one_row ? 1u : 0u);
     }
   }
 }

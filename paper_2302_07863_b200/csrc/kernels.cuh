@@ -477,6 +477,7 @@ struct HeadArgs {
   LoopPtrs loop;  // loop.st may be nullptr (single-operation entry point)
   // handles of the graph's WHILE (loop goes on) and IF (large pass wanted) nodes; 0 = not in a graph
   unsigned long long cond_while, cond_if;
+  unsigned long long cond_if1;   // IF node of the single-row large pass (0: the block branch takes every large pass)
 };
 
 constexpr int HEAD_THREADS = 256;
@@ -621,7 +622,10 @@ __global__ void __launch_bounds__(HEAD_THREADS) lm_head_kernel(HeadArgs a) {
         a.loop.st->cum_passes[a.which == 0 ? 0 : (MB == 1 ? 2 : 1)]++;
         cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
       }
-      if (a.cond_if) cudaGraphSetConditional(a.cond_if, a.loop.st->fallback ? 1u : 0u);
+      // the large pass wanted next: the single-row graph branch if it has one row (and that branch exists), else the block branch
+      const bool one_row = a.cond_if1 && a.loop.st->fallback && a.loop.descL->k == 1;
+      if (a.cond_if) cudaGraphSetConditional(a.cond_if, (a.loop.st->fallback && !one_row) ? 1u : 0u);
+      if (a.cond_if1) cudaGraphSetConditional(a.cond_if1, one_row ? 1u : 0u);
     }
   }
 }
