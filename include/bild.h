@@ -163,7 +163,11 @@ void bild_destroy(bild_ctx *ctx); /* frees the host-side context only */
 /* Run both encoders over ids[0..n_ids) and project the cross-attention K/V of
  * every decoder layer (the per-input set-up of Algorithm 1's two models).  Resets
  * the decode state: y = [start_id], both caches empty.  1 <= n_ids <= max_enc_len.
- * Asynchronous on the stream (ids are copied before returning). */
+ * Asynchronous on the stream (ids are copied before returning).  The small model's
+ * encoder runs on a stream of the context's own, forked from and joined back into the
+ * caller's stream with events, so work queued on the caller's stream after this call still
+ * sees both encoders' results (BILD_ENC_SERIAL=1 in the environment keeps everything on the
+ * caller's stream). */
 int bild_encode(bild_ctx *ctx, const int32_t *ids /*HOST*/, int n_ids);
 
 /* Reset the decode state only (keeps the encoder results of the last bild_encode). */

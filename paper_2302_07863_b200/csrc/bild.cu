@@ -112,6 +112,7 @@ struct Model {
   // encoder GEMM: descriptors of the bf16 head / remainder matrices of the layer input, by row length (d, inner, d_ff)
   CUtensorMap tmH[2][3][2];   // [buffer pair][row length d / inner / d_ff][head, remainder]
   bool enc_gemm = false;
+  int index = 0;   // 0 small, 1 large
   // whole-pass persistent kernel (bf16 only)
   MegaLayer* mega_layers = nullptr;
   unsigned* mega_sync = nullptr;
@@ -136,8 +137,14 @@ struct bild_ctx {
   int* enc_ids = nullptr;
   int* enc_len_dev = nullptr;
   int* bucket_tmp = nullptr;
-  float *ex = nullptr, *eq = nullptr, *ek = nullptr, *ev = nullptr, *eatt = nullptr, *eu = nullptr;
-  __nv_bfloat16 *exh[2] = {nullptr, nullptr}, *exl[2] = {nullptr, nullptr};   // two pairs (bf16 head, remainder) of encoder layer inputs
+  // encoder temporaries, one set per model (the two encoders run side by side on two streams)
+  struct EncBuf {
+    float *ex = nullptr, *eq = nullptr, *ek = nullptr, *ev = nullptr, *eatt = nullptr, *eu = nullptr;
+    __nv_bfloat16 *exh[2] = {nullptr, nullptr}, *exl[2] = {nullptr, nullptr};   // two pairs (bf16 head, remainder) of layer inputs
+  } eb[2];
+  cudaStream_t enc_stream = nullptr;   // the small model's encoder runs here, the large model's on the caller's stream
+  cudaEvent_t enc_fork = nullptr, enc_join = nullptr;
+  bool enc_parallel = true;
   int enc_len = 0;
   bool encoded = false;
   int64_t launches = 0;
@@ -229,13 +236,12 @@ void plan(bild_ctx* c, Bump& b) {
   c->enc_ids = b.take<int>(ecap);
   c->enc_len_dev = b.take<int>(1);
   c->bucket_tmp = b.take<int>(std::max(cap, 2 * ecap));
-  int dmax = 0, imax = 0, fmax = 0;
   for (int i = 0; i < 2; ++i) {
     Model& m = c->m[i];
     const bild_model_cfg& mc = i == 0 ? cfg.small_cfg : cfg.large_cfg;
     m.c = mc;
+    m.index = i;
     m.inner = mc.n_heads * mc.d_kv;
-    dmax = std::max(dmax, mc.d_model); imax = std::max(imax, m.inner); fmax = std::max(fmax, mc.d_ff);
     const size_t kv = (size_t)mc.n_layers * mc.n_heads * mc.d_kv;
     m.selfK = b.take<float>(kv * cap);
     m.selfV = b.take<float>(kv * cap);
@@ -260,16 +266,21 @@ void plan(bild_ctx* c, Bump& b) {
     m.mega_ll = b.take<uint2>(m.mega_ll_pairs);
   }
   const size_t ecap16 = (size_t)(ecap + MAXB - 1) / MAXB * MAXB;   // whole blocks of MAXB rows
-  c->ex = b.take<float>(ecap16 * dmax);
-  c->eq = b.take<float>(ecap16 * imax);
-  c->ek = b.take<float>((size_t)ecap * imax);
-  c->ev = b.take<float>((size_t)ecap * imax);
-  c->eatt = b.take<float>(ecap16 * imax);
-  c->eu = b.take<float>(ecap16 * fmax);
   const size_t ecap128 = (size_t)(ecap + EG_TOK - 1) / EG_TOK * EG_TOK;   // whole tiles of 128 tokens
   for (int i = 0; i < 2; ++i) {
-    c->exh[i] = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(dmax, imax), fmax));
-    c->exl[i] = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(dmax, imax), fmax));
+    const bild_model_cfg& mc = i == 0 ? cfg.small_cfg : cfg.large_cfg;
+    const size_t d = mc.d_model, I = (size_t)mc.n_heads * mc.d_kv, F = mc.d_ff;
+    bild_ctx::EncBuf& e = c->eb[i];
+    e.ex = b.take<float>(ecap16 * d);
+    e.eq = b.take<float>(ecap16 * I);
+    e.ek = b.take<float>((size_t)ecap * I);
+    e.ev = b.take<float>((size_t)ecap * I);
+    e.eatt = b.take<float>(ecap16 * I);
+    e.eu = b.take<float>(ecap16 * F);
+    for (int pr = 0; pr < 2; ++pr) {
+      e.exh[pr] = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(d, I), F));
+      e.exl[pr] = b.take<__nv_bfloat16>(ecap128 * std::max(std::max(d, I), F));
+    }
   }
   b.off = align_up(b.off, 256);
 }
@@ -575,7 +586,8 @@ void setup_umma(bild_ctx* c, Model& m) {
   const int Ks[3] = {mc.d_model, m.inner, mc.d_ff};
   for (int pr = 0; pr < 2; ++pr)
     for (int i = 0; i < 3; ++i)
-      if (!make_tmap(enc, c->exh[pr], ecap128, Ks[i], &m.tmH[pr][i][0]) || !make_tmap(enc, c->exl[pr], ecap128, Ks[i], &m.tmH[pr][i][1])) return;
+      if (!make_tmap(enc, c->eb[m.index].exh[pr], ecap128, Ks[i], &m.tmH[pr][i][0]) ||
+          !make_tmap(enc, c->eb[m.index].exl[pr], ecap128, Ks[i], &m.tmH[pr][i][1])) return;
   if (cudaFuncSetAttribute(enc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)eg_smem_bytes<false>()) != cudaSuccess ||
       cudaFuncSetAttribute(enc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)eg_smem_bytes<true>()) != cudaSuccess) {
     cudaGetLastError();
@@ -802,13 +814,13 @@ cudaError_t launch_enc_gemm(bild_ctx* c, Model& m, const LinArgs& a, int layer, 
   const int ki = a.K == m.c.d_model ? 0 : a.K == m.inner ? 1 : 2;
   if (split) {
     cudaError_t e = launch_k(c, norm_split_kernel, dim3(tiles_tok * EG_TOK / 4), dim3(128), 0, a.X, a.ldx, a.gain, a.eps, E, a.K,
-                             c->exh[pair], c->exl[pair]);
+                             c->eb[m.index].exh[pair], c->eb[m.index].exl[pair]);
     if (e != cudaSuccess) return e;
   }
   const CUtensorMap* t = &m.tmaps[(size_t)layer * TM_PER_LAYER];
   const bool gated = a.epi == EPI_GATED;
-  __nv_bfloat16* oh = out_pair >= 0 ? c->exh[out_pair] : nullptr;
-  __nv_bfloat16* ol = out_pair >= 0 ? c->exl[out_pair] : nullptr;
+  __nv_bfloat16* oh = out_pair >= 0 ? c->eb[m.index].exh[out_pair] : nullptr;
+  __nv_bfloat16* ol = out_pair >= 0 ? c->eb[m.index].exl[out_pair] : nullptr;
   dim3 grid((a.N + UM_TILE_M - 1) / UM_TILE_M, tiles_tok);
   if (gated)
     return launch_k(c, enc_gemm_kernel<true>, grid, dim3(EG_THREADS), eg_smem_bytes<true>(), a, &c->st->err, oh, ol, t[which_map],
@@ -929,44 +941,45 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
 // every decoder layer.
 int encoder_pass(bild_ctx* c, int which) {
   Model& m = c->m[which];
+  bild_ctx::EncBuf& B = c->eb[which];
   const bild_model_cfg& mc = m.c;
   const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
   const int E = c->enc_len, ecap = c->cfg.max_enc_len, dt = c->cfg.dtype;
   const int rb = (E + MAXB - 1) / MAXB;
-  CUDA_TRY(c, launch_embed(c, m.w.emb, c->enc_ids, nullptr, E, E, d, mc.vocab, c->ex));
+  CUDA_TRY(c, launch_embed(c, m.w.emb, c->enc_ids, nullptr, E, E, d, mc.vocab, B.ex));
   for (int l = 0; l < mc.n_layers; ++l) {
     const bild_enc_layer& w = m.enc[l];
     LinArgs a{};
-    a.M = E; a.eps = mc.ln_eps; a.W0 = w.wqkv; a.X = c->ex; a.ldx = d; a.gain = (const float*)w.ln1;
-    a.N = 3 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 0; a.q_out = c->eq; a.ldq = I;
-    a.kc = c->ek; a.vc = c->ev; a.cap = ecap; a.pos0_host = 0;
+    a.M = E; a.eps = mc.ln_eps; a.W0 = w.wqkv; a.X = B.ex; a.ldx = d; a.gain = (const float*)w.ln1;
+    a.N = 3 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 0; a.q_out = B.eq; a.ldq = I;
+    a.kc = B.ek; a.vc = B.ev; a.cap = ecap; a.pos0_host = 0;
     // with the GEMM path the layer inputs alternate between two (bf16 head, remainder) buffer pairs:
     // norm(x) -> pair 0 -> QKV; attention -> pair 1 -> O; norm(x) -> pair 0 -> FFN-up -> pair 1 -> FFN-down
     const bool fuse = m.enc_gemm && c->enc_attn_mma && dkv == EA_D;
     CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_EQKV, true, 0));
     BAttnArgs t{};
-    t.q = c->eq; t.ldq = I; t.kc = c->ek; t.vc = c->ev; t.cap = ecap; t.out = c->eatt; t.ldo = I;
+    t.q = B.eq; t.ldq = I; t.kc = B.ek; t.vc = B.ev; t.cap = ecap; t.out = B.eatt; t.ldo = I;
     t.bias = m.enc_bias; t.bias_ld = 2 * ecap - 1; t.bias_off = ecap - 1; t.mode = 2; t.dkv = dkv; t.H = H;
     t.n_keys_dev = c->enc_len_dev; t.M = E; t.part = m.att_part; t.counters = m.att_cnt; t.nsplit = 1;
     t.err = &c->st->err;
-    CUDA_TRY(c, launch_battn(c, MAXB, t, rb, ecap, fuse ? c->exh[1] : nullptr, fuse ? c->exl[1] : nullptr));
+    CUDA_TRY(c, launch_battn(c, MAXB, t, rb, ecap, fuse ? B.exh[1] : nullptr, fuse ? B.exl[1] : nullptr));
     LinArgs o{};
-    o.M = E; o.W0 = w.wo; o.X = c->eatt; o.ldx = I; o.N = d; o.K = I; o.epi = EPI_RESID; o.Y = c->ex; o.ldy = d;
+    o.M = E; o.W0 = w.wo; o.X = B.eatt; o.ldx = I; o.N = d; o.K = I; o.epi = EPI_RESID; o.Y = B.ex; o.ldy = d;
     CUDA_TRY(c, launch_enc_linear(c, m, o, rb, l, TM_EO, !fuse, 1));
     LinArgs up{};
-    up.M = E; up.eps = mc.ln_eps; up.W0 = w.wi0; up.W1 = w.wi1; up.X = c->ex; up.ldx = d; up.gain = (const float*)w.ln2;
-    up.N = F; up.K = d; up.Y = c->eu; up.ldy = F;
+    up.M = E; up.eps = mc.ln_eps; up.W0 = w.wi0; up.W1 = w.wi1; up.X = B.ex; up.ldx = d; up.gain = (const float*)w.ln2;
+    up.N = F; up.K = d; up.Y = B.eu; up.ldy = F;
     up.epi = mc.ffn_kind == BILD_FFN_GATED_GELU ? EPI_GATED : EPI_RELU;
     CUDA_TRY(c, launch_enc_linear(c, m, up, rb, l, TM_EWI0, true, 0, m.enc_gemm ? 1 : -1));
     LinArgs dn{};
-    dn.M = E; dn.W0 = w.wfo; dn.X = c->eu; dn.ldx = F; dn.N = d; dn.K = F; dn.epi = EPI_RESID; dn.Y = c->ex; dn.ldy = d;
+    dn.M = E; dn.W0 = w.wfo; dn.X = B.eu; dn.ldx = F; dn.N = d; dn.K = F; dn.epi = EPI_RESID; dn.Y = B.ex; dn.ldy = d;
     CUDA_TRY(c, launch_enc_linear(c, m, dn, rb, l, TM_EFO, !m.enc_gemm, 1));
   }
   // encoder memory = final norm of ex (fused into the projections); cross K/V per decoder layer
   for (int l = 0; l < mc.n_layers; ++l) {
     const size_t kvoff = (size_t)l * H * dkv;
     LinArgs a{};
-    a.M = E; a.eps = mc.ln_eps; a.W0 = m.dec[l].wckv; a.X = c->ex; a.ldx = d; a.gain = (const float*)m.w.enc_final_ln;
+    a.M = E; a.eps = mc.ln_eps; a.W0 = m.dec[l].wckv; a.X = B.ex; a.ldx = d; a.gain = (const float*)m.w.enc_final_ln;
     a.N = 2 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 1;
     a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.pos0_host = 0;
     CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_CKV, l == 0, 0));   // the normalised encoder output is split once
@@ -1188,6 +1201,8 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   if (ua && ua[0] == '0') c->unit_attn = false;
   const char* mm = std::getenv("BILD_SLICE_MMA_MIN");
   if (mm) c->slice_mma_min = std::min(5, std::max(2, std::atoi(mm)));
+  const char* es = std::getenv("BILD_ENC_SERIAL");
+  if (es && es[0] == '1') c->enc_parallel = false;
   const char* sm = std::getenv("BILD_SLICE_MIN_KB");
   if (sm) c->slice_min_bytes = (size_t)std::atoi(sm) * 1024;
   const char* np = std::getenv("BILD_NO_PDL");
@@ -1240,6 +1255,9 @@ void bild_destroy(bild_ctx* c) {
   if (!c) return;
   drop_graphs(c);
   if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+  if (c->enc_stream) { cudaStreamSynchronize(c->enc_stream); cudaStreamDestroy(c->enc_stream); }
+  if (c->enc_fork) cudaEventDestroy(c->enc_fork);
+  if (c->enc_join) cudaEventDestroy(c->enc_join);
   if (c->pin_state) cudaFreeHost(c->pin_state);
   if (c->pin_head) cudaFreeHost(c->pin_head);
   delete c;
@@ -1257,9 +1275,34 @@ int bild_encode(bild_ctx* c, const int32_t* ids, int n_ids) {
   c->enc_len = n_ids;
   CUDA_TRY(c, cudaMemcpyAsync(c->enc_ids, ids, n_ids * sizeof(int), cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(c, cudaMemcpyAsync(c->enc_len_dev, &c->enc_len, sizeof(int), cudaMemcpyHostToDevice, c->stream));
-  for (int i = 0; i < 2; ++i) {
-    int rc = encoder_pass(c, i);
-    if (rc) return rc;
+  // The two encoders are independent: the small model's runs on a side stream, forked from and joined
+  // back into the caller's stream with events, while the large model's runs on the caller's stream.
+  bool side = c->enc_parallel;
+  if (side && !c->enc_stream) {
+    if (cudaStreamCreateWithFlags(&c->enc_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->enc_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->enc_join, cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      side = c->enc_parallel = false;
+    }
+  }
+  if (side) {
+    CUDA_TRY(c, cudaEventRecord(c->enc_fork, c->stream));
+    CUDA_TRY(c, cudaStreamWaitEvent(c->enc_stream, c->enc_fork, 0));
+    cudaStream_t user_stream = c->stream;
+    c->stream = c->enc_stream;
+    int rc0 = encoder_pass(c, 0);
+    c->stream = user_stream;
+    if (rc0) return rc0;
+    CUDA_TRY(c, cudaEventRecord(c->enc_join, c->enc_stream));
+    int rc1 = encoder_pass(c, 1);
+    if (rc1) return rc1;
+    CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->enc_join, 0));
+  } else {
+    for (int i = 0; i < 2; ++i) {
+      int rc = encoder_pass(c, i);
+      if (rc) return rc;
+    }
   }
   int rc = reset_state(c, BILD_MODE_BILD, 0.f, INFINITY, c->cfg.max_dec_len - 1);
   if (rc) return rc;

@@ -231,7 +231,7 @@ def test_generate_matches_live_oracle(torch_cuda, name, alpha_fb, alpha_rb, max_
 
 @pytest.mark.parametrize("env", ["BILD_BLOCK_SIMT=1", "BILD_HOST_LOOP=1", "BILD_NO_PDL=1", "BILD_NO_UMMA=1", "BILD_MEGA=1",
                                  "BILD_SLICE=0", "BILD_SLICE=2", "BILD_SLICE_MMA_MIN=5", "BILD_UNIT_ATTN=0", "BILD_SLICE_HEAD=0",
-                                 "BILD_SLICE_HEAD=1", "BILD_ENC_GEMM=0"])
+                                 "BILD_SLICE_HEAD=1", "BILD_ENC_GEMM=0", "BILD_ENC_SERIAL=1"])
 @pytest.mark.parametrize("name", ["tiny_bf16", "odd"])
 def test_alternative_paths_match_golden(torch_cuda, name, env):
     """The switchable paths (SIMT block GEMV, host-driven loop, plain launches, no tcgen05 kernels, persistent
