@@ -55,7 +55,8 @@ def test_workspace_query_and_validation(L):
     s, l = MODEL_SHAPES["t5_s"], MODEL_SHAPES["t5_l"]
     # at least the self- and cross-attention K/V of both models (fp32)
     need = sum(2 * m.n_layers * m.inner * (65 + 512) * 4 for m in (s, l))
-    assert need <= n.value <= need + 64 * 2 ** 20
+    # ... plus activations, per-model encoder temporaries (fp32 and bf16 pairs), head partials, exchange areas
+    assert need <= n.value <= need + 96 * 2 ** 20
     n2 = C.c_size_t()
     assert L.bild_query_workspace(C.byref(_cfg(max_dec_len=257)), C.byref(n2)) == 0 and n2.value > n.value
     for bad in (dict(max_draft=0), dict(max_draft=16), dict(max_enc_len=0), dict(max_dec_len=1), dict(dtype=7),
