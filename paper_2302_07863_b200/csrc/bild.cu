@@ -351,7 +351,7 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
         c->uattn_smem_set = true;
       }
       cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(a0.H, a0.nsplit, row_blocks); cfg.blockDim = dim3(UA_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+      cfg.gridDim = dim3(a0.H, a0.nsplit, row_blocks); cfg.blockDim = dim3(MB == 1 ? UA_THREADS : UA_THREADS_MAX); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
       cudaLaunchAttribute at[2];
       int na = 0;
       if (c->use_pdl) {

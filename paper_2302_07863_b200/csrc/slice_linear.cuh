@@ -17,7 +17,9 @@
 //     a tile and added in warp order.  Rows in shared memory are padded so that the fragment
 //     loads do not collide on banks;
 //   * the epilogues are those of the other linear kernels (store, ReLU, GELU gate, residual add,
-//     scatter to q / the KV cache).
+//     scatter to q / the KV cache); a thread owns one output row of the slice and every 4th, 8th
+//     or 16th token row, the shorter the slice the more token rows per turn (a slice has 7 to 28
+//     rows for the T5-large shapes, so five to sixteen token rows finish in one turn).
 #pragma once
 #include "decode_kernels.cuh"
 #include "mega_pass.cuh"
@@ -210,17 +212,21 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
   pdl_wait();
   const int M = min(a.desc->k, MAXB), pos0 = a.desc->pos0;
   const int nkb = (K + 255) >> 8, rgl = s.x_rows;
+  // epilogue: thread <-> (output row ep_r of the slice, token rows ep_m, ep_m + ep_step, ...); short slices take
+  // more token rows per turn (16 / 8 / 4 for slices of up to 16 / 32 / 64 rows)
+  const int ep_sh = n <= 16 ? 4 : n <= 32 ? 5 : 6;
+  const int ep_r = tid & ((1 << ep_sh) - 1), ep_m = tid >> ep_sh, ep_step = SL_THREADS >> ep_sh;
   unsigned xuse = 0;
 #pragma unroll 1
   for (int m0 = 0; m0 < M; m0 += rgl, ++xuse) {
     const int mg = min(rgl, M - m0);
     // the values a residual epilogue adds to are requested now, not when the sums are ready
     float y_old[4] = {0.f, 0.f, 0.f, 0.f};
-    if (a.epi == EPI_RESID && (tid & 63) < n) {
+    if (a.epi == EPI_RESID && ep_r < n) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const int m = (tid >> 6) + 4 * i;
-        if (m < mg) y_old[i] = __ldcg(a.Y + (size_t)(m0 + m) * a.ldy + r0 + (tid & 63));
+        const int m = ep_m + ep_step * i;
+        if (m < mg) y_old[i] = __ldcg(a.Y + (size_t)(m0 + m) * a.ldy + r0 + ep_r);
       }
     }
     if (mg <= SL_PLAIN_ROWS) {
@@ -317,9 +323,9 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
     const int MT = (nrows + 15) >> 4, ks_sh = MT == 1 ? 3 : MT == 2 ? 2 : 1, NT = mg <= 8 ? 1 : 2;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const int m = (tid >> 6) + 4 * i;
+      const int m = ep_m + ep_step * i;
       if (m >= mg) break;
-      const int r = tid & 63;
+      const int r = ep_r;
       if (r >= n) continue;
       auto total = [&](int row) {
         float t = 0.f;
