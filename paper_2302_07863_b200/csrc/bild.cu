@@ -346,7 +346,8 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
     const size_t smem = uattn_smem_floats(MB, a0.dkv, a0.nsplit, bias_len) * sizeof(float);
     if (smem <= 200 * 1024) {
       if (smem > 48 * 1024 && !c->uattn_smem_set) {
-        cudaError_t e = cudaFuncSetAttribute(uattn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(uattn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(uattn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
         c->uattn_smem_set = true;
       }
@@ -366,7 +367,7 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
       }
       cfg.attrs = at; cfg.numAttrs = na;
       (*c->cnt)++;
-      return cudaLaunchKernelEx(&cfg, uattn_kernel, d, bias_len);
+      return MB == 1 ? cudaLaunchKernelEx(&cfg, uattn_kernel<true>, d, bias_len) : cudaLaunchKernelEx(&cfg, uattn_kernel<false>, d, bias_len);
     }
   }
   if (a0.mode == 2 && a0.dkv == EA_D && c->enc_attn_mma) {   // encoder: 64-row tiles on mma.sync

@@ -30,9 +30,11 @@ struct UAttnShared {
 // floats of dynamic shared memory
 inline size_t uattn_smem_floats(int MB, int dkv, int nsplit, int bias_len) {
   return (size_t)4 * UA_CK * dkv + (size_t)MB * dkv + (size_t)MB * UA_CK + (size_t)bias_len + (size_t)nsplit * MB * (dkv + 2) +
-         (sizeof(UAttnShared) + 3) / 4 + 8;
+         (sizeof(UAttnShared) + 3) / 4 + 8 + 4 * 64;   // ... + the single-row value phase's partial sums
 }
 
+// ONE: instantiation for single-row passes (its score and value phases use all 256 threads for the one row)
+template <bool ONE>
 __global__ void __launch_bounds__(UA_THREADS_MAX) uattn_kernel(DAttnArgs d, int bias_len) {
   extern __shared__ __align__(1024) float ua_smem[];
   const BAttnArgs& a = d.b;
@@ -46,6 +48,7 @@ __global__ void __launch_bounds__(UA_THREADS_MAX) uattn_kernel(DAttnArgs d, int 
   float* sBias = sS + MB * UA_CK;                      // [bias_len]
   float* sM = sBias + bias_len;                       // [ns][MB][pst] (used in the first block of the cluster)
   UAttnShared* sh = reinterpret_cast<UAttnShared*>(sM + (size_t)ns * MB * pst + ((ns * MB * pst) & 1));
+  float* sP1 = reinterpret_cast<float*>(sh + 1);     // [4 key quarters][64 channels], single-row passes
   if (tid == 0) {
     mg_mbar_init(smem_u32(&sh->kvbar[0]), 1);
     mg_mbar_init(smem_u32(&sh->kvbar[1]), 1);
@@ -103,6 +106,8 @@ __global__ void __launch_bounds__(UA_THREADS_MAX) uattn_kernel(DAttnArgs d, int 
   const int ngroups = (M + RG - 1) / RG;
   const int pv_i = tid >> dsh, pv_c = tid & (dkv - 1);   // thread <-> (row of the group, channel)
   float pv_acc[4] = {0.f, 0.f, 0.f, 0.f};               // one per group (MAXB / RG <= 4 when dkv <= 64)
+  // a single query row over 64-channel heads: the score and value phases are laid out so that all 256 threads work
+  const bool one_row = ONE && M == 1 && dkv == 64 && NT == UA_THREADS && row0 == 0;
   __syncthreads();
 #pragma unroll 1
   for (int c = 0; c < nchunks; ++c) {
@@ -118,6 +123,33 @@ __global__ void __launch_bounds__(UA_THREADS_MAX) uattn_kernel(DAttnArgs d, int 
         if (!ok) { sh->failed = 1; atomicExch(a.err, (int)BILD_ERR_TIMEOUT); }
       }
     }
+    if (one_row) {   // thread <-> (key, quarter of the channels); the quarters meet by shuffle
+      const int jj = tid >> 2, qt = tid & 3, j = jc + jj;
+      const int rot = ((qt >> 1) + 2 * (jj & 1)) & 3;   // rotated walk: the eight threads of a wavefront hit different banks
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int er = qt * 16 + (((e + rot) & 3) << 2);
+        const float4 kv = *reinterpret_cast<const float4*>(sK + jj * 64 + er);
+        const float4 qv = *reinterpret_cast<const float4*>(sQ + er);
+        s0 += kv.x * qv.x + kv.y * qv.y;
+        s1 += kv.z * qv.z + kv.w * qv.w;
+      }
+      float accs = s0 + s1;
+      accs += __shfl_xor_sync(0xffffffffu, accs, 1);
+      accs += __shfl_xor_sync(0xffffffffu, accs, 2);
+      if (qt == 0) {
+        float sc = -INFINITY;
+        if (jj < nk && (a.mode != 1 || j <= pos0)) {
+          if (a.mode != 0) {
+            const int dd = pos0 - j;
+            accs += bias_staged ? sBias[dd - dmin] : __ldg(a.bias + (size_t)h * a.bias_ld + dd);
+          }
+          sc = accs;
+        }
+        sS[jj] = sc;
+      }
+    } else
     // scores of all rows: one (row, key) pair per thread and turn
 #pragma unroll 1
     for (int idx = tid; idx < M * UA_CK; idx += NT) {
@@ -160,6 +192,18 @@ __global__ void __launch_bounds__(UA_THREADS_MAX) uattn_kernel(DAttnArgs d, int 
       }
     }
     __syncthreads();
+    if (one_row) {   // weighted values: thread <-> (quarter of the chunk's keys, channel); the quarters are added in order
+      const int kq = tid >> 6, jb = kq * 16;
+      float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+      for (int t = 0; t < 16; t += 2) {
+        if (jb + t < nk) a0 += sS[jb + t] * sV[(jb + t) * 64 + pv_c];
+        if (jb + t + 1 < nk) a1 += sS[jb + t + 1] * sV[(jb + t + 1) * 64 + pv_c];
+      }
+      sP1[tid] = a0 + a1;
+      __syncthreads();
+      if (tid < 64) pv_acc[0] = pv_acc[0] * sh->ascale[0] + (((sP1[tid] + sP1[64 + tid]) + sP1[128 + tid]) + sP1[192 + tid]);
+    } else
 #pragma unroll
     for (int gp = 0; gp < 4; ++gp) {   // weighted values: thread <-> (row gp * RG + pv_i, channel pv_c)
       const int i = gp * RG + pv_i;
