@@ -245,17 +245,24 @@ __global__ void __launch_bounds__(UA_THREADS_MAX) uattn_kernel(DAttnArgs d, int 
 #pragma unroll 1
   for (int idx = tid; idx < (M << dsh); idx += NT) {
     const int i = idx >> dsh, c = idx & (dkv - 1);
+    // at most 8 splits: the loads and exponentials of the splits are independent of each other, only the sums run in order
+    float pm[8], pl[8], pa[8];
+#pragma unroll
+    for (int s2 = 0; s2 < 8; ++s2) {
+      const float* Ps = sM + ((size_t)min(s2, ns - 1) * MB + i) * pst;
+      pm[s2] = s2 < ns ? Ps[0] : -INFINITY;
+      pl[s2] = s2 < ns ? Ps[1] : 0.f;
+      pa[s2] = Ps[2 + c];
+    }
     float gm = -INFINITY;
-#pragma unroll 1
-    for (int s2 = 0; s2 < ns; ++s2) gm = fmaxf(gm, sM[((size_t)s2 * MB + i) * pst]);
+#pragma unroll
+    for (int s2 = 0; s2 < 8; ++s2) gm = fmaxf(gm, pm[s2]);
     float num = 0.f, den = 0.f;
-#pragma unroll 1
-    for (int s2 = 0; s2 < ns; ++s2) {   // split order
-      const float* Ps = sM + ((size_t)s2 * MB + i) * pst;
-      const float l = Ps[1];
-      const float w = l > 0.f ? __expf(Ps[0] - gm) : 0.f;
-      den += l * w;
-      num += Ps[2 + c] * w;
+#pragma unroll
+    for (int s2 = 0; s2 < 8; ++s2) {   // split order
+      const float w = pl[s2] > 0.f ? __expf(pm[s2] - gm) : 0.f;
+      den += pl[s2] * w;
+      num += pa[s2] * w;
     }
     a.out[(size_t)(row0 + i) * a.ldo + h * dkv + c] = den > 0.f ? num / den : 0.f;
   }
