@@ -257,7 +257,7 @@ def main():
                      # dram__bytes_read+write of one block pass (k=5, cache 64) of the t5_sum pair: 191 of its 194
                      # launches (one of the 144 linear layers, 2 MB, and the LM head, 65.8 MB algorithmic, were
                      # outside the capture window); 814 MB algorithmic for the same launches
-                     "traffic": 828.5e6 if (dom_large and a.workload in ("t5_sum", "t5_long")) else None,
+                     "traffic": 831.2e6 if (dom_large and a.workload in ("t5_sum", "t5_long")) else None,
                      "note": "a pass is a chain of dependent kernels replayed as one CUDA graph; its duration is "
                              "measured with CUDA events over back-to-back replays"},
         "passes": {"small_step_us": t_small * 1e3, "small_step_GBs": b_small / t_small / 1e6,

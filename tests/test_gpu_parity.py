@@ -187,6 +187,51 @@ def test_steps_match_oracle_logits(torch_cuda, name):
         assert worst <= 2e-3, worst      # activations stay fp32: far inside the bf16 tolerance
 
 
+@pytest.mark.gpu
+def test_heads_of_64_channels_all_block_sizes(torch_cuda):
+    """Heads of 64 channels (the T5 / mT5 head size) at sizes the oracle runs live: single-row steps, blocks of 2 to 16
+    rows (both thread counts of the attention kernel, every epilogue turn of the row-slice linear), a self cache that
+    grows past one 64-key chunk, encoder keys split over a cluster of 4."""
+    torch = torch_cuda
+    from paper_2302_07863_b200.synthetic import make_context
+    name, scS, scL = "wide_bf16", 9.0, 11.0
+    wl = WORKLOADS[name]
+    ctx, ids, _ = make_context(name, scS, scL)
+    ctx.encode(ids)
+    S = Model(MODEL_SHAPES[wl.small], gen_model(MODEL_SHAPES[wl.small], wl.seed, wl.dtype), scS)
+    L = Model(MODEL_SHAPES[wl.large], gen_model(MODEL_SHAPES[wl.large], wl.seed, wl.dtype), scL)
+    V = S.s.vocab
+    cap = wl.gen_len + 1
+    stS, stL = S.start(ids, cap), L.start(ids, cap)
+    buf = torch.empty((16, V), dtype=torch.float32, device="cuda")
+    toks = [0] + [int(t) for t in gen_ids(V, 120, 5)]
+    worst = 0.0
+    for t in toks[:70]:   # the small model's cache passes 64 rows: second chunk of keys in the single-row kernel
+        z = S.forward_one(stS, t)
+        o = ctx.small_step(t, 0.4, buf)
+        worst = max(worst, float(np.max(np.abs(buf[0].cpu().numpy() - z))))
+        ta, pmax, lse, gap = obild.max_prob(z)
+        assert abs(o.lse - lse) <= 2e-3 and abs(o.pmax - pmax) <= 2e-2
+        if gap > 4e-3:
+            assert o.argmax == ta
+    pos = 0
+    for k in (1, 2, 3, 4, 5, 8, 9, 11, 16, 16, 13, 1):   # 89 rows in all: the large cache passes 64 rows as well
+        blk = toks[pos:pos + k]
+        Z = L.forward_block(stL, blk)
+        o = ctx.large_verify(blk, 15.0, buf)
+        worst = max(worst, float(np.max(np.abs(buf[:k].cpu().numpy() - Z))))
+        for i in range(k):
+            ta, _, lse, gap = obild.max_prob(Z[i])
+            assert abs(o.lse[i] - lse) <= 2e-3
+            if gap > 4e-3:
+                assert o.argmax[i] == ta
+            if i < k - 1:
+                assert abs(o.d[i] - (lse - Z[i][blk[i + 1]])) <= 4e-3
+        pos += k
+    assert worst <= 2e-3, worst   # activations stay fp32: far inside the 2e-2 of bf16 mode
+    ctx.close()
+
+
 # ---- whole loop against the stored oracle runs ------------------------------------------
 @pytest.mark.parametrize("name", ["tiny", "odd", "odd_bf16", "tiny_bf16"])
 def test_generate_matches_golden(torch_cuda, name):

@@ -49,6 +49,9 @@ MODEL_SHAPES = {
     # d_ff not a power of two, gated FFN.
     "odd_s": ModelShape("odd_s", 2, 64, 3, 16, 136, "gated_gelu", 773, False),
     "odd_l": ModelShape("odd_l", 3, 128, 6, 16, 328, "gated_gelu", 773, False),
+    # small pair with the 64-channel heads of the T5 / mT5 shapes (no stored run: live parity tests only)
+    "wide_s": ModelShape("wide_s", 2, 128, 2, 64, 264, "relu", 520, False),
+    "wide_l": ModelShape("wide_l", 3, 256, 4, 64, 520, "gated_gelu", 520, False),
     "t5_s": ModelShape("t5_s", 6, 512, 8, 64, 2048, "relu", 32128, False),
     "t5_l": ModelShape("t5_l", 24, 1024, 16, 64, 4096, "relu", 32128, False),
     "mt5_s": ModelShape("mt5_s", 8, 512, 6, 64, 1024, "gated_gelu", 250112, False),
@@ -73,6 +76,7 @@ WORKLOADS = {
     "odd": Workload("odd", "odd_s", "odd_l", "fp32", 19, 40),
     "odd_bf16": Workload("odd_bf16", "odd_s", "odd_l", "bf16", 19, 40),
     "tiny_bf16": Workload("tiny_bf16", "tiny_s", "tiny_l", "bf16", 32, 32),
+    "wide_bf16": Workload("wide_bf16", "wide_s", "wide_l", "bf16", 80, 100, max_draft=15),
     "t5_sum": Workload("t5_sum", "t5_s", "t5_l", "bf16", 512, 64),
     "mt5_mt": Workload("mt5_mt", "mt5_s", "mt5_l", "bf16", 64, 64),
     "t5_long": Workload("t5_long", "t5_s", "t5_l", "bf16", 1024, 256),
