@@ -246,7 +246,9 @@ int bild_op_linear(const void *W, int w_dtype, const float *X, const float *gain
 /* Fused LM head (Sections 3.3 and 3.4): for each of M rows, z = scale * W_lm rms(X),
  * and from z only: arg-max (lowest index), max, ln-sum-exp, and z[target[m]]
  * (target may be NULL).  The logits are not stored unless logits_dbg != NULL.
- * scratch: at least bild_op_lm_head_scratch_bytes(V) bytes, 256-byte aligned. */
+ * scratch: at least bild_op_lm_head_scratch_bytes(V) bytes, 256-byte aligned.
+ * K <= 4096; for M >= 2 also 16 rows of K floats must fit a block's shared memory (K up to
+ * about 3500), else BILD_ERR_CAPACITY. */
 size_t bild_op_lm_head_scratch_bytes(int V);
 int bild_op_lm_head(const void *W, int w_dtype, const float *X, const float *gain, float eps,
                     float scale, const int32_t *target, int M, int V, int K,
@@ -260,8 +262,12 @@ int bild_op_lm_head(const void *W, int w_dtype, const float *X, const float *gai
  * cudaMalloc / cudaFree, no allocating library routine.  Meant for a decode worker inside
  * a serving process whose allocator already owns the device's memory, or for a
  * latency-critical loop where cudaMalloc's device-wide synchronisation is not acceptable.
- *   - Limits: M <= 16, V <= 1048576, K <= 4096 (multiple of 8); beyond them the call
- *     returns BILD_ERR_CAPACITY (and says why on stderr) - use bild_op_lm_head then.
+ *   - Limits: M <= 16, V <= 1048576, K <= 4096 (multiple of 8), and for M >= 2 the kernel
+ *     stages 16 rows of K floats in shared memory, which a block can hold for K up to about
+ *     3500 on a B200 (the exact bound is taken from the device's attributes); beyond any of
+ *     them the call returns BILD_ERR_CAPACITY (and says why on stderr).  bild_op_lm_head
+ *     has no V limit of its own but the same shared-memory bound for M >= 2, with the same
+ *     error.
  *   - Every GPU that loads the library holds the 128 KiB until the process exits.
  *   - The first call on a device looks the array's device address up (a runtime call that
  *     is not a stream operation), so make that first call before any stream capture, with

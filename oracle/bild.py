@@ -62,6 +62,9 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
     stats   : counters,
     margins : smallest decision margins seen (top-1 vs top-2 logit of every
               arg-max that was used, |p_max - alpha_FB|, |d - alpha_RB|),
+    trace_margins : one (arg-max gap, |p_max - alpha_FB|, min |d_i - alpha_RB|) triple
+              per trace record: the margins of the decisions that produced that
+              record (inf where the record did not depend on such a decision),
     logits  : (if keep_logits) list of ("S"|"L", first position, array).
     """
     assert mode in ("bild", "small", "large")
@@ -72,7 +75,7 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
     n = 0                       # index of the last token in y
     L_len = 0                   # tokens the large model has consumed
     drafts = 0
-    trace, logits = [], []
+    trace, logits, tmg = [], [], []
     stats = dict(small_steps=0, large_calls=0, fallbacks=0, forced=0, rollbacks=0,
                  discarded=0, sum_k=0)
     mg = dict(argmax=math.inf, fallback=math.inf, rollback=math.inf)
@@ -88,6 +91,7 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
                 mg["argmax"] = min(mg["argmax"], gap)
                 y.append(t); n += 1
                 trace.append((KIND_SMALL_ACCEPT, n, t, 0, -1, pmax))
+                tmg.append((gap, math.inf, math.inf))
                 continue
             mg["fallback"] = min(mg["fallback"], abs(pmax - alpha_fb))
             confident = not (pmax < alpha_fb)                       # Section 3.3
@@ -95,6 +99,7 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
                 mg["argmax"] = min(mg["argmax"], gap)
                 y.append(t); n += 1; drafts += 1
                 trace.append((KIND_SMALL_ACCEPT, n, t, 0, -1, pmax))
+                tmg.append((gap, abs(pmax - alpha_fb), math.inf))
                 continue
             if confident:
                 stats["forced"] += 1
@@ -102,6 +107,7 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
             else:
                 stats["fallbacks"] += 1
                 trace.append((KIND_FALLBACK, n + 1, t, 0, -1, pmax))
+            tmg.append((gap, abs(pmax - alpha_fb), math.inf))   # the record names the rejected candidate
         # ---- the large model reads every token it has not seen yet ----------
         k = n - L_len + 1
         ZL = large.forward_block(stL, y[L_len:n + 1])              # Alg. 1: p_L <- LargeModel(y)
@@ -110,10 +116,11 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
         if keep_logits:
             logits.append(("L", L_len, ZL.copy()))
         rows = [max_prob(ZL[i]) for i in range(k)]
-        m_star, d_star, d_max = -1, 0.0, 0.0
+        m_star, d_star, d_max, rb_here = -1, 0.0, 0.0, math.inf
         for i in range(k - 1):                                      # pending drafts only
             d_i = rows[i][2] - float(ZL[i][y[L_len + i + 1]])       # -ln p_L(y_S)
             mg["rollback"] = min(mg["rollback"], abs(d_i - alpha_rb))
+            rb_here = min(rb_here, abs(d_i - alpha_rb))
             d_max = max(d_max, d_i)
             if d_i > alpha_rb:                                      # Eq. 3, first violation
                 m_star, d_star = i, d_i
@@ -129,10 +136,12 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
             stS.rewind(j)
             L_len = j
             trace.append((KIND_ROLLBACK, j, y[j], k, m_star, d_star))
+            tmg.append((rows[m_star][3], math.inf, rb_here))
         else:
             mg["argmax"] = min(mg["argmax"], rows[k - 1][3])
             y.append(rows[k - 1][0]); n += 1
             L_len = n
             trace.append((KIND_VERIFY_OK, n, y[n], k, -1, d_max))
+            tmg.append((rows[k - 1][3], math.inf, rb_here))
         drafts = 0
-    return dict(tokens=y[1:], trace=trace, stats=stats, margins=mg, logits=logits)
+    return dict(tokens=y[1:], trace=trace, stats=stats, margins=mg, logits=logits, trace_margins=tmg)

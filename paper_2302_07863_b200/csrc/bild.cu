@@ -10,13 +10,13 @@
 #include <vector>
 
 #include "decode_kernels.cuh"
-#include "mega_pass.cuh"
 #include "slice_linear.cuh"
 #include "unit_attention.cuh"
 #include "slice_head.cuh"
 #include "umma_linear.cuh"
 #include "enc_gemm.cuh"
 #include "enc_attention.cuh"
+#include "sublayer.cuh"
 
 using namespace bild;
 
@@ -113,15 +113,13 @@ struct Model {
   CUtensorMap tmH[2][3][2];   // [buffer pair][row length d / inner / d_ff][head, remainder]
   bool enc_gemm = false;
   int index = 0;   // 0 small, 1 large
-  // whole-pass persistent kernel (bf16 only)
-  MegaLayer* mega_layers = nullptr;
-  unsigned* mega_sync = nullptr;
-  uint2* mega_ll = nullptr;          // all (value, epoch) areas, contiguous
-  size_t mega_ll_pairs = 0;
-  int64_t mega_launch_bound = 0;     // launches since the areas and the epoch base were last cleared
-  bool mega = false;
-  MegaArgs mega_args{};
-  int mega_grid = 0;
+  // fused sub-layer kernels (bf16 only): two more residual-stream buffers, W_fo transposed per layer
+  float *xb = nullptr, *xc = nullptr;
+  __nv_bfloat16* wfoT = nullptr;     // [layers][F][d]
+  bool fused = false;
+  int sub_C = 1;                     // blocks per head (cluster size) of the attention sub-layers
+  int sub_kc = 16, sub_bias_len = 32;
+  int sub_parts = 1;                 // launches the feed-forward sub-layer is split into
 };
 
 }  // namespace
@@ -173,7 +171,8 @@ struct bild_ctx {
   size_t slice_head_min_bytes = (size_t)32 << 20;
   int slice_mma_min = 3;
   size_t slice_min_bytes = 3000 * 1024;   // single-row passes: smaller matrices stay on the GEMV (measured)
-  bool mega_coop = true;             // launch the whole-pass kernel with the cooperative attribute
+  int fused_on = 1;                  // fused sub-layer kernels where the shapes allow: 0 off, 1 single-row passes, 2 block passes too
+  int sub_parts_want = 0;            // 0: fewest launches of the feed-forward sub-layer that fit
   bool capturing = false;            // launches are being recorded into a graph, not run
   int64_t graph_counted = 0;         // launches of the loop graphs already added to `launches`
 };
@@ -222,7 +221,7 @@ int head_grid_for(int V) { return std::max(1, std::min(HEAD_GRID_MAX, (V + 63) /
 // partial records either head kernel may write (block head: grid x MAXB; single-row head: up to V / 8 blocks)
 size_t head_partial_count(int V) {
   // block head: grid x MAXB; single-row head: up to V / 8 blocks; one-block-per-SM head: SMs x MAXB
-  return std::max(std::max((size_t)head_grid_for(V) * MAXB, (size_t)(V + 7) / 8 + 8), (size_t)MG_MAX_BLOCKS * MAXB);
+  return std::max(std::max((size_t)head_grid_for(V) * MAXB, (size_t)(V + 7) / 8 + 8), (size_t)MAX_GRID_SM * MAXB);
 }
 
 // Lays out everything the context keeps on the device.
@@ -260,10 +259,9 @@ void plan(bild_ctx* c, Bump& b) {
     m.head_cnt = b.take<unsigned>(1);
     m.head_out = b.take<HeadOut>(1);
     m.desc = b.take<CallDesc>(1);
-    m.mega_layers = b.take<MegaLayer>(mc.n_layers);
-    m.mega_sync = b.take<unsigned>(4);
-    m.mega_ll_pairs = (size_t)MAXB * (6 * m.inner + 3 * mc.d_model + mc.d_ff) + 2 * mega_record_pairs(MG_MAX_BLOCKS, mc.d_kv);
-    m.mega_ll = b.take<uint2>(m.mega_ll_pairs);
+    m.xb = b.take<float>((size_t)MAXB * mc.d_model);
+    m.xc = b.take<float>((size_t)MAXB * mc.d_model);
+    m.wfoT = b.take<__nv_bfloat16>(cfg.dtype == BILD_BF16 ? (size_t)mc.n_layers * mc.d_ff * mc.d_model : 0);
   }
   const size_t ecap16 = (size_t)(ecap + MAXB - 1) / MAXB * MAXB;   // whole blocks of MAXB rows
   const size_t ecap128 = (size_t)(ecap + EG_TOK - 1) / EG_TOK * EG_TOK;   // whole tiles of 128 tokens
@@ -462,7 +460,14 @@ cudaError_t launch_head_t(bild_ctx* c, const HeadArgs& a, int grid, int64_t* lau
   const size_t smem = (size_t)MB * a.K * sizeof(float);
   auto kern = lm_head_kernel<WT, MB, RW>;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaFuncAttributes fa;
+    int dev = 0, optin = 0;
+    cudaError_t e = cudaFuncGetAttributes(&fa, kern);
+    if (e == cudaSuccess) e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return e;
+    if (smem + fa.sharedSizeBytes > (size_t)optin) return cudaErrorInvalidConfiguration;   // the staged rows do not fit a block
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   if (launches) (*launches)++;
@@ -490,9 +495,10 @@ cudaError_t launch_head1(bild_ctx* c, const HeadArgs& a, int64_t* launches) {
   return launch_head1_t<WT, 8, 1>(c, a, launches);
 }
 
-cudaError_t launch_head(cudaStream_t s, int dtype, int MB, const HeadArgs& a, int grid, int64_t* launches) {
+cudaError_t launch_head(cudaStream_t s, bool pdl, int dtype, int MB, const HeadArgs& a, int grid, int64_t* launches) {
   bild_ctx tmp;
   tmp.stream = s;
+  tmp.use_pdl = pdl;
   if (MB == 1 && head1_grid(a.V, a.K) > 0)
     return dtype == BILD_BF16 ? launch_head1<__nv_bfloat16>(&tmp, a, launches) : launch_head1<float>(&tmp, a, launches);
   if (dtype == BILD_BF16)
@@ -509,12 +515,12 @@ int pick_nsplit(int heads, int keys_cap) {
 }
 
 cudaError_t launch_embed(bild_ctx* c, const void* E, const int* tokens, const int* cnt_dev, int cnt_host, int rows,
-                         int d, int vocab, float* x) {
+                         int d, int vocab, float* x, float* x_zero = nullptr) {
   if (c->cfg.dtype == BILD_BF16)
     return launch_k(c, embed_kernel<__nv_bfloat16>, dim3(rows), dim3(128), 0, (const __nv_bfloat16*)E, tokens, cnt_dev,
-                    cnt_host, d, vocab, x);
+                    cnt_host, d, vocab, x, x_zero);
   return launch_k(c, embed_kernel<float>, dim3(rows), dim3(128), 0, (const float*)E, tokens, cnt_dev, cnt_host, d,
-                  vocab, x);
+                  vocab, x, x_zero);
 }
 
 // ---- tensor-core path of the block pass ---------------------------------------------------
@@ -597,102 +603,120 @@ void setup_umma(bild_ctx* c, Model& m) {
   m.enc_gemm = true;
 }
 
-// Decides whether the decoder passes of model `m` run as the persistent whole-pass kernel and
-// prepares its arguments (the per-layer pointer table lives in the workspace).
-int setup_mega(bild_ctx* c, Model& m) {
-  m.mega = false;
-  // Opt-in: on B200 the stage-to-stage exchange through L2 (about 2 us per hop) makes the persistent
-  // pass slower than the chain of kernels, whose boundaries cost less.
-  const char* on = std::getenv("BILD_MEGA");
-  if (!(on && on[0] == '1')) return BILD_OK;
-  if (c->cfg.dtype != BILD_BF16) return BILD_OK;
+// ---- fused sub-layer kernels ------------------------------------------------------------------
+// Decides whether the decoder passes of model `m` run on the fused sub-layer kernels, transposes the
+// FFN output matrices into the workspace and fixes the launch shapes.
+int setup_fused(bild_ctx* c, Model& m) {
+  m.fused = false;
+  if (!c->fused_on || c->cfg.dtype != BILD_BF16 || c->sms < 1) return BILD_OK;
   const bild_model_cfg& mc = m.c;
-  const int d = mc.d_model, I = m.inner, F = mc.d_ff;
+  const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
+  const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len;
   const bool gated = mc.ffn_kind == BILD_FFN_GATED_GELU;
-  if (d % 8 || I % 8 || F % 8 || d * 2 > MG_SLOT || I * 2 > MG_SLOT || F * 2 > MG_SLOT) return BILD_OK;
-  int dev = 0, sms = 0, smem_max = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
-    cudaGetLastError();
-    return BILD_OK;
-  }
-  const int nslots = std::min(MG_MAX_SLOTS, (smem_max - MG_ACT - MG_PSUM - MG_MISC) / MG_SLOT);
-  if (nslots < 4 || sms < 1 || sms > MG_MAX_BLOCKS) return BILD_OK;
-  if (mc.n_heads * 4 > sms || (d + sms - 1) / sms > MG_XRES || 8 * mc.n_layers + 2 > MG_EPOCHS_PER_LAUNCH) return BILD_OK;
-  // every stage's slice must fit the ring with room to fetch ahead, and its rows the partial-sum area
-  const int Ns[6] = {3 * I, d, I, d, F, d}, Ks[6] = {d, I, d, I, d, F};
-  for (int p = 0; p < 6; ++p) {
-    const int rows = (Ns[p] + sms - 1) / sms, nmat = (p == 4 && gated) ? 2 : 1;
-    const int rps = MG_SLOT / (Ks[p] * 2);
-    const int slots = (rows + rps - 1) / rps * nmat;
-    if (slots > nslots - 2 || rows * nmat > 4 * MG_QUADS || mc.n_layers > MG_MAX_LAYERS) return BILD_OK;
-  }
+  int C = 8;
+  while (C > 1 && (H * C > c->sms || d % (4 * C))) C >>= 1;
+  if (d % (4 * C) || d > 1024 || dkv > 64 || dkv < 16 || d / C > SUB_THREADS / 2) return BILD_OK;
+  if ((3 * dkv + C - 1) / C > SUB_MAX_ROWS) return BILD_OK;
   auto aligned = [](const void* p) { return ((uintptr_t)p & 15) == 0; };
-  std::vector<MegaLayer> tab(mc.n_layers);
   for (int l = 0; l < mc.n_layers; ++l) {
     const bild_dec_layer& w = m.dec[l];
     if (!aligned(w.wqkv) || !aligned(w.wo) || !aligned(w.wcq) || !aligned(w.wco) || !aligned(w.wi0) || !aligned(w.wfo) ||
         (gated && !aligned(w.wi1)) || !aligned(w.ln1) || !aligned(w.ln2) || !aligned(w.ln3)) return BILD_OK;
-    MegaLayer& t = tab[l];
-    t.wqkv = (const __nv_bfloat16*)w.wqkv; t.wo = (const __nv_bfloat16*)w.wo; t.wcq = (const __nv_bfloat16*)w.wcq;
-    t.wco = (const __nv_bfloat16*)w.wco; t.wi0 = (const __nv_bfloat16*)w.wi0; t.wi1 = (const __nv_bfloat16*)w.wi1;
-    t.wfo = (const __nv_bfloat16*)w.wfo;
-    t.ln1 = (const float*)w.ln1; t.ln2 = (const float*)w.ln2; t.ln3 = (const float*)w.ln3;
   }
-  if (!aligned(m.w.emb)) return BILD_OK;
-  if (cudaFuncSetAttribute(mega_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mega_smem_bytes(nslots)) != cudaSuccess) {
+  int smem_max = 0, dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
     cudaGetLastError();
     return BILD_OK;
   }
-  CUDA_TRY(c, cudaMemcpyAsync(m.mega_layers, tab.data(), tab.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice, c->stream));
-  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-  MegaArgs& a = m.mega_args;
-  a.layers = m.mega_layers; a.n_layers = mc.n_layers;
-  a.d = d; a.I = I; a.F = F; a.H = mc.n_heads; a.dkv = mc.d_kv; a.dkv_shift = ilog2(mc.d_kv); a.gated = gated ? 1 : 0;
-  a.vocab = mc.vocab; a.eps = mc.ln_eps; a.desc = m.desc; a.emb = (const __nv_bfloat16*)m.w.emb;
-  a.x = m.x;
-  {
-    uint2* p = m.mega_ll;
-    auto take = [&](size_t n) { uint2* r = p; p += n; return r; };
-    const size_t rec = mega_record_pairs(MG_MAX_BLOCKS, mc.d_kv);
-    a.ll.qkv1 = take((size_t)MAXB * 3 * I); a.ll.a2 = take((size_t)MAXB * I); a.ll.r2 = take(rec);
-    a.ll.x3 = take((size_t)MAXB * d); a.ll.q4 = take((size_t)MAXB * I); a.ll.a5 = take((size_t)MAXB * I); a.ll.r5 = take(rec);
-    a.ll.x6 = take((size_t)MAXB * d); a.ll.u7 = take((size_t)MAXB * F); a.ll.x8 = take((size_t)MAXB * d);
+  const int per_rank = (std::max(cap, ecap) + C - 1) / C;
+  int kc = std::min(64, (per_rank + 15) / 16 * 16);   // at most 64: a chunk's scores take one turn of the block
+  const int bias_len = ((cap + C - 1) / C + MAXB + 8 + 3) / 4 * 4;
+  while (kc > 16 && attn_sub_layout(d, dkv, 3, C, MAXB, kc, bias_len).total > smem_max) kc -= 16;
+  if (attn_sub_layout(d, dkv, 3, C, MAXB, kc, bias_len).total > smem_max) return BILD_OK;
+  int parts = std::max(1, c->sub_parts_want);
+  const int nmat = gated ? 2 : 1;
+  while (parts <= 8 && (ffn_sub_rows(F, c->sms * parts) * nmat > SUB_MAX_ROWS || ffn_sub_rows(F, c->sms * parts) > SUB_FO_REGS ||
+                        ffn_sub_layout(d, F, gated, c->sms * parts, c->sms, MAXB).total > smem_max)) ++parts;
+  if (parts > 8) return BILD_OK;
+  if (cudaFuncSetAttribute(attn_sub_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess ||
+      cudaFuncSetAttribute(attn_sub_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess ||
+      cudaFuncSetAttribute(ffn_sub_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess ||
+      cudaFuncSetAttribute(ffn_sub_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess) {
+    cudaGetLastError();
+    return BILD_OK;
   }
-  a.selfK = m.selfK; a.selfV = m.selfV; a.crossK = m.crossK; a.crossV = m.crossV;
-  a.cap = c->cfg.max_dec_len; a.ecap = c->cfg.max_enc_len; a.dec_bias = m.dec_bias; a.enc_len = c->enc_len_dev;
-  a.sync = m.mega_sync; a.err = &c->st->err; a.nslots = nslots;
-  m.mega_grid = sms;
-  m.mega = true;
+  for (int l = 0; l < mc.n_layers; ++l) {
+    transpose_bf16_kernel<<<dim3((F + 31) / 32, (d + 31) / 32), dim3(32, 8), 0, c->stream>>>(
+        (const __nv_bfloat16*)m.dec[l].wfo, m.wfoT + (size_t)l * F * d, d, F);
+    (*c->cnt)++;
+  }
+  CUDA_TRY(c, cudaGetLastError());
+  m.sub_C = C; m.sub_kc = kc; m.sub_bias_len = bias_len; m.sub_parts = parts;
+  m.fused = true;
   return BILD_OK;
 }
 
-// The epochs are 32-bit and grow by MG_EPOCHS_PER_LAUNCH per launch: long before they could wrap,
-// the areas and the launch counter are cleared (stream-ordered, between passes).
-cudaError_t mega_epoch_budget(bild_ctx* c, Model& m, int64_t launches) {
-  if (!m.mega) return cudaSuccess;
-  m.mega_launch_bound += launches;
-  if (m.mega_launch_bound < (int64_t)2000000) return cudaSuccess;
-  m.mega_launch_bound = launches;
-  cudaError_t e = cudaMemsetAsync(m.mega_ll, 0, m.mega_ll_pairs * sizeof(uint2), c->stream);
-  if (e != cudaSuccess) return e;
-  return cudaMemsetAsync(m.mega_sync, 0, 4 * sizeof(unsigned), c->stream);
+template <typename Arg>
+cudaError_t launch_sub(bild_ctx* c, void (*kern)(Arg), int grid, int cluster, size_t smem, const Arg& a) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(SUB_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (c->use_pdl) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (cluster > 1) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = cluster; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = at; cfg.numAttrs = na;
+  (*c->cnt)++;
+  return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
-cudaError_t launch_mega(bild_ctx* c, Model& m) {
-  if (!c->capturing) {
-    cudaError_t e = mega_epoch_budget(c, m, 1);
-    if (e != cudaSuccess) return e;
+// The layers of a decoder pass on the fused sub-layer kernels: the residual stream goes x -> xb -> xc -> x
+// per layer (self-attention, cross-attention, feed-forward), each kernel clearing the buffer after its output.
+int fused_layers(bild_ctx* c, Model& m, int MB) {
+  const bild_model_cfg& mc = m.c;
+  const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
+  const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len;
+  const bool gated = mc.ffn_kind == BILD_FFN_GATED_GELU;
+  const int C = m.sub_C;
+  for (int l = 0; l < mc.n_layers; ++l) {
+    const bild_dec_layer& w = m.dec[l];
+    const size_t kvoff = (size_t)l * H * dkv;
+    AttnSubArgs a{};
+    a.desc = m.desc; a.eps = mc.ln_eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
+    a.kc_keys = m.sub_kc; a.bias_len = m.sub_bias_len; a.mb = MB; a.err = &c->st->err;
+    a.n_keys_dev = c->enc_len_dev;
+    // S1-S3 / L1-L3
+    a.x_in = m.x; a.x_out = m.xb; a.x_zero = m.xc; a.gain = (const float*)w.ln1;
+    a.Wp = (const __nv_bfloat16*)w.wqkv; a.Wo = (const __nv_bfloat16*)w.wo;
+    a.kc = m.selfK + kvoff * cap; a.vc = m.selfV + kvoff * cap; a.cap = cap; a.bias = m.dec_bias; a.bias_ld = cap; a.self = 1;
+    a.L = attn_sub_layout(d, dkv, 3, C, MB, a.kc_keys, a.bias_len);
+    CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
+    // S4-S6 / L4-L6
+    a.x_in = m.xb; a.x_out = m.xc; a.x_zero = m.x; a.gain = (const float*)w.ln2;
+    a.Wp = (const __nv_bfloat16*)w.wcq; a.Wo = (const __nv_bfloat16*)w.wco;
+    a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.bias = nullptr; a.bias_ld = 0; a.self = 0;
+    a.L = attn_sub_layout(d, dkv, 1, C, MB, a.kc_keys, a.bias_len);
+    CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
+    // S7-S8 / L7-L8
+    FfnSubArgs f{};
+    f.desc = m.desc; f.eps = mc.ln_eps; f.d = d; f.F = F; f.gated = gated ? 1 : 0; f.mb = MB;
+    f.err = &c->st->err; f.x_in = m.xc; f.x_out = m.x; f.gain = (const float*)w.ln3;
+    f.Wi0 = (const __nv_bfloat16*)w.wi0; f.Wi1 = (const __nv_bfloat16*)w.wi1; f.WfoT = m.wfoT + (size_t)l * F * d;
+    f.nparts = m.sub_parts;
+    f.L = ffn_sub_layout(d, F, gated, c->sms * m.sub_parts, c->sms, MB);
+    for (int p = 0; p < m.sub_parts; ++p) {
+      f.part = p; f.seed = p == 0 ? 1 : 0; f.x_zero = p == 0 ? m.xb : nullptr;
+      CUDA_TRY(c, launch_sub(c, MB == 1 ? ffn_sub_kernel<true> : ffn_sub_kernel<false>, c->sms, 1, (size_t)f.L.total, f));
+    }
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(m.mega_grid); cfg.blockDim = dim3(MG_THREADS);
-  cfg.dynamicSmemBytes = mega_smem_bytes(m.mega_args.nslots); cfg.stream = c->stream;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeCooperative;   // all blocks resident at once: they wait for one another
-  at[0].val.cooperative = 1;
-  cfg.attrs = at; cfg.numAttrs = c->mega_coop ? 1 : 0;
-  (*c->cnt)++;
-  return cudaLaunchKernelEx(&cfg, mega_pass_kernel, m.mega_args);
+  return BILD_OK;
 }
 
 // Split of K over a cluster: enough blocks to pull the matrix at full bandwidth, at most 16 k blocks each.
@@ -859,15 +883,18 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   const bild_model_cfg& mc = m.c;
   const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
   const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len, dt = c->cfg.dtype;
-  if (m.mega) CUDA_TRY(c, launch_mega(c, m));
-  else
-  CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x));
+  const bool fused = m.fused && (MB == 1 || c->fused_on >= 2);
+  CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x, fused ? m.xb : nullptr));
+  if (fused) {
+    int rc = fused_layers(c, m, MB);
+    if (rc) return rc;
+  }
   // self-attention: one block per head up to 128 cached rows (no merge step); cross-attention:
   // enough splits of the encoder keys to occupy the SMs
   int ns_self = 1;
   while (ns_self < 8 && (cap + ns_self - 1) / ns_self > 256) ns_self *= 2;
   const int ns_cross = pick_nsplit(H, ecap);
-  for (int l = 0; l < (m.mega ? 0 : mc.n_layers); ++l) {
+  for (int l = 0; l < (fused ? 0 : mc.n_layers); ++l) {
     const bild_dec_layer& w = m.dec[l];
     const size_t kvoff = (size_t)l * H * dkv;
     LinArgs a{};
@@ -923,7 +950,7 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   const size_t sh_smem = slice_head_smem_bytes(d, head_tr);
   // single-row passes: only heads of 32 MB and more (smaller ones stay on the GEMV head)
   const bool big_head = (size_t)mc.vocab * d * 2 >= c->slice_head_min_bytes;
-  if (c->slice_head >= (MB == 1 ? 2 : 1) && (MB != 1 || big_head) && dt == BILD_BF16 && c->sms > 0 && c->sms <= MG_MAX_BLOCKS && sh_smem <= 200 * 1024 &&
+  if (c->slice_head >= (MB == 1 ? 2 : 1) && (MB != 1 || big_head) && dt == BILD_BF16 && c->sms > 0 && c->sms <= MAX_GRID_SM && sh_smem <= 200 * 1024 &&
       d % 8 == 0 && ((uintptr_t)m.w.lm_head & 15) == 0) {
     // tensor-core head, one block per SM
     if (!c->slice_head_smem_set) {
@@ -934,7 +961,7 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
                          &c->st->err, head_tr));
     return BILD_OK;
   }
-  CUDA_TRY(c, launch_head(c->stream, dt, MB, h, m.head_grid, c->cnt));
+  CUDA_TRY(c, launch_head(c->stream, c->use_pdl, dt, MB, h, m.head_grid, c->cnt));
   return BILD_OK;
 }
 
@@ -1068,19 +1095,16 @@ void drop_graphs(bild_ctx* c) {
 
 int build_graphs(bild_ctx* c) {
   if (c->exec[0] && c->exec[1]) return BILD_OK;
-  // what a loop body refuses (programmatic edges, cooperative kernel nodes) is dropped step by step
-  const bool want_pdl = c->use_pdl, want_coop = c->mega_coop;
-  const bool tries[3][2] = {{want_pdl, want_coop}, {want_pdl, false}, {false, false}};
-  int rc = BILD_ERR_CUDA;
-  for (int t = 0; t < 3; ++t) {
-    if (t > 0 && tries[t][0] == tries[t - 1][0] && tries[t][1] == tries[t - 1][1]) continue;
-    c->use_pdl = tries[t][0];
-    c->mega_coop = tries[t][1];
-    rc = build_graphs_once(c);
-    if (rc == BILD_OK) return rc;
+  // if a loop body refuses programmatic edges, the graphs are built again with plain launches
+  const bool want_pdl = c->use_pdl;
+  int rc = build_graphs_once(c);
+  if (rc != BILD_OK && want_pdl) {
     drop_graphs(c);
     cudaGetLastError();
+    c->use_pdl = false;
+    rc = build_graphs_once(c);
   }
+  if (rc != BILD_OK) { drop_graphs(c); cudaGetLastError(); }
   return rc;
 }
 
@@ -1206,6 +1230,10 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   if (es && es[0] == '1') c->enc_parallel = false;
   const char* sm = std::getenv("BILD_SLICE_MIN_KB");
   if (sm) c->slice_min_bytes = (size_t)std::atoi(sm) * 1024;
+  const char* fu = std::getenv("BILD_FUSED");
+  if (fu && fu[0] >= '0' && fu[0] <= '2') c->fused_on = fu[0] - '0';
+  const char* fp = std::getenv("BILD_FFN_PARTS");
+  if (fp) c->sub_parts_want = std::min(8, std::max(0, std::atoi(fp)));
   const char* np = std::getenv("BILD_NO_PDL");
   c->use_pdl = !(np && np[0] == '1');
   Bump b(workspace);
@@ -1243,7 +1271,7 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   // zero the ticket counters and the state, build the bias-by-distance tables
   if (cudaMemsetAsync(workspace, 0, c->ws_bytes, c->stream) != cudaSuccess) { bild_destroy(c); return BILD_ERR_CUDA; }
   for (int i = 0; i < 2; ++i) {
-    rc = setup_mega(c, c->m[i]);
+    rc = setup_fused(c, c->m[i]);
     if (rc) { bild_destroy(c); return rc; }
   }
   rc = build_bias_tables(c);
@@ -1399,9 +1427,6 @@ int bild_generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, i
     if (rc) return rc;
     if (max_len == 0 || c->cfg.start_id == c->cfg.eos_id) return BILD_OK;
     // passes the loop may run: bounded by the guard of the device-side policy
-    const int64_t bound = (int64_t)(max_len + 2) * (c->cfg.max_draft + 3) + 16;
-    CUDA_TRY(c, mega_epoch_budget(c, c->m[0], bound));
-    CUDA_TRY(c, mega_epoch_budget(c, c->m[1], bound));
     CUDA_TRY(c, cudaGraphLaunch(c->exec[mode == BILD_MODE_LARGE_ONLY ? 1 : 0], c->stream));
     return BILD_OK;
   }
@@ -1489,7 +1514,11 @@ int bild_op_lm_head(const void* W, int w_dtype, const float* X, const float* gai
   if (cudaMemsetAsync(h.counter, 0, sizeof(unsigned), s) != cudaSuccess) return BILD_ERR_CUDA;
   h.W = W; h.X = X; h.ldx = K; h.gain = gain; h.eps = eps; h.scale = scale; h.V = V; h.K = K; h.M = M;
   h.target = target; h.logits_dbg = logits_dbg; h.which = 1;
-  if (launch_head(s, w_dtype, M == 1 ? 1 : MAXB, h, grid, nullptr) != cudaSuccess) return BILD_ERR_CUDA;
+  {
+    const cudaError_t le = launch_head(s, false, w_dtype, M == 1 ? 1 : MAXB, h, grid, nullptr);
+    if (le == cudaErrorInvalidConfiguration) return BILD_ERR_CAPACITY;   // M >= 2: 16 rows of K floats exceed a block's shared memory
+    if (le != cudaSuccess) return BILD_ERR_CUDA;
+  }
   const HeadOut* o = h.out;
   cudaError_t e = cudaMemcpyAsync(argmax_out, o->argmax, M * sizeof(int), cudaMemcpyDeviceToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(max_out, o->zmax, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
@@ -1521,7 +1550,6 @@ int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, floa
   int64_t n_launch = 0;
   if (rc == BILD_OK) rc = capture_pass(c, g, which, k == 1 ? 1 : MAXB, 0, 0, nullptr, &n_launch);
   if (rc == BILD_OK && cudaGraphInstantiate(&ex, g, 0) != cudaSuccess) rc = BILD_ERR_CUDA;
-  if (rc == BILD_OK && mega_epoch_budget(c, c->m[which], iters + 1) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && cudaGraphUpload(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && !cold && cudaGraphLaunch(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;  // untimed first pass
   if (rc == BILD_OK && cudaEventRecord(e0, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
@@ -1540,6 +1568,18 @@ int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, floa
   *ms_per_pass = ms / (float)iters;
   return BILD_OK;
 }
+
+#ifdef BILD_STAMPS
+// Cycle stamps of the fused sub-layer kernels (debug builds only): 4 x 16 counters, optionally cleared.
+int bild_debug_stamps(unsigned long long* out, int reset) {
+  if (out && cudaMemcpyFromSymbol(out, g_sub_stamps, sizeof(g_sub_stamps)) != cudaSuccess) return BILD_ERR_CUDA;
+  if (reset) {
+    static unsigned long long zero[4][24];
+    if (cudaMemcpyToSymbol(g_sub_stamps, zero, sizeof(zero)) != cudaSuccess) return BILD_ERR_CUDA;
+  }
+  return BILD_OK;
+}
+#endif
 
 // Host-only helper for tests of the bucket tables: which = 0 decoder (delta = query - key >= 0),
 // 1 encoder (rel = key - query).

@@ -128,6 +128,54 @@ __device__ __forceinline__ void st_cluster_f1(uint32_t local_addr, uint32_t rank
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
 }
 
+// ---- mbarrier, bulk (TMA) copies, bounded polling ------------------------------------------
+constexpr unsigned SPIN_LIMIT = 1u << 20;   // polls of a barrier before a kernel gives up and reports BILD_ERR_TIMEOUT
+constexpr int MAX_GRID_SM = 256;            // per-block record areas are sized for this many blocks (one per SM)
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// global -> shared bulk copy (16-byte aligned addresses, size a multiple of 16) that reports to an mbarrier
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// barrier of the first 256 threads of a block (the computing warps of kernels with a copy-issuing extra warp)
+__device__ __forceinline__ void csync256() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// ---- sum of NP register values across the warp, one shuffle per halving ------------------
+// Returns in every lane the warp-wide sum of v[lane >> (5 - log2 NP)].
+template <int NP>
+__device__ __forceinline__ float treduce(float (&v)[NP], int lane) {
+  int s = 16;
+#pragma unroll
+  for (int n = NP; n > 1; n >>= 1) {
+    const bool up = (lane & s) != 0;
+#pragma unroll
+    for (int j = 0; j < n / 2; ++j) {
+      const float send = up ? v[j] : v[j + n / 2];
+      const float keep = up ? v[j + n / 2] : v[j];
+      v[j] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+    }
+    s >>= 1;
+  }
+  float r = v[0];
+  for (; s >= 1; s >>= 1) r += __shfl_xor_sync(0xffffffffu, r, s);
+  return r;
+}
+
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 

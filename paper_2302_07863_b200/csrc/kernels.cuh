@@ -12,7 +12,7 @@ namespace bild {
 template <typename WT>
 __global__ void embed_kernel(const WT* __restrict__ E, const int* __restrict__ tokens,
                              const int* __restrict__ count_dev, int count_host, int d,
-                             int vocab, float* __restrict__ x) {
+                             int vocab, float* __restrict__ x, float* __restrict__ x_zero) {
   const int m = blockIdx.x;
   pdl_launch_dependents();
   pdl_wait();
@@ -22,6 +22,8 @@ __global__ void embed_kernel(const WT* __restrict__ E, const int* __restrict__ t
   t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
   const WT* row = E + (size_t)t * d;
   for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)m * d + c] = to_float(row[c]);
+  // the buffer the first fused sub-layer accumulates into starts at zero
+  if (x_zero) for (int c = threadIdx.x; c < d; c += blockDim.x) x_zero[(size_t)m * d + c] = 0.f;
 }
 
 // ---------------------------------------------------------------------------------

@@ -57,12 +57,20 @@ int scratch_for_current_device(void** out) {
   return BILD_OK;
 }
 
+// *too_big: the MB staged rows of K floats plus the kernel's own shared memory exceed what a block may have
 template <typename WT, int MB, int RW>
-cudaError_t launch_t(const HeadArgs& a, int grid, cudaStream_t s) {
+cudaError_t launch_t(const HeadArgs& a, int grid, cudaStream_t s, bool* too_big) {
   const size_t smem = (size_t)MB * a.K * sizeof(float);
   auto kern = lm_head_kernel<WT, MB, RW>;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaFuncAttributes fa;
+    int dev = 0, optin = 0;
+    cudaError_t e = cudaFuncGetAttributes(&fa, kern);
+    if (e == cudaSuccess) e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return e;
+    if (smem + fa.sharedSizeBytes > (size_t)optin) { *too_big = true; return cudaSuccess; }
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   kern<<<grid, HEAD_THREADS, smem, s>>>(a);
@@ -106,11 +114,17 @@ extern "C" int bild_op_lm_head_static(const void* W, int w_dtype, const float* X
   h.W = W; h.X = X; h.ldx = K; h.gain = gain; h.eps = eps; h.scale = scale; h.V = V; h.K = K; h.M = M;
   h.target = target; h.logits_dbg = nullptr; h.which = 1;
   cudaError_t e;
+  bool too_big = false;
   const int MB = M == 1 ? 1 : MAXB;
   if (w_dtype == BILD_BF16)
-    e = MB == 1 ? launch_t<__nv_bfloat16, 1, 4>(h, grid, s) : launch_t<__nv_bfloat16, MAXB, 2>(h, grid, s);
+    e = MB == 1 ? launch_t<__nv_bfloat16, 1, 4>(h, grid, s, &too_big) : launch_t<__nv_bfloat16, MAXB, 2>(h, grid, s, &too_big);
   else
-    e = MB == 1 ? launch_t<float, 1, 4>(h, grid, s) : launch_t<float, MAXB, 2>(h, grid, s);
+    e = MB == 1 ? launch_t<float, 1, 4>(h, grid, s, &too_big) : launch_t<float, MAXB, 2>(h, grid, s, &too_big);
+  if (too_big) {
+    std::fprintf(stderr, "bild_op_lm_head_static: %d staged rows of K=%d floats do not fit a block's shared memory "
+                 "(M >= 2 takes K <= about 3500)\n", MB, K);
+    return BILD_ERR_CAPACITY;
+  }
   if (e != cudaSuccess) return BILD_ERR_CUDA;
   const HeadOut* o = h.out;
   e = cudaMemcpyAsync(argmax_out, o->argmax, M * sizeof(int), cudaMemcpyDeviceToDevice, s);

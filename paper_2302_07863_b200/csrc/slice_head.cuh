@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
   const int ntiles = (ne - nb + TR - 1) >> tr_sh;
   const __nv_bfloat16* W = (const __nv_bfloat16*)a.W;
   if (tid == 0) {
-    for (int i = 0; i < SH_TILES; ++i) { mg_mbar_init(smem_u32(&sh->full[i]), 1); mg_mbar_init(smem_u32(&sh->empty[i]), 1); }
+    for (int i = 0; i < SH_TILES; ++i) { mbar_init(smem_u32(&sh->full[i]), 1); mbar_init(smem_u32(&sh->empty[i]), 1); }
     sh->failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -59,11 +59,11 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
   auto request = [&](int t) {
     if (t >= ntiles) return;
     const int slot = t % SH_TILES;
-    if (lane == 0) mg_mbar_expect(smem_u32(&sh->full[slot]), (uint32_t)(TR * K * 2));
+    if (lane == 0) mbar_expect(smem_u32(&sh->full[slot]), (uint32_t)(TR * K * 2));
     __syncwarp();
     if (lane < TR) {
       const int n = min(nb + t * TR + lane, ne - 1);
-      mg_bulk_g2s(smem_u32(sW + slot * tile_bytes + (size_t)lane * rowst), W + (size_t)n * K, (uint32_t)(K * 2),
+      bulk_g2s(smem_u32(sW + slot * tile_bytes + (size_t)lane * rowst), W + (size_t)n * K, (uint32_t)(K * 2),
                   smem_u32(&sh->full[slot]));
     }
   };
@@ -74,9 +74,9 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
     for (int t = SH_TILES; t < ntiles; ++t) {
       const int slot = t % SH_TILES;
       const uint32_t bar = smem_u32(&sh->empty[slot]), par = ((t / SH_TILES) - 1) & 1;
-      bool ok = mg_mbar_try(bar, par);
+      bool ok = mbar_try(bar, par);
       if (!ok && !*(volatile int*)&sh->failed) {
-        for (unsigned it = 0; it < MG_SPIN && !ok; ++it) ok = mg_mbar_try(bar, par);
+        for (unsigned it = 0; it < SPIN_LIMIT && !ok; ++it) ok = mbar_try(bar, par);
         if (!ok && lane == 0) { sh->failed = 1; atomicExch(err, (int)BILD_ERR_TIMEOUT); }
       }
       request(t);
@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
       *reinterpret_cast<float4*>(Xs + (size_t)m * xst + j) = v;
     }
   }
-  mg_csync();
+  csync256();
   // thread <-> (row r of the tile, token m)
   const int er = tid & (TR - 1), em = tid >> tr_sh;
   const int ks_sh = TR == 32 ? 2 : 3;   // the K range of a 16-row tile is split over 8 (4) warps
@@ -117,17 +117,17 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
     const int slot = t % SH_TILES;
     {   // bounded wait for the tile
       const uint32_t bar = smem_u32(&sh->full[slot]), par = (t / SH_TILES) & 1;
-      bool ok = mg_mbar_try(bar, par);
+      bool ok = mbar_try(bar, par);
       if (!ok && !*(volatile int*)&sh->failed) {
-        for (unsigned it = 0; it < MG_SPIN && !ok; ++it) ok = mg_mbar_try(bar, par);
+        for (unsigned it = 0; it < SPIN_LIMIT && !ok; ++it) ok = mbar_try(bar, par);
         if (!ok) { sh->failed = 1; atomicExch(err, (int)BILD_ERR_TIMEOUT); }
       }
     }
     float* ps = psum + (t & 1) * (8 * 2 * 128);
     if (NT == 1) sl_mma<1>(sW + slot * tile_bytes, rowst, TR, K, Xs, xst, M, ps, warp, lane);
     else sl_mma<2>(sW + slot * tile_bytes, rowst, TR, K, Xs, xst, M, ps, warp, lane);
-    mg_csync();   // partial sums complete; every warp is done with the tile
-    if (tid == 0) mg_mbar_arrive(smem_u32(&sh->empty[slot]));   // the producer may refill it
+    csync256();   // partial sums complete; every warp is done with the tile
+    if (tid == 0) mbar_arrive(smem_u32(&sh->empty[slot]));   // the producer may refill it
     if (em < M) {
       // fragment layout of the accumulators: row = group (+ 8), token = 2 * (lane & 3) (+ 1)
       const int col = em & 7, mt = er >> 4, rr = er & 15;
@@ -155,13 +155,13 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
   }
   if (er == 0 && em < M) a.partials[(size_t)blockIdx.x * MAXB + em] = run;
   __threadfence();
-  mg_csync();
+  csync256();
   if (tid == 0) {
     const unsigned tk = atomicAdd(a.counter, 1u);
     sh->last = (tk == gridDim.x - 1);
     if (sh->last) *a.counter = 0;
   }
-  mg_csync();
+  csync256();
   if (!sh->last) return;
   __threadfence();
   for (int m = warp; m < M; m += SH_COMPUTE / 32) {
@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
       if (m == 0) a.out->pmax = 1.f / p.s;
     }
   }
-  mg_csync();
+  csync256();
   if (tid == 0) {
     __threadfence();
     HeadOut* o = a.out;

@@ -22,7 +22,6 @@
 //     rows for the T5-large shapes, so five to sixteen token rows finish in one turn).
 #pragma once
 #include "decode_kernels.cuh"
-#include "mega_pass.cuh"
 
 namespace bild {
 
@@ -57,10 +56,10 @@ inline size_t slice_smem_bytes(int w_bytes, int x_rows, int K) {
 
 __device__ __forceinline__ void sl_wait(SliceShared* sh, int* err, unsigned long long* bar, uint32_t parity) {
   const uint32_t b = smem_u32(bar);
-  if (mg_mbar_try(b, parity)) return;
+  if (mbar_try(b, parity)) return;
   if (*(volatile int*)&sh->failed) return;
-  for (unsigned it = 0; it < MG_SPIN; ++it)
-    if (mg_mbar_try(b, parity)) return;
+  for (unsigned it = 0; it < SPIN_LIMIT; ++it)
+    if (mbar_try(b, parity)) return;
   sh->failed = 1;
   atomicExch(err, (int)BILD_ERR_TIMEOUT);
 }
@@ -111,7 +110,7 @@ __device__ __forceinline__ void sl_items(const unsigned char* sW, int rowbytes, 
         }
       }
     }
-    const float r = mg_treduce<NP>(acc, lane);
+    const float r = treduce<NP>(acc, lane);
     if ((lane & (32 / NP - 1)) == 0) psum[(qd * 8 + warp) * 32 + (lane >> SH)] = r;
   }
 }
@@ -185,11 +184,11 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
   SliceShared* sh = reinterpret_cast<SliceShared*>(psum + SL_PSUM / 4);
   float* sG = psum + SL_PSUM / 4 + SL_MISC / 4;   // [K] norm gains
   if (tid == 0) {
-    mg_mbar_init(smem_u32(&sh->wbar), 1);
-    mg_mbar_init(smem_u32(&sh->xbar), 1);
+    mbar_init(smem_u32(&sh->wbar), 1);
+    mbar_init(smem_u32(&sh->xbar), 1);
     sh->failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    mg_mbar_expect(smem_u32(&sh->wbar), (uint32_t)(nrows * K * 2));
+    mbar_expect(smem_u32(&sh->wbar), (uint32_t)(nrows * K * 2));
   }
   __syncthreads();
   // the weights depend on nothing: request them before waiting for the kernel in front, one copy per
@@ -197,7 +196,7 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
   if (tid < nrows) {
     const int r = tid < n ? tid : tid - n;
     const __nv_bfloat16* W = (const __nv_bfloat16*)(tid < n ? a.W0 : a.W1);
-    mg_bulk_g2s(smem_u32(sW + (size_t)tid * rowbytes), W + (size_t)(r0 + r) * K, (uint32_t)(K * 2), smem_u32(&sh->wbar));
+    bulk_g2s(smem_u32(sW + (size_t)tid * rowbytes), W + (size_t)(r0 + r) * K, (uint32_t)(K * 2), smem_u32(&sh->wbar));
   }
   float4 gv[2];   // gains of the columns this thread scales (K <= 2048 where a norm precedes)
   if (a.gain) {
@@ -253,11 +252,11 @@ __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
       }
       __syncthreads();
     } else {
-    if (tid == 0) mg_mbar_expect(smem_u32(&sh->xbar), (uint32_t)(mg * K * 4));
+    if (tid == 0) mbar_expect(smem_u32(&sh->xbar), (uint32_t)(mg * K * 4));
     __syncthreads();   // the barrier expects the bytes (and the group before is done with the rows)
     if (tid < mg) {
       asm volatile("fence.proxy.async;" ::: "memory");   // rows written by the kernel in front, read by the copy engine
-      mg_bulk_g2s(smem_u32(Xs + (size_t)tid * xst), a.X + (size_t)(m0 + tid) * a.ldx, (uint32_t)(K * 4), smem_u32(&sh->xbar));
+      bulk_g2s(smem_u32(Xs + (size_t)tid * xst), a.X + (size_t)(m0 + tid) * a.ldx, (uint32_t)(K * 4), smem_u32(&sh->xbar));
     }
     sl_wait(sh, s.err, &sh->xbar, xuse & 1);
     }

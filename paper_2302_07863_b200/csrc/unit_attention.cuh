@@ -12,7 +12,6 @@
 //     warp per row, weighted values one (row, channel) pair per thread and group of rows.
 #pragma once
 #include "decode_kernels.cuh"
-#include "mega_pass.cuh"
 
 namespace bild {
 
@@ -50,8 +49,8 @@ __global__ void __launch_bounds__(UA_THREADS_MAX) uattn_kernel(DAttnArgs d, int 
   UAttnShared* sh = reinterpret_cast<UAttnShared*>(sM + (size_t)ns * MB * pst + ((ns * MB * pst) & 1));
   float* sP1 = reinterpret_cast<float*>(sh + 1);     // [4 key quarters][64 channels], single-row passes
   if (tid == 0) {
-    mg_mbar_init(smem_u32(&sh->kvbar[0]), 1);
-    mg_mbar_init(smem_u32(&sh->kvbar[1]), 1);
+    mbar_init(smem_u32(&sh->kvbar[0]), 1);
+    mbar_init(smem_u32(&sh->kvbar[1]), 1);
     sh->failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -66,9 +65,9 @@ __global__ void __launch_bounds__(UA_THREADS_MAX) uattn_kernel(DAttnArgs d, int 
       if (tid != 0) continue;
       const int jc = j0 + issued * UA_CK, nk = min(UA_CK, j1 - jc), buf = issued & 1;
       const uint32_t bar = smem_u32(&sh->kvbar[buf]), bytes = (uint32_t)(nk * dkv * 4);
-      mg_mbar_expect(bar, 2 * bytes);
-      mg_bulk_g2s(smem_u32(sKV + (size_t)buf * 2 * chunk_floats), Kh + (size_t)jc * dkv, bytes, bar);
-      mg_bulk_g2s(smem_u32(sKV + (size_t)buf * 2 * chunk_floats + chunk_floats), Vh + (size_t)jc * dkv, bytes, bar);
+      mbar_expect(bar, 2 * bytes);
+      bulk_g2s(smem_u32(sKV + (size_t)buf * 2 * chunk_floats), Kh + (size_t)jc * dkv, bytes, bar);
+      bulk_g2s(smem_u32(sKV + (size_t)buf * 2 * chunk_floats + chunk_floats), Vh + (size_t)jc * dkv, bytes, bar);
     }
   };
   auto set_range = [&](int n_all) {
@@ -117,9 +116,9 @@ __global__ void __launch_bounds__(UA_THREADS_MAX) uattn_kernel(DAttnArgs d, int 
     const int jc = j0 + c * UA_CK, nk = min(UA_CK, j1 - jc);
     {   // bounded wait for the chunk
       const uint32_t bar = smem_u32(&sh->kvbar[buf]);
-      bool ok = mg_mbar_try(bar, (c >> 1) & 1);
+      bool ok = mbar_try(bar, (c >> 1) & 1);
       if (!ok && !*(volatile int*)&sh->failed) {
-        for (unsigned it = 0; it < MG_SPIN && !ok; ++it) ok = mg_mbar_try(bar, (c >> 1) & 1);
+        for (unsigned it = 0; it < SPIN_LIMIT && !ok; ++it) ok = mbar_try(bar, (c >> 1) & 1);
         if (!ok) { sh->failed = 1; atomicExch(a.err, (int)BILD_ERR_TIMEOUT); }
       }
     }

@@ -7,7 +7,9 @@ the oracle's BiLD tokens / trace / counters / decision margins, the two greedy
 baselines, and a sample of the logits of every model call of the BiLD run
 (arg-max, log-sum-exp, max probability and the logits at a fixed set of
 vocabulary indices), which the GPU parity tests compare against without having
-to re-run the oracle at full size.  No value here comes from the CUDA path.
+to re-run the oracle at full size.  If the file exists already, its calibration
+(logit scales, thresholds) is kept and only the oracle runs are repeated
+(`--recalibrate` calibrates afresh).  No value here comes from the CUDA path.
 The paper prints no numeric worked example, so none of these are the paper's.
 """
 import json
@@ -51,8 +53,14 @@ def sample_rows(r, vocab, seed):
     return [int(i) for i in idx], out
 
 
+def fin(v):
+    """JSON has no infinity: margins that do not apply are stored as null."""
+    return None if math.isinf(v) else float(v)
+
+
 def main(names):
-    for name in names:
+    recal = "--recalibrate" in names
+    for name in [n for n in names if not n.startswith("--")]:
         t0 = time.time()
         wl = WORKLOADS[name]
         sS, sL = MODEL_SHAPES[wl.small], MODEL_SHAPES[wl.large]
@@ -60,11 +68,19 @@ def main(names):
         L = Model(sL, gen_model(sL, wl.seed, wl.dtype))
         ids = gen_ids(sS.vocab, wl.enc_len, wl.seed)
         print(f"[{name}] models ready {time.time() - t0:.1f}s", flush=True)
-        cs = calibrate.calibrate_scale(S, ids, wl.gen_len)
-        cl = calibrate.calibrate_scale(L, ids, wl.gen_len)
-        print(f"[{name}] scales {cs} {cl} {time.time() - t0:.1f}s", flush=True)
-        fb, rb, mm, runs = BANDS[name]
-        th = calibrate.calibrate_thresholds(S, L, ids, wl.gen_len, wl.max_draft, fb, rb, mm, runs)
+        path = os.path.join(HERE, name + ".json")
+        old = None
+        if os.path.exists(path) and not recal:
+            with open(path) as f:
+                old = json.load(f)
+            cs, cl, th = old["scale_small"], old["scale_large"], old["thresholds"]
+            S.logit_scale, L.logit_scale = float(cs["scale"]), float(cl["scale"])
+        else:
+            cs = calibrate.calibrate_scale(S, ids, wl.gen_len)
+            cl = calibrate.calibrate_scale(L, ids, wl.gen_len)
+            print(f"[{name}] scales {cs} {cl} {time.time() - t0:.1f}s", flush=True)
+            fb, rb, mm, runs = BANDS[name]
+            th = calibrate.calibrate_thresholds(S, L, ids, wl.gen_len, wl.max_draft, fb, rb, mm, runs)
         print(f"[{name}] thresholds {th} {time.time() - t0:.1f}s", flush=True)
         r = bild.generate(S, L, ids, th["alpha_fb"], th["alpha_rb"], wl.gen_len, max_draft=wl.max_draft,
                           keep_logits=True)
@@ -75,11 +91,16 @@ def main(names):
             workload=name, seed=wl.seed, enc_len=wl.enc_len, gen_len=wl.gen_len, max_draft=wl.max_draft,
             scale_small=cs, scale_large=cl, thresholds=th,
             bild=dict(tokens=r["tokens"], trace=[list(t) for t in r["trace"]], stats=r["stats"],
-                      margins={k: float(v) for k, v in r["margins"].items()}),
-            small_only=dict(tokens=rs["tokens"], argmax_margin=float(rs["margins"]["argmax"])),
-            large_only=dict(tokens=rl["tokens"], argmax_margin=float(rl["margins"]["argmax"])),
+                      margins={k: float(v) for k, v in r["margins"].items()},
+                      trace_margins=[[fin(v) for v in t] for t in r["trace_margins"]]),
+            small_only=dict(tokens=rs["tokens"], argmax_margin=float(rs["margins"]["argmax"]),
+                            gaps=[float(t[0]) for t in rs["trace_margins"]]),
+            large_only=dict(tokens=rl["tokens"], argmax_margin=float(rl["margins"]["argmax"]),
+                            gaps=[float(t[0]) for t in rl["trace_margins"]]),
             sample_idx=idx, sample_rows=rows)
-        with open(os.path.join(HERE, name + ".json"), "w") as f:
+        if old is not None:   # same calibration, same oracle: the runs must come out as before
+            assert old["bild"]["tokens"] == out["bild"]["tokens"] and old["bild"]["stats"] == out["bild"]["stats"], name
+        with open(path, "w") as f:
             json.dump(out, f)
         print(f"[{name}] done {time.time() - t0:.1f}s  stats {r['stats']}", flush=True)
 

@@ -66,6 +66,43 @@ def assert_trace_equal(got, want, vtol):
         assert abs(a[5] - b[5]) <= vtol * max(1.0, abs(b[5])), (a, b)
 
 
+# A logit error of at most e moves a top-1 / top-2 gap by at most 2e, ln p_max by at most 2e (so p_max by at most
+# 2e) and a distance d = lse - z[y] by at most 2e.  The bf16 tests assert e <= 2e-3 on every compared logit, the
+# fp32 tests e <= 1e-4; a decision whose oracle margin is above MARGIN[...] therefore cannot come out differently.
+MARGIN = {"fp32": 3e-4, "bf16": 5e-3}
+
+
+def assert_trace_matches_up_to_low_margin(got, want, margins, dtype, vtol=1e-3):
+    """BASELINE rule for traces: records are identical (value within vtol) up to the first record whose OWN oracle
+    margin is below the tolerance-derived bound; a difference anywhere else fails.  Returns the index of that
+    first low-margin record if the traces part there, else None (traces identical throughout)."""
+    lim = MARGIN[dtype]
+    for i, (b, mg) in enumerate(zip(want, margins)):
+        low = any(v is not None and v <= lim for v in mg)
+        if i >= len(got):
+            raise AssertionError(f"device trace ends at record {i}, oracle has {len(want)}")
+        a = got[i]
+        same = tuple(a[:5]) == tuple(b[:5]) and abs(a[5] - b[5]) <= vtol * max(1.0, abs(b[5]))
+        if same:
+            continue
+        assert low, f"trace differs at record {i} ({a} vs {b}) whose oracle margins {mg} are above {lim}"
+        return i
+    assert len(got) == len(want), (len(got), len(want))
+    return None
+
+
+def assert_tokens_match_up_to_low_gap(got, want, gaps, dtype):
+    """Greedy runs of one model: identical tokens up to the first position whose top-1 / top-2 gap is below the bound."""
+    lim = MARGIN[dtype]
+    for i, (b, gap) in enumerate(zip(want, gaps)):
+        assert i < len(got)
+        if got[i] != b:
+            assert gap <= lim, f"token {i} differs ({got[i]} vs {b}) although the oracle's gap {gap} is above {lim}"
+            return i
+    assert len(got) == len(want)
+    return None
+
+
 # ---- single kernels ---------------------------------------------------------------
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("M,N,K", [(1, 7, 64), (1, 515, 2048), (3, 96, 136), (16, 1031, 1024), (11, 257, 4096),
@@ -244,9 +281,11 @@ def test_generate_matches_golden(torch_cuda, name):
     assert r["stats"] == g["bild"]["stats"]
     assert ctx.generate(MODE_SMALL_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["small_only"]["tokens"]
     assert ctx.generate(MODE_LARGE_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["large_only"]["tokens"]
-    # twice in a row: same result (state fully reset, no stale cache rows)
+    # twice in a row: same result (state fully reset, no stale cache rows); the recorded confidences may differ
+    # in the last bits, since the fused sub-layers add their partial sums at the L2 in no fixed order
     r2 = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
-    assert r2["tokens"] == r["tokens"] and r2["trace"] == r["trace"]
+    assert r2["tokens"] == r["tokens"]
+    assert_trace_equal(r2["trace"], r["trace"], 1e-5)
 
 
 @pytest.mark.parametrize("name", ["tiny", "odd_bf16"])
@@ -263,35 +302,34 @@ def test_generate_matches_live_oracle(torch_cuda, name, alpha_fb, alpha_rb, max_
     S, L, _ = get_oracle(name)
     want = obild.generate(S, L, ids, alpha_fb, alpha_rb, wl.gen_len, max_draft=max_draft)
     got = ctx.generate(MODE_BILD, alpha_fb, alpha_rb, wl.gen_len)
-    tol = TOL[wl.dtype]
-    if min(want["margins"].values()) > 4 * tol or wl.dtype == "fp32":
+    tm = [[None if math.isinf(v) else v for v in t] for t in want["trace_margins"]]
+    n = assert_trace_matches_up_to_low_margin(got["trace"], want["trace"], tm, wl.dtype)
+    if n is None:
         assert got["tokens"] == want["tokens"]
-        assert_trace_equal(got["trace"], want["trace"], 1e-3)
         assert got["stats"] == want["stats"]
-    else:   # compare up to the first low-margin decision
-        n = next((i for i, (a, b) in enumerate(zip(got["trace"], want["trace"])) if tuple(a[:5]) != tuple(b[:5])),
-                 None)
-        assert n is None or n > 0
 
 
-@pytest.mark.parametrize("env", ["BILD_BLOCK_SIMT=1", "BILD_HOST_LOOP=1", "BILD_NO_PDL=1", "BILD_NO_UMMA=1", "BILD_MEGA=1",
-                                 "BILD_SLICE=0", "BILD_SLICE=2", "BILD_SLICE_MMA_MIN=5", "BILD_UNIT_ATTN=0", "BILD_SLICE_HEAD=0",
+@pytest.mark.parametrize("env", ["BILD_FUSED=0,BILD_BLOCK_SIMT=1", "BILD_HOST_LOOP=1", "BILD_NO_PDL=1", "BILD_NO_UMMA=1",
+                                 "BILD_FUSED=0", "BILD_FUSED=2", "BILD_FUSED=2,BILD_FFN_PARTS=2",
+                                 "BILD_FUSED=0,BILD_SLICE=0", "BILD_FUSED=0,BILD_SLICE=2", "BILD_FUSED=0,BILD_SLICE_MMA_MIN=5",
+                                 "BILD_FUSED=0,BILD_UNIT_ATTN=0", "BILD_FUSED=0,BILD_SLICE_HEAD=0",
                                  "BILD_SLICE_HEAD=1", "BILD_ENC_GEMM=0", "BILD_ENC_SERIAL=1"])
 @pytest.mark.parametrize("name", ["tiny_bf16", "odd"])
 def test_alternative_paths_match_golden(torch_cuda, name, env):
-    """The switchable paths (SIMT block GEMV, host-driven loop, plain launches, no tcgen05 kernels, persistent
-    pass, row-slice kernel off / also for single rows, SIMT items up to 4 rows, earlier attention kernel, earlier
-    block head, tensor-core head for single rows, encoder on the 16-row kernel) give the same tokens and trace as
-    the stored oracle run."""
-    env, env_value = env.split("=")
+    """The switchable paths (fused sub-layer kernels off / also for block passes / feed-forward in two launches, SIMT
+    block GEMV, host-driven loop, plain launches, no tcgen05 kernels, row-slice kernel off / also for single rows,
+    SIMT items up to 4 rows, earlier attention kernel, earlier block head, tensor-core head for single rows, encoder
+    on the 16-row kernel) give the same tokens and trace as the stored oracle run."""
     from paper_2302_07863_b200 import MODE_BILD
     from paper_2302_07863_b200.synthetic import make_context
     g = golden(name)
-    os.environ[env] = env_value
+    envs = dict(e.split("=") for e in env.split(","))
+    os.environ.update(envs)
     try:
         ctx, ids, wl = make_context(name, g["scale_small"]["scale"], g["scale_large"]["scale"])
     finally:
-        del os.environ[env]
+        for e in envs:
+            del os.environ[e]
     ctx.encode(ids)
     th = g["thresholds"]
     r = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
@@ -377,45 +415,16 @@ def test_full_size_replay_and_generate(torch_cuda, name):
     assert worst <= tol, worst
 
     # whole loop on the device
+    assert worst <= 2e-3, worst     # the bound the margin rule below is derived from
     r = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
-    mg = g["bild"]["margins"]
-    if mg["argmax"] > 2 * tol and mg["fallback"] > 2 * tol and mg["rollback"] > 2 * tol:
+    n = assert_trace_matches_up_to_low_margin(r["trace"], g["bild"]["trace"], g["bild"]["trace_margins"], wl.dtype)
+    if n is None:
         assert r["tokens"] == g["bild"]["tokens"]
         assert r["stats"] == g["bild"]["stats"]
-    else:
-        n = next((i for i, (a, b) in enumerate(zip(r["trace"], g["bild"]["trace"])) if tuple(a[:5]) != tuple(b[:5])),
-                 None)
-        if n is not None:     # a divergence is only allowed at a low-margin decision
-            lows = [i for i, row in enumerate(g["sample_rows"]) if row["gap"] <= 2 * tol
-                    or abs(row["pmax"] - th["alpha_fb"]) <= 2 * tol]
-            assert lows, "trace differs although every oracle margin is above tolerance"
-    if g["small_only"]["argmax_margin"] > 2 * tol:
-        assert ctx.generate(MODE_SMALL_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["small_only"]["tokens"]
-    if g["large_only"]["argmax_margin"] > 2 * tol:
-        assert ctx.generate(MODE_LARGE_ONLY, 0.0, INF, wl.gen_len)["tokens"] == g["large_only"]["tokens"]
-
-
-@pytest.mark.gpu
-def test_persistent_pass_full_size(torch_cuda):
-    """The opt-in whole-pass persistent kernel (BILD_MEGA=1) reproduces the stored oracle run of the
-    summarisation workload: same tokens and statistics where every decision margin is above tolerance."""
-    from paper_2302_07863_b200 import MODE_BILD
-    from paper_2302_07863_b200.synthetic import make_context
-    g = golden("t5_sum")
-    os.environ["BILD_MEGA"] = "1"
-    try:
-        ctx, ids, wl = make_context("t5_sum", g["scale_small"]["scale"], g["scale_large"]["scale"])
-    finally:
-        del os.environ["BILD_MEGA"]
-    ctx.encode(ids)
-    th = g["thresholds"]
-    tol = TOL[wl.dtype]
-    r = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
-    mg = g["bild"]["margins"]
-    if mg["argmax"] > 2 * tol and mg["fallback"] > 2 * tol and mg["rollback"] > 2 * tol:
-        assert r["tokens"] == g["bild"]["tokens"]
-        assert r["stats"] == g["bild"]["stats"]
-    ctx.close()
+    assert_tokens_match_up_to_low_gap(ctx.generate(MODE_SMALL_ONLY, 0.0, INF, wl.gen_len)["tokens"],
+                                      g["small_only"]["tokens"], g["small_only"]["gaps"], wl.dtype)
+    assert_tokens_match_up_to_low_gap(ctx.generate(MODE_LARGE_ONLY, 0.0, INF, wl.gen_len)["tokens"],
+                                      g["large_only"]["tokens"], g["large_only"]["gaps"], wl.dtype)
 
 
 @pytest.mark.gpu

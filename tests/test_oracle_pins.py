@@ -153,6 +153,69 @@ def test_threshold_endpoints_and_equality(pair):
     assert r_above["trace"][0][0] == bild.KIND_FALLBACK
 
 
+def test_rollback_threshold_is_strict(pair):
+    """Eq. 3 rolls back when the distance is strictly above alpha_RB: a threshold equal to the first scanned
+    distance leaves that draft in place, the next representable value below it rolls it back."""
+    wl, S, L, ids = pair
+    base = bild.generate(S, L, ids, 0.0, INF, 4, max_draft=2)            # two drafts, then a forced hand-over
+    v = next(t for t in base["trace"] if t[0] in (bild.KIND_VERIFY_OK, bild.KIND_ROLLBACK))
+    assert v[0] == bild.KIND_VERIFY_OK and v[3] == 3
+    # the distances of the two scanned drafts, recomputed from the large model alone
+    st = L.start(ids, 8)
+    Z = L.forward_block(st, [0] + base["tokens"][:2])
+    d = [bild.max_prob(Z[i])[2] - Z[i][base["tokens"][i]] for i in range(2)]
+    assert abs(max(d) - v[5]) < 1e-12
+    r_eq = bild.generate(S, L, ids, 0.0, d[0], 4, max_draft=2)
+    first = next(t for t in r_eq["trace"] if t[0] in (bild.KIND_VERIFY_OK, bild.KIND_ROLLBACK))
+    assert not (first[0] == bild.KIND_ROLLBACK and first[4] == 0)          # d_0 == alpha_RB: no violation at row 0
+    r_below = bild.generate(S, L, ids, 0.0, np.nextafter(d[0], -INF), 4, max_draft=2)
+    first = next(t for t in r_below["trace"] if t[0] in (bild.KIND_VERIFY_OK, bild.KIND_ROLLBACK))
+    assert first[0] == bild.KIND_ROLLBACK and first[4] == 0 and first[5] == d[0]
+
+
+def test_trace_margins_line_up_with_the_trace(pair):
+    """One margin triple per trace record; their minima are the global margins."""
+    wl, S, L, ids = pair
+    r = bild.generate(S, L, ids, 0.3, 16.0, 24, max_draft=4)
+    tm = r["trace_margins"]
+    assert len(tm) == len(r["trace"])
+    assert min(t[1] for t in tm) == r["margins"]["fallback"] and min(t[2] for t in tm) == r["margins"]["rollback"]
+    # the per-record gaps also cover the rejected candidates a fallback record names
+    used = [t[0] for rec, t in zip(r["trace"], tm) if rec[0] not in (bild.KIND_FALLBACK, bild.KIND_FORCED)]
+    assert min(used) == r["margins"]["argmax"] and min(t[0] for t in tm) <= r["margins"]["argmax"]
+    for rec, t in zip(r["trace"], tm):
+        if rec[0] in (bild.KIND_FALLBACK, bild.KIND_FORCED, bild.KIND_SMALL_ACCEPT):
+            assert t[1] == abs(rec[5] - 0.3) and t[2] == INF
+        else:
+            assert t[1] == INF and (t[2] < INF) == (rec[3] > 1)
+
+
+def test_bf16_bit_helpers_against_torch():
+    """The shared generator's fp32 -> bf16 rounding (nearest, ties to even) and the oracle's bf16 -> fp64
+    widening, against torch's bfloat16 conversions: random values, values next to a rounding boundary,
+    exact ties, signed zeros, subnormals."""
+    import torch
+    from oracle.t5 import to_f64
+    from workloads import bf16_bits_to_f32, bf16_round_bits
+    rng = np.random.default_rng(7)
+    x = (rng.standard_normal(20000) * np.exp(rng.uniform(-30, 30, 20000))).astype(np.float32)
+    base = (rng.integers(0, 1 << 15, 4000).astype(np.uint32) << 16)             # exactly representable
+    ties = (base | 0x8000).view(np.float32)                                        # half-way cases
+    near = np.concatenate([(base | 0x7FFF).view(np.float32), (base | 0x8001).view(np.float32)])
+    special = np.array([0.0, -0.0, 1e-40, -1e-40, 1.0, -1.0, 65504.0, 3.3895314e38], dtype=np.float32)
+    x = np.concatenate([x, ties, -ties, near, -near, special])
+    x = x[np.isfinite(x)]
+    bits = bf16_round_bits(x)
+    ref = torch.from_numpy(x).to(torch.bfloat16)
+    assert np.array_equal(bits.view(np.int16), ref.view(torch.int16).numpy())
+    assert np.array_equal(bf16_bits_to_f32(bits).view(np.uint32), ref.float().numpy().view(np.uint32))
+    assert np.array_equal(to_f64(bits), ref.double().numpy())
+    # a truncating conversion or a wrong shift would differ on the ties / near-boundary values
+    assert np.any(bits != (x.view(np.uint32) >> 16).astype(np.uint16))
+    f = rng.standard_normal(100).astype(np.float32)
+    assert np.array_equal(to_f64(f), f.astype(np.float64))
+
+
 def test_forced_fallback_after_max_draft(pair):
     wl, S, L, ids = pair
     r = bild.generate(S, L, ids, 0.0, INF, 12, max_draft=3)
