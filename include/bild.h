@@ -282,6 +282,14 @@ int bild_op_lm_head_static(const void *W, int w_dtype, const float *X, const flo
                            int32_t *argmax_out, float *max_out, float *lse_out, float *gather_out,
                            void *cuda_stream);
 
+/* Test helper: one decoder layer's cached keys or values as the kernels see them, copied to
+ * HOST memory (synchronises the stream).  which: 0 small, 1 large model; what: 0 cross-attention
+ * keys, 1 cross-attention values (written by bild_encode: W_ck / W_cv times the encoder output,
+ * the per-input set-up of Section 3.2's two models), 2 / 3 self-attention keys / values (rows
+ * appended by the decoder passes).  Layout [n_heads][capacity][d_kv] fp32 with capacity =
+ * max_enc_len (cross) or max_dec_len (self); count must be exactly that many floats. */
+int bild_debug_read_cache(bild_ctx *ctx, int which, int what, int layer, float *dst_host, size_t count);
+
 /* Host-only: the relative-position bucket the library uses (T5's bucket function in
  * exact integer arithmetic).  which = 0: decoder, rel = query_pos - key_pos >= 0;
  * which = 1: encoder, rel = key_pos - query_pos.  Returns -1 on invalid arguments. */

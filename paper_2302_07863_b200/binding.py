@@ -25,7 +25,8 @@ MAX_BLOCK = 16
 EXPORTS = ["bild_query_workspace", "bild_create", "bild_destroy", "bild_encode", "bild_reset",
            "bild_small_step", "bild_large_verify", "bild_rewind", "bild_generate", "bild_generate_async",
            "bild_fetch_result", "bild_time_pass", "bild_uses_tensor_cores", "bild_launch_count", "bild_last_error", "bild_op_linear",
-           "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_op_lm_head_static", "bild_debug_bucket"]
+           "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_op_lm_head_static", "bild_debug_bucket",
+           "bild_debug_read_cache"]
 
 
 class ModelCfg(C.Structure):
@@ -254,6 +255,13 @@ class Context:
         ms = C.c_float()
         self._check(self.L.bild_time_pass(self.h, which, k, cache_len, iters, C.byref(ms)))
         return ms.value
+
+    def read_cache(self, which: int, what: int, layer: int, n_heads: int, capacity: int, d_kv: int):
+        """One layer's cached keys / values [n_heads][capacity][d_kv] as a numpy array (what: 0 / 1 cross K / V, 2 / 3 self)."""
+        out = np.empty((n_heads, capacity, d_kv), dtype=np.float32)
+        self.L.bild_debug_read_cache.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
+        self._check(self.L.bild_debug_read_cache(self.h, which, what, layer, out.ctypes.data, out.size))
+        return out
 
     def uses_tensor_cores(self) -> bool:
         return bool(self.L.bild_uses_tensor_cores(self.h))

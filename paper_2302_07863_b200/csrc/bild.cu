@@ -154,7 +154,7 @@ struct bild_ctx {
   cudaGraph_t graph[2] = {nullptr, nullptr};
   cudaGraphExec_t exec[2] = {nullptr, nullptr};
   int64_t per_pass[2] = {0, 0};      // kernel launches in one small / one large pass of the graphs
-  int64_t per_pass_large1 = 0;
+  int64_t per_pass_large1 = 0, per_pass_large8 = 0;
   int64_t* cnt = &launches;         // where launches are counted (redirected while capturing)
   cudaStream_t cap_stream = nullptr;  // capture only (the legacy default stream cannot capture); nothing runs on it
   bool block_simt = false;           // block pass on the SIMT block GEMV instead of the tensor-core kernel
@@ -171,7 +171,7 @@ struct bild_ctx {
   size_t slice_head_min_bytes = (size_t)32 << 20;
   int slice_mma_min = 3;
   size_t slice_min_bytes = 3000 * 1024;   // single-row passes: smaller matrices stay on the GEMV (measured)
-  int fused_on = 1;                  // fused sub-layer kernels where the shapes allow: 0 off, 1 single-row passes, 2 block passes too
+  int fused_on = 2;                  // fused sub-layer kernels where the shapes allow: 0 off, 1 single-row passes, 2 also passes of 2 to 8 rows
   int sub_parts_want = 0;            // 0: fewest launches of the feed-forward sub-layer that fit
   bool capturing = false;            // launches are being recorded into a graph, not run
   int64_t graph_counted = 0;         // launches of the loop graphs already added to `launches`
@@ -631,12 +631,13 @@ int setup_fused(bild_ctx* c, Model& m) {
   const int per_rank = (std::max(cap, ecap) + C - 1) / C;
   int kc = std::min(64, (per_rank + 15) / 16 * 16);   // at most 64: a chunk's scores take one turn of the block
   const int bias_len = ((cap + C - 1) / C + MAXB + 8 + 3) / 4 * 4;
-  while (kc > 16 && attn_sub_layout(d, dkv, 3, C, MAXB, kc, bias_len).total > smem_max) kc -= 16;
-  if (attn_sub_layout(d, dkv, 3, C, MAXB, kc, bias_len).total > smem_max) return BILD_OK;
+  while (kc > 16 && attn_sub_layout(d, dkv, 3, C, SUB_MB, kc, bias_len).total > smem_max) kc -= 16;
+  if (attn_sub_layout(d, dkv, 3, C, SUB_MB, kc, bias_len).total > smem_max ||
+      attn_sub_layout(d, dkv, 1, C, SUB_MB, kc, bias_len).total > smem_max) return BILD_OK;
   int parts = std::max(1, c->sub_parts_want);
   const int nmat = gated ? 2 : 1;
   while (parts <= 8 && (ffn_sub_rows(F, c->sms * parts) * nmat > SUB_MAX_ROWS || ffn_sub_rows(F, c->sms * parts) > SUB_FO_REGS ||
-                        ffn_sub_layout(d, F, gated, c->sms * parts, c->sms, MAXB).total > smem_max)) ++parts;
+                        ffn_sub_layout(d, F, gated, c->sms * parts, c->sms, SUB_MB).total > smem_max)) ++parts;
   if (parts > 8) return BILD_OK;
   if (cudaFuncSetAttribute(attn_sub_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess ||
       cudaFuncSetAttribute(attn_sub_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess ||
@@ -877,16 +878,18 @@ LoopPtrs loop_ptrs(bild_ctx* c) {
 // (steps S0..S10 / L0..L10: embed, per layer [norm+QKV+append, self-attention, O+residual,
 // norm+cross-Q, cross-attention, cross-O+residual, norm+FFN-up, FFN-down+residual],
 // final norm + LM head + policy).  MB = 1 or MAXB selects the kernel variants.
-int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned long long cond_while = 0,
-                 unsigned long long cond_if = 0, unsigned long long cond_if1 = 0) {
+// MBv: rows the pass is built for: 1, SUB_MB (2 to 8 rows) or MAXB.
+int decoder_pass(bild_ctx* c, int which, int MBv, float* logits_dbg, unsigned long long cond_while = 0,
+                 unsigned long long cond_if = 0, unsigned long long cond_if1 = 0, unsigned long long cond_if8 = 0) {
+  const int MB = MBv == 1 ? 1 : MAXB;   // variant of the kernels outside the fused sub-layers
   Model& m = c->m[which];
   const bild_model_cfg& mc = m.c;
   const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
   const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len, dt = c->cfg.dtype;
-  const bool fused = m.fused && (MB == 1 || c->fused_on >= 2);
+  const bool fused = m.fused && (MBv == 1 || (MBv == SUB_MB && c->fused_on >= 2));
   CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x, fused ? m.xb : nullptr));
   if (fused) {
-    int rc = fused_layers(c, m, MB);
+    int rc = fused_layers(c, m, MBv);
     if (rc) return rc;
   }
   // self-attention: one block per head up to 128 cached rows (no merge step); cross-attention:
@@ -945,7 +948,8 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
   h.W = m.w.lm_head; h.X = m.x; h.ldx = d; h.gain = (const float*)m.w.dec_final_ln; h.eps = mc.ln_eps;
   h.scale = mc.logit_scale; h.V = mc.vocab; h.K = d; h.desc = m.desc; h.partials = m.head_part;
   h.counter = m.head_cnt; h.out = m.head_out; h.logits_dbg = logits_dbg; h.which = which; h.loop = loop_ptrs(c);
-  h.cond_while = cond_while; h.cond_if = cond_if; h.cond_if1 = cond_if1;
+  h.cond_while = cond_while; h.cond_if = cond_if; h.cond_if1 = cond_if1; h.cond_if8 = cond_if8;
+  h.pass_kind = which == 0 ? 0 : MBv == 1 ? 2 : MBv == SUB_MB ? 3 : 1;
   const int head_tr = (MB == 1 && d <= 512) ? 32 : 16;   // rows per tile of the tensor-core head
   const size_t sh_smem = slice_head_smem_bytes(d, head_tr);
   // single-row passes: only heads of 32 MB and more (smaller ones stay on the GEMV head)
@@ -957,8 +961,7 @@ int decoder_pass(bild_ctx* c, int which, int MB, float* logits_dbg, unsigned lon
       CUDA_TRY(c, cudaFuncSetAttribute(slice_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
       c->slice_head_smem_set = true;
     }
-    CUDA_TRY(c, launch_k(c, slice_head_kernel, dim3(c->sms), dim3(SH_THREADS), sh_smem, h, which == 0 ? 0 : (MB == 1 ? 2 : 1),
-                         &c->st->err, head_tr));
+    CUDA_TRY(c, launch_k(c, slice_head_kernel, dim3(c->sms), dim3(SH_THREADS), sh_smem, h, &c->st->err, head_tr));
     return BILD_OK;
   }
   CUDA_TRY(c, launch_head(c->stream, c->use_pdl, dt, MB, h, m.head_grid, c->cnt));
@@ -1053,7 +1056,7 @@ int add_cond(bild_ctx* c, cudaGraph_t g, const cudaGraphNode_t* deps, size_t nde
 
 // Captures one decoder pass into `body`; returns the leaf nodes of the capture.
 int capture_pass(bild_ctx* c, cudaGraph_t body, int which, int MB, unsigned long long hw, unsigned long long hi,
-                 std::vector<cudaGraphNode_t>* leaves, int64_t* count, unsigned long long hi1 = 0) {
+                 std::vector<cudaGraphNode_t>* leaves, int64_t* count, unsigned long long hi1 = 0, unsigned long long hi8 = 0) {
   if (!c->cap_stream) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
   CUDA_TRY(c, cudaStreamBeginCaptureToGraph(c->cap_stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed));
   int64_t n = 0;
@@ -1061,7 +1064,7 @@ int capture_pass(bild_ctx* c, cudaGraph_t body, int which, int MB, unsigned long
   c->stream = c->cap_stream;
   c->cnt = &n;
   c->capturing = true;
-  int rc = decoder_pass(c, which, MB, nullptr, hw, hi, hi1);
+  int rc = decoder_pass(c, which, MB, nullptr, hw, hi, hi1, hi8);
   c->capturing = false;
   c->cnt = &c->launches;
   c->stream = user_stream;
@@ -1111,15 +1114,18 @@ int build_graphs(bild_ctx* c) {
 int build_graphs_once(bild_ctx* c) {
   {  // BiLD (and small-only): WHILE { small pass ; IF { large block pass } ; IF { large single-row pass } }
     CUDA_TRY(c, cudaGraphCreate(&c->graph[0], 0));
-    cudaGraphConditionalHandle hw, hi, hi1;
+    cudaGraphConditionalHandle hw, hi, hi1, hi8 = 0;
     CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hw, c->graph[0], 1, cudaGraphCondAssignDefault));
     CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi, c->graph[0], 0, cudaGraphCondAssignDefault));
     CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi1, c->graph[0], 0, cudaGraphCondAssignDefault));
-    cudaGraph_t body = nullptr, ifbody = nullptr, if1body = nullptr;
+    // passes of 2 to 8 rows have a branch of their own where they run on the fused sub-layer kernels
+    const bool body8 = c->m[1].fused && c->fused_on >= 2;
+    if (body8) CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi8, c->graph[0], 0, cudaGraphCondAssignDefault));
+    cudaGraph_t body = nullptr, ifbody = nullptr, if1body = nullptr, if8body = nullptr;
     int rc = add_cond(c, c->graph[0], nullptr, 0, hw, cudaGraphCondTypeWhile, &body);
     if (rc) return rc;
     std::vector<cudaGraphNode_t> leaves;
-    rc = capture_pass(c, body, 0, 1, hw, hi, &leaves, &c->per_pass[0], hi1);
+    rc = capture_pass(c, body, 0, 1, hw, hi, &leaves, &c->per_pass[0], hi1, hi8);
     if (rc) return rc;
     rc = add_cond(c, body, leaves.data(), leaves.size(), hi, cudaGraphCondTypeIf, &ifbody);
     if (rc) return rc;
@@ -1132,6 +1138,12 @@ int build_graphs_once(bild_ctx* c) {
     rc = capture_pass(c, if1body, 1, 1, hw, 0, nullptr, &n1);
     if (rc) return rc;
     c->per_pass_large1 = n1;
+    if (body8) {
+      rc = add_cond(c, body, leaves.data(), leaves.size(), hi8, cudaGraphCondTypeIf, &if8body);
+      if (rc) return rc;
+      rc = capture_pass(c, if8body, 1, SUB_MB, hw, 0, nullptr, &c->per_pass_large8);
+      if (rc) return rc;
+    }
     CUDA_TRY(c, cudaGraphInstantiate(&c->exec[0], c->graph[0], 0));
   }
   {  // large-only greedy: WHILE { large pass with k = 1 }
@@ -1153,7 +1165,7 @@ int read_state(bild_ctx* c) {
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   {  // kernels launched by the loop graphs so far (the device counts the passes they ran)
     const long long* cp = c->pin_state->cum_passes;
-    const int64_t total = cp[0] * c->per_pass[0] + cp[1] * c->per_pass[1] + cp[2] * c->per_pass_large1;
+    const int64_t total = cp[0] * c->per_pass[0] + cp[1] * c->per_pass[1] + cp[2] * c->per_pass_large1 + cp[3] * c->per_pass_large8;
     c->launches += total - c->graph_counted;
     c->graph_counted = total;
   }
@@ -1385,7 +1397,7 @@ int bild_large_verify(bild_ctx* c, const int32_t* tokens, int k, float alpha_rb,
   set_alpha_kernel<<<1, 1, 0, c->stream>>>(c->st, c->pin_state->alpha_fb, alpha_rb);
   set_desc_kernel<<<1, 1, 0, c->stream>>>(c->m[1].desc, c->st, 1, k, t);
   c->launches += 2;
-  rc = decoder_pass(c, 1, k == 1 ? 1 : MAXB, logits_dbg);
+  rc = decoder_pass(c, 1, k == 1 ? 1 : k <= SUB_MB ? SUB_MB : MAXB, logits_dbg);
   if (rc) return rc;
   CUDA_TRY(c, cudaMemcpyAsync(c->pin_head, c->m[1].head_out, sizeof(HeadOut), cudaMemcpyDeviceToHost, c->stream));
   rc = read_state(c);
@@ -1444,7 +1456,8 @@ int bild_generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, i
       if (rc) return rc;
       if (!c->pin_state->fallback) continue;
     }
-    rc = decoder_pass(c, 1, mode == BILD_MODE_LARGE_ONLY ? 1 : MAXB, nullptr);
+    const int kk = c->pin_state->n - c->pin_state->L_len + 1;   // rows the large model has not seen
+    rc = decoder_pass(c, 1, (mode == BILD_MODE_LARGE_ONLY || kk == 1) ? 1 : kk <= SUB_MB ? SUB_MB : MAXB, nullptr);
     if (rc) return rc;
     rc = read_state(c);
     if (rc) return rc;
@@ -1548,7 +1561,7 @@ int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, floa
   cudaGraphExec_t ex = nullptr;
   if (cudaGraphCreate(&g, 0) != cudaSuccess) rc = BILD_ERR_CUDA;
   int64_t n_launch = 0;
-  if (rc == BILD_OK) rc = capture_pass(c, g, which, k == 1 ? 1 : MAXB, 0, 0, nullptr, &n_launch);
+  if (rc == BILD_OK) rc = capture_pass(c, g, which, k == 1 ? 1 : k <= SUB_MB ? SUB_MB : MAXB, 0, 0, nullptr, &n_launch);
   if (rc == BILD_OK && cudaGraphInstantiate(&ex, g, 0) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && cudaGraphUpload(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;
   if (rc == BILD_OK && !cold && cudaGraphLaunch(ex, c->stream) != cudaSuccess) rc = BILD_ERR_CUDA;  // untimed first pass
@@ -1580,6 +1593,22 @@ int bild_debug_stamps(unsigned long long* out, int reset) {
   return BILD_OK;
 }
 #endif
+
+// Test helper: copies one layer's cached keys or values to the host (synchronises the stream).
+// what: 0 cross keys, 1 cross values, 2 self keys, 3 self values; layout [n_heads][capacity][d_kv] fp32,
+// capacity = max_enc_len (cross) or max_dec_len (self); dst holds n_heads * capacity * d_kv floats.
+int bild_debug_read_cache(bild_ctx* c, int which, int what, int layer, float* dst_host, size_t count) {
+  if (!c || !dst_host || (which != 0 && which != 1) || what < 0 || what > 3) return fail(c, BILD_ERR_ARG, "null argument / which / what");
+  Model& m = c->m[which];
+  if (layer < 0 || layer >= m.c.n_layers) return fail(c, BILD_ERR_ARG, "layer out of range");
+  const size_t cap = what < 2 ? c->cfg.max_enc_len : c->cfg.max_dec_len;
+  const size_t n = (size_t)m.c.n_heads * cap * m.c.d_kv;
+  if (count != n) return fail(c, BILD_ERR_ARG, "count must be n_heads * capacity * d_kv");
+  const float* base = what == 0 ? m.crossK : what == 1 ? m.crossV : what == 2 ? m.selfK : m.selfV;
+  CUDA_TRY(c, cudaMemcpyAsync(dst_host, base + (size_t)layer * n, n * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return BILD_OK;
+}
 
 // Host-only helper for tests of the bucket tables: which = 0 decoder (delta = query - key >= 0),
 // 1 encoder (rel = key - query).

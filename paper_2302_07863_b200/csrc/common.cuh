@@ -51,7 +51,7 @@ struct DevState {
   bild_stats stats;
   int passes;   // decoder passes taken by the running loop (guards against a runaway loop)
   int pad0;
-  long long cum_passes[3];   // passes run from the loop graphs since create: small, large block, large single row
+  long long cum_passes[4];   // passes run from the loop graphs since create: small, large block, large single row, large up to 8 rows
 };
 
 struct Partial {  // running soft-max statistics of a slice of the vocabulary

@@ -697,20 +697,7 @@ __global__ void __launch_bounds__(HEAD1_THREADS) head1_kernel(HeadArgs a) {
     o->lse[0] = p.m + logf(p.s);
     o->pmax = 1.f / p.s;
     o->gather[0] = __ldcg(&o->gather[0]);
-    if (a.loop.st) {
-      policy_tests(o, a.desc, a.loop.st, a.which);
-      if (a.desc->run_policy) policy_step(a.loop, o, a.desc, a.which);
-      else if (a.which == 0) a.loop.st->S_len = a.desc->pos0 + 1;
-      else a.loop.st->L_len = a.desc->pos0 + a.desc->k;
-      if (a.cond_while) {
-        a.loop.st->cum_passes[a.which == 0 ? 0 : 2]++;
-        cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
-      }
-      // the large pass wanted next: the single-row graph branch if it has one row (and that branch exists), else the block branch
-      const bool one_row = a.cond_if1 && a.loop.st->fallback && a.loop.descL->k == 1;
-      if (a.cond_if) cudaGraphSetConditional(a.cond_if, (a.loop.st->fallback && !one_row) ? 1u : 0u);
-      if (a.cond_if1) cudaGraphSetConditional(a.cond_if1, one_row ? 1u : 0u);
-    }
+    policy_tail(a, o);
   }
 }
 

@@ -480,7 +480,31 @@ struct HeadArgs {
   // handles of the graph's WHILE (loop goes on) and IF (large pass wanted) nodes; 0 = not in a graph
   unsigned long long cond_while, cond_if;
   unsigned long long cond_if1;   // IF node of the single-row large pass (0: the block branch takes every large pass)
+  unsigned long long cond_if8;   // IF node of the large pass over 2 to 8 rows (0: the block branch takes them)
+  int pass_kind;                 // which pass counter the kernel bumps inside a loop graph: 0 small, 1 block, 2 single row, 3 up to 8 rows
 };
+
+// What the last block of every LM-head kernel does once the per-row results are complete: the policy tests, the
+// bookkeeping of Algorithm 1, and (inside a loop graph) the choice of what runs next.
+__device__ inline void policy_tail(const HeadArgs& a, HeadOut* o) {
+  if (!a.loop.st) return;
+  policy_tests(o, a.desc, a.loop.st, a.which);
+  if (a.desc->run_policy) policy_step(a.loop, o, a.desc, a.which);
+  else if (a.which == 0) a.loop.st->S_len = a.desc->pos0 + 1;
+  else a.loop.st->L_len = a.desc->pos0 + a.desc->k;
+  if (a.cond_while) {
+    a.loop.st->cum_passes[a.pass_kind]++;
+    cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
+  }
+  // the large pass wanted next: the graph branch for its row count where that branch exists, else the block branch
+  const bool fb = a.loop.st->fallback != 0;
+  const int kn = a.loop.descL->k;
+  const bool one_row = a.cond_if1 && fb && kn == 1;
+  const bool upto8 = a.cond_if8 && fb && !one_row && kn <= 8;
+  if (a.cond_if) cudaGraphSetConditional(a.cond_if, (fb && !one_row && !upto8) ? 1u : 0u);
+  if (a.cond_if1) cudaGraphSetConditional(a.cond_if1, one_row ? 1u : 0u);
+  if (a.cond_if8) cudaGraphSetConditional(a.cond_if8, upto8 ? 1u : 0u);
+}
 
 constexpr int HEAD_THREADS = 256;
 
@@ -615,20 +639,7 @@ __global__ void __launch_bounds__(HEAD_THREADS) lm_head_kernel(HeadArgs a) {
     HeadOut* o = a.out;
     // gather[] was written by other blocks before their tickets: read around L1
     for (int m = 0; m < mrows; ++m) o->gather[m] = __ldcg(&o->gather[m]);
-    if (a.loop.st) {
-      policy_tests(o, a.desc, a.loop.st, a.which);
-      if (a.desc->run_policy) policy_step(a.loop, o, a.desc, a.which);
-      else if (a.which == 0) a.loop.st->S_len = a.desc->pos0 + 1;
-      else a.loop.st->L_len = a.desc->pos0 + a.desc->k;
-      if (a.cond_while) {
-        a.loop.st->cum_passes[a.which == 0 ? 0 : (MB == 1 ? 2 : 1)]++;
-        cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
-      }
-      // the large pass wanted next: the single-row graph branch if it has one row (and that branch exists), else the block branch
-      const bool one_row = a.cond_if1 && a.loop.st->fallback && a.loop.descL->k == 1;
-      if (a.cond_if) cudaGraphSetConditional(a.cond_if, (a.loop.st->fallback && !one_row) ? 1u : 0u);
-      if (a.cond_if1) cudaGraphSetConditional(a.cond_if1, one_row ? 1u : 0u);
-    }
+    policy_tail(a, o);
   }
 }
 

@@ -32,8 +32,7 @@ inline size_t slice_head_smem_bytes(int K, int tile_rows) {
   return SH_TILES * slice_head_tile_bytes(K, tile_rows) + (size_t)MAXB * (K + SL_XPAD) * 4 + 2 * 8 * 2 * 128 * 4 + 1024;
 }
 
-// pass_kind: index of the pass counter the kernel bumps when it runs inside a loop graph
-__global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int pass_kind, int* err, int TR) {
+__global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int* err, int TR) {
   extern __shared__ __align__(1024) unsigned char shd_smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K, V = a.V, G = gridDim.x;
@@ -194,20 +193,7 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int 
     HeadOut* o = a.out;
     // gather[] was written by other blocks before their tickets: read around L1
     for (int m = 0; m < M; ++m) o->gather[m] = __ldcg(&o->gather[m]);
-    if (a.loop.st) {
-      policy_tests(o, a.desc, a.loop.st, a.which);
-      if (a.desc->run_policy) policy_step(a.loop, o, a.desc, a.which);
-      else if (a.which == 0) a.loop.st->S_len = a.desc->pos0 + 1;
-      else a.loop.st->L_len = a.desc->pos0 + a.desc->k;
-      if (a.cond_while) {
-        a.loop.st->cum_passes[pass_kind]++;
-        cudaGraphSetConditional(a.cond_while, a.loop.st->done ? 0u : 1u);
-      }
-      // the large pass wanted next: the single-row graph branch if it has one row (and that branch exists), else the block branch
-      const bool one_row = a.cond_if1 && a.loop.st->fallback && a.loop.descL->k == 1;
-      if (a.cond_if) cudaGraphSetConditional(a.cond_if, (a.loop.st->fallback && !one_row) ? 1u : 0u);
-      if (a.cond_if1) cudaGraphSetConditional(a.cond_if1, one_row ? 1u : 0u);
-    }
+    policy_tail(a, o);
   }
 }
 

@@ -139,7 +139,7 @@ __device__ __forceinline__ void sl_mma(const unsigned char* sW, int rowst, int n
   float c[NT][4];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
-#pragma unroll 2
+#pragma unroll 4
   for (int st = s0; st < s1; ++st) {
     const int k0 = st << 4;
     const bool tail = k0 + 8 >= K;   // K is a multiple of 8: the second half of the last step may not exist
