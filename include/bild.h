@@ -153,11 +153,43 @@ int bild_query_workspace(const bild_config *cfg /*HOST*/, size_t *bytes /*HOST o
 
 /* Build a context.  `workspace` is DEVICE memory, 256-byte aligned, at least
  * bild_query_workspace bytes, caller-owned, used exclusively by this context until
- * bild_destroy.  `cuda_stream` is a cudaStream_t (NULL = default stream).  Uploads a
- * few small tables; no other device work.  Errors: ARG, WORKSPACE, CUDA. */
+ * bild_destroy.  `cuda_stream` is a cudaStream_t (NULL = default stream).  Device work done
+ * here, on that stream, with a synchronisation before returning: the workspace is cleared,
+ * the relative-position bias tables are expanded by distance, and (bf16 configurations) each
+ * decoder layer's feed-forward output matrix is transposed into the workspace for the fused
+ * sub-layer kernels.  Errors: ARG, WORKSPACE, CUDA. */
 int bild_create(const bild_config *cfg /*HOST*/, const bild_weights *small_w /*HOST*/,
                 const bild_weights *large_w /*HOST*/, void *workspace /*DEVICE*/,
                 size_t workspace_bytes, void *cuda_stream, bild_ctx **out /*HOST out*/);
+
+/* Kernel selection and debugging switches (no counterpart in the paper).  The product path is
+ * what bild_tuning_default() fills in and what bild_create uses; tests and measurements set
+ * single fields to reach the comparison kernels.  Nothing is read from the environment. */
+typedef struct {
+  int32_t host_loop;         /* 1: bild_generate is driven from the host, one state read-back per pass (debug) */
+  int32_t pdl;               /* 1: kernels of a pass are launched with programmatic dependent launch */
+  int32_t fused;             /* fused sub-layer kernels: 0 off, 1 single-row passes, 2 also passes of 2 to 8 rows */
+  int32_t ffn_parts;         /* launches the fused feed-forward sub-layer is split into (0: fewest that fit) */
+  int32_t block_simt;        /* 1: unfused block passes on the SIMT block GEMV */
+  int32_t slice_mode;        /* unfused linear layers on the row-slice kernel: 0 off, 1 block passes, 2 also single rows */
+  int32_t slice_min_kb;      /* single-row passes: matrices below this size stay on the GEMV */
+  int32_t slice_mma_min;     /* row-slice kernel: row counts from this on use tensor-core tiles (2..5) */
+  int32_t slice_head;        /* tensor-core LM head: 0 off, 1 block passes, 2 also single rows of large heads */
+  int32_t slice_head_min_mb; /* single rows: heads from this size on */
+  int32_t unit_attn;         /* 1: unfused decoder attention on the chunked 256-thread kernel */
+  int32_t umma;              /* 1: tcgen05 kernels (encoder linears; unfused block linears when slice_mode = 0) */
+  int32_t enc_gemm;          /* 1: encoder linears as 128-token tcgen05 GEMM tiles */
+  int32_t enc_attn_mma;      /* 1: encoder self-attention on mma.sync tiles */
+  int32_t enc_parallel;      /* 1: the two encoders run side by side on two streams */
+  int32_t spin_limit;        /* polls before a bounded device-side wait gives up with BILD_ERR_TIMEOUT (0: 2^20) */
+  int32_t debug_skip_copies; /* 1: the fused attention kernel announces its weight copies but does not issue them, so
+                              * that its bounded wait runs out (test of the time-out path; never set in production) */
+} bild_tuning;
+void bild_tuning_default(bild_tuning *t /*HOST out*/);
+/* bild_create with explicit switches; tuning == NULL means the defaults. */
+int bild_create_tuned(const bild_config *cfg, const bild_weights *small_w, const bild_weights *large_w,
+                      void *workspace, size_t workspace_bytes, void *cuda_stream,
+                      const bild_tuning *tuning /*HOST*/, bild_ctx **out);
 void bild_destroy(bild_ctx *ctx); /* frees the host-side context only */
 
 /* Run both encoders over ids[0..n_ids) and project the cross-attention K/V of
@@ -166,8 +198,8 @@ void bild_destroy(bild_ctx *ctx); /* frees the host-side context only */
  * Asynchronous on the stream (ids are copied before returning).  The small model's
  * encoder runs on a stream of the context's own, forked from and joined back into the
  * caller's stream with events, so work queued on the caller's stream after this call still
- * sees both encoders' results (BILD_ENC_SERIAL=1 in the environment keeps everything on the
- * caller's stream). */
+ * sees both encoders' results (bild_tuning.enc_parallel = 0 keeps everything on the caller's
+ * stream). */
 int bild_encode(bild_ctx *ctx, const int32_t *ids /*HOST*/, int n_ids);
 
 /* Reset the decode state only (keeps the encoder results of the last bild_encode). */

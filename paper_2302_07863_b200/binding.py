@@ -22,7 +22,7 @@ FFN_RELU, FFN_GATED_GELU = 0, 1
 MODE_BILD, MODE_SMALL_ONLY, MODE_LARGE_ONLY = 0, 1, 2
 MAX_BLOCK = 16
 
-EXPORTS = ["bild_query_workspace", "bild_create", "bild_destroy", "bild_encode", "bild_reset",
+EXPORTS = ["bild_query_workspace", "bild_create", "bild_create_tuned", "bild_tuning_default", "bild_destroy", "bild_encode", "bild_reset",
            "bild_small_step", "bild_large_verify", "bild_rewind", "bild_generate", "bild_generate_async",
            "bild_fetch_result", "bild_time_pass", "bild_uses_tensor_cores", "bild_launch_count", "bild_last_error", "bild_op_linear",
            "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_op_lm_head_static", "bild_debug_bucket",
@@ -53,6 +53,13 @@ class Weights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("emb", "lm_head", "enc_rel_bias", "dec_rel_bias", "enc_final_ln",
                                           "dec_final_ln")] + [("enc_layers", C.POINTER(EncLayer)),
                                                               ("dec_layers", C.POINTER(DecLayer))]
+
+
+class Tuning(C.Structure):
+    """bild_tuning: kernel selection and debugging switches (defaults from bild_tuning_default)."""
+    _fields_ = [(n, C.c_int32) for n in ("host_loop", "pdl", "fused", "ffn_parts", "block_simt", "slice_mode", "slice_min_kb",
+                                         "slice_mma_min", "slice_head", "slice_head_min_mb", "unit_attn", "umma", "enc_gemm",
+                                         "enc_attn_mma", "enc_parallel", "spin_limit", "debug_skip_copies")]
 
 
 class StepOut(C.Structure):
@@ -89,6 +96,10 @@ def lib() -> C.CDLL:
         L.bild_query_workspace.argtypes = [C.POINTER(Config), C.POINTER(C.c_size_t)]
         L.bild_create.argtypes = [C.POINTER(Config), C.POINTER(Weights), C.POINTER(Weights), vp, C.c_size_t, vp,
                                   C.POINTER(vp)]
+        L.bild_create_tuned.argtypes = [C.POINTER(Config), C.POINTER(Weights), C.POINTER(Weights), vp, C.c_size_t, vp,
+                                        C.POINTER(Tuning), C.POINTER(vp)]
+        L.bild_tuning_default.argtypes = [C.POINTER(Tuning)]
+        L.bild_tuning_default.restype = None
         L.bild_destroy.argtypes = [vp]
         L.bild_destroy.restype = None
         L.bild_encode.argtypes = [vp, C.POINTER(C.c_int32), i32]
@@ -164,7 +175,7 @@ class Context:
     """Owns the workspace tensor and keeps the weight tensors alive; methods mirror the C calls."""
 
     def __init__(self, cfg: Config, small_shape, small_dev: dict, large_shape, large_dev: dict, device="cuda:0",
-                 stream=None):
+                 stream=None, tuning: dict | None = None):
         import torch
         self.L = lib()
         self.cfg = cfg
@@ -180,7 +191,17 @@ class Context:
         sp = stream.cuda_stream if stream is not None else None
         h = C.c_void_p()
         with torch.cuda.device(self.device):
-            rc = self.L.bild_create(C.byref(cfg), C.byref(ws), C.byref(wl), base, nbytes.value, sp, C.byref(h))
+            if tuning:   # bild_tuning: the defaults with the given fields replaced
+                t = Tuning()
+                self.L.bild_tuning_default(C.byref(t))
+                for key, val in tuning.items():
+                    if key not in dict(Tuning._fields_):
+                        raise KeyError(f"bild_tuning has no field {key!r}")
+                    setattr(t, key, int(val))
+                rc = self.L.bild_create_tuned(C.byref(cfg), C.byref(ws), C.byref(wl), base, nbytes.value, sp, C.byref(t),
+                                              C.byref(h))
+            else:
+                rc = self.L.bild_create(C.byref(cfg), C.byref(ws), C.byref(wl), base, nbytes.value, sp, C.byref(h))
         if rc != BILD_OK:
             raise BildError(rc, "bild_create")
         self.h = h

@@ -173,6 +173,9 @@ struct bild_ctx {
   size_t slice_min_bytes = 3000 * 1024;   // single-row passes: smaller matrices stay on the GEMV (measured)
   int fused_on = 2;                  // fused sub-layer kernels where the shapes allow: 0 off, 1 single-row passes, 2 also passes of 2 to 8 rows
   int sub_parts_want = 0;            // 0: fewest launches of the feed-forward sub-layer that fit
+  bool use_umma = true, use_enc_gemm = true;
+  unsigned spin_limit = SPIN_LIMIT;
+  bool debug_skip_copies = false;
   bool capturing = false;            // launches are being recorded into a graph, not run
   int64_t graph_counted = 0;         // launches of the loop graphs already added to `launches`
 };
@@ -544,8 +547,7 @@ enum { TM_QKV = 0, TM_O, TM_CQ, TM_CO, TM_WI0, TM_WI1, TM_FO, TM_CKV, TM_EQKV, T
 // Builds the descriptors of one model; leaves m.umma false when the shapes do not fit the kernel.
 void setup_umma(bild_ctx* c, Model& m) {
   m.umma = false;
-  const char* off = std::getenv("BILD_NO_UMMA");
-  if (off && off[0] == '1') return;
+  if (!c->use_umma) return;
   if (c->cfg.dtype != BILD_BF16) return;
   const bild_model_cfg& mc = m.c;
   if (mc.d_model % UM_KB || m.inner % UM_KB || mc.d_ff % UM_KB) return;
@@ -587,8 +589,7 @@ void setup_umma(bild_ctx* c, Model& m) {
   m.umma = true;
   // encoder GEMM over 128-token tiles
   m.enc_gemm = false;
-  const char* eg = std::getenv("BILD_ENC_GEMM");
-  if (eg && eg[0] == '0') return;
+  if (!c->use_enc_gemm) return;
   const int ecap128 = (c->cfg.max_enc_len + EG_TOK - 1) / EG_TOK * EG_TOK;
   const int Ks[3] = {mc.d_model, m.inner, mc.d_ff};
   for (int pr = 0; pr < 2; ++pr)
@@ -692,6 +693,7 @@ int fused_layers(bild_ctx* c, Model& m, int MB) {
     AttnSubArgs a{};
     a.desc = m.desc; a.eps = mc.ln_eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
     a.kc_keys = m.sub_kc; a.bias_len = m.sub_bias_len; a.mb = MB; a.err = &c->st->err;
+    a.spin = c->spin_limit; a.skip_copies = c->debug_skip_copies ? 1 : 0;
     a.n_keys_dev = c->enc_len_dev;
     // S1-S3 / L1-L3
     a.x_in = m.x; a.x_out = m.xb; a.x_zero = m.xc; a.gain = (const float*)w.ln1;
@@ -707,7 +709,7 @@ int fused_layers(bild_ctx* c, Model& m, int MB) {
     CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
     // S7-S8 / L7-L8
     FfnSubArgs f{};
-    f.desc = m.desc; f.eps = mc.ln_eps; f.d = d; f.F = F; f.gated = gated ? 1 : 0; f.mb = MB;
+    f.desc = m.desc; f.eps = mc.ln_eps; f.d = d; f.F = F; f.gated = gated ? 1 : 0; f.mb = MB; f.spin = c->spin_limit;
     f.err = &c->st->err; f.x_in = m.xc; f.x_out = m.x; f.gain = (const float*)w.ln3;
     f.Wi0 = (const __nv_bfloat16*)w.wi0; f.Wi1 = (const __nv_bfloat16*)w.wi1; f.WfoT = m.wfoT + (size_t)l * F * d;
     f.nparts = m.sub_parts;
@@ -1201,8 +1203,20 @@ int bild_query_workspace(const bild_config* cfg, size_t* bytes) {
   return BILD_OK;
 }
 
+void bild_tuning_default(bild_tuning* t) {
+  if (!t) return;
+  t->host_loop = 0; t->pdl = 1; t->fused = 2; t->ffn_parts = 0; t->block_simt = 0; t->slice_mode = 2;
+  t->slice_min_kb = 3000; t->slice_mma_min = 3; t->slice_head = 2; t->slice_head_min_mb = 32; t->unit_attn = 1;
+  t->umma = 1; t->enc_gemm = 1; t->enc_attn_mma = 1; t->enc_parallel = 1; t->spin_limit = 0; t->debug_skip_copies = 0;
+}
+
 int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_weights* large_w, void* workspace,
                 size_t workspace_bytes, void* cuda_stream, bild_ctx** out) {
+  return bild_create_tuned(cfg, small_w, large_w, workspace, workspace_bytes, cuda_stream, nullptr, out);
+}
+
+int bild_create_tuned(const bild_config* cfg, const bild_weights* small_w, const bild_weights* large_w, void* workspace,
+                      size_t workspace_bytes, void* cuda_stream, const bild_tuning* tuning, bild_ctx** out) {
   if (!out) return BILD_ERR_ARG;
   *out = nullptr;
   std::string why;
@@ -1215,12 +1229,28 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
   c->cfg = *cfg;
   c->stream = (cudaStream_t)cuda_stream;
   c->cnt = &c->launches;
-  const char* hl = std::getenv("BILD_HOST_LOOP");
-  c->host_loop = hl && hl[0] == '1';
-  const char* bs = std::getenv("BILD_BLOCK_SIMT");
-  c->block_simt = bs && bs[0] == '1';
-  const char* sl = std::getenv("BILD_SLICE");
-  if (sl && sl[0] >= '0' && sl[0] <= '2') c->slice_mode = sl[0] - '0';
+  {
+    bild_tuning t;
+    bild_tuning_default(&t);
+    if (tuning) t = *tuning;
+    c->host_loop = t.host_loop != 0;
+    c->use_pdl = t.pdl != 0;
+    c->fused_on = std::min(2, std::max(0, t.fused));
+    c->sub_parts_want = std::min(8, std::max(0, t.ffn_parts));
+    c->block_simt = t.block_simt != 0;
+    c->slice_mode = std::min(2, std::max(0, t.slice_mode));
+    c->slice_min_bytes = (size_t)std::max(0, t.slice_min_kb) * 1024;
+    c->slice_mma_min = std::min(5, std::max(2, t.slice_mma_min));
+    c->slice_head = std::min(2, std::max(0, t.slice_head));
+    c->slice_head_min_bytes = (size_t)std::max(0, t.slice_head_min_mb) << 20;
+    c->unit_attn = t.unit_attn != 0;
+    c->use_umma = t.umma != 0;
+    c->use_enc_gemm = t.enc_gemm != 0;
+    c->enc_attn_mma = t.enc_attn_mma != 0;
+    c->enc_parallel = t.enc_parallel != 0;
+    c->spin_limit = t.spin_limit > 0 ? (unsigned)t.spin_limit : SPIN_LIMIT;
+    c->debug_skip_copies = t.debug_skip_copies != 0;
+  }
   {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
@@ -1228,26 +1258,6 @@ int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_
       c->sms = 0;
     }
   }
-  const char* shm = std::getenv("BILD_SLICE_HEAD_MIN_MB");
-  if (shm) c->slice_head_min_bytes = (size_t)std::max(0, std::atoi(shm)) << 20;
-  const char* shd = std::getenv("BILD_SLICE_HEAD");
-  if (shd && shd[0] >= '0' && shd[0] <= '2') c->slice_head = shd[0] - '0';
-  const char* ea = std::getenv("BILD_ENC_ATTN_MMA");
-  if (ea && ea[0] == '0') c->enc_attn_mma = false;
-  const char* ua = std::getenv("BILD_UNIT_ATTN");
-  if (ua && ua[0] == '0') c->unit_attn = false;
-  const char* mm = std::getenv("BILD_SLICE_MMA_MIN");
-  if (mm) c->slice_mma_min = std::min(5, std::max(2, std::atoi(mm)));
-  const char* es = std::getenv("BILD_ENC_SERIAL");
-  if (es && es[0] == '1') c->enc_parallel = false;
-  const char* sm = std::getenv("BILD_SLICE_MIN_KB");
-  if (sm) c->slice_min_bytes = (size_t)std::atoi(sm) * 1024;
-  const char* fu = std::getenv("BILD_FUSED");
-  if (fu && fu[0] >= '0' && fu[0] <= '2') c->fused_on = fu[0] - '0';
-  const char* fp = std::getenv("BILD_FFN_PARTS");
-  if (fp) c->sub_parts_want = std::min(8, std::max(0, std::atoi(fp)));
-  const char* np = std::getenv("BILD_NO_PDL");
-  c->use_pdl = !(np && np[0] == '1');
   Bump b(workspace);
   plan(c, b);
   c->ws_bytes = b.off;

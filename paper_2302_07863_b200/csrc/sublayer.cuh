@@ -55,11 +55,13 @@ __host__ __device__ inline int sub_up16(int v) { return (v + 15) & ~15; }
 // row stride (floats) of staged keys / values: 16 mod 32, so the four channel quarters of two keys hit 32 distinct banks
 __host__ __device__ inline int sub_kv_stride(int dkv) { return ((dkv + 15) / 32) * 32 + 16; }
 
-__device__ __forceinline__ void sub_wait(SubShared* sh, int* err, unsigned long long* bar, uint32_t parity) {
+// Bounded wait for the weight copies: after `spin` unsuccessful polls the block records BILD_ERR_TIMEOUT for the host
+// and goes on (with whatever the shared memory holds), so that every block of the kernel still leaves.
+__device__ __forceinline__ void sub_wait(SubShared* sh, int* err, unsigned long long* bar, uint32_t parity, unsigned spin) {
   const uint32_t b = smem_u32(bar);
   if (mbar_try(b, parity)) return;
   if (*(volatile int*)&sh->failed) return;
-  for (unsigned it = 0; it < SPIN_LIMIT; ++it)
+  for (unsigned it = 0; it < spin; ++it)
     if (mbar_try(b, parity)) return;
   sh->failed = 1;
   atomicExch(err, (int)BILD_ERR_TIMEOUT);
@@ -178,6 +180,8 @@ struct AttnSubArgs {
   int kc_keys;               // keys per staged chunk (<= 64)
   int bias_len;              // floats reserved for the staged bias
   int mb;                    // token rows the shared memory is sized for
+  unsigned spin;             // polls of the weight barrier before the kernel gives up
+  int skip_copies;           // test of the time-out path: the weight copies are announced but not issued
   int* err;
   AttnSubLayout L;
 };
@@ -257,7 +261,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
   // the copies a warp issues go out one after the other (about 25 ns each), the warps issue side by side
   {
     const int i = ((tid & 31) << 3) | (tid >> 5);
-    if (i < npr) {
+    if (i < npr && !a.skip_copies) {
       const int j = pr0 + i, part = j >> a.dkv_shift, ch = j & (dkv - 1);
       bulk_g2s(smem_u32(sWq + (size_t)i * rowbytes), a.Wp + ((size_t)part * a.I + h * dkv + ch) * d, (uint32_t)(d * 2), smem_u32(&sh->wbar));
     }
@@ -330,7 +334,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
 #pragma unroll 1
   for (int i = tid + SUB_THREADS; i < bias_cnt; i += SUB_THREADS) sBias[i] = __ldg(a.bias + (size_t)h * a.bias_ld + dist_lo + i);
   SUB_STAMP();            // 2: token rows + norm
-  sub_wait(sh, a.err, &sh->wbar, 0);
+  sub_wait(sh, a.err, &sh->wbar, 0, a.spin);
   SUB_STAMP();            // 3: wait for the weights
   // ---- phase A: this rank's q|k|v rows for all token rows -----------------------------------
   if (ONE) sl_items<1>(sWq, rowbytes, npr, d, Xs, xst, psum, warp, lane);
@@ -641,6 +645,7 @@ struct FfnSubArgs {
   int part, nparts;          // this launch covers the slices blockIdx.x * nparts + part of gridDim.x * nparts
   int seed;                  // 1: the blocks add x_in for their share of the columns
   int mb;
+  unsigned spin;             // polls of the weight barrier before the kernel gives up
   int* err;
   FfnSubLayout L;
 };
@@ -737,7 +742,7 @@ __global__ void __launch_bounds__(SUB_THREADS) ffn_sub_kernel(const FfnSubArgs a
   const float inv1 = sub_load_rows<ONE>(a.x_in, k, d, g4, a.eps, Xs, xst, sh, sSeed, su0 * 4, su1 * 4, tid, lane, warp);
   SUB_STAMP();            // 2: token rows + norm
   {
-    if (nf > 0) sub_wait(sh, a.err, &sh->wbar, 0);
+    if (nf > 0) sub_wait(sh, a.err, &sh->wbar, 0, a.spin);
     SUB_STAMP();          // 3: wait for the weights
     // hidden activations of the slice
     if (ONE) sl_items<1>(sWi, rowbytes, nrows, d, Xs, xst, psum, warp, lane);

@@ -7,7 +7,7 @@ from .binding import BF16, FP32, Config, Context, model_cfg, upload_model
 
 
 def make_context(workload: str, scale_small: float, scale_large: float, device="cuda:0", max_enc_len=None,
-                 max_dec_len=None, eos_id=-1, max_draft=None):
+                 max_dec_len=None, eos_id=-1, max_draft=None, tuning=None):
     """Generate the workload's two models on the host, upload them, create a Context.
     Returns (context, encoder ids, workload)."""
     wl = WORKLOADS[workload]
@@ -16,5 +16,5 @@ def make_context(workload: str, scale_small: float, scale_large: float, device="
     devL = upload_model(gen_model(sL, wl.seed, wl.dtype), device)
     cfg = Config(model_cfg(sS, scale_small), model_cfg(sL, scale_large), BF16 if wl.dtype == "bf16" else FP32,
                  max_enc_len or wl.enc_len, max_dec_len or wl.gen_len + 1, max_draft or wl.max_draft, 0, eos_id)
-    ctx = Context(cfg, sS, devS, sL, devL, device)
+    ctx = Context(cfg, sS, devS, sL, devL, device, tuning=tuning)
     return ctx, gen_ids(sS.vocab, wl.enc_len, wl.seed), wl

@@ -225,7 +225,7 @@ def test_steps_match_oracle_logits(torch_cuda, name):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("fused", ["1", "2", "0"])
+@pytest.mark.parametrize("fused", [1, 2, 0])
 def test_heads_of_64_channels_all_block_sizes(torch_cuda, fused):
     """Heads of 64 channels (the T5 / mT5 head size) at sizes the oracle runs live: single-row steps, blocks of 2 to 16
     rows (both thread counts of the attention kernel, every epilogue turn of the row-slice linear), a self cache that
@@ -234,11 +234,8 @@ def test_heads_of_64_channels_all_block_sizes(torch_cuda, fused):
     from paper_2302_07863_b200.synthetic import make_context
     name, scS, scL = "wide_bf16", 9.0, 11.0
     wl = WORKLOADS[name]
-    os.environ["BILD_FUSED"] = fused   # fused sub-layer kernels: single-row passes only / also 2 to 8 rows / off
-    try:
-        ctx, ids, _ = make_context(name, scS, scL)
-    finally:
-        del os.environ["BILD_FUSED"]
+    # fused sub-layer kernels: single-row passes only / also 2 to 8 rows / off
+    ctx, ids, _ = make_context(name, scS, scL, tuning=dict(fused=fused))
     ctx.encode(ids)
     S = Model(MODEL_SHAPES[wl.small], gen_model(MODEL_SHAPES[wl.small], wl.seed, wl.dtype), scS)
     L = Model(MODEL_SHAPES[wl.large], gen_model(MODEL_SHAPES[wl.large], wl.seed, wl.dtype), scL)
@@ -343,27 +340,24 @@ def test_generate_matches_live_oracle(torch_cuda, name, alpha_fb, alpha_rb, max_
         assert got["stats"] == want["stats"]
 
 
-@pytest.mark.parametrize("env", ["BILD_FUSED=0,BILD_BLOCK_SIMT=1", "BILD_HOST_LOOP=1", "BILD_NO_PDL=1", "BILD_NO_UMMA=1",
-                                 "BILD_FUSED=0", "BILD_FUSED=1", "BILD_FFN_PARTS=2",
-                                 "BILD_FUSED=0,BILD_SLICE=0", "BILD_FUSED=0,BILD_SLICE=2", "BILD_FUSED=0,BILD_SLICE_MMA_MIN=5",
-                                 "BILD_FUSED=0,BILD_UNIT_ATTN=0", "BILD_FUSED=0,BILD_SLICE_HEAD=0",
-                                 "BILD_SLICE_HEAD=1", "BILD_ENC_GEMM=0", "BILD_ENC_SERIAL=1"])
+ALT_PATHS = [dict(fused=0, block_simt=1), dict(host_loop=1), dict(pdl=0), dict(umma=0), dict(fused=0), dict(fused=1),
+             dict(ffn_parts=2), dict(fused=0, slice_mode=0), dict(fused=0, slice_mode=2, slice_min_kb=0),
+             dict(fused=0, slice_mma_min=5), dict(fused=0, unit_attn=0), dict(fused=0, slice_head=0), dict(slice_head=1),
+             dict(slice_head=2, slice_head_min_mb=0), dict(enc_gemm=0), dict(enc_parallel=0), dict(enc_attn_mma=0),
+             dict(fused=0, host_loop=1)]
+
+
+@pytest.mark.parametrize("tuning", ALT_PATHS, ids=lambda t: ",".join(f"{k}={v}" for k, v in t.items()))
 @pytest.mark.parametrize("name", ["tiny_bf16", "odd"])
-def test_alternative_paths_match_golden(torch_cuda, name, env):
-    """The switchable paths (fused sub-layer kernels off / also for block passes / feed-forward in two launches, SIMT
-    block GEMV, host-driven loop, plain launches, no tcgen05 kernels, row-slice kernel off / also for single rows,
-    SIMT items up to 4 rows, earlier attention kernel, earlier block head, tensor-core head for single rows, encoder
-    on the 16-row kernel) give the same tokens and trace as the stored oracle run."""
+def test_alternative_paths_match_golden(torch_cuda, name, tuning):
+    """The switchable paths (bild_tuning: fused sub-layer kernels off / single-row passes only / feed-forward in two
+    launches, SIMT block GEMV, host-driven loop, plain launches, no tcgen05 kernels, row-slice kernel off / also for small
+    matrices, SIMT items up to 4 rows, earlier attention kernel, earlier block head, tensor-core head for single rows,
+    encoder on the 16-row kernel / on one stream / SIMT attention) give the same tokens and trace as the stored oracle run."""
     from paper_2302_07863_b200 import MODE_BILD
     from paper_2302_07863_b200.synthetic import make_context
     g = golden(name)
-    envs = dict(e.split("=") for e in env.split(","))
-    os.environ.update(envs)
-    try:
-        ctx, ids, wl = make_context(name, g["scale_small"]["scale"], g["scale_large"]["scale"])
-    finally:
-        for e in envs:
-            del os.environ[e]
+    ctx, ids, wl = make_context(name, g["scale_small"]["scale"], g["scale_large"]["scale"], tuning=tuning)
     ctx.encode(ids)
     th = g["thresholds"]
     r = ctx.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)
@@ -372,6 +366,40 @@ def test_alternative_paths_match_golden(torch_cuda, name, env):
     assert r["stats"] == g["bild"]["stats"]
     assert ctx.launch_count() > 0
     ctx.close()
+
+
+def test_bounded_wait_runs_out_and_context_recovers(torch_cuda):
+    """Time-out path of the device-side waits: with bild_tuning.debug_skip_copies the fused attention kernel announces its
+    weight copies to the barrier but does not issue them, so the bounded wait (a short limit here) runs out in every block.
+    The kernels must all leave, the call must report BILD_ERR_TIMEOUT, and after bild_encode the context must work again
+    (the same switch cannot be cleared, so a second context with the same weights checks the numbers)."""
+    from paper_2302_07863_b200 import BildError, MODE_BILD
+    from paper_2302_07863_b200.synthetic import make_context
+    g = golden("tiny_bf16")
+    ctx, ids, wl = make_context("tiny_bf16", g["scale_small"]["scale"], g["scale_large"]["scale"],
+                                tuning=dict(debug_skip_copies=1, spin_limit=200))
+    ctx.encode(ids)
+    with pytest.raises(BildError) as e:
+        ctx.small_step(0, 0.4)
+    assert e.value.code == -6                      # BILD_ERR_TIMEOUT
+    with pytest.raises(BildError) as e:
+        ctx.large_verify([0, 5, 7], 10.0)
+    assert e.value.code == -6
+    ctx.encode(ids)                                # clears the error; the set-up kernels are not affected by the switch
+    S, L, _ = get_oracle("tiny_bf16")
+    st = S.start(ids, 8)
+    for which, what, ref in ((0, 0, st.ck[0]), (0, 1, st.cv[0])):
+        sh = MODEL_SHAPES[wl.small]
+        got = ctx.read_cache(which, what, 0, sh.n_heads, wl.enc_len, sh.d_kv)[:, :len(ids), :]
+        want = ref.reshape(len(ids), sh.n_heads, sh.d_kv).transpose(1, 0, 2)
+        assert float(np.max(np.abs(got - want))) <= 2e-3
+    ctx.close()
+    # the device and the library are unharmed: a regular context reproduces the stored run
+    ctx2, ids, wl = make_context("tiny_bf16", g["scale_small"]["scale"], g["scale_large"]["scale"])
+    ctx2.encode(ids)
+    th = g["thresholds"]
+    assert ctx2.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)["tokens"] == g["bild"]["tokens"]
+    ctx2.close()
 
 
 def test_eos_and_limits(torch_cuda):
