@@ -266,8 +266,10 @@ int64_t bild_launch_count(const bild_ctx *ctx);
 const char *bild_last_error(const bild_ctx *ctx); /* HOST string owned by the context */
 
 /* ---- single operations (for unit tests and micro-benchmarks) -------------------
- * Each is the kernel the decode path uses, run once on the given stream, with every
- * pointer DEVICE unless said otherwise; no synchronisation. */
+ * One kernel (or one sub-layer) run once on the given stream, every pointer DEVICE unless said
+ * otherwise.  bild_op_linear and bild_op_lm_head run the per-operation kernels (GEMV / SIMT linear,
+ * single-row and SIMT heads) that fp32 configurations and odd shapes use; bild_op_lm_head_sliced,
+ * bild_op_attn_sublayer and bild_op_ffn_sublayer run the kernels the bf16 decoder passes use. */
 
 /* Y[m][n] = sum_j W[n][j] * H[m][j], H = X if gain == NULL, else the RMS norm of X
  * with that gain (Section 3.2's model forward; one weight pass serves all m rows).
@@ -286,6 +288,37 @@ int bild_op_lm_head(const void *W, int w_dtype, const float *X, const float *gai
                     float scale, const int32_t *target, int M, int V, int K,
                     int32_t *argmax_out, float *max_out, float *lse_out, float *gather_out,
                     float *logits_dbg, void *scratch, void *cuda_stream);
+
+/* The same fused head on the tensor-core kernel of the bf16 decoder passes (one block per SM, the
+ * vocabulary streamed through shared memory by bulk copies): W bf16 [V][K], 16-byte aligned;
+ * K * (3 * tile rows * 2 + 64) bytes must fit a block (K <= 2048), else BILD_ERR_CAPACITY.
+ * scratch as for bild_op_lm_head.  Asynchronous on the stream. */
+int bild_op_lm_head_sliced(const void *W, const float *X, const float *gain, float eps, float scale,
+                           const int32_t *target, int M, int V, int K, int32_t *argmax_out,
+                           float *max_out, float *lse_out, float *gather_out, float *logits_dbg,
+                           void *scratch, void *cuda_stream);
+
+/* One decoder sub-layer on the fused kernels of the bf16 passes (Section 3.2's model forward, one
+ * weight pass for all M rows; steps S1-S3 / S4-S6 / S7-S8 of the small step, L1-L8 of the block
+ * pass): x_out = x_in + SubLayer(rms_norm(x_in) * gain).  1 <= M <= 8; x_in, x_out fp32 [M][d];
+ * all weights bf16, row-major [out][in], 16-byte aligned.  scratch: bild_op_sublayer_scratch_bytes(d, F)
+ * bytes (F = 0 for attention), 256-byte aligned.  Both calls synchronise the stream before returning
+ * and return BILD_ERR_TIMEOUT if a bounded wait inside the kernel ran out; BILD_ERR_ARG for shapes the
+ * fused kernels do not take (d <= 1024, d_kv in {16, 32, 64}, ...).
+ *   attention: self != 0: Wp = [3 H d_kv][d] (q, k, v rows); the M rows sit at positions n_before ..
+ *     n_before + M - 1, attend causally over the n_before cached rows of kc / vc ([H][cap][d_kv] fp32)
+ *     and themselves, with bias_by_dist [H][cap] added by distance; their keys / values are appended to
+ *     kc / vc.  self == 0: Wp = [H d_kv][d]; the rows attend over the n_before rows of kc / vc.
+ *   feed-forward: Wi0 (and the GELU gate Wi1, or NULL for ReLU) [F][d], Wfo [d][F]; `parts` = launches
+ *     the slice of d_ff per block is split over (0: fewest that fit). */
+size_t bild_op_sublayer_scratch_bytes(int d, int F);
+int bild_op_attn_sublayer(int self, const void *Wp, const void *Wo, const float *gain, float eps,
+                          const float *x_in, float *x_out, float *kc, float *vc, int cap, int n_before,
+                          const float *bias_by_dist, int M, int d, int H, int dkv, void *scratch,
+                          void *cuda_stream);
+int bild_op_ffn_sublayer(const void *Wi0, const void *Wi1, const void *Wfo, const float *gain, float eps,
+                         const float *x_in, float *x_out, int M, int d, int F, int parts, void *scratch,
+                         void *cuda_stream);
 
 /* The paper has no counterpart for this call; it exists for callers that cannot allocate.
  * Same computation and outputs as bild_op_lm_head, but the kernel's scratch (block

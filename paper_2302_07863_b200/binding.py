@@ -26,7 +26,8 @@ EXPORTS = ["bild_query_workspace", "bild_create", "bild_create_tuned", "bild_tun
            "bild_small_step", "bild_large_verify", "bild_rewind", "bild_generate", "bild_generate_async",
            "bild_fetch_result", "bild_time_pass", "bild_uses_tensor_cores", "bild_launch_count", "bild_last_error", "bild_op_linear",
            "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_op_lm_head_static", "bild_debug_bucket",
-           "bild_debug_read_cache"]
+           "bild_debug_read_cache", "bild_op_lm_head_sliced", "bild_op_sublayer_scratch_bytes", "bild_op_attn_sublayer",
+           "bild_op_ffn_sublayer"]
 
 
 class ModelCfg(C.Structure):
@@ -322,6 +323,71 @@ def op_lm_head(W, X, gain, eps, scale, target, M, V, K, want_logits=False, strea
     if rc != BILD_OK:
         raise BildError(rc, "bild_op_lm_head")
     return am, mx, lse, ga, lg
+
+
+def op_lm_head_sliced(W, X, gain, eps, scale, target, M, V, K, want_logits=False):
+    """bild_op_lm_head_sliced: the tensor-core head of the bf16 decoder passes (bf16 weights only)."""
+    import torch
+    dev = X.device
+    L = lib()
+    L.bild_op_lm_head_scratch_bytes.restype = C.c_size_t
+    nb = L.bild_op_lm_head_scratch_bytes(V)
+    scratch = torch.zeros(nb + 512, dtype=torch.uint8, device=dev)
+    sp = (scratch.data_ptr() + 255) // 256 * 256
+    am = torch.empty(M, dtype=torch.int32, device=dev)
+    mx = torch.empty(M, dtype=torch.float32, device=dev)
+    lse = torch.empty(M, dtype=torch.float32, device=dev)
+    ga = torch.zeros(M, dtype=torch.float32, device=dev)
+    lg = torch.empty((M, V), dtype=torch.float32, device=dev) if want_logits else None
+    vp = C.c_void_p
+    L.bild_op_lm_head_sliced.argtypes = [vp, vp, vp, C.c_float, C.c_float, vp, C.c_int, C.c_int, C.c_int, vp, vp, vp, vp, vp, vp, vp]
+    rc = L.bild_op_lm_head_sliced(W.data_ptr(), X.data_ptr(), gain.data_ptr() if gain is not None else None, eps, scale,
+                                  target.data_ptr() if target is not None else None, M, V, K, am.data_ptr(), mx.data_ptr(),
+                                  lse.data_ptr(), ga.data_ptr(), lg.data_ptr() if lg is not None else None, sp, None)
+    if rc != BILD_OK:
+        raise BildError(rc, "bild_op_lm_head_sliced")
+    return am, mx, lse, ga, lg
+
+
+def _sub_scratch(d, F, dev):
+    import torch
+    L = lib()
+    L.bild_op_sublayer_scratch_bytes.restype = C.c_size_t
+    L.bild_op_sublayer_scratch_bytes.argtypes = [C.c_int, C.c_int]
+    scratch = torch.zeros(L.bild_op_sublayer_scratch_bytes(d, F) + 256, dtype=torch.uint8, device=dev)
+    return scratch, (scratch.data_ptr() + 255) // 256 * 256
+
+
+def op_ffn_sublayer(Wi0, Wi1, Wfo, gain, eps, x_in, M, d, F, parts=0):
+    """x_in + FFN(rms_norm(x_in)) on the fused feed-forward kernel; returns x_out [M][d]."""
+    import torch
+    scratch, sp = _sub_scratch(d, F, x_in.device)
+    x_out = torch.empty((M, d), dtype=torch.float32, device=x_in.device)
+    vp = C.c_void_p
+    L = lib()
+    L.bild_op_ffn_sublayer.argtypes = [vp, vp, vp, vp, C.c_float, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
+    rc = L.bild_op_ffn_sublayer(Wi0.data_ptr(), Wi1.data_ptr() if Wi1 is not None else None, Wfo.data_ptr(), gain.data_ptr(), eps,
+                                x_in.data_ptr(), x_out.data_ptr(), M, d, F, parts, sp, None)
+    if rc != BILD_OK:
+        raise BildError(rc, "bild_op_ffn_sublayer")
+    return x_out
+
+
+def op_attn_sublayer(self_attn, Wp, Wo, gain, eps, x_in, kc, vc, cap, n_before, bias, M, d, H, dkv):
+    """x_in + W_o Attention(...) on the fused attention kernel; kc / vc [H][cap][dkv] fp32 (appended to for self-attention)."""
+    import torch
+    scratch, sp = _sub_scratch(d, 0, x_in.device)
+    x_out = torch.empty((M, d), dtype=torch.float32, device=x_in.device)
+    vp = C.c_void_p
+    L = lib()
+    L.bild_op_attn_sublayer.argtypes = [C.c_int, vp, vp, vp, C.c_float, vp, vp, vp, vp, C.c_int, C.c_int, vp, C.c_int, C.c_int,
+                                        C.c_int, C.c_int, vp, vp]
+    rc = L.bild_op_attn_sublayer(1 if self_attn else 0, Wp.data_ptr(), Wo.data_ptr(), gain.data_ptr(), eps, x_in.data_ptr(),
+                                 x_out.data_ptr(), kc.data_ptr(), vc.data_ptr(), cap, n_before,
+                                 bias.data_ptr() if bias is not None else None, M, d, H, dkv, sp, None)
+    if rc != BILD_OK:
+        raise BildError(rc, "bild_op_attn_sublayer")
+    return x_out
 
 
 def op_lm_head_static(W, X, gain, eps, scale, target, M, V, K, stream=None):

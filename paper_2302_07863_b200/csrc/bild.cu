@@ -1551,6 +1551,154 @@ int bild_op_lm_head(const void* W, int w_dtype, const float* X, const float* gai
   return e == cudaSuccess ? BILD_OK : BILD_ERR_CUDA;
 }
 
+// ---- single operations on the hot kernels of the decoder passes ---------------------------------
+namespace {
+struct OpScratch {          // carved from the caller's scratch, 256-byte aligned pieces
+  CallDesc* desc; int* err; int* nkeys; float* zero; char* rest;
+};
+OpScratch op_scratch(void* scratch, int d) {
+  char* p = (char*)scratch;
+  OpScratch o;
+  o.desc = (CallDesc*)p; p += align_up(sizeof(CallDesc), 256);
+  o.err = (int*)p; o.nkeys = (int*)(p + 4); p += 256;
+  o.zero = (float*)p; p += align_up((size_t)MAXB * d * sizeof(float), 256);
+  o.rest = p;
+  return o;
+}
+int op_sms() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return sms;
+}
+int op_finish(cudaStream_t s, const OpScratch& o) {   // the kernels' own error flag (bounded waits) after the call
+  int err = 0;
+  if (cudaMemcpyAsync(&err, o.err, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess)
+    return BILD_ERR_CUDA;
+  return err;
+}
+}  // namespace
+
+size_t bild_op_sublayer_scratch_bytes(int d, int F) {
+  return align_up(sizeof(CallDesc), 256) + 256 + align_up((size_t)MAXB * std::max(d, 8) * sizeof(float), 256) +
+         align_up((size_t)std::max(F, 0) * d * 2, 256) + 256;
+}
+
+int bild_op_ffn_sublayer(const void* Wi0, const void* Wi1, const void* Wfo, const float* gain, float eps, const float* x_in,
+                         float* x_out, int M, int d, int F, int parts, void* scratch, void* cuda_stream) {
+  if (!Wi0 || !Wfo || !gain || !x_in || !x_out || !scratch) return BILD_ERR_ARG;
+  if (M < 1 || M > SUB_MB || d < 8 || d % 8 || d > 1024 || F < 8 || F % 8 || parts < 0 || parts > 8) return BILD_ERR_ARG;
+  if ((uintptr_t)scratch % 256) return BILD_ERR_WORKSPACE;
+  const int sms = op_sms();
+  if (sms < 1) return BILD_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const bool gated = Wi1 != nullptr;
+  const int MB = M == 1 ? 1 : SUB_MB, nmat = gated ? 2 : 1;
+  int smem_max = 0, dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return BILD_ERR_CUDA;
+  int np = std::max(1, parts);
+  while (np <= 8 && (ffn_sub_rows(F, sms * np) * nmat > SUB_MAX_ROWS || ffn_sub_rows(F, sms * np) > SUB_FO_REGS ||
+                     ffn_sub_layout(d, F, gated, sms * np, sms, MB).total > smem_max)) ++np;
+  if (np > 8) return BILD_ERR_CAPACITY;
+  OpScratch o = op_scratch(scratch, d);
+  __nv_bfloat16* WfoT = (__nv_bfloat16*)o.rest;
+  bild_ctx tmp;
+  tmp.stream = s;
+  tmp.use_pdl = false;
+  TokList t{};
+  set_desc_at_kernel<<<1, 1, 0, s>>>(o.desc, M, 0, t);
+  if (cudaMemsetAsync(o.err, 0, 8, s) != cudaSuccess) return BILD_ERR_CUDA;
+  if (cudaMemsetAsync(x_out, 0, (size_t)M * d * sizeof(float), s) != cudaSuccess) return BILD_ERR_CUDA;   // the kernel accumulates into it
+  transpose_bf16_kernel<<<dim3((F + 31) / 32, (d + 31) / 32), dim3(32, 8), 0, s>>>((const __nv_bfloat16*)Wfo, WfoT, d, F);
+  auto kern = MB == 1 ? ffn_sub_kernel<true> : ffn_sub_kernel<false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess) return BILD_ERR_CUDA;
+  FfnSubArgs f{};
+  f.desc = o.desc; f.eps = eps; f.d = d; f.F = F; f.gated = gated ? 1 : 0; f.mb = MB; f.spin = SPIN_LIMIT; f.err = o.err;
+  f.x_in = x_in; f.x_out = x_out; f.gain = gain; f.Wi0 = (const __nv_bfloat16*)Wi0; f.Wi1 = (const __nv_bfloat16*)Wi1; f.WfoT = WfoT;
+  f.nparts = np; f.L = ffn_sub_layout(d, F, gated, sms * np, sms, MB);
+  for (int p = 0; p < np; ++p) {
+    f.part = p; f.seed = p == 0 ? 1 : 0; f.x_zero = p == 0 ? o.zero : nullptr;
+    if (launch_sub(&tmp, kern, sms, 1, (size_t)f.L.total, f) != cudaSuccess) return BILD_ERR_CUDA;
+  }
+  return op_finish(s, o);
+}
+
+int bild_op_attn_sublayer(int self, const void* Wp, const void* Wo, const float* gain, float eps, const float* x_in, float* x_out,
+                          float* kc, float* vc, int cap, int n_before, const float* bias_by_dist, int M, int d, int H, int dkv,
+                          void* scratch, void* cuda_stream) {
+  if (!Wp || !Wo || !gain || !x_in || !x_out || !kc || !vc || !scratch || (self && !bias_by_dist)) return BILD_ERR_ARG;
+  if (M < 1 || M > SUB_MB || H < 1 || cap < 1 || n_before < 0) return BILD_ERR_ARG;
+  if (self ? n_before + M > cap : (n_before < 1 || n_before > cap)) return BILD_ERR_CAPACITY;
+  if ((uintptr_t)scratch % 256) return BILD_ERR_WORKSPACE;
+  const int sms = op_sms();
+  if (sms < 1) return BILD_ERR_CUDA;
+  int C = 8;
+  while (C > 1 && (H * C > sms || d % (4 * C))) C >>= 1;
+  if (d % (4 * C) || d > 1024 || d % 8 || dkv > 64 || dkv < 16 || (dkv & (dkv - 1)) || d / C > SUB_THREADS / 2 ||
+      (3 * dkv + C - 1) / C > SUB_MAX_ROWS) return BILD_ERR_ARG;   // shapes the fused kernel does not take
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int MB = M == 1 ? 1 : SUB_MB, I = H * dkv, P = self ? 3 : 1;
+  int smem_max = 0, dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return BILD_ERR_CUDA;
+  int kc_keys = std::min(64, ((cap + C - 1) / C + 15) / 16 * 16);
+  const int bias_len = ((cap + C - 1) / C + MAXB + 8 + 3) / 4 * 4;
+  while (kc_keys > 16 && attn_sub_layout(d, dkv, P, C, MB, kc_keys, bias_len).total > smem_max) kc_keys -= 16;
+  if (attn_sub_layout(d, dkv, P, C, MB, kc_keys, bias_len).total > smem_max) return BILD_ERR_CAPACITY;
+  OpScratch o = op_scratch(scratch, d);
+  bild_ctx tmp;
+  tmp.stream = s;
+  tmp.use_pdl = false;
+  TokList t{};
+  set_desc_at_kernel<<<1, 1, 0, s>>>(o.desc, M, self ? n_before : 0, t);
+  if (cudaMemsetAsync(o.err, 0, 4, s) != cudaSuccess) return BILD_ERR_CUDA;
+  if (cudaMemcpyAsync(o.nkeys, &n_before, sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess) return BILD_ERR_CUDA;
+  if (cudaMemsetAsync(x_out, 0, (size_t)M * d * sizeof(float), s) != cudaSuccess) return BILD_ERR_CUDA;   // the kernel accumulates into it
+  auto kern = MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess) return BILD_ERR_CUDA;
+  AttnSubArgs a{};
+  a.desc = o.desc; a.eps = eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
+  a.kc_keys = kc_keys; a.bias_len = bias_len; a.mb = MB; a.err = o.err; a.spin = SPIN_LIMIT; a.skip_copies = 0;
+  a.n_keys_dev = o.nkeys; a.x_in = x_in; a.x_out = x_out; a.x_zero = o.zero; a.gain = gain;
+  a.Wp = (const __nv_bfloat16*)Wp; a.Wo = (const __nv_bfloat16*)Wo; a.kc = kc; a.vc = vc; a.cap = cap;
+  a.bias = bias_by_dist; a.bias_ld = cap; a.self = self ? 1 : 0;
+  a.L = attn_sub_layout(d, dkv, P, C, MB, kc_keys, bias_len);
+  if (launch_sub(&tmp, kern, H * C, C, (size_t)a.L.total, a) != cudaSuccess) return BILD_ERR_CUDA;
+  return op_finish(s, o);
+}
+
+int bild_op_lm_head_sliced(const void* W, const float* X, const float* gain, float eps, float scale, const int32_t* target, int M,
+                           int V, int K, int32_t* argmax_out, float* max_out, float* lse_out, float* gather_out, float* logits_dbg,
+                           void* scratch, void* cuda_stream) {
+  if (!W || !X || !scratch || !argmax_out || !max_out || !lse_out) return BILD_ERR_ARG;
+  if (M < 1 || M > MAXB || V < 1 || K < 8 || K % 8 || ((uintptr_t)W & 15)) return BILD_ERR_ARG;
+  if ((uintptr_t)scratch % 256) return BILD_ERR_WORKSPACE;
+  const int sms = op_sms();
+  if (sms < 1 || sms > MAX_GRID_SM) return BILD_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int tr = (M == 1 && K <= 512) ? 32 : 16;
+  const size_t smem = slice_head_smem_bytes(K, tr);
+  if (smem > 200 * 1024) return BILD_ERR_CAPACITY;
+  char* p = (char*)scratch;
+  HeadArgs h{};
+  h.partials = (Partial*)p;
+  p += align_up(head_partial_count(V) * sizeof(Partial), 256);
+  h.counter = (unsigned*)p;
+  int* err = (int*)(p + 8);
+  p += 256;
+  h.out = (HeadOut*)p;
+  if (cudaMemsetAsync(h.counter, 0, 16, s) != cudaSuccess) return BILD_ERR_CUDA;
+  h.W = W; h.X = X; h.ldx = K; h.gain = gain; h.eps = eps; h.scale = scale; h.V = V; h.K = K; h.M = M;
+  h.target = target; h.logits_dbg = logits_dbg; h.which = 1;
+  if (cudaFuncSetAttribute(slice_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) return BILD_ERR_CUDA;
+  slice_head_kernel<<<sms, SH_THREADS, smem, s>>>(h, err, tr);
+  if (cudaGetLastError() != cudaSuccess) return BILD_ERR_CUDA;
+  const HeadOut* o = h.out;
+  cudaError_t e = cudaMemcpyAsync(argmax_out, o->argmax, M * sizeof(int), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(max_out, o->zmax, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(lse_out, o->lse, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess && gather_out && target) e = cudaMemcpyAsync(gather_out, o->gather, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
+  return e == cudaSuccess ? BILD_OK : BILD_ERR_CUDA;
+}
+
 int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, float* ms_per_pass) {
   if (!c || !ms_per_pass || (which != 0 && which != 1)) return fail(c, BILD_ERR_ARG, "null argument / which");
   if (!c->encoded) return fail(c, BILD_ERR_STATE, "bild_encode has not been called");
