@@ -15,7 +15,13 @@ where the paper is loose (each is a deliberate choice):
 * rollback iff d > alpha_RB (Eq. 3, strict), at the smallest such position;
 * only the pending, not yet verified small-model tokens are scanned; a token
   emitted by the large model is never re-judged;
-* sample() is arg-max with the lowest index on ties (greedy decoding);
+* sample() is arg-max with the lowest index on ties (greedy decoding), or, for the
+  sampling variant of the supplementary material ("BiLD with Sampling"), nucleus
+  sampling from both models with the same two policies: the fallback test still uses
+  the small model's maximum probability, the rollback distance is still -ln p_L of
+  the token the small model drew.  The uniform numbers are INPUTS (one per model and
+  output position: a token drawn again for the same position after a rollback uses
+  the same number), so a run is a deterministic function of its arguments;
 * the small model keeps at most `max_draft` tokens in a row (supplementary
   material, "maximum generation length of the small model"): once that many
   drafts are pending, the next small step still runs but control goes to the
@@ -53,9 +59,36 @@ def max_prob(z: np.ndarray):
     return t, 1.0 / sumexp, zmax + math.log(sumexp), zmax - second
 
 
+def nucleus_sample(z: np.ndarray, top_p: float, u: float):
+    """Nucleus (top-p) sampling of one token from softmax(z) with the uniform number u in [0, 1).
+
+    The tokens are put in order of decreasing probability (equal probabilities: lower index first); the
+    nucleus is the shortest prefix of that order whose probabilities add up to at least top_p; the drawn token
+    is the first of the prefix at which the running sum exceeds u times the prefix's total (inverse CDF of the
+    renormalised prefix).  Returns (token, nucleus size, margin), margin = how close (in probability) the two
+    threshold comparisons came to going the other way."""
+    zmax = float(np.max(z))
+    e = np.exp(z - zmax)
+    p = e / float(np.sum(e))
+    order = np.argsort(-p, kind="stable")
+    c = np.cumsum(p[order])
+    hit = np.nonzero(c >= top_p)[0]
+    n = int(hit[0]) + 1 if hit.size else int(z.size)            # rounding may keep the total just below 1
+    target = u * float(c[n - 1])
+    i = int(np.searchsorted(c[:n], target, side="right"))       # first running sum > target
+    i = min(i, n - 1)
+    near = [abs(float(c[n - 1]) - top_p), abs(float(c[i]) - target)]
+    if n > 1:
+        near.append(abs(float(c[n - 2]) - top_p))
+    if i > 0:
+        near.append(abs(float(c[i - 1]) - target))
+    return int(order[i]), n, min(near)
+
+
 def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: float,
              max_len: int, max_draft: int = 10, mode: str = "bild",
-             start_id: int = 0, eos_id: int = -1, keep_logits: bool = False):
+             start_id: int = 0, eos_id: int = -1, keep_logits: bool = False,
+             top_p: float = 0.0, u_small=None, u_large=None):
     """Run Algorithm 1.  Returns a dict with
     tokens  : y[1..n] (the start symbol is not included),
     trace   : list of (kind, pos, token, k, m, value),
@@ -66,7 +99,18 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
               per trace record: the margins of the decisions that produced that
               record (inf where the record did not depend on such a decision),
     logits  : (if keep_logits) list of ("S"|"L", first position, array).
+
+    top_p > 0 selects the sampling variant: every token is drawn by nucleus_sample with u_small[pos] (small
+    model) or u_large[pos] (large model), pos = the position in y the token is written to; the trace margins
+    then carry a fourth entry, the sampling margin of the record's token (in probability).
     """
+    sampling = top_p > 0.0
+
+    def pick(z, arg, u):   # the token a model emits: arg-max, or a draw
+        if not sampling:
+            return arg, math.inf
+        tok, _, near = nucleus_sample(z, top_p, float(u))
+        return tok, near
     assert mode in ("bild", "small", "large")
     cap = max_len + 1
     stS = small.start(enc_ids, cap) if mode != "large" else None
@@ -87,11 +131,14 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
             if keep_logits:
                 logits.append(("S", n, zS.copy()))
             t, pmax, _, gap = max_prob(zS)
+            t, smg = pick(zS, t, u_small[n + 1] if sampling else 0.0)
+            if sampling:
+                gap = math.inf                                      # no arg-max decision is taken
             if mode == "small":
                 mg["argmax"] = min(mg["argmax"], gap)
                 y.append(t); n += 1
                 trace.append((KIND_SMALL_ACCEPT, n, t, 0, -1, pmax))
-                tmg.append((gap, math.inf, math.inf))
+                tmg.append((gap, math.inf, math.inf) + ((smg,) if sampling else ()))
                 continue
             mg["fallback"] = min(mg["fallback"], abs(pmax - alpha_fb))
             confident = not (pmax < alpha_fb)                       # Section 3.3
@@ -99,7 +146,7 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
                 mg["argmax"] = min(mg["argmax"], gap)
                 y.append(t); n += 1; drafts += 1
                 trace.append((KIND_SMALL_ACCEPT, n, t, 0, -1, pmax))
-                tmg.append((gap, abs(pmax - alpha_fb), math.inf))
+                tmg.append((gap, abs(pmax - alpha_fb), math.inf) + ((smg,) if sampling else ()))
                 continue
             if confident:
                 stats["forced"] += 1
@@ -107,7 +154,7 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
             else:
                 stats["fallbacks"] += 1
                 trace.append((KIND_FALLBACK, n + 1, t, 0, -1, pmax))
-            tmg.append((gap, abs(pmax - alpha_fb), math.inf))   # the record names the rejected candidate
+            tmg.append((gap, abs(pmax - alpha_fb), math.inf) + ((smg,) if sampling else ()))   # the record names the rejected candidate
         # ---- the large model reads every token it has not seen yet ----------
         k = n - L_len + 1
         ZL = large.forward_block(stL, y[L_len:n + 1])              # Alg. 1: p_L <- LargeModel(y)
@@ -129,19 +176,23 @@ def generate(small: Model, large: Model, enc_ids, alpha_fb: float, alpha_rb: flo
             j = L_len + m_star + 1
             stats["rollbacks"] += 1
             stats["discarded"] += n - j + 1
-            mg["argmax"] = min(mg["argmax"], rows[m_star][3])
+            tokL, smg = pick(ZL[m_star], rows[m_star][0], u_large[j] if sampling else 0.0)
+            gapL = math.inf if sampling else rows[m_star][3]
+            mg["argmax"] = min(mg["argmax"], gapL)
             del y[j:]
-            y.append(rows[m_star][0]); n = j
+            y.append(tokL); n = j
             stL.rewind(j)
             stS.rewind(j)
             L_len = j
             trace.append((KIND_ROLLBACK, j, y[j], k, m_star, d_star))
-            tmg.append((rows[m_star][3], math.inf, rb_here))
+            tmg.append((gapL, math.inf, rb_here) + ((smg,) if sampling else ()))
         else:
-            mg["argmax"] = min(mg["argmax"], rows[k - 1][3])
-            y.append(rows[k - 1][0]); n += 1
+            tokL, smg = pick(ZL[k - 1], rows[k - 1][0], u_large[n + 1] if sampling else 0.0)
+            gapL = math.inf if sampling else rows[k - 1][3]
+            mg["argmax"] = min(mg["argmax"], gapL)
+            y.append(tokL); n += 1
             L_len = n
             trace.append((KIND_VERIFY_OK, n, y[n], k, -1, d_max))
-            tmg.append((rows[k - 1][3], math.inf, rb_here))
+            tmg.append((gapL, math.inf, rb_here) + ((smg,) if sampling else ()))
         drafts = 0
     return dict(tokens=y[1:], trace=trace, stats=stats, margins=mg, logits=logits, trace_margins=tmg)

@@ -11,7 +11,7 @@ import torch
 
 from oracle import bild
 from oracle.t5 import (Model, attend, decoder_bucket, encoder_bucket, gelu_tanh, rms_norm, softmax)
-from workloads import MODEL_SHAPES, WORKLOADS, gen_ids, gen_model
+from workloads import MODEL_SHAPES, WORKLOADS, gen_ids, gen_model, gen_uniforms
 
 INF = math.inf
 
@@ -229,6 +229,78 @@ def test_eos_stops_the_loop(pair):
     ref = bild.generate(S, L, ids, 0.0, INF, 10, mode="small")["tokens"]
     r = bild.generate(S, L, ids, 0.0, INF, 10, mode="small", eos_id=ref[4])
     assert r["tokens"] == ref[:5]
+
+
+# ---- sampling variant (supplementary material, "BiLD with Sampling") -----------------------
+def test_nucleus_sample_against_its_definition():
+    """Small vocabularies, every decision by brute force: the nucleus is the shortest prefix of the tokens sorted by
+    decreasing probability (ties: lower index) with mass >= top_p; over a fine grid of u the tokens come out with
+    frequencies proportional to their probabilities inside the nucleus and never from outside it."""
+    rng = np.random.default_rng(3)
+    for V, top_p in [(5, 0.8), (17, 0.8), (64, 0.5), (64, 1.0), (9, 0.95)]:
+        z = rng.normal(size=V) * 2
+        z[3] = z[1]                                    # a tie, resolved by index
+        p = np.exp(z) / np.exp(z).sum()
+        ranked = sorted(range(V), key=lambda i: (-p[i], i))
+        mass, keep = 0.0, []
+        for i in ranked:                               # plain loop: add tokens until the mass reaches top_p
+            keep.append(i); mass += p[i]
+            if mass >= top_p:
+                break
+        assert mass - p[keep[-1]] < top_p <= mass or len(keep) == V
+        N = 20000
+        counts = np.zeros(V)
+        for j in range(N):
+            tok, n, _ = bild.nucleus_sample(z, top_p, (j + 0.5) / N)
+            assert n == len(keep) and tok in keep
+            counts[tok] += 1
+        for i in range(V):                             # the u's that give token i form one interval of length p_i / mass
+            want = N * p[i] / mass if i in keep else 0.0
+            assert abs(counts[i] - want) <= 1.0 + 1e-9, (V, top_p, i)
+    # u = 0 gives the most probable token; top_p -> 0 keeps only that token
+    z = rng.normal(size=40)
+    assert bild.nucleus_sample(z, 0.8, 0.0)[0] == int(np.argmax(z))
+    assert all(bild.nucleus_sample(z, 1e-12, u)[:2] == (int(np.argmax(z)), 1) for u in (0.0, 0.3, 0.999999))
+
+
+def test_sampling_with_a_vanishing_nucleus_is_greedy(pair):
+    wl, S, L, ids = pair
+    uS, uL = gen_uniforms(wl.gen_len + 2, 1, "small"), gen_uniforms(wl.gen_len + 2, 1, "large")
+    ref = bild.generate(S, L, ids, 0.3, 16.0, wl.gen_len, max_draft=5)
+    got = bild.generate(S, L, ids, 0.3, 16.0, wl.gen_len, max_draft=5, top_p=1e-12, u_small=uS, u_large=uL)
+    assert got["tokens"] == ref["tokens"] and got["trace"] == ref["trace"] and got["stats"] == ref["stats"]
+
+
+@pytest.mark.parametrize("alpha_fb,alpha_rb,max_draft", [(0.3, 16.0, 10), (0.5, 14.0, 4), (0.0, 15.0, 3)])
+def test_certificate_of_a_sampled_run(pair, alpha_fb, alpha_rb, max_draft):
+    """Sampling changes how tokens are drawn and nothing else: recomputed from scratch on the final sequence, every token
+    the trace attributes to the small model is the nucleus draw from p_S with that position's number and passed the
+    fallback test; every large-model token is the nucleus draw from p_L with the large model's number of that position."""
+    wl, S, L, ids = pair
+    n = wl.gen_len
+    uS, uL = gen_uniforms(n + 2, 2, "small"), gen_uniforms(n + 2, 2, "large")
+    r = bild.generate(S, L, ids, alpha_fb, alpha_rb, n, max_draft=max_draft, top_p=0.8, u_small=uS, u_large=uL)
+    y = [0] + r["tokens"]
+    assert len(r["trace_margins"]) == len(r["trace"]) and all(len(t) == 4 for t in r["trace_margins"])
+    ZS = S.forward_full(S.start(ids, len(y)), y[:-1])
+    ZL = L.forward_full(L.start(ids, len(y)), y[:-1])
+    owner = {}
+    for kind, pos, tok, k, m, val in r["trace"]:
+        if kind == bild.KIND_SMALL_ACCEPT:
+            owner[pos] = "S"
+        elif kind in (bild.KIND_VERIFY_OK, bild.KIND_ROLLBACK):
+            for q in [q for q in owner if q > pos]:
+                del owner[q]
+            owner[pos] = "L"
+    assert sorted(owner) == list(range(1, n + 1))
+    for j in range(1, len(y)):
+        if owner[j] == "S":
+            assert y[j] == bild.nucleus_sample(ZS[j - 1], 0.8, float(uS[j]))[0]
+            assert bild.max_prob(ZS[j - 1])[1] >= alpha_fb
+        else:
+            assert y[j] == bild.nucleus_sample(ZL[j - 1], 0.8, float(uL[j]))[0]
+    assert any(bild.max_prob(ZS[j - 1])[0] != y[j] for j in range(1, len(y)) if owner[j] == "S") or alpha_fb > 0.45
+    assert r["tokens"] != bild.generate(S, L, ids, alpha_fb, alpha_rb, n, max_draft=max_draft)["tokens"]
 
 
 # ---- closed forms --------------------------------------------------------------

@@ -165,3 +165,10 @@ def gen_ids(vocab: int, n: int, seed: int) -> np.ndarray:
     """Encoder input: n token ids uniform on [2, vocab) (0 = start/pad, 1 = EOS)."""
     g = _stream(seed, "input", f"ids{n}")
     return g.integers(2, vocab, size=n, dtype=np.int64).astype(np.int32)
+
+
+def gen_uniforms(n: int, seed: int, tag: str) -> np.ndarray:
+    """n uniform numbers in [0, 1) as fp32 (multiples of 2^-24, so exact in either precision): the random
+    input of the sampling variant, one per output position; `tag` names the stream ("small" / "large")."""
+    g = _stream(seed, "uniform", tag)
+    return (g.integers(0, 1 << 24, size=n, dtype=np.int64).astype(np.float64) / float(1 << 24)).astype(np.float32)
