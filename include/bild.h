@@ -254,6 +254,22 @@ int bild_fetch_result(bild_ctx *ctx, int32_t *tokens_out /*HOST*/, int *n_tokens
  * Synchronises. */
 int bild_time_pass(bild_ctx *ctx, int which, int k, int cache_len, int iters, float *ms_per_pass /*HOST out*/);
 
+/* The sampling variant (supplementary material, section "BiLD with Sampling"): both models draw
+ * their tokens by nucleus sampling with mass top_p (0 < top_p <= 1; the paper uses 0.8) instead of
+ * taking the arg-max, while the fallback test (maximum probability of the small model) and the rollback
+ * test (-ln p_L of the token the small model drew) stay as they are.  The random numbers are inputs:
+ * u_small[j] / u_large[j] in [0, 1) is used when the small / large model draws the token written to
+ * y[j], j = 1 .. max_len (HOST arrays of max_len + 1 floats; a position drawn again after a rollback
+ * uses the same number).  Nucleus: tokens in order of decreasing probability (equal: lower index
+ * first), shortest prefix with mass >= top_p; drawn token: first of the prefix at which the running sum
+ * exceeds u times the prefix's mass.  Otherwise as bild_generate; the LM heads keep their logits in the
+ * workspace in this mode and one more kernel per pass draws the token. */
+int bild_generate_sampled(bild_ctx *ctx, int mode, float alpha_fb, float alpha_rb, int max_len,
+                          float top_p, const float *u_small /*HOST*/, const float *u_large /*HOST*/,
+                          int32_t *tokens_out /*HOST*/, int *n_tokens /*HOST out*/,
+                          bild_trace_rec *trace_out /*HOST or NULL*/, int trace_cap, int *n_trace,
+                          bild_stats *stats /*HOST or NULL*/);
+
 /* 1 if the tcgen05 tensor-core kernel is in use for this context (bf16 weights, d_model / inner /
  * d_ff multiples of 64): it runs the encoder's linear layers, and those of the large model's
  * block pass (k > 1) when the row-slice kernel is switched off (BILD_SLICE=0); 0 if everything

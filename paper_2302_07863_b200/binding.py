@@ -27,7 +27,7 @@ EXPORTS = ["bild_query_workspace", "bild_create", "bild_create_tuned", "bild_tun
            "bild_fetch_result", "bild_time_pass", "bild_uses_tensor_cores", "bild_launch_count", "bild_last_error", "bild_op_linear",
            "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_op_lm_head_static", "bild_debug_bucket",
            "bild_debug_read_cache", "bild_op_lm_head_sliced", "bild_op_sublayer_scratch_bytes", "bild_op_attn_sublayer",
-           "bild_op_ffn_sublayer"]
+           "bild_op_ffn_sublayer", "bild_generate_sampled"]
 
 
 class ModelCfg(C.Structure):
@@ -252,6 +252,25 @@ class Context:
         st = Stats()
         self._check(self.L.bild_generate(self.h, mode, alpha_fb, alpha_rb, max_len, toks, C.byref(n), tr, cap,
                                          C.byref(nt), C.byref(st)))
+        return self._unpack(toks, n, tr, nt, cap, st)
+
+    def generate_sampled(self, mode: int, alpha_fb: float, alpha_rb: float, max_len: int, top_p: float, u_small, u_large):
+        """bild_generate_sampled: nucleus sampling from both models; u_small / u_large: max_len + 1 uniform numbers each."""
+        toks = (C.c_int32 * max(1, max_len))()
+        n = C.c_int()
+        cap = (max_len + 1) * (self.cfg.max_draft + 3)
+        tr = (TraceRec * cap)()
+        nt = C.c_int()
+        st = Stats()
+        us = np.ascontiguousarray(u_small, dtype=np.float32)
+        ul = np.ascontiguousarray(u_large, dtype=np.float32)
+        assert len(us) >= max_len + 1 and len(ul) >= max_len + 1
+        fp = C.POINTER(C.c_float)
+        self.L.bild_generate_sampled.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_float, C.c_int, C.c_float, fp, fp,
+                                                 C.POINTER(C.c_int32), C.POINTER(C.c_int), C.POINTER(TraceRec), C.c_int,
+                                                 C.POINTER(C.c_int), C.POINTER(Stats)]
+        self._check(self.L.bild_generate_sampled(self.h, mode, alpha_fb, alpha_rb, max_len, top_p, us.ctypes.data_as(fp),
+                                                 ul.ctypes.data_as(fp), toks, C.byref(n), tr, cap, C.byref(nt), C.byref(st)))
         return self._unpack(toks, n, tr, nt, cap, st)
 
     def generate_async(self, mode: int, alpha_fb: float, alpha_rb: float, max_len: int):

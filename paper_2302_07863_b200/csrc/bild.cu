@@ -17,6 +17,7 @@
 #include "enc_gemm.cuh"
 #include "enc_attention.cuh"
 #include "sublayer.cuh"
+#include "sampling.cuh"
 
 using namespace bild;
 
@@ -116,6 +117,7 @@ struct Model {
   // fused sub-layer kernels (bf16 only): two more residual-stream buffers, W_fo transposed per layer
   float *xb = nullptr, *xc = nullptr;
   __nv_bfloat16* wfoT = nullptr;     // [layers][F][d]
+  float* logits = nullptr;           // [MAXB][V] logits of the last pass (sampling variant only)
   bool fused = false;
   int sub_C = 1;                     // blocks per head (cluster size) of the attention sub-layers
   int sub_kc = 16, sub_bias_len = 32;
@@ -135,6 +137,9 @@ struct bild_ctx {
   int* enc_ids = nullptr;
   int* enc_len_dev = nullptr;
   int* bucket_tmp = nullptr;
+  float* u_draw[2] = {nullptr, nullptr};   // uniform numbers by output position, small / large model (sampling variant)
+  float top_p = 0.f;                       // > 0 while a sampled generation is set up or running
+  bool draw = false;                       // decoder passes are followed by the token-drawing kernel
   // encoder temporaries, one set per model (the two encoders run side by side on two streams)
   struct EncBuf {
     float *ex = nullptr, *eq = nullptr, *ek = nullptr, *ev = nullptr, *eatt = nullptr, *eu = nullptr;
@@ -151,8 +156,10 @@ struct bild_ctx {
   HeadOut* pin_head = nullptr;
   size_t ws_bytes = 0;
   // device-side loop: WHILE { small pass; IF (fallback) { large block pass } } and WHILE { large pass }
-  cudaGraph_t graph[2] = {nullptr, nullptr};
-  cudaGraphExec_t exec[2] = {nullptr, nullptr};
+  // [0], [1]: greedy; [2], [3]: the same two loops with the token-drawing kernel after every LM head
+  cudaGraph_t graph[4] = {nullptr, nullptr, nullptr, nullptr};
+  cudaGraphExec_t exec[4] = {nullptr, nullptr, nullptr, nullptr};
+  int64_t sampled_counted = 0;
   int64_t per_pass[2] = {0, 0};      // kernel launches in one small / one large pass of the graphs
   int64_t per_pass_large1 = 0, per_pass_large8 = 0;
   int64_t* cnt = &launches;         // where launches are counted (redirected while capturing)
@@ -238,6 +245,8 @@ void plan(bild_ctx* c, Bump& b) {
   c->enc_ids = b.take<int>(ecap);
   c->enc_len_dev = b.take<int>(1);
   c->bucket_tmp = b.take<int>(std::max(cap, 2 * ecap));
+  c->u_draw[0] = b.take<float>(cap + 1);
+  c->u_draw[1] = b.take<float>(cap + 1);
   for (int i = 0; i < 2; ++i) {
     Model& m = c->m[i];
     const bild_model_cfg& mc = i == 0 ? cfg.small_cfg : cfg.large_cfg;
@@ -262,6 +271,7 @@ void plan(bild_ctx* c, Bump& b) {
     m.head_cnt = b.take<unsigned>(1);
     m.head_out = b.take<HeadOut>(1);
     m.desc = b.take<CallDesc>(1);
+    m.logits = b.take<float>((size_t)MAXB * mc.vocab);
     m.xb = b.take<float>((size_t)MAXB * mc.d_model);
     m.xc = b.take<float>((size_t)MAXB * mc.d_model);
     m.wfoT = b.take<__nv_bfloat16>(cfg.dtype == BILD_BF16 ? (size_t)mc.n_layers * mc.d_ff * mc.d_model : 0);
@@ -952,6 +962,15 @@ int decoder_pass(bild_ctx* c, int which, int MBv, float* logits_dbg, unsigned lo
   h.counter = m.head_cnt; h.out = m.head_out; h.logits_dbg = logits_dbg; h.which = which; h.loop = loop_ptrs(c);
   h.cond_while = cond_while; h.cond_if = cond_if; h.cond_if1 = cond_if1; h.cond_if8 = cond_if8;
   h.pass_kind = which == 0 ? 0 : MBv == 1 ? 2 : MBv == SUB_MB ? 3 : 1;
+  if (c->draw) {   // sampling: the head leaves its logits and the policy step to the kernel that draws the token
+    if (!h.logits_dbg) h.logits_dbg = m.logits;
+    h.defer_policy = 1;
+  }
+  auto draw_token = [&]() -> int {
+    if (!c->draw) return BILD_OK;
+    CUDA_TRY(c, launch_k(c, nucleus_policy_kernel, dim3(1), dim3(NS_THREADS), 0, h, (const float*)h.logits_dbg, (const float*)c->u_draw[which]));
+    return BILD_OK;
+  };
   const int head_tr = (MB == 1 && d <= 512) ? 32 : 16;   // rows per tile of the tensor-core head
   const size_t sh_smem = slice_head_smem_bytes(d, head_tr);
   // single-row passes: only heads of 32 MB and more (smaller ones stay on the GEMV head)
@@ -964,10 +983,10 @@ int decoder_pass(bild_ctx* c, int which, int MBv, float* logits_dbg, unsigned lo
       c->slice_head_smem_set = true;
     }
     CUDA_TRY(c, launch_k(c, slice_head_kernel, dim3(c->sms), dim3(SH_THREADS), sh_smem, h, &c->st->err, head_tr));
-    return BILD_OK;
+    return draw_token();
   }
   CUDA_TRY(c, launch_head(c->stream, c->use_pdl, dt, MB, h, m.head_grid, c->cnt));
-  return BILD_OK;
+  return draw_token();
 }
 
 // Encoder of model `which` over the ids in c->enc_ids, then the cross-attention K/V of
@@ -1087,10 +1106,10 @@ int capture_pass(bild_ctx* c, cudaGraph_t body, int which, int MB, unsigned long
 
 // Builds the two device-side loops (CUDA graphs with conditional nodes).  The head
 // kernel's last block sets the WHILE handle to "not done" and the IF handle to "fallback".
-int build_graphs_once(bild_ctx* c);
+int build_graphs_once(bild_ctx* c, int base);
 
 void drop_graphs(bild_ctx* c) {
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < 4; ++i) {
     if (c->exec[i]) cudaGraphExecDestroy(c->exec[i]);
     if (c->graph[i]) cudaGraphDestroy(c->graph[i]);
     c->exec[i] = nullptr;
@@ -1098,40 +1117,50 @@ void drop_graphs(bild_ctx* c) {
   }
 }
 
-int build_graphs(bild_ctx* c) {
-  if (c->exec[0] && c->exec[1]) return BILD_OK;
+// base 0: the greedy loops; base 2: the loops of the sampling variant (a token-drawing kernel after every LM head)
+int build_graphs(bild_ctx* c, int base) {
+  if (c->exec[base] && c->exec[base + 1]) return BILD_OK;
   // if a loop body refuses programmatic edges, the graphs are built again with plain launches
   const bool want_pdl = c->use_pdl;
-  int rc = build_graphs_once(c);
+  c->draw = base == 2;
+  int rc = build_graphs_once(c, base);
   if (rc != BILD_OK && want_pdl) {
     drop_graphs(c);
     cudaGetLastError();
     c->use_pdl = false;
-    rc = build_graphs_once(c);
+    rc = build_graphs_once(c, base);
   }
+  c->draw = false;
   if (rc != BILD_OK) { drop_graphs(c); cudaGetLastError(); }
   return rc;
 }
 
-int build_graphs_once(bild_ctx* c) {
+int build_graphs_once(bild_ctx* c, int base) {
+  // launches per pass are recorded from the greedy graphs; the drawing kernels of the sampled ones are counted on the device
+  int64_t dummy[2] = {0, 0}, dummy1 = 0, dummy8 = 0;
+  int64_t* per_pass = base == 0 ? c->per_pass : dummy;
+  int64_t& per_pass_large1 = base == 0 ? c->per_pass_large1 : dummy1;
+  int64_t& per_pass_large8 = base == 0 ? c->per_pass_large8 : dummy8;
+  cudaGraph_t* graph = c->graph + base;
+  cudaGraphExec_t* exec = c->exec + base;
   {  // BiLD (and small-only): WHILE { small pass ; IF { large block pass } ; IF { large single-row pass } }
-    CUDA_TRY(c, cudaGraphCreate(&c->graph[0], 0));
+    CUDA_TRY(c, cudaGraphCreate(&graph[0], 0));
     cudaGraphConditionalHandle hw, hi, hi1, hi8 = 0;
-    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hw, c->graph[0], 1, cudaGraphCondAssignDefault));
-    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi, c->graph[0], 0, cudaGraphCondAssignDefault));
-    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi1, c->graph[0], 0, cudaGraphCondAssignDefault));
+    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hw, graph[0], 1, cudaGraphCondAssignDefault));
+    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi, graph[0], 0, cudaGraphCondAssignDefault));
+    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi1, graph[0], 0, cudaGraphCondAssignDefault));
     // passes of 2 to 8 rows have a branch of their own where they run on the fused sub-layer kernels
     const bool body8 = c->m[1].fused && c->fused_on >= 2;
-    if (body8) CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi8, c->graph[0], 0, cudaGraphCondAssignDefault));
+    if (body8) CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hi8, graph[0], 0, cudaGraphCondAssignDefault));
     cudaGraph_t body = nullptr, ifbody = nullptr, if1body = nullptr, if8body = nullptr;
-    int rc = add_cond(c, c->graph[0], nullptr, 0, hw, cudaGraphCondTypeWhile, &body);
+    int rc = add_cond(c, graph[0], nullptr, 0, hw, cudaGraphCondTypeWhile, &body);
     if (rc) return rc;
     std::vector<cudaGraphNode_t> leaves;
-    rc = capture_pass(c, body, 0, 1, hw, hi, &leaves, &c->per_pass[0], hi1, hi8);
+    rc = capture_pass(c, body, 0, 1, hw, hi, &leaves, &per_pass[0], hi1, hi8);
     if (rc) return rc;
     rc = add_cond(c, body, leaves.data(), leaves.size(), hi, cudaGraphCondTypeIf, &ifbody);
     if (rc) return rc;
-    rc = capture_pass(c, ifbody, 1, MAXB, hw, 0, nullptr, &c->per_pass[1]);
+    rc = capture_pass(c, ifbody, 1, MAXB, hw, 0, nullptr, &per_pass[1]);
     if (rc) return rc;
     // a fallback right after a large pass verifies one row: that pass runs on the single-row kernels
     rc = add_cond(c, body, leaves.data(), leaves.size(), hi1, cudaGraphCondTypeIf, &if1body);
@@ -1139,25 +1168,25 @@ int build_graphs_once(bild_ctx* c) {
     int64_t n1 = 0;
     rc = capture_pass(c, if1body, 1, 1, hw, 0, nullptr, &n1);
     if (rc) return rc;
-    c->per_pass_large1 = n1;
+    per_pass_large1 = n1;
     if (body8) {
       rc = add_cond(c, body, leaves.data(), leaves.size(), hi8, cudaGraphCondTypeIf, &if8body);
       if (rc) return rc;
-      rc = capture_pass(c, if8body, 1, SUB_MB, hw, 0, nullptr, &c->per_pass_large8);
+      rc = capture_pass(c, if8body, 1, SUB_MB, hw, 0, nullptr, &per_pass_large8);
       if (rc) return rc;
     }
-    CUDA_TRY(c, cudaGraphInstantiate(&c->exec[0], c->graph[0], 0));
+    CUDA_TRY(c, cudaGraphInstantiate(&exec[0], graph[0], 0));
   }
   {  // large-only greedy: WHILE { large pass with k = 1 }
-    CUDA_TRY(c, cudaGraphCreate(&c->graph[1], 0));
+    CUDA_TRY(c, cudaGraphCreate(&graph[1], 0));
     cudaGraphConditionalHandle hw;
-    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hw, c->graph[1], 1, cudaGraphCondAssignDefault));
+    CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hw, graph[1], 1, cudaGraphCondAssignDefault));
     cudaGraph_t body = nullptr;
-    int rc = add_cond(c, c->graph[1], nullptr, 0, hw, cudaGraphCondTypeWhile, &body);
+    int rc = add_cond(c, graph[1], nullptr, 0, hw, cudaGraphCondTypeWhile, &body);
     if (rc) return rc;
-    rc = capture_pass(c, body, 1, 1, hw, 0, nullptr, &c->per_pass_large1);
+    rc = capture_pass(c, body, 1, 1, hw, 0, nullptr, &per_pass_large1);
     if (rc) return rc;
-    CUDA_TRY(c, cudaGraphInstantiate(&c->exec[1], c->graph[1], 0));
+    CUDA_TRY(c, cudaGraphInstantiate(&exec[1], graph[1], 0));
   }
   return BILD_OK;
 }
@@ -1170,6 +1199,8 @@ int read_state(bild_ctx* c) {
     const int64_t total = cp[0] * c->per_pass[0] + cp[1] * c->per_pass[1] + cp[2] * c->per_pass_large1 + cp[3] * c->per_pass_large8;
     c->launches += total - c->graph_counted;
     c->graph_counted = total;
+    c->launches += c->pin_state->cum_draws - c->sampled_counted;
+    c->sampled_counted = c->pin_state->cum_draws;
   }
   if (c->pin_state->err) return fail(c, c->pin_state->err, "device-side error flag set");
   return BILD_OK;
@@ -1177,7 +1208,7 @@ int read_state(bild_ctx* c) {
 
 int reset_state(bild_ctx* c, int mode, float afb, float arb, int max_len) {
   reset_state_kernel<<<1, 1, 0, c->stream>>>(loop_ptrs(c), mode, afb, arb, max_len, c->cfg.max_draft,
-                                             c->cfg.eos_id, c->cfg.start_id, c->trace_cap);
+                                             c->cfg.eos_id, c->cfg.start_id, c->trace_cap, c->top_p);
   (*c->cnt)++;
   CUDA_TRY(c, cudaGetLastError());
   return BILD_OK;
@@ -1435,25 +1466,44 @@ int bild_rewind(bild_ctx* c, int which, int new_len) {
   return BILD_OK;
 }
 
-int bild_generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, int max_len) {
+}  // extern "C"
+
+namespace {
+// top_p > 0: the sampling variant, with the uniform numbers of both models by output position (HOST, max_len + 1 each)
+int generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, int max_len, float top_p, const float* u_small,
+                   const float* u_large) {
   if (!c) return BILD_ERR_ARG;
   if (!c->encoded) return fail(c, BILD_ERR_STATE, "bild_encode has not been called");
   if (mode < 0 || mode > 2) return fail(c, BILD_ERR_ARG, "mode");
   if (max_len < 0) return fail(c, BILD_ERR_ARG, "max_len < 0");
   if (max_len + 1 > c->cfg.max_dec_len) return fail(c, BILD_ERR_CAPACITY, "max_len + 1 > max_dec_len");
+  const bool sampled = top_p > 0.f;
+  c->top_p = sampled ? top_p : 0.f;
+  if (sampled) {
+    if (!(top_p <= 1.f) || !u_small || !u_large) return fail(c, BILD_ERR_ARG, "sampling needs 0 < top_p <= 1 and both arrays of uniform numbers");
+    for (int i = 0; i <= max_len; ++i)
+      if (!(u_small[i] >= 0.f && u_small[i] < 1.f) || !(u_large[i] >= 0.f && u_large[i] < 1.f))
+        return fail(c, BILD_ERR_ARG, "uniform numbers must lie in [0, 1)");
+    CUDA_TRY(c, cudaMemcpyAsync(c->u_draw[0], u_small, (max_len + 1) * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(c->u_draw[1], u_large, (max_len + 1) * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));   // the caller's arrays may be pageable and go away
+  }
   if (!c->host_loop) {
     // device-side loop: no host involvement between the first and the last token
-    int rc = build_graphs(c);
+    const int base = sampled ? 2 : 0;
+    int rc = build_graphs(c, base);
     if (rc) return rc;
     rc = reset_state(c, mode, alpha_fb, alpha_rb, max_len);
     if (rc) return rc;
     if (max_len == 0 || c->cfg.start_id == c->cfg.eos_id) return BILD_OK;
     // passes the loop may run: bounded by the guard of the device-side policy
-    CUDA_TRY(c, cudaGraphLaunch(c->exec[mode == BILD_MODE_LARGE_ONLY ? 1 : 0], c->stream));
+    CUDA_TRY(c, cudaGraphLaunch(c->exec[base + (mode == BILD_MODE_LARGE_ONLY ? 1 : 0)], c->stream));
     return BILD_OK;
   }
   int rc = reset_state(c, mode, alpha_fb, alpha_rb, max_len);
   if (rc) return rc;
+  struct DrawGuard { bild_ctx* c; ~DrawGuard() { c->draw = false; } } guard_draw{c};
+  c->draw = sampled;
   // Debug loop driver: the policy still runs on the device; the host reads two flags per step.
   const int guard = (max_len + 1) * (c->cfg.max_draft + 3);
   rc = read_state(c);
@@ -1473,6 +1523,23 @@ int bild_generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, i
     if (rc) return rc;
   }
   return BILD_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int bild_generate_async(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, int max_len) {
+  return generate_async(c, mode, alpha_fb, alpha_rb, max_len, 0.f, nullptr, nullptr);
+}
+
+int bild_generate_sampled(bild_ctx* c, int mode, float alpha_fb, float alpha_rb, int max_len, float top_p, const float* u_small,
+                          const float* u_large, int32_t* tokens_out, int* n_tokens, bild_trace_rec* trace_out, int trace_cap,
+                          int* n_trace, bild_stats* stats) {
+  if (!c || !tokens_out || !n_tokens) return fail(c, BILD_ERR_ARG, "null argument");
+  if (!(top_p > 0.f)) return fail(c, BILD_ERR_ARG, "top_p must be positive");
+  int rc = generate_async(c, mode, alpha_fb, alpha_rb, max_len, top_p, u_small, u_large);
+  if (rc) return rc;
+  return bild_fetch_result(c, tokens_out, n_tokens, trace_out, trace_cap, n_trace, stats);
 }
 
 int bild_fetch_result(bild_ctx* c, int32_t* tokens_out, int* n_tokens, bild_trace_rec* trace_out, int trace_cap,

@@ -51,6 +51,9 @@ struct DevState {
   bild_stats stats;
   int passes;   // decoder passes taken by the running loop (guards against a runaway loop)
   int pad0;
+  float top_p;  // > 0: the sampling variant, tokens are drawn from the nucleus of this mass
+  int pad1;
+  long long cum_draws;       // token-drawing kernels run from the loop graphs since create
   long long cum_passes[4];   // passes run from the loop graphs since create: small, large block, large single row, large up to 8 rows
 };
 

@@ -482,12 +482,13 @@ struct HeadArgs {
   unsigned long long cond_if1;   // IF node of the single-row large pass (0: the block branch takes every large pass)
   unsigned long long cond_if8;   // IF node of the large pass over 2 to 8 rows (0: the block branch takes them)
   int pass_kind;                 // which pass counter the kernel bumps inside a loop graph: 0 small, 1 block, 2 single row, 3 up to 8 rows
+  int defer_policy;              // sampling: the head leaves policy and loop control to the kernel that draws the token
 };
 
 // What the last block of every LM-head kernel does once the per-row results are complete: the policy tests, the
 // bookkeeping of Algorithm 1, and (inside a loop graph) the choice of what runs next.
 __device__ inline void policy_tail(const HeadArgs& a, HeadOut* o) {
-  if (!a.loop.st) return;
+  if (!a.loop.st || a.defer_policy) return;
   policy_tests(o, a.desc, a.loop.st, a.which);
   if (a.desc->run_policy) policy_step(a.loop, o, a.desc, a.which);
   else if (a.which == 0) a.loop.st->S_len = a.desc->pos0 + 1;
@@ -678,8 +679,9 @@ __global__ void rewind_kernel(DevState* st, int which, int new_len) {
 }
 
 __global__ void reset_state_kernel(LoopPtrs L, int mode, float alpha_fb, float alpha_rb, int max_len,
-                                   int max_draft, int eos_id, int start_id, int trace_cap) {
+                                   int max_draft, int eos_id, int start_id, int trace_cap, float top_p) {
   DevState* st = L.st;
+  st->top_p = top_p;
   st->n = 0; st->S_len = 0; st->L_len = 0; st->drafts = 0;
   st->fallback = 0; st->mode = mode; st->err = 0;
   st->max_len = max_len; st->max_draft = max_draft; st->eos_id = eos_id; st->start_id = start_id;

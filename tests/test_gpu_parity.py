@@ -11,7 +11,7 @@ import pytest
 
 from oracle import bild as obild
 from oracle.t5 import Model, rms_norm
-from workloads import MODEL_SHAPES, WORKLOADS, gen_ids, gen_model
+from workloads import MODEL_SHAPES, WORKLOADS, gen_ids, gen_model, gen_uniforms
 
 pytestmark = pytest.mark.gpu
 GOLD = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
@@ -365,6 +365,67 @@ def test_alternative_paths_match_golden(torch_cuda, name, tuning):
     assert_trace_equal(r["trace"], g["bild"]["trace"], 1e-3)
     assert r["stats"] == g["bild"]["stats"]
     assert ctx.launch_count() > 0
+    ctx.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "odd", "odd_bf16", "tiny_bf16", "wide_bf16"])
+@pytest.mark.parametrize("top_p,alpha_fb,alpha_rb,max_draft,seed", [(0.8, 0.3, 16.0, 10, 1), (0.8, 0.0, 14.0, 4, 2),
+                                                                  (1.0, 0.35, 15.0, 10, 3), (0.3, 0.25, 17.0, 7, 4),
+                                                                  (1e-9, 0.3, 16.0, 10, 5)])
+def test_sampled_generate_matches_live_oracle(torch_cuda, name, top_p, alpha_fb, alpha_rb, max_draft, seed):
+    """The sampling variant (nucleus sampling from both models, same policies) against the oracle run with the same
+    uniform numbers: same tokens, trace and counters up to the first record one of whose decisions (fallback test,
+    rollback test, nucleus boundary or draw) the oracle took with a margin below what the logit error allows."""
+    from paper_2302_07863_b200 import MODE_BILD, MODE_LARGE_ONLY, MODE_SMALL_ONLY
+    from paper_2302_07863_b200.synthetic import make_context
+    wl = WORKLOADS[name]
+    if name == "wide_bf16":
+        scS, scL = 9.0, 11.0
+    else:
+        g = golden(name)
+        scS, scL = g["scale_small"]["scale"], g["scale_large"]["scale"]
+    n = min(wl.gen_len, 40)
+    ctx, ids, _ = make_context(name, scS, scL, max_draft=max_draft)
+    ctx.encode(ids)
+    S = Model(MODEL_SHAPES[wl.small], gen_model(MODEL_SHAPES[wl.small], wl.seed, wl.dtype), scS)
+    L = Model(MODEL_SHAPES[wl.large], gen_model(MODEL_SHAPES[wl.large], wl.seed, wl.dtype), scL)
+    uS, uL = gen_uniforms(n + 1, seed, "small"), gen_uniforms(n + 1, seed, "large")
+    # logit error of this pair, measured here on a few passes of both models: the margin bound of the trace rule (2.5 e
+    # covers the 2 e a probability, a running sum of probabilities or a distance can move) is derived from it
+    torch = torch_cuda
+    V = S.s.vocab
+    buf = torch.empty((16, V), dtype=torch.float32, device="cuda")
+    stS, stL = S.start(ids, 16), L.start(ids, 16)
+    toks = [0] + [int(t) for t in gen_ids(V, 12, 21)]
+    e = 0.0
+    for t in toks[:4]:
+        ctx.small_step(t, 0.4, buf)
+        e = max(e, float(np.max(np.abs(buf[0].cpu().numpy() - S.forward_one(stS, t)))))
+    for blk in (toks[:1], toks[1:6], toks[6:13]):
+        ctx.large_verify(blk, 15.0, buf)
+        e = max(e, float(np.max(np.abs(buf[:len(blk)].cpu().numpy() - L.forward_block(stL, blk)))))
+    assert e <= TOL[wl.dtype]
+    lim = 2.5 * e + 2e-6
+    complete = 0
+    for mode, omode in ((MODE_BILD, "bild"), (MODE_SMALL_ONLY, "small"), (MODE_LARGE_ONLY, "large")):
+        want = obild.generate(S, L, ids, alpha_fb, alpha_rb, n, max_draft=max_draft, mode=omode, top_p=top_p, u_small=uS, u_large=uL)
+        got = ctx.generate_sampled(mode, alpha_fb, alpha_rb, n, top_p, uS, uL)
+        tm = [[None if math.isinf(v) else v for v in t] for t in want["trace_margins"]]
+        d = assert_trace_matches_up_to_low_margin(got["trace"], want["trace"], tm, wl.dtype, lim=lim)
+        if d is None:
+            assert got["tokens"] == want["tokens"]
+            assert got["stats"] == want["stats"]
+            complete += 1
+    assert complete >= 2, "the comparison stopped early at a low-margin record in more than one of the three runs"
+    # the greedy loop still works afterwards (its own graphs, no drawing kernel)
+    if name != "wide_bf16":
+        th = g["thresholds"]
+        ctx2, ids2, _ = make_context(name, scS, scL)
+        ctx2.encode(ids2)
+        assert ctx2.generate_sampled(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len, 1e-9, gen_uniforms(wl.gen_len + 1, 9, "small"),
+                                     gen_uniforms(wl.gen_len + 1, 9, "large"))["tokens"] == g["bild"]["tokens"]
+        assert ctx2.generate(MODE_BILD, th["alpha_fb"], th["alpha_rb"], wl.gen_len)["tokens"] == g["bild"]["tokens"]
+        ctx2.close()
     ctx.close()
 
 
