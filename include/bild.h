@@ -79,6 +79,13 @@ typedef struct {
   int32_t max_draft;    /* small-model tokens in a row before a forced fallback (paper: 10); 1..15 */
   int32_t start_id;     /* y[0] */
   int32_t eos_id;       /* -1: never stop on a token */
+  /* Early-exit configuration (Section 4.4, "Early Exiting Strategy"): n > 0 makes the small model the first n
+   * decoder layers of the large model, with the large model's encoder, embedding, final norm and prediction
+   * head.  small_cfg must then equal large_cfg except for n_layers (= n) and logit_scale; the small model's
+   * weights argument is ignored (may be NULL); only the large model's encoder runs, and the two "models"
+   * share the cross-attention K/V and the self-attention cache of those n layers (a large pass rewrites the
+   * rows the small steps wrote, so the cache always holds the large model's own values).  0: two models. */
+  int32_t early_exit_layers;
 } bild_config;
 
 /* All members are DEVICE pointers.  Matrices are row-major [out][in] in

@@ -101,11 +101,24 @@ def attend(q: np.ndarray, K: np.ndarray, V: np.ndarray, bias=None) -> np.ndarray
 class Model:
     """One encoder-decoder model with fp64 weights."""
 
-    def __init__(self, shape, tensors: dict, logit_scale: float = 1.0):
+    def __init__(self, shape, tensors: dict, logit_scale: float = 1.0, exit_layers: int = 0):
+        """exit_layers > 0: the early-exit "small model" of Section 4.4: the same encoder, embedding, final norm and
+        prediction head, but only the first `exit_layers` decoder layers."""
         self.s = shape
         self.w = {k: to_f64(v) for k, v in tensors.items()}
         self.logit_scale = float(logit_scale)
         self.lm = self.w["emb"] if shape.tied_head else self.w["lm_head"]
+        self.dec_layers = exit_layers if exit_layers > 0 else shape.n_layers
+        assert 1 <= self.dec_layers <= shape.n_layers
+
+    def early_exit(self, exit_layers: int, logit_scale: float = None) -> "Model":
+        """The model that shares every tensor with this one and stops after `exit_layers` decoder layers."""
+        m = Model.__new__(Model)
+        m.s, m.w, m.lm = self.s, self.w, self.lm
+        m.logit_scale = self.logit_scale if logit_scale is None else float(logit_scale)
+        m.dec_layers = exit_layers
+        assert 1 <= exit_layers <= self.s.n_layers
+        return m
 
     # ---- feed-forward -----------------------------------------------------
     def _ffn(self, p: str, h: np.ndarray) -> np.ndarray:
@@ -148,7 +161,7 @@ class Model:
         mem = self.encode(enc_ids)
         st = DecState(s, cap)
         st.mem = mem
-        for l in range(s.n_layers):
+        for l in range(self.dec_layers):
             kv = mem @ w[f"dec.{l}.wckv"].T
             st.ck.append(kv[:, :s.inner].copy())
             st.cv.append(kv[:, s.inner:].copy())
@@ -165,7 +178,7 @@ class Model:
         assert c + k <= st.cap
         x = w["emb"][np.asarray(tokens)]
         rb = w["dec.rel_bias"]
-        for l in range(s.n_layers):
+        for l in range(self.dec_layers):
             p = f"dec.{l}."
             qkv = rms_norm(x, w[p + "ln1"], s.eps) @ w[p + "wqkv"].T
             q = qkv[:, :I]
@@ -206,7 +219,7 @@ class Model:
         for i in range(n):
             for j in range(i + 1):
                 bias[:, i, j] = rb[decoder_bucket(i - j, s.rel_buckets, s.rel_max_dist)]
-        for l in range(s.n_layers):
+        for l in range(self.dec_layers):
             p = f"dec.{l}."
             qkv = rms_norm(x, w[p + "ln1"], s.eps) @ w[p + "wqkv"].T
             q = qkv[:, :I].reshape(n, H, dk).transpose(1, 0, 2)

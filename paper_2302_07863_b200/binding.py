@@ -38,7 +38,7 @@ class ModelCfg(C.Structure):
 
 class Config(C.Structure):
     _fields_ = [("small_cfg", ModelCfg), ("large_cfg", ModelCfg)] + [
-        (n, C.c_int32) for n in ("dtype", "max_enc_len", "max_dec_len", "max_draft", "start_id", "eos_id")]
+        (n, C.c_int32) for n in ("dtype", "max_enc_len", "max_dec_len", "max_draft", "start_id", "eos_id", "early_exit_layers")]
 
 
 class EncLayer(C.Structure):

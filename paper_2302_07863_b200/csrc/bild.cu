@@ -224,6 +224,16 @@ int check_config(const bild_config* cfg, std::string& why) {
   if (cfg->max_dec_len < 2 || cfg->max_dec_len > 2048) { why = "2 <= max_dec_len <= 2048"; return BILD_ERR_ARG; }
   if (cfg->max_draft < 1 || cfg->max_draft > MAXB - 1) { why = "1 <= max_draft <= 15"; return BILD_ERR_ARG; }
   if (cfg->start_id < 0 || cfg->start_id >= cfg->small_cfg.vocab) { why = "start_id"; return BILD_ERR_ARG; }
+  if (cfg->early_exit_layers < 0) { why = "early_exit_layers"; return BILD_ERR_ARG; }
+  if (cfg->early_exit_layers > 0) {
+    const bild_model_cfg &a = cfg->small_cfg, &b = cfg->large_cfg;
+    if (a.n_layers != cfg->early_exit_layers || a.n_layers > b.n_layers || a.d_model != b.d_model || a.n_heads != b.n_heads ||
+        a.d_kv != b.d_kv || a.d_ff != b.d_ff || a.ffn_kind != b.ffn_kind || a.rel_buckets != b.rel_buckets ||
+        a.rel_max_dist != b.rel_max_dist || a.ln_eps != b.ln_eps) {
+      why = "early exit: small_cfg must be large_cfg with n_layers = early_exit_layers";
+      return BILD_ERR_ARG;
+    }
+  }
   return BILD_OK;
 }
 
@@ -1253,7 +1263,8 @@ int bild_create_tuned(const bild_config* cfg, const bild_weights* small_w, const
   std::string why;
   int rc = check_config(cfg, why);
   if (rc) return rc;
-  if (!small_w || !large_w || !workspace) return BILD_ERR_ARG;
+  const bool early = cfg->early_exit_layers > 0;
+  if ((!small_w && !early) || !large_w || !workspace) return BILD_ERR_ARG;
   if ((uintptr_t)workspace % 256) return BILD_ERR_WORKSPACE;
   bild_ctx* c = new (std::nothrow) bild_ctx;
   if (!c) return BILD_ERR_ARG;
@@ -1293,7 +1304,11 @@ int bild_create_tuned(const bild_config* cfg, const bild_weights* small_w, const
   plan(c, b);
   c->ws_bytes = b.off;
   if (workspace_bytes < b.off) { delete c; return BILD_ERR_WORKSPACE; }
-  const bild_weights* ws[2] = {small_w, large_w};
+  if (early) {   // one cache for the shared layers: [layer][head][row][channel], the small model's layers come first
+    c->m[0].selfK = c->m[1].selfK; c->m[0].selfV = c->m[1].selfV;
+    c->m[0].crossK = c->m[1].crossK; c->m[0].crossV = c->m[1].crossV;
+  }
+  const bild_weights* ws[2] = {early ? large_w : small_w, large_w};   // early exit: the small model is a prefix of the large one
   for (int i = 0; i < 2; ++i) {
     Model& m = c->m[i];
     const bild_weights* w = ws[i];
@@ -1359,7 +1374,8 @@ int bild_encode(bild_ctx* c, const int32_t* ids, int n_ids) {
   CUDA_TRY(c, cudaMemcpyAsync(c->enc_len_dev, &c->enc_len, sizeof(int), cudaMemcpyHostToDevice, c->stream));
   // The two encoders are independent: the small model's runs on a side stream, forked from and joined
   // back into the caller's stream with events, while the large model's runs on the caller's stream.
-  bool side = c->enc_parallel;
+  const bool early = c->cfg.early_exit_layers > 0;   // one encoder: the small model is a prefix of the large model's decoder
+  bool side = c->enc_parallel && !early;
   if (side && !c->enc_stream) {
     if (cudaStreamCreateWithFlags(&c->enc_stream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&c->enc_fork, cudaEventDisableTiming) != cudaSuccess ||
@@ -1381,7 +1397,7 @@ int bild_encode(bild_ctx* c, const int32_t* ids, int n_ids) {
     if (rc1) return rc1;
     CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->enc_join, 0));
   } else {
-    for (int i = 0; i < 2; ++i) {
+    for (int i = early ? 1 : 0; i < 2; ++i) {
       int rc = encoder_pass(c, i);
       if (rc) return rc;
     }

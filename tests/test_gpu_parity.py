@@ -429,6 +429,61 @@ def test_sampled_generate_matches_live_oracle(torch_cuda, name, top_p, alpha_fb,
     ctx.close()
 
 
+@pytest.mark.parametrize("name,exit_layers", [("tiny", 1), ("odd_bf16", 1), ("tiny_bf16", 2), ("wide_bf16", 1), ("mt5_mt", 1)])
+def test_early_exit_configuration_matches_oracle(torch_cuda, name, exit_layers):
+    """Section 4.4: the small model is the first layer(s) of the large model with the shared head; one encoder, one
+    cross K/V, one self-attention cache for the shared layers.  Single passes (logits) and whole generations against
+    the oracle pair built the same way; for mt5_mt the large model is replaced by the mT5-small shape the paper uses
+    (8 layers, exit after the first)."""
+    import dataclasses
+    from paper_2302_07863_b200 import MODE_BILD, MODE_SMALL_ONLY
+    from paper_2302_07863_b200.synthetic import make_context
+    torch = torch_cuda
+    wl = WORKLOADS[name]
+    if name == "mt5_mt":    # the paper's pair: mT5-small as the large model
+        wl = dataclasses.replace(wl, large=wl.small)
+    key, scS, scL = wl.large, 14.0, 9.0
+    sh = MODEL_SHAPES[key]
+    WORKLOADS["_early"] = wl
+    try:
+        ctx, ids, _ = make_context("_early", scS, scL, early_exit_layers=exit_layers, max_draft=5)
+    finally:
+        del WORKLOADS["_early"]
+    ctx.encode(ids)
+    L = Model(sh, gen_model(sh, wl.seed, wl.dtype), scL)
+    S = L.early_exit(exit_layers, logit_scale=scS)
+    V = sh.vocab
+    n = min(wl.gen_len, 24)
+    buf = torch.empty((16, V), dtype=torch.float32, device="cuda")
+    stS, stL = S.start(ids, n + 1), L.start(ids, n + 1)
+    toks = [0] + [int(t) for t in gen_ids(V, 12, 33)]
+    e = 0.0
+    # interleaved as in the loop: small steps draft over the shared cache rows, the large pass rewrites them
+    for t in toks[:4]:
+        ctx.small_step(t, 0.4, buf)
+        e = max(e, float(np.max(np.abs(buf[0].cpu().numpy() - S.forward_one(stS, t)))))
+    for blk in (toks[:4], toks[4:5]):
+        ctx.large_verify(blk, 15.0, buf)
+        e = max(e, float(np.max(np.abs(buf[:len(blk)].cpu().numpy() - L.forward_block(stL, blk)))))
+    ctx.rewind(0, 3); ctx.rewind(1, 3); stS.rewind(3); stL.rewind(3)
+    for t in toks[3:6]:     # the small model goes on from rows the large pass wrote
+        ctx.small_step(t, 0.4, buf)
+        e = max(e, float(np.max(np.abs(buf[0].cpu().numpy() - S.forward_one(stS, t)))))
+    assert e <= (1e-4 if wl.dtype == "fp32" else 2e-3), e
+    lim = 2.5 * e + 2e-6
+    for afb, arb in ((0.3, 12.0), (0.6, 8.0), (0.0, 10.0)):
+        want = obild.generate(S, L, ids, afb, arb, n, max_draft=5)
+        got = ctx.generate(MODE_BILD, afb, arb, n)
+        tm = [[None if math.isinf(v) else v for v in t] for t in want["trace_margins"]]
+        d = assert_trace_matches_up_to_low_margin(got["trace"], want["trace"], tm, wl.dtype, lim=lim)
+        if d is None:
+            assert got["tokens"] == want["tokens"] and got["stats"] == want["stats"]
+    ws = obild.generate(S, L, ids, 0.0, INF, n, mode="small")
+    assert_tokens_match_up_to_low_gap(ctx.generate(MODE_SMALL_ONLY, 0.0, INF, n)["tokens"], ws["tokens"],
+                                      [t[0] for t in ws["trace_margins"]], wl.dtype, lim=lim)
+    ctx.close()
+
+
 def test_bounded_wait_runs_out_and_context_recovers(torch_cuda):
     """Time-out path of the device-side waits: with bild_tuning.debug_skip_copies the fused attention kernel announces its
     weight copies to the barrier but does not issue them, so the bounded wait (a short limit here) runs out in every block.

@@ -303,6 +303,55 @@ def test_certificate_of_a_sampled_run(pair, alpha_fb, alpha_rb, max_draft):
     assert r["tokens"] != bild.generate(S, L, ids, alpha_fb, alpha_rb, n, max_draft=max_draft)["tokens"]
 
 
+# ---- early-exit configuration (Section 4.4) -------------------------------------------------
+def test_early_exit_model_is_the_prefix_of_the_decoder(pair):
+    """The early-exit small model shares everything with the large model and stops after its first layers: exiting
+    after the last layer is the model itself; exiting after layer 1 equals the full model whose later layers are
+    made the identity (their three output matrices set to zero)."""
+    wl, S, L, ids = pair
+    toks = [0, 5, 9, 3, 7]
+    full = L.forward_block(L.start(ids, 8), toks)
+    same = L.early_exit(L.s.n_layers)
+    assert np.array_equal(same.forward_block(same.start(ids, 8), toks), full)
+    t = gen_model(MODEL_SHAPES[wl.large], wl.seed, wl.dtype)
+    for l in range(1, L.s.n_layers):
+        for name in ("wo", "wco", "wfo"):
+            t[f"dec.{l}.{name}"] = np.zeros_like(t[f"dec.{l}.{name}"])
+    ident = Model(MODEL_SHAPES[wl.large], t, L.logit_scale)
+    e1 = L.early_exit(1)
+    z1 = e1.forward_block(e1.start(ids, 8), toks)
+    assert np.max(np.abs(z1 - ident.forward_block(ident.start(ids, 8), toks))) < 1e-10
+    assert np.max(np.abs(z1 - full)) > 1e-2                      # and it is not the full model
+    assert np.max(np.abs(e1.forward_full(e1.start(ids, 8), toks) - z1)) < 1e-10
+
+
+def test_bild_with_an_early_exit_draft_model(pair):
+    """Algorithm 1 with the small model = first layer of the large one: with the exit after the LAST layer the drafts
+    are the large model's own tokens, so nothing is ever rolled back for alpha_RB above their distances and the output
+    is the large model's greedy decode; with the exit after layer 1 the certificate of finished runs still holds."""
+    wl, S, L, ids = pair
+    ref = bild.generate(S, L, ids, 0.0, INF, wl.gen_len, mode="large")
+    same = L.early_exit(L.s.n_layers)
+    got = bild.generate(same, L, ids, 0.3, 50.0, wl.gen_len, max_draft=4)
+    assert got["tokens"] == ref["tokens"] and got["stats"]["rollbacks"] == 0
+    e1 = L.early_exit(1, logit_scale=2.0 * L.logit_scale)
+    r = bild.generate(e1, L, ids, 0.3, 16.0, wl.gen_len, max_draft=4)
+    y = [0] + r["tokens"]
+    ZS = e1.forward_full(e1.start(ids, len(y)), y[:-1])
+    ZL = L.forward_full(L.start(ids, len(y)), y[:-1])
+    owner = {}
+    for kind, pos, tok, k, m, val in r["trace"]:
+        if kind == bild.KIND_SMALL_ACCEPT:
+            owner[pos] = "S"
+        elif kind in (bild.KIND_VERIFY_OK, bild.KIND_ROLLBACK):
+            for q in [q for q in owner if q > pos]:
+                del owner[q]
+            owner[pos] = "L"
+    for j in range(1, len(y)):
+        assert y[j] == int(np.argmax(ZS[j - 1] if owner[j] == "S" else ZL[j - 1]))
+    assert r["stats"]["small_steps"] > 0 and r["stats"]["large_calls"] > 0
+
+
 # ---- closed forms --------------------------------------------------------------
 def test_softmax_identities():
     rng = np.random.default_rng(0)
