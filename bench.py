@@ -38,6 +38,18 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def measured_traffic(workload, kernel):
+    """DRAM bytes of one launch sequence of `kernel` from the committed ncu summary (profiles/dram_traffic.json:
+    dram__bytes_read.sum + dram__bytes_write.sum), or None where it was not measured for this workload and kernel."""
+    p = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(p):
+        return None
+    with open(p) as f:
+        t = json.load(f)
+    e = t.get(workload, {}).get(kernel)
+    return float(e["bytes"]) if e else None
+
+
 def pass_bytes(s, w_bytes, kv_bytes, cache_rows, enc_len, k):
     """Algorithmic bytes one decoder pass must read: every weight matrix once, the LM head,
     the self cache rows it attends to and the cross K/V (per layer), the k embedding rows."""
@@ -231,8 +243,12 @@ def main():
     t_small = ctx.time_pass(0, 1, cache_mid, 50)
     t_large = ctx.time_pass(1, k_mean, cache_mid, 20)
     t_large1 = ctx.time_pass(1, 1, cache_mid, 20)
-    b_small = pass_bytes(sS, wb, 4, cache_mid, wl.enc_len, 1)
-    b_large = pass_bytes(sL, wb, 4, cache_mid, wl.enc_len, k_mean)
+    # algorithmic bytes: keys / values at the weights' width (what the method has to move); the caches are kept in
+    # fp32 here, so the passes read somewhat more than that ("stored" figures below)
+    b_small = pass_bytes(sS, wb, wb, cache_mid, wl.enc_len, 1)
+    b_large = pass_bytes(sL, wb, wb, cache_mid, wl.enc_len, k_mean)
+    b_small_st = pass_bytes(sS, wb, 4, cache_mid, wl.enc_len, 1)
+    b_large_st = pass_bytes(sL, wb, 4, cache_mid, wl.enc_len, k_mean)
     peak, peak_kind = peaks()
     time_small_total = st["small_steps"] * t_small
     time_large_total = st["large_calls"] * t_large
@@ -247,17 +263,15 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights, f32 activations and KV cache" if wb == 2 else "f32",
         "data": "synthetic", "gpu_launches": int(launches),
         "config": dict(cfg_common, l2="inputs larger than L2: every step re-reads "
-                       f"{(b_large + b_small) / 1e6:.0f} MB of weights and K/V", parallelism="replicas only"),
+                       f"{(b_large_st + b_small_st) / 1e6:.0f} MB of weights and K/V", parallelism="replicas only"),
         "e2e": {"value": replicas.whole_job_rate(ntok * e2e_steps, world, ms_e2e), "unit": UNIT,
                 "h2d_bytes_per_step": int(ids_pinned.numel() * 4),
                 "d2h_bytes_per_step": int(4 * ntok + 24 * r["n_trace"] + 2 * 96)},
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": ("large-model block pass, k=%d" % k_mean) if dom_large else "small-model step",
                      "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "peak_kind": peak_kind,
-                     # dram__bytes_read+write of one block pass (k=5, cache 64) of the t5_sum pair: 191 of its 194
-                     # launches (one of the 144 linear layers, 2 MB, and the LM head, 65.8 MB algorithmic, were
-                     # outside the capture window); 814 MB algorithmic for the same launches
-                     "traffic": 831.2e6 if (dom_large and a.workload in ("t5_sum", "t5_long")) else None,
+                     "frac_with_fp32_kv_bytes": (b_large_st / t_large if dom_large else b_small_st / t_small) / 1e6 / peak,
+                     "traffic": measured_traffic(a.workload, ("large_block_pass_k%d" % k_mean) if dom_large else "small_step"),
                      "note": "a pass is a chain of dependent kernels replayed as one CUDA graph; its duration is "
                              "measured with CUDA events over back-to-back replays"},
         "passes": {"small_step_us": t_small * 1e3, "small_step_GBs": b_small / t_small / 1e6,

@@ -34,6 +34,7 @@ def main():
     ap.add_argument("--small", action="store_true")
     ap.add_argument("--dist", type=int, default=0, help="also time N single passes per point: median, p10, p90")
     ap.add_argument("--peak-gbs", type=float, default=0.0)
+    ap.add_argument("--tuning", default="", help="bild_tuning fields, e.g. pdl=0,fused=1")
     a = ap.parse_args()
     import torch
     assert torch.cuda.is_available(), "needs a CUDA device"
@@ -48,11 +49,16 @@ def main():
     if not peak:
         p = os.path.join(root, "MEASURED_PEAKS.json")
         peak = float(json.load(open(p))["hbm_gbs"]) if os.path.exists(p) else 6650.0
+    tf_peak = 1590.0
+    pk = os.path.join(root, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        tf_peak = float(json.load(open(pk)).get("bf16_tflops", tf_peak))
     ks = [int(x) for x in a.k.split(",")]
     caches = [int(x) for x in a.cache.split(",")]
     wl = WORKLOADS[a.workload]
+    tuning = {kv.split("=")[0]: int(kv.split("=")[1]) for kv in a.tuning.split(",") if kv}
     ctx, ids, _ = make_context(a.workload, g["scale_small"]["scale"], g["scale_large"]["scale"],
-                               max_dec_len=max(caches) + 16 + 1)
+                               max_dec_len=max(caches) + 16 + 1, tuning=tuning or None)
     ctx.encode(ids)
     wb = 2 if wl.dtype == "bf16" else 4
     sS, sL = MODEL_SHAPES[wl.small], MODEL_SHAPES[wl.large]
@@ -75,7 +81,7 @@ def main():
     for cache in caches:
         if a.small:
             ms = ctx.time_pass(0, 1, cache, a.iters)
-            b = pass_bytes(sS, wb, 4, cache, wl.enc_len, 1)
+            b = pass_bytes(sS, wb, wb, cache, wl.enc_len, 1)
             rec = {"pass": "small step", "k": 1, "cache": cache, "us": ms * 1e3, "GBs": b / ms / 1e6,
                    "frac_of_peak": b / ms / 1e6 / peak, "frac_of_nominal": b / ms / 1e6 / nominal, "bytes": b}
             rec.update(dist(0, 1, cache))
@@ -86,9 +92,14 @@ def main():
                 print(json.dumps(rec))
         for k in ks:
             ms = ctx.time_pass(1, k, cache, a.iters)
-            b = pass_bytes(sL, wb, 4, cache, wl.enc_len, k)
+            b = pass_bytes(sL, wb, wb, cache, wl.enc_len, k)
+            # tensor-pipe utilisation, derived: the pass's matrix products (2 k flops per weight; single-row passes run
+            # them on the plain ALUs) over its duration, against the measured dense bf16 rate
+            g = 3 if sL.ffn == "gated_gelu" else 2
+            flops = 2.0 * k * (sL.n_layers * (6 * sL.inner * sL.d_model + g * sL.d_model * sL.d_ff) + sL.vocab * sL.d_model)
             rec = {"pass": "large block pass", "k": k, "cache": cache, "us": ms * 1e3, "GBs": b / ms / 1e6,
-                   "frac_of_peak": b / ms / 1e6 / peak, "frac_of_nominal": b / ms / 1e6 / nominal, "bytes": b}
+                   "frac_of_peak": b / ms / 1e6 / peak, "frac_of_nominal": b / ms / 1e6 / nominal, "bytes": b,
+                   "tensor_util_derived": (flops / (ms * 1e-3) / 1e12 / tf_peak) if k > 1 else 0.0}
             rec.update(dist(1, k, cache))
             print(json.dumps(rec))
 
