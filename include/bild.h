@@ -191,6 +191,9 @@ typedef struct {
   int32_t spin_limit;        /* polls before a bounded device-side wait gives up with BILD_ERR_TIMEOUT (0: 2^20) */
   int32_t debug_skip_copies; /* 1: the fused attention kernel announces its weight copies but does not issue them, so
                               * that its bounded wait runs out (test of the time-out path; never set in production) */
+  int32_t attn_all_keys;     /* fused attention: while a head has at most this many keys (and they fit one staged chunk)
+                              * every block of the head's cluster attends over all of them, which saves the exchange
+                              * and merge of per-block partial results; 0: keys always split over the cluster */
 } bild_tuning;
 void bild_tuning_default(bild_tuning *t /*HOST out*/);
 /* bild_create with explicit switches; tuning == NULL means the defaults. */

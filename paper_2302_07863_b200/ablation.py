@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--fb", default="0.5,0.75,1.0,1.25,1.5", help="factors on the stored alpha_FB")
     ap.add_argument("--windows", default="3,4,5,6,7,8,9,10")
     ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--md", action="store_true", help="rows of a markdown table instead of JSON lines")
     a = ap.parse_args()
     import torch
     assert torch.cuda.is_available(), "needs a CUDA device"
@@ -57,13 +58,25 @@ def main():
                "fallback_rate": (st["fallbacks"] + st["forced"]) / max(1, n), "rollback_rate": st["rollbacks"] / max(1, n),
                "agree_with_large": sum(x == y for x, y in zip(r["tokens"], g["large_only"]["tokens"])) / max(1, n)}
         rec.update(extra)
-        print(json.dumps(rec), flush=True)
+        if a.md:
+            second = f"window {rec['window']} (alpha_RB {rec['alpha_rb']:.1f})" if "window" in rec else (
+                "inf" if rec["alpha_rb"] == "inf" else f"{rec['alpha_rb']:.1f}")
+            print(f"| {variant} | {rec.get('alpha_fb', 0):.3g} | {second} | {rec['tokens_per_s']:.0f} | "
+                  f"{rec['speedup_vs_large']:.2f}x | {100 * rec['fallback_rate']:.1f} % | "
+                  f"{100 * rec['rollback_rate']:.1f} % |", flush=True)
+        else:
+            print(json.dumps(rec), flush=True)
 
     ctx, ids, _ = make_context(a.workload, g["scale_small"]["scale"], g["scale_large"]["scale"])
     ctx.encode(ids)
     r, ms = timed(ctx, MODE_LARGE_ONLY, 0.0, inf)
     large_tps = len(r["tokens"]) / ms * 1e3
-    print(json.dumps({"variant": "large model alone", "tokens_per_s": large_tps}), flush=True)
+    if a.md:
+        print(f"Large model alone: {large_tps:.0f} tokens/s.\n")
+        print("| variant | alpha_FB | alpha_RB / window | tokens/s | speed-up vs large | fallback rate | rollback rate |")
+        print("|---|---|---|---|---|---|---|", flush=True)
+    else:
+        print(json.dumps({"variant": "large model alone", "tokens_per_s": large_tps}), flush=True)
     for f in [float(x) for x in a.fb.split(",")]:
         afb = th["alpha_fb"] * f
         r, ms = timed(ctx, MODE_BILD, afb, th["alpha_rb"])

@@ -120,7 +120,7 @@ struct Model {
   float* logits = nullptr;           // [MAXB][V] logits of the last pass (sampling variant only)
   bool fused = false;
   int sub_C = 1;                     // blocks per head (cluster size) of the attention sub-layers
-  int sub_kc = 16, sub_bias_len = 32;
+  AttnSubPlan sub_self{}, sub_cross{};   // chunk sizes of the attention sub-layers
   int sub_parts = 1;                 // launches the feed-forward sub-layer is split into
 };
 
@@ -170,6 +170,7 @@ struct bild_ctx {
   int slice_mode = 2;                // row-slice linear kernel: 0 off, 1 block passes, 2 block and single-row passes
   int sms = 0;
   size_t slice_smem_set = 0;
+  int attn_all_keys = 128;           // fused attention: caches up to this many keys are attended by every rank of a head
   bool unit_attn = true;             // decoder attention on the 256-thread chunked kernel
   bool uattn_smem_set = false;
   bool enc_attn_mma = true;          // encoder self-attention on the mma.sync kernel (d_kv = 64)
@@ -649,12 +650,10 @@ int setup_fused(bild_ctx* c, Model& m) {
     cudaGetLastError();
     return BILD_OK;
   }
-  const int per_rank = (std::max(cap, ecap) + C - 1) / C;
-  int kc = std::min(64, (per_rank + 15) / 16 * 16);   // at most 64: a chunk's scores take one turn of the block
-  const int bias_len = ((cap + C - 1) / C + MAXB + 8 + 3) / 4 * 4;
-  while (kc > 16 && attn_sub_layout(d, dkv, 3, C, SUB_MB, kc, bias_len).total > smem_max) kc -= 16;
-  if (attn_sub_layout(d, dkv, 3, C, SUB_MB, kc, bias_len).total > smem_max ||
-      attn_sub_layout(d, dkv, 1, C, SUB_MB, kc, bias_len).total > smem_max) return BILD_OK;
+  const int all_keys = c->attn_all_keys;
+  const AttnSubPlan ps = attn_sub_plan(d, dkv, 3, C, cap, all_keys, SUB_HALF_SM, smem_max);
+  const AttnSubPlan pc = attn_sub_plan(d, dkv, 1, C, ecap, all_keys, SUB_HALF_SM, smem_max);
+  if (!ps.ok || !pc.ok) return BILD_OK;
   int parts = std::max(1, c->sub_parts_want);
   const int nmat = gated ? 2 : 1;
   while (parts <= 8 && (ffn_sub_rows(F, c->sms * parts) * nmat > SUB_MAX_ROWS || ffn_sub_rows(F, c->sms * parts) > SUB_FO_REGS ||
@@ -673,7 +672,7 @@ int setup_fused(bild_ctx* c, Model& m) {
     (*c->cnt)++;
   }
   CUDA_TRY(c, cudaGetLastError());
-  m.sub_C = C; m.sub_kc = kc; m.sub_bias_len = bias_len; m.sub_parts = parts;
+  m.sub_C = C; m.sub_self = ps; m.sub_cross = pc; m.sub_parts = parts;
   m.fused = true;
   return BILD_OK;
 }
@@ -712,19 +711,21 @@ int fused_layers(bild_ctx* c, Model& m, int MB) {
     const size_t kvoff = (size_t)l * H * dkv;
     AttnSubArgs a{};
     a.desc = m.desc; a.eps = mc.ln_eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
-    a.kc_keys = m.sub_kc; a.bias_len = m.sub_bias_len; a.mb = MB; a.err = &c->st->err;
+    a.mb = MB; a.err = &c->st->err;
     a.spin = c->spin_limit; a.skip_copies = c->debug_skip_copies ? 1 : 0;
     a.n_keys_dev = c->enc_len_dev;
     // S1-S3 / L1-L3
     a.x_in = m.x; a.x_out = m.xb; a.x_zero = m.xc; a.gain = (const float*)w.ln1;
     a.Wp = (const __nv_bfloat16*)w.wqkv; a.Wo = (const __nv_bfloat16*)w.wo;
     a.kc = m.selfK + kvoff * cap; a.vc = m.selfV + kvoff * cap; a.cap = cap; a.bias = m.dec_bias; a.bias_ld = cap; a.self = 1;
+    a.kc_keys = m.sub_self.kc; a.bias_len = m.sub_self.bias_len; a.red_keys = m.sub_self.red_keys;
     a.L = attn_sub_layout(d, dkv, 3, C, MB, a.kc_keys, a.bias_len);
     CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
     // S4-S6 / L4-L6
     a.x_in = m.xb; a.x_out = m.xc; a.x_zero = m.x; a.gain = (const float*)w.ln2;
     a.Wp = (const __nv_bfloat16*)w.wcq; a.Wo = (const __nv_bfloat16*)w.wco;
     a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.bias = nullptr; a.bias_ld = 0; a.self = 0;
+    a.kc_keys = m.sub_cross.kc; a.bias_len = m.sub_cross.bias_len; a.red_keys = m.sub_cross.red_keys;
     a.L = attn_sub_layout(d, dkv, 1, C, MB, a.kc_keys, a.bias_len);
     CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
     // S7-S8 / L7-L8
@@ -1249,6 +1250,7 @@ void bild_tuning_default(bild_tuning* t) {
   t->host_loop = 0; t->pdl = 1; t->fused = 2; t->ffn_parts = 0; t->block_simt = 0; t->slice_mode = 2;
   t->slice_min_kb = 3000; t->slice_mma_min = 3; t->slice_head = 2; t->slice_head_min_mb = 32; t->unit_attn = 1;
   t->umma = 1; t->enc_gemm = 1; t->enc_attn_mma = 1; t->enc_parallel = 1; t->spin_limit = 0; t->debug_skip_copies = 0;
+  t->attn_all_keys = 128;
 }
 
 int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_weights* large_w, void* workspace,
@@ -1292,6 +1294,7 @@ int bild_create_tuned(const bild_config* cfg, const bild_weights* small_w, const
     c->enc_parallel = t.enc_parallel != 0;
     c->spin_limit = t.spin_limit > 0 ? (unsigned)t.spin_limit : SPIN_LIMIT;
     c->debug_skip_copies = t.debug_skip_copies != 0;
+    c->attn_all_keys = std::min(128, std::max(0, t.attn_all_keys));
   }
   {
     int dev = 0;
@@ -1722,10 +1725,9 @@ int bild_op_attn_sublayer(int self, const void* Wp, const void* Wo, const float*
   const int MB = M == 1 ? 1 : SUB_MB, I = H * dkv, P = self ? 3 : 1;
   int smem_max = 0, dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return BILD_ERR_CUDA;
-  int kc_keys = std::min(64, ((cap + C - 1) / C + 15) / 16 * 16);
-  const int bias_len = ((cap + C - 1) / C + MAXB + 8 + 3) / 4 * 4;
-  while (kc_keys > 16 && attn_sub_layout(d, dkv, P, C, MB, kc_keys, bias_len).total > smem_max) kc_keys -= 16;
-  if (attn_sub_layout(d, dkv, P, C, MB, kc_keys, bias_len).total > smem_max) return BILD_ERR_CAPACITY;
+  const AttnSubPlan pl = attn_sub_plan(d, dkv, P, C, cap, 128, SUB_HALF_SM, smem_max);
+  if (!pl.ok) return BILD_ERR_CAPACITY;
+  const int kc_keys = pl.kc, bias_len = pl.bias_len;
   OpScratch o = op_scratch(scratch, d);
   bild_ctx tmp;
   tmp.stream = s;
@@ -1739,7 +1741,7 @@ int bild_op_attn_sublayer(int self, const void* Wp, const void* Wo, const float*
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess) return BILD_ERR_CUDA;
   AttnSubArgs a{};
   a.desc = o.desc; a.eps = eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
-  a.kc_keys = kc_keys; a.bias_len = bias_len; a.mb = MB; a.err = o.err; a.spin = SPIN_LIMIT; a.skip_copies = 0;
+  a.kc_keys = kc_keys; a.bias_len = bias_len; a.red_keys = pl.red_keys; a.mb = MB; a.err = o.err; a.spin = SPIN_LIMIT; a.skip_copies = 0;
   a.n_keys_dev = o.nkeys; a.x_in = x_in; a.x_out = x_out; a.x_zero = o.zero; a.gain = gain;
   a.Wp = (const __nv_bfloat16*)Wp; a.Wo = (const __nv_bfloat16*)Wo; a.kc = kc; a.vc = vc; a.cap = cap;
   a.bias = bias_by_dist; a.bias_ld = cap; a.self = self ? 1 : 0;

@@ -25,6 +25,7 @@ constexpr int SUB_PSUM = SL_PSUM;   // bytes of partial sums of sl_items / sl_mm
 constexpr int SUB_RECPAD = 4;       // record of a rank and row = [max, sum, -, -, values[d_kv]]
 constexpr int SUB_MAX_ROWS = 4 * SL_QUADS;   // weight rows of one block and phase (limit of sl_items / sl_mma)
 constexpr int SUB_FO_REGS = 32;              // rows of the transposed W_fo a single-row block keeps in registers
+constexpr int SUB_HALF_SM = 113 * 1024;      // shared memory of a block that leaves room for a second one on the SM
 constexpr int SUB_MB = 8;                    // token rows of the block variant (one 8-token tile of the tensor-core instruction)
 
 struct SubShared {
@@ -177,7 +178,8 @@ struct AttnSubArgs {
   const int* n_keys_dev;     // cross: encoder positions
   int self;
   int d, I, H, dkv, dkv_shift, C, c_shift;
-  int kc_keys;               // keys per staged chunk (<= 64)
+  int kc_keys;               // keys per staged chunk
+  int red_keys;              // up to this many keys every rank attends over ALL keys of the head (no second exchange)
   int bias_len;              // floats reserved for the staged bias
   int mb;                    // token rows the shared memory is sized for
   unsigned spin;             // polls of the weight barrier before the kernel gives up
@@ -192,7 +194,7 @@ struct AttnSubArgs {
 inline AttnSubLayout attn_sub_layout(int d, int dkv, int P, int C, int mb, int kc, int bias_len) {
   AttnSubLayout L;
   const int npr = (P * dkv + C - 1) / C, no = (d + C - 1) / C;
-  const int wq_b = sub_up16(npr * (d * 2 + SL_WPAD)), kv_b = sub_up16(2 * kc * sub_kv_stride(dkv) * 4);
+  const int wq_b = sub_up16(npr * (d * 2 + SL_WPAD)), kv_b = sub_up16(kc * (sub_kv_stride(dkv) + dkv + 4) * 4);
   int off = 0;
   // block variant, self-attention: the keys / values of the rank are staged where the projection rows were, once the
   // products are done (they depend on the cache position anyway); otherwise they have an area of their own and the
@@ -205,7 +207,7 @@ inline AttnSubLayout attn_sub_layout(int d, int dkv, int P, int C, int mb, int k
   else { L.kv = off; off += kv_b; }
   L.qkv = off; off += sub_up16(mb * P * dkv * 4);
   // partial sums of the products; afterwards the merged head output and this rank's record
-  const int ps_b = mb == 1 ? SUB_PSUM : 8 * 128 * 4, after_b = sub_up16(mb * dkv * 4) + sub_up16(mb * (dkv + SUB_RECPAD) * 4);
+  const int ps_b = mb == 1 ? ((npr + 3) / 4) * 8 * 32 * 4 : 8 * 128 * 4, after_b = sub_up16(mb * dkv * 4) + sub_up16(mb * (dkv + SUB_RECPAD) * 4);
   L.psum = off; L.sa = off; L.recloc = off + sub_up16(mb * dkv * 4);
   off += sub_up16(ps_b > after_b ? ps_b : after_b);
   L.probs = off; off += sub_up16(mb * (kc + 4) * 4);
@@ -217,6 +219,26 @@ inline AttnSubLayout attn_sub_layout(int d, int dkv, int P, int C, int mb, int k
   L.sh = off; off += sub_up16((int)sizeof(SubShared));
   L.total = off;
   return L;
+}
+
+// Chunk size, bias room and the key count up to which the ranks attend redundantly, for a cache of keys_cap keys.
+// `all_keys` > 0 asks for a chunk that holds up to that many keys so that short caches need no second exchange; the
+// chunk shrinks until the single-row and the block layout both stay under `prefer` bytes (half an SM), else under `limit`.
+struct AttnSubPlan { int kc, bias_len, red_keys; bool ok; };
+inline AttnSubPlan attn_sub_plan(int d, int dkv, int P, int C, int keys_cap, int all_keys, int prefer, int limit) {
+  AttnSubPlan pl;
+  const int per_rank = (keys_cap + C - 1) / C;
+  const int need = std::min(64, sub_up16(per_rank)), want = std::min(128, sub_up16(std::min(all_keys, keys_cap)));
+  auto blen = [&](int kc) { return P == 3 ? (std::max(per_rank, kc) + MAXB + 8 + 3) / 4 * 4 : 4; };
+  auto fits = [&](int kc, int lim) {
+    return attn_sub_layout(d, dkv, P, C, 1, kc, blen(kc)).total <= lim && attn_sub_layout(d, dkv, P, C, SUB_MB, kc, blen(kc)).total <= lim;
+  };
+  int kc = std::max(need, want);
+  while (kc > need && !fits(kc, prefer)) kc -= 16;
+  while (kc > 16 && !fits(kc, limit)) kc -= 16;
+  pl.kc = kc; pl.bias_len = blen(kc); pl.ok = fits(kc, limit);
+  pl.red_keys = all_keys > 0 ? kc : 0;
+  return pl;
 }
 
 // ONE: a single token row (the small model's step, the large model's single-row pass): SIMT products, no loops over rows.
@@ -301,10 +323,14 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
       sub_cp16(sV + (size_t)jj * vst + u, Vh + (size_t)(c0 + jj) * dkv + u);
     }
   };
+  // Few keys: every rank attends over all of them (the keys of the cache come from the L2, those of this pass from the
+  // first exchange anyway), which costs a fraction of a microsecond and saves the exchange of the records and their merge.
   int n_keys = 0, j0 = 0, j1 = 0;
+  bool red = false;
   if (!a.self) {   // the encoder keys are static: the first chunk is requested before the wait as well
     n_keys = min(*a.n_keys_dev, a.cap);
-    j0 = (r * n_keys) >> a.c_shift; j1 = ((r + 1) * n_keys) >> a.c_shift;
+    red = n_keys <= a.red_keys;
+    j0 = red ? 0 : (r * n_keys) >> a.c_shift; j1 = red ? n_keys : ((r + 1) * n_keys) >> a.c_shift;
     stage_cached(j0, min(j1, j0 + a.kc_keys));
   }
   SUB_STAMP();            // P2: loads issued, cross keys requested
@@ -315,7 +341,8 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
   const int k = ONE ? 1 : min(a.desc->k, a.mb), pos0 = a.desc->pos0;
   if (a.self) {
     n_keys = min(pos0 + k, a.cap);
-    j0 = (r * n_keys) >> a.c_shift; j1 = ((r + 1) * n_keys) >> a.c_shift;
+    red = n_keys <= a.red_keys;
+    j0 = red ? 0 : (r * n_keys) >> a.c_shift; j1 = red ? n_keys : ((r + 1) * n_keys) >> a.c_shift;
     if (!a.L.kv_late) stage_cached(j0, min(min(j1, pos0), j0 + a.kc_keys));
   }
   // relative-position bias of the distances this rank meets
@@ -404,8 +431,10 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
     __syncthreads();
     SUB_STAMP();          // B1: keys / values staged
     {   // scores: four threads per key, one channel quarter each (16-byte units interleaved over the quarters); the
-        // quarter of the key stays in registers while the rows go by
-      const int jj = tid >> 2, qt = tid & 3;
+        // quarter of the key stays in registers while the rows go by; 64 keys per turn
+      const int qt = tid & 3;
+#pragma unroll 1
+      for (int jj = tid >> 2; jj < ((nk + 63) & ~63); jj += SUB_THREADS / 4) {
       const bool valid = jj < nk;
       float4 kq[4];
 #pragma unroll
@@ -432,6 +461,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
           }
           sP[(size_t)m * pst + jj] = s;
         }
+      }
       }
     }
     __syncthreads();
@@ -532,6 +562,14 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
   }
   __syncthreads();
   SUB_STAMP();            // 7: attention over this rank's keys
+  if (red) {   // this rank's record covers every key: the head output is its values over its sum
+#pragma unroll 1
+    for (int o = tid; o < k * dkv; o += SUB_THREADS) {
+      const int m = o >> a.dkv_shift, cc = o & (dkv - 1);
+      sA[(size_t)m * dkv + cc] = recLoc[(size_t)m * recst + SUB_RECPAD + cc] / recLoc[(size_t)m * recst + 1];
+    }
+    SUB_STAMP(); SUB_STAMP(); SUB_STAMP();
+  } else {
   {   // the record goes to every block of the cluster: one 16-byte store per thread and turn
     const int q4 = (k * recst) >> 2, tot = q4 << a.c_shift;
 #pragma unroll 1
@@ -566,8 +604,9 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
     }
     sA[(size_t)m * dkv + cc] = num / den;
   }
-  __syncthreads();
   SUB_STAMP();            // 10: merge
+  }
+  __syncthreads();
   if (ONE) {   // output projection, one row: the thread's channels of rows g and g + 8, then the four threads of a row add up
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
