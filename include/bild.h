@@ -161,10 +161,9 @@ int bild_query_workspace(const bild_config *cfg /*HOST*/, size_t *bytes /*HOST o
 /* Build a context.  `workspace` is DEVICE memory, 256-byte aligned, at least
  * bild_query_workspace bytes, caller-owned, used exclusively by this context until
  * bild_destroy.  `cuda_stream` is a cudaStream_t (NULL = default stream).  Device work done
- * here, on that stream, with a synchronisation before returning: the workspace is cleared,
- * the relative-position bias tables are expanded by distance, and (bf16 configurations) each
- * decoder layer's feed-forward output matrix is transposed into the workspace for the fused
- * sub-layer kernels.  Errors: ARG, WORKSPACE, CUDA. */
+ * here, on that stream, with a synchronisation before returning: the workspace is cleared
+ * and the relative-position bias tables are expanded by distance.  The weights are read in
+ * place by every kernel (no copies, no re-layout).  Errors: ARG, WORKSPACE, CUDA. */
 int bild_create(const bild_config *cfg /*HOST*/, const bild_weights *small_w /*HOST*/,
                 const bild_weights *large_w /*HOST*/, void *workspace /*DEVICE*/,
                 size_t workspace_bytes, void *cuda_stream, bild_ctx **out /*HOST out*/);

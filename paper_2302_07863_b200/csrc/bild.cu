@@ -116,10 +116,11 @@ struct Model {
   int index = 0;   // 0 small, 1 large
   // fused sub-layer kernels (bf16 only): two more residual-stream buffers, W_fo transposed per layer
   float *xb = nullptr, *xc = nullptr;
-  __nv_bfloat16* wfoT = nullptr;     // [layers][F][d]
   float* logits = nullptr;           // [MAXB][V] logits of the last pass (sampling variant only)
   bool fused = false;
   int sub_C = 1;                     // blocks per head (cluster size) of the attention sub-layers
+  uint4* wfo_one = nullptr;          // [layers][F / 8][d] W_fo in the load order of the fused feed-forward kernels
+  uint4* wfo_blk = nullptr;          // [layers][F / 8][pack_wfo_dpad(d)]
   AttnSubPlan sub_self{}, sub_cross{};   // chunk sizes of the attention sub-layers
   int sub_parts = 1;                 // launches the feed-forward sub-layer is split into
 };
@@ -285,7 +286,11 @@ void plan(bild_ctx* c, Bump& b) {
     m.logits = b.take<float>((size_t)MAXB * mc.vocab);
     m.xb = b.take<float>((size_t)MAXB * mc.d_model);
     m.xc = b.take<float>((size_t)MAXB * mc.d_model);
-    m.wfoT = b.take<__nv_bfloat16>(cfg.dtype == BILD_BF16 ? (size_t)mc.n_layers * mc.d_ff * mc.d_model : 0);
+    {   // W_fo of every decoder layer in the load order of the fused feed-forward kernels (two orders: one row, blocks)
+      const size_t units = cfg.dtype == BILD_BF16 && mc.d_ff % 8 == 0 ? (size_t)mc.n_layers * (mc.d_ff / 8) : 0;
+      m.wfo_one = b.take<uint4>(units * mc.d_model);
+      m.wfo_blk = b.take<uint4>(units * pack_wfo_dpad(mc.d_model));
+    }
   }
   const size_t ecap16 = (size_t)(ecap + MAXB - 1) / MAXB * MAXB;   // whole blocks of MAXB rows
   const size_t ecap128 = (size_t)(ecap + EG_TOK - 1) / EG_TOK * EG_TOK;   // whole tiles of 128 tokens
@@ -637,7 +642,7 @@ int setup_fused(bild_ctx* c, Model& m) {
   const bool gated = mc.ffn_kind == BILD_FFN_GATED_GELU;
   int C = 8;
   while (C > 1 && (H * C > c->sms || d % (4 * C))) C >>= 1;
-  if (d % (4 * C) || d > 1024 || dkv > 64 || dkv < 16 || d / C > SUB_THREADS / 2) return BILD_OK;
+  if (d % (4 * C) || d % 16 || F % 8 || d > 1024 || dkv > 64 || dkv < 16 || d / C > SUB_THREADS / 2) return BILD_OK;
   if ((3 * dkv + C - 1) / C > SUB_MAX_ROWS) return BILD_OK;
   auto aligned = [](const void* p) { return ((uintptr_t)p & 15) == 0; };
   for (int l = 0; l < mc.n_layers; ++l) {
@@ -667,8 +672,8 @@ int setup_fused(bild_ctx* c, Model& m) {
     return BILD_OK;
   }
   for (int l = 0; l < mc.n_layers; ++l) {
-    transpose_bf16_kernel<<<dim3((F + 31) / 32, (d + 31) / 32), dim3(32, 8), 0, c->stream>>>(
-        (const __nv_bfloat16*)m.dec[l].wfo, m.wfoT + (size_t)l * F * d, d, F);
+    pack_wfo_kernel<<<F / 8, 256, 0, c->stream>>>((const __nv_bfloat16*)m.dec[l].wfo, m.wfo_one + (size_t)l * (F / 8) * d,
+                                                  m.wfo_blk + (size_t)l * (F / 8) * pack_wfo_dpad(d), d, F);
     (*c->cnt)++;
   }
   CUDA_TRY(c, cudaGetLastError());
@@ -711,7 +716,7 @@ int fused_layers(bild_ctx* c, Model& m, int MB) {
     const size_t kvoff = (size_t)l * H * dkv;
     AttnSubArgs a{};
     a.desc = m.desc; a.eps = mc.ln_eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
-    a.mb = MB; a.err = &c->st->err;
+    a.mb = MB; a.err = &c->st->err; a.x_rows = MAXB;
     a.spin = c->spin_limit; a.skip_copies = c->debug_skip_copies ? 1 : 0;
     a.n_keys_dev = c->enc_len_dev;
     // S1-S3 / L1-L3
@@ -730,9 +735,10 @@ int fused_layers(bild_ctx* c, Model& m, int MB) {
     CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
     // S7-S8 / L7-L8
     FfnSubArgs f{};
+    f.x_rows = MAXB;
     f.desc = m.desc; f.eps = mc.ln_eps; f.d = d; f.F = F; f.gated = gated ? 1 : 0; f.mb = MB; f.spin = c->spin_limit;
     f.err = &c->st->err; f.x_in = m.xc; f.x_out = m.x; f.gain = (const float*)w.ln3;
-    f.Wi0 = (const __nv_bfloat16*)w.wi0; f.Wi1 = (const __nv_bfloat16*)w.wi1; f.WfoT = m.wfoT + (size_t)l * F * d;
+    f.Wi0 = (const __nv_bfloat16*)w.wi0; f.Wi1 = (const __nv_bfloat16*)w.wi1; f.Wfo1 = m.wfo_one + (size_t)l * (F / 8) * d; f.Wfo8 = m.wfo_blk + (size_t)l * (F / 8) * pack_wfo_dpad(d);
     f.nparts = m.sub_parts;
     f.L = ffn_sub_layout(d, F, gated, c->sms * m.sub_parts, c->sms, MB);
     for (int p = 0; p < m.sub_parts; ++p) {
@@ -1666,13 +1672,13 @@ int op_finish(cudaStream_t s, const OpScratch& o) {   // the kernels' own error 
 
 size_t bild_op_sublayer_scratch_bytes(int d, int F) {
   return align_up(sizeof(CallDesc), 256) + 256 + align_up((size_t)MAXB * std::max(d, 8) * sizeof(float), 256) +
-         align_up((size_t)std::max(F, 0) * d * 2, 256) + 256;
+         align_up((size_t)(std::max(F, 0) / 8) * d * 16, 256) + align_up((size_t)(std::max(F, 0) / 8) * pack_wfo_dpad(d) * 16, 256) + 256;
 }
 
 int bild_op_ffn_sublayer(const void* Wi0, const void* Wi1, const void* Wfo, const float* gain, float eps, const float* x_in,
                          float* x_out, int M, int d, int F, int parts, void* scratch, void* cuda_stream) {
   if (!Wi0 || !Wfo || !gain || !x_in || !x_out || !scratch) return BILD_ERR_ARG;
-  if (M < 1 || M > SUB_MB || d < 8 || d % 8 || d > 1024 || F < 8 || F % 8 || parts < 0 || parts > 8) return BILD_ERR_ARG;
+  if (M < 1 || M > SUB_MB || d < 16 || d % 16 || d > 1024 || F < 8 || F % 8 || parts < 0 || parts > 8) return BILD_ERR_ARG;
   if ((uintptr_t)scratch % 256) return BILD_ERR_WORKSPACE;
   const int sms = op_sms();
   if (sms < 1) return BILD_ERR_CUDA;
@@ -1686,7 +1692,9 @@ int bild_op_ffn_sublayer(const void* Wi0, const void* Wi1, const void* Wfo, cons
                      ffn_sub_layout(d, F, gated, sms * np, sms, MB).total > smem_max)) ++np;
   if (np > 8) return BILD_ERR_CAPACITY;
   OpScratch o = op_scratch(scratch, d);
-  __nv_bfloat16* WfoT = (__nv_bfloat16*)o.rest;
+  uint4* wfo_one = (uint4*)o.rest;
+  uint4* wfo_blk = (uint4*)(o.rest + align_up((size_t)(F / 8) * d * 16, 256));
+  pack_wfo_kernel<<<F / 8, 256, 0, s>>>((const __nv_bfloat16*)Wfo, wfo_one, wfo_blk, d, F);
   bild_ctx tmp;
   tmp.stream = s;
   tmp.use_pdl = false;
@@ -1694,12 +1702,11 @@ int bild_op_ffn_sublayer(const void* Wi0, const void* Wi1, const void* Wfo, cons
   set_desc_at_kernel<<<1, 1, 0, s>>>(o.desc, M, 0, t);
   if (cudaMemsetAsync(o.err, 0, 8, s) != cudaSuccess) return BILD_ERR_CUDA;
   if (cudaMemsetAsync(x_out, 0, (size_t)M * d * sizeof(float), s) != cudaSuccess) return BILD_ERR_CUDA;   // the kernel accumulates into it
-  transpose_bf16_kernel<<<dim3((F + 31) / 32, (d + 31) / 32), dim3(32, 8), 0, s>>>((const __nv_bfloat16*)Wfo, WfoT, d, F);
   auto kern = MB == 1 ? ffn_sub_kernel<true> : ffn_sub_kernel<false>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess) return BILD_ERR_CUDA;
   FfnSubArgs f{};
   f.desc = o.desc; f.eps = eps; f.d = d; f.F = F; f.gated = gated ? 1 : 0; f.mb = MB; f.spin = SPIN_LIMIT; f.err = o.err;
-  f.x_in = x_in; f.x_out = x_out; f.gain = gain; f.Wi0 = (const __nv_bfloat16*)Wi0; f.Wi1 = (const __nv_bfloat16*)Wi1; f.WfoT = WfoT;
+  f.x_in = x_in; f.x_rows = M; f.x_out = x_out; f.gain = gain; f.Wi0 = (const __nv_bfloat16*)Wi0; f.Wi1 = (const __nv_bfloat16*)Wi1; f.Wfo1 = wfo_one; f.Wfo8 = wfo_blk;
   f.nparts = np; f.L = ffn_sub_layout(d, F, gated, sms * np, sms, MB);
   for (int p = 0; p < np; ++p) {
     f.part = p; f.seed = p == 0 ? 1 : 0; f.x_zero = p == 0 ? o.zero : nullptr;
@@ -1742,7 +1749,7 @@ int bild_op_attn_sublayer(int self, const void* Wp, const void* Wo, const float*
   AttnSubArgs a{};
   a.desc = o.desc; a.eps = eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
   a.kc_keys = kc_keys; a.bias_len = bias_len; a.red_keys = pl.red_keys; a.mb = MB; a.err = o.err; a.spin = SPIN_LIMIT; a.skip_copies = 0;
-  a.n_keys_dev = o.nkeys; a.x_in = x_in; a.x_out = x_out; a.x_zero = o.zero; a.gain = gain;
+  a.n_keys_dev = o.nkeys; a.x_in = x_in; a.x_rows = M; a.x_out = x_out; a.x_zero = o.zero; a.gain = gain;
   a.Wp = (const __nv_bfloat16*)Wp; a.Wo = (const __nv_bfloat16*)Wo; a.kc = kc; a.vc = vc; a.cap = cap;
   a.bias = bias_by_dist; a.bias_ld = cap; a.self = self ? 1 : 0;
   a.L = attn_sub_layout(d, dkv, P, C, MB, kc_keys, bias_len);

@@ -136,9 +136,12 @@ __device__ __forceinline__ void sl_mma(const unsigned char* sW, int rowst, int n
   const float* xb[NT];
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) xb[nt] = Xs + (size_t)min(nt * 8 + g, mg - 1) * xst + 2 * t;
-  float c[NT][4];
+  float c[NT][4], e[NT][4];   // products with the heads and with the remainders of the activations: two independent chains
 #pragma unroll
-  for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+  for (int nt = 0; nt < NT; ++nt) {
+    c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+    e[nt][0] = e[nt][1] = e[nt][2] = e[nt][3] = 0.f;
+  }
 #pragma unroll 4
   for (int st = s0; st < s1; ++st) {
     const int k0 = st << 4;
@@ -158,13 +161,13 @@ __device__ __forceinline__ void sl_mma(const unsigned char* sW, int rowst, int n
                    : "+f"(c[nt][0]), "+f"(c[nt][1]), "+f"(c[nt][2]), "+f"(c[nt][3])
                    : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(h0), "r"(h1));
       asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                   : "+f"(c[nt][0]), "+f"(c[nt][1]), "+f"(c[nt][2]), "+f"(c[nt][3])
+                   : "+f"(e[nt][0]), "+f"(e[nt][1]), "+f"(e[nt][2]), "+f"(e[nt][3])
                    : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(l0), "r"(l1));
     }
   }
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt)
-    *reinterpret_cast<float4*>(psum + ((size_t)(warp * NT + nt) * 32 + lane) * 4) = make_float4(c[nt][0], c[nt][1], c[nt][2], c[nt][3]);
+    *reinterpret_cast<float4*>(psum + ((size_t)(warp * NT + nt) * 32 + lane) * 4) = make_float4(c[nt][0] + e[nt][0], c[nt][1] + e[nt][1], c[nt][2] + e[nt][2], c[nt][3] + e[nt][3]);
 }
 
 __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {

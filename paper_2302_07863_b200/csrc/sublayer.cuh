@@ -8,8 +8,9 @@
 //     per-rank (max, sum, weighted values) records are exchanged the same way, and every rank
 //     multiplies the merged head output with its share of the rows of W_o's column slice;
 //   * ffn_sub_kernel: x_out = x_in + W_fo * act(W_i * rms_norm(x_in))   (S7-S8 / L7-L8).  Block b owns a
-//     slice of d_ff: the rows of W_i (and of the gate matrix) and the matching rows of the transposed
-//     W_fo, so the hidden activations never leave the block.
+//     slice of d_ff (a multiple of 8 rows): the rows of W_i (and of the gate matrix) in shared memory and the
+//     matching columns of W_fo in registers (from a copy laid out in load order), so the hidden activations never
+//     leave the block.
 // Both kernels produce partial sums over heads / slices of d_ff of the d_model outputs.  They are added
 // into x_out with vector reductions at the L2 (red.global.add); x_out was zeroed by the kernel before the
 // previous one, one designated block adds x_in (the residual term), and every kernel zeroes the buffer
@@ -24,7 +25,7 @@ constexpr int SUB_THREADS = 256;
 constexpr int SUB_PSUM = SL_PSUM;   // bytes of partial sums of sl_items / sl_mma
 constexpr int SUB_RECPAD = 4;       // record of a rank and row = [max, sum, -, -, values[d_kv]]
 constexpr int SUB_MAX_ROWS = 4 * SL_QUADS;   // weight rows of one block and phase (limit of sl_items / sl_mma)
-constexpr int SUB_FO_REGS = 32;              // rows of the transposed W_fo a single-row block keeps in registers
+constexpr int SUB_FO_REGS = 32;              // most rows of d_ff a block takes: its columns of W_fo fill 64 registers of a thread
 constexpr int SUB_HALF_SM = 113 * 1024;      // shared memory of a block that leaves room for a second one on the SM
 constexpr int SUB_MB = 8;                    // token rows of the block variant (one 8-token tile of the tensor-core instruction)
 
@@ -100,18 +101,32 @@ __device__ __forceinline__ float sub_total(const float* psum, int row, int m, in
   return t;
 }
 
-// Token rows, after the dependency wait (d <= 1024: one 128-bit load per thread and row, all rows of a turn in
-// flight together): x * gain into Xs, 1 / rms into sh->inv (returned for the single row of ONE).  The raw values of the
-// columns [seed0, seed1) (multiples of 4) also go to sSeed[m][column - seed0]: the residual term the block adds.
+// Token rows, after the dependency wait (d <= 1024: one 128-bit load per thread and row).  The loads are issued first
+// thing after the wait, for all rows the variant can take (which rows count is known only once the call descriptor
+// has been read, a round trip to the L2 of its own); sub_rows_finish then writes x * gain into Xs and 1 / rms into
+// sh->inv (returned for the single row of ONE).  The raw values of the columns [seed0, seed1) (multiples of 4) also go
+// to sSeed[m][column - seed0]: the residual term the block adds.
 template <bool ONE>
-__device__ __forceinline__ float sub_load_rows(const float* __restrict__ x_in, int k, int d, float4 g, float eps, float* Xs, int xst,
-                                               SubShared* sh, float* sSeed, int seed0, int seed1, int tid, int lane, int warp) {
+struct SubRows { float4 v[ONE ? 1 : SUB_MB]; };
+
+template <bool ONE>
+__device__ __forceinline__ void sub_rows_issue(const float* __restrict__ x_in, int rows, int d, int tid, SubRows<ONE>& rw) {
+  if (tid * 4 < d) {   // rows: how many rows of x_in exist (a launch parameter, known without a load)
+#pragma unroll
+    for (int i = 0; i < (ONE ? 1 : SUB_MB); ++i)
+      if (i < rows) rw.v[i] = __ldcg(reinterpret_cast<const float4*>(x_in + (size_t)i * d) + tid);
+  }
+}
+
+template <bool ONE>
+__device__ __forceinline__ float sub_rows_finish(const SubRows<ONE>& rw, int k, int d, float4 g, float eps, float* Xs, int xst,
+                                                 SubShared* sh, float* sSeed, int seed0, int seed1, int tid, int lane, int warp) {
   const int d4 = d >> 2, c = tid * 4;
   const bool on = tid < d4, sd = c >= seed0 && c < seed1;
   if (ONE) {
     float ss = 0.f;
     if (on) {
-      float4 w = __ldcg(reinterpret_cast<const float4*>(x_in) + tid);
+      float4 w = rw.v[0];
       ss = w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
       if (sd) *reinterpret_cast<float4*>(sSeed + (c - seed0)) = w;
       w.x *= g.x; w.y *= g.y; w.z *= g.z; w.w *= g.w;
@@ -124,18 +139,13 @@ __device__ __forceinline__ float sub_load_rows(const float* __restrict__ x_in, i
 #pragma unroll
     for (int wv = 0; wv < 8; ++wv) ss += sh->ssq[wv][0];
     return rsqrtf(ss / (float)d + eps);
-  }
-  {
-    float4 v[SUB_MB];
+  } else {
     float q[SUB_MB];
-#pragma unroll
-    for (int i = 0; i < SUB_MB; ++i)
-      if (on && i < k) v[i] = __ldcg(reinterpret_cast<const float4*>(x_in + (size_t)i * d) + tid);
 #pragma unroll
     for (int i = 0; i < SUB_MB; ++i) {
       q[i] = 0.f;
       if (on && i < k) {
-        float4 w = v[i];
+        float4 w = rw.v[i];
         q[i] = w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
         if (sd) *reinterpret_cast<float4*>(sSeed + (size_t)i * (seed1 - seed0) + (c - seed0)) = w;
         w.x *= g.x; w.y *= g.y; w.z *= g.z; w.w *= g.w;
@@ -144,16 +154,16 @@ __device__ __forceinline__ float sub_load_rows(const float* __restrict__ x_in, i
     }
     const float r8 = treduce<8>(q, lane);   // lanes 4 i hold the warp's sum of row i
     if ((lane & 3) == 0) sh->ssq[warp][lane >> 2] = r8;
-  }
-  __syncthreads();
-  if (tid < k) {
-    float ss = 0.f;
+    __syncthreads();
+    if (tid < k) {
+      float ss = 0.f;
 #pragma unroll
-    for (int wv = 0; wv < 8; ++wv) ss += sh->ssq[wv][tid];
-    sh->inv[tid] = rsqrtf(ss / (float)d + eps);
+      for (int wv = 0; wv < 8; ++wv) ss += sh->ssq[wv][tid];
+      sh->inv[tid] = rsqrtf(ss / (float)d + eps);
+    }
+    __syncthreads();
+    return 0.f;
   }
-  __syncthreads();
-  return 0.f;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -163,7 +173,8 @@ struct AttnSubLayout { int wq, xs, kv, kv_late, qkv, psum, probs, bias, seed, sa
 
 struct AttnSubArgs {
   const CallDesc* desc;
-  const float* x_in;    // [MAXB][d] residual stream (complete)
+  const float* x_in;    // [x_rows][d] residual stream (complete)
+  int x_rows;           // rows x_in has (at least the rows of the pass)
   float* x_out;         // [MAXB][d] zero on entry; receives x_in + the sub-layer's output
   float* x_zero;        // [MAXB][d] cleared for the kernel after this one
   const float* gain;
@@ -213,7 +224,7 @@ inline AttnSubLayout attn_sub_layout(int d, int dkv, int P, int C, int mb, int k
   L.probs = off; off += sub_up16(mb * (kc + 4) * 4);
   L.bias = off; off += sub_up16(bias_len * 4);
   L.seed = off; off += sub_up16(mb * no * 4);
-  L.red = off; off += sub_up16(SUB_THREADS * 4 + 64);
+  L.red = off; off += sub_up16(SUB_THREADS * 16 + 64 * 4);   // single row: [key part][d_kv] weighted values, then the parts' sums
   L.loc = off; off += sub_up16(mb * npr * 4);
   L.out = off; off += mb == 1 ? 0 : sub_up16(SUB_MB * (no + 4) * 4);
   L.sh = off; off += sub_up16((int)sizeof(SubShared));
@@ -338,6 +349,8 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
   SUB_STAMP();            // 0: prologue
   pdl_wait();
   SUB_STAMP();            // 1: dependency wait
+  SubRows<ONE> rw;
+  sub_rows_issue<ONE>(a.x_in, a.x_rows, d, tid, rw);
   const int k = ONE ? 1 : min(a.desc->k, a.mb), pos0 = a.desc->pos0;
   if (a.self) {
     n_keys = min(pos0 + k, a.cap);
@@ -356,7 +369,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
     for (int i = blockIdx.x * SUB_THREADS + tid; i < n4; i += gridDim.x * SUB_THREADS)
       reinterpret_cast<float4*>(a.x_zero)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  const float inv1 = sub_load_rows<ONE>(a.x_in, k, d, g4, a.eps, Xs, xst, sh, sSeed, h == 0 ? o0 : 0, h == 0 ? o0 + no : 0, tid, lane, warp);
+  const float inv1 = sub_rows_finish<ONE>(rw, k, d, g4, a.eps, Xs, xst, sh, sSeed, h == 0 ? o0 : 0, h == 0 ? o0 + no : 0, tid, lane, warp);
   if (tid < bias_cnt) sBias[tid] = bias0;
 #pragma unroll 1
   for (int i = tid + SUB_THREADS; i < bias_cnt; i += SUB_THREADS) sBias[i] = __ldg(a.bias + (size_t)h * a.bias_ld + dist_lo + i);
@@ -404,7 +417,9 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
   sub_cluster_wait();
   SUB_STAMP();            // 6: cluster barrier 1
   // ---- phase B: attention of the k rows over the keys [j0, j1) ---------------------------------
-  const int ch = tid & (dkv - 1), part = tid >> a.dkv_shift, nparts = SUB_THREADS >> a.dkv_shift;
+  // single row, value phase: thread = (group of four channels, key part)
+  const int cg4 = tid & ((dkv >> 2) - 1), part4 = tid >> (a.dkv_shift - 2), nparts4 = SUB_THREADS >> (a.dkv_shift - 2);
+  float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
   const int dq4 = dkv >> 4;   // 16-byte units per channel quarter (d_kv <= 64)
   constexpr int RPP = ONE ? 1 : 2;   // rows per thread in the value phase (up to 8 rows over at least 4 parts)
   float acc[RPP], run1 = -INFINITY, lsum1 = 0.f;
@@ -430,56 +445,105 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
     sub_cp_wait();
     __syncthreads();
     SUB_STAMP();          // B1: keys / values staged
-    {   // scores: four threads per key, one channel quarter each (16-byte units interleaved over the quarters); the
-        // quarter of the key stays in registers while the rows go by; 64 keys per turn
+    if (ONE) {   // scores: four threads per key, one channel quarter each (16-byte units interleaved over the quarters);
+                 // two keys (64 apart) per thread and turn so that their loads are in flight together
       const int qt = tid & 3;
+      const float* qp = sQKV;
 #pragma unroll 1
-      for (int jj = tid >> 2; jj < ((nk + 63) & ~63); jj += SUB_THREADS / 4) {
-      const bool valid = jj < nk;
-      float4 kq[4];
+      for (int j0b = 0; j0b < nk; j0b += SUB_THREADS / 2) {   // (the same trip count for every thread: the quads shuffle)
+        const int jb = j0b + (tid >> 2), jc = jb + SUB_THREADS / 4;
+        const bool va = jb < nk, vb = jc < nk;
+        const float* pa = sK + (size_t)(va ? jb : 0) * kvst;
+        const float* pb = sK + (size_t)(vb ? jc : 0) * kvst;
+        float sa = 0.f, sb = 0.f;
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (valid && u < dq4) kq[u] = *reinterpret_cast<const float4*>(sK + (size_t)jj * kvst + (u * 4 + qt) * 4);
-#pragma unroll 1
-      for (int m = 0; m < k; ++m) {
-        float s = 0.f;
-        if (valid) {
-          const float* qp = sQKV + (size_t)m * R;
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-            if (u < dq4) {
-              const float4 q4 = *reinterpret_cast<const float4*>(qp + (u * 4 + qt) * 4);
-              s += q4.x * kq[u].x + q4.y * kq[u].y + q4.z * kq[u].z + q4.w * kq[u].w;
-            }
-        }
-        s += __shfl_xor_sync(0xffffffffu, s, 1);
-        s += __shfl_xor_sync(0xffffffffu, s, 2);
-        if (valid && qt == 0) {
-          if (a.self) {
-            const int dist = pos0 + m - (c0 + jj);   // causal inside the block: row m sees keys up to its own position
-            s = dist >= 0 ? s + sBias[min(dist - dist_lo, a.bias_len - 1)] : -INFINITY;
+        for (int u = 0; u < 4; ++u)
+          if (u < dq4) {
+            const float4 q4 = *reinterpret_cast<const float4*>(qp + (u * 4 + qt) * 4);
+            const float4 ka = *reinterpret_cast<const float4*>(pa + (u * 4 + qt) * 4);
+            const float4 kb = *reinterpret_cast<const float4*>(pb + (u * 4 + qt) * 4);
+            sa += q4.x * ka.x + q4.y * ka.y + q4.z * ka.z + q4.w * ka.w;
+            sb += q4.x * kb.x + q4.y * kb.y + q4.z * kb.z + q4.w * kb.w;
           }
-          sP[(size_t)m * pst + jj] = s;
+        sa += __shfl_xor_sync(0xffffffffu, sa, 1); sb += __shfl_xor_sync(0xffffffffu, sb, 1);
+        sa += __shfl_xor_sync(0xffffffffu, sa, 2); sb += __shfl_xor_sync(0xffffffffu, sb, 2);
+        if (qt == 0) {
+          if (a.self) {   // (a single row sees every key up to its own position: all of them)
+            if (va) sa += sBias[min(pos0 - (c0 + jb) - dist_lo, a.bias_len - 1)];
+            if (vb) sb += sBias[min(pos0 - (c0 + jc) - dist_lo, a.bias_len - 1)];
+          }
+          if (va) sP[jb] = sa;
+          if (vb) sP[jc] = sb;
         }
       }
+    } else {
+      // scores on mma.sync m16n8k16: 16 keys of the chunk are the rows of the left operand, the token rows the columns of
+      // the right one, 16 channels per step; keys and queries each as a bf16 head and a bf16 remainder, three products kept.
+      // Warp w takes the key tiles w, w + 8, ...
+      const int g = lane >> 2, t = lane & 3;
+#pragma unroll 1
+      for (int t0 = warp * 16; t0 < nk; t0 += 16 * (SUB_THREADS / 32)) {
+        float c0a = 0.f, c1a = 0.f, c2a = 0.f, c3a = 0.f;
+        const float* ka = sK + (size_t)min(t0 + g, nk - 1) * kvst + 2 * t;
+        const float* kb = sK + (size_t)min(t0 + g + 8, nk - 1) * kvst + 2 * t;
+        const float* qp = sQKV + (size_t)min(g, k - 1) * R + 2 * t;
+#pragma unroll
+        for (int st = 0; st < 4; ++st)
+          if (st * 16 < dkv) {
+            const float2 a0 = *reinterpret_cast<const float2*>(ka + st * 16), a1 = *reinterpret_cast<const float2*>(kb + st * 16);
+            const float2 a2 = *reinterpret_cast<const float2*>(ka + st * 16 + 8), a3 = *reinterpret_cast<const float2*>(kb + st * 16 + 8);
+            float2 b0 = *reinterpret_cast<const float2*>(qp + st * 16), b1 = *reinterpret_cast<const float2*>(qp + st * 16 + 8);
+            if (g >= k) { b0 = make_float2(0.f, 0.f); b1 = b0; }
+            const uint32_t ah0 = sl_pack_bf16(a0.x, a0.y), ah1 = sl_pack_bf16(a1.x, a1.y), ah2 = sl_pack_bf16(a2.x, a2.y), ah3 = sl_pack_bf16(a3.x, a3.y);
+            const uint32_t al0 = sl_pack_bf16(a0.x - __uint_as_float(ah0 << 16), a0.y - __uint_as_float(ah0 & 0xffff0000u));
+            const uint32_t al1 = sl_pack_bf16(a1.x - __uint_as_float(ah1 << 16), a1.y - __uint_as_float(ah1 & 0xffff0000u));
+            const uint32_t al2 = sl_pack_bf16(a2.x - __uint_as_float(ah2 << 16), a2.y - __uint_as_float(ah2 & 0xffff0000u));
+            const uint32_t al3 = sl_pack_bf16(a3.x - __uint_as_float(ah3 << 16), a3.y - __uint_as_float(ah3 & 0xffff0000u));
+            const uint32_t bh0 = sl_pack_bf16(b0.x, b0.y), bh1 = sl_pack_bf16(b1.x, b1.y);
+            const uint32_t bl0 = sl_pack_bf16(b0.x - __uint_as_float(bh0 << 16), b0.y - __uint_as_float(bh0 & 0xffff0000u));
+            const uint32_t bl1 = sl_pack_bf16(b1.x - __uint_as_float(bh1 << 16), b1.y - __uint_as_float(bh1 & 0xffff0000u));
+#define SUB_MMA_S(A0, A1, A2, A3, B0, B1)                                                                                        \
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};" \
+                         : "+f"(c0a), "+f"(c1a), "+f"(c2a), "+f"(c3a) : "r"(A0), "r"(A1), "r"(A2), "r"(A3), "r"(B0), "r"(B1))
+            SUB_MMA_S(ah0, ah1, ah2, ah3, bh0, bh1);
+            SUB_MMA_S(al0, al1, al2, al3, bh0, bh1);
+            SUB_MMA_S(ah0, ah1, ah2, ah3, bl0, bl1);
+#undef SUB_MMA_S
+          }
+        // accumulators: keys t0 + g and t0 + g + 8, token rows 2 t and 2 t + 1
+        const float cv[4] = {c0a, c1a, c2a, c3a};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int jj = t0 + g + 8 * (i >> 1), m = 2 * t + (i & 1);
+          if (jj < nk && m < k) {
+            float sc = cv[i];
+            if (a.self) {
+              const int dist = pos0 + m - (c0 + jj);   // causal inside the block: row m sees keys up to its own position
+              sc = dist >= 0 ? sc + sBias[min(dist - dist_lo, a.bias_len - 1)] : -INFINITY;
+            }
+            sP[(size_t)m * pst + jj] = sc;
+          }
+        }
       }
     }
     __syncthreads();
     SUB_STAMP();          // B2: scores
     if (ONE) {
-      // every warp finds the chunk's maximum; thread (channel, key part) then exponentiates and weighs its keys
+      // every warp finds the chunk's maximum; thread (group of four channels, key part) then exponentiates and weighs its keys
       float mx = -INFINITY;
       for (int jj = lane; jj < nk; jj += 32) mx = fmaxf(mx, sP[jj]);
       mx = warp_max(mx);
       const float nw = fmaxf(run1, mx), sc = run1 == -INFINITY ? 0.f : __expf(run1 - nw);
-      float t = acc[0] * sc, l = lsum1 * sc;
-#pragma unroll 4
-      for (int jj = part; jj < nk; jj += nparts) {
+      float4 t4 = make_float4(acc4.x * sc, acc4.y * sc, acc4.z * sc, acc4.w * sc);
+      float l = lsum1 * sc;
+#pragma unroll 2
+      for (int jj = part4; jj < nk; jj += nparts4) {
         const float p = __expf(sP[jj] - nw);
+        const float4 v = *reinterpret_cast<const float4*>(sV + (size_t)jj * vst + cg4 * 4);
         l += p;
-        t += p * sV[(size_t)jj * vst + ch];
+        t4.x += p * v.x; t4.y += p * v.y; t4.z += p * v.z; t4.w += p * v.w;
       }
-      acc[0] = t; lsum1 = l; run1 = nw;
+      acc4 = t4; lsum1 = l; run1 = nw;
     } else {
       // running soft-max, one warp per row
 #pragma unroll 1
@@ -513,7 +577,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
         acc[0] *= rs; acc[1] *= rs;
         float c2 = 0.f, c3 = 0.f;
         const uint32_t zero = 0u;
-#pragma unroll 1
+#pragma unroll 2
         for (int k0 = 0; k0 < nk; k0 += 16) {
           float2 p0 = make_float2(0.f, 0.f), p1 = p0;
           if (g < k) {
@@ -542,18 +606,19 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
   }
   // this rank's record (max, sum, weighted values per row), assembled locally
   if (ONE) {
-    sRed[part * dkv + ch] = acc[0];
-    if (ch == 0) sRed[SUB_THREADS + part] = lsum1;
+    *reinterpret_cast<float4*>(sRed + (size_t)part4 * dkv + cg4 * 4) = acc4;
+    if (cg4 == 0) sRed[SUB_THREADS * 4 + part4] = lsum1;
     __syncthreads();
     if (tid < dkv) {
       float t = 0.f;
-      for (int p2 = 0; p2 < nparts; ++p2) t += sRed[p2 * dkv + tid];
+#pragma unroll 4
+      for (int p2 = 0; p2 < nparts4; ++p2) t += sRed[p2 * dkv + tid];
       recLoc[SUB_RECPAD + tid] = t;
-    }
-    if (tid == 0) {
+    } else if (warp == SUB_THREADS / 32 - 1) {   // the parts' sums, added by one warp
       float l = 0.f;
-      for (int p2 = 0; p2 < nparts; ++p2) l += sRed[SUB_THREADS + p2];
-      recLoc[0] = run1; recLoc[1] = l; recLoc[2] = 0.f; recLoc[3] = 0.f;
+      for (int p2 = lane; p2 < nparts4; p2 += 32) l += sRed[SUB_THREADS * 4 + p2];
+      l = warp_sum(l);
+      if (lane == 0) { recLoc[0] = run1; recLoc[1] = l; recLoc[2] = 0.f; recLoc[3] = 0.f; }
     }
   } else {
     if (warp * 8 < dkv && (lane >> 2) < k)   // accumulators of the tile: row lane / 4, channels 8 warp + 2 (lane % 4) (+ 1)
@@ -668,18 +733,37 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
 // ------------------------------------------------------------------------------------------------
 // Feed-forward sub-layer
 // ------------------------------------------------------------------------------------------------
-struct FfnSubLayout { int wi, wfo, xs, psum, u, seed, sh, total; };
+// W_fo [d][F] in the order the feed-forward kernels load it, in units of 8 columns (16 bytes of a row).  Unit u holds
+//   one: [i < 4][tid < d / 4]            the piece of row 4 tid + i                  (d pieces)
+//   blk: [i][rr < 2][w < 8][g < 8]       the piece of row (w + 8 i) 16 + g + 8 rr    (pack_wfo_dpad(d) pieces, zero past d)
+// so that the threads of a warp read neighbouring pieces.  Built once, when the context is created.
+__host__ __device__ inline int pack_wfo_dpad(int d) { return (d + 127) / 128 * 128; }
+__global__ void pack_wfo_kernel(const __nv_bfloat16* __restrict__ W, uint4* __restrict__ one, uint4* __restrict__ blk, int d, int F) {
+  const int u = blockIdx.x, d4 = d >> 2, dpad = pack_wfo_dpad(d);
+  for (int p = threadIdx.x; p < d; p += blockDim.x) {
+    const int i = p / d4, tt = p - i * d4;
+    one[(size_t)u * d + p] = *reinterpret_cast<const uint4*>(W + (size_t)(4 * tt + i) * F + 8 * u);
+  }
+  for (int p = threadIdx.x; p < dpad; p += blockDim.x) {
+    const int g = p & 7, w = (p >> 3) & 7, rr = (p >> 6) & 1, i = p >> 7, n = (w + 8 * i) * 16 + g + 8 * rr;
+    blk[(size_t)u * dpad + p] = n < d ? *reinterpret_cast<const uint4*>(W + (size_t)n * F + 8 * u) : make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+
+struct FfnSubLayout { int wi, xs, psum, u, seed, sh, total; };
 
 struct FfnSubArgs {
   const CallDesc* desc;
   const float* x_in;
+  int x_rows;                // rows x_in has (at least the rows of the pass)
   float* x_out;
   float* x_zero;             // nullptr: nothing to clear (second part of a split launch)
   const float* gain;
   float eps;
   const __nv_bfloat16* Wi0;  // [F][d]
   const __nv_bfloat16* Wi1;  // [F][d] gate matrix (gated GELU) or nullptr
-  const __nv_bfloat16* WfoT; // [F][d]: W_fo transposed
+  const uint4* Wfo1;         // W_fo in the load order of the single-row variant (pack_wfo_kernel)
+  const uint4* Wfo8;         // ... and of the block variant
   int d, F, gated;
   int part, nparts;          // this launch covers the slices blockIdx.x * nparts + part of gridDim.x * nparts
   int seed;                  // 1: the blocks add x_in for their share of the columns
@@ -689,16 +773,14 @@ struct FfnSubArgs {
   FfnSubLayout L;
 };
 
-inline int ffn_sub_rows(int F, int slices) { return (F + slices - 1) / slices; }
+// most rows of a slice when F (a multiple of 8) is dealt out in units of 8 rows
+inline int ffn_sub_rows(int F, int slices) { return 8 * ((F / 8 + slices - 1) / slices); }
 inline FfnSubLayout ffn_sub_layout(int d, int F, int gated, int slices, int grid, int mb) {
   FfnSubLayout L;
   const int nf = ffn_sub_rows(F, slices), nmat = gated ? 2 : 1;
   int off = 0;
   L.wi = off; off += sub_up16(nf * nmat * (d * 2 + SL_WPAD));
-  // a single-row block keeps the rows of the transposed W_fo in registers; the block variant stages SUB_FO_REGS padded
-  // rows (those past the slice are zero) for the tensor-core tiles of the output products
-  L.wfo = off; off += mb == 1 ? 0 : SUB_FO_REGS * (d * 2 + SL_WPAD);
-  L.xs = off; off += sub_up16(mb * (d + SL_XPAD) * 4);
+  L.xs = off; off += sub_up16(mb * (d + SL_XPAD) * 4);   // token rows; the block variant later collects its output tile here
   L.psum = off; off += mb == 1 ? SUB_PSUM : 8 * 128 * 4;
   L.u = off; off += sub_up16(mb * (SUB_FO_REGS + 4) * 4);
   L.seed = off; off += sub_up16(mb * 4 * ((d / 4 + grid - 1) / grid + 1) * 4);
@@ -712,11 +794,10 @@ __global__ void __launch_bounds__(SUB_THREADS) ffn_sub_kernel(const FfnSubArgs a
   extern __shared__ __align__(1024) unsigned char sub_smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = a.d, F = a.F, G = gridDim.x, S = G * a.nparts, s = blockIdx.x * a.nparts + a.part;
-  const int f0 = (int)(((long long)s * F) / S), f1 = (int)(((long long)(s + 1) * F) / S), nf = f1 - f0;
+  const int f0 = 8 * (int)(((long long)s * (F >> 3)) / S), f1 = 8 * (int)(((long long)(s + 1) * (F >> 3)) / S), nf = f1 - f0;
   const int nmat = a.gated ? 2 : 1, nrows = nf * nmat;
   const int rowbytes = d * 2 + SL_WPAD, xst = d + SL_XPAD;
   unsigned char* sWi = sub_smem + a.L.wi;
-  const unsigned char* sWfo = sub_smem + a.L.wfo;
   float* Xs = reinterpret_cast<float*>(sub_smem + a.L.xs);
   float* psum = reinterpret_cast<float*>(sub_smem + a.L.psum);
   float* sU = reinterpret_cast<float*>(sub_smem + a.L.u);
@@ -732,7 +813,7 @@ __global__ void __launch_bounds__(SUB_THREADS) ffn_sub_kernel(const FfnSubArgs a
     mbar_init(smem_u32(&sh->wbar), 1);
     sh->failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    mbar_expect(smem_u32(&sh->wbar), (uint32_t)((nrows + (ONE ? 0 : nf)) * d * 2));
+    mbar_expect(smem_u32(&sh->wbar), (uint32_t)(nrows * d * 2));
   }
   __syncthreads();
   pdl_launch_dependents();
@@ -744,33 +825,53 @@ __global__ void __launch_bounds__(SUB_THREADS) ffn_sub_kernel(const FfnSubArgs a
       bulk_g2s(smem_u32(sWi + (size_t)i * rowbytes), W + (size_t)(f0 + rr) * d, (uint32_t)(d * 2), smem_u32(&sh->wbar));
     }
   }
-  // the slice of the transposed W_fo: ONE keeps it in registers (thread <-> four columns of every row), else one bulk copy
-  constexpr int NFR = ONE ? SUB_FO_REGS : 1;
-  uint2 wfr[NFR];
-  if (ONE) {
+  // The block's columns [f0, f1) of W_fo stay in registers, 16 bytes (8 columns of a row) per load, from the copies of
+  // W_fo that pack_wfo_kernel lays out so that the loads of a warp are contiguous (8 columns of a row in place are 16
+  // bytes every 2 F bytes: a fraction of the memory's rate).  ONE: thread <-> the four output rows 4 tid .. 4 tid + 3,
+  // chunk q = columns 8 q .. 8 q + 7.  Block variant: warp w owns the output tiles w, w + 8, ... (16 rows each); thread
+  // (g, t) keeps, of rows g and g + 8 of a tile, the columns 8 t .. 8 t + 7: read as the left operand of mma.sync m16n8k16
+  // they are two steps of 16 slice rows, with the slice rows dealt to the steps' positions so that one 16-byte load
+  // fills them (the right operand, the hidden activations, follows the same order).
+  uint4 wf[8][2];
 #pragma unroll
-    for (int i = 0; i < NFR; ++i) {
-      wfr[i] = make_uint2(0u, 0u);
-      if (i < nf && tid * 4 < d) {
-        const __nv_bfloat16* p = a.WfoT + (size_t)(f0 + i) * d + tid * 4;
-        asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(wfr[i].x), "=r"(wfr[i].y) : "l"(p));
-      }
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 2; ++j) wf[i][j] = make_uint4(0u, 0u, 0u, 0u);
+  if (ONE) {
+    if (tid * 4 < d) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (8 * q < nf) {
+          const uint4* p = a.Wfo1 + (size_t)((f0 >> 3) + q) * d + tid;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4& w = wf[i * 2 + (q >> 1)][q & 1];
+            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w) : "l"(p + i * (d >> 2)));
+          }
+        }
     }
   } else {
-    const int i = (((tid & 31) << 3) | (tid >> 5)) - nrows;   // the rows after those of W_i, spread over the warps in the same way
-    if (i >= 0 && i < nf)
-      bulk_g2s(smem_u32(sWfo + (size_t)i * rowbytes), a.WfoT + (size_t)(f0 + i) * d, (uint32_t)(d * 2), smem_u32(&sh->wbar));
-    // rows past the slice take part in the tiles: they must be zero
-    const int z16 = (SUB_FO_REGS - nf) * (rowbytes >> 4);
-#pragma unroll 1
-    for (int z = tid; z < z16; z += SUB_THREADS)
-      *reinterpret_cast<uint4*>(sub_smem + a.L.wfo + (size_t)nf * rowbytes + (size_t)z * 16) = make_uint4(0u, 0u, 0u, 0u);
+    const int g = lane >> 2, t = lane & 3;
+    if (8 * t < nf) {
+      const uint4* p = a.Wfo8 + (size_t)((f0 >> 3) + t) * pack_wfo_dpad(d) + warp * 8 + g;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if ((warp + 8 * i) * 16 < d) {
+#pragma unroll
+          for (int rr = 0; rr < 2; ++rr) {
+            uint4& w = wf[i][rr];
+            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w) : "l"(p + (i * 2 + rr) * 64));
+          }
+        }
+    }
   }
   float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f);
   if (tid * 4 < d) g4 = __ldg(reinterpret_cast<const float4*>(a.gain) + tid);
   SUB_STAMP();            // 0: prologue
   pdl_wait();
   SUB_STAMP();            // 1: dependency wait
+  SubRows<ONE> rw;
+  sub_rows_issue<ONE>(a.x_in, a.x_rows, d, tid, rw);
   const int k = ONE ? 1 : min(a.desc->k, a.mb);
   if (a.x_zero) {
     const int n4 = k * d4;
@@ -778,7 +879,7 @@ __global__ void __launch_bounds__(SUB_THREADS) ffn_sub_kernel(const FfnSubArgs a
     for (int i = blockIdx.x * SUB_THREADS + tid; i < n4; i += G * SUB_THREADS)
       reinterpret_cast<float4*>(a.x_zero)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  const float inv1 = sub_load_rows<ONE>(a.x_in, k, d, g4, a.eps, Xs, xst, sh, sSeed, su0 * 4, su1 * 4, tid, lane, warp);
+  const float inv1 = sub_rows_finish<ONE>(rw, k, d, g4, a.eps, Xs, xst, sh, sSeed, su0 * 4, su1 * 4, tid, lane, warp);
   SUB_STAMP();            // 2: token rows + norm
   {
     if (nf > 0) sub_wait(sh, a.err, &sh->wbar, 0, a.spin);
@@ -805,82 +906,79 @@ __global__ void __launch_bounds__(SUB_THREADS) ffn_sub_kernel(const FfnSubArgs a
     SUB_STAMP();          // 4: hidden activations
   }
   if (ONE) {
-    // this slice's share of all d outputs: thread <-> four columns, the rows of the transposed W_fo from its registers
+    // this slice's share of all d outputs: thread <-> four output rows, their columns of W_fo from its registers
     if (tid < d4) {
       const bool seeds = tid >= su0 && tid < su1;
-      float o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
+      float o[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int i = 0; i < NFR; ++i) {   // (registers past the slice hold zeros)
-        const float uv = i < nf ? sU[i] : 0.f;
-        o0 += __uint_as_float(wfr[i].x << 16) * uv; o1 += __uint_as_float(wfr[i].x & 0xffff0000u) * uv;
-        o2 += __uint_as_float(wfr[i].y << 16) * uv; o3 += __uint_as_float(wfr[i].y & 0xffff0000u) * uv;
-      }
+      for (int q = 0; q < 4; ++q)
+        if (8 * q < nf) {
+          const float4 u0 = *reinterpret_cast<const float4*>(sU + 8 * q), u1 = *reinterpret_cast<const float4*>(sU + 8 * q + 4);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint4 w = wf[i * 2 + (q >> 1)][q & 1];
+            o[i] += __uint_as_float(w.x << 16) * u0.x + __uint_as_float(w.x & 0xffff0000u) * u0.y + __uint_as_float(w.y << 16) * u0.z +
+                    __uint_as_float(w.y & 0xffff0000u) * u0.w + __uint_as_float(w.z << 16) * u1.x + __uint_as_float(w.z & 0xffff0000u) * u1.y +
+                    __uint_as_float(w.w << 16) * u1.z + __uint_as_float(w.w & 0xffff0000u) * u1.w;
+          }
+        }
       if (seeds) {
         const float4 xr = *reinterpret_cast<const float4*>(sSeed + (tid - su0) * 4);
-        o0 += xr.x; o1 += xr.y; o2 += xr.z; o3 += xr.w;
+        o[0] += xr.x; o[1] += xr.y; o[2] += xr.z; o[3] += xr.w;
       }
       if (nf > 0 || seeds)
-        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(a.x_out + tid * 4), "f"(o0), "f"(o1), "f"(o2), "f"(o3) : "memory");
+        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(a.x_out + tid * 4), "f"(o[0]), "f"(o[1]), "f"(o[2]), "f"(o[3]) : "memory");
     }
   } else {
-    // out[token][column] = sum_i u[token][i] * WfoT[i][column] on mma.sync m16n8k16: the token rows are the 16 rows of
-    // the left operand (rows 8..15 zero), each activation as a bf16 head and a bf16 remainder; the right operand
-    // (32 slice rows x 8 columns, two steps of 16) comes out of the padded rows with one transposing matrix load
+    // out[column][token] = sum_i W_fo[column][f0 + i] * u[token][i] on mma.sync m16n8k16: 16 output columns are the rows of
+    // the left operand (from the registers), the token rows the columns of the right one, each activation as a bf16 head and
+    // a bf16 remainder.  Step s of thread (g, t) covers the slice rows 8 t + 4 s .. 8 t + 4 s + 3.
     const int g = lane >> 2, t = lane & 3;
-    uint32_t ah[2][2], al[2][2];
+    uint32_t bh[2][2], bl[2][2];
 #pragma unroll
-    for (int st = 0; st < 2; ++st)
+    for (int st = 0; st < 2; ++st) {
+      const float4 u4 = *reinterpret_cast<const float4*>(sU + (size_t)g * ust + 8 * t + 4 * st);
+      bh[st][0] = sl_pack_bf16(u4.x, u4.y); bh[st][1] = sl_pack_bf16(u4.z, u4.w);
+      bl[st][0] = sl_pack_bf16(u4.x - __uint_as_float(bh[st][0] << 16), u4.y - __uint_as_float(bh[st][0] & 0xffff0000u));
+      bl[st][1] = sl_pack_bf16(u4.z - __uint_as_float(bh[st][1] << 16), u4.w - __uint_as_float(bh[st][1] & 0xffff0000u));
+    }
+    float* sOut = Xs;   // [token][column], row stride xst: the token rows are done with
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        const float2 u2 = *reinterpret_cast<const float2*>(sU + (size_t)g * ust + 16 * st + 8 * hh + 2 * t);
-        ah[st][hh] = sl_pack_bf16(u2.x, u2.y);
-        al[st][hh] = sl_pack_bf16(u2.x - __uint_as_float(ah[st][hh] << 16), u2.y - __uint_as_float(ah[st][hh] & 0xffff0000u));
-      }
-    const uint32_t brow = smem_u32(sWfo + (size_t)lane * rowbytes);   // lane l addresses slice row l of each 8 x 8 piece
-    const uint32_t zero = 0u;
-#pragma unroll 1
-    for (int nt = warp; nt < (d >> 3); nt += SUB_THREADS / 32) {
-      uint32_t b0, b1, b2, b3;
-      asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-                   : "=r"(b0), "=r"(b1), "=r"(b2), "=r"(b3) : "r"(brow + (uint32_t)nt * 16u));
-      float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
-#define SUB_MMA(A0, A2, B0, B1)                                                                                              \
-      asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};" \
-                   : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3) : "r"(A0), "r"(zero), "r"(A2), "r"(zero), "r"(B0), "r"(B1))
-      SUB_MMA(ah[0][0], ah[0][1], b0, b1);
-      SUB_MMA(al[0][0], al[0][1], b0, b1);
-      SUB_MMA(ah[1][0], ah[1][1], b2, b3);
-      SUB_MMA(al[1][0], al[1][1], b2, b3);
+    for (int i = 0; i < 8; ++i) {
+      const int n0 = (warp + 8 * i) * 16;
+      if (n0 < d) {
+        float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
+#define SUB_MMA(A0, A1, A2, A3, B0, B1)                                                                                          \
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};" \
+                     : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3) : "r"(A0), "r"(A1), "r"(A2), "r"(A3), "r"(B0), "r"(B1))
+        SUB_MMA(wf[i][0].x, wf[i][1].x, wf[i][0].y, wf[i][1].y, bh[0][0], bh[0][1]);
+        SUB_MMA(wf[i][0].x, wf[i][1].x, wf[i][0].y, wf[i][1].y, bl[0][0], bl[0][1]);
+        SUB_MMA(wf[i][0].z, wf[i][1].z, wf[i][0].w, wf[i][1].w, bh[1][0], bh[1][1]);
+        SUB_MMA(wf[i][0].z, wf[i][1].z, wf[i][0].w, wf[i][1].w, bl[1][0], bl[1][1]);
 #undef SUB_MMA
-      // c0, c1: token row g, columns 8 nt + 2 t (+ 1)
-      const int col = nt * 8 + 2 * t, un = col >> 2;
+        // accumulators: columns n0 + g and n0 + g + 8, token rows 2 t and 2 t + 1
+        sOut[(size_t)(2 * t) * xst + n0 + g] = c0; sOut[(size_t)(2 * t + 1) * xst + n0 + g] = c1;
+        sOut[(size_t)(2 * t) * xst + n0 + g + 8] = c2; sOut[(size_t)(2 * t + 1) * xst + n0 + g + 8] = c3;
+      }
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int idx = tid; idx < k * d4; idx += SUB_THREADS) {   // added four columns at a time
+      const int m = idx / d4, un = idx - m * d4;
       const bool seeds = un >= su0 && un < su1;
-      if (g < k && (nf > 0 || seeds)) {
+      if (nf > 0 || seeds) {
+        float4 v = *reinterpret_cast<const float4*>(sOut + (size_t)m * xst + un * 4);
         if (seeds) {
-          const float2 xr = *reinterpret_cast<const float2*>(sSeed + (size_t)g * (su1 - su0) * 4 + (col - su0 * 4));
-          c0 += xr.x; c1 += xr.y;
+          const float4 xr = *reinterpret_cast<const float4*>(sSeed + (size_t)m * (su1 - su0) * 4 + (un - su0) * 4);
+          v.x += xr.x; v.y += xr.y; v.z += xr.z; v.w += xr.w;
         }
-        asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(a.x_out + (size_t)g * d + col), "f"(c0), "f"(c1) : "memory");
+        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(a.x_out + (size_t)m * d + un * 4), "f"(v.x), "f"(v.y), "f"(v.z),
+                     "f"(v.w) : "memory");
       }
     }
   }
   SUB_STAMP();            // 5: output products + reductions issued
   SUB_STAMP_END(2);
-}
-
-// W_fo [d][F] -> [F][d] (once, when the context is created)
-__global__ void transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out, int rows, int cols) {
-  __shared__ __nv_bfloat16 tile[32][33];
-  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
-    const int r = r0 + i, c = c0 + threadIdx.x;
-    if (r < rows && c < cols) tile[i][threadIdx.x] = in[(size_t)r * cols + c];
-  }
-  __syncthreads();
-  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
-    const int c = c0 + i, r = r0 + threadIdx.x;
-    if (r < rows && c < cols) out[(size_t)c * rows + r] = tile[threadIdx.x][i];
-  }
 }
 
 }  // namespace bild

@@ -67,7 +67,9 @@ def _ref_attention(self_attn, x, g, Wp, Wo, K, V, n_before, bias, H, dkv):
 @pytest.mark.parametrize("self_attn,d,H,dkv,cap,n_before", [
     (True, 1024, 16, 64, 81, 0), (True, 1024, 16, 64, 81, 64), (True, 1024, 16, 64, 1040, 1000),
     (False, 1024, 16, 64, 512, 512), (False, 1024, 16, 64, 1024, 1000), (False, 512, 8, 64, 512, 512),
-    (True, 512, 6, 64, 300, 257), (False, 512, 6, 64, 64, 64), (True, 128, 4, 32, 40, 7), (False, 64, 4, 16, 32, 19)])
+    (True, 512, 6, 64, 300, 257), (False, 512, 6, 64, 64, 64), (True, 128, 4, 32, 40, 7), (False, 64, 4, 16, 32, 19),
+    # around the key count up to which every block of a head attends over all keys (one staged chunk)
+    (True, 1024, 16, 64, 200, 72), (True, 1024, 16, 64, 200, 75), (True, 512, 8, 64, 257, 100), (False, 1024, 16, 64, 96, 70)])
 def test_attention_sublayer_matches_numpy(M, self_attn, d, H, dkv, cap, n_before):
     import torch
     from paper_2302_07863_b200.binding import op_attn_sublayer

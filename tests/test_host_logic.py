@@ -55,8 +55,8 @@ def test_workspace_query_and_validation(L):
     s, l = MODEL_SHAPES["t5_s"], MODEL_SHAPES["t5_l"]
     # at least the self- and cross-attention K/V of both models (fp32)
     need = sum(2 * m.n_layers * m.inner * (65 + 512) * 4 for m in (s, l))
-    # ... plus the transposed feed-forward output matrices of both decoders (bf16 configurations)
-    need += sum(m.n_layers * m.d_ff * m.d_model * 2 for m in (s, l))
+    # ... plus two re-ordered copies of the feed-forward output matrices of both decoders (bf16 configurations)
+    need += sum(2 * m.n_layers * m.d_ff * m.d_model * 2 for m in (s, l))
     # ... plus activations, per-model encoder temporaries (fp32 and bf16 pairs), head partials
     assert need <= n.value <= need + 96 * 2 ** 20
     n2 = C.c_size_t()
