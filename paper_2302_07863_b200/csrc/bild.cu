@@ -1837,7 +1837,7 @@ int bild_time_pass(bild_ctx* c, int which, int k, int cache_len, int iters, floa
 int bild_debug_stamps(unsigned long long* out, int reset) {
   if (out && cudaMemcpyFromSymbol(out, g_sub_stamps, sizeof(g_sub_stamps)) != cudaSuccess) return BILD_ERR_CUDA;
   if (reset) {
-    static unsigned long long zero[4][24];
+    static unsigned long long zero[3][4][24];
     if (cudaMemcpyToSymbol(g_sub_stamps, zero, sizeof(zero)) != cudaSuccess) return BILD_ERR_CUDA;
   }
   return BILD_OK;

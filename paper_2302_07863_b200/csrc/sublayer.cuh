@@ -37,15 +37,22 @@ struct SubShared {
   int failed;
 };
 
-// Optional cycle stamps of block 0 (build with -DBILD_STAMPS): summed per kernel kind and phase boundary.
+// Optional cycle stamps (build with -DBILD_STAMPS), summed per kernel kind and phase boundary: [0] block 0, [1] every
+// block, [2] the longest a block took ([..][23]: how many blocks were added).
 #ifdef BILD_STAMPS
-__device__ unsigned long long g_sub_stamps[4][24];
+__device__ unsigned long long g_sub_stamps[3][4][24];
 #define SUB_STAMP_BEGIN() long long st_t[20]; int st_n = 0; st_t[st_n++] = clock64()
 #define SUB_STAMP() st_t[st_n++] = clock64()
 #define SUB_STAMP_END(kind)                                                                                \
-  if (blockIdx.x == 0 && threadIdx.x == 0) {                                                              \
-    for (int i_ = 1; i_ < st_n; ++i_) atomicAdd(&g_sub_stamps[kind][i_ - 1], (unsigned long long)(st_t[i_] - st_t[i_ - 1])); \
-    atomicAdd(&g_sub_stamps[kind][23], 1ull);                                                              \
+  if (threadIdx.x == 0) {                                                                                 \
+    for (int i_ = 1; i_ < st_n; ++i_) {                                                                   \
+      const unsigned long long dt_ = (unsigned long long)(st_t[i_] - st_t[i_ - 1]);                      \
+      if (blockIdx.x == 0) atomicAdd(&g_sub_stamps[0][kind][i_ - 1], dt_);                                \
+      atomicAdd(&g_sub_stamps[1][kind][i_ - 1], dt_);                                                     \
+      atomicMax(&g_sub_stamps[2][kind][i_ - 1], dt_);                                                     \
+    }                                                                                                     \
+    if (blockIdx.x == 0) atomicAdd(&g_sub_stamps[0][kind][23], 1ull);                                     \
+    atomicAdd(&g_sub_stamps[1][kind][23], 1ull);                                                          \
   }
 #else
 #define SUB_STAMP_BEGIN()

@@ -19,10 +19,12 @@ def bench(fn, n=30):
         e0.record(); fn(); e1.record(); torch.cuda.synchronize()
         ts.append(e0.elapsed_time(e1) * 1e3)
     ts.sort(); return ts[len(ts) // 2]
-for V, K, M, which in [(32128, 512, 1, "simt"), (32128, 512, 1, "sliced"), (32128, 1024, 1, "simt"), (32128, 1024, 1, "sliced"), (32128, 1024, 5, "sliced"),
-                       (250112, 512, 1, "sliced"), (250112, 1024, 1, "sliced"), (250112, 1024, 5, "sliced")]:
+# "rows": bild_op_lm_head (single rows: weights of a warp's vocabulary rows in registers); "sliced": the streaming tensor-core head
+for V, K, M, which in [(32128, 512, 1, "rows"), (32128, 512, 1, "sliced"), (32128, 1024, 1, "rows"), (32128, 1024, 1, "sliced"), (32128, 1024, 5, "sliced"),
+                       (250112, 512, 1, "rows"), (250112, 512, 1, "sliced"), (250112, 1024, 1, "rows"), (250112, 1024, 1, "sliced"),
+                       (250112, 1024, 5, "sliced")]:
     W = (torch.randn(V, K, device="cuda") * 0.05).to(torch.bfloat16)
     X = torch.randn(M, K, device="cuda"); g = torch.ones(K, device="cuda"); t = torch.zeros(M, dtype=torch.int32, device="cuda")
-    f = (lambda: op_lm_head(W, X, g, 1e-6, 5.0, t, M, V, K)) if which == "simt" else (lambda: op_lm_head_sliced(W, X, g, 1e-6, 5.0, t, M, V, K))
+    f = (lambda: op_lm_head(W, X, g, 1e-6, 5.0, t, M, V, K)) if which == "rows" else (lambda: op_lm_head_sliced(W, X, g, 1e-6, 5.0, t, M, V, K))
     us = bench(f)
     print(f"V={V} K={K} M={M} {which}: {us:.1f} us (L2 flushed; includes the entry point's small copies) -> {V*K*2/us/1e3:.0f} GB/s")

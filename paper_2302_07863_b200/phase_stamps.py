@@ -1,4 +1,5 @@
-"""Cycle stamps of the fused sub-layer kernels, phase by phase (block 0, averaged over the launches of a pass):
+"""Cycle stamps of the fused sub-layer kernels, phase by phase (per launch: block 0 / mean of all blocks / the longest
+any block took in any launch):
 
     python -m paper_2302_07863_b200.phase_stamps [workload] [k,...]
 
@@ -28,18 +29,21 @@ names = {0: ["P0 init", "P1 copies", "P2 loads", "arrive", "dep wait", "rows+nor
          1: None, 2: ["prologue", "dep wait", "rows+norm", "weights wait", "hidden", "out+red"]}
 names[1] = names[0]
 def run(which, k):
-    buf = (C.c_ulonglong * 96)()
+    buf = (C.c_ulonglong * 288)()
     L.bild_debug_stamps(buf, 1)
     us = ctx.time_pass(which, k, 64, 10) * 1000
     L.bild_debug_stamps(buf, 0)
     print(f"== model {which} k={k}: {us:.1f} us per pass")
     for kind, nm in (("self", 0), ("cross", 1), ("ffn", 2)):
-        n = buf[nm * 24 + 23]
-        if not n: continue
+        n0, na = buf[nm * 24 + 23], buf[96 + nm * 24 + 23]
+        if not n0: continue
         # single-row kernels have no separate soft-max phase (it is part of the value phase)
         nms = [x for x in names[nm] if not (k == 1 and x == "B3 softmax")]
-        ph = [buf[nm * 24 + i] / n / 1965.0 for i in range(len(nms))]
+        ph0 = [buf[nm * 24 + i] / n0 / 1965.0 for i in range(len(nms))]
+        pha = [buf[96 + nm * 24 + i] / na / 1965.0 for i in range(len(nms))]
+        phm = [buf[192 + nm * 24 + i] / 1965.0 for i in range(len(nms))]
         off = 5 if nm < 2 else 2
-        print(f"  {kind:5s} total {sum(ph[off:]):.2f} us after wait | " + " ".join(f"{a}={b:.2f}" for a, b in zip(nms, ph)))
+        print(f"  {kind:5s} after wait: block 0 {sum(ph0[off:]):.2f} us, mean of blocks {sum(pha[off:]):.2f} us | " +
+              " ".join(f"{a}={b:.2f}/{c:.2f}/{e:.2f}" for a, b, c, e in zip(nms, ph0, pha, phm)))
 run(0, 1)
 for k in ks: run(1, k)
