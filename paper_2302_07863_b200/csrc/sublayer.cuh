@@ -113,6 +113,42 @@ __device__ __forceinline__ float sub_total(const float* psum, int row, int m, in
 // has been read, a round trip to the L2 of its own); sub_rows_finish then writes x * gain into Xs and 1 / rms into
 // sh->inv (returned for the single row of ONE).  The raw values of the columns [seed0, seed1) (multiples of 4) also go
 // to sSeed[m][column - seed0]: the residual term the block adds.
+// Block variant: the normalised token rows wait in shared memory as bf16 heads [SUB_MB][d / 2 + 4] (two values a word)
+// followed by their bf16 remainders in the same layout: d + 8 words a row in all, as for the fp32 rows of the single-row
+// variant.  The row stride of d / 2 + 4 words is 4 times an odd number for d a multiple of 32: the eight rows a warp
+// reads side by side fall into different banks.
+__host__ __device__ inline int sub_split_stride(int d) { return (d >> 1) + 4; }
+
+// Products of up to 48 weight rows (shared memory, row stride rowst bytes) with the token rows on mma.sync m16n8k16, one tile
+// of 8 token rows: warp w works on row tile w / KS and on the w % KS-th part of K (KS = 8, 4 or 2 for 1, 2 or 3 row tiles),
+// as sl_mma<1>, with the right operand read ready-made; partial sums in the same place and layout (sub_total<false>).
+__device__ __forceinline__ void sub_mma_split(const unsigned char* sW, int rowst, int nrows, int K, const float* Xs, int mg, float* psum,
+                                              int warp, int lane) {
+  const int MT = (nrows + 15) >> 4, ks_sh = MT == 1 ? 3 : MT == 2 ? 2 : 1, KS = 1 << ks_sh;
+  if (warp >= MT * KS) return;
+  const int mt = warp >> ks_sh, ks = warp & (KS - 1);
+  const int steps = K >> 4, per = (steps + KS - 1) >> ks_sh;   // K is a multiple of 16 here
+  const int s0 = ks * per, s1 = min(steps, s0 + per);
+  const int g = lane >> 2, t = lane & 3, hw = sub_split_stride(K);
+  const unsigned char* pa0 = sW + (size_t)min(mt * 16 + g, nrows - 1) * rowst + t * 4;
+  const unsigned char* pa1 = sW + (size_t)min(mt * 16 + g + 8, nrows - 1) * rowst + t * 4;
+  const uint32_t* xh = reinterpret_cast<const uint32_t*>(Xs) + (size_t)min(g, mg - 1) * hw + t;
+  const uint32_t* xl = xh + (size_t)SUB_MB * hw;
+  float c[4] = {0.f, 0.f, 0.f, 0.f}, e[4] = {0.f, 0.f, 0.f, 0.f};   // heads and remainders: two independent chains
+#pragma unroll 4
+  for (int st = s0; st < s1; ++st) {
+    const int k0 = st << 4;
+    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(pa0 + k0 * 2), a1 = *reinterpret_cast<const uint32_t*>(pa1 + k0 * 2);
+    const uint32_t a2 = *reinterpret_cast<const uint32_t*>(pa0 + k0 * 2 + 16), a3 = *reinterpret_cast<const uint32_t*>(pa1 + k0 * 2 + 16);
+    const uint32_t h0 = xh[k0 >> 1], h1 = xh[(k0 >> 1) + 4], l0 = xl[k0 >> 1], l1 = xl[(k0 >> 1) + 4];
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(h0), "r"(h1));
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(e[0]), "+f"(e[1]), "+f"(e[2]), "+f"(e[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(l0), "r"(l1));
+  }
+  *reinterpret_cast<float4*>(psum + ((size_t)warp * 32 + lane) * 4) = make_float4(c[0] + e[0], c[1] + e[1], c[2] + e[2], c[3] + e[3]);
+}
+
 template <bool ONE>
 struct SubRows { float4 v[ONE ? 1 : SUB_MB]; };
 
@@ -156,7 +192,14 @@ __device__ __forceinline__ float sub_rows_finish(const SubRows<ONE>& rw, int k, 
         q[i] = w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
         if (sd) *reinterpret_cast<float4*>(sSeed + (size_t)i * (seed1 - seed0) + (c - seed0)) = w;
         w.x *= g.x; w.y *= g.y; w.z *= g.z; w.w *= g.w;
-        *reinterpret_cast<float4*>(Xs + (size_t)i * xst + c) = w;
+        // stored as bf16 heads and bf16 remainders, the form the tensor-core products read (sub_mma_split)
+        const uint32_t h0 = sl_pack_bf16(w.x, w.y), h1 = sl_pack_bf16(w.z, w.w);
+        const uint32_t l0 = sl_pack_bf16(w.x - __uint_as_float(h0 << 16), w.y - __uint_as_float(h0 & 0xffff0000u));
+        const uint32_t l1 = sl_pack_bf16(w.z - __uint_as_float(h1 << 16), w.w - __uint_as_float(h1 & 0xffff0000u));
+        uint32_t* xh = reinterpret_cast<uint32_t*>(Xs);
+        const int hw = sub_split_stride(d);
+        *reinterpret_cast<uint2*>(xh + (size_t)i * hw + 2 * tid) = make_uint2(h0, h1);
+        *reinterpret_cast<uint2*>(xh + (size_t)(SUB_MB + i) * hw + 2 * tid) = make_uint2(l0, l1);
       }
     }
     const float r8 = treduce<8>(q, lane);   // lanes 4 i hold the warp's sum of row i
@@ -385,7 +428,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
   SUB_STAMP();            // 3: wait for the weights
   // ---- phase A: this rank's q|k|v rows for all token rows -----------------------------------
   if (ONE) sl_items<1>(sWq, rowbytes, npr, d, Xs, xst, psum, warp, lane);
-  else sl_mma<1>(sWq, rowbytes, npr, d, Xs, xst, k, psum, warp, lane);
+  else sub_mma_split(sWq, rowbytes, npr, d, Xs, k, psum, warp, lane);
   __syncthreads();
   if (a.L.kv_late) stage_cached(j0, min(min(j1, pos0), j0 + a.kc_keys));   // the projection rows are done with: their place takes the keys
   SUB_STAMP();            // 4: q|k|v products
@@ -893,7 +936,7 @@ __global__ void __launch_bounds__(SUB_THREADS) ffn_sub_kernel(const FfnSubArgs a
     SUB_STAMP();          // 3: wait for the weights
     // hidden activations of the slice
     if (ONE) sl_items<1>(sWi, rowbytes, nrows, d, Xs, xst, psum, warp, lane);
-    else sl_mma<1>(sWi, rowbytes, nrows, d, Xs, xst, k, psum, warp, lane);
+    else sub_mma_split(sWi, rowbytes, nrows, d, Xs, k, psum, warp, lane);
     __syncthreads();   // (both product routines do nothing for a block without rows)
     if (ONE) {
       if (tid < nf) {
