@@ -193,6 +193,11 @@ typedef struct {
   int32_t attn_all_keys;     /* fused attention: while a head has at most this many keys (and they fit one staged chunk)
                               * every block of the head's cluster attends over all of them, which saves the exchange
                               * and merge of per-block partial results; 0: keys always split over the cluster */
+  int32_t graph_switch;      /* 1: in the loop graph the large pass of an iteration hangs off ONE conditional node of the
+                              * SWITCH kind (bodies: block pass, single-row pass, pass of 2 to 8 rows); 0: one IF node per
+                              * kind of pass */
+  int32_t enc_split_k;       /* 1: encoder GEMMs that add to the residual stream (output projection, second FFN matrix)
+                              * split K over more blocks, partial tiles added with reductions at the L2 */
 } bild_tuning;
 void bild_tuning_default(bild_tuning *t /*HOST out*/);
 /* bild_create with explicit switches; tuning == NULL means the defaults. */

@@ -171,6 +171,10 @@ struct bild_ctx {
   int slice_mode = 2;                // row-slice linear kernel: 0 off, 1 block passes, 2 block and single-row passes
   int sms = 0;
   size_t slice_smem_set = 0;
+  bool enc_split_k = true;           // encoder GEMMs that add to the residual stream split K over grid.z (reductions at the L2)
+  bool graph_switch = true;          // the large pass of a loop iteration hangs off one SWITCH node (else: one IF node per kind of pass)
+  unsigned long long sw_handle = 0;  // while the small pass of such a loop is captured: the SWITCH node's handle and body count
+  int sw_bodies = 0;
   int attn_all_keys = 128;           // fused attention: caches up to this many keys are attended by every rank of a head
   bool unit_attn = true;             // decoder attention on the 256-thread chunked kernel
   bool uattn_smem_set = false;
@@ -877,6 +881,12 @@ cudaError_t launch_enc_gemm(bild_ctx* c, Model& m, const LinArgs& a, int layer, 
   __nv_bfloat16* oh = out_pair >= 0 ? c->eb[m.index].exh[out_pair] : nullptr;
   __nv_bfloat16* ol = out_pair >= 0 ? c->eb[m.index].exl[out_pair] : nullptr;
   dim3 grid((a.N + UM_TILE_M - 1) / UM_TILE_M, tiles_tok);
+  if (a.epi == EPI_RESID && c->enc_split_k) {   // few tiles, long K: split K until the grid covers the SMs (at least 4 K blocks each)
+    const int tiles = (int)(grid.x * grid.y), nkb = a.K / UM_KB;
+    int z = 1;
+    while (z < 8 && tiles * (z * 2) <= c->sms && nkb / (z * 2) >= 4) z *= 2;
+    grid.z = z;
+  }
   if (gated)
     return launch_k(c, enc_gemm_kernel<true>, grid, dim3(EG_THREADS), eg_smem_bytes<true>(), a, &c->st->err, oh, ol, t[which_map],
                     t[which_map == TM_EWI0 ? TM_EWI1 : which_map], m.tmH[pair][ki][0], m.tmH[pair][ki][1]);
@@ -978,6 +988,7 @@ int decoder_pass(bild_ctx* c, int which, int MBv, float* logits_dbg, unsigned lo
   h.scale = mc.logit_scale; h.V = mc.vocab; h.K = d; h.desc = m.desc; h.partials = m.head_part;
   h.counter = m.head_cnt; h.out = m.head_out; h.logits_dbg = logits_dbg; h.which = which; h.loop = loop_ptrs(c);
   h.cond_while = cond_while; h.cond_if = cond_if; h.cond_if1 = cond_if1; h.cond_if8 = cond_if8;
+  if (which == 0) { h.cond_switch = c->sw_handle; h.sw_bodies = c->sw_bodies; }
   h.pass_kind = which == 0 ? 0 : MBv == 1 ? 2 : MBv == SUB_MB ? 3 : 1;
   if (c->draw) {   // sampling: the head leaves its logits and the policy step to the kernel that draws the token
     if (!h.logits_dbg) h.logits_dbg = m.logits;
@@ -1141,6 +1152,12 @@ int build_graphs(bild_ctx* c, int base) {
   const bool want_pdl = c->use_pdl;
   c->draw = base == 2;
   int rc = build_graphs_once(c, base);
+  if (rc != BILD_OK && c->graph_switch) {   // no SWITCH nodes here: one IF node per kind of pass
+    drop_graphs(c);
+    cudaGetLastError();
+    c->graph_switch = false;
+    rc = build_graphs_once(c, base);
+  }
   if (rc != BILD_OK && want_pdl) {
     drop_graphs(c);
     cudaGetLastError();
@@ -1173,6 +1190,32 @@ int build_graphs_once(bild_ctx* c, int base) {
     int rc = add_cond(c, graph[0], nullptr, 0, hw, cudaGraphCondTypeWhile, &body);
     if (rc) return rc;
     std::vector<cudaGraphNode_t> leaves;
+    if (c->graph_switch) {   // one conditional node per iteration: SWITCH { block pass | single-row pass | pass of 2 to 8 rows }
+      const int nb = body8 ? 3 : 2;
+      cudaGraphConditionalHandle hs;
+      CUDA_TRY(c, cudaGraphConditionalHandleCreate(&hs, graph[0], (unsigned)nb, cudaGraphCondAssignDefault));
+      c->sw_handle = hs; c->sw_bodies = nb;
+      rc = capture_pass(c, body, 0, 1, hw, 0, &leaves, &per_pass[0]);
+      c->sw_handle = 0; c->sw_bodies = 0;
+      if (rc) return rc;
+      cudaGraphNodeParams p = {cudaGraphNodeTypeConditional};
+      p.conditional.handle = hs;
+      p.conditional.type = cudaGraphCondTypeSwitch;
+      p.conditional.size = (unsigned)nb;
+      cudaGraphNode_t node;
+      CUDA_TRY(c, cudaGraphAddNode(&node, body, leaves.data(), leaves.size(), &p));
+      rc = capture_pass(c, p.conditional.phGraph_out[0], 1, MAXB, hw, 0, nullptr, &per_pass[1]);
+      if (rc) return rc;
+      int64_t n1 = 0;
+      rc = capture_pass(c, p.conditional.phGraph_out[1], 1, 1, hw, 0, nullptr, &n1);
+      if (rc) return rc;
+      per_pass_large1 = n1;
+      if (body8) {
+        rc = capture_pass(c, p.conditional.phGraph_out[2], 1, SUB_MB, hw, 0, nullptr, &per_pass_large8);
+        if (rc) return rc;
+      }
+      CUDA_TRY(c, cudaGraphInstantiate(&exec[0], graph[0], 0));
+    } else {
     rc = capture_pass(c, body, 0, 1, hw, hi, &leaves, &per_pass[0], hi1, hi8);
     if (rc) return rc;
     rc = add_cond(c, body, leaves.data(), leaves.size(), hi, cudaGraphCondTypeIf, &ifbody);
@@ -1193,6 +1236,7 @@ int build_graphs_once(bild_ctx* c, int base) {
       if (rc) return rc;
     }
     CUDA_TRY(c, cudaGraphInstantiate(&exec[0], graph[0], 0));
+    }
   }
   {  // large-only greedy: WHILE { large pass with k = 1 }
     CUDA_TRY(c, cudaGraphCreate(&graph[1], 0));
@@ -1256,7 +1300,7 @@ void bild_tuning_default(bild_tuning* t) {
   t->host_loop = 0; t->pdl = 1; t->fused = 2; t->ffn_parts = 0; t->block_simt = 0; t->slice_mode = 2;
   t->slice_min_kb = 3000; t->slice_mma_min = 3; t->slice_head = 2; t->slice_head_min_mb = 32; t->unit_attn = 1;
   t->umma = 1; t->enc_gemm = 1; t->enc_attn_mma = 1; t->enc_parallel = 1; t->spin_limit = 0; t->debug_skip_copies = 0;
-  t->attn_all_keys = 128;
+  t->attn_all_keys = 128; t->graph_switch = 1; t->enc_split_k = 1;
 }
 
 int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_weights* large_w, void* workspace,
@@ -1301,6 +1345,8 @@ int bild_create_tuned(const bild_config* cfg, const bild_weights* small_w, const
     c->spin_limit = t.spin_limit > 0 ? (unsigned)t.spin_limit : SPIN_LIMIT;
     c->debug_skip_copies = t.debug_skip_copies != 0;
     c->attn_all_keys = std::min(128, std::max(0, t.attn_all_keys));
+    c->graph_switch = t.graph_switch != 0;
+    c->enc_split_k = t.enc_split_k != 0;
   }
   {
     int dev = 0;

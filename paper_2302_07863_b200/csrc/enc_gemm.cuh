@@ -13,6 +13,9 @@
 //     scatter to q and the K/V layout, writing 32 consecutive outputs of one token per warp;
 //   * the FFN's first matrix can write its output directly as the bf16 head / remainder pair that
 //     the second matrix reads (no fp32 round trip, no separate split);
+//   * matrices with few output rows and a long K (output projection, second FFN matrix: 32 tiles for 512 tokens of the
+//     T5-large shape) are split over K as well (grid.z): every split adds its partial tile to the residual stream with
+//     reductions at the L2 (the stream holds the old values already), so that the GEMM covers the SMs;
 //   * every wait on an mbarrier is bounded (error code, then the block carries on and frees its
 //     tensor memory).
 #pragma once
@@ -100,7 +103,9 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
   extern __shared__ unsigned char eg_raw[];
   const int tid = threadIdx.x, warp = tid >> 5;
   const int n_base = blockIdx.x * UM_TILE_M, tok0 = blockIdx.y * EG_TOK;
-  const int nkb = a.K / UM_KB;
+  // this block's share of the K blocks (gridDim.z splits, EPI_RESID only)
+  const int nkb_all = a.K / UM_KB, kb0 = (int)(((long long)blockIdx.z * nkb_all) / gridDim.z);
+  const int nkb = (int)(((long long)(blockIdx.z + 1) * nkb_all) / gridDim.z) - kb0;
   unsigned char* base = (unsigned char*)(((uintptr_t)eg_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* full = (uint64_t*)(base + (size_t)NST * STAGE);
   uint64_t* empty = full + NST;
@@ -125,14 +130,14 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
     unsigned char* st = base + (size_t)(kb % NST) * STAGE;
     uint64_t* bar = &full[kb % NST];
     mbar_expect_tx(bar, STAGE);
-    tma_load_2d(st, &tmW0, kb * UM_KB, n_base, bar);
-    if (GATED) tma_load_2d(st + 16384, &tmW1, kb * UM_KB, n_base, bar);
+    tma_load_2d(st, &tmW0, (kb0 + kb) * UM_KB, n_base, bar);
+    if (GATED) tma_load_2d(st + 16384, &tmW1, (kb0 + kb) * UM_KB, n_base, bar);
   };
   auto load_acts = [&](int kb) {
     unsigned char* st = base + (size_t)(kb % NST) * STAGE;
     uint64_t* bar = &full[kb % NST];
-    tma_load_2d(st + NMAT * 16384, &tmHh, kb * UM_KB, tok0, bar);
-    tma_load_2d(st + (NMAT + 1) * 16384, &tmHl, kb * UM_KB, tok0, bar);
+    tma_load_2d(st + NMAT * 16384, &tmHh, (kb0 + kb) * UM_KB, tok0, bar);
+    tma_load_2d(st + (NMAT + 1) * 16384, &tmHl, (kb0 + kb) * UM_KB, tok0, bar);
   };
   if (tid == 0)
     for (int kb = 0; kb < nkb && kb < NST; ++kb) load_weights(kb);
@@ -192,6 +197,12 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
       for (int j = 0; j < 16; ++j) v1[j] += lo16[j];
     }
     if (!row_ok) continue;
+    if (a.epi == EPI_RESID && gridDim.z > 1) {   // split over K: the partial tile is added to the stream where it lies
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (tok0 + c0 + j < a.M) atomicAdd(a.Y + (size_t)(tok0 + c0 + j) * a.ldy + n, v0[j]);
+      continue;
+    }
     if (a.epi == EPI_RESID) {   // all 16 old values are requested before any of them is needed
       float old[16];
 #pragma unroll

@@ -481,6 +481,10 @@ struct HeadArgs {
   unsigned long long cond_while, cond_if;
   unsigned long long cond_if1;   // IF node of the single-row large pass (0: the block branch takes every large pass)
   unsigned long long cond_if8;   // IF node of the large pass over 2 to 8 rows (0: the block branch takes them)
+  // one SWITCH node instead of the IF nodes: body 0 the block pass, body 1 the single-row pass, body 2 (if sw_bodies is 3)
+  // the pass over 2 to 8 rows; the value sw_bodies runs none
+  unsigned long long cond_switch;
+  int sw_bodies;
   int pass_kind;                 // which pass counter the kernel bumps inside a loop graph: 0 small, 1 block, 2 single row, 3 up to 8 rows
   int defer_policy;              // sampling: the head leaves policy and loop control to the kernel that draws the token
 };
@@ -505,6 +509,8 @@ __device__ inline void policy_tail(const HeadArgs& a, HeadOut* o) {
   if (a.cond_if) cudaGraphSetConditional(a.cond_if, (fb && !one_row && !upto8) ? 1u : 0u);
   if (a.cond_if1) cudaGraphSetConditional(a.cond_if1, one_row ? 1u : 0u);
   if (a.cond_if8) cudaGraphSetConditional(a.cond_if8, upto8 ? 1u : 0u);
+  if (a.cond_switch)
+    cudaGraphSetConditional(a.cond_switch, !fb ? (unsigned)a.sw_bodies : kn == 1 ? 1u : (a.sw_bodies == 3 && kn <= 8) ? 2u : 0u);
 }
 
 constexpr int HEAD_THREADS = 256;

@@ -17,6 +17,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="t5_sum")
     ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--tuning", default="", help="bild_tuning fields, e.g. enc_split_k=0,enc_parallel=0")
     a = ap.parse_args()
     import torch
     assert torch.cuda.is_available(), "needs a CUDA device"
@@ -26,7 +27,8 @@ def main():
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     with open(os.path.join(root, "tests", "golden", a.workload + ".json")) as f:
         g = json.load(f)
-    ctx, ids, wl = make_context(a.workload, g["scale_small"]["scale"], g["scale_large"]["scale"])
+    tuning = {k: int(v) for k, v in (kv.split("=") for kv in a.tuning.split(",") if kv)} or None
+    ctx, ids, wl = make_context(a.workload, g["scale_small"]["scale"], g["scale_large"]["scale"], tuning=tuning)
     for _ in range(3):
         ctx.encode(ids)
     torch.cuda.synchronize()
