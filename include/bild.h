@@ -174,7 +174,9 @@ int bild_create(const bild_config *cfg /*HOST*/, const bild_weights *small_w /*H
 typedef struct {
   int32_t host_loop;         /* 1: bild_generate is driven from the host, one state read-back per pass (debug) */
   int32_t pdl;               /* 1: kernels of a pass are launched with programmatic dependent launch */
-  int32_t fused;             /* fused sub-layer kernels: 0 off, 1 single-row passes, 2 also passes of 2 to 8 rows */
+  int32_t fused;             /* fused sub-layer kernels: 0 off, 1 single-row passes, 2 also passes of 2 to 8 rows, 3 also
+                              * blocks of 9 to 16 rows (as two chunks of up to 8 rows on two streams, layer l of the second
+                              * chunk waiting for the self-attention of layer l of the first) */
   int32_t ffn_parts;         /* launches the fused feed-forward sub-layer is split into (0: fewest that fit) */
   int32_t block_simt;        /* 1: unfused block passes on the SIMT block GEMV */
   int32_t slice_mode;        /* unfused linear layers on the row-slice kernel: 0 off, 1 block passes, 2 also single rows */

@@ -121,6 +121,8 @@ struct Model {
   int sub_C = 1;                     // blocks per head (cluster size) of the attention sub-layers
   uint4* wfo_one = nullptr;          // [layers][F / 8][d] W_fo in the load order of the fused feed-forward kernels
   uint4* wfo_blk = nullptr;          // [layers][F / 8][pack_wfo_dpad(d)]
+  CallDesc* desc_lo = nullptr;       // the two chunks of a block of 9 to 16 rows (split_desc_kernel)
+  CallDesc* desc_hi = nullptr;
   AttnSubPlan sub_self{}, sub_cross{};   // chunk sizes of the attention sub-layers
   int sub_parts = 1;                 // launches the feed-forward sub-layer is split into
 };
@@ -164,6 +166,8 @@ struct bild_ctx {
   int64_t per_pass[2] = {0, 0};      // kernel launches in one small / one large pass of the graphs
   int64_t per_pass_large1 = 0, per_pass_large8 = 0;
   int64_t* cnt = &launches;         // where launches are counted (redirected while capturing)
+  cudaStream_t side2 = nullptr;       // second chunk of a block of 9 to 16 rows (fused sub-layer kernels)
+  std::vector<cudaEvent_t> chunk_ev;  // per layer: first chunk's self-attention done; then fork and join
   cudaStream_t cap_stream = nullptr;  // capture only (the legacy default stream cannot capture); nothing runs on it
   bool block_simt = false;           // block pass on the SIMT block GEMV instead of the tensor-core kernel
   bool use_pdl = true;               // launch pass kernels with programmatic stream serialization
@@ -184,7 +188,7 @@ struct bild_ctx {
   size_t slice_head_min_bytes = (size_t)32 << 20;
   int slice_mma_min = 3;
   size_t slice_min_bytes = 3000 * 1024;   // single-row passes: smaller matrices stay on the GEMV (measured)
-  int fused_on = 2;                  // fused sub-layer kernels where the shapes allow: 0 off, 1 single-row passes, 2 also passes of 2 to 8 rows
+  int fused_on = 3;                  // fused sub-layer kernels where the shapes allow: 0 off, 1 single-row passes, 2 also passes of 2 to 8 rows, 3 also 9 to 16 rows (two chunks)
   int sub_parts_want = 0;            // 0: fewest launches of the feed-forward sub-layer that fit
   bool use_umma = true, use_enc_gemm = true;
   unsigned spin_limit = SPIN_LIMIT;
@@ -287,6 +291,8 @@ void plan(bild_ctx* c, Bump& b) {
     m.head_cnt = b.take<unsigned>(1);
     m.head_out = b.take<HeadOut>(1);
     m.desc = b.take<CallDesc>(1);
+    m.desc_lo = b.take<CallDesc>(1);
+    m.desc_hi = b.take<CallDesc>(1);
     m.logits = b.take<float>((size_t)MAXB * mc.vocab);
     m.xb = b.take<float>((size_t)MAXB * mc.d_model);
     m.xc = b.take<float>((size_t)MAXB * mc.d_model);
@@ -687,12 +693,12 @@ int setup_fused(bild_ctx* c, Model& m) {
 }
 
 template <typename Arg>
-cudaError_t launch_sub(bild_ctx* c, void (*kern)(Arg), int grid, int cluster, size_t smem, const Arg& a) {
+cudaError_t launch_sub(bild_ctx* c, void (*kern)(Arg), int grid, int cluster, size_t smem, const Arg& a, bool pdl_ok = true) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid); cfg.blockDim = dim3(SUB_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
   cudaLaunchAttribute at[2];
   int na = 0;
-  if (c->use_pdl) {
+  if (c->use_pdl && pdl_ok) {
     at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[na].val.programmaticStreamSerializationAllowed = 1;
     ++na;
@@ -707,49 +713,100 @@ cudaError_t launch_sub(bild_ctx* c, void (*kern)(Arg), int grid, int cluster, si
   return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
-// The layers of a decoder pass on the fused sub-layer kernels: the residual stream goes x -> xb -> xc -> x
-// per layer (self-attention, cross-attention, feed-forward), each kernel clearing the buffer after its output.
-int fused_layers(bild_ctx* c, Model& m, int MB) {
+// One layer of a decoder pass on the fused sub-layer kernels: the residual stream goes x -> xb -> xc -> x (self-attention,
+// cross-attention, feed-forward), each kernel clearing the buffer after its output.  desc / row0: the rows the kernels
+// work on (a whole pass, or one chunk of a block of 9 to 16 rows); first_plain: the layer's first kernel follows a
+// dependency on another stream and is launched without the programmatic-launch attribute; after_self: called once the
+// self-attention kernel is in the stream (its keys and values are what the next chunk's same layer waits for).
+template <typename F>
+int fused_layer(bild_ctx* c, Model& m, int MB, int l, const CallDesc* desc, int row0, bool first_plain, F after_self) {
   const bild_model_cfg& mc = m.c;
-  const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
+  const int d = mc.d_model, I = m.inner, Fd = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
   const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len;
   const bool gated = mc.ffn_kind == BILD_FFN_GATED_GELU;
   const int C = m.sub_C;
-  for (int l = 0; l < mc.n_layers; ++l) {
-    const bild_dec_layer& w = m.dec[l];
-    const size_t kvoff = (size_t)l * H * dkv;
-    AttnSubArgs a{};
-    a.desc = m.desc; a.eps = mc.ln_eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
-    a.mb = MB; a.err = &c->st->err; a.x_rows = MAXB;
-    a.spin = c->spin_limit; a.skip_copies = c->debug_skip_copies ? 1 : 0;
-    a.n_keys_dev = c->enc_len_dev;
-    // S1-S3 / L1-L3
-    a.x_in = m.x; a.x_out = m.xb; a.x_zero = m.xc; a.gain = (const float*)w.ln1;
-    a.Wp = (const __nv_bfloat16*)w.wqkv; a.Wo = (const __nv_bfloat16*)w.wo;
-    a.kc = m.selfK + kvoff * cap; a.vc = m.selfV + kvoff * cap; a.cap = cap; a.bias = m.dec_bias; a.bias_ld = cap; a.self = 1;
-    a.kc_keys = m.sub_self.kc; a.bias_len = m.sub_self.bias_len; a.red_keys = m.sub_self.red_keys;
-    a.L = attn_sub_layout(d, dkv, 3, C, MB, a.kc_keys, a.bias_len);
-    CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
-    // S4-S6 / L4-L6
-    a.x_in = m.xb; a.x_out = m.xc; a.x_zero = m.x; a.gain = (const float*)w.ln2;
-    a.Wp = (const __nv_bfloat16*)w.wcq; a.Wo = (const __nv_bfloat16*)w.wco;
-    a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.bias = nullptr; a.bias_ld = 0; a.self = 0;
-    a.kc_keys = m.sub_cross.kc; a.bias_len = m.sub_cross.bias_len; a.red_keys = m.sub_cross.red_keys;
-    a.L = attn_sub_layout(d, dkv, 1, C, MB, a.kc_keys, a.bias_len);
-    CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
-    // S7-S8 / L7-L8
-    FfnSubArgs f{};
-    f.x_rows = MAXB;
-    f.desc = m.desc; f.eps = mc.ln_eps; f.d = d; f.F = F; f.gated = gated ? 1 : 0; f.mb = MB; f.spin = c->spin_limit;
-    f.err = &c->st->err; f.x_in = m.xc; f.x_out = m.x; f.gain = (const float*)w.ln3;
-    f.Wi0 = (const __nv_bfloat16*)w.wi0; f.Wi1 = (const __nv_bfloat16*)w.wi1; f.Wfo1 = m.wfo_one + (size_t)l * (F / 8) * d; f.Wfo8 = m.wfo_blk + (size_t)l * (F / 8) * pack_wfo_dpad(d);
-    f.nparts = m.sub_parts;
-    f.L = ffn_sub_layout(d, F, gated, c->sms * m.sub_parts, c->sms, MB);
-    for (int p = 0; p < m.sub_parts; ++p) {
-      f.part = p; f.seed = p == 0 ? 1 : 0; f.x_zero = p == 0 ? m.xb : nullptr;
-      CUDA_TRY(c, launch_sub(c, MB == 1 ? ffn_sub_kernel<true> : ffn_sub_kernel<false>, c->sms, 1, (size_t)f.L.total, f));
-    }
+  float* x = m.x + (size_t)row0 * d;
+  float* xb = m.xb + (size_t)row0 * d;
+  float* xc = m.xc + (size_t)row0 * d;
+  const bild_dec_layer& w = m.dec[l];
+  const size_t kvoff = (size_t)l * H * dkv;
+  AttnSubArgs a{};
+  a.desc = desc; a.eps = mc.ln_eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
+  a.mb = MB; a.err = &c->st->err; a.x_rows = MAXB - row0;
+  a.spin = c->spin_limit; a.skip_copies = c->debug_skip_copies ? 1 : 0;
+  a.n_keys_dev = c->enc_len_dev;
+  // S1-S3 / L1-L3
+  a.x_in = x; a.x_out = xb; a.x_zero = xc; a.gain = (const float*)w.ln1;
+  a.Wp = (const __nv_bfloat16*)w.wqkv; a.Wo = (const __nv_bfloat16*)w.wo;
+  a.kc = m.selfK + kvoff * cap; a.vc = m.selfV + kvoff * cap; a.cap = cap; a.bias = m.dec_bias; a.bias_ld = cap; a.self = 1;
+  a.kc_keys = m.sub_self.kc; a.bias_len = m.sub_self.bias_len; a.red_keys = m.sub_self.red_keys;
+  a.L = attn_sub_layout(d, dkv, 3, C, MB, a.kc_keys, a.bias_len);
+  CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a, !first_plain));
+  int rc = after_self();
+  if (rc) return rc;
+  // S4-S6 / L4-L6
+  a.x_in = xb; a.x_out = xc; a.x_zero = x; a.gain = (const float*)w.ln2;
+  a.Wp = (const __nv_bfloat16*)w.wcq; a.Wo = (const __nv_bfloat16*)w.wco;
+  a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.bias = nullptr; a.bias_ld = 0; a.self = 0;
+  a.kc_keys = m.sub_cross.kc; a.bias_len = m.sub_cross.bias_len; a.red_keys = m.sub_cross.red_keys;
+  a.L = attn_sub_layout(d, dkv, 1, C, MB, a.kc_keys, a.bias_len);
+  CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
+  // S7-S8 / L7-L8
+  FfnSubArgs f{};
+  f.x_rows = MAXB - row0;
+  f.desc = desc; f.eps = mc.ln_eps; f.d = d; f.F = Fd; f.gated = gated ? 1 : 0; f.mb = MB; f.spin = c->spin_limit;
+  f.err = &c->st->err; f.x_in = xc; f.x_out = x; f.gain = (const float*)w.ln3;
+  f.Wi0 = (const __nv_bfloat16*)w.wi0; f.Wi1 = (const __nv_bfloat16*)w.wi1;
+  f.Wfo1 = m.wfo_one + (size_t)l * (Fd / 8) * d; f.Wfo8 = m.wfo_blk + (size_t)l * (Fd / 8) * pack_wfo_dpad(d);
+  f.nparts = m.sub_parts;
+  f.L = ffn_sub_layout(d, Fd, gated, c->sms * m.sub_parts, c->sms, MB);
+  for (int p = 0; p < m.sub_parts; ++p) {
+    f.part = p; f.seed = p == 0 ? 1 : 0; f.x_zero = p == 0 ? xb : nullptr;
+    CUDA_TRY(c, launch_sub(c, MB == 1 ? ffn_sub_kernel<true> : ffn_sub_kernel<false>, c->sms, 1, (size_t)f.L.total, f));
   }
+  return BILD_OK;
+}
+
+int fused_layers(bild_ctx* c, Model& m, int MB) {
+  for (int l = 0; l < m.c.n_layers; ++l) {
+    int rc = fused_layer(c, m, MB, l, m.desc, 0, false, [] { return (int)BILD_OK; });
+    if (rc) return rc;
+  }
+  return BILD_OK;
+}
+
+// A block of 9 to 16 rows on the fused sub-layer kernels: two chunks (rows 0..7, then the rest) on two streams, layer l of
+// the second chunk waiting only for the self-attention kernel of layer l of the first (whose keys and values it attends
+// over), so that the two chunks run side by side, one layer apart.  On return the context's stream has both behind it.
+int fused_layers_two_chunks(bild_ctx* c, Model& m) {
+  const int L = m.c.n_layers;
+  if (!c->side2) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->side2, cudaStreamNonBlocking));
+  while ((int)c->chunk_ev.size() < L + 2) {
+    cudaEvent_t e;
+    CUDA_TRY(c, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    c->chunk_ev.push_back(e);
+  }
+  cudaStream_t s0 = c->stream, s1 = c->side2;
+  split_desc_kernel<<<1, 1, 0, s0>>>(m.desc, m.desc_lo, m.desc_hi);
+  (*c->cnt)++;
+  CUDA_TRY(c, cudaGetLastError());
+  CUDA_TRY(c, cudaEventRecord(c->chunk_ev[L], s0));
+  CUDA_TRY(c, cudaStreamWaitEvent(s1, c->chunk_ev[L], 0));
+  int rc = BILD_OK;
+  for (int l = 0; l < L && rc == BILD_OK; ++l) {
+    rc = fused_layer(c, m, SUB_MB, l, m.desc_lo, 0, l == 0, [&] {
+      CUDA_TRY(c, cudaEventRecord(c->chunk_ev[l], s0));
+      return (int)BILD_OK;
+    });
+    if (rc) break;
+    CUDA_TRY(c, cudaStreamWaitEvent(s1, c->chunk_ev[l], 0));
+    c->stream = s1;
+    rc = fused_layer(c, m, SUB_MB, l, m.desc_hi, SUB_CHUNK, true, [] { return (int)BILD_OK; });
+    c->stream = s0;
+  }
+  if (rc) return rc;
+  CUDA_TRY(c, cudaEventRecord(c->chunk_ev[L + 1], s1));
+  CUDA_TRY(c, cudaStreamWaitEvent(s0, c->chunk_ev[L + 1], 0));
   return BILD_OK;
 }
 
@@ -925,12 +982,17 @@ int decoder_pass(bild_ctx* c, int which, int MBv, float* logits_dbg, unsigned lo
   const bild_model_cfg& mc = m.c;
   const int d = mc.d_model, I = m.inner, F = mc.d_ff, H = mc.n_heads, dkv = mc.d_kv;
   const int cap = c->cfg.max_dec_len, ecap = c->cfg.max_enc_len, dt = c->cfg.dtype;
-  const bool fused = m.fused && (MBv == 1 || (MBv == SUB_MB && c->fused_on >= 2));
+  // blocks of 9 to 16 rows: two chunks of the 8-row kernels side by side (the caller guarantees more than 8 rows)
+  const bool chunked = m.fused && which == 1 && MBv == MAXB && c->fused_on >= 3;
+  const bool fused = chunked || (m.fused && (MBv == 1 || (MBv == SUB_MB && c->fused_on >= 2)));
   CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x, fused ? m.xb : nullptr));
   if (fused) {
-    int rc = fused_layers(c, m, MBv);
+    int rc = chunked ? fused_layers_two_chunks(c, m) : fused_layers(c, m, MBv);
     if (rc) return rc;
   }
+  const bool pdl_was = c->use_pdl;
+  if (chunked) c->use_pdl = false;   // the head follows the join of two streams: a plain launch
+  struct PdlRestore { bild_ctx* c; bool v; ~PdlRestore() { c->use_pdl = v; } } pdl_restore{c, pdl_was};
   // self-attention: one block per head up to 128 cached rows (no merge step); cross-attention:
   // enough splits of the encoder keys to occupy the SMs
   int ns_self = 1;
@@ -1297,7 +1359,7 @@ int bild_query_workspace(const bild_config* cfg, size_t* bytes) {
 
 void bild_tuning_default(bild_tuning* t) {
   if (!t) return;
-  t->host_loop = 0; t->pdl = 1; t->fused = 2; t->ffn_parts = 0; t->block_simt = 0; t->slice_mode = 2;
+  t->host_loop = 0; t->pdl = 1; t->fused = 3; t->ffn_parts = 0; t->block_simt = 0; t->slice_mode = 2;
   t->slice_min_kb = 3000; t->slice_mma_min = 3; t->slice_head = 2; t->slice_head_min_mb = 32; t->unit_attn = 1;
   t->umma = 1; t->enc_gemm = 1; t->enc_attn_mma = 1; t->enc_parallel = 1; t->spin_limit = 0; t->debug_skip_copies = 0;
   t->attn_all_keys = 128; t->graph_switch = 1; t->enc_split_k = 1;
@@ -1329,7 +1391,7 @@ int bild_create_tuned(const bild_config* cfg, const bild_weights* small_w, const
     if (tuning) t = *tuning;
     c->host_loop = t.host_loop != 0;
     c->use_pdl = t.pdl != 0;
-    c->fused_on = std::min(2, std::max(0, t.fused));
+    c->fused_on = std::min(3, std::max(0, t.fused));
     c->sub_parts_want = std::min(8, std::max(0, t.ffn_parts));
     c->block_simt = t.block_simt != 0;
     c->slice_mode = std::min(2, std::max(0, t.slice_mode));
@@ -1407,6 +1469,8 @@ void bild_destroy(bild_ctx* c) {
   if (!c) return;
   drop_graphs(c);
   if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+  if (c->side2) { cudaStreamSynchronize(c->side2); cudaStreamDestroy(c->side2); }
+  for (cudaEvent_t e : c->chunk_ev) cudaEventDestroy(e);
   if (c->enc_stream) { cudaStreamSynchronize(c->enc_stream); cudaStreamDestroy(c->enc_stream); }
   if (c->enc_fork) cudaEventDestroy(c->enc_fork);
   if (c->enc_join) cudaEventDestroy(c->enc_join);

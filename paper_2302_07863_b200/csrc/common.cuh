@@ -13,6 +13,8 @@ constexpr int MAXB = BILD_MAX_BLOCK;  // largest block of tokens one decoder pas
 // What one decoder pass works on.  Written on the device by the policy code (or by a
 // tiny set-up kernel for the single-step entry points), read by every kernel of the
 // pass, so that a captured launch sequence can be replayed with new values.
+constexpr int SUB_CHUNK = 8;   // rows of a chunk when a block of 9 to 16 rows runs on the fused sub-layer kernels
+
 struct CallDesc {
   int k;              // rows in this pass (1 for a small-model step)
   int pos0;           // position of row 0 = number of rows already in the self cache

@@ -675,6 +675,14 @@ __global__ void set_desc_at_kernel(CallDesc* d, int k, int pos0, TokList toks) {
   }
 }
 
+// A block of 9 to 16 rows as two chunks for the fused sub-layer kernels: rows 0..7 and the rest, the second chunk at
+// the cache position right after the first.
+__global__ void split_desc_kernel(const CallDesc* d, CallDesc* lo, CallDesc* hi) {
+  const int k = d->k, klo = k < SUB_CHUNK ? k : SUB_CHUNK;
+  lo->k = klo; lo->pos0 = d->pos0; lo->run_policy = 0;
+  hi->k = k - klo; hi->pos0 = d->pos0 + klo; hi->run_policy = 0;
+}
+
 __global__ void set_alpha_kernel(DevState* st, float alpha_fb, float alpha_rb) {
   st->alpha_fb = alpha_fb;
   st->alpha_rb = alpha_rb;
