@@ -200,6 +200,8 @@ typedef struct {
                               * kind of pass */
   int32_t enc_split_k;       /* 1: encoder GEMMs that add to the residual stream (output projection, second FFN matrix)
                               * split K over more blocks, partial tiles added with reductions at the L2 */
+  int32_t head_stream;       /* single-row bf16 LM heads (rows of at most 1024 columns) on the streaming kernel: 0 off,
+                              * 1 heads of slice_head_min_mb and more, 2 all */
 } bild_tuning;
 void bild_tuning_default(bild_tuning *t /*HOST out*/);
 /* bild_create with explicit switches; tuning == NULL means the defaults. */
@@ -301,7 +303,8 @@ const char *bild_last_error(const bild_ctx *ctx); /* HOST string owned by the co
  * One kernel (or one sub-layer) run once on the given stream, every pointer DEVICE unless said
  * otherwise.  bild_op_linear and bild_op_lm_head run the per-operation kernels (GEMV / SIMT linear,
  * single-row and SIMT heads) that fp32 configurations and odd shapes use; bild_op_lm_head_sliced,
- * bild_op_attn_sublayer and bild_op_ffn_sublayer run the kernels the bf16 decoder passes use. */
+ * bild_op_lm_head_stream, bild_op_attn_sublayer and bild_op_ffn_sublayer run the kernels the bf16
+ * decoder passes use. */
 
 /* Y[m][n] = sum_j W[n][j] * H[m][j], H = X if gain == NULL, else the RMS norm of X
  * with that gain (Section 3.2's model forward; one weight pass serves all m rows).
@@ -329,6 +332,14 @@ int bild_op_lm_head_sliced(const void *W, const float *X, const float *gain, flo
                            const int32_t *target, int M, int V, int K, int32_t *argmax_out,
                            float *max_out, float *lse_out, float *gather_out, float *logits_dbg,
                            void *scratch, void *cuda_stream);
+
+/* The same fused head for ONE row on the streaming kernel of the bf16 single-row passes (two blocks per SM walk the
+ * vocabulary, weights through registers): W bf16 [V][K], 16-byte aligned, K <= 1024 (else BILD_ERR_CAPACITY), X [K].
+ * scratch as for bild_op_lm_head.  Asynchronous on the stream. */
+int bild_op_lm_head_stream(const void *W, const float *X, const float *gain, float eps, float scale,
+                           const int32_t *target, int V, int K, int32_t *argmax_out, float *max_out,
+                           float *lse_out, float *gather_out, float *logits_dbg, void *scratch,
+                           void *cuda_stream);
 
 /* One decoder sub-layer on the fused kernels of the bf16 passes (Section 3.2's model forward, one
  * weight pass for all M rows; steps S1-S3 / S4-S6 / S7-S8 of the small step, L1-L8 of the block

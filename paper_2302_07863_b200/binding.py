@@ -26,7 +26,7 @@ EXPORTS = ["bild_query_workspace", "bild_create", "bild_create_tuned", "bild_tun
            "bild_small_step", "bild_large_verify", "bild_rewind", "bild_generate", "bild_generate_async",
            "bild_fetch_result", "bild_time_pass", "bild_uses_tensor_cores", "bild_launch_count", "bild_last_error", "bild_op_linear",
            "bild_op_lm_head_scratch_bytes", "bild_op_lm_head", "bild_op_lm_head_static", "bild_debug_bucket",
-           "bild_debug_read_cache", "bild_op_lm_head_sliced", "bild_op_sublayer_scratch_bytes", "bild_op_attn_sublayer",
+           "bild_debug_read_cache", "bild_op_lm_head_sliced", "bild_op_lm_head_stream", "bild_op_sublayer_scratch_bytes", "bild_op_attn_sublayer",
            "bild_op_ffn_sublayer", "bild_generate_sampled"]
 
 
@@ -60,7 +60,7 @@ class Tuning(C.Structure):
     """bild_tuning: kernel selection and debugging switches (defaults from bild_tuning_default)."""
     _fields_ = [(n, C.c_int32) for n in ("host_loop", "pdl", "fused", "ffn_parts", "block_simt", "slice_mode", "slice_min_kb",
                                          "slice_mma_min", "slice_head", "slice_head_min_mb", "unit_attn", "umma", "enc_gemm",
-                                         "enc_attn_mma", "enc_parallel", "spin_limit", "debug_skip_copies", "attn_all_keys", "graph_switch", "enc_split_k")]
+                                         "enc_attn_mma", "enc_parallel", "spin_limit", "debug_skip_copies", "attn_all_keys", "graph_switch", "enc_split_k", "head_stream")]
 
 
 class StepOut(C.Structure):
@@ -365,6 +365,30 @@ def op_lm_head_sliced(W, X, gain, eps, scale, target, M, V, K, want_logits=False
                                   lse.data_ptr(), ga.data_ptr(), lg.data_ptr() if lg is not None else None, sp, None)
     if rc != BILD_OK:
         raise BildError(rc, "bild_op_lm_head_sliced")
+    return am, mx, lse, ga, lg
+
+
+def op_lm_head_stream(W, X, gain, eps, scale, target, V, K, want_logits=False):
+    """bild_op_lm_head_stream: the streaming head of the bf16 single-row passes (one row, bf16 weights, K <= 1024)."""
+    import torch
+    dev = X.device
+    L = lib()
+    L.bild_op_lm_head_scratch_bytes.restype = C.c_size_t
+    nb = L.bild_op_lm_head_scratch_bytes(V)
+    scratch = torch.zeros(nb + 512, dtype=torch.uint8, device=dev)
+    sp = (scratch.data_ptr() + 255) // 256 * 256
+    am = torch.empty(1, dtype=torch.int32, device=dev)
+    mx = torch.empty(1, dtype=torch.float32, device=dev)
+    lse = torch.empty(1, dtype=torch.float32, device=dev)
+    ga = torch.zeros(1, dtype=torch.float32, device=dev)
+    lg = torch.empty((1, V), dtype=torch.float32, device=dev) if want_logits else None
+    vp = C.c_void_p
+    L.bild_op_lm_head_stream.argtypes = [vp, vp, vp, C.c_float, C.c_float, vp, C.c_int, C.c_int, vp, vp, vp, vp, vp, vp, vp]
+    rc = L.bild_op_lm_head_stream(W.data_ptr(), X.data_ptr(), gain.data_ptr() if gain is not None else None, eps, scale,
+                                  target.data_ptr() if target is not None else None, V, K, am.data_ptr(), mx.data_ptr(),
+                                  lse.data_ptr(), ga.data_ptr(), lg.data_ptr() if lg is not None else None, sp, None)
+    if rc != BILD_OK:
+        raise BildError(rc, "bild_op_lm_head_stream")
     return am, mx, lse, ga, lg
 
 

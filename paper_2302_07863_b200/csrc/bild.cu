@@ -175,6 +175,7 @@ struct bild_ctx {
   int slice_mode = 2;                // row-slice linear kernel: 0 off, 1 block passes, 2 block and single-row passes
   int sms = 0;
   size_t slice_smem_set = 0;
+  int head_stream = 2;               // single-row bf16 heads on the streaming kernel: 0 off, 1 heads of slice_head_min_mb and more, 2 all
   bool enc_split_k = true;           // encoder GEMMs that add to the residual stream split K over grid.z (reductions at the L2)
   bool graph_switch = true;          // the large pass of a loop iteration hangs off one SWITCH node (else: one IF node per kind of pass)
   unsigned long long sw_handle = 0;  // while the small pass of such a loop is captured: the SWITCH node's handle and body count
@@ -532,6 +533,18 @@ cudaError_t launch_head1(bild_ctx* c, const HeadArgs& a, int64_t* launches) {
   if (nch <= 2) return launch_head1_t<WT, 2, 4>(c, a, launches);
   if (nch <= 4) return launch_head1_t<WT, 4, 2>(c, a, launches);
   return launch_head1_t<WT, 8, 1>(c, a, launches);
+}
+
+// Single row, bf16 weights, rows of at most 1024 columns: the streaming head (two blocks per SM walk the vocabulary).
+bool head_stream_fits(int dtype, int MB, const HeadArgs& a) {
+  return MB == 1 && dtype == BILD_BF16 && a.K % 8 == 0 && a.K <= 1024 && ((uintptr_t)a.W & 15) == 0;
+}
+cudaError_t launch_head_stream(bild_ctx* c, const HeadArgs& a, int sms) {
+  const int r = a.K <= 512 ? 8 : 4;
+  const dim3 grid(std::max(1, std::min(2 * sms, (a.V + 8 * r - 1) / (8 * r)))), block(HEAD1_THREADS);
+  if (a.K <= 256) return launch_k(c, head_stream_kernel<1, 8>, grid, block, 0, a);
+  if (a.K <= 512) return launch_k(c, head_stream_kernel<2, 8>, grid, block, 0, a);
+  return launch_k(c, head_stream_kernel<4, 4>, grid, block, 0, a);
 }
 
 cudaError_t launch_head(cudaStream_t s, bool pdl, int dtype, int MB, const HeadArgs& a, int grid, int64_t* launches) {
@@ -1065,6 +1078,10 @@ int decoder_pass(bild_ctx* c, int which, int MBv, float* logits_dbg, unsigned lo
   const size_t sh_smem = slice_head_smem_bytes(d, head_tr);
   // single-row passes: only heads of 32 MB and more (smaller ones stay on the GEMV head)
   const bool big_head = (size_t)mc.vocab * d * 2 >= c->slice_head_min_bytes;
+  if (c->head_stream >= (big_head ? 1 : 2) && c->sms > 0 && 2 * c->sms <= MAX_GRID_SM * 2 && head_stream_fits(dt, MB, h)) {
+    CUDA_TRY(c, launch_head_stream(c, h, c->sms));   // single row: the vocabulary streamed through registers
+    return draw_token();
+  }
   if (c->slice_head >= (MB == 1 ? 2 : 1) && (MB != 1 || big_head) && dt == BILD_BF16 && c->sms > 0 && c->sms <= MAX_GRID_SM && sh_smem <= 200 * 1024 &&
       d % 8 == 0 && ((uintptr_t)m.w.lm_head & 15) == 0) {
     // tensor-core head, one block per SM
@@ -1362,7 +1379,7 @@ void bild_tuning_default(bild_tuning* t) {
   t->host_loop = 0; t->pdl = 1; t->fused = 3; t->ffn_parts = 0; t->block_simt = 0; t->slice_mode = 2;
   t->slice_min_kb = 3000; t->slice_mma_min = 3; t->slice_head = 2; t->slice_head_min_mb = 32; t->unit_attn = 1;
   t->umma = 1; t->enc_gemm = 1; t->enc_attn_mma = 1; t->enc_parallel = 1; t->spin_limit = 0; t->debug_skip_copies = 0;
-  t->attn_all_keys = 128; t->graph_switch = 1; t->enc_split_k = 1;
+  t->attn_all_keys = 128; t->graph_switch = 1; t->enc_split_k = 1; t->head_stream = 2;
 }
 
 int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_weights* large_w, void* workspace,
@@ -1409,6 +1426,7 @@ int bild_create_tuned(const bild_config* cfg, const bild_weights* small_w, const
     c->attn_all_keys = std::min(128, std::max(0, t.attn_all_keys));
     c->graph_switch = t.graph_switch != 0;
     c->enc_split_k = t.enc_split_k != 0;
+    c->head_stream = std::min(2, std::max(0, t.head_stream));
   }
   {
     int dev = 0;
@@ -1898,6 +1916,38 @@ int bild_op_lm_head_sliced(const void* W, const float* X, const float* gain, flo
   if (e == cudaSuccess) e = cudaMemcpyAsync(max_out, o->zmax, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(lse_out, o->lse, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
   if (e == cudaSuccess && gather_out && target) e = cudaMemcpyAsync(gather_out, o->gather, M * sizeof(float), cudaMemcpyDeviceToDevice, s);
+  return e == cudaSuccess ? BILD_OK : BILD_ERR_CUDA;
+}
+
+int bild_op_lm_head_stream(const void* W, const float* X, const float* gain, float eps, float scale, const int32_t* target, int V,
+                           int K, int32_t* argmax_out, float* max_out, float* lse_out, float* gather_out, float* logits_dbg,
+                           void* scratch, void* cuda_stream) {
+  if (!W || !X || !scratch || !argmax_out || !max_out || !lse_out) return BILD_ERR_ARG;
+  if (V < 1 || K < 8 || K % 8 || ((uintptr_t)W & 15)) return BILD_ERR_ARG;
+  if (K > 1024) return BILD_ERR_CAPACITY;
+  if ((uintptr_t)scratch % 256) return BILD_ERR_WORKSPACE;
+  const int sms = op_sms();
+  if (sms < 1) return BILD_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  char* p = (char*)scratch;
+  HeadArgs h{};
+  h.partials = (Partial*)p;
+  p += align_up(head_partial_count(V) * sizeof(Partial), 256);
+  h.counter = (unsigned*)p;
+  p += 256;
+  h.out = (HeadOut*)p;
+  if (cudaMemsetAsync(h.counter, 0, 16, s) != cudaSuccess) return BILD_ERR_CUDA;
+  h.W = W; h.X = X; h.ldx = K; h.gain = gain; h.eps = eps; h.scale = scale; h.V = V; h.K = K; h.M = 1;
+  h.target = target; h.logits_dbg = logits_dbg; h.which = 1;
+  bild_ctx tmp;
+  tmp.stream = s;
+  tmp.use_pdl = false;
+  if (launch_head_stream(&tmp, h, sms) != cudaSuccess) return BILD_ERR_CUDA;
+  const HeadOut* o = h.out;
+  cudaError_t e = cudaMemcpyAsync(argmax_out, o->argmax, sizeof(int), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(max_out, o->zmax, sizeof(float), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(lse_out, o->lse, sizeof(float), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess && gather_out && target) e = cudaMemcpyAsync(gather_out, o->gather, sizeof(float), cudaMemcpyDeviceToDevice, s);
   return e == cudaSuccess ? BILD_OK : BILD_ERR_CUDA;
 }
 

@@ -702,6 +702,151 @@ __global__ void __launch_bounds__(HEAD1_THREADS) head1_kernel(HeadArgs a) {
 }
 
 // ---------------------------------------------------------------------------------
+// LM head for one row, bf16 weights, streaming variant: two blocks per SM stay for the whole vocabulary; every warp
+// owns a contiguous range of vocabulary rows and walks it R rows at a time, each batch requested with 16-byte loads
+// (R x NCH per lane, all issued before any is used; the first batch before the dependency wait), reduced R rows at
+// once (one shuffle per halving), with the running (max, arg, sum-exp) kept by the lane that ends up with a row's
+// total.  Sixteen warps an SM with 8 KB in flight each keep the memory busy without a ring in shared memory and
+// without the per-wave launch and load latency of the register-resident head above (one wave of 296 blocks holds a
+// third of a 32 MB head; a 256 MB head would take 26 waves).
+// ---------------------------------------------------------------------------------
+template <int NCH, int R>   // NCH chunks of 256 columns per row, R rows per batch
+__global__ void __launch_bounds__(HEAD1_THREADS, 2) head_stream_kernel(HeadArgs a) {
+  constexpr int NW = HEAD1_THREADS / 32, SH = R == 8 ? 2 : R == 4 ? 3 : 4;   // lane >> SH: the row of the batch this lane ends up with
+  __shared__ Partial s_p[HEAD1_THREADS];
+  __shared__ int s_last;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int K = a.K, V = a.V;
+  const int tw = gridDim.x * NW, gw = blockIdx.x * NW + warp;
+  const int per = ((V + tw - 1) / tw + R - 1) / R * R;   // rows per warp, whole batches
+  const int w0 = min(V, gw * per), w1 = min(V, w0 + per);
+  const __nv_bfloat16* W = (const __nv_bfloat16*)a.W;
+  uint4 w[R][NCH];
+  auto request = [&](int b) {
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int p = 0; p < NCH; ++p) {
+        const int c = p * 256 + lane * 8;
+        if (c < K) {
+          const __nv_bfloat16* src = W + (size_t)min(b + r, V - 1) * K + c;
+          asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[r][p].x), "=r"(w[r][p].y), "=r"(w[r][p].z), "=r"(w[r][p].w) : "l"(src));
+        }
+      }
+  };
+  if (w0 < w1) request(w0);
+  float gn[NCH][8];   // the norm gains are weights too
+  if (a.gain) {
+#pragma unroll
+    for (int p = 0; p < NCH; ++p) {
+      const int c = p * 256 + lane * 8;
+      if (c < K) {
+        const float4 g0 = __ldg(reinterpret_cast<const float4*>(a.gain + c)), g1 = __ldg(reinterpret_cast<const float4*>(a.gain + c + 4));
+        gn[p][0] = g0.x; gn[p][1] = g0.y; gn[p][2] = g0.z; gn[p][3] = g0.w; gn[p][4] = g1.x; gn[p][5] = g1.y; gn[p][6] = g1.z; gn[p][7] = g1.w;
+      }
+    }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  const int target = a.desc ? a.desc->targets[0] : (a.target ? a.target[0] : -1);
+  float h[NCH][8], ss = 0.f;
+#pragma unroll
+  for (int p = 0; p < NCH; ++p) {
+    const int c = p * 256 + lane * 8;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) h[p][i] = 0.f;
+    if (c < K) {
+      const float4 x0 = __ldcg(reinterpret_cast<const float4*>(a.X + c)), x1 = __ldcg(reinterpret_cast<const float4*>(a.X + c + 4));
+      h[p][0] = x0.x; h[p][1] = x0.y; h[p][2] = x0.z; h[p][3] = x0.w; h[p][4] = x1.x; h[p][5] = x1.y; h[p][6] = x1.z; h[p][7] = x1.w;
+      if (a.gain) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { ss += h[p][i] * h[p][i]; h[p][i] *= gn[p][i]; }
+      }
+    }
+  }
+  ss = warp_sum(ss);
+  const float mul = (a.gain ? rsqrtf(ss / (float)K + a.eps) : 1.f) * a.scale;
+  Partial run;
+  run.m = -INFINITY; run.s = 0.f; run.idx = 0x7fffffff;
+#pragma unroll 1
+  for (int b = w0; b < w1; b += R) {
+    float acc[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      float t = 0.f;
+#pragma unroll
+      for (int p = 0; p < NCH; ++p) {
+        if (p * 256 + lane * 8 < K) {
+          const uint4 q = w[r][p];
+          t += __uint_as_float(q.x << 16) * h[p][0] + __uint_as_float(q.x & 0xffff0000u) * h[p][1] + __uint_as_float(q.y << 16) * h[p][2] +
+               __uint_as_float(q.y & 0xffff0000u) * h[p][3] + __uint_as_float(q.z << 16) * h[p][4] + __uint_as_float(q.z & 0xffff0000u) * h[p][5] +
+               __uint_as_float(q.w << 16) * h[p][6] + __uint_as_float(q.w & 0xffff0000u) * h[p][7];
+        }
+      }
+      acc[r] = t;
+    }
+    if (b + R < w1) request(b + R);   // the next batch is on its way while this one is reduced
+    const float z = treduce<R>(acc, lane) * mul;
+    const int n = b + (lane >> SH);
+    if ((lane & ((1 << SH) - 1)) == 0 && n < w1) {
+      if (z > run.m) { run.s = run.s * __expf(run.m - z) + 1.f; run.m = z; run.idx = n; }
+      else run.s += __expf(z - run.m);
+      if (n == target) a.out->gather[0] = z;
+      if (a.logits_dbg) a.logits_dbg[n] = z;
+    }
+  }
+  // rows of a batch are in index order over the lanes, batches in index order over time: combining the lanes in lane
+  // order keeps the lowest index among equal maxima
+#pragma unroll
+  for (int o = 1 << SH; o < 32; o <<= 1) {
+    Partial q;
+    q.m = __shfl_xor_sync(0xffffffffu, run.m, o);
+    q.s = __shfl_xor_sync(0xffffffffu, run.s, o);
+    q.idx = __shfl_xor_sync(0xffffffffu, run.idx, o);
+    run = ((lane & o) == 0) ? combine(run, q) : combine(q, run);
+  }
+  if (lane == 0) s_p[warp] = run;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    Partial p = s_p[0];
+    for (int w2 = 1; w2 < NW; ++w2) p = combine(p, s_p[w2]);
+    a.partials[blockIdx.x] = p;
+    __threadfence();
+    const unsigned t = atomicAdd(a.counter, 1u);
+    s_last = (t == gridDim.x - 1);
+    if (s_last) *a.counter = 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  {   // merge: the grid has at most two blocks per SM, one partial each
+    Partial p;
+    p.m = -INFINITY; p.s = 0.f; p.idx = 0x7fffffff;
+    for (int b = threadIdx.x; b < (int)gridDim.x; b += HEAD1_THREADS) {
+      Partial t2;
+      t2.m = __ldcg(&a.partials[b].m); t2.s = __ldcg(&a.partials[b].s); t2.idx = __ldcg(&a.partials[b].idx);
+      p = combine(p, t2);
+    }
+    s_p[threadIdx.x] = p;
+  }
+  __syncthreads();
+  for (int stride = HEAD1_THREADS / 2; stride > 0; stride >>= 1) {
+    if (threadIdx.x < stride) s_p[threadIdx.x] = combine(s_p[threadIdx.x], s_p[threadIdx.x + stride]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const Partial p = s_p[0];
+    HeadOut* o = a.out;
+    o->argmax[0] = p.idx;
+    o->zmax[0] = p.m;
+    o->lse[0] = p.m + logf(p.s);
+    o->pmax = 1.f / p.s;
+    o->gather[0] = __ldcg(&o->gather[0]);
+    policy_tail(a, o);
+  }
+}
+
+// ---------------------------------------------------------------------------------
 // Decode attention, compact version of the block attention above for the decoder passes
 // (modes 0 and 1 only).  Keys and values of the block's split are staged in shared memory
 // (cross-attention: before the dependency wait), scores are taken one (row, key) pair per

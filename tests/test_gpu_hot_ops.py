@@ -123,3 +123,29 @@ def test_sliced_head_matches_numpy_over_the_whole_vocabulary(M, V, K):
         assert abs(float(mx[m]) - zmax) <= 2e-4
         assert abs(float(lse[m]) - (zmax + np.log(np.exp(Z[m] - zmax).sum()))) <= 2e-4
         assert abs(float(ga[m]) - Z[m][tgt[m]]) <= 2e-4
+
+
+@pytest.mark.parametrize("V,K", [(32128, 512), (32128, 1024), (250112, 512), (250112, 1024), (1001, 264), (40, 64), (5000, 256)])
+def test_streaming_head_matches_numpy_over_the_whole_vocabulary(V, K):
+    """The single-row streaming head: all V logits (debug dump), arg-max, max, log-sum-exp and gathered logit against
+    fp64; vocabularies that do not fill the grid or the last batch of a warp included."""
+    import torch
+    from paper_2302_07863_b200.binding import op_lm_head_stream
+    rng = np.random.default_rng(V + K)
+    W, Wd = _bf16(torch, rng, (V, K), 0.05)
+    X = rng.standard_normal((1, K)).astype(np.float32)
+    g = (1 + 0.1 * rng.standard_normal(K)).astype(np.float32)
+    tgt = rng.integers(0, V, 1).astype(np.int32)
+    scale = 9.0
+    Z = scale * (rms_norm(X.astype(np.float64), g.astype(np.float64), 1e-6) @ W.T)
+    am, mx, lse, ga, lg = op_lm_head_stream(Wd, torch.from_numpy(X).cuda(), torch.from_numpy(g).cuda(), 1e-6, scale,
+                                            torch.from_numpy(tgt).cuda(), V, K, want_logits=True)
+    torch.cuda.synchronize()
+    assert np.max(np.abs(lg.cpu().numpy() - Z)) <= 2e-4          # every logit: a skipped row or batch would show here
+    srt = np.sort(Z[0])
+    if srt[-1] - srt[-2] > 1e-3:
+        assert int(am[0]) == int(np.argmax(Z[0]))
+    zmax = Z[0].max()
+    assert abs(float(mx[0]) - zmax) <= 2e-4
+    assert abs(float(lse[0]) - (zmax + np.log(np.exp(Z[0] - zmax).sum()))) <= 2e-4
+    assert abs(float(ga[0]) - Z[0][tgt[0]]) <= 2e-4

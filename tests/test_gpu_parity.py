@@ -344,7 +344,7 @@ ALT_PATHS = [dict(fused=0, block_simt=1), dict(host_loop=1), dict(pdl=0), dict(u
              dict(ffn_parts=2), dict(fused=0, slice_mode=0), dict(fused=0, slice_mode=2, slice_min_kb=0),
              dict(fused=0, slice_mma_min=5), dict(fused=0, unit_attn=0), dict(fused=0, slice_head=0), dict(slice_head=1),
              dict(slice_head=2, slice_head_min_mb=0), dict(enc_gemm=0), dict(enc_parallel=0), dict(enc_attn_mma=0),
-             dict(fused=0, host_loop=1), dict(attn_all_keys=0), dict(attn_all_keys=16), dict(graph_switch=0), dict(enc_split_k=0), dict(fused=2)]
+             dict(fused=0, host_loop=1), dict(attn_all_keys=0), dict(attn_all_keys=16), dict(graph_switch=0), dict(enc_split_k=0), dict(fused=2), dict(head_stream=0), dict(head_stream=1)]
 
 
 @pytest.mark.parametrize("tuning", ALT_PATHS, ids=lambda t: ",".join(f"{k}={v}" for k, v in t.items()))
@@ -354,7 +354,8 @@ def test_alternative_paths_match_golden(torch_cuda, name, tuning):
     launches, SIMT block GEMV, host-driven loop, plain launches, no tcgen05 kernels, row-slice kernel off / also for small
     matrices, SIMT items up to 4 rows, earlier attention kernel, earlier block head, tensor-core head for single rows,
     encoder on the 16-row kernel / on one stream / SIMT attention, fused attention with the keys always split over the
-    cluster / attended by every block only up to 16 keys, one IF node per kind of large pass instead of the SWITCH node, encoder GEMMs without the split over K, blocks of 9 to 16 rows on the one-kernel-per-operation path) give the same tokens and trace as the stored oracle run."""
+    cluster / attended by every block only up to 16 keys, one IF node per kind of large pass instead of the SWITCH node, encoder GEMMs without the split over K, blocks of 9 to 16 rows on the one-kernel-per-operation path, single-row heads on the register-resident / tensor-core
+    kernels instead of the streaming one) give the same tokens and trace as the stored oracle run."""
     from paper_2302_07863_b200 import MODE_BILD
     from paper_2302_07863_b200.synthetic import make_context
     g = golden(name)
