@@ -1078,7 +1078,7 @@ int decoder_pass(bild_ctx* c, int which, int MBv, float* logits_dbg, unsigned lo
   const size_t sh_smem = slice_head_smem_bytes(d, head_tr);
   // single-row passes: only heads of 32 MB and more (smaller ones stay on the GEMV head)
   const bool big_head = (size_t)mc.vocab * d * 2 >= c->slice_head_min_bytes;
-  if (c->head_stream >= (big_head ? 1 : 2) && c->sms > 0 && 2 * c->sms <= MAX_GRID_SM * 2 && head_stream_fits(dt, MB, h)) {
+  if (c->head_stream >= (big_head ? 1 : 2) && c->sms > 0 && (size_t)2 * c->sms <= head_partial_count(mc.vocab) && head_stream_fits(dt, MB, h)) {
     CUDA_TRY(c, launch_head_stream(c, h, c->sms));   // single row: the vocabulary streamed through registers
     return draw_token();
   }
