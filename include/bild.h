@@ -288,10 +288,11 @@ int bild_generate_sampled(bild_ctx *ctx, int mode, float alpha_fb, float alpha_r
                           bild_trace_rec *trace_out /*HOST or NULL*/, int trace_cap, int *n_trace,
                           bild_stats *stats /*HOST or NULL*/);
 
-/* 1 if the tcgen05 tensor-core kernel is in use for this context (bf16 weights, d_model / inner /
- * d_ff multiples of 64): it runs the encoder's linear layers, and those of the large model's
- * block pass (k > 1) when the row-slice kernel is switched off (BILD_SLICE=0); 0 if everything
- * runs on the SIMT kernels. */
+/* 1 if the tcgen05 kernels are in use for this context (bf16 weights, d_model / inner / d_ff
+ * multiples of 64): they run the ENCODER's linear layers (the set-up step) and, with
+ * bild_tuning.fused = 0 and slice_mode = 0, the linear layers of block passes.  The decoder passes of
+ * the product path multiply on mma.sync tiles (blocks of 2 rows and more) or plain multiply-adds
+ * (single rows): they are latency-bound, see the per-pass tables.  0: no tcgen05 kernel runs. */
 int bild_uses_tensor_cores(const bild_ctx *ctx);
 
 /* Number of kernel launches this context has enqueued since it was created. */
