@@ -7,6 +7,8 @@
 //   * the key tile is staged as [key][d] (the "col" operand of Q K^T), the value tile transposed as
 //     [d][key] (the "col" operand of P V), both as head and remainder, rows padded against bank
 //     conflicts;
+//   * the next tile's keys and values are on their way (asynchronous 16-byte copies into a raw fp32 area) while the
+//     current tile is multiplied; staging then converts from shared memory;
 //   * the score fragment of a warp (16 rows x 64 keys) stays in registers, is turned into
 //     probabilities and re-used as the left operand of P V (accumulator fragment of two 8-key
 //     tiles = operand fragment of one 16-key step).
@@ -20,6 +22,7 @@ constexpr int EA_ROWS = 64;    // query rows per block
 constexpr int EA_KEYS = 64;    // keys per tile
 constexpr int EA_D = 64;       // d_kv
 constexpr int EA_PAD = 8;      // bf16 elements of padding per staged row
+constexpr int EA_RVS = EA_D + 4;   // row stride (floats) of the raw value tile: two keys 2 rows apart fall into different banks
 
 __device__ __forceinline__ uint32_t ea_pack(float a, float b) {
   __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
@@ -36,7 +39,7 @@ __device__ __forceinline__ void ea_mma(float (&c)[4], uint32_t a0, uint32_t a1, 
 }
 
 inline size_t enc_attn_smem_bytes(int max_keys) {
-  return (size_t)4 * EA_KEYS * (EA_D + EA_PAD) * 2 + (size_t)(max_keys + EA_ROWS) * 4;
+  return (size_t)4 * EA_KEYS * (EA_D + EA_PAD) * 2 + (size_t)EA_KEYS * (EA_D + EA_RVS) * 4 + (size_t)((max_keys + EA_ROWS + 3) & ~3) * 4;
 }
 
 // q [E][ldq], kc / vc [H][cap][64], out [E][ldo]; bias [H][bias_ld] indexed by bias_off + key - query
@@ -49,7 +52,9 @@ __global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_
   __nv_bfloat16* sKl = sKh + EA_KEYS * ST;
   __nv_bfloat16* sVh = sKl + EA_KEYS * ST;                          // [d][key]
   __nv_bfloat16* sVl = sVh + EA_D * ST;
-  float* sBias = reinterpret_cast<float*>(sVl + EA_D * ST);        // [E + 63]: entry (key - query + r0 + 63)
+  float* sRawK = reinterpret_cast<float*>(sVl + EA_D * ST);        // [key][64] fp32 as it lies in the cache
+  float* sRawV = sRawK + EA_KEYS * EA_D;                            // [key][EA_RVS]
+  float* sBias = sRawV + EA_KEYS * EA_RVS;                          // [E + 63]: entry (key - query + r0 + 63)
   const int h = blockIdx.x, r0 = blockIdx.y * EA_ROWS;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   pdl_launch_dependents();
@@ -86,14 +91,24 @@ __global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_
   const float* Kg = a.kc + (size_t)h * a.cap * EA_D;
   const float* Vg = a.vc + (size_t)h * a.cap * EA_D;
   const int qa_pos = r0 + warp * 16 + g, qb_pos = qa_pos + 8;
-#pragma unroll 1
-  for (int k0 = 0; k0 < E; k0 += EA_KEYS) {
-    __syncthreads();   // the previous tile is no longer read
-    // stage the tile.  Keys: thread -> (key, 4 channels), rows written 8 bytes at a time.
+  auto fetch = [&](int k0) {   // the raw tile: 16-byte asynchronous copies, keys past the end repeat the last one
     for (int idx = tid; idx < EA_KEYS * (EA_D / 4); idx += EA_THREADS) {
       const int key = idx >> 4, c4 = (idx & 15) << 2;
       const int kg = min(k0 + key, E - 1);
-      const float4 kv = __ldcg(reinterpret_cast<const float4*>(Kg + (size_t)kg * EA_D + c4));
+      cp_async16(sRawK + key * EA_D + c4, Kg + (size_t)kg * EA_D + c4);
+      cp_async16(sRawV + key * EA_RVS + c4, Vg + (size_t)kg * EA_D + c4);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  fetch(0);
+#pragma unroll 1
+  for (int k0 = 0; k0 < E; k0 += EA_KEYS) {
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();   // the raw tile has arrived for everybody; the previous tile is no longer read
+    // stage the tile.  Keys: thread -> (key, 4 channels), rows written 8 bytes at a time.
+    for (int idx = tid; idx < EA_KEYS * (EA_D / 4); idx += EA_THREADS) {
+      const int key = idx >> 4, c4 = (idx & 15) << 2;
+      const float4 kv = *reinterpret_cast<const float4*>(sRawK + key * EA_D + c4);
       uint32_t h0, l0, h1, l1;
       ea_split(kv.x, kv.y, h0, l0);
       ea_split(kv.z, kv.w, h1, l1);
@@ -104,9 +119,8 @@ __global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_
     // warp writes 32 consecutive words of one transposed row
     for (int idx = tid; idx < (EA_KEYS / 2) * (EA_D / 4); idx += EA_THREADS) {
       const int kp = idx & 31, c4 = (idx >> 5) << 2;
-      const int ka = min(k0 + 2 * kp, E - 1), kb = min(k0 + 2 * kp + 1, E - 1);
-      const float4 va = *reinterpret_cast<const float4*>(Vg + (size_t)ka * EA_D + c4);
-      const float4 vb = *reinterpret_cast<const float4*>(Vg + (size_t)kb * EA_D + c4);
+      const float4 va = *reinterpret_cast<const float4*>(sRawV + (2 * kp) * EA_RVS + c4);
+      const float4 vb = *reinterpret_cast<const float4*>(sRawV + (2 * kp + 1) * EA_RVS + c4);
       const float ea[4] = {va.x, va.y, va.z, va.w}, eb[4] = {vb.x, vb.y, vb.z, vb.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -117,6 +131,7 @@ __global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_
       }
     }
     __syncthreads();
+    if (k0 + EA_KEYS < E) fetch(k0 + EA_KEYS);   // (the raw area is free again: everybody has converted its share)
     // scores of 16 rows x 64 keys
     float s[8][4];
 #pragma unroll
