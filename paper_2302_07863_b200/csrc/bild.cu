@@ -166,6 +166,9 @@ struct bild_ctx {
   int64_t per_pass[2] = {0, 0};      // kernel launches in one small / one large pass of the graphs
   int64_t per_pass_large1 = 0, per_pass_large8 = 0;
   int64_t* cnt = &launches;         // where launches are counted (redirected while capturing)
+  bool enc_kv_streams = true;         // cross K/V projections of the decoder layers dealt to three streams
+  cudaStream_t kv_stream[2] = {nullptr, nullptr};
+  cudaEvent_t kv_fork = nullptr, kv_join[2] = {nullptr, nullptr};
   cudaStream_t side2 = nullptr;       // second chunk of a block of 9 to 16 rows (fused sub-layer kernels)
   std::vector<cudaEvent_t> chunk_ev;  // per layer: first chunk's self-attention done; then fork and join
   cudaStream_t cap_stream = nullptr;  // capture only (the legacy default stream cannot capture); nothing runs on it
@@ -1134,16 +1137,39 @@ int encoder_pass(bild_ctx* c, int which) {
     dn.M = E; dn.W0 = w.wfo; dn.X = B.eu; dn.ldx = F; dn.N = d; dn.K = F; dn.epi = EPI_RESID; dn.Y = B.ex; dn.ldy = d;
     CUDA_TRY(c, launch_enc_linear(c, m, dn, rb, l, TM_EFO, !m.enc_gemm, 1));
   }
-  // encoder memory = final norm of ex (fused into the projections); cross K/V per decoder layer
-  for (int l = 0; l < mc.n_layers; ++l) {
+  // encoder memory = final norm of ex (fused into the projections); cross K/V per decoder layer.  The projections of the
+  // layers are independent of one another (each covers a fraction of the SMs): after the first, which also writes the
+  // normalised encoder output, they are dealt to this stream and two more.
+  cudaStream_t base = c->stream;
+  bool spread = c->enc_kv_streams && m.enc_gemm && mc.n_layers >= 4;
+  if (spread && !c->kv_stream[0]) {
+    bool ok = cudaEventCreateWithFlags(&c->kv_fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+      ok = cudaStreamCreateWithFlags(&c->kv_stream[i], cudaStreamNonBlocking) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->kv_join[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); spread = c->enc_kv_streams = false; }
+  }
+  int rc = BILD_OK;
+  for (int l = 0; l < mc.n_layers && rc == BILD_OK; ++l) {
     const size_t kvoff = (size_t)l * H * dkv;
     LinArgs a{};
     a.M = E; a.eps = mc.ln_eps; a.W0 = m.dec[l].wckv; a.X = B.ex; a.ldx = d; a.gain = (const float*)m.w.enc_final_ln;
     a.N = 2 * I; a.K = d; a.epi = EPI_HEADS; a.inner = I; a.dkv = dkv; a.first_part = 1;
     a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.pos0_host = 0;
-    CUDA_TRY(c, launch_enc_linear(c, m, a, rb, l, TM_CKV, l == 0, 0));   // the normalised encoder output is split once
+    if (spread && l > 0 && l % 3) c->stream = c->kv_stream[l % 3 - 1];
+    const cudaError_t e = launch_enc_linear(c, m, a, rb, l, TM_CKV, l == 0, 0);   // the normalised encoder output is split once
+    c->stream = base;
+    if (e != cudaSuccess) rc = fail(c, BILD_ERR_CUDA, std::string("cross K/V projection: ") + cudaGetErrorString(e));
+    if (spread && l == 0 && rc == BILD_OK) {   // the other streams start once the split rows exist
+      if (cudaEventRecord(c->kv_fork, base) != cudaSuccess || cudaStreamWaitEvent(c->kv_stream[0], c->kv_fork, 0) != cudaSuccess ||
+          cudaStreamWaitEvent(c->kv_stream[1], c->kv_fork, 0) != cudaSuccess) rc = fail(c, BILD_ERR_CUDA, "cross K/V projection: fork");
+    }
   }
-  return BILD_OK;
+  if (spread)   // joined in any case, so that nothing is left running beside the caller's stream
+    for (int i = 0; i < 2; ++i)
+      if (cudaEventRecord(c->kv_join[i], c->kv_stream[i]) != cudaSuccess || cudaStreamWaitEvent(base, c->kv_join[i], 0) != cudaSuccess)
+        rc = rc ? rc : fail(c, BILD_ERR_CUDA, "cross K/V projection: join");
+  return rc;
 }
 
 int build_bias_tables(bild_ctx* c) {
@@ -1421,6 +1447,7 @@ int bild_create_tuned(const bild_config* cfg, const bild_weights* small_w, const
     c->use_enc_gemm = t.enc_gemm != 0;
     c->enc_attn_mma = t.enc_attn_mma != 0;
     c->enc_parallel = t.enc_parallel != 0;
+    c->enc_kv_streams = t.enc_parallel != 0;   // (one switch: everything of the set-up step on one stream, or not)
     c->spin_limit = t.spin_limit > 0 ? (unsigned)t.spin_limit : SPIN_LIMIT;
     c->debug_skip_copies = t.debug_skip_copies != 0;
     c->attn_all_keys = std::min(128, std::max(0, t.attn_all_keys));
@@ -1488,6 +1515,11 @@ void bild_destroy(bild_ctx* c) {
   drop_graphs(c);
   if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
   if (c->side2) { cudaStreamSynchronize(c->side2); cudaStreamDestroy(c->side2); }
+  for (int i = 0; i < 2; ++i) {
+    if (c->kv_stream[i]) { cudaStreamSynchronize(c->kv_stream[i]); cudaStreamDestroy(c->kv_stream[i]); }
+    if (c->kv_join[i]) cudaEventDestroy(c->kv_join[i]);
+  }
+  if (c->kv_fork) cudaEventDestroy(c->kv_fork);
   for (cudaEvent_t e : c->chunk_ev) cudaEventDestroy(e);
   if (c->enc_stream) { cudaStreamSynchronize(c->enc_stream); cudaStreamDestroy(c->enc_stream); }
   if (c->enc_fork) cudaEventDestroy(c->enc_fork);
