@@ -188,7 +188,8 @@ typedef struct {
   int32_t umma;              /* 1: tcgen05 kernels (encoder linears; unfused block linears when slice_mode = 0) */
   int32_t enc_gemm;          /* 1: encoder linears as 128-token tcgen05 GEMM tiles */
   int32_t enc_attn_mma;      /* 1: encoder self-attention on mma.sync tiles */
-  int32_t enc_parallel;      /* 1: the two encoders run side by side on two streams */
+  int32_t enc_parallel;      /* 1: the two encoders run side by side on two streams, and the cross K/V projections of the
+                              * decoder layers on three; 0: the whole set-up step on the context's stream */
   int32_t spin_limit;        /* polls before a bounded device-side wait gives up with BILD_ERR_TIMEOUT (0: 2^20) */
   int32_t debug_skip_copies; /* 1: the fused attention kernel announces its weight copies but does not issue them, so
                               * that its bounded wait runs out (test of the time-out path; never set in production) */
