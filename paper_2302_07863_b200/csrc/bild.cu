@@ -748,7 +748,7 @@ int fused_layer(bild_ctx* c, Model& m, int MB, int l, const CallDesc* desc, int 
   const size_t kvoff = (size_t)l * H * dkv;
   AttnSubArgs a{};
   a.desc = desc; a.eps = mc.ln_eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
-  a.mb = MB; a.err = &c->st->err; a.x_rows = MAXB - row0;
+  a.mb = MB; a.err = &c->st->err;
   a.spin = c->spin_limit; a.skip_copies = c->debug_skip_copies ? 1 : 0;
   a.n_keys_dev = c->enc_len_dev;
   // S1-S3 / L1-L3
@@ -769,7 +769,6 @@ int fused_layer(bild_ctx* c, Model& m, int MB, int l, const CallDesc* desc, int 
   CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
   // S7-S8 / L7-L8
   FfnSubArgs f{};
-  f.x_rows = MAXB - row0;
   f.desc = desc; f.eps = mc.ln_eps; f.d = d; f.F = Fd; f.gated = gated ? 1 : 0; f.mb = MB; f.spin = c->spin_limit;
   f.err = &c->st->err; f.x_in = xc; f.x_out = x; f.gain = (const float*)w.ln3;
   f.Wi0 = (const __nv_bfloat16*)w.wi0; f.Wi1 = (const __nv_bfloat16*)w.wi1;
@@ -1866,7 +1865,7 @@ int bild_op_ffn_sublayer(const void* Wi0, const void* Wi1, const void* Wfo, cons
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max) != cudaSuccess) return BILD_ERR_CUDA;
   FfnSubArgs f{};
   f.desc = o.desc; f.eps = eps; f.d = d; f.F = F; f.gated = gated ? 1 : 0; f.mb = MB; f.spin = SPIN_LIMIT; f.err = o.err;
-  f.x_in = x_in; f.x_rows = M; f.x_out = x_out; f.gain = gain; f.Wi0 = (const __nv_bfloat16*)Wi0; f.Wi1 = (const __nv_bfloat16*)Wi1; f.Wfo1 = wfo_one; f.Wfo8 = wfo_blk;
+  f.x_in = x_in; f.x_out = x_out; f.gain = gain; f.Wi0 = (const __nv_bfloat16*)Wi0; f.Wi1 = (const __nv_bfloat16*)Wi1; f.Wfo1 = wfo_one; f.Wfo8 = wfo_blk;
   f.nparts = np; f.L = ffn_sub_layout(d, F, gated, sms * np, sms, MB);
   for (int p = 0; p < np; ++p) {
     f.part = p; f.seed = p == 0 ? 1 : 0; f.x_zero = p == 0 ? o.zero : nullptr;
@@ -1909,7 +1908,7 @@ int bild_op_attn_sublayer(int self, const void* Wp, const void* Wo, const float*
   AttnSubArgs a{};
   a.desc = o.desc; a.eps = eps; a.d = d; a.I = I; a.H = H; a.dkv = dkv; a.dkv_shift = ilog2(dkv); a.C = C; a.c_shift = ilog2(C);
   a.kc_keys = kc_keys; a.bias_len = bias_len; a.red_keys = pl.red_keys; a.mb = MB; a.err = o.err; a.spin = SPIN_LIMIT; a.skip_copies = 0;
-  a.n_keys_dev = o.nkeys; a.x_in = x_in; a.x_rows = M; a.x_out = x_out; a.x_zero = o.zero; a.gain = gain;
+  a.n_keys_dev = o.nkeys; a.x_in = x_in; a.x_out = x_out; a.x_zero = o.zero; a.gain = gain;
   a.Wp = (const __nv_bfloat16*)Wp; a.Wo = (const __nv_bfloat16*)Wo; a.kc = kc; a.vc = vc; a.cap = cap;
   a.bias = bias_by_dist; a.bias_ld = cap; a.self = self ? 1 : 0;
   a.L = attn_sub_layout(d, dkv, P, C, MB, kc_keys, bias_len);

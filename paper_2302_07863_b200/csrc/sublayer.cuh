@@ -109,8 +109,8 @@ __device__ __forceinline__ float sub_total(const float* psum, int row, int m, in
 }
 
 // Token rows, after the dependency wait (d <= 1024: one 128-bit load per thread and row).  The loads are issued first
-// thing after the wait, for all rows the variant can take (which rows count is known only once the call descriptor
-// has been read, a round trip to the L2 of its own); sub_rows_finish then writes x * gain into Xs and 1 / rms into
+// thing after the wait, for the rows of the pass (the row count is read before the wait); sub_rows_finish then writes
+// x * gain into Xs and 1 / rms into
 // sh->inv (returned for the single row of ONE).  The raw values of the columns [seed0, seed1) (multiples of 4) also go
 // to sSeed[m][column - seed0]: the residual term the block adds.
 // Block variant: the normalised token rows wait in shared memory as bf16 heads [SUB_MB][d / 2 + 4] (two values a word)
@@ -154,7 +154,7 @@ struct SubRows { float4 v[ONE ? 1 : SUB_MB]; };
 
 template <bool ONE>
 __device__ __forceinline__ void sub_rows_issue(const float* __restrict__ x_in, int rows, int d, int tid, SubRows<ONE>& rw) {
-  if (tid * 4 < d) {   // rows: how many rows of x_in exist (a launch parameter, known without a load)
+  if (tid * 4 < d) {   // rows: the rows of the pass
 #pragma unroll
     for (int i = 0; i < (ONE ? 1 : SUB_MB); ++i)
       if (i < rows) rw.v[i] = __ldcg(reinterpret_cast<const float4*>(x_in + (size_t)i * d) + tid);
@@ -223,8 +223,7 @@ struct AttnSubLayout { int wq, xs, kv, kv_late, qkv, psum, probs, bias, seed, sa
 
 struct AttnSubArgs {
   const CallDesc* desc;
-  const float* x_in;    // [x_rows][d] residual stream (complete)
-  int x_rows;           // rows x_in has (at least the rows of the pass)
+  const float* x_in;    // [rows of the pass][d] residual stream (complete)
   float* x_out;         // [MAXB][d] zero on entry; receives x_in + the sub-layer's output
   float* x_zero;        // [MAXB][d] cleared for the kernel after this one
   const float* gain;
@@ -394,13 +393,11 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
     j0 = red ? 0 : (r * n_keys) >> a.c_shift; j1 = red ? n_keys : ((r + 1) * n_keys) >> a.c_shift;
     stage_cached(j0, min(j1, j0 + a.kc_keys));
   }
-  SUB_STAMP();            // P2: loads issued, cross keys requested
-  sub_cluster_arrive_relaxed();   // (0) this block is up: its shared memory may be written by the cluster
-  SUB_STAMP();            // 0: prologue
-  pdl_wait();
-  SUB_STAMP();            // 1: dependency wait
-  SubRows<ONE> rw;
-  sub_rows_issue<ONE>(a.x_in, a.x_rows, d, tid, rw);
+  // The call descriptor (row count, cache position) is written by kernels that have finished before the first kernel of a
+  // pass starts -- the head of the pass before, or a set-up kernel in front of the embedding -- never by the kernel in
+  // front of this one: it is read before the dependency wait, and with it the cached keys and values (rows below the
+  // cache position, written by earlier passes; a second chunk of a block is launched only when the first chunk's rows
+  // of this layer are complete) and the bias by distance.
   const int k = ONE ? 1 : min(a.desc->k, a.mb), pos0 = a.desc->pos0;
   if (a.self) {
     n_keys = min(pos0 + k, a.cap);
@@ -411,8 +408,15 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
   // relative-position bias of the distances this rank meets
   const int dist_lo = max(0, pos0 - (j1 - 1));
   const int bias_cnt = a.self ? min(pos0 + k - j0 - dist_lo, a.bias_len) : 0;
-  float bias0 = 0.f;   // requested now, stored once the token rows are requested too
-  if (tid < bias_cnt) bias0 = __ldg(a.bias + (size_t)h * a.bias_ld + dist_lo + tid);
+#pragma unroll 1
+  for (int i = tid; i < bias_cnt; i += SUB_THREADS) sBias[i] = __ldg(a.bias + (size_t)h * a.bias_ld + dist_lo + i);
+  SUB_STAMP();            // P2: loads issued, keys requested
+  sub_cluster_arrive_relaxed();   // (0) this block is up: its shared memory may be written by the cluster
+  SUB_STAMP();            // 0: prologue
+  pdl_wait();
+  SUB_STAMP();            // 1: dependency wait
+  SubRows<ONE> rw;
+  sub_rows_issue<ONE>(a.x_in, k, d, tid, rw);
   {   // clear the buffer the next kernel accumulates into
     const int n4 = k * (d >> 2);
 #pragma unroll 1
@@ -420,9 +424,6 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
       reinterpret_cast<float4*>(a.x_zero)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
   const float inv1 = sub_rows_finish<ONE>(rw, k, d, g4, a.eps, Xs, xst, sh, sSeed, h == 0 ? o0 : 0, h == 0 ? o0 + no : 0, tid, lane, warp);
-  if (tid < bias_cnt) sBias[tid] = bias0;
-#pragma unroll 1
-  for (int i = tid + SUB_THREADS; i < bias_cnt; i += SUB_THREADS) sBias[i] = __ldg(a.bias + (size_t)h * a.bias_ld + dist_lo + i);
   SUB_STAMP();            // 2: token rows + norm
   sub_wait(sh, a.err, &sh->wbar, 0, a.spin);
   SUB_STAMP();            // 3: wait for the weights
@@ -805,7 +806,6 @@ struct FfnSubLayout { int wi, xs, psum, u, seed, sh, total; };
 struct FfnSubArgs {
   const CallDesc* desc;
   const float* x_in;
-  int x_rows;                // rows x_in has (at least the rows of the pass)
   float* x_out;
   float* x_zero;             // nullptr: nothing to clear (second part of a split launch)
   const float* gain;
@@ -917,12 +917,12 @@ __global__ void __launch_bounds__(SUB_THREADS) ffn_sub_kernel(const FfnSubArgs a
   }
   float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f);
   if (tid * 4 < d) g4 = __ldg(reinterpret_cast<const float4*>(a.gain) + tid);
+  const int k = ONE ? 1 : min(a.desc->k, a.mb);   // (written before the pass began: see the attention kernel)
   SUB_STAMP();            // 0: prologue
   pdl_wait();
   SUB_STAMP();            // 1: dependency wait
   SubRows<ONE> rw;
-  sub_rows_issue<ONE>(a.x_in, a.x_rows, d, tid, rw);
-  const int k = ONE ? 1 : min(a.desc->k, a.mb);
+  sub_rows_issue<ONE>(a.x_in, k, d, tid, rw);
   if (a.x_zero) {
     const int n4 = k * d4;
 #pragma unroll 1
