@@ -166,6 +166,7 @@ struct bild_ctx {
   int64_t per_pass[2] = {0, 0};      // kernel launches in one small / one large pass of the graphs
   int64_t per_pass_large1 = 0, per_pass_large8 = 0;
   int64_t* cnt = &launches;         // where launches are counted (redirected while capturing)
+  bool fused_embed = true;            // the first fused sub-layer kernel of a pass gathers the embedding rows (no embedding kernel)
   bool enc_kv_streams = true;         // cross K/V projections of the decoder layers dealt to three streams
   cudaStream_t kv_stream[2] = {nullptr, nullptr};
   cudaEvent_t kv_fork = nullptr, kv_join[2] = {nullptr, nullptr};
@@ -676,6 +677,7 @@ int setup_fused(bild_ctx* c, Model& m) {
     if (!aligned(w.wqkv) || !aligned(w.wo) || !aligned(w.wcq) || !aligned(w.wco) || !aligned(w.wi0) || !aligned(w.wfo) ||
         (gated && !aligned(w.wi1)) || !aligned(w.ln1) || !aligned(w.ln2) || !aligned(w.ln3)) return BILD_OK;
   }
+  if (!aligned(m.w.emb)) return BILD_OK;   // (the first sub-layer kernel gathers the embedding rows, 8 bytes per load)
   int smem_max = 0, dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
     cudaGetLastError();
@@ -751,7 +753,10 @@ int fused_layer(bild_ctx* c, Model& m, int MB, int l, const CallDesc* desc, int 
   a.mb = MB; a.err = &c->st->err;
   a.spin = c->spin_limit; a.skip_copies = c->debug_skip_copies ? 1 : 0;
   a.n_keys_dev = c->enc_len_dev;
-  // S1-S3 / L1-L3
+  // S1-S3 / L1-L3 (layer 0: with S0 / L0, the rows come from the embedding table)
+  if (l == 0 && c->fused_embed) {
+    a.emb = (const __nv_bfloat16*)m.w.emb; a.tokens = m.desc->tokens + row0; a.vocab = mc.vocab;
+  }
   a.x_in = x; a.x_out = xb; a.x_zero = xc; a.gain = (const float*)w.ln1;
   a.Wp = (const __nv_bfloat16*)w.wqkv; a.Wo = (const __nv_bfloat16*)w.wo;
   a.kc = m.selfK + kvoff * cap; a.vc = m.selfV + kvoff * cap; a.cap = cap; a.bias = m.dec_bias; a.bias_ld = cap; a.self = 1;
@@ -761,6 +766,7 @@ int fused_layer(bild_ctx* c, Model& m, int MB, int l, const CallDesc* desc, int 
   int rc = after_self();
   if (rc) return rc;
   // S4-S6 / L4-L6
+  a.emb = nullptr;
   a.x_in = xb; a.x_out = xc; a.x_zero = x; a.gain = (const float*)w.ln2;
   a.Wp = (const __nv_bfloat16*)w.wcq; a.Wo = (const __nv_bfloat16*)w.wco;
   a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.bias = nullptr; a.bias_ld = 0; a.self = 0;
@@ -1000,7 +1006,10 @@ int decoder_pass(bild_ctx* c, int which, int MBv, float* logits_dbg, unsigned lo
   // blocks of 9 to 16 rows: two chunks of the 8-row kernels side by side (the caller guarantees more than 8 rows)
   const bool chunked = m.fused && which == 1 && MBv == MAXB && c->fused_on >= 3;
   const bool fused = chunked || (m.fused && (MBv == 1 || (MBv == SUB_MB && c->fused_on >= 2)));
-  CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x, fused ? m.xb : nullptr));
+  // (fused sub-layer kernels: the first one gathers the embedding rows itself; the buffer it adds into is clear, every
+  // pass leaves it so and a generation starts with it cleared)
+  if (!(fused && c->fused_embed))
+    CUDA_TRY(c, launch_embed(c, m.w.emb, m.desc->tokens, &m.desc->k, 0, MB, d, mc.vocab, m.x, fused ? m.xb : nullptr));
   if (fused) {
     int rc = chunked ? fused_layers_two_chunks(c, m) : fused_layers(c, m, MBv);
     if (rc) return rc;
@@ -1376,6 +1385,10 @@ int reset_state(bild_ctx* c, int mode, float afb, float arb, int max_len) {
                                              c->cfg.eos_id, c->cfg.start_id, c->trace_cap, c->top_p);
   (*c->cnt)++;
   CUDA_TRY(c, cudaGetLastError());
+  // the buffer the first fused sub-layer kernel of a pass adds into: every pass leaves it clear; cleared here as well, so
+  // that a pass that ended in an error cannot leak into the next generation
+  for (int i = 0; i < 2; ++i)
+    if (c->m[i].fused && c->m[i].xb) CUDA_TRY(c, cudaMemsetAsync(c->m[i].xb, 0, (size_t)MAXB * c->m[i].c.d_model * sizeof(float), c->stream));
   return BILD_OK;
 }
 

@@ -161,6 +161,23 @@ __device__ __forceinline__ void sub_rows_issue(const float* __restrict__ x_in, i
   }
 }
 
+// The first sub-layer of a pass takes its rows from the embedding table (S0 / L0): row i = E[token_i], bf16.
+template <bool ONE>
+__device__ __forceinline__ void sub_rows_embed(const __nv_bfloat16* __restrict__ E, const int* __restrict__ tokens, int vocab, int rows,
+                                               int d, int tid, SubRows<ONE>& rw) {
+  if (tid * 4 < d) {
+#pragma unroll
+    for (int i = 0; i < (ONE ? 1 : SUB_MB); ++i)
+      if (i < rows) {
+        int t = tokens[i];
+        t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
+        const uint2 w = __ldg(reinterpret_cast<const uint2*>(E + (size_t)t * d) + tid);
+        rw.v[i] = make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u), __uint_as_float(w.y << 16),
+                              __uint_as_float(w.y & 0xffff0000u));
+      }
+  }
+}
+
 template <bool ONE>
 __device__ __forceinline__ float sub_rows_finish(const SubRows<ONE>& rw, int k, int d, float4 g, float eps, float* Xs, int xst,
                                                  SubShared* sh, float* sSeed, int seed0, int seed1, int tid, int lane, int warp) {
@@ -224,6 +241,9 @@ struct AttnSubLayout { int wq, xs, kv, kv_late, qkv, psum, probs, bias, seed, sa
 struct AttnSubArgs {
   const CallDesc* desc;
   const float* x_in;    // [rows of the pass][d] residual stream (complete)
+  const __nv_bfloat16* emb;  // not null: the first sub-layer of a pass, its rows are E[tokens[i]] instead of x_in (S0 / L0)
+  const int* tokens;
+  int vocab;
   float* x_out;         // [MAXB][d] zero on entry; receives x_in + the sub-layer's output
   float* x_zero;        // [MAXB][d] cleared for the kernel after this one
   const float* gain;
@@ -410,13 +430,14 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
   const int bias_cnt = a.self ? min(pos0 + k - j0 - dist_lo, a.bias_len) : 0;
 #pragma unroll 1
   for (int i = tid; i < bias_cnt; i += SUB_THREADS) sBias[i] = __ldg(a.bias + (size_t)h * a.bias_ld + dist_lo + i);
+  SubRows<ONE> rw;
+  if (a.emb) sub_rows_embed<ONE>(a.emb, a.tokens, a.vocab, k, d, tid, rw);   // (tokens: part of the descriptor; the table: weights)
   SUB_STAMP();            // P2: loads issued, keys requested
   sub_cluster_arrive_relaxed();   // (0) this block is up: its shared memory may be written by the cluster
   SUB_STAMP();            // 0: prologue
   pdl_wait();
   SUB_STAMP();            // 1: dependency wait
-  SubRows<ONE> rw;
-  sub_rows_issue<ONE>(a.x_in, k, d, tid, rw);
+  if (!a.emb) sub_rows_issue<ONE>(a.x_in, k, d, tid, rw);
   {   // clear the buffer the next kernel accumulates into
     const int n4 = k * (d >> 2);
 #pragma unroll 1
