@@ -1,12 +1,14 @@
-// Decoder sub-layers as ONE kernel each (bf16 weights, up to MAXB token rows), so that a layer
-// of a decoder pass is three or four dependent kernels instead of eight:
+// Decoder sub-layers as ONE kernel each (bf16 weights, up to 8 token rows a launch), so that a layer
+// of a decoder pass is three dependent kernels instead of eight:
 //   * attn_sub_kernel: x_out = x_in + W_o * Attention(W_q|k|v * rms_norm(x_in))   (steps S1-S3 / L1-L3
 //     for self-attention, S4-S6 / L4-L6 for cross-attention).  A cluster of C blocks owns one head:
 //     rank r multiplies its share of the head's q|k|v rows (weights fetched by bulk copies BEFORE
 //     the dependency wait of the programmatic launch), the cluster exchanges the k x 3 x d_kv results
 //     through distributed shared memory, rank r then attends over its share of the keys, the
 //     per-rank (max, sum, weighted values) records are exchanged the same way, and every rank
-//     multiplies the merged head output with its share of the rows of W_o's column slice;
+//     multiplies the merged head output with its share of the rows of W_o's column slice; while a head has few keys
+//     (they fit one staged chunk) every rank attends over all of them instead and the second exchange falls away;
+//     the first kernel of a pass takes its rows from the embedding table (S0 / L0);
 //   * ffn_sub_kernel: x_out = x_in + W_fo * act(W_i * rms_norm(x_in))   (S7-S8 / L7-L8).  Block b owns a
 //     slice of d_ff (a multiple of 8 rows): the rows of W_i (and of the gate matrix) in shared memory and the
 //     matching columns of W_fo in registers (from a copy laid out in load order), so the hidden activations never
