@@ -203,6 +203,8 @@ typedef struct {
                               * split K over more blocks, partial tiles added with reductions at the L2 */
   int32_t head_stream;       /* single-row bf16 LM heads (rows of at most 1024 columns) on the streaming kernel: 0 off,
                               * 1 heads of slice_head_min_mb and more, 2 all */
+  int32_t enc_attn_groups;   /* encoder self-attention (enc_attn_mma): groups of four warps per block, each visiting every
+                              * n-th tile of 64 keys, partial results merged at the end; 1..3 */
 } bild_tuning;
 void bild_tuning_default(bild_tuning *t /*HOST out*/);
 /* bild_create with explicit switches; tuning == NULL means the defaults. */

@@ -60,7 +60,7 @@ class Tuning(C.Structure):
     """bild_tuning: kernel selection and debugging switches (defaults from bild_tuning_default)."""
     _fields_ = [(n, C.c_int32) for n in ("host_loop", "pdl", "fused", "ffn_parts", "block_simt", "slice_mode", "slice_min_kb",
                                          "slice_mma_min", "slice_head", "slice_head_min_mb", "unit_attn", "umma", "enc_gemm",
-                                         "enc_attn_mma", "enc_parallel", "spin_limit", "debug_skip_copies", "attn_all_keys", "graph_switch", "enc_split_k", "head_stream")]
+                                         "enc_attn_mma", "enc_parallel", "spin_limit", "debug_skip_copies", "attn_all_keys", "graph_switch", "enc_split_k", "head_stream", "enc_attn_groups")]
 
 
 class StepOut(C.Structure):

@@ -188,6 +188,7 @@ struct bild_ctx {
   bool unit_attn = true;             // decoder attention on the 256-thread chunked kernel
   bool uattn_smem_set = false;
   bool enc_attn_mma = true;          // encoder self-attention on the mma.sync kernel (d_kv = 64)
+  int enc_attn_groups = EA_MAX_GROUPS;   // key groups per block of that kernel (1..3)
   int slice_head = 2;                // tensor-core LM head: 0 off, 1 block passes, 2 also single-row passes (large heads)
   bool slice_head_smem_set = false;
   size_t slice_head_min_bytes = (size_t)32 << 20;
@@ -413,12 +414,14 @@ cudaError_t launch_battn(bild_ctx* c, int MB, const BAttnArgs& a0, int row_block
     }
   }
   if (a0.mode == 2 && a0.dkv == EA_D && c->enc_attn_mma) {   // encoder: 64-row tiles on mma.sync
-    const size_t smem = enc_attn_smem_bytes(keys_cap);
+    const int groups = std::min(enc_attn_groups(keys_cap), std::max(1, c->enc_attn_groups));
+    const size_t smem = enc_attn_smem_bytes(keys_cap, groups);
+    auto kern = groups == 1 ? enc_attn_kernel<1> : groups == 2 ? enc_attn_kernel<2> : enc_attn_kernel<3>;
     if (smem > 48 * 1024) {
-      cudaError_t e = cudaFuncSetAttribute(enc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
     }
-    return launch_k(c, enc_attn_kernel, dim3(a0.H, (a0.M + EA_ROWS - 1) / EA_ROWS), dim3(EA_THREADS), smem, a0, oh, ol);
+    return launch_k(c, kern, dim3(a0.H, (a0.M + EA_ROWS - 1) / EA_ROWS), dim3(EA_THREADS * groups), smem, a0, oh, ol);
   }
   if (a0.mode == 2) return launch_battn_t<MAXB, false>(c, a0, row_blocks, keys_cap);
   BAttnArgs a = a0;
@@ -1417,7 +1420,7 @@ void bild_tuning_default(bild_tuning* t) {
   t->host_loop = 0; t->pdl = 1; t->fused = 3; t->ffn_parts = 0; t->block_simt = 0; t->slice_mode = 2;
   t->slice_min_kb = 3000; t->slice_mma_min = 3; t->slice_head = 2; t->slice_head_min_mb = 32; t->unit_attn = 1;
   t->umma = 1; t->enc_gemm = 1; t->enc_attn_mma = 1; t->enc_parallel = 1; t->spin_limit = 0; t->debug_skip_copies = 0;
-  t->attn_all_keys = 128; t->graph_switch = 1; t->enc_split_k = 1; t->head_stream = 2;
+  t->attn_all_keys = 128; t->graph_switch = 1; t->enc_split_k = 1; t->head_stream = 2; t->enc_attn_groups = EA_MAX_GROUPS;
 }
 
 int bild_create(const bild_config* cfg, const bild_weights* small_w, const bild_weights* large_w, void* workspace,
@@ -1466,6 +1469,7 @@ int bild_create_tuned(const bild_config* cfg, const bild_weights* small_w, const
     c->graph_switch = t.graph_switch != 0;
     c->enc_split_k = t.enc_split_k != 0;
     c->head_stream = std::min(2, std::max(0, t.head_stream));
+    c->enc_attn_groups = std::min(EA_MAX_GROUPS, std::max(1, t.enc_attn_groups));
   }
   {
     int dev = 0;

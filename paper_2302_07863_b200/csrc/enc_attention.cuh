@@ -1,7 +1,8 @@
 // Self-attention of the encoder (set-up step) for d_kv = 64: softmax(Q K^T + bias) V per head over
 // all encoder positions, bias by signed relative position.
-// One block per (head, 64 query rows), 4 warps of 16 rows each; keys and values are visited in tiles
-// of 64 with a running soft-max (no score matrix in memory).  Both products run on mma.sync
+// One block per (head, 64 query rows); a group of 4 warps (16 rows each) visits keys and values in tiles
+// of 64 with a running soft-max (no score matrix in memory); G such groups share a block, group i taking the
+// tiles i, i + G, ... with staging areas of its own, and their (maximum, sum, weighted values) are merged at the end.  Both products run on mma.sync
 // m16n8k16 with every fp32 operand split into a bf16 head and a bf16 remainder and three products
 // kept (head x head, head x remainder, remainder x head), i.e. ~16 mantissa bits per operand:
 //   * the key tile is staged as [key][d] (the "col" operand of Q K^T), the value tile transposed as
@@ -38,29 +39,35 @@ __device__ __forceinline__ void ea_mma(float (&c)[4], uint32_t a0, uint32_t a1, 
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-inline size_t enc_attn_smem_bytes(int max_keys) {
-  return (size_t)4 * EA_KEYS * (EA_D + EA_PAD) * 2 + (size_t)EA_KEYS * (EA_D + EA_RVS) * 4 + (size_t)((max_keys + EA_ROWS + 3) & ~3) * 4;
+constexpr size_t EA_GROUP_BYTES = (size_t)4 * EA_KEYS * (EA_D + EA_PAD) * 2 + (size_t)EA_KEYS * (EA_D + EA_RVS) * 4;   // one group's areas
+constexpr int EA_MAX_GROUPS = 3;   // what fits the shared memory of an SM
+inline size_t enc_attn_smem_bytes(int max_keys, int groups) {
+  return groups * EA_GROUP_BYTES + (size_t)((max_keys + EA_ROWS + 3) & ~3) * 4;
 }
+inline int enc_attn_groups(int max_keys) { return std::max(1, std::min(EA_MAX_GROUPS, (max_keys + EA_KEYS - 1) / EA_KEYS)); }
+__device__ __forceinline__ void ea_group_sync(int grp) { asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "n"(EA_THREADS) : "memory"); }
 
 // q [E][ldq], kc / vc [H][cap][64], out [E][ldo]; bias [H][bias_ld] indexed by bias_off + key - query
 // oh / ol != nullptr: the output is written as its bf16 head and remainder [E][H * 64] (what the
 // output projection reads) instead of fp32
-__global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_bfloat16* oh, __nv_bfloat16* ol) {
+template <int G>
+__global__ void __launch_bounds__(EA_THREADS * G) enc_attn_kernel(BAttnArgs a, __nv_bfloat16* oh, __nv_bfloat16* ol) {
   extern __shared__ __align__(16) unsigned char ea_smem[];
   constexpr int ST = EA_D + EA_PAD;   // staged row length (bf16 elements)
-  __nv_bfloat16* sKh = reinterpret_cast<__nv_bfloat16*>(ea_smem);   // [key][d]
+  const int grp = threadIdx.x / EA_THREADS;   // key group of this warp
+  __nv_bfloat16* sKh = reinterpret_cast<__nv_bfloat16*>(ea_smem + grp * EA_GROUP_BYTES);   // [key][d]
   __nv_bfloat16* sKl = sKh + EA_KEYS * ST;
   __nv_bfloat16* sVh = sKl + EA_KEYS * ST;                          // [d][key]
   __nv_bfloat16* sVl = sVh + EA_D * ST;
   float* sRawK = reinterpret_cast<float*>(sVl + EA_D * ST);        // [key][64] fp32 as it lies in the cache
   float* sRawV = sRawK + EA_KEYS * EA_D;                            // [key][EA_RVS]
-  float* sBias = sRawV + EA_KEYS * EA_RVS;                          // [E + 63]: entry (key - query + r0 + 63)
+  float* sBias = reinterpret_cast<float*>(ea_smem + G * EA_GROUP_BYTES);   // [E + 63]: entry (key - query + r0 + 63)
   const int h = blockIdx.x, r0 = blockIdx.y * EA_ROWS;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int tid = threadIdx.x % EA_THREADS, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;   // (within the group)
   pdl_launch_dependents();
   pdl_wait();
   const int E = min(min(a.M, *a.n_keys_dev), a.cap);
-  for (int i = tid; i < E + EA_ROWS - 1; i += EA_THREADS) {
+  for (int i = threadIdx.x; i < E + EA_ROWS - 1; i += EA_THREADS * G) {
     // key - query for query r0 + 63 - ... : entry i stands for key - query = i - (r0 + 63)
     const int rel = i - (r0 + EA_ROWS - 1);
     const int idx = a.bias_off + rel;
@@ -100,11 +107,12 @@ __global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  fetch(0);
+  if (grp * EA_KEYS < E) fetch(grp * EA_KEYS);
+  __syncthreads();   // the bias table is complete
 #pragma unroll 1
-  for (int k0 = 0; k0 < E; k0 += EA_KEYS) {
+  for (int k0 = grp * EA_KEYS; k0 < E; k0 += EA_KEYS * G) {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();   // the raw tile has arrived for everybody; the previous tile is no longer read
+    ea_group_sync(grp);   // the raw tile has arrived for the whole group; the previous tile is no longer read
     // stage the tile.  Keys: thread -> (key, 4 channels), rows written 8 bytes at a time.
     for (int idx = tid; idx < EA_KEYS * (EA_D / 4); idx += EA_THREADS) {
       const int key = idx >> 4, c4 = (idx & 15) << 2;
@@ -130,8 +138,8 @@ __global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_
         *reinterpret_cast<uint32_t*>(sVl + (c4 + e) * ST + 2 * kp) = lv;
       }
     }
-    __syncthreads();
-    if (k0 + EA_KEYS < E) fetch(k0 + EA_KEYS);   // (the raw area is free again: everybody has converted its share)
+    ea_group_sync(grp);
+    if (k0 + EA_KEYS * G < E) fetch(k0 + EA_KEYS * G);   // (the raw area is free again: everybody has converted its share)
     // scores of 16 rows x 64 keys
     float s[8][4];
 #pragma unroll
@@ -200,6 +208,42 @@ __global__ void __launch_bounds__(EA_THREADS) enc_attn_kernel(BAttnArgs a, __nv_
         ea_mma(o[dt], ph[0], ph[1], ph[2], ph[3], bh0, bh1);
         ea_mma(o[dt], ph[0], ph[1], ph[2], ph[3], bl0, bl1);
         ea_mma(o[dt], pl[0], pl[1], pl[2], pl[3], bh0, bh1);
+      }
+    }
+  }
+  if (G > 1) {   // the groups' partial results meet in group 0 (thread to thread: the same rows and channels), in group order
+    float* sM = reinterpret_cast<float*>(sKh);   // [36][EA_THREADS] in the group's own staging area
+    ea_group_sync(grp);                          // the last tile is no longer read
+    if (grp > 0) {
+#pragma unroll
+      for (int dt = 0; dt < 8; ++dt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sM[(dt * 4 + e) * EA_THREADS + tid] = o[dt][e];
+      sM[32 * EA_THREADS + tid] = m_a; sM[33 * EA_THREADS + tid] = m_b;
+      sM[34 * EA_THREADS + tid] = l_a; sM[35 * EA_THREADS + tid] = l_b;
+    }
+    __syncthreads();
+    if (grp > 0) return;
+    float gm_a = m_a, gm_b = m_b;
+#pragma unroll
+    for (int j = 1; j < G; ++j) {
+      const float* sJ = reinterpret_cast<const float*>(ea_smem + j * EA_GROUP_BYTES);
+      gm_a = fmaxf(gm_a, sJ[32 * EA_THREADS + tid]); gm_b = fmaxf(gm_b, sJ[33 * EA_THREADS + tid]);
+    }
+    const float w_a = m_a == -INFINITY ? 0.f : __expf(m_a - gm_a), w_b = m_b == -INFINITY ? 0.f : __expf(m_b - gm_b);
+    l_a *= w_a; l_b *= w_b;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) { o[dt][0] *= w_a; o[dt][1] *= w_a; o[dt][2] *= w_b; o[dt][3] *= w_b; }
+#pragma unroll
+    for (int j = 1; j < G; ++j) {
+      const float* sJ = reinterpret_cast<const float*>(ea_smem + j * EA_GROUP_BYTES);
+      const float mj_a = sJ[32 * EA_THREADS + tid], mj_b = sJ[33 * EA_THREADS + tid];
+      const float v_a = mj_a == -INFINITY ? 0.f : __expf(mj_a - gm_a), v_b = mj_b == -INFINITY ? 0.f : __expf(mj_b - gm_b);
+      l_a += sJ[34 * EA_THREADS + tid] * v_a; l_b += sJ[35 * EA_THREADS + tid] * v_b;
+#pragma unroll
+      for (int dt = 0; dt < 8; ++dt) {
+        o[dt][0] += sJ[(dt * 4 + 0) * EA_THREADS + tid] * v_a; o[dt][1] += sJ[(dt * 4 + 1) * EA_THREADS + tid] * v_a;
+        o[dt][2] += sJ[(dt * 4 + 2) * EA_THREADS + tid] * v_b; o[dt][3] += sJ[(dt * 4 + 3) * EA_THREADS + tid] * v_b;
       }
     }
   }

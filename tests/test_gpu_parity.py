@@ -300,6 +300,28 @@ def test_encode_cross_kv_match_oracle(torch_cuda, name):
     ctx.close()
 
 
+@pytest.mark.parametrize("groups", [1, 2, 3])
+@pytest.mark.parametrize("E", [130, 192, 210])
+def test_encode_long_sources_match_oracle(torch_cuda, E, groups):
+    """Sources of three and four key tiles (ragged and full last tile) through the encoder's attention kernel with one,
+    two and three key groups per block: cross-attention keys and values against oracle.t5.Model.start."""
+    from paper_2302_07863_b200.synthetic import make_context
+    wl = WORKLOADS["wide_bf16"]
+    ctx, _, _ = make_context("wide_bf16", 10.0, 10.0, max_enc_len=210, tuning=dict(enc_attn_groups=groups))
+    ids = gen_ids(MODEL_SHAPES[wl.small].vocab, E, wl.seed + 3)
+    ctx.encode(ids)
+    for which, key in ((0, wl.small), (1, wl.large)):
+        sh = MODEL_SHAPES[key]
+        st = Model(sh, gen_model(sh, wl.seed, wl.dtype), 1.0).start(ids, 4)
+        for l in range(sh.n_layers):
+            for what, ref in ((0, st.ck[l]), (1, st.cv[l])):
+                got = ctx.read_cache(which, what, l, sh.n_heads, 210, sh.d_kv)[:, :E, :]
+                want = ref.reshape(E, sh.n_heads, sh.d_kv).transpose(1, 0, 2)
+                err = float(np.max(np.abs(got - want)))
+                assert err <= 2e-3 * max(1.0, float(np.max(np.abs(want)))), (E, groups, which, l, what, err)
+    ctx.close()
+
+
 # ---- whole loop against the stored oracle runs ------------------------------------------
 @pytest.mark.parametrize("name", ["tiny", "odd", "odd_bf16", "tiny_bf16"])
 def test_generate_matches_golden(torch_cuda, name):
