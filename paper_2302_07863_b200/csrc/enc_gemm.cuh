@@ -9,7 +9,7 @@
 //     thread issues tcgen05.mma M128 N256 K16: the H_hi and H_lo tiles sit back to back in the
 //     stage and form one 256-row operand, so each weight tile is read once per k step; the
 //     accumulator in tensor memory has 128 columns for hi and 128 for lo (a second accumulator
-//     for the gate matrix of a gated FFN); the epilogue reads 16 token columns of both at a time, adds them and applies store / ReLU / GELU gate / residual add /
+//     for the gate matrix of a gated FFN); the epilogue (all 16 warps: four per quarter of the rows, 32 token columns each) adds them and applies store / ReLU / GELU gate / residual add /
 //     scatter to q and the K/V layout, writing 32 consecutive outputs of one token per warp;
 //   * the FFN's first matrix can write its output directly as the bf16 head / remainder pair that
 //     the second matrix reads (no fp32 round trip, no separate split);
@@ -23,7 +23,7 @@
 
 namespace bild {
 
-constexpr int EG_THREADS = 128;
+constexpr int EG_THREADS = 512;   // thread 0 feeds the ring, thread 32 issues the MMAs, all 16 warps share the epilogue
 constexpr int EG_TOK = 128;   // tokens per tile
 
 // H_hi / H_lo of one row per warp; rows >= M are written as zeros (the last tile's padding)
@@ -173,65 +173,89 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
   if (!mbar_wait(done, 0)) *err = BILD_ERR_TIMEOUT;
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
-  // ---- epilogue: thread t holds weight row n_base + t; 16 token columns at a time ----
-  const int n = n_base + tid;
+  // ---- epilogue: a warp reads the 32 lanes (weight rows) of tensor memory that its number modulo 4 gives it access to; the
+  // four warps of a lane quarter share the 128 token columns, 32 each.  One warp per scheduler would be bound by the
+  // latency of its own instruction stream (measured: 5-10 us for the 128 columns), so all 16 warps of the block take part.
+  const int quarter = warp & 3, colgrp = warp >> 2;
+  const int n = n_base + quarter * 32 + (tid & 31);
   const bool row_ok = n < a.N;
-  const uint32_t t0 = tmem + ((uint32_t)(warp * 32) << 16);
+  const uint32_t t0 = tmem + ((uint32_t)(quarter * 32) << 16);
   int part = a.first_part, rr = n;
   if (a.epi == EPI_HEADS) {
     if (rr >= a.inner) { rr -= a.inner; ++part; }
     if (rr >= a.inner) { rr -= a.inner; ++part; }
   }
   const int hh = a.epi == EPI_HEADS ? rr / a.dkv : 0, hc = a.epi == EPI_HEADS ? rr % a.dkv : 0;
+  constexpr int CH = GATED ? 16 : 32;   // token columns per turn (registers: four loads of CH columns in flight when gated)
 #pragma unroll 1
-  for (int c0 = 0; c0 < EG_TOK; c0 += 16) {
-    float v0[16], v1[16], lo16[16];
-    tmem_ld16(t0 + c0, v0);
-    tmem_ld16(t0 + 128 + c0, lo16);
+  for (int c0 = colgrp * 32; c0 < colgrp * 32 + 32; c0 += CH) {
+    uint32_t rh[CH], rl[CH], gh[GATED ? CH : 1], gl[GATED ? CH : 1];
+    if constexpr (GATED) {
+      tmem_ld16_issue(t0 + c0, rh); tmem_ld16_issue(t0 + 128 + c0, rl);
+      tmem_ld16_issue(t0 + 256 + c0, gh); tmem_ld16_issue(t0 + 384 + c0, gl);
+    } else {
+      tmem_ld32_issue(t0 + c0, rh); tmem_ld32_issue(t0 + 128 + c0, rl);
+    }
+    tmem_ld_wait();
+    tmem_ld_pin(rh); tmem_ld_pin(rl);
+    if constexpr (GATED) { tmem_ld_pin(gh); tmem_ld_pin(gl); }
+    float v0[CH];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) v0[j] += lo16[j];
-    if (GATED) {
-      tmem_ld16(t0 + 256 + c0, v1);
-      tmem_ld16(t0 + 384 + c0, lo16);
-#pragma unroll
-      for (int j = 0; j < 16; ++j) v1[j] += lo16[j];
+    for (int j = 0; j < CH; ++j) {
+      v0[j] = __uint_as_float(rh[j]) + __uint_as_float(rl[j]);
+      if constexpr (GATED) v0[j] = gelu_tanh(v0[j]) * (__uint_as_float(gh[j]) + __uint_as_float(gl[j]));
     }
     if (!row_ok) continue;
-    if (a.epi == EPI_RESID && gridDim.z > 1) {   // split over K: the partial tile is added to the stream where it lies
+    const int tokb = tok0 + c0;
+    int lim = a.M - tokb;   // token columns of this turn that exist
+    if (a.epi == EPI_RESID) {
+      float* p = a.Y + (size_t)tokb * a.ldy + n;
+      if (gridDim.z > 1) {   // split over K: the partial tile is added to the stream where it lies
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if (tok0 + c0 + j < a.M) atomicAdd(a.Y + (size_t)(tok0 + c0 + j) * a.ldy + n, v0[j]);
-      continue;
-    }
-    if (a.epi == EPI_RESID) {   // all 16 old values are requested before any of them is needed
-      float old[16];
+        for (int j = 0; j < CH; ++j)
+          if (j < lim) atomicAdd(p + (size_t)j * a.ldy, v0[j]);
+      } else {   // all old values are requested before any of them is needed
+        float old[CH];
 #pragma unroll
-      for (int j = 0; j < 16; ++j) old[j] = tok0 + c0 + j < a.M ? __ldcg(a.Y + (size_t)(tok0 + c0 + j) * a.ldy + n) : 0.f;
+        for (int j = 0; j < CH; ++j) old[j] = j < lim ? __ldcg(p + (size_t)j * a.ldy) : 0.f;
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if (tok0 + c0 + j < a.M) a.Y[(size_t)(tok0 + c0 + j) * a.ldy + n] = old[j] + v0[j];
-      continue;
-    }
+        for (int j = 0; j < CH; ++j)
+          if (j < lim) p[(size_t)j * a.ldy] = old[j] + v0[j];
+      }
+    } else if (a.epi == EPI_HEADS) {
+      if (part == 0) {
+        float* p = a.q_out + (size_t)tokb * a.ldq + rr;
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const int tok = tok0 + c0 + j;
-      if (tok >= a.M) break;
-      float y = v0[j];
-      if (a.epi == EPI_STORE) a.Y[(size_t)tok * a.ldy + n] = y;
-      else if (a.epi == EPI_RELU || a.epi == EPI_GATED) {
-        if (a.epi == EPI_RELU) y = fmaxf(y, 0.f);
-        else if (GATED) y = gelu_tanh(y) * v1[j];
-        if (oh) {   // the next layer reads this as bf16 head + remainder: write that form directly
-          const __nv_bfloat16 hv = __float2bfloat16_rn(y);
-          oh[(size_t)tok * a.N + n] = hv;
-          ol[(size_t)tok * a.N + n] = __float2bfloat16_rn(y - __bfloat162float(hv));
-        } else {
-          a.Y[(size_t)tok * a.ldy + n] = y;
-        }
+        for (int j = 0; j < CH; ++j)
+          if (j < lim) p[(size_t)j * a.ldq] = v0[j];
       } else {
-        const int row = a.pos0_host + tok;
-        if (part == 0) a.q_out[(size_t)tok * a.ldq + rr] = y;
-        else if (row < a.cap) (part == 1 ? a.kc : a.vc)[((size_t)hh * a.cap + row) * a.dkv + hc] = y;
+        const int row0 = a.pos0_host + tokb;
+        lim = min(lim, a.cap - row0);
+        float* p = (part == 1 ? a.kc : a.vc) + ((size_t)hh * a.cap + row0) * a.dkv + hc;
+#pragma unroll
+        for (int j = 0; j < CH; ++j)
+          if (j < lim) p[(size_t)j * a.dkv] = v0[j];
+      }
+    } else {
+      if (a.epi == EPI_RELU) {
+#pragma unroll
+        for (int j = 0; j < CH; ++j) v0[j] = fmaxf(v0[j], 0.f);
+      }
+      if (oh && a.epi != EPI_STORE) {   // the next layer reads this as bf16 head + remainder: write that form directly
+        __nv_bfloat16* ph = oh + (size_t)tokb * a.N + n;
+        __nv_bfloat16* pl = ol + (size_t)tokb * a.N + n;
+#pragma unroll
+        for (int j = 0; j < CH; ++j)
+          if (j < lim) {
+            const __nv_bfloat16 hv = __float2bfloat16_rn(v0[j]);
+            ph[(size_t)j * a.N] = hv;
+            pl[(size_t)j * a.N] = __float2bfloat16_rn(v0[j] - __bfloat162float(hv));
+          }
+      } else {
+        float* p = a.Y + (size_t)tokb * a.ldy + n;
+#pragma unroll
+        for (int j = 0; j < CH; ++j)
+          if (j < lim) p[(size_t)j * a.ldy] = v0[j];
       }
     }
   }
