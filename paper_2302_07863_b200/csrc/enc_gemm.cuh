@@ -43,6 +43,54 @@ __global__ void __launch_bounds__(128) norm_split_kernel(const float* __restrict
     return;
   }
   const float* x = X + (size_t)row * ldx;
+  auto split8 = [&](int c, const float (&h)[8]) {
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(h[2 * i]), h1 = __float2bfloat16_rn(h[2 * i + 1]);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(h[2 * i] - __bfloat162float(h0));
+      const __nv_bfloat16 l1 = __float2bfloat16_rn(h[2 * i + 1] - __bfloat162float(h1));
+      hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    }
+    *reinterpret_cast<uint4*>(oh + c) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(ol + c) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  };
+  if (K <= 1024) {   // the row stays in registers between the sum of squares and the split: one round of loads
+    float h[4][8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int c = lane * 8 + 256 * i;
+      float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+      if (c < K) { a0 = *reinterpret_cast<const float4*>(x + c); a1 = *reinterpret_cast<const float4*>(x + c + 4); }
+      h[i][0] = a0.x; h[i][1] = a0.y; h[i][2] = a0.z; h[i][3] = a0.w; h[i][4] = a1.x; h[i][5] = a1.y; h[i][6] = a1.z; h[i][7] = a1.w;
+    }
+    if (gain) {
+      float ss = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ss += h[i][e] * h[i][e];
+      ss = warp_sum(ss);
+      const float inv = rsqrtf(ss / (float)K + eps);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int c = lane * 8 + 256 * i;
+        if (c < K) {
+          const float4 g0 = __ldg(reinterpret_cast<const float4*>(gain + c)), g1 = __ldg(reinterpret_cast<const float4*>(gain + c + 4));
+          const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+          for (int e = 0; e < 8; ++e) h[i][e] = h[i][e] * g[e] * inv;
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int c = lane * 8 + 256 * i;
+      if (c < K) split8(c, h[i]);
+    }
+    return;
+  }
   float inv = 1.f;
   if (gain) {
     float ss = 0.f;
@@ -62,17 +110,7 @@ __global__ void __launch_bounds__(128) norm_split_kernel(const float* __restrict
 #pragma unroll
       for (int i = 0; i < 8; ++i) h[i] = h[i] * g[i] * inv;
     }
-    uint32_t hi[4], lo[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const __nv_bfloat16 h0 = __float2bfloat16_rn(h[2 * i]), h1 = __float2bfloat16_rn(h[2 * i + 1]);
-      const __nv_bfloat16 l0 = __float2bfloat16_rn(h[2 * i] - __bfloat162float(h0));
-      const __nv_bfloat16 l1 = __float2bfloat16_rn(h[2 * i + 1] - __bfloat162float(h1));
-      hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-      lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-    }
-    *reinterpret_cast<uint4*>(oh + c) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-    *reinterpret_cast<uint4*>(ol + c) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    split8(c, h);
   }
 }
 
