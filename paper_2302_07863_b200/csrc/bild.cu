@@ -2050,6 +2050,15 @@ int bild_debug_stamps(unsigned long long* out, int reset) {
   }
   return BILD_OK;
 }
+// Cycle stamps of the encoder GEMM (debug builds only): 3 x 16 counters, optionally cleared.
+int bild_debug_gemm_stamps(unsigned long long* out, int reset) {
+  if (out && cudaMemcpyFromSymbol(out, g_eg_stamps, sizeof(g_eg_stamps)) != cudaSuccess) return BILD_ERR_CUDA;
+  if (reset) {
+    static unsigned long long zero[3][16];
+    if (cudaMemcpyToSymbol(g_eg_stamps, zero, sizeof(zero)) != cudaSuccess) return BILD_ERR_CUDA;
+  }
+  return BILD_OK;
+}
 #endif
 
 // Test helper: copies one layer's cached keys or values to the host (synchronises the stream).

@@ -26,6 +26,18 @@ namespace bild {
 constexpr int EG_THREADS = 512;   // thread 0 feeds the ring, thread 32 issues the MMAs, all 16 warps share the epilogue
 constexpr int EG_TOK = 128;   // tokens per tile
 
+// Optional cycle stamps (build with -DBILD_STAMPS), summed over the blocks of the T5-large-shaped GEMMs of 512 tokens:
+// [class: QKV (24 row tiles), FFN-up (32), residual (8, K split)][slot]; slot 15 counts the blocks.  Slots 0-4: a thread
+// of warp 2 (start -> tensor memory allocated -> dependency wait returned -> all MMAs done -> epilogue done; 4: its loads
+// from tensor memory); 8, 9: the MMA thread (wait -> first stage full -> last MMA issued); 12: the producer (wait ->
+// last copy issued).
+#ifdef BILD_STAMPS
+__device__ unsigned long long g_eg_stamps[3][16];
+#define EG_STAMP(v) v = clock64()
+#else
+#define EG_STAMP(v)
+#endif
+
 // H_hi / H_lo of one row per warp; rows >= M are written as zeros (the last tile's padding)
 __global__ void __launch_bounds__(128) norm_split_kernel(const float* __restrict__ X, int ldx, const float* __restrict__ gain,
                                                          float eps, int M, int K, __nv_bfloat16* __restrict__ Hh,
@@ -140,6 +152,10 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
   constexpr int TCOLS = 256 * NMAT;
   extern __shared__ unsigned char eg_raw[];
   const int tid = threadIdx.x, warp = tid >> 5;
+#ifdef BILD_STAMPS
+  long long T0, T1 = 0, T2 = 0, T3 = 0, T4 = 0, TM1 = 0, TM2 = 0, TP1 = 0, TL = 0, TA = 0;
+#endif
+  EG_STAMP(T0);
   const int n_base = blockIdx.x * UM_TILE_M, tok0 = blockIdx.y * EG_TOK;
   // this block's share of the K blocks (gridDim.z splits, EPI_RESID only)
   const int nkb_all = a.K / UM_KB, kb0 = (int)(((long long)blockIdx.z * nkb_all) / gridDim.z);
@@ -162,6 +178,7 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
+  EG_STAMP(T1);
   // thread 0 feeds the ring; the weight tiles depend on nothing and are requested before the dependency wait
   // for the first NST stages, the activation tiles of those stages follow after it (same barrier per stage)
   auto load_weights = [&](int kb) {
@@ -181,6 +198,7 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
     for (int kb = 0; kb < nkb && kb < NST; ++kb) load_weights(kb);
   pdl_launch_dependents();
   pdl_wait();   // the activation tiles were written by the kernel in front
+  EG_STAMP(T2);
   if (tid == 0) {
     asm volatile("fence.proxy.async;" ::: "memory");   // rows written with ordinary stores, read by the copy engine
     for (int kb = 0; kb < nkb; ++kb) {
@@ -190,11 +208,15 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
       }
       load_acts(kb);
     }
+    EG_STAMP(TP1);
   } else if (tid == 32) {
     for (int kb = 0; kb < nkb; ++kb) {
       const int st = kb % NST;
       if (!mbar_wait(&full[st], (kb / NST) & 1)) *err = BILD_ERR_TIMEOUT;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#ifdef BILD_STAMPS
+      if (kb == 0) TM1 = clock64();
+#endif
       const uint32_t a0 = smem_u32(base + (size_t)st * STAGE);
       const uint32_t bh = a0 + NMAT * 16384;   // hi tile, lo tile right behind it: one operand of 256 rows
 #pragma unroll
@@ -206,10 +228,12 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
       umma_commit(&empty[st]);   // the stage may be refilled once these MMAs have read it
     }
     umma_commit(done);
+    EG_STAMP(TM2);
   }
   __syncwarp();
   if (!mbar_wait(done, 0)) *err = BILD_ERR_TIMEOUT;
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  EG_STAMP(T3);
 
   // ---- epilogue: a warp reads the 32 lanes (weight rows) of tensor memory that its number modulo 4 gives it access to; the
   // four warps of a lane quarter share the 128 token columns, 32 each.  One warp per scheduler would be bound by the
@@ -228,6 +252,7 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
 #pragma unroll 1
   for (int c0 = colgrp * 32; c0 < colgrp * 32 + 32; c0 += CH) {
     uint32_t rh[CH], rl[CH], gh[GATED ? CH : 1], gl[GATED ? CH : 1];
+    EG_STAMP(TA);
     if constexpr (GATED) {
       tmem_ld16_issue(t0 + c0, rh); tmem_ld16_issue(t0 + 128 + c0, rl);
       tmem_ld16_issue(t0 + 256 + c0, gh); tmem_ld16_issue(t0 + 384 + c0, gl);
@@ -236,6 +261,9 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
     }
     tmem_ld_wait();
     tmem_ld_pin(rh); tmem_ld_pin(rl);
+#ifdef BILD_STAMPS
+    TL += clock64() - TA;
+#endif
     if constexpr (GATED) { tmem_ld_pin(gh); tmem_ld_pin(gl); }
     float v0[CH];
 #pragma unroll
@@ -297,6 +325,20 @@ __global__ void __launch_bounds__(EG_THREADS) enc_gemm_kernel(LinArgs a, int* er
       }
     }
   }
+#ifdef BILD_STAMPS
+  T4 = clock64();
+  const int cls = a.M != 512 ? -1 : gridDim.x == 24 ? 0 : gridDim.x == 32 ? 1 : (gridDim.x == 8 && a.epi == EPI_RESID) ? 2 : -1;
+  if (cls >= 0) {
+    unsigned long long* S = g_eg_stamps[cls];
+    if (tid == 64) {
+      atomicAdd(S + 0, (unsigned long long)(T1 - T0)); atomicAdd(S + 1, (unsigned long long)(T2 - T1));
+      atomicAdd(S + 2, (unsigned long long)(T3 - T2)); atomicAdd(S + 3, (unsigned long long)(T4 - T3));
+      atomicAdd(S + 4, (unsigned long long)TL); atomicAdd(S + 15, 1ull);
+    }
+    if (tid == 32) { atomicAdd(S + 8, (unsigned long long)(TM1 - T2)); atomicAdd(S + 9, (unsigned long long)(TM2 - TM1)); }
+    if (tid == 0) atomicAdd(S + 12, (unsigned long long)(TP1 - T2));
+  }
+#endif
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(TCOLS) : "memory");

@@ -5,7 +5,8 @@ any block took in any launch):
 
 Builds a second copy of the library with -DBILD_STAMPS (libbild_stamps.so beside libbild.so: the same kernels plus
 clock64() reads at the phase boundaries and a debug entry point that returns the sums) and replays the small step
-and the large pass for the given row counts.  The stamped build is a few percent slower than the product build."""
+and the large pass for the given row counts, then the set-up step (phases of the encoder GEMM's blocks, T5-large shapes
+at 512 tokens).  The stamped build is a few percent slower than the product build."""
 import ctypes as C, json, os, sys
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 sys.path.insert(0, ROOT)
@@ -47,3 +48,21 @@ def run(which, k):
               " ".join(f"{a}={b:.2f}/{c:.2f}/{e:.2f}" for a, b, c, e in zip(nms, ph0, pha, phm)))
 run(0, 1)
 for k in ks: run(1, k)
+
+# ---- encoder GEMM: phases of a block (sources of 512 ids) ----
+import torch
+L.bild_debug_gemm_stamps.argtypes = [C.POINTER(C.c_ulonglong), C.c_int]
+gb = (C.c_ulonglong * 48)()
+for _ in range(3): ctx.encode(ids)
+torch.cuda.synchronize()
+L.bild_debug_gemm_stamps(gb, 1)
+for _ in range(5): ctx.encode(ids)
+torch.cuda.synchronize()
+L.bild_debug_gemm_stamps(gb, 0)
+for cls, nm in enumerate(["QKV (24 x 4 tiles)", "FFN-up (32 x 4)", "residual (8 x 4, K split)"]):
+    n = gb[cls * 16 + 15]
+    if not n: continue
+    f = lambda i: gb[cls * 16 + i] / n / 1965.0
+    print(f"== encoder GEMM {nm}: {n} blocks | start -> tensor memory allocated {f(0):.2f} us | -> dependency wait returned {f(1):.2f} | "
+          f"-> all MMAs done {f(2):.2f} (MMA thread: wait -> first stage full {f(8):.2f}, first -> last MMA issued {f(9):.2f}; "
+          f"producer: wait -> last copy issued {f(12):.2f}) | epilogue {f(3):.2f} (loads from tensor memory {f(4):.2f})")
