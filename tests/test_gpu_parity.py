@@ -301,10 +301,10 @@ def test_encode_cross_kv_match_oracle(torch_cuda, name):
 
 
 @pytest.mark.parametrize("groups", [1, 2, 3])
-@pytest.mark.parametrize("E", [130, 192, 210])
+@pytest.mark.parametrize("E", [40, 130, 192, 210])
 def test_encode_long_sources_match_oracle(torch_cuda, E, groups):
-    """Sources of three and four key tiles (ragged and full last tile) through the encoder's attention kernel with one,
-    two and three key groups per block: cross-attention keys and values against oracle.t5.Model.start."""
+    """Sources of one, three and four key tiles (ragged and full last tile; one tile leaves the other groups of a block
+    without work) through the encoder's attention kernel with one, two and three key groups per block: cross-attention keys and values against oracle.t5.Model.start."""
     from paper_2302_07863_b200.synthetic import make_context
     wl = WORKLOADS["wide_bf16"]
     ctx, _, _ = make_context("wide_bf16", 10.0, 10.0, max_enc_len=210, tuning=dict(enc_attn_groups=groups))
