@@ -123,7 +123,7 @@ struct Model {
   uint4* wfo_blk = nullptr;          // [layers][F / 8][pack_wfo_dpad(d)]
   CallDesc* desc_lo = nullptr;       // the two chunks of a block of 9 to 16 rows (split_desc_kernel)
   CallDesc* desc_hi = nullptr;
-  AttnSubPlan sub_self{}, sub_cross{};   // chunk sizes of the attention sub-layers
+  AttnSubPlan sub_self[2]{}, sub_cross[2]{};   // chunk sizes of the attention sub-layers: [0] single-row kernel, [1] block kernel
   int sub_parts = 1;                 // launches the feed-forward sub-layer is split into
 };
 
@@ -687,9 +687,12 @@ int setup_fused(bild_ctx* c, Model& m) {
     return BILD_OK;
   }
   const int all_keys = c->attn_all_keys;
-  const AttnSubPlan ps = attn_sub_plan(d, dkv, 3, C, cap, all_keys, SUB_HALF_SM, smem_max);
-  const AttnSubPlan pc = attn_sub_plan(d, dkv, 1, C, ecap, all_keys, SUB_HALF_SM, smem_max);
-  if (!ps.ok || !pc.ok) return BILD_OK;
+  AttnSubPlan ps[2], pc[2];
+  for (int v = 0; v < 2; ++v) {
+    ps[v] = attn_sub_plan(d, dkv, 3, C, cap, all_keys, SUB_HALF_SM, smem_max, v ? SUB_MB : 1);
+    pc[v] = attn_sub_plan(d, dkv, 1, C, ecap, all_keys, SUB_HALF_SM, smem_max, v ? SUB_MB : 1);
+    if (!ps[v].ok || !pc[v].ok) return BILD_OK;
+  }
   int parts = std::max(1, c->sub_parts_want);
   const int nmat = gated ? 2 : 1;
   while (parts <= 8 && (ffn_sub_rows(F, c->sms * parts) * nmat > SUB_MAX_ROWS || ffn_sub_rows(F, c->sms * parts) > SUB_FO_REGS ||
@@ -708,7 +711,8 @@ int setup_fused(bild_ctx* c, Model& m) {
     (*c->cnt)++;
   }
   CUDA_TRY(c, cudaGetLastError());
-  m.sub_C = C; m.sub_self = ps; m.sub_cross = pc; m.sub_parts = parts;
+  m.sub_C = C; m.sub_parts = parts;
+  for (int v = 0; v < 2; ++v) { m.sub_self[v] = ps[v]; m.sub_cross[v] = pc[v]; }
   m.fused = true;
   return BILD_OK;
 }
@@ -763,7 +767,8 @@ int fused_layer(bild_ctx* c, Model& m, int MB, int l, const CallDesc* desc, int 
   a.x_in = x; a.x_out = xb; a.x_zero = xc; a.gain = (const float*)w.ln1;
   a.Wp = (const __nv_bfloat16*)w.wqkv; a.Wo = (const __nv_bfloat16*)w.wo;
   a.kc = m.selfK + kvoff * cap; a.vc = m.selfV + kvoff * cap; a.cap = cap; a.bias = m.dec_bias; a.bias_ld = cap; a.self = 1;
-  a.kc_keys = m.sub_self.kc; a.bias_len = m.sub_self.bias_len; a.red_keys = m.sub_self.red_keys;
+  const AttnSubPlan& pls = m.sub_self[MB == 1 ? 0 : 1];
+  a.kc_keys = pls.kc; a.bias_len = pls.bias_len; a.red_keys = pls.red_keys;
   a.L = attn_sub_layout(d, dkv, 3, C, MB, a.kc_keys, a.bias_len);
   CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a, !first_plain));
   int rc = after_self();
@@ -773,7 +778,8 @@ int fused_layer(bild_ctx* c, Model& m, int MB, int l, const CallDesc* desc, int 
   a.x_in = xb; a.x_out = xc; a.x_zero = x; a.gain = (const float*)w.ln2;
   a.Wp = (const __nv_bfloat16*)w.wcq; a.Wo = (const __nv_bfloat16*)w.wco;
   a.kc = m.crossK + kvoff * ecap; a.vc = m.crossV + kvoff * ecap; a.cap = ecap; a.bias = nullptr; a.bias_ld = 0; a.self = 0;
-  a.kc_keys = m.sub_cross.kc; a.bias_len = m.sub_cross.bias_len; a.red_keys = m.sub_cross.red_keys;
+  const AttnSubPlan& plc = m.sub_cross[MB == 1 ? 0 : 1];
+  a.kc_keys = plc.kc; a.bias_len = plc.bias_len; a.red_keys = plc.red_keys;
   a.L = attn_sub_layout(d, dkv, 1, C, MB, a.kc_keys, a.bias_len);
   CUDA_TRY(c, launch_sub(c, MB == 1 ? attn_sub_kernel<true> : attn_sub_kernel<false>, H * C, C, (size_t)a.L.total, a));
   // S7-S8 / L7-L8
@@ -1908,7 +1914,7 @@ int bild_op_attn_sublayer(int self, const void* Wp, const void* Wo, const float*
   const int MB = M == 1 ? 1 : SUB_MB, I = H * dkv, P = self ? 3 : 1;
   int smem_max = 0, dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return BILD_ERR_CUDA;
-  const AttnSubPlan pl = attn_sub_plan(d, dkv, P, C, cap, 128, SUB_HALF_SM, smem_max);
+  const AttnSubPlan pl = attn_sub_plan(d, dkv, P, C, cap, 128, SUB_HALF_SM, smem_max, MB);
   if (!pl.ok) return BILD_ERR_CAPACITY;
   const int kc_keys = pl.kc, bias_len = pl.bias_len;
   OpScratch o = op_scratch(scratch, d);

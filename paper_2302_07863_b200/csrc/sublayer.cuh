@@ -305,15 +305,16 @@ inline AttnSubLayout attn_sub_layout(int d, int dkv, int P, int C, int mb, int k
 
 // Chunk size, bias room and the key count up to which the ranks attend redundantly, for a cache of keys_cap keys.
 // `all_keys` > 0 asks for a chunk that holds up to that many keys so that short caches need no second exchange; the
-// chunk shrinks until the single-row and the block layout both stay under `prefer` bytes (half an SM), else under `limit`.
+// chunk shrinks until the layout for passes of `mb` rows (1: the single-row kernel, SUB_MB: the block kernel; each has a plan
+// of its own) stays under `prefer` bytes (half an SM), else under `limit`.
 struct AttnSubPlan { int kc, bias_len, red_keys; bool ok; };
-inline AttnSubPlan attn_sub_plan(int d, int dkv, int P, int C, int keys_cap, int all_keys, int prefer, int limit) {
+inline AttnSubPlan attn_sub_plan(int d, int dkv, int P, int C, int keys_cap, int all_keys, int prefer, int limit, int mb) {
   AttnSubPlan pl;
   const int per_rank = (keys_cap + C - 1) / C;
   const int need = std::min(64, sub_up16(per_rank)), want = std::min(128, sub_up16(std::min(all_keys, keys_cap)));
   auto blen = [&](int kc) { return P == 3 ? (std::max(per_rank, kc) + MAXB + 8 + 3) / 4 * 4 : 4; };
   auto fits = [&](int kc, int lim) {
-    return attn_sub_layout(d, dkv, P, C, 1, kc, blen(kc)).total <= lim && attn_sub_layout(d, dkv, P, C, SUB_MB, kc, blen(kc)).total <= lim;
+    return attn_sub_layout(d, dkv, P, C, mb, kc, blen(kc)).total <= lim;
   };
   int kc = std::max(need, want);
   while (kc > need && !fits(kc, prefer)) kc -= 16;

@@ -557,6 +557,12 @@ def test_eos_and_limits(torch_cuda):
         ctx.large_verify([1] * 17, 1.0)
     with pytest.raises(BildError):
         ctx.rewind(0, 10 ** 6)
+    # an empty source and one beyond the configured capacity are refused on the host; the context then needs a valid encode
+    for bad in (np.zeros(0, np.int32), np.full(wl.enc_len + 1, 2, np.int32)):
+        with pytest.raises(BildError) as e:
+            ctx.encode(bad)
+        assert e.value.code == -4
+    ctx.encode(ids)
     # still usable after errors
     assert ctx.generate(MODE_SMALL_ONLY, 0.0, INF, 3)["tokens"] == g["small_only"]["tokens"][:3]
 
