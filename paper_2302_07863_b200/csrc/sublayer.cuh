@@ -415,6 +415,14 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
     red = n_keys <= a.red_keys;
     j0 = red ? 0 : (r * n_keys) >> a.c_shift; j1 = red ? n_keys : ((r + 1) * n_keys) >> a.c_shift;
     stage_cached(j0, min(j1, j0 + a.kc_keys));
+    // a share of more than one chunk: the later chunks are asked into the L2 now (they are staged when the first is used up)
+    const int later = (j1 - j0 - a.kc_keys) * (dkv >> 5);   // 128-byte lines of keys (as many again of values)
+#pragma unroll 1
+    for (int i = tid; i < later; i += SUB_THREADS) {
+      const size_t o = (size_t)(j0 + a.kc_keys) * dkv + (size_t)i * 32;
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(Kh + o));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(Vh + o));
+    }
   }
   // The call descriptor (row count, cache position) is written by kernels that have finished before the first kernel of a
   // pass starts -- the head of the pass before, or a set-up kernel in front of the embedding -- never by the kernel in
