@@ -1,7 +1,8 @@
 // Fused LM head (steps S9+S10 / L9+L10) for up to MAXB rows, bf16 weights, one block per SM.
 //   z[m][n] = scale * sum_j W[n][j] * rms_norm(x_m)[j]
 // Block b owns the vocabulary rows [b V / G, (b + 1) V / G).  They stream through a ring of
-// 16-row tiles in shared memory (one bulk copy per row, rows padded against bank conflicts; the
+// 16-row tiles in shared memory (one bulk copy per tile where the width allows the products of sl_mma_perm,
+// else one copy per row with the rows padded against bank conflicts; the
 // first tiles are requested before the dependency wait of the programmatic launch) by a ninth warp
 // that does nothing else (issuing a tile's copies costs about as much as multiplying it).  A tile
 // times the (up to 16) normalised token rows goes through mma.sync m16n8k16 (each activation as
@@ -55,9 +56,22 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int*
   // the last warp requests tile t: lane 0 announces the bytes, lanes 0..15 copy one row each (rows past
   // the end of the slice repeat its last row; their logits are masked).  Issuing the copies takes about
   // as long as multiplying a tile, which is why the eight computing warps do not do it themselves.
+  // usual widths (K a multiple of 256 up to 1024, or of 128 up to 512 for 32-row tiles): ONE bulk copy brings a tile, which
+  // then lies unpadded, and the products read it with 16-byte loads (sl_mma_perm); otherwise one copy per padded row
+  const bool whole = sl_perm_fits(TR, K);
+  const int wrow = whole ? K * 2 : rowst;   // bytes from one weight row of a tile to the next
   auto request = [&](int t) {
     if (t >= ntiles) return;
     const int slot = t % SH_TILES;
+    if (whole) {
+      if (lane == 0) {
+        const int n0 = nb + t * TR;
+        const uint32_t bytes = (uint32_t)(min(TR, ne - n0) * K * 2);   // (rows past the end of the slice keep what the slot held: masked)
+        mbar_expect(smem_u32(&sh->full[slot]), bytes);
+        bulk_g2s(smem_u32(sW + slot * tile_bytes), W + (size_t)n0 * K, bytes, smem_u32(&sh->full[slot]));
+      }
+      return;
+    }
     if (lane == 0) mbar_expect(smem_u32(&sh->full[slot]), (uint32_t)(TR * K * 2));
     __syncwarp();
     if (lane < TR) {
@@ -111,6 +125,12 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int*
   Partial run;
   run.m = -INFINITY; run.s = 0.f; run.idx = 0x7fffffff;
   const int NT = M <= 8 ? 1 : 2;
+  SlPermFrags<1> f1;
+  SlPermFrags<2> f2;
+  if (whole) {   // the token rows as operand fragments of this warp's K range, built once for all tiles
+    if (NT == 1) sl_perm_frags<1>(TR, K, Xs, xst, M, warp, lane, f1);
+    else sl_perm_frags<2>(TR, K, Xs, xst, M, warp, lane, f2);
+  }
 #pragma unroll 1
   for (int t = 0; t < ntiles; ++t) {
     const int slot = t % SH_TILES;
@@ -123,7 +143,10 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int*
       }
     }
     float* ps = psum + (t & 1) * (8 * 2 * 128);
-    if (NT == 1) sl_mma<1>(sW + slot * tile_bytes, rowst, TR, K, Xs, xst, M, ps, warp, lane);
+    if (whole) {
+      if (NT == 1) sl_mma_perm<1>(sW + slot * tile_bytes, wrow, TR, K, f1, ps, warp, lane);
+      else sl_mma_perm<2>(sW + slot * tile_bytes, wrow, TR, K, f2, ps, warp, lane);
+    } else if (NT == 1) sl_mma<1>(sW + slot * tile_bytes, rowst, TR, K, Xs, xst, M, ps, warp, lane);
     else sl_mma<2>(sW + slot * tile_bytes, rowst, TR, K, Xs, xst, M, ps, warp, lane);
     csync256();   // partial sums complete; every warp is done with the tile
     if (tid == 0) mbar_arrive(smem_u32(&sh->empty[slot]));   // the producer may refill it

@@ -170,6 +170,76 @@ __device__ __forceinline__ void sl_mma(const unsigned char* sW, int rowst, int n
     *reinterpret_cast<float4*>(psum + ((size_t)(warp * NT + nt) * 32 + lane) * 4) = make_float4(c[nt][0] + e[nt][0], c[nt][1] + e[nt][1], c[nt][2] + e[nt][2], c[nt][3] + e[nt][3]);
 }
 
+// Products of a weight tile in shared memory (rows `rowst` bytes apart) with token rows whose operand fragments were built
+// once (a caller that multiplies many tiles with the same rows: the LM head).  A thread loads 16 bytes of a weight row -- the columns
+// 8 t .. 8 t + 7 of a 32-column chunk -- and uses them as the left operands of two m16n8k16 instructions: within a chunk
+// the instruction's column positions are dealt to the threads' columns (position 2 t, 2 t + 1 | 2 t + 8, 2 t + 9 of
+// instruction m <-> columns 8 t + 4 m + 0, 1 | 2, 3), and the fragments of the token rows follow the same order, so every
+// product meets its partner.
+constexpr int SL_PERM_CHUNKS = 4;   // 32-column chunks of a warp's K range (K / 8 or K / 4 columns: K <= 1024 or 512)
+template <int NT>
+struct SlPermFrags { uint32_t h[NT][SL_PERM_CHUNKS][2][2], l[NT][SL_PERM_CHUNKS][2][2]; };
+__host__ __device__ inline bool sl_perm_fits(int nrows, int K) {
+  const int MT = (nrows + 15) >> 4, ks_sh = MT == 1 ? 3 : MT == 2 ? 2 : 1;
+  return (nrows == 16 || nrows == 32) && K % (32 << ks_sh) == 0 && (K >> ks_sh) / 32 <= SL_PERM_CHUNKS;
+}
+template <int NT>
+__device__ __forceinline__ void sl_perm_frags(int nrows, int K, const float* Xs, int xst, int mg, int warp, int lane, SlPermFrags<NT>& f) {
+  const int MT = (nrows + 15) >> 4, ks_sh = MT == 1 ? 3 : MT == 2 ? 2 : 1, KS = 1 << ks_sh;
+  const int ks = warp & (KS - 1), cols = K >> ks_sh, chunks = cols >> 5;
+  const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const float* xb = Xs + (size_t)min(nt * 8 + g, mg - 1) * xst + ks * cols + 8 * t;
+#pragma unroll
+    for (int ch = 0; ch < SL_PERM_CHUNKS; ++ch)
+#pragma unroll
+      for (int m = 0; m < 2; ++m) {
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ch < chunks) x = *reinterpret_cast<const float4*>(xb + ch * 32 + 4 * m);
+        const uint32_t h0 = sl_pack_bf16(x.x, x.y), h1 = sl_pack_bf16(x.z, x.w);
+        f.h[nt][ch][m][0] = h0; f.h[nt][ch][m][1] = h1;
+        f.l[nt][ch][m][0] = sl_pack_bf16(x.x - __uint_as_float(h0 << 16), x.y - __uint_as_float(h0 & 0xffff0000u));
+        f.l[nt][ch][m][1] = sl_pack_bf16(x.z - __uint_as_float(h1 << 16), x.w - __uint_as_float(h1 & 0xffff0000u));
+      }
+  }
+}
+template <int NT>
+__device__ __forceinline__ void sl_mma_perm(const unsigned char* sW, int rowst, int nrows, int K, const SlPermFrags<NT>& f, float* psum, int warp,
+                                            int lane) {
+  const int MT = (nrows + 15) >> 4, ks_sh = MT == 1 ? 3 : MT == 2 ? 2 : 1, KS = 1 << ks_sh;
+  if (warp >= MT * KS) return;
+  const int mt = warp >> ks_sh, ks = warp & (KS - 1), cols = K >> ks_sh, chunks = cols >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const unsigned char* pa0 = sW + (size_t)(mt * 16 + g) * rowst + (size_t)(ks * cols + 8 * t) * 2;
+  const unsigned char* pa1 = pa0 + (size_t)8 * rowst;
+  float c[NT][4], e[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+    e[nt][0] = e[nt][1] = e[nt][2] = e[nt][3] = 0.f;
+  }
+#pragma unroll
+  for (int ch = 0; ch < SL_PERM_CHUNKS; ++ch)
+    if (ch < chunks) {
+      const uint4 a0 = *reinterpret_cast<const uint4*>(pa0 + ch * 64), a1 = *reinterpret_cast<const uint4*>(pa1 + ch * 64);
+#define SL_MMA_P(ACC, A0, A1, A2, A3, B0, B1)                                                                                    \
+      asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"   \
+                   : "+f"(ACC[0]), "+f"(ACC[1]), "+f"(ACC[2]), "+f"(ACC[3]) : "r"(A0), "r"(A1), "r"(A2), "r"(A3), "r"(B0), "r"(B1))
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        SL_MMA_P(c[nt], a0.x, a1.x, a0.y, a1.y, f.h[nt][ch][0][0], f.h[nt][ch][0][1]);
+        SL_MMA_P(e[nt], a0.x, a1.x, a0.y, a1.y, f.l[nt][ch][0][0], f.l[nt][ch][0][1]);
+        SL_MMA_P(c[nt], a0.z, a1.z, a0.w, a1.w, f.h[nt][ch][1][0], f.h[nt][ch][1][1]);
+        SL_MMA_P(e[nt], a0.z, a1.z, a0.w, a1.w, f.l[nt][ch][1][0], f.l[nt][ch][1][1]);
+      }
+#undef SL_MMA_P
+    }
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+    *reinterpret_cast<float4*>(psum + ((size_t)(warp * NT + nt) * 32 + lane) * 4) = make_float4(c[nt][0] + e[nt][0], c[nt][1] + e[nt][1], c[nt][2] + e[nt][2], c[nt][3] + e[nt][3]);
+}
+
 __global__ void __launch_bounds__(SL_THREADS) slice_linear_kernel(SliceArgs s) {
   extern __shared__ __align__(1024) unsigned char sl_smem[];
   const LinArgs& a = s.lin;
