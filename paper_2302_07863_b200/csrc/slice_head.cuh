@@ -155,12 +155,21 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int*
       const int col = em & 7, mt = er >> 4, rr = er & 15;
       const float* p = ps + ((size_t)((mt << ks_sh) * NT + (em >> 3)) * 32 + (rr & 7) * 4 + (col >> 1)) * 4 + (rr >> 3) * 2 + (col & 1);
       float z = 0.f;
-      for (int w = 0; w < (1 << ks_sh); ++w) z += p[(size_t)w * NT * 128];
+      if (ks_sh == 3) {   // the eight partial sums are requested together, then added in warp order
+        float v[8];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v[w] = p[(size_t)w * NT * 128];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) z += v[w];
+      } else {
+        for (int w = 0; w < (1 << ks_sh); ++w) z += p[(size_t)w * NT * 128];
+      }
       const int n = nb + t * TR + er;
       if (n < ne) {
         z *= a.scale;
-        if (z > run.m) { run.s = run.s * expf(run.m - z) + 1.f; run.m = z; run.idx = n; }
-        else run.s += expf(z - run.m);
+        const float dz = z - run.m, ez = expf(-fabsf(dz));   // one exponential for either case (the lanes of a warp take both)
+        if (dz > 0.f) { run.s = run.s * ez + 1.f; run.m = z; run.idx = n; }
+        else run.s += ez;
         if (n == my_target) a.out->gather[em] = z;
         if (a.logits_dbg) a.logits_dbg[(size_t)em * V + n] = z;
       }
