@@ -566,7 +566,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
       const int g = lane >> 2, t = lane & 3;
 #pragma unroll 1
       for (int t0 = warp * 16; t0 < nk; t0 += 16 * (SUB_THREADS / 32)) {
-        float c0a = 0.f, c1a = 0.f, c2a = 0.f, c3a = 0.f;
+        float c0a = 0.f, c1a = 0.f, c2a = 0.f, c3a = 0.f, c0b = 0.f, c1b = 0.f, c2b = 0.f, c3b = 0.f, c0c = 0.f, c1c = 0.f, c2c = 0.f, c3c = 0.f;
         const float* ka = sK + (size_t)min(t0 + g, nk - 1) * kvst + 2 * t;
         const float* kb = sK + (size_t)min(t0 + g + 8, nk - 1) * kvst + 2 * t;
         const float* qp = sQKV + (size_t)min(g, k - 1) * R + 2 * t;
@@ -585,16 +585,16 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
             const uint32_t bh0 = sl_pack_bf16(b0.x, b0.y), bh1 = sl_pack_bf16(b1.x, b1.y);
             const uint32_t bl0 = sl_pack_bf16(b0.x - __uint_as_float(bh0 << 16), b0.y - __uint_as_float(bh0 & 0xffff0000u));
             const uint32_t bl1 = sl_pack_bf16(b1.x - __uint_as_float(bh1 << 16), b1.y - __uint_as_float(bh1 & 0xffff0000u));
-#define SUB_MMA_S(A0, A1, A2, A3, B0, B1)                                                                                        \
+#define SUB_MMA_S(C0, C1, C2, C3, A0, A1, A2, A3, B0, B1)                                                                        \
             asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};" \
-                         : "+f"(c0a), "+f"(c1a), "+f"(c2a), "+f"(c3a) : "r"(A0), "r"(A1), "r"(A2), "r"(A3), "r"(B0), "r"(B1))
-            SUB_MMA_S(ah0, ah1, ah2, ah3, bh0, bh1);
-            SUB_MMA_S(al0, al1, al2, al3, bh0, bh1);
-            SUB_MMA_S(ah0, ah1, ah2, ah3, bl0, bl1);
+                         : "+f"(C0), "+f"(C1), "+f"(C2), "+f"(C3) : "r"(A0), "r"(A1), "r"(A2), "r"(A3), "r"(B0), "r"(B1))
+            SUB_MMA_S(c0a, c1a, c2a, c3a, ah0, ah1, ah2, ah3, bh0, bh1);
+            SUB_MMA_S(c0b, c1b, c2b, c3b, al0, al1, al2, al3, bh0, bh1);
+            SUB_MMA_S(c0c, c1c, c2c, c3c, ah0, ah1, ah2, ah3, bl0, bl1);
 #undef SUB_MMA_S
           }
         // accumulators: keys t0 + g and t0 + g + 8, token rows 2 t and 2 t + 1
-        const float cv[4] = {c0a, c1a, c2a, c3a};
+        const float cv[4] = {c0a + (c0b + c0c), c1a + (c1b + c1c), c2a + (c2b + c2c), c3a + (c3b + c3c)};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int jj = t0 + g + 8 * (i >> 1), m = 2 * t + (i & 1);
@@ -658,7 +658,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
         const int g = lane >> 2, t = lane & 3, n0 = warp * 8;
         const float rs = g < k ? sh->rscale[g] : 1.f;
         acc[0] *= rs; acc[1] *= rs;
-        float c2 = 0.f, c3 = 0.f;
+        float c2 = 0.f, c3 = 0.f, d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;   // (d: the products with the remainders, a chain of their own)
         const uint32_t zero = 0u;
 #pragma unroll 2
         for (int k0 = 0; k0 < nk; k0 += 16) {
@@ -680,10 +680,13 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
           asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};" \
                        : "+f"(acc[0]), "+f"(acc[1]), "+f"(c2), "+f"(c3) : "r"(A0), "r"(zero), "r"(A2), "r"(zero), "r"(B0), "r"(B1))
           SUB_MMA(ah0, ah2, bh0, bh1);
-          SUB_MMA(al0, al2, bh0, bh1);
-          SUB_MMA(ah0, ah2, bl0, bl1);
+          asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                       : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3) : "r"(al0), "r"(zero), "r"(al2), "r"(zero), "r"(bh0), "r"(bh1));
+          asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                       : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3) : "r"(ah0), "r"(zero), "r"(ah2), "r"(zero), "r"(bl0), "r"(bl1));
 #undef SUB_MMA
         }
+        acc[0] += d0; acc[1] += d1;
       }
     }
   }
@@ -774,7 +777,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
     float* sOut = reinterpret_cast<float*>(sub_smem + a.L.out);
     const int ost = no + 4;
     if (warp * 16 < no) {
-      float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
+      float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f;   // (heads | remainders: two chains)
 #pragma unroll
       for (int st = 0; st < 4; ++st)
         if (st * 16 < dkv) {
@@ -787,9 +790,10 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
                        : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3)
                        : "r"(wr[0][2 * st]), "r"(wr[1][2 * st]), "r"(wr[0][2 * st + 1]), "r"(wr[1][2 * st + 1]), "r"(bh0), "r"(bh1));
           asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                       : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3)
+                       : "+f"(e0), "+f"(e1), "+f"(e2), "+f"(e3)
                        : "r"(wr[0][2 * st]), "r"(wr[1][2 * st]), "r"(wr[0][2 * st + 1]), "r"(wr[1][2 * st + 1]), "r"(bl0), "r"(bl1));
         }
+      c0 += e0; c1 += e1; c2 += e2; c3 += e3;
       // accumulators: rows g and g + 8 of the tile, token rows 2 t and 2 t + 1
       const int row = warp * 16 + og;
       if (row < no) { sOut[(size_t)(2 * ot) * ost + row] = c0; sOut[(size_t)(2 * ot + 1) * ost + row] = c1; }
