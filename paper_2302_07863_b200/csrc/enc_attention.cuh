@@ -141,21 +141,30 @@ __global__ void __launch_bounds__(EA_THREADS * G) enc_attn_kernel(BAttnArgs a, _
     ea_group_sync(grp);
     if (k0 + EA_KEYS * G < E) fetch(k0 + EA_KEYS * G);   // (the raw area is free again: everybody has converted its share)
     // scores of 16 rows x 64 keys
+    // (consecutive instructions go to different accumulators, four key tiles side by side: an instruction that adds to the
+    // accumulator of the one in front waits for its result)
     float s[8][4];
 #pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-      s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-      const __nv_bfloat16* kh = sKh + (nt * 8 + g) * ST + 2 * t;
-      const __nv_bfloat16* kl = sKl + (nt * 8 + g) * ST + 2 * t;
+    for (int nt = 0; nt < 8; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
 #pragma unroll
-      for (int ks = 0; ks < 4; ++ks) {
-        const uint32_t bh0 = *reinterpret_cast<const uint32_t*>(kh + ks * 16), bh1 = *reinterpret_cast<const uint32_t*>(kh + ks * 16 + 8);
-        const uint32_t bl0 = *reinterpret_cast<const uint32_t*>(kl + ks * 16), bl1 = *reinterpret_cast<const uint32_t*>(kl + ks * 16 + 8);
-        ea_mma(s[nt], qh[ks][0], qh[ks][1], qh[ks][2], qh[ks][3], bh0, bh1);
-        ea_mma(s[nt], qh[ks][0], qh[ks][1], qh[ks][2], qh[ks][3], bl0, bl1);
-        ea_mma(s[nt], ql[ks][0], ql[ks][1], ql[ks][2], ql[ks][3], bh0, bh1);
+    for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+      for (int n4 = 0; n4 < 8; n4 += 4) {
+        uint32_t bh[4][2], bl[4][2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const __nv_bfloat16* kh = sKh + ((n4 + i) * 8 + g) * ST + 2 * t + ks * 16;
+          const __nv_bfloat16* kl = sKl + ((n4 + i) * 8 + g) * ST + 2 * t + ks * 16;
+          bh[i][0] = *reinterpret_cast<const uint32_t*>(kh); bh[i][1] = *reinterpret_cast<const uint32_t*>(kh + 8);
+          bl[i][0] = *reinterpret_cast<const uint32_t*>(kl); bl[i][1] = *reinterpret_cast<const uint32_t*>(kl + 8);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ea_mma(s[n4 + i], qh[ks][0], qh[ks][1], qh[ks][2], qh[ks][3], bh[i][0], bh[i][1]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ea_mma(s[n4 + i], qh[ks][0], qh[ks][1], qh[ks][2], qh[ks][3], bl[i][0], bl[i][1]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ea_mma(s[n4 + i], ql[ks][0], ql[ks][1], ql[ks][2], ql[ks][3], bh[i][0], bh[i][1]);
       }
-    }
     // bias, mask of the keys past the end, tile maxima
     float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
@@ -200,14 +209,21 @@ __global__ void __launch_bounds__(EA_THREADS * G) enc_attn_kernel(BAttnArgs a, _
       ea_split(s[2 * j + 1][0], s[2 * j + 1][1], ph[2], pl[2]);
       ea_split(s[2 * j + 1][2], s[2 * j + 1][3], ph[3], pl[3]);
 #pragma unroll
-      for (int dt = 0; dt < 8; ++dt) {
-        const __nv_bfloat16* vh = sVh + (dt * 8 + g) * ST + j * 16 + 2 * t;
-        const __nv_bfloat16* vl = sVl + (dt * 8 + g) * ST + j * 16 + 2 * t;
-        const uint32_t bh0 = *reinterpret_cast<const uint32_t*>(vh), bh1 = *reinterpret_cast<const uint32_t*>(vh + 8);
-        const uint32_t bl0 = *reinterpret_cast<const uint32_t*>(vl), bl1 = *reinterpret_cast<const uint32_t*>(vl + 8);
-        ea_mma(o[dt], ph[0], ph[1], ph[2], ph[3], bh0, bh1);
-        ea_mma(o[dt], ph[0], ph[1], ph[2], ph[3], bl0, bl1);
-        ea_mma(o[dt], pl[0], pl[1], pl[2], pl[3], bh0, bh1);
+      for (int d4 = 0; d4 < 8; d4 += 4) {   // four channel tiles side by side, as above
+        uint32_t bh[4][2], bl[4][2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const __nv_bfloat16* vh = sVh + ((d4 + i) * 8 + g) * ST + j * 16 + 2 * t;
+          const __nv_bfloat16* vl = sVl + ((d4 + i) * 8 + g) * ST + j * 16 + 2 * t;
+          bh[i][0] = *reinterpret_cast<const uint32_t*>(vh); bh[i][1] = *reinterpret_cast<const uint32_t*>(vh + 8);
+          bl[i][0] = *reinterpret_cast<const uint32_t*>(vl); bl[i][1] = *reinterpret_cast<const uint32_t*>(vl + 8);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ea_mma(o[d4 + i], ph[0], ph[1], ph[2], ph[3], bh[i][0], bh[i][1]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ea_mma(o[d4 + i], ph[0], ph[1], ph[2], ph[3], bl[i][0], bl[i][1]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ea_mma(o[d4 + i], pl[0], pl[1], pl[2], pl[3], bh[i][0], bh[i][1]);
       }
     }
   }
