@@ -614,12 +614,13 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
     if (ONE) {
       // every warp finds the chunk's maximum; thread (group of four channels, key part) then exponentiates and weighs its keys
       float mx = -INFINITY;
-      for (int jj = lane; jj < nk; jj += 32) mx = fmaxf(mx, sP[jj]);
+#pragma unroll 4
+      for (int jj = lane; jj < nk; jj += 32) mx = fmaxf(mx, sP[jj]);   // (unrolled: the loads of a thread side by side)
       mx = warp_max(mx);
       const float nw = fmaxf(run1, mx), sc = run1 == -INFINITY ? 0.f : __expf(run1 - nw);
       float4 t4 = make_float4(acc4.x * sc, acc4.y * sc, acc4.z * sc, acc4.w * sc);
       float l = lsum1 * sc;
-#pragma unroll 2
+#pragma unroll 4
       for (int jj = part4; jj < nk; jj += nparts4) {
         const float p = __expf(sP[jj] - nw);
         const float4 v = *reinterpret_cast<const float4*>(sV + (size_t)jj * vst + cg4 * 4);
@@ -697,7 +698,7 @@ __global__ void __launch_bounds__(SUB_THREADS) attn_sub_kernel(const AttnSubArgs
     __syncthreads();
     if (tid < dkv) {
       float t = 0.f;
-#pragma unroll 4
+#pragma unroll 16
       for (int p2 = 0; p2 < nparts4; ++p2) t += sRed[p2 * dkv + tid];
       recLoc[SUB_RECPAD + tid] = t;
     } else if (warp == SUB_THREADS / 32 - 1) {   // the parts' sums, added by one warp
