@@ -198,11 +198,20 @@ __global__ void __launch_bounds__(SH_THREADS) slice_head_kernel(HeadArgs a, int*
   for (int m = warp; m < M; m += SH_COMPUTE / 32) {
     Partial p;
     p.m = -INFINITY; p.s = 0.f; p.idx = 0x7fffffff;
-    for (int b = lane; b < (int)gridDim.x; b += 32) {
-      Partial q;
-      const Partial* src = &a.partials[(size_t)b * MAXB + m];
-      q.m = __ldcg(&src->m); q.s = __ldcg(&src->s); q.idx = __ldcg(&src->idx);
-      p = combine(p, q);
+    // (the blocks' partial results of a lane are requested together, eight at a time, then combined in block order)
+    for (int b0 = lane; b0 < (int)gridDim.x; b0 += 8 * 32) {
+      Partial q[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int b = b0 + 32 * j;
+        q[j].m = -INFINITY; q[j].s = 0.f; q[j].idx = 0x7fffffff;
+        if (b < (int)gridDim.x) {
+          const Partial* src = &a.partials[(size_t)b * MAXB + m];
+          q[j].m = __ldcg(&src->m); q[j].s = __ldcg(&src->s); q[j].idx = __ldcg(&src->idx);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) p = combine(p, q[j]);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
